@@ -1,0 +1,295 @@
+"""ctypes front end of the CPU oracle (ecospa_oracle.cpp) -- TEST INFRASTRUCTURE ONLY.
+
+Nothing in the product package imports this module.  It marshals numpy / torch CPU
+tensors into the plain-C oracle and returns numpy fp64 (or int32 / raw byte) results.
+It performs no arithmetic of the method itself.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional, Sequence
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ecospa_oracle.cpp")
+_LIB = os.path.join(_HERE, "libecospa_oracle.so")
+
+F32, BF16, F64 = 0, 1, 2
+SHARED_COLS, SHARED_ROWS = 0, 1
+ACT_GELU_ERF, ACT_GELU_TANH, ACT_SWIGLU = 1, 2, 3
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with g++ (plain -O2, no fast-math) if it is stale."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-o", _LIB, _SRC])
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.eco_coupled_single.restype = C.c_int32
+        _lib.eco_frob_removed.restype = C.c_double
+    return _lib
+
+
+# ---------------------------------------------------------------------------
+# marshalling helpers
+# ---------------------------------------------------------------------------
+
+class _Buf:
+    """Keeps a contiguous CPU buffer alive and exposes (pointer, dtype code, leading dim)."""
+
+    def __init__(self, t):
+        if t is None:
+            self.arr, self.ptr, self.dtype, self.ld = None, None, F64, 0
+            return
+        if isinstance(t, torch.Tensor):
+            t = t.detach().cpu().contiguous()
+            assert t.dim() <= 2, "2-D or 1-D tensors only"
+            ld = t.shape[1] if t.dim() == 2 else t.numel()
+            if t.dtype == torch.bfloat16:
+                arr, code = t.view(torch.int16).numpy(), BF16
+            elif t.dtype == torch.float32:
+                arr, code = t.numpy(), F32
+            elif t.dtype == torch.float64:
+                arr, code = t.numpy(), F64
+            else:
+                raise TypeError(t.dtype)
+        else:
+            arr = np.ascontiguousarray(t)
+            ld = arr.shape[1] if arr.ndim == 2 else arr.size
+            code = {np.dtype(np.float32): F32, np.dtype(np.float64): F64}[arr.dtype]
+        self.arr, self.dtype, self.ld = arr, code, int(ld)
+        self.ptr = C.c_void_p(arr.ctypes.data)
+
+
+def _i32(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int32))
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else C.c_void_p(a.ctypes.data)
+
+
+def _shared_dims(t, layout):
+    """(other, D) of a matrix with a shared axis."""
+    r, c = t.shape
+    return (r, c) if layout == SHARED_COLS else (c, r)
+
+
+# ---------------------------------------------------------------------------
+# scores, Fisher, selection, compaction
+# ---------------------------------------------------------------------------
+
+def sumsq_shared(w, layout: int) -> np.ndarray:
+    b = _Buf(w)
+    other, D = _shared_dims(w, layout)
+    out = np.empty(D, dtype=np.float64)
+    lib().eco_sumsq_shared(b.ptr, b.dtype, layout, C.c_int64(other), C.c_int64(D), C.c_int64(b.ld), _p(out))
+    return out
+
+
+def sumsq_shared_hadamard(gate, up, layout: int) -> np.ndarray:
+    g, u = _Buf(gate), _Buf(up)
+    assert g.dtype == u.dtype and gate.shape == up.shape
+    other, D = _shared_dims(gate, layout)
+    out = np.empty(D, dtype=np.float64)
+    lib().eco_sumsq_shared_hadamard(g.ptr, u.ptr, g.dtype, layout, C.c_int64(other), C.c_int64(D),
+                                    C.c_int64(g.ld), C.c_int64(u.ld), _p(out))
+    return out
+
+
+def upsilon(c1: np.ndarray, c2: np.ndarray, n_seg: int, seg_len: int):
+    c1 = np.ascontiguousarray(c1, dtype=np.float64)
+    c2 = np.ascontiguousarray(c2, dtype=np.float64)
+    assert c1.size == c2.size == n_seg * seg_len
+    raw = np.empty_like(c1)
+    ups = np.empty_like(c1)
+    lib().eco_upsilon(_p(c1), _p(c2), n_seg, seg_len, _p(raw), _p(ups))
+    return raw, ups
+
+
+def score_pair(w1, w2, layout1: int, layout2: int, n_seg: int, seg_len: int, w1b=None):
+    """(raw, upsilon) of a coupled pair; w1b given = SwiGLU pair with W_1 = w1 (.) w1b."""
+    c1 = sumsq_shared(w1, layout1) if w1b is None else sumsq_shared_hadamard(w1, w1b, layout1)
+    c2 = sumsq_shared(w2, layout2)
+    return upsilon(c1, c2, n_seg, seg_len)
+
+
+def fisher_pair(g1, g2, layout1: int, layout2: int, n_seg: int, seg_len: int, n_samples: float, g1b=None):
+    a, b, ab = _Buf(g1), _Buf(g2), _Buf(g1b)
+    other1, D1 = _shared_dims(g1, layout1)
+    other2, D2 = _shared_dims(g2, layout2)
+    assert D1 == D2 == n_seg * seg_len and a.dtype == b.dtype
+    out = np.empty(n_seg, dtype=np.float64)
+    lib().eco_fisher_pair(a.ptr, ab.ptr, b.ptr, a.dtype, layout1, layout2, C.c_int64(other1), C.c_int64(other2),
+                          C.c_int64(a.ld), C.c_int64(ab.ld), C.c_int64(b.ld), n_seg, seg_len,
+                          C.c_double(n_samples), _p(out))
+    return out
+
+
+def select_topk(ups, n_seg: int, seg_len: int, k: Sequence[int]) -> np.ndarray:
+    """Ascending global kept indices, segment after segment.  fp32 input is ranked as fp32."""
+    k = _i32(k)
+    assert k.size == n_seg and (k >= 0).all() and (k <= seg_len).all()
+    kept = np.empty(int(k.sum()), dtype=np.int32)
+    ups = np.ascontiguousarray(ups)
+    assert ups.size == n_seg * seg_len
+    if ups.dtype == np.float32:
+        lib().eco_select_topk_f32(_p(ups), n_seg, seg_len, _p(k), _p(kept))
+    else:
+        ups = ups.astype(np.float64, copy=False)
+        lib().eco_select_topk_f64(_p(ups), n_seg, seg_len, _p(k), _p(kept))
+    return kept
+
+
+def compact(t: torch.Tensor, layout: int, kept, ld_out: Optional[int] = None) -> torch.Tensor:
+    """Gather the kept shared indices of `t` (2-D, or 1-D = a bias over the shared axis)."""
+    kept = _i32(kept)
+    vec = t.dim() == 1
+    t2 = t.reshape(1, -1) if vec else t
+    if vec:
+        layout = SHARED_COLS
+    t2 = t2.detach().cpu().contiguous()
+    other, D = _shared_dims(t2, layout)
+    eb = t2.element_size()
+    n_kept = kept.size
+    if layout == SHARED_COLS:
+        ld = ld_out if ld_out is not None else n_kept
+        out = torch.empty((other, ld), dtype=t2.dtype)
+    else:
+        ld = ld_out if ld_out is not None else other
+        out = torch.empty((n_kept, ld), dtype=t2.dtype)
+    src = t2.view(torch.uint8).numpy() if eb == 1 else t2.view(torch.int16 if eb == 2 else torch.int32 if eb == 4 else torch.int64).numpy()
+    dst_t = out.view(torch.int16 if eb == 2 else torch.int32 if eb == 4 else torch.int64)
+    dst = dst_t.numpy()
+    lib().eco_compact_bytes(_p(src), eb, layout, C.c_int64(other), C.c_int64(t2.stride(0)), _p(kept),
+                            C.c_int64(n_kept), _p(dst), C.c_int64(ld))
+    return out.reshape(-1) if vec else out
+
+
+# ---------------------------------------------------------------------------
+# Appendix A comparators
+# ---------------------------------------------------------------------------
+
+def coupled_single(A: np.ndarray, B: np.ndarray) -> int:
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    B = np.ascontiguousarray(B, dtype=np.float64)
+    m, n = A.shape
+    p = B.shape[1]
+    return int(lib().eco_coupled_single(_p(A), _p(B), C.c_int64(m), C.c_int64(n), C.c_int64(p)))
+
+
+def individual_single(A: np.ndarray, B: np.ndarray):
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    B = np.ascontiguousarray(B, dtype=np.float64)
+    m, n = A.shape
+    p = B.shape[1]
+    ks, ls = C.c_int32(0), C.c_int32(0)
+    lib().eco_individual_single(_p(A), _p(B), C.c_int64(m), C.c_int64(n), C.c_int64(p), C.byref(ks), C.byref(ls))
+    return int(ks.value), int(ls.value)
+
+
+def frob_removed(A: np.ndarray, B: np.ndarray, keptA, keptB) -> float:
+    A = np.ascontiguousarray(A, dtype=np.float64)
+    B = np.ascontiguousarray(B, dtype=np.float64)
+    ka, kb = _i32(keptA), _i32(keptB)
+    assert ka.size == kb.size
+    m, n = A.shape
+    p = B.shape[1]
+    return float(lib().eco_frob_removed(_p(A), _p(B), C.c_int64(m), C.c_int64(n), C.c_int64(p), _p(ka), _p(kb),
+                                        C.c_int64(ka.size)))
+
+
+# ---------------------------------------------------------------------------
+# layer math
+# ---------------------------------------------------------------------------
+
+def _wdims(w, layout):
+    other, D = _shared_dims(w, layout)
+    return other, D
+
+
+def proj_fwd(X, W, wlayout: int, n: int, bias=None) -> np.ndarray:
+    """Y = X W^c + b with W^c a (d_m x n) shared-cols or (n x d_m) shared-rows matrix (n real columns)."""
+    x, w, b = _Buf(X), _Buf(W), _Buf(bias)
+    T, d_m = X.shape
+    Y = np.empty((T, n), dtype=np.float64)
+    lib().eco_proj_fwd(x.ptr, x.dtype, C.c_int64(T), C.c_int64(d_m), C.c_int64(x.ld), w.ptr, w.dtype, wlayout,
+                       C.c_int64(n), C.c_int64(w.ld), b.ptr, _p(Y))
+    return Y
+
+
+def proj_bwd(X, W, wlayout: int, n: int, dY, want_db: bool = False, dX: Optional[np.ndarray] = None):
+    x, w, dy = _Buf(X), _Buf(W), _Buf(dY)
+    assert x.dtype == dy.dtype
+    T, d_m = X.shape
+    if dX is None:
+        dX = np.zeros((T, d_m), dtype=np.float64)
+    dW = np.empty((d_m, n), dtype=np.float64)
+    db = np.empty(n, dtype=np.float64) if want_db else None
+    lib().eco_proj_bwd(x.ptr, x.dtype, C.c_int64(T), C.c_int64(d_m), C.c_int64(x.ld), w.ptr, w.dtype, wlayout,
+                       C.c_int64(n), C.c_int64(w.ld), dy.ptr, C.c_int64(dy.ld), _p(dX), _p(dW), _p(db))
+    return dX, dW, db
+
+
+def outproj_fwd(Ctx, W, wlayout: int, n: int, d_m: int, bias=None) -> np.ndarray:
+    c, w, b = _Buf(Ctx), _Buf(W), _Buf(bias)
+    T = Ctx.shape[0]
+    Out = np.empty((T, d_m), dtype=np.float64)
+    lib().eco_outproj_fwd(c.ptr, c.dtype, C.c_int64(T), C.c_int64(n), C.c_int64(c.ld), w.ptr, w.dtype, wlayout,
+                          C.c_int64(d_m), C.c_int64(w.ld), b.ptr, _p(Out))
+    return Out
+
+
+def outproj_bwd(Ctx, W, wlayout: int, n: int, d_m: int, dOut, want_db: bool = False):
+    c, w, do = _Buf(Ctx), _Buf(W), _Buf(dOut)
+    T = Ctx.shape[0]
+    dCtx = np.empty((T, n), dtype=np.float64)
+    dW = np.empty((d_m, n), dtype=np.float64)
+    db = np.empty(d_m, dtype=np.float64) if want_db else None
+    lib().eco_outproj_bwd(c.ptr, c.dtype, C.c_int64(T), C.c_int64(n), C.c_int64(c.ld), w.ptr, w.dtype, wlayout,
+                          C.c_int64(d_m), C.c_int64(w.ld), do.ptr, C.c_int64(do.ld), _p(dCtx), _p(dW), _p(db))
+    return dCtx, dW, db
+
+
+def ffn_fwd(X, act: int, W1, W2, layout1: int, layout2: int, k: int, W1b=None, b1=None, b2=None):
+    """Returns dict(Y, H, Hb, A) in fp64."""
+    x, w1, w1b, w2, bb1, bb2 = _Buf(X), _Buf(W1), _Buf(W1b), _Buf(W2), _Buf(b1), _Buf(b2)
+    T, d_m = X.shape
+    Y = np.empty((T, d_m), dtype=np.float64)
+    H = np.empty((T, k), dtype=np.float64)
+    A = np.empty((T, k), dtype=np.float64)
+    Hb = np.empty((T, k), dtype=np.float64) if act == ACT_SWIGLU else None
+    lib().eco_ffn_fwd(x.ptr, x.dtype, C.c_int64(T), C.c_int64(d_m), C.c_int64(x.ld), act, w1.ptr, w1b.ptr, w2.ptr,
+                      w1.dtype, layout1, layout2, C.c_int64(k), C.c_int64(w1.ld), C.c_int64(w1b.ld),
+                      C.c_int64(w2.ld), bb1.ptr, bb2.ptr, _p(Y), _p(H), _p(Hb), _p(A))
+    return {"Y": Y, "H": H, "Hb": Hb, "A": A}
+
+
+def ffn_bwd(X, act: int, W1, W2, layout1: int, layout2: int, k: int, dY, W1b=None, b1=None, want_bias: bool = False):
+    """Returns dict(dX, dW1, dW1b, dW2, db1, db2); weight grads in math orientation (d_m x k)."""
+    x, w1, w1b, w2, bb1, dy = _Buf(X), _Buf(W1), _Buf(W1b), _Buf(W2), _Buf(b1), _Buf(dY)
+    assert x.dtype == dy.dtype
+    T, d_m = X.shape
+    dX = np.empty((T, d_m), dtype=np.float64)
+    dW1 = np.empty((d_m, k), dtype=np.float64)
+    dW2 = np.empty((d_m, k), dtype=np.float64)
+    dW1b = np.empty((d_m, k), dtype=np.float64) if act == ACT_SWIGLU else None
+    db1 = np.empty(k, dtype=np.float64) if want_bias else None
+    db2 = np.empty(d_m, dtype=np.float64) if want_bias else None
+    lib().eco_ffn_bwd(x.ptr, x.dtype, C.c_int64(T), C.c_int64(d_m), C.c_int64(x.ld), act, w1.ptr, w1b.ptr, w2.ptr,
+                      w1.dtype, layout1, layout2, C.c_int64(k), C.c_int64(w1.ld), C.c_int64(w1b.ld),
+                      C.c_int64(w2.ld), bb1.ptr, dy.ptr, C.c_int64(dy.ld), _p(dX), _p(dW1), _p(dW1b), _p(dW2),
+                      _p(db1), _p(db2))
+    return {"dX": dX, "dW1": dW1, "dW1b": dW1b, "dW2": dW2, "db1": db1, "db2": db2}
