@@ -1,0 +1,229 @@
+// Aligned top-k per segment (Definition 1 applied to the lowest-scored indices).
+//
+// One CTA per segment.  The k-th largest score is found by a 4-pass radix select over an
+// order-preserving 32-bit key; the kept indices are then emitted in ascending order with a
+// block-wide stream compaction, taking equal-to-threshold scores lowest index first.  The score
+// vector of a segment (<= 44 KB at the shapes of interest) is re-read from L1/L2 in each pass.
+
+#include <vector>
+
+#include "common.cuh"
+
+namespace ecospa {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kMaxSegs = 4096;   // per launch (16 KB of offsets)
+constexpr int kMaxPairs = 256;   // per launch
+
+struct SelPair {
+    int32_t seg_start;  // first segment (within this launch) of the pair
+    int32_t seg_len;
+    int32_t d_off;      // offset of the pair's scores in upsilon, and base added to nothing: kept
+                        // indices are relative to the pair group (segment offset included)
+    int32_t pad_;
+};
+
+struct SelectParams {
+    const float* upsilon;
+    int32_t* kept;
+    int32_t* seg_offsets;   // may be null; global prefix sums of k
+    int32_t n_pairs, n_segs;
+    int32_t seg_base;       // global index of this launch's first segment
+    int32_t is_last;        // this launch writes the final seg_offsets entry
+    SelPair pairs[kMaxPairs];
+    int32_t out_off[kMaxSegs + 1];  // global offsets into kept
+};
+
+// fp32 -> uint32 whose unsigned order is the float order; -0 and +0 map to the same key.
+__device__ __forceinline__ uint32_t order_key(float f) {
+    uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ SelectParams P) {
+    __shared__ int hist[256];
+    __shared__ int warp_tot[kWarps];
+    __shared__ uint32_t sh_prefix;
+    __shared__ int sh_want, sh_cnt_eq;
+
+    const int seg = blockIdx.x;
+    int lo = 0, hi = P.n_pairs - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (P.pairs[mid].seg_start <= seg) lo = mid; else hi = mid - 1;
+    }
+    const SelPair& Q = P.pairs[lo];
+    const int n = Q.seg_len;
+    const int seg_in_pair = seg - Q.seg_start;
+    const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg_in_pair) * n;
+    const int out0 = P.out_off[seg];
+    const int k = P.out_off[seg + 1] - out0;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+    if (P.seg_offsets && tid == 0) {
+        P.seg_offsets[P.seg_base + seg] = out0;
+        if (P.is_last && seg == P.n_segs - 1) P.seg_offsets[P.seg_base + seg + 1] = out0 + k;
+    }
+    if (k <= 0) return;
+
+    // ---- radix select: key of the k-th largest element
+    uint32_t prefix = 0, mask = 0;
+    int want = k, cnt_eq = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+        hist[tid] = 0;
+        __syncthreads();
+        for (int j = tid; j < n; j += kThreads) {
+            const uint32_t key = order_key(__ldg(sc + j));
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane l owns bins 255-8l ... 248-8l (descending)
+            int local[8], s = 0;
+#pragma unroll
+            for (int b = 0; b < 8; ++b) {
+                local[b] = hist[255 - 8 * lane - b];
+                s += local[b];
+            }
+            int incl = s;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const int excl = incl - s;
+            if (excl < want && want <= incl) {
+                int cum = excl;
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    if (cum < want && want <= cum + local[b]) {
+                        sh_prefix = prefix | (static_cast<uint32_t>(255 - 8 * lane - b) << shift);
+                        sh_want = want - cum;
+                        sh_cnt_eq = local[b];
+                    }
+                    cum += local[b];
+                }
+            }
+        }
+        __syncthreads();
+        prefix = sh_prefix;
+        want = sh_want;
+        cnt_eq = sh_cnt_eq;
+        mask |= 255u << shift;
+        __syncthreads();
+    }
+    const uint32_t thr = prefix;            // key of the k-th largest
+    const bool all_eq = (want == cnt_eq);   // every element equal to the threshold is kept
+
+    // ---- emit ascending: key > thr, plus the first `want` elements with key == thr
+    const int seg_first = seg_in_pair * n;  // kept indices are shared indices of the pair group
+    int run_eq = 0, run_out = 0;
+    for (int base = 0; base < n; base += kThreads) {
+        const int j = base + tid;
+        uint32_t key = 0;
+        bool valid = j < n;
+        if (valid) key = order_key(__ldg(sc + j));
+        const bool gt = valid && key > thr;
+        const bool eq = valid && key == thr;
+        bool sel;
+        if (all_eq) {
+            sel = gt || eq;
+        } else {
+            const unsigned beq = __ballot_sync(0xffffffffu, eq);
+            if (lane == 0) warp_tot[warp] = __popc(beq);
+            __syncthreads();
+            int rank = run_eq + __popc(beq & ((1u << lane) - 1u));
+            int tot = 0;
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                if (w < warp) rank += warp_tot[w];
+                tot += warp_tot[w];
+            }
+            run_eq += tot;
+            sel = gt || (eq && rank < want);
+            __syncthreads();
+        }
+        const unsigned bs = __ballot_sync(0xffffffffu, sel);
+        if (lane == 0) warp_tot[warp] = __popc(bs);
+        __syncthreads();
+        int pos = run_out + __popc(bs & ((1u << lane) - 1u));
+        int tot = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            if (w < warp) pos += warp_tot[w];
+            tot += warp_tot[w];
+        }
+        run_out += tot;
+        if (sel && pos < k) P.kept[out0 + pos] = seg_first + j;
+        __syncthreads();
+    }
+}
+
+}  // namespace
+
+}  // namespace ecospa
+
+using namespace ecospa;
+
+extern "C" ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, const int32_t* n_seg,
+                                                      const int32_t* seg_len, const int32_t* k_per_seg,
+                                                      int32_t n_pairs, int32_t* kept, int32_t* seg_offsets,
+                                                      void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!upsilon || !n_seg || !seg_len || !k_per_seg || n_pairs < 1 || !kept) return ECOSPA_ERR_INVALID;
+    int64_t total_segs = 0, total_d = 0, total_k = 0;
+    for (int p = 0; p < n_pairs; ++p) {
+        if (n_seg[p] < 1 || seg_len[p] < 1) return ECOSPA_ERR_INVALID;
+        if (seg_len[p] > (1 << 20)) return ECOSPA_ERR_UNSUPPORTED;
+        for (int s = 0; s < n_seg[p]; ++s) {
+            const int32_t k = k_per_seg[total_segs + s];
+            if (k < 0 || k > seg_len[p]) return ECOSPA_ERR_INVALID;
+            total_k += k;
+        }
+        total_segs += n_seg[p];
+        total_d += static_cast<int64_t>(n_seg[p]) * seg_len[p];
+    }
+    if (total_d > INT32_MAX || total_k > INT32_MAX) return ECOSPA_ERR_UNSUPPORTED;
+
+    static thread_local SelectParams sp;
+    int p = 0, s_in_p = 0;          // walk position: pair, segment inside pair
+    int32_t d_off = 0, out = 0, seg_global = 0;
+    while (p < n_pairs) {
+        int np = 0, ns = 0;
+        sp.seg_base = seg_global;
+        // a pair can be split across launches; each launch sees it as a pair starting at s_in_p
+        while (p < n_pairs && np < kMaxPairs && ns < kMaxSegs) {
+            const int take = std::min(n_seg[p] - s_in_p, kMaxSegs - ns);
+            SelPair& Q = sp.pairs[np++];
+            Q.seg_start = ns - s_in_p;   // so that (seg - seg_start) is the segment index inside the pair
+            Q.seg_len = seg_len[p];
+            Q.d_off = d_off;
+            Q.pad_ = 0;
+            for (int s = 0; s < take; ++s) {
+                sp.out_off[ns++] = out;
+                out += k_per_seg[seg_global++];
+            }
+            s_in_p += take;
+            if (s_in_p == n_seg[p]) {
+                d_off += n_seg[p] * seg_len[p];
+                ++p;
+                s_in_p = 0;
+            }
+        }
+        sp.out_off[ns] = out;
+        sp.upsilon = upsilon;
+        sp.kept = kept;
+        sp.seg_offsets = seg_offsets;
+        sp.n_pairs = np;
+        sp.n_segs = ns;
+        sp.is_last = (p >= n_pairs) ? 1 : 0;
+        select_kernel<<<ns, kThreads, 0, stream>>>(sp);
+        ecospa_status_t st = check_launch("select_kernel");
+        if (st != ECOSPA_OK) return st;
+    }
+    return ECOSPA_OK;
+}
