@@ -1,0 +1,661 @@
+// Grouped persistent bf16 GEMM for sm_100a: TMA -> shared memory ring -> tcgen05.mma (cta_group::1,
+// 128x256x16, fp32 accumulators in TMEM, double buffered) -> fused epilogues.
+//
+// One launch computes up to kMaxGemmOps independent products ("ops"), each C = sum over one or two
+// K segments of A_seg * B_seg with K-major or MN-major operands (chosen per segment, so that weights
+// and activations are consumed in whatever row-major orientation they are stored).  Warp roles:
+//   warp 0      producer: one elected lane issues the TMA loads of a k-block into a 4-stage ring
+//   warp 1      owns the 512 TMEM columns; one elected lane issues the MMAs and the commits
+//   warps 2..9  epilogue: two warps per TMEM lane quadrant, each takes half of the tile's columns
+// The tile list of all ops is walked with a static stride (tile = blockIdx.x + i * gridDim.x);
+// ops are ordered by decreasing contraction length so the long tiles start first.
+// Every mbarrier wait is bounded in time; on expiry the CTA records an error code in a device
+// status word, waits for its copies in flight, frees its TMEM and returns.
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+#include "gemm.cuh"
+
+namespace ecospa {
+
+namespace {
+
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kStages = 4;
+constexpr int kAStage = BM * BK * 2;        // 16 KB
+constexpr int kBStage = BN * BK * 2;        // 32 KB
+constexpr int kBHalf = kBStage / 2;
+constexpr int kAtomBytes = 64 * 64 * 2;     // one 64x64 bf16 swizzle atom of an MN-major operand
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kTmemCols = 512;
+constexpr int kMapsPerOp = 6;
+constexpr int kSmemBytes = kStages * (kAStage + kBStage) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+
+struct DevProblem {
+    int32_t M, N;
+    int32_t kblocks0, kblocks;   // k-blocks of segment 0, of both segments
+    int32_t tiles_m, tiles_n, tile_start;
+    int32_t n_per_tile;          // output columns per tile: 256, or 128 hidden units for EPI_SWIGLU
+    int32_t half1_n_off;         // n-coordinate of B half 1 relative to half 0
+    int32_t epi;
+    uint8_t a_mn[2], b_mn[2];
+    uint8_t map_a[2], map_b[2][2];
+    uint8_t out_f32, accumulate, bias_f32, pad_[5];
+    void* C;
+    void* C2;
+    void* C3;
+    const void* bias;
+    const void* H;
+    const void* Hb;
+    int64_t ldc, ldh;
+};
+
+struct GemmParams {
+    alignas(64) CUtensorMap maps[kMaxGemmOps * kMapsPerOp];
+    DevProblem prob[kMaxGemmOps];
+    int32_t n_problems, total_tiles;
+    int* status;
+};
+
+__device__ int g_gemm_status = 0;
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false if the wait gave up (or another thread of the CTA already did).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                atomicCAS(status, 0, code);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((addr >> 4) & 0x3fffu);
+    d |= static_cast<uint64_t>((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= static_cast<uint64_t>((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= 1ull << 46;   // descriptor version of this architecture
+    d |= 2ull << 61;   // 128-byte swizzle
+    return d;
+}
+
+// ------------------------------------------------------------------------------------------------
+// epilogue math (fp32)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
+__device__ __forceinline__ float dgelu_erf(float x) {
+    return 0.5f * (1.f + erff(x * 0.70710678118654752f)) + x * 0.39894228040143268f * __expf(-0.5f * x * x);
+}
+__device__ __forceinline__ float gelu_tanh(float x) {
+    const float u = 0.79788456080286536f * (x + 0.044715f * x * x * x);
+    return 0.5f * x * (1.f + tanhf(u));
+}
+__device__ __forceinline__ float dgelu_tanh(float x) {
+    const float u = 0.79788456080286536f * (x + 0.044715f * x * x * x);
+    const float t = tanhf(u);
+    const float du = 0.79788456080286536f * (1.f + 3.f * 0.044715f * x * x);
+    return 0.5f * (1.f + t) + 0.5f * x * (1.f - t * t) * du;
+}
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// 32 consecutive values of one row -> bf16 (or fp32) at `row_off` + n; nv = valid columns (<= 32)
+__device__ __forceinline__ void store_row32(void* base, int64_t row_off, int n, int nv, const float (&v)[32], bool f32) {
+    if (f32) {
+        float* p = static_cast<float*>(base) + row_off + n;
+        if (nv == 32) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                *reinterpret_cast<float4*>(p + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < nv) p[i] = v[i];
+        }
+    } else {
+        __nv_bfloat16* p = static_cast<__nv_bfloat16*>(base) + row_off + n;
+        if (nv == 32) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint4 q;
+                q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
+                q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
+                q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
+                q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
+                *reinterpret_cast<uint4*>(p + 8 * i) = q;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (i < nv) p[i] = __float2bfloat16_rn(v[i]);
+        }
+    }
+}
+
+__device__ __forceinline__ void load_row32(const void* base, int64_t row_off, int n, int nv, float (&v)[32], bool f32) {
+    if (f32) {
+        const float* p = static_cast<const float*>(base) + row_off + n;
+        if (nv == 32) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 q = *reinterpret_cast<const float4*>(p + 4 * i);
+                v[4 * i] = q.x; v[4 * i + 1] = q.y; v[4 * i + 2] = q.z; v[4 * i + 3] = q.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = i < nv ? p[i] : 0.f;
+        }
+    } else {
+        const unsigned short* p = static_cast<const unsigned short*>(base) + row_off + n;
+        if (nv == 32) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint4 q = *reinterpret_cast<const uint4*>(p + 8 * i);
+                v[8 * i + 0] = bf16_lo(q.x); v[8 * i + 1] = bf16_hi(q.x);
+                v[8 * i + 2] = bf16_lo(q.y); v[8 * i + 3] = bf16_hi(q.y);
+                v[8 * i + 4] = bf16_lo(q.z); v[8 * i + 5] = bf16_hi(q.z);
+                v[8 * i + 6] = bf16_lo(q.w); v[8 * i + 7] = bf16_hi(q.w);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = i < nv ? __uint_as_float(static_cast<uint32_t>(p[i]) << 16) : 0.f;
+        }
+    }
+}
+
+__device__ __forceinline__ const DevProblem& find_problem(const GemmParams& P, int tile) {
+    int pi = 0;
+#pragma unroll
+    for (int i = 1; i < kMaxGemmOps; ++i)
+        if (i < P.n_problems && P.prob[i].tile_start <= tile) pi = i;
+    return P.prob[pi];
+}
+
+// ------------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;       // 1024-byte aligned stage memory
+    uint8_t* smem = smem_raw + (base - raw_addr);
+    const uint32_t sA = base, sB = base + kStages * kAStage;
+    uint8_t* tail = smem + kStages * (kAStage + kBStage);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);        // full[4], empty[4], tmem_full[2], tmem_empty[2]
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 12 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 12 * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
+    auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), kEpiWarps);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+                const DevProblem& Q = find_problem(P, tile);
+                const int local = tile - Q.tile_start;
+                const int m0 = (local % Q.tiles_m) * BM;
+                const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
+                for (int kb = 0; kb < Q.kblocks; ++kb) {
+                    const int seg = kb >= Q.kblocks0 ? 1 : 0;
+                    const int k0 = (seg ? kb - Q.kblocks0 : kb) * BK;
+                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
+                    mbar_expect_tx(full_bar(stage), kAStage + kBStage);
+                    const uint32_t a_dst = sA + stage * kAStage, b_dst = sB + stage * kBStage;
+                    const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
+                    if (!Q.a_mn[seg]) {
+                        tma_load_2d(a_dst, ma, k0, m0, full_bar(stage));                    // box 64(k) x 128(m)
+                    } else {
+                        tma_load_2d(a_dst, ma, m0, k0, full_bar(stage));                    // box 64(m) x 64(k)
+                        tma_load_2d(a_dst + kAtomBytes, ma, m0 + 64, k0, full_bar(stage));
+                    }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const CUtensorMap* mb = &P.maps[Q.map_b[seg][h]];
+                        const int nc = n0 + h * Q.half1_n_off;
+                        const uint32_t dst = b_dst + h * kBHalf;
+                        if (!Q.b_mn[seg]) {
+                            tma_load_2d(dst, mb, k0, nc, full_bar(stage));                  // box 64(k) x 128(n)
+                        } else {
+                            tma_load_2d(dst, mb, nc, k0, full_bar(stage));                  // box 64(n) x 64(k)
+                            tma_load_2d(dst + kAtomBytes, mb, nc + 64, k0, full_bar(stage));
+                        }
+                    }
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++it) {
+                const DevProblem& Q = find_problem(P, tile);
+                const int acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1u;
+                if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 2, P.status))) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < Q.kblocks; ++kb) {
+                    const int seg = kb >= Q.kblocks0 ? 1 : 0;
+                    if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, 3, P.status))) break;
+                    tc_fence_after();
+                    const uint32_t a_mn = Q.a_mn[seg], b_mn = Q.b_mn[seg];
+                    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) |
+                                           (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
+                    const uint64_t a_desc = make_smem_desc(sA + stage * kAStage, a_mn ? kAtomBytes : 16, 1024);
+                    const uint64_t b_desc = make_smem_desc(sB + stage * kBStage, b_mn ? kAtomBytes : 16, 1024);
+                    const uint64_t a_step = a_mn ? (2048 >> 4) : (32 >> 4);   // per 16 k: two 8-row groups, or 32 bytes
+                    const uint64_t b_step = b_mn ? (2048 >> 4) : (32 >> 4);
+#pragma unroll
+                    for (int ks = 0; ks < BK / 16; ++ks)
+                        tc_mma_bf16(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
+                    tc_commit(empty_bar(stage));      // the stage is free once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) tc_commit(tfull_bar(acc));    // accumulator complete
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int ew = warp - 2;
+        const int quad = warp & 3;            // TMEM lanes this warp may read: [32*quad, 32*quad + 32)
+        const int half = ew >> 2;             // which half of the tile's columns
+        int it = 0;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++it) {
+            const DevProblem& Q = find_problem(P, tile);
+            const int local = tile - Q.tile_start;
+            const int m = (local % Q.tiles_m) * BM + quad * 32 + lane;
+            const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
+            const int acc = it & 1;
+            const uint32_t acc_phase = (it >> 1) & 1u;
+            if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 4, P.status))) break;
+            tc_fence_after();
+            const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
+            const bool row_ok = m < Q.M;
+            const int64_t c_off = static_cast<int64_t>(m) * Q.ldc;
+            const int64_t h_off = static_cast<int64_t>(m) * Q.ldh;
+            const int epi = Q.epi;
+            if (epi == EPI_SWIGLU) {
+                // accumulator columns [0,128) = gate, [128,256) = up for hidden units n0 .. n0+127
+#pragma unroll 1
+                for (int c = 0; c < 2; ++c) {
+                    const int hc = half * 64 + c * 32;
+                    uint32_t rg[32], ru[32];
+                    tc_ld32(t_row + hc, rg);
+                    tc_ld32(t_row + 128 + hc, ru);
+                    tc_wait_ld();
+                    const int n = n0 + hc;
+                    const int nv = min(32, Q.N - n);
+                    if (row_ok && nv > 0) {
+                        float g[32], u[32], a[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            g[i] = __uint_as_float(rg[i]);
+                            u[i] = __uint_as_float(ru[i]);
+                            a[i] = g[i] * sigmoidf_(g[i]) * u[i];
+                        }
+                        store_row32(Q.C, c_off, n, nv, g, false);
+                        store_row32(Q.C2, c_off, n, nv, u, false);
+                        store_row32(Q.C3, c_off, n, nv, a, false);
+                    }
+                }
+            } else {
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    const int col = half * 128 + c * 32;
+                    uint32_t r[32];
+                    tc_ld32(t_row + col, r);
+                    tc_wait_ld();
+                    const int n = n0 + col;
+                    const int nv = min(32, Q.N - n);
+                    if (!(row_ok && nv > 0)) continue;
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                    if (Q.bias) {
+                        float b[32];
+                        load_row32(Q.bias, 0, n, nv, b, Q.bias_f32 != 0);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] += b[i];
+                    }
+                    if (epi == EPI_STORE) {
+                        if (Q.accumulate) {
+                            float o[32];
+                            load_row32(Q.C, c_off, n, nv, o, Q.out_f32 != 0);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] += o[i];
+                        }
+                        store_row32(Q.C, c_off, n, nv, v, Q.out_f32 != 0);
+                    } else if (epi == EPI_GELU_ERF || epi == EPI_GELU_TANH) {
+                        store_row32(Q.C, c_off, n, nv, v, false);
+                        float a[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) a[i] = epi == EPI_GELU_ERF ? gelu_erf(v[i]) : gelu_tanh(v[i]);
+                        store_row32(Q.C2, c_off, n, nv, a, false);
+                    } else if (epi == EPI_DGELU_ERF || epi == EPI_DGELU_TANH) {
+                        float h[32];
+                        load_row32(Q.H, h_off, n, nv, h, false);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] *= epi == EPI_DGELU_ERF ? dgelu_erf(h[i]) : dgelu_tanh(h[i]);
+                        store_row32(Q.C, c_off, n, nv, v, false);
+                    } else {  // EPI_DSWIGLU
+                        float hg[32], hu[32], dg[32];
+                        load_row32(Q.H, h_off, n, nv, hg, false);
+                        load_row32(Q.Hb, h_off, n, nv, hu, false);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float s = sigmoidf_(hg[i]);
+                            dg[i] = v[i] * hu[i] * s * (1.f + hg[i] * (1.f - s));
+                            v[i] = v[i] * hg[i] * s;
+                        }
+                        store_row32(Q.C, c_off, n, nv, dg, false);
+                        store_row32(Q.C2, c_off, n, nv, v, false);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        // give copies that are still in flight time to land before the shared memory is released
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeFn get_encode() {
+    static EncodeFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    });
+    return fn;
+}
+
+// Tensor map of a stored row-major bf16 matrix; box = 64 elements along the row x box_rows rows.
+ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows) {
+    EncodeFn enc = get_encode();
+    if (!enc) {
+        set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
+        return ECOSPA_ERR_CUDA;
+    }
+    if (!s.ptr || s.rows < 1 || s.cols < 1 || s.ld < s.cols) return ECOSPA_ERR_INVALID;
+    if (!aligned16(s.ptr) || (s.ld * 2) % 16 != 0) return ECOSPA_ERR_ALIGNMENT;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(s.cols), static_cast<cuuint64_t>(s.rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(s.ld) * 2};
+    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(s.ptr), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+        return ECOSPA_ERR_CUDA;
+    }
+    return ECOSPA_OK;
+}
+
+int g_num_sms = 0;
+int* g_status_ptr = nullptr;
+
+ecospa_status_t gemm_setup() {
+    static std::once_flag once;
+    static ecospa_status_t st = ECOSPA_OK;
+    std::call_once(once, [] {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&g_status_ptr), g_gemm_status);
+        if (e != cudaSuccess) {
+            set_cuda_error(e, "gemm setup");
+            st = ECOSPA_ERR_CUDA;
+        }
+    });
+    return st;
+}
+
+}  // namespace
+
+ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t stream) {
+    if (!ops || n_ops < 1 || n_ops > kMaxGemmOps) return ECOSPA_ERR_INVALID;
+    ecospa_status_t st = gemm_setup();
+    if (st != ECOSPA_OK) return st;
+
+    // longest contraction first
+    int order[kMaxGemmOps];
+    int64_t ktot[kMaxGemmOps];
+    for (int i = 0; i < n_ops; ++i) {
+        order[i] = i;
+        ktot[i] = 0;
+        for (int s = 0; s < ops[i].n_kseg; ++s) ktot[i] += ceil_div(ops[i].seg[s].K, BK);
+    }
+    std::stable_sort(order, order + n_ops, [&](int a, int b) { return ktot[a] > ktot[b]; });
+
+    static thread_local GemmParams gp;
+    int tiles = 0;
+    for (int oi = 0; oi < n_ops; ++oi) {
+        const GemmOp& op = ops[order[oi]];
+        DevProblem& Q = gp.prob[oi];
+        std::memset(&Q, 0, sizeof(Q));
+        if (op.M < 1 || op.N < 1 || op.n_kseg < 1 || op.n_kseg > 2 || !op.C || op.ldc < 1) return ECOSPA_ERR_INVALID;
+        if (op.M > INT32_MAX || op.N > INT32_MAX) return ECOSPA_ERR_INVALID;
+        const bool swiglu = op.epi == EPI_SWIGLU;
+        const int out_eb = op.out_f32 ? 4 : 2;
+        if (!aligned16(op.C) || (op.ldc * out_eb) % 16) return ECOSPA_ERR_ALIGNMENT;
+        if ((op.epi == EPI_GELU_ERF || op.epi == EPI_GELU_TANH || op.epi == EPI_DSWIGLU || swiglu) && (!op.C2 || !aligned16(op.C2)))
+            return op.C2 ? ECOSPA_ERR_ALIGNMENT : ECOSPA_ERR_INVALID;
+        if (swiglu && (!op.C3 || !aligned16(op.C3))) return op.C3 ? ECOSPA_ERR_ALIGNMENT : ECOSPA_ERR_INVALID;
+        if (op.epi >= EPI_DGELU_ERF) {
+            if (!op.H || (op.epi == EPI_DSWIGLU && !op.Hb)) return ECOSPA_ERR_INVALID;
+            if (!aligned16(op.H) || (op.Hb && !aligned16(op.Hb)) || (op.ldh * 2) % 16) return ECOSPA_ERR_ALIGNMENT;
+        }
+        if (op.out_f32 && op.epi != EPI_STORE) return ECOSPA_ERR_UNSUPPORTED;
+        if (op.bias && !aligned16(op.bias)) return ECOSPA_ERR_ALIGNMENT;
+        Q.M = static_cast<int32_t>(op.M);
+        Q.N = static_cast<int32_t>(op.N);
+        Q.n_per_tile = swiglu ? 128 : BN;
+        Q.half1_n_off = swiglu ? 0 : 128;
+        Q.epi = op.epi;
+        Q.out_f32 = op.out_f32;
+        Q.accumulate = op.accumulate;
+        Q.bias_f32 = op.bias_f32;
+        Q.C = op.C; Q.C2 = op.C2; Q.C3 = op.C3;
+        Q.bias = op.bias; Q.H = op.H; Q.Hb = op.Hb;
+        Q.ldc = op.ldc; Q.ldh = op.ldh;
+        for (int s = 0; s < op.n_kseg; ++s) {
+            const KSegment& ks = op.seg[s];
+            if (ks.K < 1) return ECOSPA_ERR_INVALID;
+            // stored shapes must match the logical (M, N, K)
+            const Stored& a = ks.a;
+            if (ks.a_mn ? (a.rows != ks.K || a.cols != op.M) : (a.rows != op.M || a.cols != ks.K)) return ECOSPA_ERR_INVALID;
+            const int mi = oi * kMapsPerOp;
+            if ((st = encode_map(&gp.maps[mi + s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
+            Q.map_a[s] = static_cast<uint8_t>(mi + s);
+            for (int h = 0; h < 2; ++h) {
+                const Stored& b = (swiglu && h == 1) ? ks.b[1] : ks.b[0];
+                if (ks.b_mn ? (b.rows != ks.K || b.cols != op.N) : (b.rows != op.N || b.cols != ks.K)) return ECOSPA_ERR_INVALID;
+                if ((st = encode_map(&gp.maps[mi + 2 + 2 * s + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
+                Q.map_b[s][h] = static_cast<uint8_t>(mi + 2 + 2 * s + h);
+            }
+            Q.a_mn[s] = ks.a_mn;
+            Q.b_mn[s] = ks.b_mn;
+            const int32_t kb = static_cast<int32_t>(ceil_div(ks.K, BK));
+            if (s == 0) Q.kblocks0 = kb;
+            Q.kblocks += kb;
+        }
+        Q.tiles_m = static_cast<int32_t>(ceil_div(op.M, BM));
+        Q.tiles_n = static_cast<int32_t>(ceil_div(op.N, Q.n_per_tile));
+        Q.tile_start = tiles;
+        tiles += Q.tiles_m * Q.tiles_n;
+    }
+    gp.n_problems = n_ops;
+    gp.total_tiles = tiles;
+    gp.status = g_status_ptr;
+    const int grid = std::min(tiles, g_num_sms);
+    gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(gp);
+    return check_launch("gemm_kernel");
+}
+
+}  // namespace ecospa
+
+extern "C" ecospa_status_t ecospa_device_status(void* stream, int32_t* code) {
+    if (!code) return ECOSPA_ERR_INVALID;
+    ecospa_status_t st = ecospa::gemm_setup();
+    if (st != ECOSPA_OK) return st;
+    cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+    int v = 0;
+    if (e == cudaSuccess) e = cudaMemcpy(&v, ecospa::g_status_ptr, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) {
+        ecospa::set_cuda_error(e, "ecospa_device_status");
+        return ECOSPA_ERR_CUDA;
+    }
+    *code = v;
+    if (v != 0) {
+        cudaMemset(ecospa::g_status_ptr, 0, sizeof(int));
+        return ECOSPA_ERR_TIMEOUT;
+    }
+    return ECOSPA_OK;
+}
