@@ -150,6 +150,92 @@ ecospa_status_t ecospa_compact_pair(const ecospa_pair_t* pair, const int32_t* ke
                                     const ecospa_mat_t* w1_out, const ecospa_mat_t* w1b_out,
                                     const ecospa_mat_t* w2_out, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Step 4: forward / backward of the compacted coupled pairs.
+ *
+ * The dense layer math of Eq. 2 (Q, K, V projections), Eq. 5 (output projection with W^O as a stack of
+ * per-head row blocks) and Eq. 3 (FFN; SwiGLU variant per the footnote to Eq. 8) evaluated on the
+ * matrices that aligned removal leaves, and the reverse-mode derivatives of the same expressions.
+ * bf16 operands on the tensor cores with fp32 accumulation; the FFN activation (and, in the backward
+ * pass, its derivative) is fused into the epilogue of the W_1 (resp. dY W_2^T) product.
+ *
+ * Common conventions
+ *   T, d_m        tokens (batch*seq) and model width; n / k = real number of kept shared indices.
+ *   dtype         taken from the first weight descriptor.  ECOSPA_BF16: every activation, gradient and
+ *                 output below is bf16.  ECOSPA_F32: X, upstream gradients, biases, Y/Q/K/V/Out, dX and all
+ *                 weight/bias gradients are fp32; operands are rounded to bf16 in the workspace first.
+ *                 The saved FFN tensors H, Hb, A are bf16 in both cases.
+ *   weights       compacted matrices as written by step 3: W_Q^c, W_K^c, W_V^c, W_1^c (W_gate^c, W_up^c)
+ *                 are ECOSPA_SHARED_COLS (d_m x n, pitch ld); W_O^c, W_2^c are ECOSPA_SHARED_ROWS
+ *                 (n x d_m).  other_dim must equal d_m.  The other storage orientation returns
+ *                 ECOSPA_ERR_UNSUPPORTED.
+ *   pitches       all ld* in elements.  Every base pointer must be 16-byte aligned and every pitch a
+ *                 multiple of 16 bytes (ECOSPA_ERR_ALIGNMENT otherwise); gradient outputs use the pitch
+ *                 of a compacted weight (padded), pad columns are left untouched.
+ *   workspace     DEVICE scratch, 16-byte aligned, at least ecospa_proj_workspace_bytes /
+ *                 ecospa_ffn_workspace_bytes; may be NULL when that function returns 0.
+ *   1/sqrt(d_h)   is not applied: Q^c and K^c are the plain projections.
+ * All DEVICE pointers; results are deterministic (fixed summation order).  A device-side wait that
+ * expires records a code readable with ecospa_device_status.
+ */
+size_t ecospa_proj_workspace_bytes(int64_t T, int64_t d_m, int64_t n, int32_t dtype);
+size_t ecospa_ffn_workspace_bytes(int64_t T, int64_t d_m, int64_t k, int32_t act, int32_t dtype);
+
+/* Q^c = X W_Q^c + b_Q^c, K^c = X W_K^c + b_K^c (Eq. 2 on the compacted pair).  X: T x d_m (pitch ldx);
+ * Qc, Kc: T x n (pitch ld_out).  bq_c / bk_c may be NULL.  wk_c == NULL computes Q^c only. */
+ecospa_status_t ecospa_coupled_qk_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, const ecospa_mat_t* wq_c,
+                                      const ecospa_mat_t* wk_c, int64_t n, const void* bq_c, const void* bk_c,
+                                      void* Qc, void* Kc, int64_t ld_out, void* workspace, size_t workspace_bytes,
+                                      void* stream);
+/* Given dQc, dKc (T x n, pitch ld_dqk): dX = dQc W_Q^cT + dKc W_K^cT (added to dX if accumulate_dX),
+ * dW_Q^c = X^T dQc, dW_K^c = X^T dKc (d_m x n, pitch ld_dw), db = column sums (may be NULL). */
+ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, const ecospa_mat_t* wq_c,
+                                      const ecospa_mat_t* wk_c, int64_t n, const void* dQc, const void* dKc,
+                                      int64_t ld_dqk, void* dX, int64_t ld_dx, int32_t accumulate_dX, void* dWq_c,
+                                      void* dWk_c, int64_t ld_dw, void* dbq_c, void* dbk_c, void* workspace,
+                                      size_t workspace_bytes, void* stream);
+
+/* V^c = X W_V^c + b_V^c;  Out = Ctx W_O^c + b_O, where Ctx (T x n) is the attention-mixed values of the
+ * compacted heads supplied by the caller (Eq. 5).  */
+ecospa_status_t ecospa_coupled_vo_fwd_v(const void* X, int64_t ldx, int64_t T, int64_t d_m, const ecospa_mat_t* wv_c,
+                                        int64_t n, const void* bv_c, void* Vc, int64_t ld_out, void* workspace,
+                                        size_t workspace_bytes, void* stream);
+ecospa_status_t ecospa_coupled_vo_fwd_o(const void* Ctx, int64_t ld_ctx, int64_t T, int64_t d_m,
+                                        const ecospa_mat_t* wo_c, int64_t n, const void* bo, void* Out, int64_t ld_out,
+                                        void* workspace, size_t workspace_bytes, void* stream);
+/* dCtx = dOut W_O^cT, dW_O^c = Ctx^T dOut (n x d_m), dbo = colsum(dOut); dW_V^c = X^T dVc, dX (+)= dVc W_V^cT,
+ * dbv = colsum(dVc). */
+ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, const void* Ctx, int64_t ld_ctx, int64_t T,
+                                      int64_t d_m, const ecospa_mat_t* wv_c, const ecospa_mat_t* wo_c, int64_t n,
+                                      const void* dVc, int64_t ld_dv, const void* dOut, int64_t ld_dout, void* dX,
+                                      int64_t ld_dx, int32_t accumulate_dX, void* dCtx, int64_t ld_dctx, void* dWv_c,
+                                      int64_t ld_dwv, void* dWo_c, int64_t ld_dwo, void* dbv_c, void* dbo,
+                                      void* workspace, size_t workspace_bytes, void* stream);
+
+/* FFN on a compacted pair with k hidden units (Eq. 3):
+ *   GELU   : H = X W_1^c + b_1^c, A = GELU(H), Y = A W_2^c + b_2
+ *   SwiGLU : H = X W_gate^c, Hb = X W_up^c, A = silu(H) (.) Hb, Y = A W_2^c        (w1_c = gate, w1b_c = up)
+ * H, Hb, A: bf16 T x k (pitch ld_h), written for the backward pass; Y: T x d_m (pitch ld_y). */
+ecospa_status_t ecospa_coupled_ffn_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, int32_t act,
+                                       const ecospa_mat_t* w1_c, const ecospa_mat_t* w1b_c, const ecospa_mat_t* w2_c,
+                                       int64_t k, const void* b1_c, const void* b2, void* Y, int64_t ld_y, void* H,
+                                       void* Hb, void* A, int64_t ld_h, void* workspace, size_t workspace_bytes,
+                                       void* stream);
+/* Given dY (T x d_m): dH = (dY W_2^cT) (.) act'(H)  [SwiGLU: dH = dA (.) Hb (.) silu'(H), dHb = dA (.) silu(H)],
+ * dW_2^c = A^T dY (k x d_m, pitch ld_dw2), dW_1^c = X^T dH (d_m x k, pitch ld_dw1; dW1b_c = X^T dHb),
+ * dX = dH W_1^cT (+ dHb W_up^cT), db1 = colsum(dH) (GELU only), db2 = colsum(dY); db* may be NULL. */
+ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, int32_t act,
+                                       const ecospa_mat_t* w1_c, const ecospa_mat_t* w1b_c, const ecospa_mat_t* w2_c,
+                                       int64_t k, const void* H, const void* Hb, const void* A, int64_t ld_h,
+                                       const void* dY, int64_t ld_dy, void* dX, int64_t ld_dx, void* dW1_c,
+                                       void* dW1b_c, int64_t ld_dw1, void* dW2_c, int64_t ld_dw2, void* db1_c,
+                                       void* db2, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Synchronises `stream` and reports the device status word: ECOSPA_OK and *code = 0, or
+ * ECOSPA_ERR_TIMEOUT and *code = which bounded wait expired (1 producer, 2 accumulator-free,
+ * 3 operands-ready, 4 accumulator-ready); the word is cleared.  This is the one call that blocks. */
+ecospa_status_t ecospa_device_status(void* stream, int32_t* code);
+
 #ifdef __cplusplus
 }
 #endif

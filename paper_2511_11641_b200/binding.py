@@ -181,3 +181,158 @@ def ecospa_compact_pair(p: Pair, kept: torch.Tensor, n_kept: int, w1_out: torch.
                                    _stream(stream))
     if st != 0:
         raise EcospaError(st, "ecospa_compact_pair")
+
+
+# ---------------------------------------------------------------------------------------------
+# compacted-pair forward / backward
+# ---------------------------------------------------------------------------------------------
+
+_LAYER_SIGS = {
+    "ecospa_proj_workspace_bytes": (C.c_size_t, [C.c_int64, C.c_int64, C.c_int64, C.c_int32]),
+    "ecospa_ffn_workspace_bytes": (C.c_size_t, [C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.c_int32]),
+    "ecospa_coupled_qk_fwd": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64,
+                                        C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                        C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_qk_bwd": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64,
+                                        C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32,
+                                        C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p,
+                                        C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_vo_fwd_v": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p,
+                                          C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_vo_fwd_o": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p,
+                                          C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_vo_bwd": (C.c_int, [C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int64, C.c_int64,
+                                        C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                        C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                                        C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_ffn_fwd": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_ffn_bwd": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                         C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64,
+                                         C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
+}
+_sigs_done = False
+
+
+def _fn(name: str):
+    global _sigs_done
+    l = lib()
+    if not _sigs_done:
+        for n, (res, args) in _LAYER_SIGS.items():
+            f = getattr(l, n)
+            f.restype, f.argtypes = res, args
+        _sigs_done = True
+    return getattr(l, name)
+
+
+def _ws(ws: Optional[torch.Tensor]):
+    return (None, 0) if ws is None else (ws.data_ptr(), ws.numel() * ws.element_size())
+
+
+def _ref(m: Optional[Mat]):
+    return None if m is None else C.addressof(m)
+
+
+def _check(st: int, where: str) -> None:
+    if st != 0:
+        raise EcospaError(st, where)
+
+
+def ecospa_proj_workspace_bytes(T: int, d_m: int, n: int, dtype: int) -> int:
+    return int(_fn("ecospa_proj_workspace_bytes")(T, d_m, n, dtype))
+
+
+def ecospa_ffn_workspace_bytes(T: int, d_m: int, k: int, act: int, dtype: int) -> int:
+    return int(_fn("ecospa_ffn_workspace_bytes")(T, d_m, k, act, dtype))
+
+
+def ecospa_coupled_qk_fwd(X, wq_c, wk_c, n: int, Qc, Kc, bq_c=None, bk_c=None, workspace=None, stream=None) -> None:
+    """wq_c / wk_c: compacted weight buffers of shape (d_m, pitch); Qc / Kc: (T, pitch_out)."""
+    T, d_m = X.shape
+    mq = mat(wq_c, SHARED_COLS)
+    mk = mat(wk_c, SHARED_COLS) if wk_c is not None else None
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_qk_fwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), n, _ptr(bq_c), _ptr(bk_c),
+                                        Qc.data_ptr(), _ptr(Kc), Qc.stride(0), wp, wb, _stream(stream)),
+           "ecospa_coupled_qk_fwd")
+
+
+def ecospa_coupled_qk_bwd(X, wq_c, wk_c, n: int, dQc, dKc, dX, dWq_c, dWk_c, dbq_c=None, dbk_c=None,
+                          accumulate_dX: bool = False, workspace=None, stream=None) -> None:
+    T, d_m = X.shape
+    mq = mat(wq_c, SHARED_COLS)
+    mk = mat(wk_c, SHARED_COLS) if wk_c is not None else None
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_qk_bwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), n, dQc.data_ptr(), _ptr(dKc),
+                                        dQc.stride(0), dX.data_ptr(), dX.stride(0), int(accumulate_dX), dWq_c.data_ptr(),
+                                        _ptr(dWk_c), dWq_c.stride(0), _ptr(dbq_c), _ptr(dbk_c), wp, wb, _stream(stream)),
+           "ecospa_coupled_qk_bwd")
+
+
+def ecospa_coupled_vo_fwd_v(X, wv_c, n: int, Vc, bv_c=None, workspace=None, stream=None) -> None:
+    T, d_m = X.shape
+    mv = mat(wv_c, SHARED_COLS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_vo_fwd_v")(X.data_ptr(), X.stride(0), T, d_m, _ref(mv), n, _ptr(bv_c), Vc.data_ptr(),
+                                          Vc.stride(0), wp, wb, _stream(stream)), "ecospa_coupled_vo_fwd_v")
+
+
+def ecospa_coupled_vo_fwd_o(Ctx, wo_c, n: int, Out, bo=None, workspace=None, stream=None) -> None:
+    T = Ctx.shape[0]
+    d_m = wo_c.shape[1]
+    mo = mat(wo_c, SHARED_ROWS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_vo_fwd_o")(Ctx.data_ptr(), Ctx.stride(0), T, d_m, _ref(mo), n, _ptr(bo), Out.data_ptr(),
+                                          Out.stride(0), wp, wb, _stream(stream)), "ecospa_coupled_vo_fwd_o")
+
+
+def ecospa_coupled_vo_bwd(X, Ctx, wv_c, wo_c, n: int, dVc, dOut, dX, dCtx, dWv_c, dWo_c, dbv_c=None, dbo=None,
+                          accumulate_dX: bool = False, workspace=None, stream=None) -> None:
+    T, d_m = X.shape
+    mv, mo = mat(wv_c, SHARED_COLS), mat(wo_c, SHARED_ROWS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_vo_bwd")(X.data_ptr(), X.stride(0), Ctx.data_ptr(), Ctx.stride(0), T, d_m, _ref(mv), _ref(mo),
+                                        n, dVc.data_ptr(), dVc.stride(0), dOut.data_ptr(), dOut.stride(0), dX.data_ptr(),
+                                        dX.stride(0), int(accumulate_dX), dCtx.data_ptr(), dCtx.stride(0), dWv_c.data_ptr(),
+                                        dWv_c.stride(0), dWo_c.data_ptr(), dWo_c.stride(0), _ptr(dbv_c), _ptr(dbo), wp, wb,
+                                        _stream(stream)), "ecospa_coupled_vo_bwd")
+
+
+def ecospa_coupled_ffn_fwd(X, act: int, w1_c, w2_c, k: int, Y, H, A, w1b_c=None, Hb=None, b1_c=None, b2=None,
+                           workspace=None, stream=None) -> None:
+    T, d_m = X.shape
+    m1 = mat(w1_c, SHARED_COLS)
+    m1b = mat(w1b_c, SHARED_COLS) if w1b_c is not None else None
+    m2 = mat(w2_c, SHARED_ROWS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_ffn_fwd")(X.data_ptr(), X.stride(0), T, d_m, act, _ref(m1), _ref(m1b), _ref(m2), k, _ptr(b1_c),
+                                         _ptr(b2), Y.data_ptr(), Y.stride(0), H.data_ptr(), _ptr(Hb), A.data_ptr(),
+                                         H.stride(0), wp, wb, _stream(stream)), "ecospa_coupled_ffn_fwd")
+
+
+def ecospa_coupled_ffn_bwd(X, act: int, w1_c, w2_c, k: int, H, A, dY, dX, dW1_c, dW2_c, w1b_c=None, Hb=None,
+                           dW1b_c=None, db1_c=None, db2=None, workspace=None, stream=None) -> None:
+    T, d_m = X.shape
+    m1 = mat(w1_c, SHARED_COLS)
+    m1b = mat(w1b_c, SHARED_COLS) if w1b_c is not None else None
+    m2 = mat(w2_c, SHARED_ROWS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_ffn_bwd")(X.data_ptr(), X.stride(0), T, d_m, act, _ref(m1), _ref(m1b), _ref(m2), k, H.data_ptr(),
+                                         _ptr(Hb), A.data_ptr(), H.stride(0), dY.data_ptr(), dY.stride(0), dX.data_ptr(),
+                                         dX.stride(0), dW1_c.data_ptr(), _ptr(dW1b_c), dW1_c.stride(0), dW2_c.data_ptr(),
+                                         dW2_c.stride(0), _ptr(db1_c), _ptr(db2), wp, wb, _stream(stream)),
+           "ecospa_coupled_ffn_bwd")
+
+
+def ecospa_device_status(stream=None) -> int:
+    """Synchronises the stream; returns 0 or raises EcospaError(ERR_TIMEOUT) carrying the wait code."""
+    code = C.c_int32(0)
+    st = _fn("ecospa_device_status")(_stream(stream), C.addressof(code))
+    if st != 0:
+        e = EcospaError(st, f"ecospa_device_status (wait code {code.value})")
+        e.code = code.value
+        raise e
+    return 0

@@ -1,0 +1,445 @@
+// Forward / backward of the compacted coupled pairs (Eq. 2, 3, 5 after aligned removal), expressed as
+// grouped launches of the tcgen05 GEMM engine plus two small helper kernels (fp32 -> bf16 staging for
+// fp32 models, and column sums for the bias gradients).
+//
+// Storage convention accepted here (the one the equations are written in):
+//   W_Q^c, W_K^c, W_V^c, W_1^c (gate/up): d_m x n row-major  (ECOSPA_SHARED_COLS, pitch ld >= n)
+//   W_O^c, W_2^c (down)                 : n x d_m row-major  (ECOSPA_SHARED_ROWS)
+// so every product below consumes its operands as stored (K-major or MN-major UMMA operands); nothing
+// is transposed in memory.
+
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+#include "common.cuh"
+#include "gemm.cuh"
+
+namespace ecospa {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// ------------------------------------------------------------------------------------------------
+// helper kernels
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) cast_f32_bf16_kernel(const float* __restrict__ in, int64_t ld_in,
+                                                                 uint16_t* __restrict__ out, int64_t ld_out, int64_t rows,
+                                                                 int64_t cols, int64_t cols_out) {
+    // one thread per 4 output columns; columns [cols, cols_out) are zero-filled
+    const int64_t per_row = (cols_out + 3) / 4;
+    const int64_t total = rows * per_row;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(kThreads) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * kThreads) {
+        const int64_t r = i / per_row, c = (i % per_row) * 4;
+        for (int e = 0; e < 4; ++e) {
+            if (c + e < cols_out) {
+                const float v = (c + e < cols) ? in[r * ld_in + c + e] : 0.f;
+                __nv_bfloat16 b = __float2bfloat16_rn(v);
+                out[r * ld_out + c + e] = *reinterpret_cast<uint16_t*>(&b);
+            }
+        }
+    }
+}
+
+// partial[chunk][c] = sum over the chunk's rows of M[r][c];  M is bf16 (rows x cols, pitch ld)
+constexpr int kSumRows = 256;
+__global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const uint16_t* __restrict__ M, int64_t ld, int64_t rows,
+                                                                  int64_t cols, float* __restrict__ partial) {
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kSumRows;
+    const int64_t r1 = r0 + kSumRows < rows ? r0 + kSumRows : rows;
+    if (c >= cols) return;
+    float s = 0.f;
+    for (int64_t r = r0; r < r1; ++r) s += __uint_as_float(static_cast<uint32_t>(M[r * ld + c]) << 16);
+    partial[static_cast<int64_t>(blockIdx.y) * cols + c] = s;
+}
+__global__ void __launch_bounds__(kThreads) colsum_final_kernel(const float* __restrict__ partial, int chunks, int64_t cols,
+                                                                void* out, int out_f32) {
+    const int c = blockIdx.x * kThreads + threadIdx.x;
+    if (c >= cols) return;
+    float s = 0.f;
+    for (int k = 0; k < chunks; ++k) s += partial[static_cast<int64_t>(k) * cols + c];
+    if (out_f32) static_cast<float*>(out)[c] = s;
+    else static_cast<__nv_bfloat16*>(out)[c] = __float2bfloat16_rn(s);
+}
+
+// ------------------------------------------------------------------------------------------------
+// workspace bump allocator and operand staging
+// ------------------------------------------------------------------------------------------------
+struct Arena {
+    char* base = nullptr;
+    size_t size = 0, used = 0;
+    void* take(size_t bytes) {
+        const size_t a = (used + 255) & ~size_t(255);
+        if (!base || a + bytes > size) return nullptr;
+        used = a + bytes;
+        return base + a;
+    }
+};
+inline size_t arena_need(size_t bytes) { return ((bytes + 255) & ~size_t(255)) + 256; }
+
+struct Ctx {
+    cudaStream_t stream = nullptr;
+    Arena arena;
+    int dtype = ECOSPA_BF16;  // of the model (activations, weights, outputs)
+    ecospa_status_t st = ECOSPA_OK;
+};
+
+// A (rows x cols, pitch ld) matrix of the model dtype as a bf16 Stored operand (staged if fp32).
+Stored as_bf16(Ctx& cx, const void* p, int64_t rows, int64_t cols, int64_t ld) {
+    Stored s;
+    if (cx.st != ECOSPA_OK) return s;
+    if (!p || rows < 1 || cols < 1 || ld < cols) {
+        cx.st = ECOSPA_ERR_INVALID;
+        return s;
+    }
+    if (cx.dtype == ECOSPA_BF16) {
+        s.ptr = p; s.rows = rows; s.cols = cols; s.ld = ld;
+        return s;
+    }
+    const int64_t ldo = round_up(cols, 8);
+    void* buf = cx.arena.take(static_cast<size_t>(rows) * ldo * 2);
+    if (!buf) {
+        cx.st = ECOSPA_ERR_WORKSPACE;
+        return s;
+    }
+    const int64_t total = rows * ((ldo + 3) / 4);
+    const int grid = static_cast<int>(std::min<int64_t>(ceil_div(total, kThreads), 148 * 16));
+    cast_f32_bf16_kernel<<<grid, kThreads, 0, cx.stream>>>(static_cast<const float*>(p), ld, static_cast<uint16_t*>(buf), ldo,
+                                                           rows, cols, ldo);
+    cx.st = check_launch("cast_f32_bf16_kernel");
+    s.ptr = buf; s.rows = rows; s.cols = cols; s.ld = ldo;
+    return s;
+}
+
+// bf16 scratch matrix (rows x cols) from the workspace.
+Stored scratch_bf16(Ctx& cx, int64_t rows, int64_t cols) {
+    Stored s;
+    if (cx.st != ECOSPA_OK) return s;
+    const int64_t ld = round_up(cols, 8);
+    void* buf = cx.arena.take(static_cast<size_t>(rows) * ld * 2);
+    if (!buf) {
+        cx.st = ECOSPA_ERR_WORKSPACE;
+        return s;
+    }
+    s.ptr = buf; s.rows = rows; s.cols = cols; s.ld = ld;
+    return s;
+}
+
+// out[c] = sum_r M[r][c] for a bf16 matrix; out has the model dtype.
+void colsum(Ctx& cx, const Stored& M, void* out) {
+    if (cx.st != ECOSPA_OK || !out) return;
+    const int chunks = static_cast<int>(ceil_div(M.rows, kSumRows));
+    float* partial = static_cast<float*>(cx.arena.take(static_cast<size_t>(chunks) * M.cols * 4));
+    if (!partial) {
+        cx.st = ECOSPA_ERR_WORKSPACE;
+        return;
+    }
+    dim3 grid(static_cast<unsigned>(ceil_div(M.cols, kThreads)), chunks);
+    colsum_partial_kernel<<<grid, kThreads, 0, cx.stream>>>(static_cast<const uint16_t*>(M.ptr), M.ld, M.rows, M.cols, partial);
+    if ((cx.st = check_launch("colsum_partial_kernel")) != ECOSPA_OK) return;
+    colsum_final_kernel<<<grid.x, kThreads, 0, cx.stream>>>(partial, chunks, M.cols, out, cx.dtype == ECOSPA_F32);
+    cx.st = check_launch("colsum_final_kernel");
+}
+
+// Compacted weight with n real shared indices, as stored: shared-cols d_m x n, or shared-rows n x d_m.
+ecospa_status_t check_weight(const ecospa_mat_t* w, int64_t d_m, int64_t n, int want_layout, int dtype) {
+    if (!w || !w->ptr) return ECOSPA_ERR_INVALID;
+    if (w->dtype != dtype || w->other_dim != d_m) return ECOSPA_ERR_INVALID;
+    if (w->layout != want_layout) return ECOSPA_ERR_UNSUPPORTED;
+    if (w->ld < (want_layout == ECOSPA_SHARED_COLS ? n : d_m)) return ECOSPA_ERR_INVALID;
+    return ECOSPA_OK;
+}
+Stored weight_bf16(Ctx& cx, const ecospa_mat_t* w, int64_t d_m, int64_t n) {
+    if (w->layout == ECOSPA_SHARED_COLS) return as_bf16(cx, w->ptr, d_m, n, w->ld);
+    return as_bf16(cx, w->ptr, n, d_m, w->ld);
+}
+
+ecospa_status_t begin(Ctx& cx, int dtype, void* workspace, size_t workspace_bytes, void* stream, int64_t T, int64_t d_m, int64_t n) {
+    if (dtype != ECOSPA_F32 && dtype != ECOSPA_BF16) return ECOSPA_ERR_INVALID;
+    if (T < 1 || d_m < 1 || n < 1) return ECOSPA_ERR_INVALID;
+    if (workspace && !aligned16(workspace)) return ECOSPA_ERR_ALIGNMENT;
+    cx.stream = static_cast<cudaStream_t>(stream);
+    cx.arena.base = static_cast<char*>(workspace);
+    cx.arena.size = workspace ? workspace_bytes : 0;
+    cx.dtype = dtype;
+    return ECOSPA_OK;
+}
+
+size_t staged(int dtype, int64_t rows, int64_t cols) {  // bytes as_bf16 takes from the arena
+    return dtype == ECOSPA_F32 ? arena_need(static_cast<size_t>(rows) * round_up(cols, 8) * 2) : 0;
+}
+size_t scratch(int64_t rows, int64_t cols) { return arena_need(static_cast<size_t>(rows) * round_up(cols, 8) * 2); }
+size_t colsum_need(int64_t rows, int64_t cols) { return arena_need(static_cast<size_t>(ceil_div(rows, kSumRows)) * cols * 4); }
+
+// C (T x n) = X (stored T x d_m, K-major) * W (shared-cols weight d_m x n, consumed MN-major) [+ bias]
+GemmOp proj_op(const Stored& X, const Stored& W, int64_t T, int64_t d_m, int64_t n, const void* bias, void* out, int64_t ld_out, int dtype) {
+    GemmOp op;
+    op.M = T; op.N = n; op.n_kseg = 1;
+    op.seg[0].a = X; op.seg[0].a_mn = false;
+    op.seg[0].b[0] = W; op.seg[0].b_mn = true;
+    op.seg[0].K = d_m;
+    op.epi = EPI_STORE;
+    op.C = out; op.ldc = ld_out; op.out_f32 = dtype == ECOSPA_F32;
+    op.bias = bias; op.bias_f32 = dtype == ECOSPA_F32;
+    return op;
+}
+// dW (rows_out x cols_out) = Xs^T dYs  with Xs stored T x rows_out and dYs stored T x cols_out
+GemmOp wgrad_op(const Stored& Xs, const Stored& dYs, int64_t rows_out, int64_t cols_out, int64_t T, void* out, int64_t ld_out, int dtype) {
+    GemmOp op;
+    op.M = rows_out; op.N = cols_out; op.n_kseg = 1;
+    op.seg[0].a = Xs; op.seg[0].a_mn = true;
+    op.seg[0].b[0] = dYs; op.seg[0].b_mn = true;
+    op.seg[0].K = T;
+    op.epi = EPI_STORE;
+    op.C = out; op.ldc = ld_out; op.out_f32 = dtype == ECOSPA_F32;
+    return op;
+}
+
+}  // namespace
+
+}  // namespace ecospa
+
+using namespace ecospa;
+
+extern "C" size_t ecospa_proj_workspace_bytes(int64_t T, int64_t d_m, int64_t n, int32_t dtype) {
+    // worst case over the qk / vo calls: staged X, Ctx, upstream grads, weights, and the column-sum partials
+    return staged(dtype, T, d_m) * 2 + staged(dtype, d_m, n) * 2 + staged(dtype, n, d_m) + staged(dtype, T, n) * 3 +
+           colsum_need(T, n) * 2 + colsum_need(T, d_m) + 1024;
+}
+
+extern "C" size_t ecospa_ffn_workspace_bytes(int64_t T, int64_t d_m, int64_t k, int32_t act, int32_t dtype) {
+    const int nw = act == ECOSPA_ACT_SWIGLU ? 2 : 1;
+    return staged(dtype, T, d_m) * 2 + staged(dtype, d_m, k) * nw + staged(dtype, k, d_m) + scratch(T, k) * nw +
+           colsum_need(T, k) + colsum_need(T, d_m) + 1024;
+}
+
+extern "C" ecospa_status_t ecospa_coupled_qk_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m,
+                                                 const ecospa_mat_t* wq_c, const ecospa_mat_t* wk_c, int64_t n,
+                                                 const void* bq_c, const void* bk_c, void* Qc, void* Kc, int64_t ld_out,
+                                                 void* workspace, size_t workspace_bytes, void* stream) {
+    if (!wq_c || !Qc) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if (wk_c && (st = check_weight(wk_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if (wk_c && !Kc) return ECOSPA_ERR_INVALID;
+    const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
+    GemmOp ops[2];
+    int n_ops = 0;
+    ops[n_ops++] = proj_op(Xs, weight_bf16(cx, wq_c, d_m, n), T, d_m, n, bq_c, Qc, ld_out, cx.dtype);
+    if (wk_c) ops[n_ops++] = proj_op(Xs, weight_bf16(cx, wk_c, d_m, n), T, d_m, n, bk_c, Kc, ld_out, cx.dtype);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    return launch_grouped_gemm(ops, n_ops, cx.stream);
+}
+
+extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int64_t T, int64_t d_m,
+                                                 const ecospa_mat_t* wq_c, const ecospa_mat_t* wk_c, int64_t n,
+                                                 const void* dQc, const void* dKc, int64_t ld_dqk, void* dX, int64_t ld_dx,
+                                                 int32_t accumulate_dX, void* dWq_c, void* dWk_c, int64_t ld_dw,
+                                                 void* dbq_c, void* dbk_c, void* workspace, size_t workspace_bytes,
+                                                 void* stream) {
+    if (!wq_c || !dQc || !dX || !dWq_c) return ECOSPA_ERR_INVALID;
+    if (wk_c && (!dKc || !dWk_c)) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if (wk_c && (st = check_weight(wk_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    const bool f32 = cx.dtype == ECOSPA_F32;
+    const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
+    const Stored dQs = as_bf16(cx, dQc, T, n, ld_dqk);
+    const Stored Wq = weight_bf16(cx, wq_c, d_m, n);
+    Stored dKs, Wk;
+    if (wk_c) {
+        dKs = as_bf16(cx, dKc, T, n, ld_dqk);
+        Wk = weight_bf16(cx, wk_c, d_m, n);
+    }
+    if (cx.st != ECOSPA_OK) return cx.st;
+    GemmOp ops[3];
+    int n_ops = 0;
+    ops[n_ops++] = wgrad_op(Xs, dQs, d_m, n, T, dWq_c, ld_dw, cx.dtype);
+    if (wk_c) ops[n_ops++] = wgrad_op(Xs, dKs, d_m, n, T, dWk_c, ld_dw, cx.dtype);
+    // dX = dQ W_Q^T (+ dK W_K^T): weights stored d_m x n are K-major B operands here
+    GemmOp& dx = ops[n_ops++];
+    dx.M = T; dx.N = d_m; dx.n_kseg = wk_c ? 2 : 1;
+    dx.seg[0].a = dQs; dx.seg[0].b[0] = Wq; dx.seg[0].K = n;
+    if (wk_c) {
+        dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].K = n;
+    }
+    dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
+    if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
+    colsum(cx, dQs, dbq_c);
+    if (wk_c) colsum(cx, dKs, dbk_c);
+    return cx.st;
+}
+
+extern "C" ecospa_status_t ecospa_coupled_vo_fwd_v(const void* X, int64_t ldx, int64_t T, int64_t d_m,
+                                                   const ecospa_mat_t* wv_c, int64_t n, const void* bv_c, void* Vc,
+                                                   int64_t ld_out, void* workspace, size_t workspace_bytes, void* stream) {
+    return ecospa_coupled_qk_fwd(X, ldx, T, d_m, wv_c, nullptr, n, bv_c, nullptr, Vc, nullptr, ld_out, workspace,
+                                 workspace_bytes, stream);
+}
+
+extern "C" ecospa_status_t ecospa_coupled_vo_fwd_o(const void* Ctxm, int64_t ld_ctx, int64_t T, int64_t d_m,
+                                                   const ecospa_mat_t* wo_c, int64_t n, const void* bo, void* Out,
+                                                   int64_t ld_out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!wo_c || !Out) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, wo_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(wo_c, d_m, n, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    GemmOp op;
+    op.M = T; op.N = d_m; op.n_kseg = 1;
+    op.seg[0].a = as_bf16(cx, Ctxm, T, n, ld_ctx);
+    op.seg[0].b[0] = weight_bf16(cx, wo_c, d_m, n);   // stored n x d_m = [K][N]
+    op.seg[0].b_mn = true;
+    op.seg[0].K = n;
+    op.epi = EPI_STORE; op.C = Out; op.ldc = ld_out; op.out_f32 = cx.dtype == ECOSPA_F32;
+    op.bias = bo; op.bias_f32 = cx.dtype == ECOSPA_F32;
+    if (cx.st != ECOSPA_OK) return cx.st;
+    return launch_grouped_gemm(&op, 1, cx.stream);
+}
+
+extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, const void* Ctxm, int64_t ld_ctx, int64_t T,
+                                                 int64_t d_m, const ecospa_mat_t* wv_c, const ecospa_mat_t* wo_c, int64_t n,
+                                                 const void* dVc, int64_t ld_dv, const void* dOut, int64_t ld_dout,
+                                                 void* dX, int64_t ld_dx, int32_t accumulate_dX, void* dCtx, int64_t ld_dctx,
+                                                 void* dWv_c, int64_t ld_dwv, void* dWo_c, int64_t ld_dwo, void* dbv_c,
+                                                 void* dbo, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!wv_c || !wo_c || !dVc || !dOut || !dX || !dCtx || !dWv_c || !dWo_c) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, wv_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(wv_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wo_c, d_m, n, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    const bool f32 = cx.dtype == ECOSPA_F32;
+    const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
+    const Stored Cs = as_bf16(cx, Ctxm, T, n, ld_ctx);
+    const Stored dVs = as_bf16(cx, dVc, T, n, ld_dv);
+    const Stored dOs = as_bf16(cx, dOut, T, d_m, ld_dout);
+    const Stored Wv = weight_bf16(cx, wv_c, d_m, n);
+    const Stored Wo = weight_bf16(cx, wo_c, d_m, n);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    GemmOp ops[4];
+    // dW_O (n x d_m) = Ctx^T dOut ; dW_V (d_m x n) = X^T dV
+    ops[0] = wgrad_op(Cs, dOs, n, d_m, T, dWo_c, ld_dwo, cx.dtype);
+    ops[1] = wgrad_op(Xs, dVs, d_m, n, T, dWv_c, ld_dwv, cx.dtype);
+    // dCtx (T x n) = dOut W_O^T : W_O stored n x d_m = [N][K]
+    GemmOp& dc = ops[2];
+    dc.M = T; dc.N = n; dc.n_kseg = 1;
+    dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].K = d_m;
+    dc.epi = EPI_STORE; dc.C = dCtx; dc.ldc = ld_dctx; dc.out_f32 = f32;
+    // dX (T x d_m) = dV W_V^T : W_V stored d_m x n = [N][K]
+    GemmOp& dx = ops[3];
+    dx.M = T; dx.N = d_m; dx.n_kseg = 1;
+    dx.seg[0].a = dVs; dx.seg[0].b[0] = Wv; dx.seg[0].K = n;
+    dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
+    if ((st = launch_grouped_gemm(ops, 4, cx.stream)) != ECOSPA_OK) return st;
+    colsum(cx, dVs, dbv_c);
+    colsum(cx, dOs, dbo);
+    return cx.st;
+}
+
+extern "C" ecospa_status_t ecospa_coupled_ffn_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, int32_t act,
+                                                  const ecospa_mat_t* w1_c, const ecospa_mat_t* w1b_c,
+                                                  const ecospa_mat_t* w2_c, int64_t k, const void* b1_c, const void* b2,
+                                                  void* Y, int64_t ld_y, void* H, void* Hb, void* A, int64_t ld_h,
+                                                  void* workspace, size_t workspace_bytes, void* stream) {
+    if (!w1_c || !w2_c || !Y || !H || !A) return ECOSPA_ERR_INVALID;
+    if (act != ECOSPA_ACT_GELU_ERF && act != ECOSPA_ACT_GELU_TANH && act != ECOSPA_ACT_SWIGLU) return ECOSPA_ERR_INVALID;
+    const bool sw = act == ECOSPA_ACT_SWIGLU;
+    if (sw && (!w1b_c || !Hb)) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, w1_c->dtype, workspace, workspace_bytes, stream, T, d_m, k);
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(w1_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if (sw && (st = check_weight(w1b_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(w2_c, d_m, k, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    if (ld_h < k || (ld_h * 2) % 16) return ld_h < k ? ECOSPA_ERR_INVALID : ECOSPA_ERR_ALIGNMENT;
+    const bool f32 = cx.dtype == ECOSPA_F32;
+    const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
+    GemmOp up;   // H = X W_1 (+ b_1), A = act(H): activation fused into the W_1 epilogue
+    up.M = T; up.N = k; up.n_kseg = 1;
+    up.seg[0].a = Xs;
+    up.seg[0].b[0] = weight_bf16(cx, w1_c, d_m, k);
+    if (sw) up.seg[0].b[1] = weight_bf16(cx, w1b_c, d_m, k);
+    up.seg[0].b_mn = true;
+    up.seg[0].K = d_m;
+    up.epi = sw ? EPI_SWIGLU : (act == ECOSPA_ACT_GELU_ERF ? EPI_GELU_ERF : EPI_GELU_TANH);
+    up.C = H; up.C2 = sw ? Hb : A; up.C3 = sw ? A : nullptr; up.ldc = ld_h;
+    up.bias = sw ? nullptr : b1_c; up.bias_f32 = f32;
+    GemmOp down;  // Y = A W_2 (+ b_2)
+    down.M = T; down.N = d_m; down.n_kseg = 1;
+    down.seg[0].a.ptr = A; down.seg[0].a.rows = T; down.seg[0].a.cols = k; down.seg[0].a.ld = ld_h;
+    down.seg[0].b[0] = weight_bf16(cx, w2_c, d_m, k);  // stored k x d_m = [K][N]
+    down.seg[0].b_mn = true;
+    down.seg[0].K = k;
+    down.epi = EPI_STORE; down.C = Y; down.ldc = ld_y; down.out_f32 = f32;
+    down.bias = b2; down.bias_f32 = f32;
+    if (cx.st != ECOSPA_OK) return cx.st;
+    if ((st = launch_grouped_gemm(&up, 1, cx.stream)) != ECOSPA_OK) return st;
+    return launch_grouped_gemm(&down, 1, cx.stream);
+}
+
+extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, int32_t act,
+                                                  const ecospa_mat_t* w1_c, const ecospa_mat_t* w1b_c,
+                                                  const ecospa_mat_t* w2_c, int64_t k, const void* H, const void* Hb,
+                                                  const void* A, int64_t ld_h, const void* dY, int64_t ld_dy, void* dX,
+                                                  int64_t ld_dx, void* dW1_c, void* dW1b_c, int64_t ld_dw1, void* dW2_c,
+                                                  int64_t ld_dw2, void* db1_c, void* db2, void* workspace,
+                                                  size_t workspace_bytes, void* stream) {
+    if (!w1_c || !w2_c || !H || !A || !dY || !dX || !dW1_c || !dW2_c) return ECOSPA_ERR_INVALID;
+    if (act != ECOSPA_ACT_GELU_ERF && act != ECOSPA_ACT_GELU_TANH && act != ECOSPA_ACT_SWIGLU) return ECOSPA_ERR_INVALID;
+    const bool sw = act == ECOSPA_ACT_SWIGLU;
+    if (sw && (!w1b_c || !Hb || !dW1b_c)) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, w1_c->dtype, workspace, workspace_bytes, stream, T, d_m, k);
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(w1_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if (sw && (st = check_weight(w1b_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(w2_c, d_m, k, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    if (ld_h < k || (ld_h * 2) % 16) return ld_h < k ? ECOSPA_ERR_INVALID : ECOSPA_ERR_ALIGNMENT;
+    const bool f32 = cx.dtype == ECOSPA_F32;
+    const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
+    const Stored dYs = as_bf16(cx, dY, T, d_m, ld_dy);
+    const Stored W1 = weight_bf16(cx, w1_c, d_m, k);
+    Stored W1b;
+    if (sw) W1b = weight_bf16(cx, w1b_c, d_m, k);
+    const Stored W2 = weight_bf16(cx, w2_c, d_m, k);
+    const Stored dH = scratch_bf16(cx, T, k);
+    Stored dHb;
+    if (sw) dHb = scratch_bf16(cx, T, k);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    Stored As;
+    As.ptr = A; As.rows = T; As.cols = k; As.ld = ld_h;
+
+    // dH = (dY W_2^T) (.) act'(H): W_2 stored k x d_m = [N][K]; derivative fused into the epilogue
+    GemmOp da;
+    da.M = T; da.N = k; da.n_kseg = 1;
+    da.seg[0].a = dYs; da.seg[0].b[0] = W2; da.seg[0].K = d_m;
+    da.epi = sw ? EPI_DSWIGLU : (act == ECOSPA_ACT_GELU_ERF ? EPI_DGELU_ERF : EPI_DGELU_TANH);
+    da.C = const_cast<void*>(dH.ptr); da.C2 = sw ? const_cast<void*>(dHb.ptr) : nullptr; da.ldc = dH.ld;
+    da.H = H; da.Hb = Hb; da.ldh = ld_h;
+    if ((st = launch_grouped_gemm(&da, 1, cx.stream)) != ECOSPA_OK) return st;
+
+    GemmOp ops[4];
+    int n_ops = 0;
+    ops[n_ops++] = wgrad_op(As, dYs, k, d_m, T, dW2_c, ld_dw2, cx.dtype);          // dW_2 (k x d_m) = A^T dY
+    ops[n_ops++] = wgrad_op(Xs, dH, d_m, k, T, dW1_c, ld_dw1, cx.dtype);           // dW_1 (d_m x k) = X^T dH
+    if (sw) ops[n_ops++] = wgrad_op(Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, cx.dtype); // dW_up = X^T dH_up
+    GemmOp& dx = ops[n_ops++];                                                    // dX = dH W_1^T (+ dH_up W_up^T)
+    dx.M = T; dx.N = d_m; dx.n_kseg = sw ? 2 : 1;
+    dx.seg[0].a = dH; dx.seg[0].b[0] = W1; dx.seg[0].K = k;
+    if (sw) {
+        dx.seg[1].a = dHb; dx.seg[1].b[0] = W1b; dx.seg[1].K = k;
+    }
+    dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32;
+    if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
+    if (!sw) colsum(cx, dH, db1_c);
+    colsum(cx, dYs, db2);
+    return cx.st;
+}

@@ -1,0 +1,70 @@
+"""Buffer plumbing for the compacted-pair forward/backward calls (allocation and argument order only)."""
+from __future__ import annotations
+
+from typing import Dict
+
+import torch
+
+from . import binding as B
+from .block import pad8
+
+
+def ffn_buffers(T: int, d_m: int, k: int, act: int, dtype: torch.dtype, device) -> Dict[str, torch.Tensor]:
+    """Outputs and saved tensors of one FFN forward+backward (H, Hb, A are always bf16)."""
+    kp = pad8(k, 2)
+    kpw = pad8(k, 2 if dtype == torch.bfloat16 else 4)
+    sw = act == B.ACT_SWIGLU
+    d = {
+        "Y": torch.empty((T, d_m), dtype=dtype, device=device),
+        "H": torch.empty((T, kp), dtype=torch.bfloat16, device=device),
+        "A": torch.empty((T, kp), dtype=torch.bfloat16, device=device),
+        "dX": torch.empty((T, d_m), dtype=dtype, device=device),
+        "dW1": torch.zeros((d_m, kpw), dtype=dtype, device=device),
+        "dW2": torch.empty((k, d_m), dtype=dtype, device=device),
+        "db2": torch.empty((d_m,), dtype=dtype, device=device),
+    }
+    if sw:
+        d["Hb"] = torch.empty((T, kp), dtype=torch.bfloat16, device=device)
+        d["dW1b"] = torch.zeros((d_m, kpw), dtype=dtype, device=device)
+    else:
+        d["db1"] = torch.empty((k,), dtype=dtype, device=device)
+    code = B.F32 if dtype == torch.float32 else B.BF16
+    d["ws"] = torch.empty(max(16, B.ecospa_ffn_workspace_bytes(T, d_m, k, act, code)), dtype=torch.uint8, device=device)
+    return d
+
+
+def ffn_fwd_bwd(X, dY, act: int, w1c, w2c, k: int, buf: Dict[str, torch.Tensor], w1bc=None, b1c=None, b2=None) -> None:
+    B.ecospa_coupled_ffn_fwd(X, act, w1c, w2c, k, buf["Y"], buf["H"], buf["A"], w1b_c=w1bc, Hb=buf.get("Hb"),
+                             b1_c=b1c, b2=b2, workspace=buf["ws"])
+    B.ecospa_coupled_ffn_bwd(X, act, w1c, w2c, k, buf["H"], buf["A"], dY, buf["dX"], buf["dW1"], buf["dW2"],
+                             w1b_c=w1bc, Hb=buf.get("Hb"), dW1b_c=buf.get("dW1b"), db1_c=buf.get("db1"),
+                             db2=buf["db2"], workspace=buf["ws"])
+
+
+def smoke_layer_check(wl, w1c, w1bc, w2c, k: int, dev) -> None:
+    """One tiny compacted SwiGLU FFN forward/backward on the GPU against the fp64 oracle."""
+    import numpy as np
+    from oracle import oracle as O
+    from . import workloads as WL
+
+    acts = WL.activations(wl, 0, kinds=["x", "dy"])
+    X, dY = acts["x"].to(dev), acts["dy"].to(dev)
+    T = X.shape[0]
+    buf = ffn_buffers(T, wl.d_m, k, B.ACT_SWIGLU, torch.bfloat16, dev)
+    ffn_fwd_bwd(X, dY, B.ACT_SWIGLU, w1c, w2c, k, buf, w1bc=w1bc)
+    B.ecospa_device_status()
+    ref_f = O.ffn_fwd(acts["x"], O.ACT_SWIGLU, w1c.cpu(), w2c.cpu(), O.SHARED_COLS, O.SHARED_ROWS, k, W1b=w1bc.cpu())
+    ref_b = O.ffn_bwd(acts["x"], O.ACT_SWIGLU, w1c.cpu(), w2c.cpu(), O.SHARED_COLS, O.SHARED_ROWS, k, acts["dy"],
+                      W1b=w1bc.cpu())
+
+    def rel(a, b):
+        return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
+
+    errs = {
+        "Y": rel(buf["Y"].double().cpu().numpy(), ref_f["Y"]),
+        "dX": rel(buf["dX"].double().cpu().numpy(), ref_b["dX"]),
+        "dW1": rel(buf["dW1"][:, :k].double().cpu().numpy(), ref_b["dW1"]),
+        "dW2": rel(buf["dW2"].double().cpu().numpy(), ref_b["dW2"].T),
+    }
+    bad = {n: e for n, e in errs.items() if not e <= 2e-2}
+    assert not bad, f"layer mismatch vs oracle: {bad}"
