@@ -1,0 +1,442 @@
+"""Benchmark of the coupled-sparsity hot path on a GPT-2-Medium-shaped model (or another workload).
+
+One step = one pass of the whole hot path over every layer of the model:
+  score (+ Fisher) of all coupled pairs -> aligned top-k -> compaction of weights, biases and
+  gradients -> forward and backward of every compacted QK / VO / FFN pair.
+
+    python bench.py --gpus 1 --steps 10 --warmup 3
+    python bench.py --impl reference            # the CPU oracle on a bounded sample of the same step
+
+Prints one JSON line (rank 0).  `value` is the tensor-core throughput of the step (algorithmic
+flops of the compacted-pair GEMMs / whole step time); the memory-bound phase is reported
+alongside as GB/s.  With N > 1 every rank runs an independent replica (the path has no exchange
+step); times are the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "compacted-pair fwd/bwd TFLOP/s over the whole coupled-sparsity step (score+select+compact GB/s alongside)"
+
+
+# ---------------------------------------------------------------------------------------------
+# workload accounting (algorithmic bytes and flops; see the design doc for the derivation)
+# ---------------------------------------------------------------------------------------------
+
+def step_flops(wl, n_attn: int, k_ffn: int) -> float:
+    """2*M*N*K of every compacted-pair product, forward (x1) and backward (x2), all layers."""
+    T, d = wl.tokens, wl.d_m
+    ffn_mats = 3 if wl.ffn == "swiglu" else 2
+    fwd = 2.0 * T * d * (2 * n_attn) + 2.0 * T * d * (2 * n_attn) + 2.0 * T * d * k_ffn * ffn_mats
+    return 3.0 * fwd * wl.n_layers
+
+
+def sparsify_bytes(wl, rho: float, with_grads: bool = True) -> float:
+    """Weights (and gradients) read once for the scores; compaction reads a shared-cols tensor in
+    full and a shared-rows tensor at the kept fraction, and writes the kept fraction of both."""
+    D = wl.n_heads * wl.d_h
+    e = wl.elem_bytes
+    cols = (3 * wl.d_m * D + (2 if wl.ffn == "swiglu" else 1) * wl.d_m * wl.d_ffn) * e * wl.n_layers
+    rows = (wl.d_m * D + wl.d_m * wl.d_ffn) * e * wl.n_layers
+    mult = 2 if with_grads else 1
+    score = (cols + rows) * mult
+    compact = (cols * (1 + rho) + rows * 2 * rho) * mult
+    return float(score + compact)
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ---------------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons of one GPU while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([f.strip() for f in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 6:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------------------------
+# the GPU step
+# ---------------------------------------------------------------------------------------------
+
+class Model:
+    """Device-resident synthetic model plus every buffer a step writes (allocated once)."""
+
+    def __init__(self, wl, sparsity: float, device, n_act_sets: int = 4):
+        import torch
+        from paper_2511_11641_b200 import binding as B, block as BL, workloads as WL
+        self.wl, self.dev, self.B, self.BL = wl, device, B, BL
+        self.torch = torch
+        self.w, self.g, self.pairs = [], [], []
+        for l in range(wl.n_layers):
+            w = WL.layer_weights(wl, l, device=device)
+            g = WL.layer_grads(wl, l, device=device)
+            self.w.append(w); self.g.append(g)
+            self.pairs += BL.block_pairs(w, wl.n_heads, wl.d_h, wl.d_ffn, g)
+        plan = WL.kept_plan(wl, sparsity)
+        self.n_attn, self.k_ffn = sum(plan["qk"]), plan["ffn"][0]
+        self.k_per_seg = (plan["qk"] + plan["vo"] + plan["ffn"]) * wl.n_layers
+        self.n_seg = [wl.n_heads, wl.n_heads, 1] * wl.n_layers
+        self.seg_len = [wl.d_h, wl.d_h, wl.d_ffn] * wl.n_layers
+        D_layer = 2 * wl.n_heads * wl.d_h + wl.d_ffn
+        f32, i32 = torch.float32, torch.int32
+        self.ups = torch.empty(D_layer * wl.n_layers, dtype=f32, device=device)
+        self.fis = torch.empty((2 * wl.n_heads + 1) * wl.n_layers, dtype=f32, device=device)
+        self.kept = torch.empty(sum(self.k_per_seg), dtype=i32, device=device)
+        self.score_ws = torch.empty(B.ecospa_score_workspace_bytes(self.pairs), dtype=torch.uint8, device=device)
+        # compaction jobs: weights, biases and gradients of every pair group
+        self.c, self.jobs = [], []
+        off = 0
+        D_attn = wl.n_heads * wl.d_h
+        groups = [(["wq", "wk", "bq", "bk"], ["gq", "gk"], self.n_attn, D_attn),
+                  (["wv", "wo", "bv"], ["gv", "go"], self.n_attn, D_attn),
+                  (["w1", "w1b", "w2", "b1"], ["g1", "g1b", "g2"], self.k_ffn, wl.d_ffn)]
+        layout = {"wq": 0, "wk": 0, "wv": 0, "wo": 1, "w1": 0, "w1b": 0, "w2": 1, "bq": 0, "bk": 0, "bv": 0, "b1": 0,
+                  "gq": 0, "gk": 0, "gv": 0, "go": 1, "g1": 0, "g1b": 0, "g2": 1}
+        for l in range(wl.n_layers):
+            c = {}
+            for wn, gn, nk, D in groups:
+                kd = self.kept[off:off + nk]
+                for nm in wn + gn:
+                    src = self.w[l].get(nm) if nm in self.w[l] else self.g[l].get(nm)
+                    if src is None:
+                        continue
+                    o = BL.alloc_compacted(src, layout[nm], nk)
+                    c[nm] = o
+                    self.jobs.append(B.gather(src, o, layout[nm], kd, nk, D))
+                off += nk
+            self.c.append(c)
+        # activations and upstream gradients: a small pool of distinct sets cycled over the layers
+        T, d, n, k = wl.tokens, wl.d_m, self.n_attn, self.k_ffn
+        npad = BL.pad8(n)
+        dt = wl.torch_dtype
+        self.acts = []
+        for s in range(n_act_sets):
+            self.acts.append(WL.activations(wl, s, kinds=["x", "dy", "dout", "dq", "dk", "dv", "ctx"],
+                                            widths={"dq": npad, "dk": npad, "dv": npad, "ctx": npad}, device=device))
+        e = lambda *shape: torch.empty(shape, dtype=dt, device=device)
+        self.o = {"Q": e(T, npad), "K": e(T, npad), "V": e(T, npad), "Out": e(T, d), "dX": e(T, d), "dCtx": e(T, npad),
+                  "dWq": e(d, npad), "dWk": e(d, npad), "dWv": e(d, npad), "dWo": e(n, d),
+                  "dbq": e(n), "dbk": e(n), "dbv": e(n), "dbo": e(d)}
+        from paper_2511_11641_b200 import layers as L
+        self.L = L
+        self.act = B.ACT_SWIGLU if wl.ffn == "swiglu" else B.ACT_GELU_ERF
+        self.ffn = L.ffn_buffers(T, d, k, self.act, dt, device)
+        self.proj_ws = torch.empty(B.ecospa_proj_workspace_bytes(T, d, n, B.BF16 if dt == torch.bfloat16 else B.F32) + 16,
+                                   dtype=torch.uint8, device=device)
+
+    def sparsify(self):
+        B = self.B
+        B.ecospa_score_pairs(self.pairs, float(self.wl.tokens), self.ups, None, self.fis, self.score_ws)
+        B.ecospa_select_aligned_topk(self.ups, self.n_seg, self.seg_len, self.k_per_seg, self.kept)
+        B.ecospa_compact_tensors(self.jobs)
+
+    def layers(self):
+        B, o, n, k = self.B, self.o, self.n_attn, self.k_ffn
+        bias = self.wl.bias
+        for l in range(self.wl.n_layers):
+            c, a = self.c[l], self.acts[l % len(self.acts)]
+            B.ecospa_coupled_qk_fwd(a["x"], c["wq"], c["wk"], n, o["Q"], o["K"], bq_c=c.get("bq"), bk_c=c.get("bk"),
+                                    workspace=self.proj_ws)
+            B.ecospa_coupled_vo_fwd_v(a["x"], c["wv"], n, o["V"], bv_c=c.get("bv"), workspace=self.proj_ws)
+            B.ecospa_coupled_vo_fwd_o(a["ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws)
+            self.L.ffn_fwd_bwd(a["x"], a["dy"], self.act, c["w1"], c["w2"], k, self.ffn, w1bc=c.get("w1b"),
+                               b1c=c.get("b1"), b2=self.w[l].get("b2"))
+            B.ecospa_coupled_vo_bwd(a["x"], a["ctx"], c["wv"], c["wo"], n, a["dv"], a["dout"], o["dX"], o["dCtx"],
+                                    o["dWv"], o["dWo"], o["dbv"] if bias else None, o["dbo"] if bias else None,
+                                    workspace=self.proj_ws)
+            B.ecospa_coupled_qk_bwd(a["x"], c["wq"], c["wk"], n, a["dq"], a["dk"], o["dX"], o["dWq"], o["dWk"],
+                                    o["dbq"] if bias else None, o["dbk"] if bias else None, accumulate_dX=True,
+                                    workspace=self.proj_ws)
+
+    def host_copies(self):
+        """Pinned host mirrors of every input of a step (weights, gradients, activations)."""
+        torch = self.torch
+        pairs = []
+        for d in self.w + self.g + self.acts:
+            for t in d.values():
+                h = torch.empty(t.shape, dtype=t.dtype, pin_memory=True)
+                h.copy_(t)
+                pairs.append((h, t))
+        return pairs
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2511_11641_b200 import binding as B, workloads as WL
+    import __graft_entry__ as ge
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if rank == 0:
+        ge.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    dev = torch.device("cuda", local)
+    wl = WL.WORKLOADS[args.workload]
+    m = Model(wl, args.sparsity, dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        m.sparsify(); m.layers()
+    B.ecospa_device_status()
+    # ---- device-resident timing
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = B.ecospa_launch_count()
+    marks = []
+    barrier()
+    t_all0, t_all1 = ev(), ev()
+    t_all0.record()
+    for _ in range(args.steps):
+        e0, e1, e2 = ev(), ev(), ev()
+        e0.record(); m.sparsify(); e1.record(); m.layers(); e2.record()
+        marks.append((e0, e1, e2))
+    t_all1.record()
+    barrier()
+    launches = (B.ecospa_launch_count() - launches0) // args.steps
+    clocks = sampler.stop() if rank == 0 else None
+    B.ecospa_device_status()
+    ms_total = t_all0.elapsed_time(t_all1)
+    ms_sp = sum(a.elapsed_time(b) for a, b, _ in marks) / args.steps
+    ms_gemm = sum(b.elapsed_time(c) for _, b, c in marks) / args.steps
+    ms_step = ms_total / args.steps
+
+    # ---- end to end: inputs start in pinned host memory, results are read back
+    host = m.host_copies()
+    h2d = sum(h.numel() * h.element_size() for h, _ in host)
+    res_host = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (m.kept, m.fis, m.ups)]
+    chk_host = torch.empty(1, dtype=torch.float32, pin_memory=True)
+    d2h = sum(t.numel() * t.element_size() for t in res_host) + 4
+
+    def e2e_step():
+        for h, d in host:
+            d.copy_(h, non_blocking=True)
+        m.sparsify(); m.layers()
+        for h, d in zip(res_host, (m.kept, m.fis, m.ups)):
+            h.copy_(d, non_blocking=True)
+        chk_host.copy_(m.o["dX"][0, :1].float(), non_blocking=True)
+
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_step()
+    barrier()
+    e0, e1 = ev(), ev()
+    e0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    ms_e2e = e0.elapsed_time(e1) / e2e_steps
+
+    if world > 1:
+        t = torch.tensor([ms_step, ms_sp, ms_gemm, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, ms_sp, ms_gemm, ms_e2e = t.tolist()
+
+    flops = step_flops(wl, m.n_attn, m.k_ffn)
+    sbytes = sparsify_bytes(wl, 1.0 - args.sparsity)
+    peaks = measured_peaks()
+    n_gemm_launches = wl.n_layers * 9
+    out = {
+        "metric": METRIC, "value": world * flops / ms_step / 1e9, "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic (seeded N(0,sigma) tensors)",
+        "config": {"workload": f"{wl.name}: {wl.n_layers} layers d_model={wl.d_m} heads={wl.n_heads}x{wl.d_h} "
+                               f"ffn={wl.d_ffn} {wl.ffn} T={wl.tokens} sparsity={args.sparsity}",
+                   "l2": "inputs larger than L2: 1.7 GB of weights/gradients per step, activations cycled over 4 sets",
+                   "replicas": world},
+        "phases": {
+            "sparsify": {"ms": ms_sp, "GB/s": sbytes / ms_sp / 1e6, "bytes": sbytes,
+                         "frac_of_measured_hbm": sbytes / ms_sp / 1e6 / peaks["hbm_gbs"],
+                         "frac_of_nominal_8TBs": sbytes / ms_sp / 1e6 / 8000.0},
+            "gemm": {"ms": ms_gemm, "TFLOP/s": flops / ms_gemm / 1e9, "flops": flops,
+                     "frac_of_nominal_2250": flops / ms_gemm / 1e9 / 2250.0},
+        },
+        "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": flops / ms_gemm / 1e9,
+                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                     "frac": flops / ms_gemm / 1e9 / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
+                     "launches_per_step": n_gemm_launches, "avg_launch_ms": ms_gemm / n_gemm_launches},
+        "e2e": {"value": world * flops / ms_e2e / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            out["cpu_baseline"] = cpu_sample(wl, args.sparsity)
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+# the CPU oracle on a bounded sample of the same step
+# ---------------------------------------------------------------------------------------------
+
+def cpu_sample(wl, sparsity: float, tokens: int = 256):
+    """Layer 0 of the workload through the oracle: score + Fisher + select + compact at full size,
+    then forward/backward of the compacted pairs on `tokens` token rows.  Returns the metric
+    (algorithmic flops / wall time) for that sample."""
+    import numpy as np
+    from oracle import oracle as O
+    from paper_2511_11641_b200 import workloads as WL
+    from paper_2511_11641_b200.block import pad8
+    w = WL.layer_weights(wl, 0)
+    g = WL.layer_grads(wl, 0)
+    plan = WL.kept_plan(wl, sparsity)
+    n_attn, k_ffn = sum(plan["qk"]), plan["ffn"][0]
+    acts = WL.activations(wl, 0, tokens=tokens, kinds=["x", "dy", "dout", "dq", "dk", "dv", "ctx"],
+                          widths={kk: n_attn for kk in ("dq", "dk", "dv", "ctx")})
+    sw = wl.ffn == "swiglu"
+    act = O.ACT_SWIGLU if sw else O.ACT_GELU_ERF
+    t0 = time.perf_counter()
+    groups = [("wq", "wk", None, "gq", "gk", None, 0, 0, wl.n_heads, wl.d_h, plan["qk"]),
+              ("wv", "wo", None, "gv", "go", None, 0, 1, wl.n_heads, wl.d_h, plan["vo"]),
+              ("w1", "w2", "w1b" if sw else None, "g1", "g2", "g1b" if sw else None, 0, 1, 1, wl.d_ffn, plan["ffn"])]
+    c = {}
+    for n1, n2, n1b, g1, g2, g1b, l1, l2, n_seg, seg_len, k in groups:
+        _, ups = O.score_pair(w[n1], w[n2], l1, l2, n_seg, seg_len, w1b=w.get(n1b) if n1b else None)
+        O.fisher_pair(g[g1], g[g2], l1, l2, n_seg, seg_len, float(wl.tokens), g1b=g.get(g1b) if g1b else None)
+        kept = O.select_topk(ups.astype(np.float32), n_seg, seg_len, k)
+        for nm, lay in ((n1, l1), (n2, l2), (n1b, l1), (g1, l1), (g2, l2), (g1b, l1)):
+            if nm:
+                src = w[nm] if nm in w else g[nm]
+                c[nm] = O.compact(src, lay, kept, ld_out=pad8(len(kept), wl.elem_bytes) if lay == 0 else None)
+    t1 = time.perf_counter()
+    x = acts["x"]
+    O.proj_fwd(x, c["wq"], 0, n_attn); O.proj_fwd(x, c["wk"], 0, n_attn); O.proj_fwd(x, c["wv"], 0, n_attn)
+    O.outproj_fwd(acts["ctx"], c["wo"], 1, n_attn, wl.d_m)
+    dX, _, _ = O.proj_bwd(x, c["wq"], 0, n_attn, acts["dq"])
+    O.proj_bwd(x, c["wk"], 0, n_attn, acts["dk"], dX=dX)
+    O.proj_bwd(x, c["wv"], 0, n_attn, acts["dv"])
+    O.outproj_bwd(acts["ctx"], c["wo"], 1, n_attn, wl.d_m, acts["dout"])
+    O.ffn_fwd(x, act, c["w1"], c["w2"], 0, 1, k_ffn, W1b=c.get("w1b"))
+    O.ffn_bwd(x, act, c["w1"], c["w2"], 0, 1, k_ffn, acts["dy"], W1b=c.get("w1b"))
+    t2 = time.perf_counter()
+    flops = step_flops(wl, n_attn, k_ffn) / wl.n_layers * tokens / wl.tokens
+    sbytes = sparsify_bytes(wl, 1.0 - sparsity) / wl.n_layers
+    return {"value": flops / (t2 - t0) / 1e12, "unit": "TFLOP/s", "cores": 1, "kind": "oracle",
+            "sample": f"layer 0 of {wl.name}: score+Fisher+select+compact at full size ({t1 - t0:.2f} s, "
+                      f"{sbytes / (t1 - t0) / 1e9:.3f} GB/s), then fwd+bwd of the compacted QK/VO/FFN pairs on "
+                      f"{tokens} of {wl.tokens} tokens ({t2 - t1:.2f} s)",
+            "seconds": t2 - t0, "gemm_tflops": flops / (t2 - t1) / 1e12, "sparsify_GB/s": sbytes / (t1 - t0) / 1e9}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import oracle as O
+    from paper_2511_11641_b200 import workloads as WL
+    O.build()
+    wl = WL.WORKLOADS[args.workload]
+    tokens = 32
+    steps, warm = max(1, min(args.steps, 5)), max(1, min(args.warmup, 1))
+    for _ in range(warm):
+        cpu_sample(wl, args.sparsity, tokens)
+    t0 = time.perf_counter()
+    last = None
+    for _ in range(steps):
+        last = cpu_sample(wl, args.sparsity, tokens)
+    dt = (time.perf_counter() - t0) / steps
+    plan = WL.kept_plan(wl, args.sparsity)
+    flops = step_flops(wl, sum(plan["qk"]), plan["ffn"][0]) / wl.n_layers * tokens / wl.tokens
+    v = flops / dt / 1e12
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": steps,
+        "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic (seeded N(0,sigma) tensors)",
+        "config": {"workload": f"{wl.name}: bounded sample of the step (layer 0, {tokens} of {wl.tokens} tokens), "
+                               f"sparsity={args.sparsity}"},
+        "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": 1, "kind": "oracle", "sample": last["sample"]},
+        "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="gpt2m")
+    ap.add_argument("--sparsity", type=float, default=0.5)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -85,6 +85,8 @@ typedef struct {
 const char* ecospa_status_string(ecospa_status_t s);
 /* Text of the last CUDA error this thread's calls ran into ("" if none). */
 const char* ecospa_last_cuda_error(void);
+/* Number of kernels this process has launched through the library so far (all threads). */
+uint64_t ecospa_launch_count(void);
 
 /* ---------------------------------------------------------------------------------------------
  * Step 1: coupled importance scores.   Eq. "l2norm" (per-index score upsilon) and

@@ -327,6 +327,12 @@ def ecospa_coupled_ffn_bwd(X, act: int, w1_c, w2_c, k: int, H, A, dY, dX, dW1_c,
            "ecospa_coupled_ffn_bwd")
 
 
+def ecospa_launch_count() -> int:
+    f = lib().ecospa_launch_count
+    f.restype = C.c_uint64
+    return int(f())
+
+
 def ecospa_device_status(stream=None) -> int:
     """Synchronises the stream; returns 0 or raises EcospaError(ERR_TIMEOUT) carrying the wait code."""
     code = C.c_int32(0)

@@ -1,4 +1,5 @@
 // Status strings and per-thread CUDA error record of libecospa.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 
@@ -7,6 +8,7 @@
 namespace ecospa {
 
 static thread_local char g_cuda_error[256] = "";
+static std::atomic<uint64_t> g_launches{0};
 
 void set_cuda_error(cudaError_t e, const char* where) {
     std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s (%s)", where, cudaGetErrorName(e), cudaGetErrorString(e));
@@ -14,6 +16,7 @@ void set_cuda_error(cudaError_t e, const char* where) {
 
 ecospa_status_t check_launch(const char* where) {
     const cudaError_t e = cudaGetLastError();
+    g_launches.fetch_add(1, std::memory_order_relaxed);
     if (e == cudaSuccess) return ECOSPA_OK;
     set_cuda_error(e, where);
     return ECOSPA_ERR_CUDA;
@@ -35,3 +38,5 @@ extern "C" const char* ecospa_status_string(ecospa_status_t s) {
 }
 
 extern "C" const char* ecospa_last_cuda_error(void) { return ecospa::g_cuda_error; }
+
+extern "C" uint64_t ecospa_launch_count(void) { return ecospa::g_launches.load(std::memory_order_relaxed); }
