@@ -114,6 +114,30 @@ ecospa_status_t ecospa_score_pairs(const ecospa_pair_t* pairs, int32_t n_pairs, 
                                    float* raw, float* fisher, void* workspace, size_t workspace_bytes,
                                    void* stream);
 
+/* Scores of ONE pair group without any workspace argument.  (The paper has no counterpart: this entry
+ * point exists only for the sake of callers that cannot allocate.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or unavailable -- a plug-in invoked
+ * from inside another framework's memory-managed region, a real-time loop that must not touch the
+ * allocator, a process whose memory pool is fixed up front -- and therefore has no way to obtain the
+ * scratch buffer that ecospa_score_pairs asks for.  Here the scratch is a fixed 4 MiB array inside the
+ * library's device image (ecospa_score_pair_static_max_bytes()); every GPU that loads the library holds
+ * it until the process exits.  The call itself allocates nothing on the device.
+ *
+ * Same inputs, outputs and results as ecospa_score_pairs with n_pairs == 1.  Differences:
+ *   - a pair group whose scratch need exceeds the array returns ECOSPA_ERR_UNSUPPORTED (the text from
+ *     ecospa_last_cuda_error says so) and launches nothing; ecospa_score_workspace_bytes(pair, 1) tells
+ *     the need in advance;
+ *   - the first call on each device looks up the array's device address (with that device current); make
+ *     that first call before starting any stream capture;
+ *   - every call on a device shares the one array and finds the previous call's data in it.  Nothing in
+ *     it has to start at zero (each value is written before it is read), but two calls that overlap on
+ *     the GPU (different streams, or several host threads) race on it: serialise them.
+ */
+size_t ecospa_score_pair_static_max_bytes(void);
+ecospa_status_t ecospa_score_pair_static(const ecospa_pair_t* pair, double n_samples, float* upsilon, float* raw,
+                                         float* fisher, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Step 2: aligned top-k per pair.   Definition 1 (coupled sparsification), App. A.2, applied to the
  * seg_len - k lowest-scored indices of each segment; Alg. 1 "remove smallest upsilon_i".

@@ -28,7 +28,7 @@ class EcospaError(RuntimeError):
         l = lib()
         msg = l.ecospa_status_string(status).decode()
         cuda = l.ecospa_last_cuda_error().decode()
-        super().__init__(f"{where}: {msg} (status {status})" + (f" [{cuda}]" if status == 4 and cuda else ""))
+        super().__init__(f"{where}: {msg} (status {status})" + (f" [{cuda}]" if status in (3, 4) and cuda else ""))
         self.status = status
 
 
@@ -136,6 +136,23 @@ def ecospa_score_pairs(pairs: Sequence[Pair], n_samples: float, upsilon: torch.T
                                   _ptr(fisher), _ptr(workspace), workspace.numel(), _stream(stream))
     if st != 0:
         raise EcospaError(st, "ecospa_score_pairs")
+
+
+def ecospa_score_pair_static_max_bytes() -> int:
+    f = lib().ecospa_score_pair_static_max_bytes
+    f.restype = C.c_size_t
+    return int(f())
+
+
+def ecospa_score_pair_static(p: Pair, n_samples: float, upsilon: torch.Tensor, raw: Optional[torch.Tensor] = None,
+                             fisher: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Scores of one pair group using the library's built-in scratch array; allocates nothing."""
+    f = lib().ecospa_score_pair_static
+    f.restype = C.c_int
+    f.argtypes = [C.c_void_p, C.c_double, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+    st = f(C.addressof(p), float(n_samples), _ptr(upsilon), _ptr(raw), _ptr(fisher), _stream(stream))
+    if st != 0:
+        raise EcospaError(st, "ecospa_score_pair_static")
 
 
 def ecospa_select_aligned_topk(upsilon: torch.Tensor, n_seg: Sequence[int], seg_len: Sequence[int],

@@ -10,6 +10,7 @@
 // Everything is summed in a fixed order, so results are bit-identical run to run.
 
 #include <algorithm>
+#include <mutex>
 #include <vector>
 
 #include "common.cuh"
@@ -491,4 +492,63 @@ extern "C" ecospa_status_t ecospa_score_pairs(const ecospa_pair_t* pairs, int32_
         if (st != ECOSPA_OK) return st;
     }
     return ECOSPA_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free variant: scores of ONE pair group with the scratch taken from a fixed array that
+// lives in the library's device image instead of from a caller-provided workspace.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kStaticScratchBytes = size_t(4) << 20;  // 4 MiB, held by every GPU that loads the library
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};
+
+// Device address of g_static_scratch on the current device (looked up once per device).
+ecospa_status_t static_scratch_ptr(void** out) {
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        set_cuda_error(e == cudaSuccess ? cudaErrorInvalidDevice : e, "ecospa_score_pair_static: cudaGetDevice");
+        return ECOSPA_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);   // the symbol itself is not a device pointer on the host
+        if (e != cudaSuccess || !p) {
+            set_cuda_error(e, "ecospa_score_pair_static: cudaGetSymbolAddress");
+            return ECOSPA_ERR_CUDA;
+        }
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return ECOSPA_OK;
+}
+
+}  // namespace
+
+extern "C" size_t ecospa_score_pair_static_max_bytes(void) { return kStaticScratchBytes; }
+
+extern "C" ecospa_status_t ecospa_score_pair_static(const ecospa_pair_t* pair, double n_samples, float* upsilon,
+                                                    float* raw, float* fisher, void* stream) {
+    if (!pair || !upsilon) return ECOSPA_ERR_INVALID;
+    const ecospa_status_t vs = validate_pair(*pair, fisher != nullptr);
+    if (vs != ECOSPA_OK) return vs;
+    std::vector<StatPlan> stats;
+    const size_t need = plan_stats(pair, 1, fisher != nullptr, &stats) * sizeof(float);
+    if (need > kStaticScratchBytes) {
+        set_cuda_error(cudaErrorMemoryAllocation,
+                       "ecospa_score_pair_static: this pair needs more scratch than the built-in 4 MiB array; "
+                       "use ecospa_score_pairs with a workspace");
+        return ECOSPA_ERR_UNSUPPORTED;
+    }
+    void* scratch = nullptr;
+    const ecospa_status_t st = static_scratch_ptr(&scratch);
+    if (st != ECOSPA_OK) return st;
+    return ecospa_score_pairs(pair, 1, n_samples, upsilon, raw, fisher, scratch, kStaticScratchBytes, stream);
 }
