@@ -220,6 +220,22 @@ class Model:
         return pairs
 
 
+def max_over_ranks(values, device=None):
+    """Element-wise maximum of per-rank timings over all ranks (identity without a process group)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return list(values)
+    t = torch.tensor(list(values), dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(world: int, units_per_rank: float, ms: float) -> float:
+    """Whole-job rate: every rank processed `units_per_rank` in `ms` (already the max over ranks)."""
+    return world * units_per_rank / ms
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -297,17 +313,14 @@ def run_gpu(args):
     barrier()
     ms_e2e = e0.elapsed_time(e1) / e2e_steps
 
-    if world > 1:
-        t = torch.tensor([ms_step, ms_sp, ms_gemm, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step, ms_sp, ms_gemm, ms_e2e = t.tolist()
+    ms_step, ms_sp, ms_gemm, ms_e2e = max_over_ranks([ms_step, ms_sp, ms_gemm, ms_e2e], dev)
 
     flops = step_flops(wl, m.n_attn, m.k_ffn)
     sbytes = sparsify_bytes(wl, 1.0 - args.sparsity)
     peaks = measured_peaks()
     n_gemm_launches = wl.n_layers * 9
     out = {
-        "metric": METRIC, "value": world * flops / ms_step / 1e9, "unit": "TFLOP/s", "n_gpus": world,
+        "metric": METRIC, "value": job_throughput(world, flops, ms_step) / 1e9, "unit": "TFLOP/s", "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic (seeded N(0,sigma) tensors)",
         "config": {"workload": f"{wl.name}: {wl.n_layers} layers d_model={wl.d_m} heads={wl.n_heads}x{wl.d_h} "
@@ -326,7 +339,7 @@ def run_gpu(args):
                      "frac": flops / ms_gemm / 1e9 / peaks["bf16_tflops_sustained"], "traffic": None,
                      "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                      "launches_per_step": n_gemm_launches, "avg_launch_ms": ms_gemm / n_gemm_launches},
-        "e2e": {"value": world * flops / ms_e2e / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
+        "e2e": {"value": job_throughput(world, flops, ms_e2e) / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": int(launches), "clocks": clocks,
     }
