@@ -165,21 +165,44 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
 // ------------------------------------------------------------------------------------------------
 // epilogue math (fp32)
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ float gelu_erf(float x) { return 0.5f * x * (1.f + erff(x * 0.70710678118654752f)); }
-__device__ __forceinline__ float dgelu_erf(float x) {
-    return 0.5f * (1.f + erff(x * 0.70710678118654752f)) + x * 0.39894228040143268f * __expf(-0.5f * x * x);
+// Phi(x) (standard normal CDF) and phi(x) (its density) from one exponential: erf by the rational
+// approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), whose exp(-z^2) factor at
+// z = |x|/sqrt(2) is exp(-x^2/2), the same exponential the density needs.
+__device__ __forceinline__ void normal_cdf_pdf(float x, float& cdf, float& pdf) {
+    const float z = fabsf(x) * 0.70710678118654752f;
+    const float e = __expf(-0.5f * x * x);
+    const float t = __fdividef(1.f, fmaf(0.3275911f, z, 1.f));
+    float p = fmaf(t, 1.061405429f, -1.453152027f);
+    p = fmaf(t, p, 1.421413741f);
+    p = fmaf(t, p, -0.284496736f);
+    p = fmaf(t, p, 0.254829592f);
+    const float half_erfc = 0.5f * p * t * e;          // 0.5 * erfc(z), z >= 0
+    cdf = x >= 0.f ? 1.f - half_erfc : half_erfc;
+    pdf = 0.39894228040143268f * e;
 }
+__device__ __forceinline__ float gelu_erf(float x) {
+    float c, d;
+    normal_cdf_pdf(x, c, d);
+    return x * c;
+}
+__device__ __forceinline__ float dgelu_erf(float x) {
+    float c, d;
+    normal_cdf_pdf(x, c, d);
+    return fmaf(x, d, c);
+}
+// tanh(u) = 1 - 2 / (1 + exp(2u)); saturates correctly for large |u|
+__device__ __forceinline__ float tanh_fast(float u) { return 1.f - __fdividef(2.f, 1.f + __expf(2.f * u)); }
 __device__ __forceinline__ float gelu_tanh(float x) {
     const float u = 0.79788456080286536f * (x + 0.044715f * x * x * x);
-    return 0.5f * x * (1.f + tanhf(u));
+    return 0.5f * x * (1.f + tanh_fast(u));
 }
 __device__ __forceinline__ float dgelu_tanh(float x) {
     const float u = 0.79788456080286536f * (x + 0.044715f * x * x * x);
-    const float t = tanhf(u);
+    const float t = tanh_fast(u);
     const float du = 0.79788456080286536f * (1.f + 3.f * 0.044715f * x * x);
     return 0.5f * (1.f + t) + 0.5f * x * (1.f - t * t) * du;
 }
-__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + __expf(-x)); }
+__device__ __forceinline__ float sigmoidf_(float x) { return __fdividef(1.f, 1.f + __expf(-x)); }
 
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);

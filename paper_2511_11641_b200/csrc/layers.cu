@@ -43,17 +43,56 @@ __global__ void __launch_bounds__(kThreads) cast_f32_bf16_kernel(const float* __
     }
 }
 
-// partial[chunk][c] = sum over the chunk's rows of M[r][c];  M is bf16 (rows x cols, pitch ld)
-constexpr int kSumRows = 256;
+// partial[chunk][c] = sum over the chunk's rows of M[r][c];  M is bf16 (rows x cols, pitch ld).
+// Tile = kSumRows rows x 256 columns: a lane owns 16 bytes (8 columns) of a row, the 8 warps stride
+// over the rows with 4 independent vector loads in flight, then add up through shared memory in warp order.
+constexpr int kSumRows = 512;
+constexpr int kSumCols = 256;
 __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const uint16_t* __restrict__ M, int64_t ld, int64_t rows,
-                                                                  int64_t cols, float* __restrict__ partial) {
-    const int c = blockIdx.x * kThreads + threadIdx.x;
+                                                                  int64_t cols, int vec_ok, float* __restrict__ partial) {
+    __shared__ float red[8][kSumCols + 4];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t c0 = static_cast<int64_t>(blockIdx.x) * kSumCols + lane * 8;
     const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kSumRows;
     const int64_t r1 = r0 + kSumRows < rows ? r0 + kSumRows : rows;
-    if (c >= cols) return;
-    float s = 0.f;
-    for (int64_t r = r0; r < r1; ++r) s += __uint_as_float(static_cast<uint32_t>(M[r * ld + c]) << 16);
-    partial[static_cast<int64_t>(blockIdx.y) * cols + c] = s;
+    float acc[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+    if (c0 < cols) {
+        if (vec_ok && c0 + 8 <= cols) {
+            const uint16_t* p = M + c0;
+            for (int64_t r = r0 + warp; r < r1; r += 32) {
+                uint4 v[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int64_t rr = r + 8 * u;
+                    v[u] = rr < r1 ? ldg_stream16(p + rr * ld) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    acc[0] += bf16_lo(v[u].x); acc[1] += bf16_hi(v[u].x);
+                    acc[2] += bf16_lo(v[u].y); acc[3] += bf16_hi(v[u].y);
+                    acc[4] += bf16_lo(v[u].z); acc[5] += bf16_hi(v[u].z);
+                    acc[6] += bf16_lo(v[u].w); acc[7] += bf16_hi(v[u].w);
+                }
+            }
+        } else {
+            for (int64_t r = r0 + warp; r < r1; r += 8)
+#pragma unroll
+                for (int e = 0; e < 8; ++e)
+                    if (c0 + e < cols) acc[e] += __uint_as_float(static_cast<uint32_t>(M[r * ld + c0 + e]) << 16);
+        }
+    }
+#pragma unroll
+    for (int e = 0; e < 8; ++e) red[warp][lane * 8 + e] = acc[e];
+    __syncthreads();
+    const int64_t c = static_cast<int64_t>(blockIdx.x) * kSumCols + threadIdx.x;
+    if (c < cols) {
+        float s = 0.f;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) s += red[w][threadIdx.x];
+        partial[static_cast<int64_t>(blockIdx.y) * cols + c] = s;
+    }
 }
 __global__ void __launch_bounds__(kThreads) colsum_final_kernel(const float* __restrict__ partial, int chunks, int64_t cols,
                                                                 void* out, int out_f32) {
@@ -137,10 +176,13 @@ void colsum(Ctx& cx, const Stored& M, void* out) {
         cx.st = ECOSPA_ERR_WORKSPACE;
         return;
     }
-    dim3 grid(static_cast<unsigned>(ceil_div(M.cols, kThreads)), chunks);
-    colsum_partial_kernel<<<grid, kThreads, 0, cx.stream>>>(static_cast<const uint16_t*>(M.ptr), M.ld, M.rows, M.cols, partial);
+    dim3 grid(static_cast<unsigned>(ceil_div(M.cols, kSumCols)), chunks);
+    const int vec_ok = aligned16(M.ptr) && M.ld % 8 == 0;
+    colsum_partial_kernel<<<grid, kThreads, 0, cx.stream>>>(static_cast<const uint16_t*>(M.ptr), M.ld, M.rows, M.cols, vec_ok,
+                                                            partial);
     if ((cx.st = check_launch("colsum_partial_kernel")) != ECOSPA_OK) return;
-    colsum_final_kernel<<<grid.x, kThreads, 0, cx.stream>>>(partial, chunks, M.cols, out, cx.dtype == ECOSPA_F32);
+    colsum_final_kernel<<<static_cast<unsigned>(ceil_div(M.cols, kThreads)), kThreads, 0, cx.stream>>>(
+        partial, chunks, M.cols, out, cx.dtype == ECOSPA_F32);
     cx.st = check_launch("colsum_final_kernel");
 }
 
