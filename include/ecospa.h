@@ -197,7 +197,9 @@ ecospa_status_t ecospa_compact_pair(const ecospa_pair_t* pair, const int32_t* ke
  *                 ECOSPA_ERR_UNSUPPORTED.
  *   pitches       all ld* in elements.  Every base pointer must be 16-byte aligned and every pitch a
  *                 multiple of 16 bytes (ECOSPA_ERR_ALIGNMENT otherwise); gradient outputs use the pitch
- *                 of a compacted weight (padded), pad columns are left untouched.
+ *                 of a compacted weight (padded).  Outputs are written in 16-byte units: the pad columns
+ *                 between n and the next multiple of 8 (bf16) elements may be overwritten (with what a zero
+ *                 weight column yields); columns beyond that are left untouched.
  *   workspace     DEVICE scratch, 16-byte aligned, at least ecospa_proj_workspace_bytes /
  *                 ecospa_ffn_workspace_bytes; may be NULL when that function returns 0.
  *   1/sqrt(d_h)   is not applied: Q^c and K^c are the plain projections.

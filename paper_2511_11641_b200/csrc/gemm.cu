@@ -35,8 +35,10 @@ constexpr int kAtomBytes = 64 * 64 * 2;     // one 64x64 bf16 swizzle atom of an
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
-constexpr int kMapsPerOp = 6;
-constexpr int kSmemBytes = kStages * (kAStage + kBStage) + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kMapsPerOp = 9;              // 2 A + 4 B operand maps, 3 output maps
+constexpr int kEpiSlotBytes = 32 * 32 * 2;  // one 32-row x 32-column bf16 store box
+constexpr int kEpiBytes = kEpiWarps * 2 * kEpiSlotBytes;
+constexpr int kSmemBytes = kStages * (kAStage + kBStage) + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct DevProblem {
@@ -48,7 +50,7 @@ struct DevProblem {
     int32_t epi;
     uint8_t a_mn[2], b_mn[2];
     uint8_t map_a[2], map_b[2][2];
-    uint8_t out_f32, accumulate, bias_f32, pad_[5];
+    uint8_t out_f32, accumulate, bias_f32, tma_store, map_c[3], pad_;
     void* C;
     void* C2;
     void* C3;
@@ -122,6 +124,17 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+
+// Shared -> global tile store; the tensor map clips rows and columns beyond the tensor's extent.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(x), "r"(y)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read_1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -242,6 +255,34 @@ __device__ __forceinline__ void store_row32(void* base, int64_t row_off, int n, 
     }
 }
 
+// Per-warp staging of 32 rows x 32 bf16 columns for a TMA store: lane = row, 64 bytes per row,
+// 16-byte chunks permuted by the 64-byte swizzle (chunk ^ ((row >> 1) & 3)) that the store's tensor map undoes.
+struct EpiStage {
+    uint32_t base;   // shared address of this warp's two 2 KB slots
+    int slot;
+};
+__device__ __forceinline__ void stage_store32(EpiStage& st, const CUtensorMap* map, int x, int y, const float (&v)[32], int lane) {
+    if (lane == 0) bulk_wait_read_1();       // the slot about to be rewritten has been read out
+    __syncwarp();
+    const uint32_t row = st.base + st.slot * kEpiSlotBytes + lane * 64;
+    const int sw = (lane >> 1) & 3;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint32_t a = row + ((c ^ sw) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(a), "r"(pack_bf16(v[8 * c + 0], v[8 * c + 1])),
+                     "r"(pack_bf16(v[8 * c + 2], v[8 * c + 3])), "r"(pack_bf16(v[8 * c + 4], v[8 * c + 5])),
+                     "r"(pack_bf16(v[8 * c + 6], v[8 * c + 7]))
+                     : "memory");
+    }
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        tma_store_2d(map, st.base + st.slot * kEpiSlotBytes, x, y);
+        bulk_commit();
+    }
+    st.slot ^= 1;
+}
+
 __device__ __forceinline__ void load_row32(const void* base, int64_t row_off, int n, int nv, float (&v)[32], bool f32) {
     if (f32) {
         const float* p = static_cast<const float*>(base) + row_off + n;
@@ -290,7 +331,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     const uint32_t base = (raw_addr + 1023u) & ~1023u;       // 1024-byte aligned stage memory
     uint8_t* smem = smem_raw + (base - raw_addr);
     const uint32_t sA = base, sB = base + kStages * kAStage;
-    uint8_t* tail = smem + kStages * (kAStage + kBStage);
+    const uint32_t sEpi = base + kStages * (kAStage + kBStage);
+    uint8_t* tail = smem + kStages * (kAStage + kBStage) + kEpiBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);        // full[4], empty[4], tmem_full[2], tmem_empty[2]
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 12 * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 12 * 8 + 8);
@@ -402,12 +444,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         const int ew = warp - 2;
         const int quad = warp & 3;            // TMEM lanes this warp may read: [32*quad, 32*quad + 32)
         const int half = ew >> 2;             // which half of the tile's columns
+        EpiStage stg{sEpi + ew * 2 * kEpiSlotBytes, 0};
         int it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++it) {
             const DevProblem& Q = find_problem(P, tile);
             const int local = tile - Q.tile_start;
-            const int m = (local % Q.tiles_m) * BM + quad * 32 + lane;
+            const int m_warp = (local % Q.tiles_m) * BM + quad * 32;   // first row of this warp
+            const int m = m_warp + lane;
             const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1u;
@@ -415,9 +459,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             tc_fence_after();
             const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
             const bool row_ok = m < Q.M;
+            const bool warp_rows = m_warp < Q.M;          // any row of this warp inside the output
             const int64_t c_off = static_cast<int64_t>(m) * Q.ldc;
             const int64_t h_off = static_cast<int64_t>(m) * Q.ldh;
             const int epi = Q.epi;
+            const bool tma = Q.tma_store != 0;
+            // writes 32 columns starting at n of output `which` (0: C, 1: C2, 2: C3)
+            auto emit = [&](int which, void* ptr, int n, int nv, const float (&v)[32]) {
+                if (tma) {
+                    if (warp_rows) stage_store32(stg, &P.maps[Q.map_c[which]], n, m_warp, v, lane);
+                } else if (row_ok) {
+                    store_row32(ptr, c_off, n, nv, v, Q.out_f32 != 0);
+                }
+            };
             if (epi == EPI_SWIGLU) {
                 // accumulator columns [0,128) = gate, [128,256) = up for hidden units n0 .. n0+127
 #pragma unroll 1
@@ -429,18 +483,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     tc_wait_ld();
                     const int n = n0 + hc;
                     const int nv = min(32, Q.N - n);
-                    if (row_ok && nv > 0) {
-                        float g[32], u[32], a[32];
+                    if (nv <= 0) continue;
+                    float g[32], u[32];
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) {
-                            g[i] = __uint_as_float(rg[i]);
-                            u[i] = __uint_as_float(ru[i]);
-                            a[i] = g[i] * sigmoidf_(g[i]) * u[i];
-                        }
-                        store_row32(Q.C, c_off, n, nv, g, false);
-                        store_row32(Q.C2, c_off, n, nv, u, false);
-                        store_row32(Q.C3, c_off, n, nv, a, false);
+                    for (int i = 0; i < 32; ++i) {
+                        g[i] = __uint_as_float(rg[i]);
+                        u[i] = __uint_as_float(ru[i]);
                     }
+                    emit(0, Q.C, n, nv, g);
+                    emit(1, Q.C2, n, nv, u);
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) g[i] = g[i] * sigmoidf_(g[i]) * u[i];
+                    emit(2, Q.C3, n, nv, g);
                 }
             } else {
 #pragma unroll 1
@@ -451,7 +505,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     tc_wait_ld();
                     const int n = n0 + col;
                     const int nv = min(32, Q.N - n);
-                    if (!(row_ok && nv > 0)) continue;
+                    if (nv <= 0) continue;
                     float v[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
@@ -462,37 +516,36 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         for (int i = 0; i < 32; ++i) v[i] += b[i];
                     }
                     if (epi == EPI_STORE) {
-                        if (Q.accumulate) {
+                        if (Q.accumulate && row_ok) {
                             float o[32];
                             load_row32(Q.C, c_off, n, nv, o, Q.out_f32 != 0);
 #pragma unroll
                             for (int i = 0; i < 32; ++i) v[i] += o[i];
                         }
-                        store_row32(Q.C, c_off, n, nv, v, Q.out_f32 != 0);
+                        emit(0, Q.C, n, nv, v);
                     } else if (epi == EPI_GELU_ERF || epi == EPI_GELU_TANH) {
-                        store_row32(Q.C, c_off, n, nv, v, false);
-                        float a[32];
+                        emit(0, Q.C, n, nv, v);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) a[i] = epi == EPI_GELU_ERF ? gelu_erf(v[i]) : gelu_tanh(v[i]);
-                        store_row32(Q.C2, c_off, n, nv, a, false);
+                        for (int i = 0; i < 32; ++i) v[i] = epi == EPI_GELU_ERF ? gelu_erf(v[i]) : gelu_tanh(v[i]);
+                        emit(1, Q.C2, n, nv, v);
                     } else if (epi == EPI_DGELU_ERF || epi == EPI_DGELU_TANH) {
                         float h[32];
-                        load_row32(Q.H, h_off, n, nv, h, false);
+                        load_row32(Q.H, h_off, n, row_ok ? nv : 0, h, false);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] *= epi == EPI_DGELU_ERF ? dgelu_erf(h[i]) : dgelu_tanh(h[i]);
-                        store_row32(Q.C, c_off, n, nv, v, false);
+                        emit(0, Q.C, n, nv, v);
                     } else {  // EPI_DSWIGLU
-                        float hg[32], hu[32], dg[32];
-                        load_row32(Q.H, h_off, n, nv, hg, false);
-                        load_row32(Q.Hb, h_off, n, nv, hu, false);
+                        float hg[32], hu[32];
+                        load_row32(Q.H, h_off, n, row_ok ? nv : 0, hg, false);
+                        load_row32(Q.Hb, h_off, n, row_ok ? nv : 0, hu, false);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float s = sigmoidf_(hg[i]);
-                            dg[i] = v[i] * hu[i] * s * (1.f + hg[i] * (1.f - s));
-                            v[i] = v[i] * hg[i] * s;
+                            hu[i] = v[i] * hu[i] * s * (1.f + hg[i] * (1.f - s));   // dH_gate
+                            v[i] = v[i] * hg[i] * s;                                // dH_up
                         }
-                        store_row32(Q.C, c_off, n, nv, dg, false);
-                        store_row32(Q.C2, c_off, n, nv, v, false);
+                        emit(0, Q.C, n, nv, hu);
+                        emit(1, Q.C2, n, nv, v);
                     }
                 }
             }
@@ -500,6 +553,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(acc));
         }
+        if (lane == 0) bulk_wait_all();       // every tile store of this warp has completed
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -537,8 +591,9 @@ EncodeFn get_encode() {
     return fn;
 }
 
-// Tensor map of a stored row-major bf16 matrix; box = 64 elements along the row x box_rows rows.
-ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows) {
+// Tensor map of a stored row-major bf16 matrix; box = 64 elements along the row x box_rows rows
+// (128-byte swizzle, operand loads), or 32 x 32 with the 64-byte swizzle (epilogue stores).
+ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows, bool store_box = false) {
     EncodeFn enc = get_encode();
     if (!enc) {
         set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
@@ -548,10 +603,11 @@ ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows) {
     if (!aligned16(s.ptr) || (s.ld * 2) % 16 != 0) return ECOSPA_ERR_ALIGNMENT;
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(s.cols), static_cast<cuuint64_t>(s.rows)};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(s.ld) * 2};
-    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
+    const cuuint32_t box[2] = {store_box ? 32u : 64u, static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(s.ptr), dims, strides, box, estr,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, store_box ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
@@ -648,6 +704,19 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
             const int32_t kb = static_cast<int32_t>(ceil_div(ks.K, BK));
             if (s == 0) Q.kblocks0 = kb;
             Q.kblocks += kb;
+        }
+        // bf16 outputs that are not read-modify-write go out as TMA tile stores
+        Q.tma_store = (!op.out_f32 && !op.accumulate) ? 1 : 0;
+        if (Q.tma_store) {
+            void* outs[3] = {op.C, op.C2, op.C3};
+            for (int w = 0; w < 3; ++w) {
+                if (!outs[w]) continue;
+                Stored o;
+                o.ptr = outs[w]; o.rows = op.M; o.cols = op.N; o.ld = op.ldc;
+                const int mi = oi * kMapsPerOp + 6 + w;
+                if ((st = encode_map(&gp.maps[mi], o, 32, true)) != ECOSPA_OK) return st;
+                Q.map_c[w] = static_cast<uint8_t>(mi);
+            }
         }
         Q.tiles_m = static_cast<int32_t>(ceil_div(op.M, BM));
         Q.tiles_n = static_cast<int32_t>(ceil_div(op.N, Q.n_per_tile));

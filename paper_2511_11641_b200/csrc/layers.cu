@@ -46,7 +46,7 @@ __global__ void __launch_bounds__(kThreads) cast_f32_bf16_kernel(const float* __
 // partial[chunk][c] = sum over the chunk's rows of M[r][c];  M is bf16 (rows x cols, pitch ld).
 // Tile = kSumRows rows x 256 columns: a lane owns 16 bytes (8 columns) of a row, the 8 warps stride
 // over the rows with 4 independent vector loads in flight, then add up through shared memory in warp order.
-constexpr int kSumRows = 512;
+constexpr int kSumRows = 64;
 constexpr int kSumCols = 256;
 __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const uint16_t* __restrict__ M, int64_t ld, int64_t rows,
                                                                   int64_t cols, int vec_ok, float* __restrict__ partial) {
@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const uint16_t
     if (c0 < cols) {
         if (vec_ok && c0 + 8 <= cols) {
             const uint16_t* p = M + c0;
-            for (int64_t r = r0 + warp; r < r1; r += 32) {
+            for (int64_t r = r0 + warp; r < r1; r += 32) {   // two rounds of 4 rows per warp
                 uint4 v[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
