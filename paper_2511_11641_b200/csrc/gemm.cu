@@ -1,5 +1,10 @@
-// Grouped persistent bf16 GEMM for sm_100a: TMA -> shared memory ring -> tcgen05.mma (cta_group::1,
-// 128x256x16, fp32 accumulators in TMEM, double buffered) -> fused epilogues.
+// Grouped persistent bf16 GEMM for sm_100a: TMA -> shared memory ring -> tcgen05.mma (fp32 accumulators
+// in TMEM, double buffered) -> fused epilogues.  Two forms of the same kernel:
+//   single  cta_group::1, one CTA per SM computes 128x256 tiles (4-stage ring of 16 KB A + 32 KB B)
+//   pair    cta_group::2, a cluster of two CTAs computes 256x256 tiles: each CTA loads its 128 rows of A
+//           and its half of B (6-stage ring of 16 KB + 16 KB), the leader CTA issues the MMAs for both,
+//           so every SM fetches a third less operand data per flop.  No cluster multicast is used: the
+//           peer's loads signal the leader's barrier, and completion is committed to each CTA's barrier.
 //
 // One launch computes up to kMaxGemmOps independent products ("ops"), each C = sum over one or two
 // K segments of A_seg * B_seg with K-major or MN-major operands (chosen per segment, so that weights
@@ -16,6 +21,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <mutex>
 
@@ -27,10 +33,11 @@ namespace ecospa {
 namespace {
 
 constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages = 4;
 constexpr int kAStage = BM * BK * 2;        // 16 KB
 constexpr int kBStage = BN * BK * 2;        // 32 KB
 constexpr int kBHalf = kBStage / 2;
+constexpr int kRingBytes = 4 * (kAStage + kBStage);   // = 6 * (kAStage + kBHalf) = 192 KB
+constexpr int kMaxStages = 6;
 constexpr int kAtomBytes = 64 * 64 * 2;     // one 64x64 bf16 swizzle atom of an MN-major operand
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
@@ -38,7 +45,7 @@ constexpr int kTmemCols = 512;
 constexpr int kMapsPerOp = 9;              // 2 A + 4 B operand maps, 3 output maps
 constexpr int kEpiSlotBytes = 32 * 32 * 2;  // one 32-row x 32-column bf16 store box
 constexpr int kEpiBytes = kEpiWarps * 2 * kEpiSlotBytes;
-constexpr int kSmemBytes = kStages * (kAStage + kBStage) + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr int kSmemBytes = kRingBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct DevProblem {
@@ -101,12 +108,16 @@ __device__ __forceinline__ unsigned long long global_ns() {
 }
 
 // Bounded wait.  Returns false if the wait gave up (or another thread of the CTA already did).
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity);
+
+template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code, int* status) {
-    if (mbar_try_wait(bar, parity)) return true;
+    auto poll = [&]() { return CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
+    if (poll()) return true;
     const unsigned long long t0 = global_ns();
     uint32_t spins = 0;
     while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (poll()) return true;
         if ((++spins & 255u) == 0) {
             if (*abort_flag) return false;
             if (global_ns() - t0 > kWaitLimitNs) {
@@ -116,6 +127,59 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             }
         }
     }
+}
+
+// --- cluster (CTA pair) helpers
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of `addr` (a shared::cta address of this CTA) in the CTA of rank `rank`
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(uint32_t cluster_addr, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// TMA load issued by one CTA of a pair; the completion may be signalled on the peer's (leader's) barrier.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(x), "r"(y)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar_cluster) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar_cluster) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
 }
 
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -325,17 +389,22 @@ __device__ __forceinline__ const DevProblem& find_problem(const GemmParams& P, i
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
+template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams P) {
+    constexpr int kStages = PAIR ? 6 : 4;
+    constexpr int kBLocal = PAIR ? kBHalf : kBStage;        // B bytes this CTA holds per stage
+    constexpr int kTileM = PAIR ? 2 * BM : BM;               // rows of one scheduled tile
+    constexpr uint32_t kStageTx = kAStage + kBLocal;         // bytes this CTA's loads deliver per stage
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;       // 1024-byte aligned stage memory
     uint8_t* smem = smem_raw + (base - raw_addr);
     const uint32_t sA = base, sB = base + kStages * kAStage;
-    const uint32_t sEpi = base + kStages * (kAStage + kBStage);
-    uint8_t* tail = smem + kStages * (kAStage + kBStage) + kEpiBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);        // full[4], empty[4], tmem_full[2], tmem_empty[2]
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 12 * 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 12 * 8 + 8);
+    const uint32_t sEpi = base + kRingBytes;
+    uint8_t* tail = smem + kRingBytes + kEpiBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);        // full[S], empty[S], tmem_full[2], tmem_empty[2]
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + (2 * kMaxStages + 4) * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + (2 * kMaxStages + 4) * 8 + 8);
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
@@ -343,62 +412,92 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;   // 0 = leader: issues the MMAs, owns full/tmem_empty
+    const bool leader = cta_rank == 0;
+    const int worker = PAIR ? blockIdx.x >> 1 : blockIdx.x;
+    const int n_workers = PAIR ? gridDim.x >> 1 : gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar(s), 1);
+            mbar_init(full_bar(s), PAIR ? 2 : 1);     // one expect_tx arrival per CTA of the pair
             mbar_init(empty_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), kEpiWarps);
+            mbar_init(tempty_bar(a), PAIR ? 2 * kEpiWarps : kEpiWarps);
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_holder)), "r"(kTmemCols) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();     // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ producer
+        // ------------------------------------------------------------------ producer (both CTAs of a pair)
         if (lane == 0) {
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x) {
+            for (int tile = worker; ok && tile < P.total_tiles; tile += n_workers) {
                 const DevProblem& Q = find_problem(P, tile);
                 const int local = tile - Q.tile_start;
-                const int m0 = (local % Q.tiles_m) * BM;
+                const int m0 = (local % Q.tiles_m) * kTileM + static_cast<int>(cta_rank) * BM;
                 const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
                 for (int kb = 0; kb < Q.kblocks; ++kb) {
                     const int seg = kb >= Q.kblocks0 ? 1 : 0;
                     const int k0 = (seg ? kb - Q.kblocks0 : kb) * BK;
-                    if (!(ok = mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
-                    mbar_expect_tx(full_bar(stage), kAStage + kBStage);
-                    const uint32_t a_dst = sA + stage * kAStage, b_dst = sB + stage * kBStage;
+                    if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
+                    const uint32_t a_dst = sA + stage * kAStage, b_dst = sB + stage * kBLocal;
                     const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
-                    if (!Q.a_mn[seg]) {
-                        tma_load_2d(a_dst, ma, k0, m0, full_bar(stage));                    // box 64(k) x 128(m)
-                    } else {
-                        tma_load_2d(a_dst, ma, m0, k0, full_bar(stage));                    // box 64(m) x 64(k)
-                        tma_load_2d(a_dst + kAtomBytes, ma, m0 + 64, k0, full_bar(stage));
-                    }
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const CUtensorMap* mb = &P.maps[Q.map_b[seg][h]];
-                        const int nc = n0 + h * Q.half1_n_off;
-                        const uint32_t dst = b_dst + h * kBHalf;
-                        if (!Q.b_mn[seg]) {
-                            tma_load_2d(dst, mb, k0, nc, full_bar(stage));                  // box 64(k) x 128(n)
+                    if (PAIR) {
+                        // this CTA's share of the stage, signalled on the leader's barrier
+                        const uint32_t fb = map_to_cta(full_bar(stage), 0);
+                        mbar_expect_tx_cluster(fb, kStageTx);
+                        if (!Q.a_mn[seg]) {
+                            tma_load_2d_pair(a_dst, ma, k0, m0, fb);
                         } else {
-                            tma_load_2d(dst, mb, nc, k0, full_bar(stage));                  // box 64(n) x 64(k)
-                            tma_load_2d(dst + kAtomBytes, mb, nc + 64, k0, full_bar(stage));
+                            tma_load_2d_pair(a_dst, ma, m0, k0, fb);
+                            tma_load_2d_pair(a_dst + kAtomBytes, ma, m0 + 64, k0, fb);
+                        }
+                        const CUtensorMap* mb = &P.maps[Q.map_b[seg][cta_rank]];
+                        const int nc = n0 + static_cast<int>(cta_rank) * Q.half1_n_off;
+                        if (!Q.b_mn[seg]) {
+                            tma_load_2d_pair(b_dst, mb, k0, nc, fb);
+                        } else {
+                            tma_load_2d_pair(b_dst, mb, nc, k0, fb);
+                            tma_load_2d_pair(b_dst + kAtomBytes, mb, nc + 64, k0, fb);
+                        }
+                    } else {
+                        mbar_expect_tx(full_bar(stage), kStageTx);
+                        if (!Q.a_mn[seg]) {
+                            tma_load_2d(a_dst, ma, k0, m0, full_bar(stage));                    // box 64(k) x 128(m)
+                        } else {
+                            tma_load_2d(a_dst, ma, m0, k0, full_bar(stage));                    // box 64(m) x 64(k)
+                            tma_load_2d(a_dst + kAtomBytes, ma, m0 + 64, k0, full_bar(stage));
+                        }
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const CUtensorMap* mb = &P.maps[Q.map_b[seg][h]];
+                            const int nc = n0 + h * Q.half1_n_off;
+                            const uint32_t dst = b_dst + h * kBHalf;
+                            if (!Q.b_mn[seg]) {
+                                tma_load_2d(dst, mb, k0, nc, full_bar(stage));                  // box 64(k) x 128(n)
+                            } else {
+                                tma_load_2d(dst, mb, nc, k0, full_bar(stage));                  // box 64(n) x 64(k)
+                                tma_load_2d(dst + kAtomBytes, mb, nc + 64, k0, full_bar(stage));
+                            }
                         }
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
@@ -406,37 +505,52 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (lane == 0 && leader) {
             int stage = 0;
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++it) {
+            for (int tile = worker; ok && tile < P.total_tiles; tile += n_workers, ++it) {
                 const DevProblem& Q = find_problem(P, tile);
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1u;
-                if (!(ok = mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 2, P.status))) break;
+                if (!(ok = mbar_wait<PAIR>(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 2, P.status))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < Q.kblocks; ++kb) {
                     const int seg = kb >= Q.kblocks0 ? 1 : 0;
-                    if (!(ok = mbar_wait(full_bar(stage), phase, abort_flag, 3, P.status))) break;
+                    if (!(ok = mbar_wait<PAIR>(full_bar(stage), phase, abort_flag, 3, P.status))) break;
                     tc_fence_after();
                     const uint32_t a_mn = Q.a_mn[seg], b_mn = Q.b_mn[seg];
                     const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) |
-                                           (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(BM >> 4) << 24);
+                                           (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
                     const uint64_t a_desc = make_smem_desc(sA + stage * kAStage, a_mn ? kAtomBytes : 16, 1024);
-                    const uint64_t b_desc = make_smem_desc(sB + stage * kBStage, b_mn ? kAtomBytes : 16, 1024);
+                    const uint64_t b_desc = make_smem_desc(sB + stage * kBLocal, b_mn ? kAtomBytes : 16, 1024);
                     const uint64_t a_step = a_mn ? (2048 >> 4) : (32 >> 4);   // per 16 k: two 8-row groups, or 32 bytes
                     const uint64_t b_step = b_mn ? (2048 >> 4) : (32 >> 4);
 #pragma unroll
-                    for (int ks = 0; ks < BK / 16; ++ks)
-                        tc_mma_bf16(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
-                    tc_commit(empty_bar(stage));      // the stage is free once these MMAs have read it
+                    for (int ks = 0; ks < BK / 16; ++ks) {
+                        if (PAIR) tc_mma_bf16_pair(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
+                        else tc_mma_bf16(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
+                    }
+                    // the stage is free (in both CTAs) once these MMAs have read it
+                    if (PAIR) {
+                        tc_commit_pair(map_to_cta(empty_bar(stage), 0));
+                        tc_commit_pair(map_to_cta(empty_bar(stage), 1));
+                    } else {
+                        tc_commit(empty_bar(stage));
+                    }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
-                if (ok) tc_commit(tfull_bar(acc));    // accumulator complete
+                if (ok) {                              // accumulator complete (in both CTAs)
+                    if (PAIR) {
+                        tc_commit_pair(map_to_cta(tfull_bar(acc), 0));
+                        tc_commit_pair(map_to_cta(tfull_bar(acc), 1));
+                    } else {
+                        tc_commit(tfull_bar(acc));
+                    }
+                }
             }
         }
     } else {
@@ -447,15 +561,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         EpiStage stg{sEpi + ew * 2 * kEpiSlotBytes, 0};
         int it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < P.total_tiles; tile += gridDim.x, ++it) {
+        for (int tile = worker; ok && tile < P.total_tiles; tile += n_workers, ++it) {
             const DevProblem& Q = find_problem(P, tile);
             const int local = tile - Q.tile_start;
-            const int m_warp = (local % Q.tiles_m) * BM + quad * 32;   // first row of this warp
+            const int m_warp = (local % Q.tiles_m) * kTileM + static_cast<int>(cta_rank) * BM + quad * 32;   // first row of this warp
             const int m = m_warp + lane;
             const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1u;
-            if (!(ok = mbar_wait(tfull_bar(acc), acc_phase, abort_flag, 4, P.status))) break;
+            if (!(ok = mbar_wait<PAIR>(tfull_bar(acc), acc_phase, abort_flag, 4, P.status))) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
             const bool row_ok = m < Q.M;
@@ -551,7 +665,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(tempty_bar(acc));
+            if (lane == 0) {                       // the accumulator may be overwritten: tell the MMA issuer
+                if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
+                else mbar_arrive(tempty_bar(acc));
+            }
         }
         if (lane == 0) bulk_wait_all();       // every tile store of this warp has completed
     }
@@ -565,9 +682,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();     // neither CTA leaves while the other may still signal its barriers
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -618,6 +737,7 @@ ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows, bool
 
 int g_num_sms = 0;
 int* g_status_ptr = nullptr;
+int g_pair_mode = 1;   // 1: CTA pairs (cta_group::2) whenever an op has more than one 128-row tile; 0: never
 
 ecospa_status_t gemm_setup() {
     static std::once_flag once;
@@ -626,7 +746,9 @@ ecospa_status_t gemm_setup() {
         int dev = 0;
         cudaError_t e = cudaGetDevice(&dev);
         if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+        if (const char* v = std::getenv("ECOSPA_GEMM_PAIR")) g_pair_mode = std::atoi(v);
         if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&g_status_ptr), g_gemm_status);
         if (e != cudaSuccess) {
             set_cuda_error(e, "gemm setup");
@@ -652,6 +774,15 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
         for (int s = 0; s < ops[i].n_kseg; ++s) ktot[i] += ceil_div(ops[i].seg[s].K, BK);
     }
     std::stable_sort(order, order + n_ops, [&](int a, int b) { return ktot[a] > ktot[b]; });
+
+    // CTA pairs pay off as soon as there is more than one 128-row tile to share a B tile between
+    bool pair = g_pair_mode != 0 && g_num_sms >= 2;
+    if (pair) {
+        bool any_tall = false;
+        for (int i = 0; i < n_ops; ++i) any_tall = any_tall || ops[i].M > BM;
+        pair = any_tall;
+    }
+    const int tile_m = pair ? 2 * BM : BM;
 
     static thread_local GemmParams gp;
     int tiles = 0;
@@ -718,7 +849,7 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
                 Q.map_c[w] = static_cast<uint8_t>(mi);
             }
         }
-        Q.tiles_m = static_cast<int32_t>(ceil_div(op.M, BM));
+        Q.tiles_m = static_cast<int32_t>(ceil_div(op.M, tile_m));
         Q.tiles_n = static_cast<int32_t>(ceil_div(op.N, Q.n_per_tile));
         Q.tile_start = tiles;
         tiles += Q.tiles_m * Q.tiles_n;
@@ -726,9 +857,30 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
     gp.n_problems = n_ops;
     gp.total_tiles = tiles;
     gp.status = g_status_ptr;
-    const int grid = std::min(tiles, g_num_sms);
-    gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(gp);
-    return check_launch("gemm_kernel");
+    if (!pair) {
+        const int grid = std::min(tiles, g_num_sms);
+        gemm_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(gp);
+        return check_launch("gemm_kernel");
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(2 * std::min(tiles, g_num_sms / 2));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<true>, gp);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "gemm_kernel (pair) launch");
+        cudaGetLastError();
+        return ECOSPA_ERR_CUDA;
+    }
+    return check_launch("gemm_kernel (pair)");
 }
 
 }  // namespace ecospa
