@@ -259,6 +259,10 @@ ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, int64_t T, in
                                        void* dW1b_c, int64_t ld_dw1, void* dW2_c, int64_t ld_dw2, void* db1_c,
                                        void* db2, void* workspace, size_t workspace_bytes, void* stream);
 
+/* How many CTA pairs (2-SM clusters) of the GEMM engine are resident at once on the current device; 0 when
+ * pair mode is off (environment ECOSPA_GEMM_PAIR=0), -1 on a CUDA error.  Informational. */
+int32_t ecospa_gemm_resident_pairs(void);
+
 /* Synchronises `stream` and reports the device status word: ECOSPA_OK and *code = 0, or
  * ECOSPA_ERR_TIMEOUT and *code = which bounded wait expired (1 producer, 2 accumulator-free,
  * 3 operands-ready, 4 accumulator-ready); the word is cleared.  This is the one call that blocks. */

@@ -112,15 +112,17 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t par
 
 template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code, int* status) {
-    auto poll = [&]() { return CLUSTER ? mbar_try_wait_cluster(bar, parity) : mbar_try_wait(bar, parity); };
-    if (poll()) return true;
-    const unsigned long long t0 = global_ns();
+    // Fast path: plain polling.  The (slow) global timer is only consulted every 1024 failed polls,
+    // so a wait that completes normally never touches it.
+    unsigned long long t0 = 0;
     uint32_t spins = 0;
     while (true) {
-        if (poll()) return true;
-        if ((++spins & 255u) == 0) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 1023u) == 0) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > kWaitLimitNs) {
+            const unsigned long long now = global_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitNs) {
                 *abort_flag = 1;
                 atomicCAS(status, 0, code);
                 return false;
@@ -419,7 +421,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(full_bar(s), PAIR ? 2 : 1);     // one expect_tx arrival per CTA of the pair
+            mbar_init(full_bar(s), 1);                // the leader's producer announces the bytes of both CTAs
             mbar_init(empty_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -464,7 +466,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     if (PAIR) {
                         // this CTA's share of the stage, signalled on the leader's barrier
                         const uint32_t fb = map_to_cta(full_bar(stage), 0);
-                        mbar_expect_tx_cluster(fb, kStageTx);
+                        if (leader) mbar_expect_tx(full_bar(stage), 2 * kStageTx);
                         if (!Q.a_mn[seg]) {
                             tma_load_2d_pair(a_dst, ma, k0, m0, fb);
                         } else {
@@ -737,6 +739,7 @@ ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows, bool
 
 int g_num_sms = 0;
 int* g_status_ptr = nullptr;
+int g_max_pairs = 0;   // CTA pairs that can be resident at once (clusters must fit inside a GPC)
 int g_pair_mode = 1;   // 1: CTA pairs (cta_group::2) whenever an op has more than one 128-row tile; 0: never
 
 ecospa_status_t gemm_setup() {
@@ -749,6 +752,24 @@ ecospa_status_t gemm_setup() {
         if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (const char* v = std::getenv("ECOSPA_GEMM_PAIR")) g_pair_mode = std::atoi(v);
+        if (e == cudaSuccess) {
+            // the tile schedule is static, so only as many pairs as can run at the same time are launched
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(2 * (g_num_sms / 2));
+            cfg.blockDim = dim3(kThreads);
+            cfg.dynamicSmemBytes = kSmemBytes;
+            cudaLaunchAttribute attr[1];
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = 2;
+            attr[0].val.clusterDim.y = 1;
+            attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true>, &cfg) == cudaSuccess && n > 0) g_max_pairs = n;
+            else cudaGetLastError();
+            if (g_max_pairs < 1) g_pair_mode = 0;
+        }
         if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&g_status_ptr), g_gemm_status);
         if (e != cudaSuccess) {
             set_cuda_error(e, "gemm setup");
@@ -776,7 +797,7 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
     std::stable_sort(order, order + n_ops, [&](int a, int b) { return ktot[a] > ktot[b]; });
 
     // CTA pairs pay off as soon as there is more than one 128-row tile to share a B tile between
-    bool pair = g_pair_mode != 0 && g_num_sms >= 2;
+    bool pair = g_pair_mode != 0 && g_max_pairs >= 1;
     if (pair) {
         bool any_tall = false;
         for (int i = 0; i < n_ops; ++i) any_tall = any_tall || ops[i].M > BM;
@@ -863,7 +884,7 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
         return check_launch("gemm_kernel");
     }
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * std::min(tiles, g_num_sms / 2));
+    cfg.gridDim = dim3(2 * std::min(tiles, g_max_pairs));
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
@@ -902,4 +923,10 @@ extern "C" ecospa_status_t ecospa_device_status(void* stream, int32_t* code) {
         return ECOSPA_ERR_TIMEOUT;
     }
     return ECOSPA_OK;
+}
+
+// Number of CTA pairs the GEMM engine runs at once on the current device (0 = pair mode off).
+extern "C" int32_t ecospa_gemm_resident_pairs(void) {
+    if (ecospa::gemm_setup() != ECOSPA_OK) return -1;
+    return ecospa::g_pair_mode ? ecospa::g_max_pairs : 0;
 }
