@@ -43,30 +43,46 @@ __global__ void __launch_bounds__(kThreads) cast_f32_bf16_kernel(const float* __
     }
 }
 
-// partial[chunk][c] = sum over the chunk's rows of M[r][c];  M is bf16 (rows x cols, pitch ld).
-// Tile = kSumRows rows x 256 columns: a lane owns 16 bytes (8 columns) of a row, the 8 warps stride
-// over the rows with 4 independent vector loads in flight, then add up through shared memory in warp order.
-constexpr int kSumRows = 64;
-constexpr int kSumCols = 256;
-__global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const uint16_t* __restrict__ M, int64_t ld, int64_t rows,
-                                                                  int64_t cols, int vec_ok, float* __restrict__ partial) {
-    __shared__ float red[8][kSumCols + 4];
+// Column sums (bias gradients) of up to two bf16 matrices with the same number of rows, two launches:
+// partial[chunk][c] over tiles of kSumRows rows x 64 columns (8 lanes cover a row's 128 bytes with
+// 16-byte loads, the block covers 32 rows per pass, 4 passes in flight), then a fixed-order sum of the chunks.
+constexpr int kSumRows = 512;
+constexpr int kSumCols = 64;
+struct ColsumJob {
+    const uint16_t* M;
+    float* partial;
+    void* out;
+    int64_t ld, cols;
+    int32_t col_tiles, vec_ok;
+};
+struct ColsumParams {
+    ColsumJob job[2];
+    int64_t rows;
+    int32_t n_jobs, chunks, out_f32;
+};
+
+__global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const __grid_constant__ ColsumParams P) {
+    __shared__ float red[32][kSumCols + 1];
+    const int ji = (P.n_jobs > 1 && static_cast<int>(blockIdx.x) >= P.job[0].col_tiles) ? 1 : 0;
+    const ColsumJob& J = P.job[ji];
+    const int ct = blockIdx.x - (ji ? P.job[0].col_tiles : 0);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t c0 = static_cast<int64_t>(blockIdx.x) * kSumCols + lane * 8;
+    const int rowoff = (lane >> 3) + 4 * warp;              // 0..31
+    const int64_t c0 = static_cast<int64_t>(ct) * kSumCols + (lane & 7) * 8;
     const int64_t r0 = static_cast<int64_t>(blockIdx.y) * kSumRows;
-    const int64_t r1 = r0 + kSumRows < rows ? r0 + kSumRows : rows;
+    const int64_t r1 = r0 + kSumRows < P.rows ? r0 + kSumRows : P.rows;
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-    if (c0 < cols) {
-        if (vec_ok && c0 + 8 <= cols) {
-            const uint16_t* p = M + c0;
-            for (int64_t r = r0 + warp; r < r1; r += 32) {   // two rounds of 4 rows per warp
+    if (c0 < J.cols) {
+        if (J.vec_ok && c0 + 8 <= J.cols) {
+            const uint16_t* p = J.M + c0;
+            for (int64_t r = r0 + rowoff; r < r1; r += 128) {
                 uint4 v[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int64_t rr = r + 8 * u;
-                    v[u] = rr < r1 ? ldg_stream16(p + rr * ld) : make_uint4(0, 0, 0, 0);
+                    const int64_t rr = r + 32 * u;
+                    v[u] = rr < r1 ? ldg_stream16(p + rr * J.ld) : make_uint4(0, 0, 0, 0);
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
@@ -77,31 +93,38 @@ __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const uint16_t
                 }
             }
         } else {
-            for (int64_t r = r0 + warp; r < r1; r += 8)
+            for (int64_t r = r0 + rowoff; r < r1; r += 32)
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
-                    if (c0 + e < cols) acc[e] += __uint_as_float(static_cast<uint32_t>(M[r * ld + c0 + e]) << 16);
+                    if (c0 + e < J.cols) acc[e] += __uint_as_float(static_cast<uint32_t>(J.M[r * J.ld + c0 + e]) << 16);
         }
     }
 #pragma unroll
-    for (int e = 0; e < 8; ++e) red[warp][lane * 8 + e] = acc[e];
+    for (int e = 0; e < 8; ++e) red[rowoff][(lane & 7) * 8 + e] = acc[e];
     __syncthreads();
-    const int64_t c = static_cast<int64_t>(blockIdx.x) * kSumCols + threadIdx.x;
-    if (c < cols) {
-        float s = 0.f;
+    if (threadIdx.x < kSumCols) {
+        const int64_t c = static_cast<int64_t>(ct) * kSumCols + threadIdx.x;
+        if (c < J.cols) {
+            float s = 0.f;
 #pragma unroll
-        for (int w = 0; w < 8; ++w) s += red[w][threadIdx.x];
-        partial[static_cast<int64_t>(blockIdx.y) * cols + c] = s;
+            for (int w = 0; w < 32; ++w) s += red[w][threadIdx.x];
+            J.partial[static_cast<int64_t>(blockIdx.y) * J.cols + c] = s;
+        }
     }
 }
-__global__ void __launch_bounds__(kThreads) colsum_final_kernel(const float* __restrict__ partial, int chunks, int64_t cols,
-                                                                void* out, int out_f32) {
-    const int c = blockIdx.x * kThreads + threadIdx.x;
-    if (c >= cols) return;
+__global__ void __launch_bounds__(kThreads) colsum_final_kernel(const __grid_constant__ ColsumParams P) {
+    int64_t c = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
+    int ji = 0;
+    if (c >= P.job[0].cols) {
+        c -= P.job[0].cols;
+        ji = 1;
+        if (P.n_jobs < 2 || c >= P.job[1].cols) return;
+    }
+    const ColsumJob& J = P.job[ji];
     float s = 0.f;
-    for (int k = 0; k < chunks; ++k) s += partial[static_cast<int64_t>(k) * cols + c];
-    if (out_f32) static_cast<float*>(out)[c] = s;
-    else static_cast<__nv_bfloat16*>(out)[c] = __float2bfloat16_rn(s);
+    for (int k = 0; k < P.chunks; ++k) s += J.partial[static_cast<int64_t>(k) * J.cols + c];
+    if (P.out_f32) static_cast<float*>(J.out)[c] = s;
+    else static_cast<__nv_bfloat16*>(J.out)[c] = __float2bfloat16_rn(s);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -167,22 +190,41 @@ Stored scratch_bf16(Ctx& cx, int64_t rows, int64_t cols) {
     return s;
 }
 
-// out[c] = sum_r M[r][c] for a bf16 matrix; out has the model dtype.
-void colsum(Ctx& cx, const Stored& M, void* out) {
-    if (cx.st != ECOSPA_OK || !out) return;
-    const int chunks = static_cast<int>(ceil_div(M.rows, kSumRows));
-    float* partial = static_cast<float*>(cx.arena.take(static_cast<size_t>(chunks) * M.cols * 4));
-    if (!partial) {
-        cx.st = ECOSPA_ERR_WORKSPACE;
-        return;
+// out[c] = sum_r M[r][c] for one or two bf16 matrices with the same row count; outputs have the model
+// dtype.  A null output skips that matrix.
+void colsum(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), void* out2 = nullptr) {
+    if (cx.st != ECOSPA_OK) return;
+    ColsumParams P = {};
+    const Stored* mats[2] = {&M1, &M2};
+    void* outs[2] = {out1, out2};
+    for (int i = 0; i < 2; ++i) {
+        if (!outs[i] || !mats[i]->ptr) continue;
+        ColsumJob& J = P.job[P.n_jobs++];
+        J.M = static_cast<const uint16_t*>(mats[i]->ptr);
+        J.out = outs[i];
+        J.ld = mats[i]->ld;
+        J.cols = mats[i]->cols;
+        J.col_tiles = static_cast<int32_t>(ceil_div(J.cols, kSumCols));
+        J.vec_ok = aligned16(J.M) && J.ld % 8 == 0;
+        P.rows = mats[i]->rows;
     }
-    dim3 grid(static_cast<unsigned>(ceil_div(M.cols, kSumCols)), chunks);
-    const int vec_ok = aligned16(M.ptr) && M.ld % 8 == 0;
-    colsum_partial_kernel<<<grid, kThreads, 0, cx.stream>>>(static_cast<const uint16_t*>(M.ptr), M.ld, M.rows, M.cols, vec_ok,
-                                                            partial);
+    if (P.n_jobs == 0) return;
+    P.chunks = static_cast<int32_t>(ceil_div(P.rows, kSumRows));
+    P.out_f32 = cx.dtype == ECOSPA_F32;
+    int64_t total_cols = 0;
+    int tiles = 0;
+    for (int i = 0; i < P.n_jobs; ++i) {
+        P.job[i].partial = static_cast<float*>(cx.arena.take(static_cast<size_t>(P.chunks) * P.job[i].cols * 4));
+        if (!P.job[i].partial) {
+            cx.st = ECOSPA_ERR_WORKSPACE;
+            return;
+        }
+        total_cols += P.job[i].cols;
+        tiles += P.job[i].col_tiles;
+    }
+    colsum_partial_kernel<<<dim3(tiles, P.chunks), kThreads, 0, cx.stream>>>(P);
     if ((cx.st = check_launch("colsum_partial_kernel")) != ECOSPA_OK) return;
-    colsum_final_kernel<<<static_cast<unsigned>(ceil_div(M.cols, kThreads)), kThreads, 0, cx.stream>>>(
-        partial, chunks, M.cols, out, cx.dtype == ECOSPA_F32);
+    colsum_final_kernel<<<static_cast<unsigned>(ceil_div(total_cols, kThreads)), kThreads, 0, cx.stream>>>(P);
     cx.st = check_launch("colsum_final_kernel");
 }
 
@@ -314,8 +356,7 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    colsum(cx, dQs, dbq_c);
-    if (wk_c) colsum(cx, dKs, dbk_c);
+    colsum(cx, dQs, dbq_c, dKs, wk_c ? dbk_c : nullptr);
     return cx.st;
 }
 
@@ -381,8 +422,7 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     dx.seg[0].a = dVs; dx.seg[0].b[0] = Wv; dx.seg[0].K = n;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, 4, cx.stream)) != ECOSPA_OK) return st;
-    colsum(cx, dVs, dbv_c);
-    colsum(cx, dOs, dbo);
+    colsum(cx, dVs, dbv_c, dOs, dbo);
     return cx.st;
 }
 
@@ -481,7 +521,6 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    if (!sw) colsum(cx, dH, db1_c);
-    colsum(cx, dYs, db2);
+    colsum(cx, dYs, db2, dH, sw ? nullptr : db1_c);
     return cx.st;
 }
