@@ -380,38 +380,47 @@ __device__ __forceinline__ void staged_store32(uint32_t buf, __nv_bfloat16* C, i
     __syncwarp();
 }
 
-// global (bf16, rows m_warp.. x columns n..n+31, coalesced) -> buffer -> registers (one row per lane)
-__device__ __forceinline__ void staged_load32(uint32_t buf, const unsigned short* H, int64_t ldh, int m_warp, int n, int M, int N,
-                                              float (&v)[32], int lane) {
+// global (bf16, rows m_warp.. x columns n..n+31) -> registers in the coalesced "line" pattern.  Split in
+// two so that the global loads of the next chunk are in flight while the current one is processed.
+__device__ __forceinline__ void staged_load32_issue(const unsigned short* H, int64_t ldh, int m_warp, int n, int M, int N,
+                                                    uint4 (&q)[4], int lane) {
     const int c = lane & 3;
     const int col = n + 8 * c;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int row = 8 * i + (lane >> 2);
-        uint4 q = make_uint4(0, 0, 0, 0);
+        q[i] = make_uint4(0, 0, 0, 0);
         if (m_warp + row < M && col < N) {
             const unsigned short* g = H + static_cast<int64_t>(m_warp + row) * ldh + col;
             if (col + 8 <= N) {
-                q = *reinterpret_cast<const uint4*>(g);
+                q[i] = *reinterpret_cast<const uint4*>(g);
             } else {
                 uint32_t w[4] = {0, 0, 0, 0};
 #pragma unroll
                 for (int e = 0; e < 8; ++e)
                     if (col + e < N) w[e >> 1] |= static_cast<uint32_t>(g[e]) << ((e & 1) * 16);
-                q = make_uint4(w[0], w[1], w[2], w[3]);
+                q[i] = make_uint4(w[0], w[1], w[2], w[3]);
             }
         }
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(epi_chunk_addr(buf, row, c)), "r"(q.x), "r"(q.y), "r"(q.z), "r"(q.w) : "memory");
+    }
+}
+// registers ("line" pattern) -> buffer -> registers (one row per lane, fp32)
+__device__ __forceinline__ void staged_load32_finish(uint32_t buf, const uint4 (&q)[4], float (&v)[32], int lane) {
+    const int c = lane & 3;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = 8 * i + (lane >> 2);
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(epi_chunk_addr(buf, row, c)), "r"(q[i].x), "r"(q[i].y), "r"(q[i].z), "r"(q[i].w) : "memory");
     }
     __syncwarp();
 #pragma unroll
     for (int cc = 0; cc < 4; ++cc) {
-        uint4 q;
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w) : "r"(epi_chunk_addr(buf, lane, cc)));
-        v[8 * cc + 0] = bf16_lo(q.x); v[8 * cc + 1] = bf16_hi(q.x);
-        v[8 * cc + 2] = bf16_lo(q.y); v[8 * cc + 3] = bf16_hi(q.y);
-        v[8 * cc + 4] = bf16_lo(q.z); v[8 * cc + 5] = bf16_hi(q.z);
-        v[8 * cc + 6] = bf16_lo(q.w); v[8 * cc + 7] = bf16_hi(q.w);
+        uint4 t;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(t.x), "=r"(t.y), "=r"(t.z), "=r"(t.w) : "r"(epi_chunk_addr(buf, lane, cc)));
+        v[8 * cc + 0] = bf16_lo(t.x); v[8 * cc + 1] = bf16_hi(t.x);
+        v[8 * cc + 2] = bf16_lo(t.y); v[8 * cc + 3] = bf16_hi(t.y);
+        v[8 * cc + 4] = bf16_lo(t.z); v[8 * cc + 5] = bf16_hi(t.z);
+        v[8 * cc + 6] = bf16_lo(t.w); v[8 * cc + 7] = bf16_hi(t.w);
     }
     __syncwarp();
 }
@@ -638,6 +647,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1u;
+            // saved activations of the derivative epilogues: first chunk requested before the accumulator is ready
+            const bool need_h = Q.epi >= EPI_DGELU_ERF;
+            const bool need_hb = Q.epi == EPI_DSWIGLU;
+            const unsigned short* Hp = static_cast<const unsigned short*>(Q.H);
+            const unsigned short* Hbp = static_cast<const unsigned short*>(Q.Hb);
+            uint4 hq[4], hbq[4];
+            if (need_h) staged_load32_issue(Hp, Q.ldh, m_warp, n0 + half * 128, Q.M, Q.N, hq, lane);
+            if (need_hb) staged_load32_issue(Hbp, Q.ldh, m_warp, n0 + half * 128, Q.M, Q.N, hbq, lane);
             if (!(ok = mbar_wait<PAIR>(tfull_bar(acc), acc_phase, abort_flag, 4, P.status))) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
@@ -717,7 +734,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         emit(Q.C2, n, nv, v, false);
                     } else if (epi == EPI_DGELU_ERF || epi == EPI_DGELU_TANH) {
                         float h[32];
-                        staged_load32(buf_in, static_cast<const unsigned short*>(Q.H), Q.ldh, m_warp, n, Q.M, Q.N, h, lane);
+                        staged_load32_finish(buf_in, hq, h, lane);
+                        if (c < 3) staged_load32_issue(Hp, Q.ldh, m_warp, n + 32, Q.M, Q.N, hq, lane);
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             if (epi != EPI_DGELU_ERF) v[i] *= dgelu_tanh(h[i]);
@@ -725,8 +743,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         emit(Q.C, n, nv, v, false);
                     } else {  // EPI_DSWIGLU
                         float hg[32], hu[32];
-                        staged_load32(buf_in, static_cast<const unsigned short*>(Q.H), Q.ldh, m_warp, n, Q.M, Q.N, hg, lane);
-                        staged_load32(buf_in, static_cast<const unsigned short*>(Q.Hb), Q.ldh, m_warp, n, Q.M, Q.N, hu, lane);
+                        staged_load32_finish(buf_in, hq, hg, lane);
+                        staged_load32_finish(buf_in, hbq, hu, lane);
+                        if (c < 3) {
+                            staged_load32_issue(Hp, Q.ldh, m_warp, n + 32, Q.M, Q.N, hq, lane);
+                            staged_load32_issue(Hbp, Q.ldh, m_warp, n + 32, Q.M, Q.N, hbq, lane);
+                        }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
                             const float s = sigmoidf_(hg[i]);
