@@ -55,6 +55,7 @@ struct DevProblem {
     int32_t n_per_tile;          // output columns per tile: 256, or 128 hidden units for EPI_SWIGLU
     int32_t half1_n_off;         // n-coordinate of B half 1 relative to half 0
     int32_t epi;
+    int32_t k_off[2];            // first contraction index of each segment
     uint8_t a_mn[2], b_mn[2];
     uint8_t map_a[2], map_b[2][2];
     uint8_t out_f32, accumulate, bias_f32, pad_[5];
@@ -535,7 +536,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
                 for (int kb = 0; kb < Q.kblocks; ++kb) {
                     const int seg = kb >= Q.kblocks0 ? 1 : 0;
-                    const int k0 = (seg ? kb - Q.kblocks0 : kb) * BK;
+                    const int k0 = (seg ? kb - Q.kblocks0 : kb) * BK + Q.k_off[seg];
                     if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
                     const uint32_t a_dst = sA + stage * kAStage, b_dst = sB + stage * kBLocal;
                     const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
@@ -932,21 +933,25 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
         Q.ldc = op.ldc; Q.ldh = op.ldh;
         for (int s = 0; s < op.n_kseg; ++s) {
             const KSegment& ks = op.seg[s];
-            if (ks.K < 1) return ECOSPA_ERR_INVALID;
-            // stored shapes must match the logical (M, N, K)
+            if (ks.K < 1 || ks.k_begin < 0 || ks.k_begin % BK) return ECOSPA_ERR_INVALID;
+            // stored shapes must cover the logical (M, N, [k_begin, k_begin + K))
+            const int64_t k_end = ks.k_begin + ks.K;
             const Stored& a = ks.a;
-            if (ks.a_mn ? (a.rows != ks.K || a.cols != op.M) : (a.rows != op.M || a.cols != ks.K)) return ECOSPA_ERR_INVALID;
+            // a range that stops before the end of the stored tensor must end on a k-block boundary
+            if (k_end < (ks.a_mn ? a.rows : a.cols) && ks.K % BK) return ECOSPA_ERR_INVALID;
+            if (ks.a_mn ? (a.rows < k_end || a.cols != op.M) : (a.rows != op.M || a.cols < k_end)) return ECOSPA_ERR_INVALID;
             const int mi = oi * kMapsPerOp;
             if ((st = encode_map(&gp.maps[mi + s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
             Q.map_a[s] = static_cast<uint8_t>(mi + s);
             for (int h = 0; h < 2; ++h) {
                 const Stored& b = (swiglu && h == 1) ? ks.b[1] : ks.b[0];
-                if (ks.b_mn ? (b.rows != ks.K || b.cols != op.N) : (b.rows != op.N || b.cols != ks.K)) return ECOSPA_ERR_INVALID;
+                if (ks.b_mn ? (b.rows < k_end || b.cols != op.N) : (b.rows != op.N || b.cols < k_end)) return ECOSPA_ERR_INVALID;
                 if ((st = encode_map(&gp.maps[mi + 2 + 2 * s + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
                 Q.map_b[s][h] = static_cast<uint8_t>(mi + 2 + 2 * s + h);
             }
             Q.a_mn[s] = ks.a_mn;
             Q.b_mn[s] = ks.b_mn;
+            Q.k_off[s] = static_cast<int32_t>(ks.k_begin);
             const int32_t kb = static_cast<int32_t>(ceil_div(ks.K, BK));
             if (s == 0) Q.kblocks0 = kb;
             Q.kblocks += kb;

@@ -32,7 +32,8 @@ struct KSegment {
     Stored a;
     Stored b[2];
     bool a_mn = false, b_mn = false;
-    int64_t K = 0;
+    int64_t K = 0;        // length of this segment's contraction
+    int64_t k_begin = 0;  // first contraction index used (multiple of 64): lets several ops split one K range
 };
 
 struct GemmOp {
@@ -53,7 +54,7 @@ struct GemmOp {
     int64_t ldh = 0;
 };
 
-constexpr int kMaxGemmOps = 4;
+constexpr int kMaxGemmOps = 16;
 
 // Enqueues one persistent launch that computes every op (tiles of the ops with the longest
 // contraction are scheduled first).  Operands must be 16-byte aligned with 16-byte pitches.

@@ -127,6 +127,31 @@ __global__ void __launch_bounds__(kThreads) colsum_final_kernel(const __grid_con
     else static_cast<__nv_bfloat16*>(J.out)[c] = __float2bfloat16_rn(s);
 }
 
+// out[r][c] = sum over s of partial[s][r][c]  (split-K partial products, summed in split order)
+__global__ void __launch_bounds__(kThreads) splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t rows,
+                                                                 int64_t cols, int64_t ldp, void* out, int64_t ld_out,
+                                                                 int out_f32) {
+    const int64_t per_row = (cols + 3) / 4;
+    const int64_t total = rows * per_row;
+    const int64_t plane = rows * ldp;
+    for (int64_t i = blockIdx.x * static_cast<int64_t>(kThreads) + threadIdx.x; i < total;
+         i += static_cast<int64_t>(gridDim.x) * kThreads) {
+        const int64_t r = i / per_row, c = (i % per_row) * 4;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int s2 = 0; s2 < splits; ++s2) {
+            const float4 v = *reinterpret_cast<const float4*>(partial + s2 * plane + r * ldp + c);
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+        for (int e = 0; e < 4; ++e) {
+            if (c + e < cols) {
+                if (out_f32) static_cast<float*>(out)[r * ld_out + c + e] = a[e];
+                else static_cast<__nv_bfloat16*>(out)[r * ld_out + c + e] = __float2bfloat16_rn(a[e]);
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // workspace bump allocator and operand staging
 // ------------------------------------------------------------------------------------------------
@@ -270,16 +295,80 @@ GemmOp proj_op(const Stored& X, const Stored& W, int64_t T, int64_t d_m, int64_t
     op.bias = bias; op.bias_f32 = dtype == ECOSPA_F32;
     return op;
 }
-// dW (rows_out x cols_out) = Xs^T dYs  with Xs stored T x rows_out and dYs stored T x cols_out
-GemmOp wgrad_op(const Stored& Xs, const Stored& dYs, int64_t rows_out, int64_t cols_out, int64_t T, void* out, int64_t ld_out, int dtype) {
+// Weight gradients contract over the T tokens and have few output tiles, so on their own they would keep
+// most SMs idle behind one long tile.  The token range is therefore cut into `splits` ranges computed as
+// separate ops of the same launch into fp32 partial buffers, which splitk_reduce_kernel adds up in order.
+int wgrad_splits(int64_t rows_out, int64_t cols_out, int64_t T) {
+    const int64_t tiles = ceil_div(rows_out, 256) * ceil_div(cols_out, 256);
+    int64_t s = 74 / tiles;                       // aim at one wave of CTA pairs
+    if (s < 3) s = 1;                             // a 2-way split does not pay for its reduction pass
+    s = std::min<int64_t>(s, T / 1024);            // at least 16 k-blocks per range
+    s = std::min<int64_t>(s, 6);
+    return static_cast<int>(std::max<int64_t>(s, 1));
+}
+size_t wgrad_need(int64_t rows_out, int64_t cols_out, int64_t T) {
+    const int S = wgrad_splits(rows_out, cols_out, T);
+    return S > 1 ? arena_need(static_cast<size_t>(S) * rows_out * round_up(cols_out, 4) * 4) : 0;
+}
+struct PendingReduce {
+    const float* partial = nullptr;
+    int splits = 0;
+    int64_t rows = 0, cols = 0, ldp = 0, ld_out = 0;
+    void* out = nullptr;
+};
+// dW (rows_out x cols_out) = Xs^T dYs  with Xs stored T x rows_out and dYs stored T x cols_out.
+// Appends 1 or `splits` ops to ops[n_ops...] and returns the new op count.  `reserve` = ops the caller
+// still has to append after this one; the split count is reduced so that everything fits kMaxGemmOps.
+int add_wgrad(Ctx& cx, GemmOp* ops, int n_ops, const Stored& Xs, const Stored& dYs, int64_t rows_out, int64_t cols_out,
+              int64_t T, void* out, int64_t ld_out, PendingReduce* red, int reserve) {
     GemmOp op;
     op.M = rows_out; op.N = cols_out; op.n_kseg = 1;
     op.seg[0].a = Xs; op.seg[0].a_mn = true;
     op.seg[0].b[0] = dYs; op.seg[0].b_mn = true;
-    op.seg[0].K = T;
     op.epi = EPI_STORE;
-    op.C = out; op.ldc = ld_out; op.out_f32 = dtype == ECOSPA_F32;
-    return op;
+    int S = wgrad_splits(rows_out, cols_out, T);
+    S = std::max(1, std::min(S, kMaxGemmOps - n_ops - reserve));
+    if (cx.st != ECOSPA_OK) return n_ops;
+    if (n_ops + 1 + reserve > kMaxGemmOps) {
+        cx.st = ECOSPA_ERR_INVALID;
+        return n_ops;
+    }
+    if (S == 1) {
+        op.seg[0].K = T;
+        op.C = out; op.ldc = ld_out; op.out_f32 = cx.dtype == ECOSPA_F32;
+        ops[n_ops++] = op;
+        return n_ops;
+    }
+    const int64_t ldp = round_up(cols_out, 4);
+    float* partial = static_cast<float*>(cx.arena.take(static_cast<size_t>(S) * rows_out * ldp * 4));
+    if (!partial) {
+        cx.st = ECOSPA_ERR_WORKSPACE;
+        return n_ops;
+    }
+    const int64_t per = round_up(ceil_div(T, S), 64);
+    int used = 0;
+    for (int i = 0; i < S; ++i) {
+        const int64_t k0 = i * per;
+        if (k0 >= T) break;
+        op.seg[0].k_begin = k0;
+        op.seg[0].K = std::min<int64_t>(per, T - k0);
+        op.C = partial + static_cast<int64_t>(i) * rows_out * ldp;
+        op.ldc = ldp;
+        op.out_f32 = true;
+        ops[n_ops++] = op;
+        ++used;
+    }
+    red->partial = partial; red->splits = used; red->rows = rows_out; red->cols = cols_out; red->ldp = ldp;
+    red->out = out; red->ld_out = ld_out;
+    return n_ops;
+}
+void run_reduce(Ctx& cx, const PendingReduce& r) {
+    if (cx.st != ECOSPA_OK || r.splits == 0) return;
+    const int64_t total = r.rows * ((r.cols + 3) / 4);
+    const int grid = static_cast<int>(std::min<int64_t>(ceil_div(total, kThreads), 148 * 8));
+    splitk_reduce_kernel<<<grid, kThreads, 0, cx.stream>>>(r.partial, r.splits, r.rows, r.cols, r.ldp, r.out, r.ld_out,
+                                                           cx.dtype == ECOSPA_F32);
+    cx.st = check_launch("splitk_reduce_kernel");
 }
 
 }  // namespace
@@ -291,13 +380,13 @@ using namespace ecospa;
 extern "C" size_t ecospa_proj_workspace_bytes(int64_t T, int64_t d_m, int64_t n, int32_t dtype) {
     // worst case over the qk / vo calls: staged X, Ctx, upstream grads, weights, and the column-sum partials
     return staged(dtype, T, d_m) * 2 + staged(dtype, d_m, n) * 2 + staged(dtype, n, d_m) + staged(dtype, T, n) * 3 +
-           colsum_need(T, n) * 2 + colsum_need(T, d_m) + 1024;
+           colsum_need(T, n) * 2 + colsum_need(T, d_m) + wgrad_need(d_m, n, T) * 2 + wgrad_need(n, d_m, T) + 1024;
 }
 
 extern "C" size_t ecospa_ffn_workspace_bytes(int64_t T, int64_t d_m, int64_t k, int32_t act, int32_t dtype) {
     const int nw = act == ECOSPA_ACT_SWIGLU ? 2 : 1;
     return staged(dtype, T, d_m) * 2 + staged(dtype, d_m, k) * nw + staged(dtype, k, d_m) + scratch(T, k) * nw +
-           colsum_need(T, k) + colsum_need(T, d_m) + 1024;
+           colsum_need(T, k) + colsum_need(T, d_m) + wgrad_need(d_m, k, T) * nw + wgrad_need(k, d_m, T) + 1024;
 }
 
 extern "C" ecospa_status_t ecospa_coupled_qk_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m,
@@ -343,10 +432,12 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
         Wk = weight_bf16(cx, wk_c, d_m, n);
     }
     if (cx.st != ECOSPA_OK) return cx.st;
-    GemmOp ops[3];
+    GemmOp ops[kMaxGemmOps];
+    PendingReduce red[2];
     int n_ops = 0;
-    ops[n_ops++] = wgrad_op(Xs, dQs, d_m, n, T, dWq_c, ld_dw, cx.dtype);
-    if (wk_c) ops[n_ops++] = wgrad_op(Xs, dKs, d_m, n, T, dWk_c, ld_dw, cx.dtype);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n, T, dWq_c, ld_dw, &red[0], wk_c ? 2 : 1);
+    if (wk_c) n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n, T, dWk_c, ld_dw, &red[1], 1);
+    if (cx.st != ECOSPA_OK) return cx.st;
     // dX = dQ W_Q^T (+ dK W_K^T): weights stored d_m x n are K-major B operands here
     GemmOp& dx = ops[n_ops++];
     dx.M = T; dx.N = d_m; dx.n_kseg = wk_c ? 2 : 1;
@@ -356,6 +447,8 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
+    run_reduce(cx, red[0]);
+    run_reduce(cx, red[1]);
     colsum(cx, dQs, dbq_c, dKs, wk_c ? dbk_c : nullptr);
     return cx.st;
 }
@@ -407,21 +500,26 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     const Stored Wv = weight_bf16(cx, wv_c, d_m, n);
     const Stored Wo = weight_bf16(cx, wo_c, d_m, n);
     if (cx.st != ECOSPA_OK) return cx.st;
-    GemmOp ops[4];
+    GemmOp ops[kMaxGemmOps];
+    PendingReduce red[2];
+    int n_ops = 0;
     // dW_O (n x d_m) = Ctx^T dOut ; dW_V (d_m x n) = X^T dV
-    ops[0] = wgrad_op(Cs, dOs, n, d_m, T, dWo_c, ld_dwo, cx.dtype);
-    ops[1] = wgrad_op(Xs, dVs, d_m, n, T, dWv_c, ld_dwv, cx.dtype);
+    n_ops = add_wgrad(cx, ops, n_ops, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red[0], 3);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n, T, dWv_c, ld_dwv, &red[1], 2);
+    if (cx.st != ECOSPA_OK) return cx.st;
     // dCtx (T x n) = dOut W_O^T : W_O stored n x d_m = [N][K]
-    GemmOp& dc = ops[2];
+    GemmOp& dc = ops[n_ops++];
     dc.M = T; dc.N = n; dc.n_kseg = 1;
     dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].K = d_m;
     dc.epi = EPI_STORE; dc.C = dCtx; dc.ldc = ld_dctx; dc.out_f32 = f32;
     // dX (T x d_m) = dV W_V^T : W_V stored d_m x n = [N][K]
-    GemmOp& dx = ops[3];
+    GemmOp& dx = ops[n_ops++];
     dx.M = T; dx.N = d_m; dx.n_kseg = 1;
     dx.seg[0].a = dVs; dx.seg[0].b[0] = Wv; dx.seg[0].K = n;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
-    if ((st = launch_grouped_gemm(ops, 4, cx.stream)) != ECOSPA_OK) return st;
+    if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
+    run_reduce(cx, red[0]);
+    run_reduce(cx, red[1]);
     colsum(cx, dVs, dbv_c, dOs, dbo);
     return cx.st;
 }
@@ -508,11 +606,13 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     da.H = H; da.Hb = Hb; da.ldh = ld_h;
     if ((st = launch_grouped_gemm(&da, 1, cx.stream)) != ECOSPA_OK) return st;
 
-    GemmOp ops[4];
+    GemmOp ops[kMaxGemmOps];
+    PendingReduce red[3];
     int n_ops = 0;
-    ops[n_ops++] = wgrad_op(As, dYs, k, d_m, T, dW2_c, ld_dw2, cx.dtype);          // dW_2 (k x d_m) = A^T dY
-    ops[n_ops++] = wgrad_op(Xs, dH, d_m, k, T, dW1_c, ld_dw1, cx.dtype);           // dW_1 (d_m x k) = X^T dH
-    if (sw) ops[n_ops++] = wgrad_op(Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, cx.dtype); // dW_up = X^T dH_up
+    n_ops = add_wgrad(cx, ops, n_ops, As, dYs, k, d_m, T, dW2_c, ld_dw2, &red[0], sw ? 3 : 2);          // dW_2 (k x d_m) = A^T dY
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1);           // dW_1 (d_m x k) = X^T dH
+    if (sw) n_ops = add_wgrad(cx, ops, n_ops, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1); // dW_up = X^T dH_up
+    if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& dx = ops[n_ops++];                                                    // dX = dH W_1^T (+ dH_up W_up^T)
     dx.M = T; dx.N = d_m; dx.n_kseg = sw ? 2 : 1;
     dx.seg[0].a = dH; dx.seg[0].b[0] = W1; dx.seg[0].K = k;
@@ -521,6 +621,7 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
+    for (int i = 0; i < 3; ++i) run_reduce(cx, red[i]);
     colsum(cx, dYs, db2, dH, sw ? nullptr : db1_c);
     return cx.st;
 }
