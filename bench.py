@@ -252,6 +252,9 @@ def run_gpu(args):
         dist.barrier()
     dev = torch.device("cuda", local)
     wl = WL.WORKLOADS[args.workload]
+    if args.layers:
+        import dataclasses
+        wl = dataclasses.replace(wl, n_layers=args.layers)   # smaller model of the same shape (profiler captures)
     m = Model(wl, args.sparsity, dev)
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
@@ -458,6 +461,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="gpt2m")
     ap.add_argument("--sparsity", type=float, default=0.5)
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small cases for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="issue every launch from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
