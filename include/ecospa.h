@@ -240,6 +240,34 @@ ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, const void* Ct
                                       int64_t ld_dwv, void* dWo_c, int64_t ld_dwo, void* dbv_c, void* dbo,
                                       void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same products grouped the way a training step meets them (one launch each):
+ *   ecospa_coupled_qkv_fwd   Q^c, K^c (n_qk columns) and V^c (n_vo columns) from one X; the QK and VO pairs of
+ *                            a block may keep different numbers of columns.
+ *   ecospa_coupled_vo_bwd_o  what follows from dOut alone: dCtx = dOut W_O^cT (input of the caller's attention
+ *                            backward), dW_O^c = Ctx^T dOut, dbo.
+ *   ecospa_coupled_qkv_bwd   what follows once dQ^c, dK^c, dV^c are known: dW_Q^c, dW_K^c, dW_V^c, the three bias
+ *                            gradients and dX = dQ^c W_Q^cT + dK^c W_K^cT + dV^c W_V^cT (added to dX if accumulate_dX).
+ *   ecospa_coupled_vo_bwd_v  the V part of the above on its own.
+ * Arguments as in the calls above (ld_dwqk / ld_dwv: pitches of the weight-gradient outputs). */
+ecospa_status_t ecospa_coupled_qkv_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, const ecospa_mat_t* wq_c,
+                                       const ecospa_mat_t* wk_c, const ecospa_mat_t* wv_c, int64_t n_qk, int64_t n_vo,
+                                       const void* bq_c, const void* bk_c, const void* bv_c, void* Qc, void* Kc, void* Vc,
+                                       int64_t ld_qk, int64_t ld_v, void* workspace, size_t workspace_bytes, void* stream);
+ecospa_status_t ecospa_coupled_qkv_bwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, const ecospa_mat_t* wq_c,
+                                       const ecospa_mat_t* wk_c, const ecospa_mat_t* wv_c, int64_t n_qk, int64_t n_vo,
+                                       const void* dQc, const void* dKc, const void* dVc, int64_t ld_dqk, int64_t ld_dv,
+                                       void* dX, int64_t ld_dx, int32_t accumulate_dX, void* dWq_c, void* dWk_c,
+                                       void* dWv_c, int64_t ld_dwqk, int64_t ld_dwv, void* dbq_c, void* dbk_c,
+                                       void* dbv_c, void* workspace, size_t workspace_bytes, void* stream);
+ecospa_status_t ecospa_coupled_vo_bwd_o(const void* Ctx, int64_t ld_ctx, int64_t T, int64_t d_m,
+                                        const ecospa_mat_t* wo_c, int64_t n, const void* dOut, int64_t ld_dout,
+                                        void* dCtx, int64_t ld_dctx, void* dWo_c, int64_t ld_dwo, void* dbo,
+                                        void* workspace, size_t workspace_bytes, void* stream);
+ecospa_status_t ecospa_coupled_vo_bwd_v(const void* X, int64_t ldx, int64_t T, int64_t d_m, const ecospa_mat_t* wv_c,
+                                        int64_t n, const void* dVc, int64_t ld_dv, void* dX, int64_t ld_dx,
+                                        int32_t accumulate_dX, void* dWv_c, int64_t ld_dwv, void* dbv_c, void* workspace,
+                                        size_t workspace_bytes, void* stream);
+
 /* FFN on a compacted pair with k hidden units (Eq. 3):
  *   GELU   : H = X W_1^c + b_1^c, A = GELU(H), Y = A W_2^c + b_2
  *   SwiGLU : H = X W_gate^c, Hb = X W_up^c, A = silu(H) (.) Hb, Y = A W_2^c        (w1_c = gate, w1b_c = up)

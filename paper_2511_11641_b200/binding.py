@@ -229,6 +229,19 @@ _LAYER_SIGS = {
                                          C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
                                          C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_int64,
                                          C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_qkv_fwd": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_qkv_bwd": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64,
+                                         C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int64,
+                                         C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_vo_bwd_o": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p,
+                                          C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p,
+                                          C.c_void_p, C.c_size_t, C.c_void_p]),
+    "ecospa_coupled_vo_bwd_v": (C.c_int, [C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p,
+                                          C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_int64, C.c_void_p,
+                                          C.c_void_p, C.c_size_t, C.c_void_p]),
     "ecospa_device_status": (C.c_int, [C.c_void_p, C.c_void_p]),
 }
 _sigs_done = False
@@ -316,6 +329,50 @@ def ecospa_coupled_vo_bwd(X, Ctx, wv_c, wo_c, n: int, dVc, dOut, dX, dCtx, dWv_c
                                         dX.stride(0), int(accumulate_dX), dCtx.data_ptr(), dCtx.stride(0), dWv_c.data_ptr(),
                                         dWv_c.stride(0), dWo_c.data_ptr(), dWo_c.stride(0), _ptr(dbv_c), _ptr(dbo), wp, wb,
                                         _stream(stream)), "ecospa_coupled_vo_bwd")
+
+
+def ecospa_coupled_qkv_fwd(X, wq_c, wk_c, wv_c, n_qk: int, n_vo: int, Qc, Kc, Vc, bq_c=None, bk_c=None, bv_c=None,
+                           workspace=None, stream=None) -> None:
+    T, d_m = X.shape
+    mq, mk, mv = mat(wq_c, SHARED_COLS), mat(wk_c, SHARED_COLS), mat(wv_c, SHARED_COLS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_qkv_fwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), _ref(mv), n_qk, n_vo,
+                                         _ptr(bq_c), _ptr(bk_c), _ptr(bv_c), Qc.data_ptr(), Kc.data_ptr(), Vc.data_ptr(),
+                                         Qc.stride(0), Vc.stride(0), wp, wb, _stream(stream)), "ecospa_coupled_qkv_fwd")
+
+
+def ecospa_coupled_qkv_bwd(X, wq_c, wk_c, wv_c, n_qk: int, n_vo: int, dQc, dKc, dVc, dX, dWq_c, dWk_c, dWv_c,
+                           dbq_c=None, dbk_c=None, dbv_c=None, accumulate_dX: bool = False, workspace=None,
+                           stream=None) -> None:
+    T, d_m = X.shape
+    mq, mk, mv = mat(wq_c, SHARED_COLS), mat(wk_c, SHARED_COLS), mat(wv_c, SHARED_COLS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_qkv_bwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), _ref(mv), n_qk, n_vo,
+                                         dQc.data_ptr(), dKc.data_ptr(), dVc.data_ptr(), dQc.stride(0), dVc.stride(0),
+                                         dX.data_ptr(), dX.stride(0), int(accumulate_dX), dWq_c.data_ptr(),
+                                         dWk_c.data_ptr(), dWv_c.data_ptr(), dWq_c.stride(0), dWv_c.stride(0),
+                                         _ptr(dbq_c), _ptr(dbk_c), _ptr(dbv_c), wp, wb, _stream(stream)),
+           "ecospa_coupled_qkv_bwd")
+
+
+def ecospa_coupled_vo_bwd_o(Ctx, wo_c, n: int, dOut, dCtx, dWo_c, dbo=None, workspace=None, stream=None) -> None:
+    T = Ctx.shape[0]
+    d_m = wo_c.shape[1]
+    mo = mat(wo_c, SHARED_ROWS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_vo_bwd_o")(Ctx.data_ptr(), Ctx.stride(0), T, d_m, _ref(mo), n, dOut.data_ptr(),
+                                          dOut.stride(0), dCtx.data_ptr(), dCtx.stride(0), dWo_c.data_ptr(),
+                                          dWo_c.stride(0), _ptr(dbo), wp, wb, _stream(stream)), "ecospa_coupled_vo_bwd_o")
+
+
+def ecospa_coupled_vo_bwd_v(X, wv_c, n: int, dVc, dX, dWv_c, dbv_c=None, accumulate_dX: bool = False, workspace=None,
+                            stream=None) -> None:
+    T, d_m = X.shape
+    mv = mat(wv_c, SHARED_COLS)
+    wp, wb = _ws(workspace)
+    _check(_fn("ecospa_coupled_vo_bwd_v")(X.data_ptr(), X.stride(0), T, d_m, _ref(mv), n, dVc.data_ptr(), dVc.stride(0),
+                                          dX.data_ptr(), dX.stride(0), int(accumulate_dX), dWv_c.data_ptr(),
+                                          dWv_c.stride(0), _ptr(dbv_c), wp, wb, _stream(stream)), "ecospa_coupled_vo_bwd_v")
 
 
 def ecospa_coupled_ffn_fwd(X, act: int, w1_c, w2_c, k: int, Y, H, A, w1b_c=None, Hb=None, b1_c=None, b2=None,

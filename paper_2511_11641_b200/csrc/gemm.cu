@@ -42,7 +42,8 @@ constexpr int kAtomBytes = 64 * 64 * 2;     // one 64x64 bf16 swizzle atom of an
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
-constexpr int kMapsPerOp = 6;              // 2 A + 4 B operand maps
+constexpr int kMaxSeg = 3;
+constexpr int kMapsPerOp = 3 * kMaxSeg;     // per K segment: one A map and two B (half) maps
 constexpr int kEpiSlotBytes = 32 * 32 * 2;  // one 32-row x 32-column bf16 store box
 constexpr int kEpiBytes = kEpiWarps * 2 * kEpiSlotBytes;
 constexpr int kSmemBytes = kRingBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
@@ -50,14 +51,16 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 
 struct DevProblem {
     int32_t M, N;
-    int32_t kblocks0, kblocks;   // k-blocks of segment 0, of both segments
+    int32_t kb_end[kMaxSeg];     // cumulative k-blocks: segment s covers [kb_end[s-1], kb_end[s])
+    int32_t kblocks;             // k-blocks of all segments
     int32_t tiles_m, tiles_n, tile_start;
     int32_t n_per_tile;          // output columns per tile: 256, or 128 hidden units for EPI_SWIGLU
     int32_t half1_n_off;         // n-coordinate of B half 1 relative to half 0
     int32_t epi;
-    int32_t k_off[2];            // first contraction index of each segment
-    uint8_t a_mn[2], b_mn[2];
-    uint8_t map_a[2], map_b[2][2];
+    int32_t k_off[kMaxSeg];      // first contraction index of each segment
+    uint8_t a_mn[kMaxSeg], b_mn[kMaxSeg];
+    uint8_t map_a[kMaxSeg], map_b[kMaxSeg][2];
+    uint8_t pad2_[1];
     uint8_t out_f32, accumulate, bias_f32, pad_[5];
     void* C;
     void* C2;
@@ -535,8 +538,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 const int m0 = (local % Q.tiles_m) * kTileM + static_cast<int>(cta_rank) * BM;
                 const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
                 for (int kb = 0; kb < Q.kblocks; ++kb) {
-                    const int seg = kb >= Q.kblocks0 ? 1 : 0;
-                    const int k0 = (seg ? kb - Q.kblocks0 : kb) * BK + Q.k_off[seg];
+                    const int seg = (kb >= Q.kb_end[0] ? 1 : 0) + (kb >= Q.kb_end[1] ? 1 : 0);
+                    const int k0 = (kb - (seg ? Q.kb_end[seg - 1] : 0)) * BK + Q.k_off[seg];
                     if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
                     const uint32_t a_dst = sA + stage * kAStage, b_dst = sB + stage * kBLocal;
                     const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
@@ -598,7 +601,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < Q.kblocks; ++kb) {
-                    const int seg = kb >= Q.kblocks0 ? 1 : 0;
+                    const int seg = (kb >= Q.kb_end[0] ? 1 : 0) + (kb >= Q.kb_end[1] ? 1 : 0);
                     if (!(ok = mbar_wait<PAIR>(full_bar(stage), phase, abort_flag, 3, P.status))) break;
                     tc_fence_after();
                     const uint32_t a_mn = Q.a_mn[seg], b_mn = Q.b_mn[seg];
@@ -906,7 +909,7 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
         const GemmOp& op = ops[order[oi]];
         DevProblem& Q = gp.prob[oi];
         std::memset(&Q, 0, sizeof(Q));
-        if (op.M < 1 || op.N < 1 || op.n_kseg < 1 || op.n_kseg > 2 || !op.C || op.ldc < 1) return ECOSPA_ERR_INVALID;
+        if (op.M < 1 || op.N < 1 || op.n_kseg < 1 || op.n_kseg > kMaxSeg || !op.C || op.ldc < 1) return ECOSPA_ERR_INVALID;
         if (op.M > INT32_MAX || op.N > INT32_MAX) return ECOSPA_ERR_INVALID;
         const bool swiglu = op.epi == EPI_SWIGLU;
         const int out_eb = op.out_f32 ? 4 : 2;
@@ -941,21 +944,21 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
             if (k_end < (ks.a_mn ? a.rows : a.cols) && ks.K % BK) return ECOSPA_ERR_INVALID;
             if (ks.a_mn ? (a.rows < k_end || a.cols != op.M) : (a.rows != op.M || a.cols < k_end)) return ECOSPA_ERR_INVALID;
             const int mi = oi * kMapsPerOp;
-            if ((st = encode_map(&gp.maps[mi + s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
-            Q.map_a[s] = static_cast<uint8_t>(mi + s);
+            if ((st = encode_map(&gp.maps[mi + 3 * s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
+            Q.map_a[s] = static_cast<uint8_t>(mi + 3 * s);
             for (int h = 0; h < 2; ++h) {
                 const Stored& b = (swiglu && h == 1) ? ks.b[1] : ks.b[0];
                 if (ks.b_mn ? (b.rows < k_end || b.cols != op.N) : (b.rows != op.N || b.cols < k_end)) return ECOSPA_ERR_INVALID;
-                if ((st = encode_map(&gp.maps[mi + 2 + 2 * s + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
-                Q.map_b[s][h] = static_cast<uint8_t>(mi + 2 + 2 * s + h);
+                if ((st = encode_map(&gp.maps[mi + 3 * s + 1 + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
+                Q.map_b[s][h] = static_cast<uint8_t>(mi + 3 * s + 1 + h);
             }
             Q.a_mn[s] = ks.a_mn;
             Q.b_mn[s] = ks.b_mn;
             Q.k_off[s] = static_cast<int32_t>(ks.k_begin);
-            const int32_t kb = static_cast<int32_t>(ceil_div(ks.K, BK));
-            if (s == 0) Q.kblocks0 = kb;
-            Q.kblocks += kb;
+            Q.kblocks += static_cast<int32_t>(ceil_div(ks.K, BK));
+            Q.kb_end[s] = Q.kblocks;
         }
+        for (int s2 = op.n_kseg; s2 < kMaxSeg; ++s2) Q.kb_end[s2] = Q.kblocks;
         Q.tiles_m = static_cast<int32_t>(ceil_div(op.M, tile_m));
         Q.tiles_n = static_cast<int32_t>(ceil_div(op.N, Q.n_per_tile));
         Q.tile_start = tiles;

@@ -38,8 +38,8 @@ struct KSegment {
 
 struct GemmOp {
     int64_t M = 0, N = 0;     // output extent (EPI_SWIGLU: N = hidden units)
-    int n_kseg = 1;
-    KSegment seg[2];
+    int n_kseg = 1;           // 1..3 segments accumulated into the same output
+    KSegment seg[3];
     int epi = EPI_STORE;
     void* C = nullptr;
     void* C2 = nullptr;

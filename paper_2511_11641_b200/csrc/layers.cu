@@ -56,16 +56,19 @@ struct ColsumJob {
     int32_t col_tiles, vec_ok;
 };
 struct ColsumParams {
-    ColsumJob job[2];
+    ColsumJob job[3];
     int64_t rows;
     int32_t n_jobs, chunks, out_f32;
 };
 
 __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const __grid_constant__ ColsumParams P) {
     __shared__ float red[32][kSumCols + 1];
-    const int ji = (P.n_jobs > 1 && static_cast<int>(blockIdx.x) >= P.job[0].col_tiles) ? 1 : 0;
+    int ji = 0, ct = blockIdx.x;
+    while (ji + 1 < P.n_jobs && ct >= P.job[ji].col_tiles) {
+        ct -= P.job[ji].col_tiles;
+        ++ji;
+    }
     const ColsumJob& J = P.job[ji];
-    const int ct = blockIdx.x - (ji ? P.job[0].col_tiles : 0);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int rowoff = (lane >> 3) + 4 * warp;              // 0..31
     const int64_t c0 = static_cast<int64_t>(ct) * kSumCols + (lane & 7) * 8;
@@ -115,11 +118,11 @@ __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const __grid_c
 __global__ void __launch_bounds__(kThreads) colsum_final_kernel(const __grid_constant__ ColsumParams P) {
     int64_t c = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
     int ji = 0;
-    if (c >= P.job[0].cols) {
-        c -= P.job[0].cols;
-        ji = 1;
-        if (P.n_jobs < 2 || c >= P.job[1].cols) return;
+    while (ji < P.n_jobs && c >= P.job[ji].cols) {
+        c -= P.job[ji].cols;
+        ++ji;
     }
+    if (ji >= P.n_jobs) return;
     const ColsumJob& J = P.job[ji];
     float s = 0.f;
     for (int k = 0; k < P.chunks; ++k) s += J.partial[static_cast<int64_t>(k) * J.cols + c];
@@ -215,14 +218,15 @@ Stored scratch_bf16(Ctx& cx, int64_t rows, int64_t cols) {
     return s;
 }
 
-// out[c] = sum_r M[r][c] for one or two bf16 matrices with the same row count; outputs have the model
+// out[c] = sum_r M[r][c] for up to three bf16 matrices with the same row count; outputs have the model
 // dtype.  A null output skips that matrix.
-void colsum(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), void* out2 = nullptr) {
+void colsum(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), void* out2 = nullptr,
+            const Stored& M3 = Stored(), void* out3 = nullptr) {
     if (cx.st != ECOSPA_OK) return;
     ColsumParams P = {};
-    const Stored* mats[2] = {&M1, &M2};
-    void* outs[2] = {out1, out2};
-    for (int i = 0; i < 2; ++i) {
+    const Stored* mats[3] = {&M1, &M2, &M3};
+    void* outs[3] = {out1, out2, out3};
+    for (int i = 0; i < 3; ++i) {
         if (!outs[i] || !mats[i]->ptr) continue;
         ColsumJob& J = P.job[P.n_jobs++];
         J.M = static_cast<const uint16_t*>(mats[i]->ptr);
@@ -380,7 +384,8 @@ using namespace ecospa;
 extern "C" size_t ecospa_proj_workspace_bytes(int64_t T, int64_t d_m, int64_t n, int32_t dtype) {
     // worst case over the qk / vo calls: staged X, Ctx, upstream grads, weights, and the column-sum partials
     return staged(dtype, T, d_m) * 2 + staged(dtype, d_m, n) * 2 + staged(dtype, n, d_m) + staged(dtype, T, n) * 3 +
-           colsum_need(T, n) * 2 + colsum_need(T, d_m) + wgrad_need(d_m, n, T) * 2 + wgrad_need(n, d_m, T) + 1024;
+           colsum_need(T, n) * 3 + colsum_need(T, d_m) + wgrad_need(d_m, n, T) * 3 + wgrad_need(n, d_m, T) + staged(dtype, d_m, n) +
+           staged(dtype, T, n) + 1024;
 }
 
 extern "C" size_t ecospa_ffn_workspace_bytes(int64_t T, int64_t d_m, int64_t k, int32_t act, int32_t dtype) {
@@ -522,6 +527,112 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     run_reduce(cx, red[1]);
     colsum(cx, dVs, dbv_c, dOs, dbo);
     return cx.st;
+}
+
+// Q^c, K^c and V^c in one launch (the QK and VO pairs of a block read the same X).
+extern "C" ecospa_status_t ecospa_coupled_qkv_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m,
+                                                  const ecospa_mat_t* wq_c, const ecospa_mat_t* wk_c,
+                                                  const ecospa_mat_t* wv_c, int64_t n_qk, int64_t n_vo, const void* bq_c,
+                                                  const void* bk_c, const void* bv_c, void* Qc, void* Kc, void* Vc,
+                                                  int64_t ld_qk, int64_t ld_v, void* workspace, size_t workspace_bytes,
+                                                  void* stream) {
+    if (!wq_c || !wk_c || !wv_c || !Qc || !Kc || !Vc) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, std::min(n_qk, n_vo));
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wk_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wv_c, d_m, n_vo, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
+    GemmOp ops[3];
+    ops[0] = proj_op(Xs, weight_bf16(cx, wq_c, d_m, n_qk), T, d_m, n_qk, bq_c, Qc, ld_qk, cx.dtype);
+    ops[1] = proj_op(Xs, weight_bf16(cx, wk_c, d_m, n_qk), T, d_m, n_qk, bk_c, Kc, ld_qk, cx.dtype);
+    ops[2] = proj_op(Xs, weight_bf16(cx, wv_c, d_m, n_vo), T, d_m, n_vo, bv_c, Vc, ld_v, cx.dtype);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    return launch_grouped_gemm(ops, 3, cx.stream);
+}
+
+// Backward of the three projections in one launch: dW_Q^c, dW_K^c, dW_V^c (split over the tokens when they
+// have few tiles) and dX = dQ W_Q^cT + dK W_K^cT + dV W_V^cT as one product over three K segments.
+extern "C" ecospa_status_t ecospa_coupled_qkv_bwd(const void* X, int64_t ldx, int64_t T, int64_t d_m,
+                                                  const ecospa_mat_t* wq_c, const ecospa_mat_t* wk_c,
+                                                  const ecospa_mat_t* wv_c, int64_t n_qk, int64_t n_vo, const void* dQc,
+                                                  const void* dKc, const void* dVc, int64_t ld_dqk, int64_t ld_dv,
+                                                  void* dX, int64_t ld_dx, int32_t accumulate_dX, void* dWq_c,
+                                                  void* dWk_c, void* dWv_c, int64_t ld_dwqk, int64_t ld_dwv, void* dbq_c,
+                                                  void* dbk_c, void* dbv_c, void* workspace, size_t workspace_bytes,
+                                                  void* stream) {
+    if (!wq_c || !wk_c || !wv_c || !dQc || !dKc || !dVc || !dX || !dWq_c || !dWk_c || !dWv_c) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, std::min(n_qk, n_vo));
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wk_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wv_c, d_m, n_vo, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
+    const Stored dQs = as_bf16(cx, dQc, T, n_qk, ld_dqk);
+    const Stored dKs = as_bf16(cx, dKc, T, n_qk, ld_dqk);
+    const Stored dVs = as_bf16(cx, dVc, T, n_vo, ld_dv);
+    const Stored Wq = weight_bf16(cx, wq_c, d_m, n_qk);
+    const Stored Wk = weight_bf16(cx, wk_c, d_m, n_qk);
+    const Stored Wv = weight_bf16(cx, wv_c, d_m, n_vo);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    GemmOp ops[kMaxGemmOps];
+    PendingReduce red[3];
+    int n_ops = 0;
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n_qk, T, dWq_c, ld_dwqk, &red[0], 3);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n_qk, T, dWk_c, ld_dwqk, &red[1], 2);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n_vo, T, dWv_c, ld_dwv, &red[2], 1);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    GemmOp& dx = ops[n_ops++];
+    dx.M = T; dx.N = d_m; dx.n_kseg = 3;
+    dx.seg[0].a = dQs; dx.seg[0].b[0] = Wq; dx.seg[0].K = n_qk;
+    dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].K = n_qk;
+    dx.seg[2].a = dVs; dx.seg[2].b[0] = Wv; dx.seg[2].K = n_vo;
+    dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = cx.dtype == ECOSPA_F32; dx.accumulate = accumulate_dX != 0;
+    if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
+    for (int i = 0; i < 3; ++i) run_reduce(cx, red[i]);
+    colsum(cx, dQs, dbq_c, dKs, dbk_c, dVs, dbv_c);
+    return cx.st;
+}
+
+// Output-projection half of the VO backward: everything that only needs dOut (dCtx feeds the caller's
+// attention backward, which produces the dV^c that ecospa_coupled_qkv_bwd / _vo_bwd_v consume).
+extern "C" ecospa_status_t ecospa_coupled_vo_bwd_o(const void* Ctxm, int64_t ld_ctx, int64_t T, int64_t d_m,
+                                                   const ecospa_mat_t* wo_c, int64_t n, const void* dOut, int64_t ld_dout,
+                                                   void* dCtx, int64_t ld_dctx, void* dWo_c, int64_t ld_dwo, void* dbo,
+                                                   void* workspace, size_t workspace_bytes, void* stream) {
+    if (!wo_c || !Ctxm || !dOut || !dCtx || !dWo_c) return ECOSPA_ERR_INVALID;
+    Ctx cx;
+    ecospa_status_t st = begin(cx, wo_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
+    if (st != ECOSPA_OK) return st;
+    if ((st = check_weight(wo_c, d_m, n, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    const Stored Cs = as_bf16(cx, Ctxm, T, n, ld_ctx);
+    const Stored dOs = as_bf16(cx, dOut, T, d_m, ld_dout);
+    const Stored Wo = weight_bf16(cx, wo_c, d_m, n);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    GemmOp ops[kMaxGemmOps];
+    PendingReduce red;
+    int n_ops = add_wgrad(cx, ops, 0, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red, 1);   // dW_O (n x d_m) = Ctx^T dOut
+    if (cx.st != ECOSPA_OK) return cx.st;
+    GemmOp& dc = ops[n_ops++];                                                        // dCtx = dOut W_O^T
+    dc.M = T; dc.N = n; dc.n_kseg = 1;
+    dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].K = d_m;
+    dc.epi = EPI_STORE; dc.C = dCtx; dc.ldc = ld_dctx; dc.out_f32 = cx.dtype == ECOSPA_F32;
+    if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
+    run_reduce(cx, red);
+    colsum(cx, dOs, dbo);
+    return cx.st;
+}
+
+// Value-projection half of the VO backward: dW_V^c = X^T dV^c, dX (+)= dV^c W_V^cT, dbv = colsum(dV^c).
+extern "C" ecospa_status_t ecospa_coupled_vo_bwd_v(const void* X, int64_t ldx, int64_t T, int64_t d_m,
+                                                   const ecospa_mat_t* wv_c, int64_t n, const void* dVc, int64_t ld_dv,
+                                                   void* dX, int64_t ld_dx, int32_t accumulate_dX, void* dWv_c,
+                                                   int64_t ld_dwv, void* dbv_c, void* workspace, size_t workspace_bytes,
+                                                   void* stream) {
+    return ecospa_coupled_qk_bwd(X, ldx, T, d_m, wv_c, nullptr, n, dVc, nullptr, ld_dv, dX, ld_dx, accumulate_dX, dWv_c,
+                                 nullptr, ld_dwv, dbv_c, nullptr, workspace, workspace_bytes, stream);
 }
 
 extern "C" ecospa_status_t ecospa_coupled_ffn_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, int32_t act,

@@ -113,6 +113,28 @@ def run_block_full(wl, k_heads, k_ffn, act, T=None, seed=0):
     errs["dCtx"] = rel(dCtx[:, :n], rdCtx); errs["dWo"] = rel(dWo, rdWo.T); errs["dbo"] = rel(dbo, rdbo)
     errs["vo.dX"] = rel(dX, rdXv); errs["dWv"] = rel(dWv[:, :n], rdWv); errs["dbv"] = rel(dbv, rdbv)
 
+    # ---- the same attention-side products through the grouped calls (one launch each)
+    Q2 = torch.empty_like(Q); K2 = torch.empty_like(K); V2 = torch.empty_like(V)
+    B.ecospa_coupled_qkv_fwd(a["x"], d["wq"], d["wk"], d["wv"], n, n, Q2, K2, V2, bq_c=d.get("bq"), bk_c=d.get("bk"),
+                             bv_c=d.get("bv"), workspace=ws)
+    errs["qkv.Q"] = rel(Q2[:, :n], O.proj_fwd(acts["x"], wc["wq"], O.SHARED_COLS, n, bias=wc.get("bq")))
+    errs["qkv.K"] = rel(K2[:, :n], O.proj_fwd(acts["x"], wc["wk"], O.SHARED_COLS, n, bias=wc.get("bk")))
+    errs["qkv.V"] = rel(V2[:, :n], O.proj_fwd(acts["x"], wc["wv"], O.SHARED_COLS, n, bias=wc.get("bv")))
+    dCtx2 = torch.empty_like(dCtx); dWo2 = torch.empty_like(dWo); dbo2 = torch.empty_like(dbo)
+    B.ecospa_coupled_vo_bwd_o(a["ctx"], d["wo"], n, a["dout"], dCtx2, dWo2, dbo2, workspace=ws)
+    errs["vo_o.dCtx"] = rel(dCtx2[:, :n], rdCtx); errs["vo_o.dWo"] = rel(dWo2, rdWo.T); errs["vo_o.dbo"] = rel(dbo2, rdbo)
+    dX3 = torch.empty_like(dX)
+    dWq3 = torch.zeros_like(dWq); dWk3 = torch.zeros_like(dWk); dWv3 = torch.zeros_like(dWv)
+    dbq3 = torch.empty_like(dbq); dbk3 = torch.empty_like(dbk); dbv3 = torch.empty_like(dbv)
+    B.ecospa_coupled_qkv_bwd(a["x"], d["wq"], d["wk"], d["wv"], n, n, a["dq"], a["dk"], a["dv"], dX3, dWq3, dWk3, dWv3,
+                             dbq3, dbk3, dbv3, workspace=ws)
+    errs["qkv.dX"] = rel(dX3, rdX + rdXv)
+    errs["qkv.dWq"] = rel(dWq3[:, :n], rdWq); errs["qkv.dWk"] = rel(dWk3[:, :n], rdWk); errs["qkv.dWv"] = rel(dWv3[:, :n], rdWv)
+    errs["qkv.dbq"] = rel(dbq3, rdbq); errs["qkv.dbk"] = rel(dbk3, rdbk); errs["qkv.dbv"] = rel(dbv3, rdbv)
+    dX4 = torch.empty_like(dX); dWv4 = torch.zeros_like(dWv)
+    B.ecospa_coupled_vo_bwd_v(a["x"], d["wv"], n, a["dv"], dX4, dWv4, workspace=ws)
+    errs["vo_v.dX"] = rel(dX4, rdXv); errs["vo_v.dWv"] = rel(dWv4[:, :n], rdWv)
+
     # ---- FFN
     sw = act == B.ACT_SWIGLU
     buf = L.ffn_buffers(T, wl.d_m, k, act, dt, DEV)
