@@ -544,22 +544,28 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     const uint32_t a_dst = sA + stage * kAStage, b_dst = sB + stage * kBLocal;
                     const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
                     if (PAIR) {
-                        // this CTA's share of the stage, signalled on the leader's barrier
-                        const uint32_t fb = map_to_cta(full_bar(stage), 0);
-                        if (leader) mbar_expect_tx(full_bar(stage), 2 * kStageTx);
+                        // This CTA's share of the stage, completed on the leader's barrier: the leader uses the
+                        // plain form on its own barrier (measurably cheaper), the peer the pair form that may
+                        // signal the other CTA's barrier.
+                        const uint32_t fb = leader ? full_bar(stage) : map_to_cta(full_bar(stage), 0);
+                        if (leader) mbar_expect_tx(fb, 2 * kStageTx);
+                        auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
+                            if (leader) tma_load_2d(dst, map, x, y, fb);
+                            else tma_load_2d_pair(dst, map, x, y, fb);
+                        };
                         if (!Q.a_mn[seg]) {
-                            tma_load_2d_pair(a_dst, ma, k0, m0, fb);
+                            load(a_dst, ma, k0, m0);
                         } else {
-                            tma_load_2d_pair(a_dst, ma, m0, k0, fb);
-                            tma_load_2d_pair(a_dst + kAtomBytes, ma, m0 + 64, k0, fb);
+                            load(a_dst, ma, m0, k0);
+                            load(a_dst + kAtomBytes, ma, m0 + 64, k0);
                         }
                         const CUtensorMap* mb = &P.maps[Q.map_b[seg][cta_rank]];
                         const int nc = n0 + static_cast<int>(cta_rank) * Q.half1_n_off;
                         if (!Q.b_mn[seg]) {
-                            tma_load_2d_pair(b_dst, mb, k0, nc, fb);
+                            load(b_dst, mb, k0, nc);
                         } else {
-                            tma_load_2d_pair(b_dst, mb, nc, k0, fb);
-                            tma_load_2d_pair(b_dst + kAtomBytes, mb, nc + 64, k0, fb);
+                            load(b_dst, mb, nc, k0);
+                            load(b_dst + kAtomBytes, mb, nc + 64, k0);
                         }
                     } else {
                         mbar_expect_tx(full_bar(stage), kStageTx);
