@@ -547,10 +547,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         // This CTA's share of the stage, completed on the leader's barrier: the leader uses the
                         // plain form on its own barrier (measurably cheaper), the peer the pair form that may
                         // signal the other CTA's barrier.
-                        const uint32_t fb = leader ? full_bar(stage) : map_to_cta(full_bar(stage), 0);
-                        if (leader) mbar_expect_tx(fb, 2 * kStageTx);
+                        const uint32_t fb = map_to_cta(full_bar(stage), 0);
+                        if (leader) mbar_expect_tx(full_bar(stage), 2 * kStageTx);
                         auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
-                            if (leader) tma_load_2d(dst, map, x, y, fb);
+                            if (leader) tma_load_2d(dst, map, x, y, full_bar(stage));
                             else tma_load_2d_pair(dst, map, x, y, fb);
                         };
                         if (!Q.a_mn[seg]) {
