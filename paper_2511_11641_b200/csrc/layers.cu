@@ -115,44 +115,57 @@ __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const __grid_c
         }
     }
 }
-__global__ void __launch_bounds__(kThreads) colsum_final_kernel(const __grid_constant__ ColsumParams P) {
-    int64_t c = static_cast<int64_t>(blockIdx.x) * kThreads + threadIdx.x;
-    int ji = 0;
-    while (ji < P.n_jobs && c >= P.job[ji].cols) {
-        c -= P.job[ji].cols;
-        ++ji;
-    }
-    if (ji >= P.n_jobs) return;
-    const ColsumJob& J = P.job[ji];
-    float s = 0.f;
-    for (int k = 0; k < P.chunks; ++k) s += J.partial[static_cast<int64_t>(k) * J.cols + c];
-    if (P.out_f32) static_cast<float*>(J.out)[c] = s;
-    else static_cast<__nv_bfloat16*>(J.out)[c] = __float2bfloat16_rn(s);
-}
-
-// out[r][c] = sum over s of partial[s][r][c]  (split-K partial products, summed in split order)
-__global__ void __launch_bounds__(kThreads) splitk_reduce_kernel(const float* __restrict__ partial, int splits, int64_t rows,
-                                                                 int64_t cols, int64_t ldp, void* out, int64_t ld_out,
-                                                                 int out_f32) {
-    const int64_t per_row = (cols + 3) / 4;
-    const int64_t total = rows * per_row;
-    const int64_t plane = rows * ldp;
-    for (int64_t i = blockIdx.x * static_cast<int64_t>(kThreads) + threadIdx.x; i < total;
-         i += static_cast<int64_t>(gridDim.x) * kThreads) {
-        const int64_t r = i / per_row, c = (i % per_row) * 4;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int s2 = 0; s2 < splits; ++s2) {
-            const float4 v = *reinterpret_cast<const float4*>(partial + s2 * plane + r * ldp + c);
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-        }
-        const float a[4] = {acc.x, acc.y, acc.z, acc.w};
-        for (int e = 0; e < 4; ++e) {
-            if (c + e < cols) {
-                if (out_f32) static_cast<float*>(out)[r * ld_out + c + e] = a[e];
-                else static_cast<__nv_bfloat16*>(out)[r * ld_out + c + e] = __float2bfloat16_rn(a[e]);
+// One launch that finishes a call: out[r][c] = sum over s of partial[s][r][c] for up to three split-K weight
+// gradients (summed in split order), and the fixed-order sum of the column-sum chunks.
+struct ReduceJob {
+    const float* partial;
+    void* out;
+    int64_t rows, cols, ldp, ld_out;
+    int32_t splits, blk_start, n_blk, pad_;
+};
+struct PostParams {
+    ReduceJob red[3];
+    ColsumParams cs;
+    int32_t n_red, red_blocks, out_f32, pad_;
+};
+__global__ void __launch_bounds__(kThreads) post_kernel(const __grid_constant__ PostParams P) {
+    if (static_cast<int>(blockIdx.x) < P.red_blocks) {
+        int ji = 0;
+        while (ji + 1 < P.n_red && static_cast<int>(blockIdx.x) >= P.red[ji + 1].blk_start) ++ji;
+        const ReduceJob& J = P.red[ji];
+        const int64_t per_row = (J.cols + 3) / 4;
+        const int64_t total = J.rows * per_row;
+        const int64_t plane = J.rows * J.ldp;
+        for (int64_t i = (blockIdx.x - J.blk_start) * static_cast<int64_t>(kThreads) + threadIdx.x; i < total;
+             i += static_cast<int64_t>(J.n_blk) * kThreads) {
+            const int64_t r = i / per_row, c = (i % per_row) * 4;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int s2 = 0; s2 < J.splits; ++s2) {
+                const float4 v = *reinterpret_cast<const float4*>(J.partial + s2 * plane + r * J.ldp + c);
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+            for (int e = 0; e < 4; ++e) {
+                if (c + e < J.cols) {
+                    if (P.out_f32) static_cast<float*>(J.out)[r * J.ld_out + c + e] = a[e];
+                    else static_cast<__nv_bfloat16*>(J.out)[r * J.ld_out + c + e] = __float2bfloat16_rn(a[e]);
+                }
             }
         }
+        return;
     }
+    int64_t c = static_cast<int64_t>(blockIdx.x - P.red_blocks) * kThreads + threadIdx.x;
+    int ji = 0;
+    while (ji < P.cs.n_jobs && c >= P.cs.job[ji].cols) {
+        c -= P.cs.job[ji].cols;
+        ++ji;
+    }
+    if (ji >= P.cs.n_jobs) return;
+    const ColsumJob& J = P.cs.job[ji];
+    float s = 0.f;
+    for (int k = 0; k < P.cs.chunks; ++k) s += J.partial[static_cast<int64_t>(k) * J.cols + c];
+    if (P.out_f32) static_cast<float*>(J.out)[c] = s;
+    else static_cast<__nv_bfloat16*>(J.out)[c] = __float2bfloat16_rn(s);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -218,12 +231,12 @@ Stored scratch_bf16(Ctx& cx, int64_t rows, int64_t cols) {
     return s;
 }
 
-// out[c] = sum_r M[r][c] for up to three bf16 matrices with the same row count; outputs have the model
-// dtype.  A null output skips that matrix.
-void colsum(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), void* out2 = nullptr,
-            const Stored& M3 = Stored(), void* out3 = nullptr) {
-    if (cx.st != ECOSPA_OK) return;
+// Column sums of up to three bf16 matrices with the same row count: launches the chunk-partial kernel and
+// returns the description the finishing launch needs.  A null output skips that matrix.
+ColsumParams colsum_begin(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), void* out2 = nullptr,
+                          const Stored& M3 = Stored(), void* out3 = nullptr) {
     ColsumParams P = {};
+    if (cx.st != ECOSPA_OK) return P;
     const Stored* mats[3] = {&M1, &M2, &M3};
     void* outs[3] = {out1, out2, out3};
     for (int i = 0; i < 3; ++i) {
@@ -237,24 +250,22 @@ void colsum(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), 
         J.vec_ok = aligned16(J.M) && J.ld % 8 == 0;
         P.rows = mats[i]->rows;
     }
-    if (P.n_jobs == 0) return;
+    if (P.n_jobs == 0) return P;
     P.chunks = static_cast<int32_t>(ceil_div(P.rows, kSumRows));
     P.out_f32 = cx.dtype == ECOSPA_F32;
-    int64_t total_cols = 0;
     int tiles = 0;
     for (int i = 0; i < P.n_jobs; ++i) {
         P.job[i].partial = static_cast<float*>(cx.arena.take(static_cast<size_t>(P.chunks) * P.job[i].cols * 4));
         if (!P.job[i].partial) {
             cx.st = ECOSPA_ERR_WORKSPACE;
-            return;
+            P.n_jobs = 0;
+            return P;
         }
-        total_cols += P.job[i].cols;
         tiles += P.job[i].col_tiles;
     }
     colsum_partial_kernel<<<dim3(tiles, P.chunks), kThreads, 0, cx.stream>>>(P);
-    if ((cx.st = check_launch("colsum_partial_kernel")) != ECOSPA_OK) return;
-    colsum_final_kernel<<<static_cast<unsigned>(ceil_div(total_cols, kThreads)), kThreads, 0, cx.stream>>>(P);
-    cx.st = check_launch("colsum_final_kernel");
+    cx.st = check_launch("colsum_partial_kernel");
+    return P;
 }
 
 // Compacted weight with n real shared indices, as stored: shared-cols d_m x n, or shared-rows n x d_m.
@@ -301,7 +312,7 @@ GemmOp proj_op(const Stored& X, const Stored& W, int64_t T, int64_t d_m, int64_t
 }
 // Weight gradients contract over the T tokens and have few output tiles, so on their own they would keep
 // most SMs idle behind one long tile.  The token range is therefore cut into `splits` ranges computed as
-// separate ops of the same launch into fp32 partial buffers, which splitk_reduce_kernel adds up in order.
+// separate ops of the same launch into fp32 partial buffers, which the finishing launch (post_kernel) adds up in split order.
 int wgrad_splits(int64_t rows_out, int64_t cols_out, int64_t T) {
     const int64_t tiles = ceil_div(rows_out, 256) * ceil_div(cols_out, 256);
     int64_t s = 74 / tiles;                       // aim at one wave of CTA pairs
@@ -366,13 +377,31 @@ int add_wgrad(Ctx& cx, GemmOp* ops, int n_ops, const Stored& Xs, const Stored& d
     red->out = out; red->ld_out = ld_out;
     return n_ops;
 }
-void run_reduce(Ctx& cx, const PendingReduce& r) {
-    if (cx.st != ECOSPA_OK || r.splits == 0) return;
-    const int64_t total = r.rows * ((r.cols + 3) / 4);
-    const int grid = static_cast<int>(std::min<int64_t>(ceil_div(total, kThreads), 148 * 8));
-    splitk_reduce_kernel<<<grid, kThreads, 0, cx.stream>>>(r.partial, r.splits, r.rows, r.cols, r.ldp, r.out, r.ld_out,
-                                                           cx.dtype == ECOSPA_F32);
-    cx.st = check_launch("splitk_reduce_kernel");
+// The finishing launch of a call: split-K reductions and column-sum finals together.
+void finish(Ctx& cx, const PendingReduce* red, int n_red, const ColsumParams& cs) {
+    if (cx.st != ECOSPA_OK) return;
+    PostParams P = {};
+    P.cs = cs;
+    P.out_f32 = cx.dtype == ECOSPA_F32;
+    int blocks = 0;
+    for (int i = 0; i < n_red; ++i) {
+        const PendingReduce& r = red[i];
+        if (r.splits == 0) continue;
+        ReduceJob& J = P.red[P.n_red++];
+        J.partial = r.partial; J.out = r.out; J.rows = r.rows; J.cols = r.cols; J.ldp = r.ldp; J.ld_out = r.ld_out;
+        J.splits = r.splits;
+        const int64_t total = r.rows * ((r.cols + 3) / 4);
+        J.n_blk = static_cast<int32_t>(std::min<int64_t>(ceil_div(total, kThreads), 148 * 4));
+        J.blk_start = blocks;
+        blocks += J.n_blk;
+    }
+    P.red_blocks = blocks;
+    int64_t total_cols = 0;
+    for (int i = 0; i < cs.n_jobs; ++i) total_cols += cs.job[i].cols;
+    blocks += static_cast<int>(ceil_div(total_cols, kThreads));
+    if (blocks == 0) return;
+    post_kernel<<<blocks, kThreads, 0, cx.stream>>>(P);
+    cx.st = check_launch("post_kernel");
 }
 
 }  // namespace
@@ -452,9 +481,7 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    run_reduce(cx, red[0]);
-    run_reduce(cx, red[1]);
-    colsum(cx, dQs, dbq_c, dKs, wk_c ? dbk_c : nullptr);
+    finish(cx, red, 2, colsum_begin(cx, dQs, dbq_c, dKs, wk_c ? dbk_c : nullptr));
     return cx.st;
 }
 
@@ -523,9 +550,7 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     dx.seg[0].a = dVs; dx.seg[0].b[0] = Wv; dx.seg[0].K = n;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    run_reduce(cx, red[0]);
-    run_reduce(cx, red[1]);
-    colsum(cx, dVs, dbv_c, dOs, dbo);
+    finish(cx, red, 2, colsum_begin(cx, dVs, dbv_c, dOs, dbo));
     return cx.st;
 }
 
@@ -591,8 +616,7 @@ extern "C" ecospa_status_t ecospa_coupled_qkv_bwd(const void* X, int64_t ldx, in
     dx.seg[2].a = dVs; dx.seg[2].b[0] = Wv; dx.seg[2].K = n_vo;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = cx.dtype == ECOSPA_F32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    for (int i = 0; i < 3; ++i) run_reduce(cx, red[i]);
-    colsum(cx, dQs, dbq_c, dKs, dbk_c, dVs, dbv_c);
+    finish(cx, red, 3, colsum_begin(cx, dQs, dbq_c, dKs, dbk_c, dVs, dbv_c));
     return cx.st;
 }
 
@@ -620,8 +644,7 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd_o(const void* Ctxm, int64_t ld_
     dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].K = d_m;
     dc.epi = EPI_STORE; dc.C = dCtx; dc.ldc = ld_dctx; dc.out_f32 = cx.dtype == ECOSPA_F32;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    run_reduce(cx, red);
-    colsum(cx, dOs, dbo);
+    finish(cx, &red, 1, colsum_begin(cx, dOs, dbo));
     return cx.st;
 }
 
@@ -732,7 +755,6 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    for (int i = 0; i < 3; ++i) run_reduce(cx, red[i]);
-    colsum(cx, dYs, db2, dH, sw ? nullptr : db1_c);
+    finish(cx, red, 3, colsum_begin(cx, dYs, db2, dH, sw ? nullptr : db1_c));
     return cx.st;
 }
