@@ -60,7 +60,8 @@ struct DevProblem {
     int32_t k_off[kMaxSeg];      // first contraction index of each segment
     uint8_t a_mn[kMaxSeg], b_mn[kMaxSeg];
     uint8_t map_a[kMaxSeg], map_b[kMaxSeg][2];
-    uint8_t pad2_[1];
+    uint8_t a_3d[kMaxSeg], b_3d[kMaxSeg];   // MN-major operand fetched as one 3-D box (both 64-wide atoms)
+    uint8_t pad2_[3];
     uint8_t out_f32, accumulate, bias_f32, pad_[5];
     void* C;
     void* C2;
@@ -171,6 +172,18 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         : "memory");
 }
 
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
@@ -553,8 +566,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                             if (leader) tma_load_2d(dst, map, x, y, full_bar(stage));
                             else tma_load_2d_pair(dst, map, x, y, fb);
                         };
+                        auto load3 = [&](uint32_t dst, const CUtensorMap* map, int y, int z) {
+                            if (leader) tma_load_3d(dst, map, 0, y, z, full_bar(stage));
+                            else tma_load_3d_pair(dst, map, 0, y, z, fb);
+                        };
                         if (!Q.a_mn[seg]) {
                             load(a_dst, ma, k0, m0);
+                        } else if (Q.a_3d[seg]) {
+                            load3(a_dst, ma, k0, m0 >> 6);
                         } else {
                             load(a_dst, ma, m0, k0);
                             load(a_dst + kAtomBytes, ma, m0 + 64, k0);
@@ -563,6 +582,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         const int nc = n0 + static_cast<int>(cta_rank) * Q.half1_n_off;
                         if (!Q.b_mn[seg]) {
                             load(b_dst, mb, k0, nc);
+                        } else if (Q.b_3d[seg]) {
+                            load3(b_dst, mb, k0, nc >> 6);
                         } else {
                             load(b_dst, mb, nc, k0);
                             load(b_dst + kAtomBytes, mb, nc + 64, k0);
@@ -571,6 +592,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         mbar_expect_tx(full_bar(stage), kStageTx);
                         if (!Q.a_mn[seg]) {
                             tma_load_2d(a_dst, ma, k0, m0, full_bar(stage));                    // box 64(k) x 128(m)
+                        } else if (Q.a_3d[seg]) {
+                            tma_load_3d(a_dst, ma, 0, k0, m0 >> 6, full_bar(stage));            // box 64 x 64(k) x 2 atoms
                         } else {
                             tma_load_2d(a_dst, ma, m0, k0, full_bar(stage));                    // box 64(m) x 64(k)
                             tma_load_2d(a_dst + kAtomBytes, ma, m0 + 64, k0, full_bar(stage));
@@ -582,6 +605,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                             const uint32_t dst = b_dst + h * kBHalf;
                             if (!Q.b_mn[seg]) {
                                 tma_load_2d(dst, mb, k0, nc, full_bar(stage));                  // box 64(k) x 128(n)
+                            } else if (Q.b_3d[seg]) {
+                                tma_load_3d(dst, mb, 0, k0, nc >> 6, full_bar(stage));
                             } else {
                                 tma_load_2d(dst, mb, nc, k0, full_bar(stage));                  // box 64(n) x 64(k)
                                 tma_load_2d(dst + kAtomBytes, mb, nc + 64, k0, full_bar(stage));
@@ -816,6 +841,21 @@ EncodeFn get_encode() {
     return fn;
 }
 
+// MN-major operand whose row length is a multiple of 64: the matrix [K][MN] viewed as (64, K, MN/64) with strides
+// (2 B, pitch, 128 B), so that one box of 64 x 64 x 2 brings both 64-wide swizzle atoms of a 128-wide slab
+// in the atom-major order the MMA descriptor expects.  Returns false when the view cannot be encoded.
+bool encode_map_mn3d(CUtensorMap* out, const Stored& s) {
+    EncodeFn enc = get_encode();
+    if (!enc || !s.ptr || s.cols % 64 != 0 || !aligned16(s.ptr) || (s.ld * 2) % 16 != 0) return false;
+    const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(s.rows), static_cast<cuuint64_t>(s.cols / 64)};
+    const cuuint64_t strides[2] = {static_cast<cuuint64_t>(s.ld) * 2, 128};
+    const cuuint32_t box[3] = {64, 64, 2};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(s.ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tensor map of a stored row-major bf16 matrix; box = 64 elements along the row x box_rows rows
 // (128-byte swizzle, operand loads), or 32 x 32 with the 64-byte swizzle (epilogue stores).
 ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows, bool store_box = false) {
@@ -950,12 +990,16 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
             if (k_end < (ks.a_mn ? a.rows : a.cols) && ks.K % BK) return ECOSPA_ERR_INVALID;
             if (ks.a_mn ? (a.rows < k_end || a.cols != op.M) : (a.rows != op.M || a.cols < k_end)) return ECOSPA_ERR_INVALID;
             const int mi = oi * kMapsPerOp;
-            if ((st = encode_map(&gp.maps[mi + 3 * s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
+            Q.a_3d[s] = ks.a_mn && encode_map_mn3d(&gp.maps[mi + 3 * s], a);
+            if (!Q.a_3d[s] && (st = encode_map(&gp.maps[mi + 3 * s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
             Q.map_a[s] = static_cast<uint8_t>(mi + 3 * s);
             for (int h = 0; h < 2; ++h) {
                 const Stored& b = (swiglu && h == 1) ? ks.b[1] : ks.b[0];
                 if (ks.b_mn ? (b.rows < k_end || b.cols != op.N) : (b.rows != op.N || b.cols < k_end)) return ECOSPA_ERR_INVALID;
-                if ((st = encode_map(&gp.maps[mi + 3 * s + 1 + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
+                const bool b3 = ks.b_mn && encode_map_mn3d(&gp.maps[mi + 3 * s + 1 + h], b);
+                if (h == 0) Q.b_3d[s] = b3;
+                else if (b3 != (Q.b_3d[s] != 0)) return ECOSPA_ERR_UNSUPPORTED;   // both halves take the same path
+                if (!b3 && (st = encode_map(&gp.maps[mi + 3 * s + 1 + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
                 Q.map_b[s][h] = static_cast<uint8_t>(mi + 3 * s + 1 + h);
             }
             Q.a_mn[s] = ks.a_mn;
