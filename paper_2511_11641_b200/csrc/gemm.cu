@@ -486,15 +486,16 @@ __device__ __forceinline__ const DevProblem& find_problem(const GemmParams& P, i
 // ------------------------------------------------------------------------------------------------
 template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams P) {
-    constexpr int kStages = PAIR ? 6 : 4;
-    constexpr int kBLocal = PAIR ? kBHalf : kBStage;        // B bytes this CTA holds per stage
+    constexpr int kSub = PAIR ? 2 : 1;                       // 64-deep k-blocks per pipeline stage
+    constexpr int kStages = PAIR ? 3 : 4;
+    constexpr int kBLocal = PAIR ? kBHalf : kBStage;        // B bytes this CTA holds per k-block
     constexpr int kTileM = PAIR ? 2 * BM : BM;               // rows of one scheduled tile
-    constexpr uint32_t kStageTx = kAStage + kBLocal;         // bytes this CTA's loads deliver per stage
+    constexpr uint32_t kBlockTx = kAStage + kBLocal;         // bytes this CTA's loads deliver per k-block
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;       // 1024-byte aligned stage memory
     uint8_t* smem = smem_raw + (base - raw_addr);
-    const uint32_t sA = base, sB = base + kStages * kAStage;
+    const uint32_t sA = base, sB = base + kStages * kSub * kAStage;
     const uint32_t sEpi = base + kRingBytes;
     uint8_t* tail = smem + kRingBytes + kEpiBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);        // full[S], empty[S], tmem_full[2], tmem_empty[2]
@@ -550,18 +551,27 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 const int local = tile - Q.tile_start;
                 const int m0 = (local % Q.tiles_m) * kTileM + static_cast<int>(cta_rank) * BM;
                 const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
-                for (int kb = 0; kb < Q.kblocks; ++kb) {
+                for (int kb0 = 0; kb0 < Q.kblocks; kb0 += kSub) {
+                    const int nsub = min(kSub, Q.kblocks - kb0);      // k-blocks this stage carries
+                    if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
+                    if (PAIR) {
+                        if (leader) mbar_expect_tx(full_bar(stage), 2 * kBlockTx * nsub);   // both CTAs' bytes
+                    } else {
+                        mbar_expect_tx(full_bar(stage), kBlockTx * nsub);
+                    }
+#pragma unroll
+                    for (int sub = 0; sub < kSub; ++sub) {
+                    if (sub >= nsub) break;
+                    const int kb = kb0 + sub;
                     const int seg = (kb >= Q.kb_end[0] ? 1 : 0) + (kb >= Q.kb_end[1] ? 1 : 0);
                     const int k0 = (kb - (seg ? Q.kb_end[seg - 1] : 0)) * BK + Q.k_off[seg];
-                    if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
-                    const uint32_t a_dst = sA + stage * kAStage, b_dst = sB + stage * kBLocal;
+                    const uint32_t a_dst = sA + (stage * kSub + sub) * kAStage, b_dst = sB + (stage * kSub + sub) * kBLocal;
                     const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
                     if (PAIR) {
                         // This CTA's share of the stage, completed on the leader's barrier: the leader uses the
                         // plain form on its own barrier (measurably cheaper), the peer the pair form that may
                         // signal the other CTA's barrier.
                         const uint32_t fb = map_to_cta(full_bar(stage), 0);
-                        if (leader) mbar_expect_tx(full_bar(stage), 2 * kStageTx);
                         auto load = [&](uint32_t dst, const CUtensorMap* map, int x, int y) {
                             if (leader) tma_load_2d(dst, map, x, y, full_bar(stage));
                             else tma_load_2d_pair(dst, map, x, y, fb);
@@ -589,7 +599,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                             load(b_dst + kAtomBytes, mb, nc + 64, k0);
                         }
                     } else {
-                        mbar_expect_tx(full_bar(stage), kStageTx);
                         if (!Q.a_mn[seg]) {
                             tma_load_2d(a_dst, ma, k0, m0, full_bar(stage));                    // box 64(k) x 128(m)
                         } else if (Q.a_3d[seg]) {
@@ -613,6 +622,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                             }
                         }
                     }
+                    }   // sub
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -631,21 +641,27 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 if (!(ok = mbar_wait<PAIR>(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 2, P.status))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb = 0; kb < Q.kblocks; ++kb) {
-                    const int seg = (kb >= Q.kb_end[0] ? 1 : 0) + (kb >= Q.kb_end[1] ? 1 : 0);
+                for (int kb0 = 0; kb0 < Q.kblocks; kb0 += kSub) {
+                    const int nsub = min(kSub, Q.kblocks - kb0);
                     if (!(ok = mbar_wait<PAIR>(full_bar(stage), phase, abort_flag, 3, P.status))) break;
                     tc_fence_after();
-                    const uint32_t a_mn = Q.a_mn[seg], b_mn = Q.b_mn[seg];
-                    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) |
-                                           (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
-                    const uint64_t a_desc = make_smem_desc(sA + stage * kAStage, a_mn ? kAtomBytes : 16, 1024);
-                    const uint64_t b_desc = make_smem_desc(sB + stage * kBLocal, b_mn ? kAtomBytes : 16, 1024);
-                    const uint64_t a_step = a_mn ? (2048 >> 4) : (32 >> 4);   // per 16 k: two 8-row groups, or 32 bytes
-                    const uint64_t b_step = b_mn ? (2048 >> 4) : (32 >> 4);
 #pragma unroll
-                    for (int ks = 0; ks < BK / 16; ++ks) {
-                        if (PAIR) tc_mma_bf16_pair(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
-                        else tc_mma_bf16(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
+                    for (int sub = 0; sub < kSub; ++sub) {
+                        if (sub >= nsub) break;
+                        const int kb = kb0 + sub;
+                        const int seg = (kb >= Q.kb_end[0] ? 1 : 0) + (kb >= Q.kb_end[1] ? 1 : 0);
+                        const uint32_t a_mn = Q.a_mn[seg], b_mn = Q.b_mn[seg];
+                        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) |
+                                               (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
+                        const uint64_t a_desc = make_smem_desc(sA + (stage * kSub + sub) * kAStage, a_mn ? kAtomBytes : 16, 1024);
+                        const uint64_t b_desc = make_smem_desc(sB + (stage * kSub + sub) * kBLocal, b_mn ? kAtomBytes : 16, 1024);
+                        const uint64_t a_step = a_mn ? (2048 >> 4) : (32 >> 4);   // per 16 k: two 8-row groups, or 32 bytes
+                        const uint64_t b_step = b_mn ? (2048 >> 4) : (32 >> 4);
+#pragma unroll
+                        for (int ks = 0; ks < BK / 16; ++ks) {
+                            if (PAIR) tc_mma_bf16_pair(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
+                            else tc_mma_bf16(d_tmem, a_desc + ks * a_step, b_desc + ks * b_step, idesc, (kb | ks) != 0 ? 1u : 0u);
+                        }
                     }
                     // the stage is free (in both CTAs) once these MMAs have read it
                     if (PAIR) {
