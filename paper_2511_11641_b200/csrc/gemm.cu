@@ -1,15 +1,15 @@
 // Grouped persistent bf16 GEMM for sm_100a: TMA -> shared memory ring -> tcgen05.mma (fp32 accumulators
 // in TMEM, double buffered) -> fused epilogues.  Two forms of the same kernel:
-//   single  cta_group::1, one CTA per SM computes 128x256 tiles (4-stage ring of 16 KB A + 32 KB B)
+//   single  cta_group::1, one CTA per SM computes 128x256 tiles (2 stages of 2 x (16 KB A + 32 KB B))
 //   pair    cta_group::2, a cluster of two CTAs computes 256x256 tiles: each CTA loads its 128 rows of A
-//           and its half of B (6-stage ring of 16 KB + 16 KB), the leader CTA issues the MMAs for both,
+//           and its half of B (3 stages of 2 x (16 KB + 16 KB)), the leader CTA issues the MMAs for both,
 //           so every SM fetches a third less operand data per flop.  No cluster multicast is used: the
 //           peer's loads signal the leader's barrier, and completion is committed to each CTA's barrier.
 //
-// One launch computes up to kMaxGemmOps independent products ("ops"), each C = sum over one or two
+// One launch computes up to kMaxGemmOps independent products ("ops"), each C = sum over one to three
 // K segments of A_seg * B_seg with K-major or MN-major operands (chosen per segment, so that weights
 // and activations are consumed in whatever row-major orientation they are stored).  Warp roles:
-//   warp 0      producer: one elected lane issues the TMA loads of a k-block into a 4-stage ring
+//   warp 0      producer: one elected lane issues the TMA loads of a stage (two 64-deep k-blocks)
 //   warp 1      owns the 512 TMEM columns; one elected lane issues the MMAs and the commits
 //   warps 2..9  epilogue: two warps per TMEM lane quadrant, each takes half of the tile's columns
 // The tile list of all ops is walked with a static stride (tile = blockIdx.x + i * gridDim.x);
@@ -61,7 +61,8 @@ struct DevProblem {
     uint8_t a_mn[kMaxSeg], b_mn[kMaxSeg];
     uint8_t map_a[kMaxSeg], map_b[kMaxSeg][2];
     uint8_t a_3d[kMaxSeg], b_3d[kMaxSeg];   // MN-major operand fetched as one 3-D box (both 64-wide atoms)
-    uint8_t pad2_[3];
+    uint8_t a_big[kMaxSeg], b_big[kMaxSeg]; // pair mode: one box brings both k-blocks of a stage
+    uint8_t pad2_[5];
     uint8_t out_f32, accumulate, bias_f32, pad_[5];
     void* C;
     void* C2;
@@ -172,6 +173,18 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t a_des
         : "memory");
 }
 
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int y, int z, int w, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(0), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, int y, int z, int w, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(0), "r"(y), "r"(z), "r"(w)
+        : "memory");
+}
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
@@ -486,11 +499,10 @@ __device__ __forceinline__ const DevProblem& find_problem(const GemmParams& P, i
 // ------------------------------------------------------------------------------------------------
 template <bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant__ GemmParams P) {
-    constexpr int kSub = PAIR ? 2 : 1;                       // 64-deep k-blocks per pipeline stage
-    constexpr int kStages = PAIR ? 3 : 4;
+    constexpr int kSub = 2;                                  // 64-deep k-blocks per pipeline stage
+    constexpr int kStages = PAIR ? 3 : 2;
     constexpr int kBLocal = PAIR ? kBHalf : kBStage;        // B bytes this CTA holds per k-block
     constexpr int kTileM = PAIR ? 2 * BM : BM;               // rows of one scheduled tile
-    constexpr uint32_t kBlockTx = kAStage + kBLocal;         // bytes this CTA's loads deliver per k-block
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;       // 1024-byte aligned stage memory
@@ -551,20 +563,52 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 const int local = tile - Q.tile_start;
                 const int m0 = (local % Q.tiles_m) * kTileM + static_cast<int>(cta_rank) * BM;
                 const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
-                for (int kb0 = 0; kb0 < Q.kblocks; kb0 += kSub) {
-                    const int nsub = min(kSub, Q.kblocks - kb0);      // k-blocks this stage carries
+                // a stage carries up to kSub k-blocks of one K segment
+                for (int seg = 0; ok && seg < kMaxSeg; ++seg) {
+                const int kb_lo = seg ? Q.kb_end[seg - 1] : 0, kb_hi = Q.kb_end[seg];
+                for (int kb0 = kb_lo; kb0 < kb_hi; kb0 += kSub) {
+                    const int nsub = min(kSub, kb_hi - kb0);
                     if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
+                    // "big" operands arrive as one box holding both k-blocks (zero-filled past the end of K)
+                    const bool a_big = PAIR && Q.a_big[seg], b_big = PAIR && Q.b_big[seg];
+                    const uint32_t tx = (a_big ? kSub : nsub) * kAStage + (b_big ? kSub : nsub) * kBLocal;
                     if (PAIR) {
-                        if (leader) mbar_expect_tx(full_bar(stage), 2 * kBlockTx * nsub);   // both CTAs' bytes
+                        if (leader) mbar_expect_tx(full_bar(stage), 2 * tx);   // both CTAs' bytes
                     } else {
-                        mbar_expect_tx(full_bar(stage), kBlockTx * nsub);
+                        mbar_expect_tx(full_bar(stage), tx);
+                    }
+                    if (PAIR && (a_big || b_big)) {
+                        const int k0 = (kb0 - kb_lo) * BK + Q.k_off[seg];
+                        const uint32_t fb = map_to_cta(full_bar(stage), 0);
+                        if (a_big) {
+                            const uint32_t dst = sA + stage * kSub * kAStage;
+                            const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
+                            if (!Q.a_mn[seg]) {           // (64 k, 128 rows, 2 k-blocks)
+                                if (leader) tma_load_3d(dst, ma, 0, m0, k0 >> 6, full_bar(stage));
+                                else tma_load_3d_pair(dst, ma, 0, m0, k0 >> 6, fb);
+                            } else {                      // (64 m, 64 k, 2 atoms, 2 k-blocks)
+                                if (leader) tma_load_4d(dst, ma, 0, m0 >> 6, k0 >> 6, full_bar(stage));
+                                else tma_load_4d_pair(dst, ma, 0, m0 >> 6, k0 >> 6, fb);
+                            }
+                        }
+                        if (b_big) {
+                            const uint32_t dst = sB + stage * kSub * kBLocal;
+                            const CUtensorMap* mb = &P.maps[Q.map_b[seg][cta_rank]];
+                            const int nc = n0 + static_cast<int>(cta_rank) * Q.half1_n_off;
+                            if (!Q.b_mn[seg]) {
+                                if (leader) tma_load_3d(dst, mb, 0, nc, k0 >> 6, full_bar(stage));
+                                else tma_load_3d_pair(dst, mb, 0, nc, k0 >> 6, fb);
+                            } else {
+                                if (leader) tma_load_4d(dst, mb, 0, nc >> 6, k0 >> 6, full_bar(stage));
+                                else tma_load_4d_pair(dst, mb, 0, nc >> 6, k0 >> 6, fb);
+                            }
+                        }
                     }
 #pragma unroll
                     for (int sub = 0; sub < kSub; ++sub) {
                     if (sub >= nsub) break;
                     const int kb = kb0 + sub;
-                    const int seg = (kb >= Q.kb_end[0] ? 1 : 0) + (kb >= Q.kb_end[1] ? 1 : 0);
-                    const int k0 = (kb - (seg ? Q.kb_end[seg - 1] : 0)) * BK + Q.k_off[seg];
+                    const int k0 = (kb - kb_lo) * BK + Q.k_off[seg];
                     const uint32_t a_dst = sA + (stage * kSub + sub) * kAStage, b_dst = sB + (stage * kSub + sub) * kBLocal;
                     const CUtensorMap* ma = &P.maps[Q.map_a[seg]];
                     if (PAIR) {
@@ -580,7 +624,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                             if (leader) tma_load_3d(dst, map, 0, y, z, full_bar(stage));
                             else tma_load_3d_pair(dst, map, 0, y, z, fb);
                         };
-                        if (!Q.a_mn[seg]) {
+                        if (a_big) {
+                        } else if (!Q.a_mn[seg]) {
                             load(a_dst, ma, k0, m0);
                         } else if (Q.a_3d[seg]) {
                             load3(a_dst, ma, k0, m0 >> 6);
@@ -590,7 +635,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         }
                         const CUtensorMap* mb = &P.maps[Q.map_b[seg][cta_rank]];
                         const int nc = n0 + static_cast<int>(cta_rank) * Q.half1_n_off;
-                        if (!Q.b_mn[seg]) {
+                        if (b_big) {
+                        } else if (!Q.b_mn[seg]) {
                             load(b_dst, mb, k0, nc);
                         } else if (Q.b_3d[seg]) {
                             load3(b_dst, mb, k0, nc >> 6);
@@ -624,6 +670,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     }
                     }   // sub
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }   // kb0
                 }
             }
         }
@@ -641,15 +688,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 if (!(ok = mbar_wait<PAIR>(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 2, P.status))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
-                for (int kb0 = 0; kb0 < Q.kblocks; kb0 += kSub) {
-                    const int nsub = min(kSub, Q.kblocks - kb0);
+                for (int seg = 0; ok && seg < kMaxSeg; ++seg) {
+                const int kb_lo = seg ? Q.kb_end[seg - 1] : 0, kb_hi = Q.kb_end[seg];
+                for (int kb0 = kb_lo; kb0 < kb_hi; kb0 += kSub) {
+                    const int nsub = min(kSub, kb_hi - kb0);
                     if (!(ok = mbar_wait<PAIR>(full_bar(stage), phase, abort_flag, 3, P.status))) break;
                     tc_fence_after();
 #pragma unroll
                     for (int sub = 0; sub < kSub; ++sub) {
                         if (sub >= nsub) break;
                         const int kb = kb0 + sub;
-                        const int seg = (kb >= Q.kb_end[0] ? 1 : 0) + (kb >= Q.kb_end[1] ? 1 : 0);
                         const uint32_t a_mn = Q.a_mn[seg], b_mn = Q.b_mn[seg];
                         const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (a_mn << 15) | (b_mn << 16) |
                                                (static_cast<uint32_t>(BN >> 3) << 17) | (static_cast<uint32_t>(kTileM >> 4) << 24);
@@ -672,6 +720,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     }
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
+                }   // seg
                 if (ok) {                              // accumulator complete (in both CTAs)
                     if (PAIR) {
                         tc_commit_pair(map_to_cta(tfull_bar(acc), 0));
@@ -872,6 +921,31 @@ bool encode_map_mn3d(CUtensorMap* out, const Stored& s) {
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Pair mode, one box per operand per stage (two 64-deep k-blocks), when the extents are multiples of 64:
+//   K-major  [rows][K]  viewed as (64, rows, K/64)          box 64 x 128 x 2        -> [k-block][row][64 k]
+//   MN-major [K][MN]    viewed as (64, 64, MN/64, K/64)     box 64 x 64 x 2 x 2     -> [k-block][atom][k][64 mn]
+// Both orders are exactly two consecutive k-block images of the per-k-block layout.
+bool encode_map_big(CUtensorMap* out, const Stored& s, bool mn) {
+    EncodeFn enc = get_encode();
+    if (!enc || !s.ptr || s.cols % 64 != 0 || !aligned16(s.ptr) || (s.ld * 2) % 16 != 0) return false;
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (!mn) {
+        const cuuint64_t dims[3] = {64, static_cast<cuuint64_t>(s.rows), static_cast<cuuint64_t>(s.cols / 64)};
+        const cuuint64_t strides[2] = {static_cast<cuuint64_t>(s.ld) * 2, 128};
+        const cuuint32_t box[3] = {64, 128, 2};
+        return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(s.ptr), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+    }
+    if (s.rows % 64 != 0) return false;
+    const cuuint64_t dims[4] = {64, 64, static_cast<cuuint64_t>(s.cols / 64), static_cast<cuuint64_t>(s.rows / 64)};
+    const cuuint64_t strides[3] = {static_cast<cuuint64_t>(s.ld) * 2, 128, static_cast<cuuint64_t>(s.ld) * 128};
+    const cuuint32_t box[4] = {64, 64, 2, 2};
+    return enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(s.ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tensor map of a stored row-major bf16 matrix; box = 64 elements along the row x box_rows rows
 // (128-byte swizzle, operand loads), or 32 x 32 with the 64-byte swizzle (epilogue stores).
 ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows, bool store_box = false) {
@@ -1006,16 +1080,22 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
             if (k_end < (ks.a_mn ? a.rows : a.cols) && ks.K % BK) return ECOSPA_ERR_INVALID;
             if (ks.a_mn ? (a.rows < k_end || a.cols != op.M) : (a.rows != op.M || a.cols < k_end)) return ECOSPA_ERR_INVALID;
             const int mi = oi * kMapsPerOp;
-            Q.a_3d[s] = ks.a_mn && encode_map_mn3d(&gp.maps[mi + 3 * s], a);
-            if (!Q.a_3d[s] && (st = encode_map(&gp.maps[mi + 3 * s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
+            Q.a_big[s] = pair && encode_map_big(&gp.maps[mi + 3 * s], a, ks.a_mn);
+            Q.a_3d[s] = !Q.a_big[s] && ks.a_mn && encode_map_mn3d(&gp.maps[mi + 3 * s], a);
+            if (!Q.a_big[s] && !Q.a_3d[s] && (st = encode_map(&gp.maps[mi + 3 * s], a, ks.a_mn ? 64 : 128)) != ECOSPA_OK) return st;
             Q.map_a[s] = static_cast<uint8_t>(mi + 3 * s);
             for (int h = 0; h < 2; ++h) {
                 const Stored& b = (swiglu && h == 1) ? ks.b[1] : ks.b[0];
                 if (ks.b_mn ? (b.rows < k_end || b.cols != op.N) : (b.rows != op.N || b.cols < k_end)) return ECOSPA_ERR_INVALID;
-                const bool b3 = ks.b_mn && encode_map_mn3d(&gp.maps[mi + 3 * s + 1 + h], b);
-                if (h == 0) Q.b_3d[s] = b3;
-                else if (b3 != (Q.b_3d[s] != 0)) return ECOSPA_ERR_UNSUPPORTED;   // both halves take the same path
-                if (!b3 && (st = encode_map(&gp.maps[mi + 3 * s + 1 + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
+                const bool bb = pair && encode_map_big(&gp.maps[mi + 3 * s + 1 + h], b, ks.b_mn);
+                const bool b3 = !bb && ks.b_mn && encode_map_mn3d(&gp.maps[mi + 3 * s + 1 + h], b);
+                if (h == 0) {
+                    Q.b_big[s] = bb;
+                    Q.b_3d[s] = b3;
+                } else if (bb != (Q.b_big[s] != 0) || b3 != (Q.b_3d[s] != 0)) {
+                    return ECOSPA_ERR_UNSUPPORTED;   // both halves take the same path
+                }
+                if (!bb && !b3 && (st = encode_map(&gp.maps[mi + 3 * s + 1 + h], b, ks.b_mn ? 64 : 128)) != ECOSPA_OK) return st;
                 Q.map_b[s][h] = static_cast<uint8_t>(mi + 3 * s + 1 + h);
             }
             Q.a_mn[s] = ks.a_mn;
