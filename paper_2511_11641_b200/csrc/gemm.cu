@@ -43,8 +43,9 @@ constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kTmemCols = 512;
 constexpr int kMaxSeg = 3;
-constexpr int kMapsPerOp = 3 * kMaxSeg;     // per K segment: one A map and two B (half) maps
-constexpr int kEpiSlotBytes = 32 * 32 * 2;  // one 32-row x 32-column bf16 store box
+constexpr int kOperandMaps = 3 * kMaxSeg;   // per K segment: one A map and two B (half) maps
+constexpr int kMapsPerOp = kOperandMaps + 3; // + one store map per output (C, C2, C3)
+constexpr int kEpiSlotBytes = 32 * 32 * 2;  // one 32-row x 64-byte staging image; a warp owns two (= one 32 x 128-byte image)
 constexpr int kEpiBytes = kEpiWarps * 2 * kEpiSlotBytes;
 constexpr int kSmemBytes = kRingBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
@@ -62,7 +63,9 @@ struct DevProblem {
     uint8_t map_a[kMaxSeg], map_b[kMaxSeg][2];
     uint8_t a_3d[kMaxSeg], b_3d[kMaxSeg];   // MN-major operand fetched as one 3-D box (both 64-wide atoms)
     uint8_t a_big[kMaxSeg], b_big[kMaxSeg]; // pair mode: one box brings both k-blocks of a stage
-    uint8_t pad2_[5];
+    uint8_t map_c[3];            // store maps of C, C2, C3 (valid when tma_out)
+    uint8_t tma_out;             // outputs leave through TMA tile stores (everything except accumulate)
+    uint8_t pad2_[1];
     uint8_t out_f32, accumulate, bias_f32, pad_[5];
     void* C;
     void* C2;
@@ -202,6 +205,20 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(x), "r"(y)
         : "memory");
+}
+
+// --- TMA tile stores (shared memory -> global), tracked per issuing thread in bulk groups
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all but the newest N stores of this thread have finished reading their shared-memory source
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -355,6 +372,59 @@ __device__ __forceinline__ void store_row32(void* base, int64_t row_off, int n, 
                 if (i < nv) p[i] = __float2bfloat16_rn(v[i]);
         }
     }
+}
+
+// Staging images for the TMA tile stores.  A warp owns 4 KB: either one image of 32 rows x 128 bytes in the
+// 128-byte swizzle (64 bf16 or 32 fp32 columns; 16-byte chunk j of row r sits at chunk j ^ (r & 7)), or two
+// "slots" of 32 rows x 64 bytes in the 64-byte swizzle (32 bf16 columns; chunk j of row r at j ^ ((r >> 1) & 3)).
+// Lane = row (what tcgen05.ld delivers); both layouts are bank-conflict free for that access.
+// Before an image is overwritten the issuing lane waits until the stores that still read it are done
+// (KEEP = stores that may stay in flight because they read the other slot).
+template <int KEEP>
+__device__ __forceinline__ void stage_begin(int lane) {
+    if (lane == 0) bulk_wait_read<KEEP>();
+    __syncwarp();
+}
+__device__ __forceinline__ void stage_commit(const CUtensorMap* map, uint32_t buf, int x, int y, int lane) {
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        tma_store_2d(map, buf, x, y);
+        bulk_commit();
+    }
+}
+// 32 words (128 bytes) per lane
+__device__ __forceinline__ void stage_row128(uint32_t buf, int lane, const uint32_t (&w)[32]) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + lane * 128 + ((j ^ (lane & 7)) << 4)),
+                     "r"(w[4 * j]), "r"(w[4 * j + 1]), "r"(w[4 * j + 2]), "r"(w[4 * j + 3]) : "memory");
+}
+// 64 fp32 values of one row -> 64 bf16 columns (one 128-byte image row)
+__device__ __forceinline__ void stage_bf16x64(uint32_t buf, int lane, const float (&v0)[32], const float (&v1)[32]) {
+    uint32_t w[32];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        w[i] = pack_bf16(v0[2 * i], v0[2 * i + 1]);
+        w[16 + i] = pack_bf16(v1[2 * i], v1[2 * i + 1]);
+    }
+    stage_row128(buf, lane, w);
+}
+// 32 fp32 values of one row -> 32 fp32 columns (one 128-byte image row)
+__device__ __forceinline__ void stage_f32x32(uint32_t buf, int lane, const float (&v)[32]) {
+    uint32_t w[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) w[i] = __float_as_uint(v[i]);
+    stage_row128(buf, lane, w);
+}
+// 32 fp32 values of one row -> 32 bf16 columns (one 64-byte slot row)
+__device__ __forceinline__ void stage_bf16x32(uint32_t slot, int lane, const float (&v)[32]) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slot + lane * 64 + ((c ^ ((lane >> 1) & 3)) << 4)),
+                     "r"(pack_bf16(v[8 * c + 0], v[8 * c + 1])), "r"(pack_bf16(v[8 * c + 2], v[8 * c + 3])),
+                     "r"(pack_bf16(v[8 * c + 4], v[8 * c + 5])), "r"(pack_bf16(v[8 * c + 6], v[8 * c + 7]))
+                     : "memory");
 }
 
 // Per-warp transposition buffers: 32 rows x 32 bf16 columns, 64 bytes per row, the four 16-byte chunks
@@ -536,6 +606,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (worker < P.total_tiles) {
+            // warm the descriptors of the first tile while TMEM is allocated and the CTAs meet
+            const DevProblem& Q0 = find_problem(P, worker);
+            prefetch_tensormap(&P.maps[Q0.map_a[0]]);
+            prefetch_tensormap(&P.maps[Q0.map_b[0][cta_rank]]);
+        }
     }
     if (warp == 1) {
         if (PAIR) {
@@ -747,41 +823,40 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1u;
+            const int epi = Q.epi;
+            const int QM = Q.M, QN = Q.N;
+            const bool tma = Q.tma_out != 0;
+            const CUtensorMap* mc0 = &P.maps[Q.map_c[0]];
+            const CUtensorMap* mc1 = &P.maps[Q.map_c[1]];
+            const CUtensorMap* mc2 = &P.maps[Q.map_c[2]];
             // saved activations of the derivative epilogues: first chunk requested before the accumulator is ready
-            const bool need_h = Q.epi >= EPI_DGELU_ERF;
-            const bool need_hb = Q.epi == EPI_DSWIGLU;
+            const bool need_h = epi >= EPI_DGELU_ERF;
+            const bool need_hb = epi == EPI_DSWIGLU;
             const unsigned short* Hp = static_cast<const unsigned short*>(Q.H);
             const unsigned short* Hbp = static_cast<const unsigned short*>(Q.Hb);
             uint4 hq[4], hbq[4];
-            if (need_h) staged_load32_issue(Hp, Q.ldh, m_warp, n0 + half * 128, Q.M, Q.N, hq, lane);
-            if (need_hb) staged_load32_issue(Hbp, Q.ldh, m_warp, n0 + half * 128, Q.M, Q.N, hbq, lane);
+            if (need_h) staged_load32_issue(Hp, Q.ldh, m_warp, n0 + half * 128, QM, QN, hq, lane);
+            if (need_hb) staged_load32_issue(Hbp, Q.ldh, m_warp, n0 + half * 128, QM, QN, hbq, lane);
+            // the second slot doubles as the landing buffer of those loads: no store of an earlier tile may still read it
+            if (need_h) stage_begin<0>(lane);
             if (!(ok = mbar_wait<PAIR>(tfull_bar(acc), acc_phase, abort_flag, 4, P.status))) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
-            const bool row_ok = m < Q.M;
-            const bool warp_rows = m_warp < Q.M;          // any row of this warp inside the output
-            const int64_t c_off = static_cast<int64_t>(m) * Q.ldc;
-            const int epi = Q.epi;
-            const bool staged = Q.out_f32 == 0;          // bf16 outputs go through the transposition buffer
-            // writes 32 columns starting at n of one output
-            auto emit = [&](void* ptr, int n, int nv, const float (&v)[32], bool accumulate) {
-                if (staged) {
-                    if (warp_rows) staged_store32(buf_out, static_cast<__nv_bfloat16*>(ptr), Q.ldc, m_warp, n, Q.M, Q.N, v, lane, accumulate);
-                } else if (row_ok) {
-                    if (accumulate) {
-                        float o[32];
-                        load_row32(ptr, c_off, n, nv, o, true);
-                        float t[32];
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) t[i] = v[i] + o[i];
-                        store_row32(ptr, c_off, n, nv, t, true);
-                    } else {
-                        store_row32(ptr, c_off, n, nv, v, true);
-                    }
-                }
-            };
+            const bool row_ok = m < QM;
+            const bool warp_rows = m_warp < QM;          // any row of this warp inside the output
             if (epi == EPI_SWIGLU) {
-                // accumulator columns [0,128) = gate, [128,256) = up for hidden units n0 .. n0+127
+                // accumulator columns [0,128) = gate, [128,256) = up for hidden units n0 .. n0+127.
+                // The three outputs of a chunk alternate between the two slots, one store may stay in flight.
+                int slot = 0;
+                bool fresh = true;
+                auto put = [&](const CUtensorMap* map, int n, const float (&v)[32]) {
+                    if (fresh) stage_begin<0>(lane); else stage_begin<1>(lane);
+                    fresh = false;
+                    const uint32_t sb = buf_out + slot * kEpiSlotBytes;
+                    stage_bf16x32(sb, lane, v);
+                    stage_commit(map, sb, n, m_warp, lane);
+                    slot ^= 1;
+                };
 #pragma unroll 1
                 for (int c = 0; c < 2; ++c) {
                     const int hc = half * 64 + c * 32;
@@ -790,21 +865,95 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     tc_ld32(t_row + 128 + hc, ru);
                     tc_wait_ld();
                     const int n = n0 + hc;
-                    const int nv = min(32, Q.N - n);
-                    if (nv <= 0) continue;
+                    if (n >= QN || !warp_rows) continue;
                     float g[32], u[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) {
                         g[i] = __uint_as_float(rg[i]);
                         u[i] = __uint_as_float(ru[i]);
                     }
-                    emit(Q.C, n, nv, g, false);
-                    emit(Q.C2, n, nv, u, false);
+                    put(mc0, n, g);
+                    put(mc1, n, u);
 #pragma unroll
                     for (int i = 0; i < 32; ++i) g[i] = g[i] * sigmoidf_(g[i]) * u[i];
-                    emit(Q.C3, n, nv, g, false);
+                    put(mc2, n, g);
+                }
+            } else if (epi == EPI_STORE && tma && !Q.out_f32) {
+                // bf16 output: two chunks of 64 columns, each one 32 x 128-byte image
+#pragma unroll 1
+                for (int c = 0; c < 2; ++c) {
+                    const int col = half * 128 + c * 64;
+                    uint32_t r0[32], r1[32];
+                    tc_ld32(t_row + col, r0);
+                    tc_ld32(t_row + col + 32, r1);
+                    tc_wait_ld();
+                    const int n = n0 + col;
+                    if (n >= QN || !warp_rows) continue;
+                    float v0[32], v1[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        v0[i] = __uint_as_float(r0[i]);
+                        v1[i] = __uint_as_float(r1[i]);
+                    }
+                    if (Q.bias) {
+                        float b[32];
+                        load_row32(Q.bias, 0, n, min(32, QN - n), b, Q.bias_f32 != 0);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v0[i] += b[i];
+                        load_row32(Q.bias, 0, n + 32, min(32, QN - n - 32), b, Q.bias_f32 != 0);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v1[i] += b[i];
+                    }
+                    stage_begin<0>(lane);
+                    stage_bf16x64(buf_out, lane, v0, v1);
+                    stage_commit(mc0, buf_out, n, m_warp, lane);
+                }
+            } else if (epi == EPI_GELU_ERF || epi == EPI_GELU_TANH) {
+                // H = acc + bias and A = GELU(H), 64 columns at a time
+#pragma unroll 1
+                for (int c = 0; c < 2; ++c) {
+                    const int col = half * 128 + c * 64;
+                    uint32_t r0[32], r1[32];
+                    tc_ld32(t_row + col, r0);
+                    tc_ld32(t_row + col + 32, r1);
+                    tc_wait_ld();
+                    const int n = n0 + col;
+                    if (n >= QN || !warp_rows) continue;
+                    float v0[32], v1[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        v0[i] = __uint_as_float(r0[i]);
+                        v1[i] = __uint_as_float(r1[i]);
+                    }
+                    if (Q.bias) {
+                        float b[32];
+                        load_row32(Q.bias, 0, n, min(32, QN - n), b, Q.bias_f32 != 0);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v0[i] += b[i];
+                        load_row32(Q.bias, 0, n + 32, min(32, QN - n - 32), b, Q.bias_f32 != 0);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v1[i] += b[i];
+                    }
+                    stage_begin<0>(lane);
+                    stage_bf16x64(buf_out, lane, v0, v1);
+                    stage_commit(mc0, buf_out, n, m_warp, lane);
+                    if (epi == EPI_GELU_ERF) {
+                        gelu_erf32(v0);
+                        gelu_erf32(v1);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            v0[i] = gelu_tanh(v0[i]);
+                            v1[i] = gelu_tanh(v1[i]);
+                        }
+                    }
+                    stage_begin<0>(lane);
+                    stage_bf16x64(buf_out, lane, v0, v1);
+                    stage_commit(mc1, buf_out, n, m_warp, lane);
                 }
             } else {
+                // 32 columns at a time: fp32 outputs, accumulating outputs and the derivative epilogues
+                const int64_t c_off = static_cast<int64_t>(m) * Q.ldc;
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
                     const int col = half * 128 + c * 32;
@@ -812,7 +961,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     tc_ld32(t_row + col, r);
                     tc_wait_ld();
                     const int n = n0 + col;
-                    const int nv = min(32, Q.N - n);
+                    const int nv = min(32, QN - n);
                     if (nv <= 0) continue;
                     float v[32];
 #pragma unroll
@@ -824,30 +973,41 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         for (int i = 0; i < 32; ++i) v[i] += b[i];
                     }
                     if (epi == EPI_STORE) {
-                        emit(Q.C, n, nv, v, Q.accumulate != 0);
-                    } else if (epi == EPI_GELU_ERF || epi == EPI_GELU_TANH) {
-                        emit(Q.C, n, nv, v, false);
+                        if (tma) {                         // fp32 output: one 32 x 128-byte image
+                            if (warp_rows) {
+                                stage_begin<0>(lane);
+                                stage_f32x32(buf_out, lane, v);
+                                stage_commit(mc0, buf_out, n, m_warp, lane);
+                            }
+                        } else if (!Q.out_f32) {           // C += acc, bf16
+                            if (warp_rows) staged_store32(buf_out, static_cast<__nv_bfloat16*>(Q.C), Q.ldc, m_warp, n, QM, QN, v, lane, true);
+                        } else if (row_ok) {               // C += acc, fp32
+                            float o[32];
+                            load_row32(Q.C, c_off, n, nv, o, true);
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (epi != EPI_GELU_ERF) v[i] = gelu_tanh(v[i]);
-                        if (epi == EPI_GELU_ERF) gelu_erf32(v);
-                        emit(Q.C2, n, nv, v, false);
+                            for (int i = 0; i < 32; ++i) v[i] += o[i];
+                            store_row32(Q.C, c_off, n, nv, v, true);
+                        }
                     } else if (epi == EPI_DGELU_ERF || epi == EPI_DGELU_TANH) {
                         float h[32];
                         staged_load32_finish(buf_in, hq, h, lane);
-                        if (c < 3) staged_load32_issue(Hp, Q.ldh, m_warp, n + 32, Q.M, Q.N, hq, lane);
+                        if (c < 3) staged_load32_issue(Hp, Q.ldh, m_warp, n + 32, QM, QN, hq, lane);
 #pragma unroll
                         for (int i = 0; i < 32; ++i)
                             if (epi != EPI_DGELU_ERF) v[i] *= dgelu_tanh(h[i]);
                         if (epi == EPI_DGELU_ERF) dgelu_erf32(v, h);
-                        emit(Q.C, n, nv, v, false);
+                        if (warp_rows) {
+                            stage_begin<0>(lane);
+                            stage_bf16x32(buf_out, lane, v);
+                            stage_commit(mc0, buf_out, n, m_warp, lane);
+                        }
                     } else {  // EPI_DSWIGLU
                         float hg[32], hu[32];
                         staged_load32_finish(buf_in, hq, hg, lane);
                         staged_load32_finish(buf_in, hbq, hu, lane);
                         if (c < 3) {
-                            staged_load32_issue(Hp, Q.ldh, m_warp, n + 32, Q.M, Q.N, hq, lane);
-                            staged_load32_issue(Hbp, Q.ldh, m_warp, n + 32, Q.M, Q.N, hbq, lane);
+                            staged_load32_issue(Hp, Q.ldh, m_warp, n + 32, QM, QN, hq, lane);
+                            staged_load32_issue(Hbp, Q.ldh, m_warp, n + 32, QM, QN, hbq, lane);
                         }
 #pragma unroll
                         for (int i = 0; i < 32; ++i) {
@@ -855,8 +1015,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                             hu[i] = v[i] * hu[i] * s * (1.f + hg[i] * (1.f - s));   // dH_gate
                             v[i] = v[i] * hg[i] * s;                                // dH_up
                         }
-                        emit(Q.C, n, nv, hu, false);
-                        emit(Q.C2, n, nv, v, false);
+                        if (warp_rows) {
+                            stage_begin<0>(lane);
+                            stage_bf16x32(buf_out, lane, hu);
+                            stage_commit(mc0, buf_out, n, m_warp, lane);
+                            stage_begin<0>(lane);
+                            stage_bf16x32(buf_out, lane, v);
+                            stage_commit(mc1, buf_out, n, m_warp, lane);
+                        }
                     }
                 }
             }
@@ -867,6 +1033,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 else mbar_arrive(tempty_bar(acc));
             }
         }
+        if (lane == 0) bulk_wait_all();            // this warp's tile stores have landed
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -966,6 +1133,29 @@ ecospa_status_t encode_map(CUtensorMap* out, const Stored& s, int box_rows, bool
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+        return ECOSPA_ERR_CUDA;
+    }
+    return ECOSPA_OK;
+}
+
+// Store map of an output (rows x cols, pitch ld elements): boxes of 32 rows x 64 bf16 or 32 fp32 columns
+// (128-byte swizzle) or 32 rows x 32 bf16 columns (64-byte swizzle), matching the staging images.
+ecospa_status_t encode_out_map(CUtensorMap* out, void* ptr, int64_t rows, int64_t cols, int64_t ld, bool f32, bool wide) {
+    EncodeFn enc = get_encode();
+    if (!enc) {
+        set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
+        return ECOSPA_ERR_CUDA;
+    }
+    const int eb = f32 ? 4 : 2;
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * eb};
+    const cuuint32_t box[2] = {(f32 || !wide) ? 32u : 64u, 32u};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(out, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, ptr, dims, strides, box,
+                           estr, CU_TENSOR_MAP_INTERLEAVE_NONE, (f32 || wide) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                           CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (output)");
         return ECOSPA_ERR_CUDA;
     }
     return ECOSPA_OK;
@@ -1103,6 +1293,17 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
             Q.k_off[s] = static_cast<int32_t>(ks.k_begin);
             Q.kblocks += static_cast<int32_t>(ceil_div(ks.K, BK));
             Q.kb_end[s] = Q.kblocks;
+        }
+        // outputs leave through TMA tile stores unless they are added to what C already holds
+        Q.tma_out = op.accumulate ? 0 : 1;
+        if (Q.tma_out) {
+            const bool wide = op.epi == EPI_STORE || op.epi == EPI_GELU_ERF || op.epi == EPI_GELU_TANH;
+            void* outs[3] = {op.C, op.C2, op.C3};
+            for (int o = 0; o < 3; ++o) {
+                Q.map_c[o] = static_cast<uint8_t>(oi * kMapsPerOp + kOperandMaps + o);
+                if (!outs[o]) continue;
+                if ((st = encode_out_map(&gp.maps[Q.map_c[o]], outs[o], op.M, op.N, op.ldc, op.out_f32, wide)) != ECOSPA_OK) return st;
+            }
         }
         for (int s2 = op.n_kseg; s2 < kMaxSeg; ++s2) Q.kb_end[s2] = Q.kblocks;
         Q.tiles_m = static_cast<int32_t>(ceil_div(op.M, tile_m));
