@@ -63,9 +63,8 @@ struct DevProblem {
     uint8_t map_a[kMaxSeg], map_b[kMaxSeg][2];
     uint8_t a_3d[kMaxSeg], b_3d[kMaxSeg];   // MN-major operand fetched as one 3-D box (both 64-wide atoms)
     uint8_t a_big[kMaxSeg], b_big[kMaxSeg]; // pair mode: one box brings both k-blocks of a stage
-    uint8_t map_c[3];            // store maps of C, C2, C3 (valid when tma_out)
-    uint8_t tma_out;             // outputs leave through TMA tile stores (everything except accumulate)
-    uint8_t pad2_[1];
+    uint8_t map_c[3];            // store maps of C, C2, C3
+    uint8_t pad2_[2];
     uint8_t out_f32, accumulate, bias_f32, pad_[5];
     void* C;
     void* C2;
@@ -76,10 +75,15 @@ struct DevProblem {
     int64_t ldc, ldh;
 };
 
+constexpr int kMaxOrder = 2048;              // entries of the explicit tile schedule
+constexpr uint16_t kNoTile = 0xffff;
 struct GemmParams {
     alignas(64) CUtensorMap maps[kMaxGemmOps * kMapsPerOp];
     DevProblem prob[kMaxGemmOps];
-    int32_t n_problems, total_tiles;
+    // Worker w runs, in round i, tile order[w + i * workers] (kNoTile = nothing) when use_order is set,
+    // otherwise tile w + i * workers.
+    uint16_t order[kMaxOrder];
+    int32_t n_problems, total_tiles, rounds, use_order;
     int* status;
 };
 
@@ -211,6 +215,10 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
 }
+// C += tile: the addition is done by the memory system in the output's type, once per element
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // all but the newest N stores of this thread have finished reading their shared-memory source
 template <int N>
@@ -341,39 +349,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// 32 consecutive values of one row -> bf16 (or fp32) at `row_off` + n; nv = valid columns (<= 32)
-__device__ __forceinline__ void store_row32(void* base, int64_t row_off, int n, int nv, const float (&v)[32], bool f32) {
-    if (f32) {
-        float* p = static_cast<float*>(base) + row_off + n;
-        if (nv == 32) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-                *reinterpret_cast<float4*>(p + 4 * i) = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (i < nv) p[i] = v[i];
-        }
-    } else {
-        __nv_bfloat16* p = static_cast<__nv_bfloat16*>(base) + row_off + n;
-        if (nv == 32) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint4 q;
-                q.x = pack_bf16(v[8 * i + 0], v[8 * i + 1]);
-                q.y = pack_bf16(v[8 * i + 2], v[8 * i + 3]);
-                q.z = pack_bf16(v[8 * i + 4], v[8 * i + 5]);
-                q.w = pack_bf16(v[8 * i + 6], v[8 * i + 7]);
-                *reinterpret_cast<uint4*>(p + 8 * i) = q;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (i < nv) p[i] = __float2bfloat16_rn(v[i]);
-        }
-    }
-}
-
 // Staging images for the TMA tile stores.  A warp owns 4 KB: either one image of 32 rows x 128 bytes in the
 // 128-byte swizzle (64 bf16 or 32 fp32 columns; 16-byte chunk j of row r sits at chunk j ^ (r & 7)), or two
 // "slots" of 32 rows x 64 bytes in the 64-byte swizzle (32 bf16 columns; chunk j of row r at j ^ ((r >> 1) & 3)).
@@ -385,11 +360,12 @@ __device__ __forceinline__ void stage_begin(int lane) {
     if (lane == 0) bulk_wait_read<KEEP>();
     __syncwarp();
 }
-__device__ __forceinline__ void stage_commit(const CUtensorMap* map, uint32_t buf, int x, int y, int lane) {
+__device__ __forceinline__ void stage_commit(const CUtensorMap* map, uint32_t buf, int x, int y, int lane, bool add = false) {
     fence_async_smem();
     __syncwarp();
     if (lane == 0) {
-        tma_store_2d(map, buf, x, y);
+        if (add) tma_reduce_add_2d(map, buf, x, y);
+        else tma_store_2d(map, buf, x, y);
         bulk_commit();
     }
 }
@@ -427,57 +403,12 @@ __device__ __forceinline__ void stage_bf16x32(uint32_t slot, int lane, const flo
                      : "memory");
 }
 
-// Per-warp transposition buffers: 32 rows x 32 bf16 columns, 64 bytes per row, the four 16-byte chunks
-// of a row permuted by (chunk ^ ((row >> 1) & 3)) so that both access patterns below are conflict-free.
-//   "row" pattern:  lane = row, a lane touches the four chunks of its row (what tcgen05.ld delivers);
-//   "line" pattern: 4 lanes per row, 8 rows per instruction (coalesced 64-byte global segments).
+// Landing buffer of the saved activations: 32 rows x 32 bf16 columns, 64 bytes per row, the four 16-byte
+// chunks of a row permuted by (chunk ^ ((row >> 1) & 3)) so that both access patterns are conflict-free:
+//   "line" pattern: 4 lanes per row, 8 rows per instruction (coalesced 64-byte global segments);
+//   "row" pattern:  lane = row, a lane touches the four chunks of its row (the layout of tcgen05.ld).
 __device__ __forceinline__ uint32_t epi_chunk_addr(uint32_t buf, int row, int chunk) {
     return buf + row * 64 + ((chunk ^ ((row >> 1) & 3)) << 4);
-}
-
-// registers (one row per lane) -> buffer -> global, bf16.  Rows >= M and columns >= N are not written.
-// accumulate: the previous contents of C are added (in fp32) before the store.
-__device__ __forceinline__ void staged_store32(uint32_t buf, __nv_bfloat16* C, int64_t ldc, int m_warp, int n, int M, int N,
-                                               const float (&v)[32], int lane, bool accumulate) {
-#pragma unroll
-    for (int c = 0; c < 4; ++c)
-        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(epi_chunk_addr(buf, lane, c)),
-                     "r"(pack_bf16(v[8 * c + 0], v[8 * c + 1])), "r"(pack_bf16(v[8 * c + 2], v[8 * c + 3])),
-                     "r"(pack_bf16(v[8 * c + 4], v[8 * c + 5])), "r"(pack_bf16(v[8 * c + 6], v[8 * c + 7]))
-                     : "memory");
-    __syncwarp();
-    const int c = lane & 3;
-    const int col = n + 8 * c;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int row = 8 * i + (lane >> 2);
-        uint4 q;
-        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(q.x), "=r"(q.y), "=r"(q.z), "=r"(q.w) : "r"(epi_chunk_addr(buf, row, c)));
-        if (m_warp + row < M && col < N) {
-            __nv_bfloat16* g = C + static_cast<int64_t>(m_warp + row) * ldc + col;
-            if (col + 8 <= N) {
-                if (accumulate) {
-                    const uint4 o = *reinterpret_cast<const uint4*>(g);
-                    q.x = pack_bf16(bf16_lo(q.x) + bf16_lo(o.x), bf16_hi(q.x) + bf16_hi(o.x));
-                    q.y = pack_bf16(bf16_lo(q.y) + bf16_lo(o.y), bf16_hi(q.y) + bf16_hi(o.y));
-                    q.z = pack_bf16(bf16_lo(q.z) + bf16_lo(o.z), bf16_hi(q.z) + bf16_hi(o.z));
-                    q.w = pack_bf16(bf16_lo(q.w) + bf16_lo(o.w), bf16_hi(q.w) + bf16_hi(o.w));
-                }
-                *reinterpret_cast<uint4*>(g) = q;
-            } else {
-                const uint32_t w[4] = {q.x, q.y, q.z, q.w};
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                    if (col + e < N) {
-                        float f = (e & 1) ? bf16_hi(w[e >> 1]) : bf16_lo(w[e >> 1]);
-                        if (accumulate) f += __bfloat162float(g[e]);
-                        g[e] = __float2bfloat16_rn(f);
-                    }
-                }
-            }
-        }
-    }
-    __syncwarp();
 }
 
 // global (bf16, rows m_warp.. x columns n..n+31) -> registers in the coalesced "line" pattern.  Split in
@@ -525,35 +456,20 @@ __device__ __forceinline__ void staged_load32_finish(uint32_t buf, const uint4 (
     __syncwarp();
 }
 
-__device__ __forceinline__ void load_row32(const void* base, int64_t row_off, int n, int nv, float (&v)[32], bool f32) {
-    if (f32) {
-        const float* p = static_cast<const float*>(base) + row_off + n;
-        if (nv == 32) {
-#pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float4 q = *reinterpret_cast<const float4*>(p + 4 * i);
-                v[4 * i] = q.x; v[4 * i + 1] = q.y; v[4 * i + 2] = q.z; v[4 * i + 3] = q.w;
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = i < nv ? p[i] : 0.f;
-        }
-    } else {
-        const unsigned short* p = static_cast<const unsigned short*>(base) + row_off + n;
-        if (nv == 32) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint4 q = *reinterpret_cast<const uint4*>(p + 8 * i);
-                v[8 * i + 0] = bf16_lo(q.x); v[8 * i + 1] = bf16_hi(q.x);
-                v[8 * i + 2] = bf16_lo(q.y); v[8 * i + 3] = bf16_hi(q.y);
-                v[8 * i + 4] = bf16_lo(q.z); v[8 * i + 5] = bf16_hi(q.z);
-                v[8 * i + 6] = bf16_lo(q.w); v[8 * i + 7] = bf16_hi(q.w);
-            }
-        } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = i < nv ? __uint_as_float(static_cast<uint32_t>(p[i]) << 16) : 0.f;
-        }
+// tile of worker `worker` in round `i`, or -1
+__device__ __forceinline__ int scheduled_tile(const GemmParams& P, int worker, int n_workers, int i) {
+    const int pos = worker + i * n_workers;
+    if (P.use_order) {
+        const int t = P.order[pos];
+        return t == kNoTile ? -1 : t;
     }
+    return pos < P.total_tiles ? pos : -1;
+}
+
+// v[i] += bias of column i, where lane i of the warp holds that column's bias
+__device__ __forceinline__ void add_bias32(float (&v)[32], float b) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] += __shfl_sync(0xffffffffu, b, i);
 }
 
 __device__ __forceinline__ const DevProblem& find_problem(const GemmParams& P, int tile) {
@@ -589,6 +505,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     auto tfull_bar = [&](int a) { return bar0 + 8u * (2 * kStages + a); };
     auto tempty_bar = [&](int a) { return bar0 + 8u * (2 * kStages + 2 + a); };
 
+    // Launched with programmatic stream serialization: the next launch of this engine may place its CTAs as
+    // soon as SMs free up and set itself up; it reads or writes no global memory before the wait below.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;   // 0 = leader: issues the MMAs, owns full/tmem_empty
     const bool leader = cta_rank == 0;
@@ -606,9 +525,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        if (worker < P.total_tiles) {
+        const int tile0 = P.rounds > 0 ? scheduled_tile(P, worker, n_workers, 0) : -1;
+        if (tile0 >= 0) {
             // warm the descriptors of the first tile while TMEM is allocated and the CTAs meet
-            const DevProblem& Q0 = find_problem(P, worker);
+            const DevProblem& Q0 = find_problem(P, tile0);
             prefetch_tensormap(&P.maps[Q0.map_a[0]]);
             prefetch_tensormap(&P.maps[Q0.map_b[0][cta_rank]]);
         }
@@ -627,6 +547,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
     if (PAIR) cluster_sync_all();     // the peer's barriers are initialised before anything signals them
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
+    // everything earlier in the stream has completed and its writes are visible after this
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer (both CTAs of a pair)
@@ -634,7 +556,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             int stage = 0;
             uint32_t phase = 0;
             bool ok = true;
-            for (int tile = worker; ok && tile < P.total_tiles; tile += n_workers) {
+            for (int round = 0; ok && round < P.rounds; ++round) {
+                const int tile = scheduled_tile(P, worker, n_workers, round);
+                if (tile < 0) continue;
                 const DevProblem& Q = find_problem(P, tile);
                 const int local = tile - Q.tile_start;
                 const int m0 = (local % Q.tiles_m) * kTileM + static_cast<int>(cta_rank) * BM;
@@ -757,7 +681,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             uint32_t phase = 0;
             int it = 0;
             bool ok = true;
-            for (int tile = worker; ok && tile < P.total_tiles; tile += n_workers, ++it) {
+            for (int round = 0; ok && round < P.rounds; ++round) {
+                const int tile = scheduled_tile(P, worker, n_workers, round);
+                if (tile < 0) continue;
                 const DevProblem& Q = find_problem(P, tile);
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1u;
@@ -805,6 +731,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         tc_commit(tfull_bar(acc));
                     }
                 }
+                ++it;
             }
         }
     } else {
@@ -815,17 +742,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
         const uint32_t buf_out = sEpi + ew * 2 * kEpiSlotBytes, buf_in = buf_out + kEpiSlotBytes;
         int it = 0;
         bool ok = true;
-        for (int tile = worker; ok && tile < P.total_tiles; tile += n_workers, ++it) {
+        for (int round = 0; ok && round < P.rounds; ++round) {
+            const int tile = scheduled_tile(P, worker, n_workers, round);
+            if (tile < 0) continue;
             const DevProblem& Q = find_problem(P, tile);
             const int local = tile - Q.tile_start;
             const int m_warp = (local % Q.tiles_m) * kTileM + static_cast<int>(cta_rank) * BM + quad * 32;   // first row of this warp
-            const int m = m_warp + lane;
             const int n0 = (local / Q.tiles_m) * Q.n_per_tile;
             const int acc = it & 1;
             const uint32_t acc_phase = (it >> 1) & 1u;
             const int epi = Q.epi;
             const int QM = Q.M, QN = Q.N;
-            const bool tma = Q.tma_out != 0;
             const CUtensorMap* mc0 = &P.maps[Q.map_c[0]];
             const CUtensorMap* mc1 = &P.maps[Q.map_c[1]];
             const CUtensorMap* mc2 = &P.maps[Q.map_c[2]];
@@ -839,10 +766,21 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
             if (need_hb) staged_load32_issue(Hbp, Q.ldh, m_warp, n0 + half * 128, QM, QN, hbq, lane);
             // the second slot doubles as the landing buffer of those loads: no store of an earlier tile may still read it
             if (need_h) stage_begin<0>(lane);
+            // bias of this warp's 128 columns, one column per lane and 32-column chunk (fetched while the tile is computed)
+            float breg[4] = {0.f, 0.f, 0.f, 0.f};
+            const bool has_bias = Q.bias != nullptr;
+            if (has_bias) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int col = n0 + half * 128 + 32 * j + lane;
+                    if (col < QN)
+                        breg[j] = Q.bias_f32 ? static_cast<const float*>(Q.bias)[col]
+                                             : __uint_as_float(static_cast<uint32_t>(static_cast<const unsigned short*>(Q.bias)[col]) << 16);
+                }
+            }
             if (!(ok = mbar_wait<PAIR>(tfull_bar(acc), acc_phase, abort_flag, 4, P.status))) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
-            const bool row_ok = m < QM;
             const bool warp_rows = m_warp < QM;          // any row of this warp inside the output
             if (epi == EPI_SWIGLU) {
                 // accumulator columns [0,128) = gate, [128,256) = up for hidden units n0 .. n0+127.
@@ -878,7 +816,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     for (int i = 0; i < 32; ++i) g[i] = g[i] * sigmoidf_(g[i]) * u[i];
                     put(mc2, n, g);
                 }
-            } else if (epi == EPI_STORE && tma && !Q.out_f32) {
+            } else if (epi == EPI_STORE && !Q.out_f32) {
                 // bf16 output: two chunks of 64 columns, each one 32 x 128-byte image
 #pragma unroll 1
                 for (int c = 0; c < 2; ++c) {
@@ -895,18 +833,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         v0[i] = __uint_as_float(r0[i]);
                         v1[i] = __uint_as_float(r1[i]);
                     }
-                    if (Q.bias) {
-                        float b[32];
-                        load_row32(Q.bias, 0, n, min(32, QN - n), b, Q.bias_f32 != 0);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v0[i] += b[i];
-                        load_row32(Q.bias, 0, n + 32, min(32, QN - n - 32), b, Q.bias_f32 != 0);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v1[i] += b[i];
+                    if (has_bias) {
+                        add_bias32(v0, c ? breg[2] : breg[0]);
+                        add_bias32(v1, c ? breg[3] : breg[1]);
                     }
                     stage_begin<0>(lane);
                     stage_bf16x64(buf_out, lane, v0, v1);
-                    stage_commit(mc0, buf_out, n, m_warp, lane);
+                    stage_commit(mc0, buf_out, n, m_warp, lane, Q.accumulate != 0);
                 }
             } else if (epi == EPI_GELU_ERF || epi == EPI_GELU_TANH) {
                 // H = acc + bias and A = GELU(H), 64 columns at a time
@@ -925,14 +858,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                         v0[i] = __uint_as_float(r0[i]);
                         v1[i] = __uint_as_float(r1[i]);
                     }
-                    if (Q.bias) {
-                        float b[32];
-                        load_row32(Q.bias, 0, n, min(32, QN - n), b, Q.bias_f32 != 0);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v0[i] += b[i];
-                        load_row32(Q.bias, 0, n + 32, min(32, QN - n - 32), b, Q.bias_f32 != 0);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v1[i] += b[i];
+                    if (has_bias) {
+                        add_bias32(v0, c ? breg[2] : breg[0]);
+                        add_bias32(v1, c ? breg[3] : breg[1]);
                     }
                     stage_begin<0>(lane);
                     stage_bf16x64(buf_out, lane, v0, v1);
@@ -952,8 +880,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     stage_commit(mc1, buf_out, n, m_warp, lane);
                 }
             } else {
-                // 32 columns at a time: fp32 outputs, accumulating outputs and the derivative epilogues
-                const int64_t c_off = static_cast<int64_t>(m) * Q.ldc;
+                // 32 columns at a time: fp32 outputs and the derivative epilogues
 #pragma unroll 1
                 for (int c = 0; c < 4; ++c) {
                     const int col = half * 128 + c * 32;
@@ -966,27 +893,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                     float v[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    if (Q.bias) {
-                        float b[32];
-                        load_row32(Q.bias, 0, n, nv, b, Q.bias_f32 != 0);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] += b[i];
-                    }
-                    if (epi == EPI_STORE) {
-                        if (tma) {                         // fp32 output: one 32 x 128-byte image
-                            if (warp_rows) {
-                                stage_begin<0>(lane);
-                                stage_f32x32(buf_out, lane, v);
-                                stage_commit(mc0, buf_out, n, m_warp, lane);
-                            }
-                        } else if (!Q.out_f32) {           // C += acc, bf16
-                            if (warp_rows) staged_store32(buf_out, static_cast<__nv_bfloat16*>(Q.C), Q.ldc, m_warp, n, QM, QN, v, lane, true);
-                        } else if (row_ok) {               // C += acc, fp32
-                            float o[32];
-                            load_row32(Q.C, c_off, n, nv, o, true);
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) v[i] += o[i];
-                            store_row32(Q.C, c_off, n, nv, v, true);
+                    if (has_bias) add_bias32(v, c == 0 ? breg[0] : c == 1 ? breg[1] : c == 2 ? breg[2] : breg[3]);
+                    if (epi == EPI_STORE) {                // fp32 output: one 32 x 128-byte image
+                        if (warp_rows) {
+                            stage_begin<0>(lane);
+                            stage_f32x32(buf_out, lane, v);
+                            stage_commit(mc0, buf_out, n, m_warp, lane, Q.accumulate != 0);
                         }
                     } else if (epi == EPI_DGELU_ERF || epi == EPI_DGELU_TANH) {
                         float h[32];
@@ -1032,6 +944,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 if (PAIR) mbar_arrive_cluster(map_to_cta(tempty_bar(acc), 0));
                 else mbar_arrive(tempty_bar(acc));
             }
+            ++it;
         }
         if (lane == 0) bulk_wait_all();            // this warp's tile stores have landed
     }
@@ -1203,6 +1116,40 @@ ecospa_status_t gemm_setup() {
     return st;
 }
 
+// Tile schedule.  Tiles are numbered op by op, longest contraction first.  With few tiles per worker the
+// plain stride (worker w takes w, w + workers, ...) can leave one worker with several long tiles, so the
+// tiles are handed out longest first to the least-loaded worker (ties: lowest worker) and the result is
+// written as a table; with many tiles per worker the stride is balanced enough and needs no table.
+void build_schedule(GemmParams& gp, int workers) {
+    const int tiles = gp.total_tiles;
+    gp.use_order = 0;
+    gp.rounds = static_cast<int32_t>(ceil_div(tiles, workers));
+    if (tiles <= workers || tiles > kMaxOrder || tiles >= kNoTile) return;
+    static thread_local int64_t load[256];
+    static thread_local int32_t len[256];
+    static thread_local uint16_t lists[256][64];
+    if (workers > 256) return;
+    for (int w = 0; w < workers; ++w) load[w] = len[w] = 0;
+    int max_len = 0;
+    int pi = 0;
+    for (int t = 0; t < tiles; ++t) {
+        while (pi + 1 < gp.n_problems && gp.prob[pi + 1].tile_start <= t) ++pi;
+        const int64_t cost = gp.prob[pi].kblocks + 4;     // main loop + a fixed per-tile share
+        int best = 0;
+        for (int w = 1; w < workers; ++w)
+            if (load[w] < load[best]) best = w;
+        if (len[best] >= 64) return;                       // not expected; keep the stride
+        lists[best][len[best]++] = static_cast<uint16_t>(t);
+        load[best] += cost;
+        max_len = std::max(max_len, static_cast<int>(len[best]));
+    }
+    if (static_cast<int64_t>(max_len) * workers > kMaxOrder) return;
+    for (int i = 0; i < max_len; ++i)
+        for (int w = 0; w < workers; ++w) gp.order[w + i * workers] = i < len[w] ? lists[w][i] : kNoTile;
+    gp.rounds = max_len;
+    gp.use_order = 1;
+}
+
 }  // namespace
 
 ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t stream) {
@@ -1294,9 +1241,8 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
             Q.kblocks += static_cast<int32_t>(ceil_div(ks.K, BK));
             Q.kb_end[s] = Q.kblocks;
         }
-        // outputs leave through TMA tile stores unless they are added to what C already holds
-        Q.tma_out = op.accumulate ? 0 : 1;
-        if (Q.tma_out) {
+        // outputs leave through TMA tile stores (a reducing store when they are added to what C holds)
+        {
             const bool wide = op.epi == EPI_STORE || op.epi == EPI_GELU_ERF || op.epi == EPI_GELU_TANH;
             void* outs[3] = {op.C, op.C2, op.C3};
             for (int o = 0; o < 3; ++o) {
@@ -1314,30 +1260,29 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
     gp.n_problems = n_ops;
     gp.total_tiles = tiles;
     gp.status = g_status_ptr;
-    if (!pair) {
-        const int grid = std::min(tiles, g_num_sms);
-        gemm_kernel<false><<<grid, kThreads, kSmemBytes, stream>>>(gp);
-        return check_launch("gemm_kernel");
-    }
+    const int workers = pair ? std::min(tiles, g_max_pairs) : std::min(tiles, g_num_sms);
+    build_schedule(gp, workers);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(2 * std::min(tiles, g_max_pairs));
+    cfg.gridDim = dim3(pair ? 2 * workers : workers);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kSmemBytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 2;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    const cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_kernel<true>, gp);
+    cfg.numAttrs = pair ? 2 : 1;
+    const cudaError_t e = pair ? cudaLaunchKernelEx(&cfg, gemm_kernel<true>, gp) : cudaLaunchKernelEx(&cfg, gemm_kernel<false>, gp);
     if (e != cudaSuccess) {
-        set_cuda_error(e, "gemm_kernel (pair) launch");
+        set_cuda_error(e, "gemm_kernel launch");
         cudaGetLastError();
         return ECOSPA_ERR_CUDA;
     }
-    return check_launch("gemm_kernel (pair)");
+    return check_launch("gemm_kernel");
 }
 
 }  // namespace ecospa

@@ -313,16 +313,21 @@ GemmOp proj_op(const Stored& X, const Stored& W, int64_t T, int64_t d_m, int64_t
 // Weight gradients contract over the T tokens and have few output tiles, so on their own they would keep
 // most SMs idle behind one long tile.  The token range is therefore cut into `splits` ranges computed as
 // separate ops of the same launch into fp32 partial buffers, which the finishing launch (post_kernel) adds up in split order.
-int wgrad_splits(int64_t rows_out, int64_t cols_out, int64_t T) {
-    const int64_t tiles = ceil_div(rows_out, 256) * ceil_div(cols_out, 256);
-    int64_t s = 74 / tiles;                       // aim at one wave of CTA pairs
-    if (s < 3) s = 1;                             // a 2-way split does not pay for its reduction pass
+constexpr int64_t kWorkers = 74;                  // CTA pairs the engine keeps resident
+// Cost of a product in k-blocks of 256x256 tiles (what one worker spends on it if it ran alone).
+int64_t gemm_cost(int64_t M, int64_t N, int64_t K) { return ceil_div(M, 256) * ceil_div(N, 256) * ceil_div(K, 64); }
+// `launch_cost` = cost of every product of the launch.  The scheduler hands tiles out longest first, so a
+// tile longer than a worker's fair share of the launch sets the duration: cut the tokens until it is not.
+int wgrad_splits(int64_t rows_out, int64_t cols_out, int64_t T, int64_t launch_cost) {
+    const int64_t share = std::max<int64_t>(launch_cost / kWorkers, 1);
+    int64_t s = ceil_div(ceil_div(T, 64), share);
     s = std::min<int64_t>(s, T / 1024);            // at least 16 k-blocks per range
     s = std::min<int64_t>(s, 6);
     return static_cast<int>(std::max<int64_t>(s, 1));
 }
+// Upper bound of the partial buffers over every launch this product can be part of (its own cost alone).
 size_t wgrad_need(int64_t rows_out, int64_t cols_out, int64_t T) {
-    const int S = wgrad_splits(rows_out, cols_out, T);
+    const int S = wgrad_splits(rows_out, cols_out, T, gemm_cost(rows_out, cols_out, T));
     return S > 1 ? arena_need(static_cast<size_t>(S) * rows_out * round_up(cols_out, 4) * 4) : 0;
 }
 struct PendingReduce {
@@ -335,14 +340,14 @@ struct PendingReduce {
 // Appends 1 or `splits` ops to ops[n_ops...] and returns the new op count.  `reserve` = ops the caller
 // still has to append after this one; the split count is reduced so that everything fits kMaxGemmOps.
 int add_wgrad(Ctx& cx, GemmOp* ops, int n_ops, const Stored& Xs, const Stored& dYs, int64_t rows_out, int64_t cols_out,
-              int64_t T, void* out, int64_t ld_out, PendingReduce* red, int reserve) {
+              int64_t T, void* out, int64_t ld_out, PendingReduce* red, int reserve, int64_t launch_cost) {
     GemmOp op;
     op.M = rows_out; op.N = cols_out; op.n_kseg = 1;
     op.seg[0].a = Xs; op.seg[0].a_mn = true;
     op.seg[0].b[0] = dYs; op.seg[0].b_mn = true;
     op.epi = EPI_STORE;
-    int S = wgrad_splits(rows_out, cols_out, T);
-    S = std::max(1, std::min(S, kMaxGemmOps - n_ops - reserve));
+    int S = wgrad_splits(rows_out, cols_out, T, launch_cost);
+    S = std::max(1, std::min(S, (kMaxGemmOps - n_ops - reserve) / std::max(1, reserve)));
     if (cx.st != ECOSPA_OK) return n_ops;
     if (n_ops + 1 + reserve > kMaxGemmOps) {
         cx.st = ECOSPA_ERR_INVALID;
@@ -469,8 +474,9 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
     GemmOp ops[kMaxGemmOps];
     PendingReduce red[2];
     int n_ops = 0;
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n, T, dWq_c, ld_dw, &red[0], wk_c ? 2 : 1);
-    if (wk_c) n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n, T, dWk_c, ld_dw, &red[1], 1);
+    const int64_t cost = (wk_c ? 2 : 1) * (gemm_cost(d_m, n, T) + gemm_cost(T, d_m, n));
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n, T, dWq_c, ld_dw, &red[0], wk_c ? 2 : 1, cost);
+    if (wk_c) n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n, T, dWk_c, ld_dw, &red[1], 1, cost);
     if (cx.st != ECOSPA_OK) return cx.st;
     // dX = dQ W_Q^T (+ dK W_K^T): weights stored d_m x n are K-major B operands here
     GemmOp& dx = ops[n_ops++];
@@ -536,8 +542,9 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     PendingReduce red[2];
     int n_ops = 0;
     // dW_O (n x d_m) = Ctx^T dOut ; dW_V (d_m x n) = X^T dV
-    n_ops = add_wgrad(cx, ops, n_ops, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red[0], 3);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n, T, dWv_c, ld_dwv, &red[1], 2);
+    const int64_t cost = gemm_cost(n, d_m, T) + gemm_cost(d_m, n, T) + gemm_cost(T, n, d_m) + gemm_cost(T, d_m, n);
+    n_ops = add_wgrad(cx, ops, n_ops, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red[0], 3, cost);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n, T, dWv_c, ld_dwv, &red[1], 2, cost);
     if (cx.st != ECOSPA_OK) return cx.st;
     // dCtx (T x n) = dOut W_O^T : W_O stored n x d_m = [N][K]
     GemmOp& dc = ops[n_ops++];
@@ -605,9 +612,10 @@ extern "C" ecospa_status_t ecospa_coupled_qkv_bwd(const void* X, int64_t ldx, in
     GemmOp ops[kMaxGemmOps];
     PendingReduce red[3];
     int n_ops = 0;
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n_qk, T, dWq_c, ld_dwqk, &red[0], 3);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n_qk, T, dWk_c, ld_dwqk, &red[1], 2);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n_vo, T, dWv_c, ld_dwv, &red[2], 1);
+    const int64_t cost = 2 * gemm_cost(d_m, n_qk, T) + gemm_cost(d_m, n_vo, T) + gemm_cost(T, d_m, 2 * n_qk + n_vo);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n_qk, T, dWq_c, ld_dwqk, &red[0], 3, cost);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n_qk, T, dWk_c, ld_dwqk, &red[1], 2, cost);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n_vo, T, dWv_c, ld_dwv, &red[2], 1, cost);
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& dx = ops[n_ops++];
     dx.M = T; dx.N = d_m; dx.n_kseg = 3;
@@ -637,7 +645,8 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd_o(const void* Ctxm, int64_t ld_
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp ops[kMaxGemmOps];
     PendingReduce red;
-    int n_ops = add_wgrad(cx, ops, 0, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red, 1);   // dW_O (n x d_m) = Ctx^T dOut
+    const int64_t cost = gemm_cost(n, d_m, T) + gemm_cost(T, n, d_m);
+    int n_ops = add_wgrad(cx, ops, 0, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red, 1, cost);   // dW_O (n x d_m) = Ctx^T dOut
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& dc = ops[n_ops++];                                                        // dCtx = dOut W_O^T
     dc.M = T; dc.N = n; dc.n_kseg = 1;
@@ -743,9 +752,11 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     GemmOp ops[kMaxGemmOps];
     PendingReduce red[3];
     int n_ops = 0;
-    n_ops = add_wgrad(cx, ops, n_ops, As, dYs, k, d_m, T, dW2_c, ld_dw2, &red[0], sw ? 3 : 2);          // dW_2 (k x d_m) = A^T dY
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1);           // dW_1 (d_m x k) = X^T dH
-    if (sw) n_ops = add_wgrad(cx, ops, n_ops, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1); // dW_up = X^T dH_up
+    const int nw = sw ? 2 : 1;
+    const int64_t cost = gemm_cost(k, d_m, T) + nw * gemm_cost(d_m, k, T) + gemm_cost(T, d_m, nw * k);
+    n_ops = add_wgrad(cx, ops, n_ops, As, dYs, k, d_m, T, dW2_c, ld_dw2, &red[0], sw ? 3 : 2, cost);          // dW_2 (k x d_m) = A^T dY
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1, cost);           // dW_1 (d_m x k) = X^T dH
+    if (sw) n_ops = add_wgrad(cx, ops, n_ops, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1, cost); // dW_up = X^T dH_up
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& dx = ops[n_ops++];                                                    // dX = dH W_1^T (+ dH_up W_up^T)
     dx.M = T; dx.N = d_m; dx.n_kseg = sw ? 2 : 1;
