@@ -45,8 +45,9 @@ __global__ void __launch_bounds__(kThreads) cast_f32_bf16_kernel(const float* __
 
 // Column sums (bias gradients) of up to two bf16 matrices with the same number of rows, two launches:
 // partial[chunk][c] over tiles of kSumRows rows x 64 columns (8 lanes cover a row's 128 bytes with
-// 16-byte loads, the block covers 32 rows per pass, 4 passes in flight), then a fixed-order sum of the chunks.
-constexpr int kSumRows = 512;
+// 16-byte loads, the block covers 32 rows per pass, all 4 passes in flight at once: the kernel is one round
+// of loads deep and its grid is large), then a fixed-order sum of the chunks.
+constexpr int kSumRows = 128;
 constexpr int kSumCols = 64;
 struct ColsumJob {
     const uint16_t* M;
