@@ -295,6 +295,11 @@ __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
     asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
 }
+__device__ __forceinline__ float ex2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 // Phi of two values
 __device__ __forceinline__ f32x2 normal_cdf2(float x0, float x1) {
     const f32x2 xc = pack2(fminf(fmaxf(x0, -4.5f), 4.5f), fminf(fmaxf(x1, -4.5f), 4.5f));
@@ -323,8 +328,12 @@ __device__ __forceinline__ void dgelu_erf32(float (&v)[32], const float (&h)[32]
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
         const f32x2 hh = pack2(h[i], h[i + 1]);
-        const f32x2 pdf = pack2(0.39894228040143268f * __expf(-0.5f * h[i] * h[i]),
-                                0.39894228040143268f * __expf(-0.5f * h[i + 1] * h[i + 1]));
+        // phi(h) = 2^(-h^2 log2(e)/2 - log2(sqrt(2 pi))): one packed multiply-add and one exponential per element
+        const f32x2 ex = fma2(mul2(hh, hh), pack2(-0.72134752044448170f, -0.72134752044448170f),
+                              pack2(-1.3257480647361593f, -1.3257480647361593f));
+        float e0, e1;
+        unpack2(ex, e0, e1);
+        const f32x2 pdf = pack2(ex2_fast(e0), ex2_fast(e1));
         const f32x2 d = fma2(hh, pdf, normal_cdf2(h[i], h[i + 1]));
         const f32x2 r = mul2(pack2(v[i], v[i + 1]), d);
         unpack2(r, v[i], v[i + 1]);

@@ -43,6 +43,25 @@ __global__ void __launch_bounds__(kThreads) cast_f32_bf16_kernel(const float* __
     }
 }
 
+// These helpers are launched with programmatic stream serialization, like the GEMM engine: their blocks may be
+// placed while the previous kernel drains, and touch no global memory before pdl_wait().
+__device__ __forceinline__ void pdl_start() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <typename Params>
+cudaError_t launch_pdl(void (*kernel)(Params), dim3 grid, cudaStream_t stream, const Params& p) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, p);
+}
+
 // Column sums (bias gradients) of up to two bf16 matrices with the same number of rows, two launches:
 // partial[chunk][c] over tiles of kSumRows rows x 64 columns (8 lanes cover a row's 128 bytes with
 // 16-byte loads, the block covers 32 rows per pass, all 4 passes in flight at once: the kernel is one round
@@ -64,6 +83,8 @@ struct ColsumParams {
 
 __global__ void __launch_bounds__(kThreads) colsum_partial_kernel(const __grid_constant__ ColsumParams P) {
     __shared__ float red[32][kSumCols + 1];
+    pdl_start();
+    pdl_wait();
     int ji = 0, ct = blockIdx.x;
     while (ji + 1 < P.n_jobs && ct >= P.job[ji].col_tiles) {
         ct -= P.job[ji].col_tiles;
@@ -129,7 +150,11 @@ struct PostParams {
     ColsumParams cs;
     int32_t n_red, red_blocks, out_f32, pad_;
 };
+__host__ __device__ inline int64_t round_up32(int64_t v) { return (v + 31) & ~int64_t(31); }
 __global__ void __launch_bounds__(kThreads) post_kernel(const __grid_constant__ PostParams P) {
+    __shared__ float part[8][32];
+    pdl_start();
+    pdl_wait();
     if (static_cast<int>(blockIdx.x) < P.red_blocks) {
         int ji = 0;
         while (ji + 1 < P.n_red && static_cast<int>(blockIdx.x) >= P.red[ji + 1].blk_start) ++ji;
@@ -155,18 +180,30 @@ __global__ void __launch_bounds__(kThreads) post_kernel(const __grid_constant__ 
         }
         return;
     }
-    int64_t c = static_cast<int64_t>(blockIdx.x - P.red_blocks) * kThreads + threadIdx.x;
+    // column-sum finals: a block takes 32 columns; warp g adds chunks g, g + 8, ... and warp 0 adds the 8 sums
+    const int g = threadIdx.x >> 5;
+    int64_t c = static_cast<int64_t>(blockIdx.x - P.red_blocks) * 32 + (threadIdx.x & 31);
     int ji = 0;
-    while (ji < P.cs.n_jobs && c >= P.cs.job[ji].cols) {
-        c -= P.cs.job[ji].cols;
+    while (ji < P.cs.n_jobs && c >= round_up32(P.cs.job[ji].cols)) {
+        c -= round_up32(P.cs.job[ji].cols);
         ++ji;
     }
-    if (ji >= P.cs.n_jobs) return;
-    const ColsumJob& J = P.cs.job[ji];
+    const bool live = ji < P.cs.n_jobs && c < P.cs.job[ji].cols;
     float s = 0.f;
-    for (int k = 0; k < P.cs.chunks; ++k) s += J.partial[static_cast<int64_t>(k) * J.cols + c];
-    if (P.out_f32) static_cast<float*>(J.out)[c] = s;
-    else static_cast<__nv_bfloat16*>(J.out)[c] = __float2bfloat16_rn(s);
+    if (live) {
+        const float* p = P.cs.job[ji].partial + c;
+        const int64_t cols = P.cs.job[ji].cols;
+        for (int k = g; k < P.cs.chunks; k += 8) s += p[static_cast<int64_t>(k) * cols];
+    }
+    part[g][threadIdx.x & 31] = s;
+    __syncthreads();
+    if (g == 0 && live) {
+        float t = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t += part[i][threadIdx.x];
+        if (P.out_f32) static_cast<float*>(P.cs.job[ji].out)[c] = t;
+        else static_cast<__nv_bfloat16*>(P.cs.job[ji].out)[c] = __float2bfloat16_rn(t);
+    }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -264,7 +301,13 @@ ColsumParams colsum_begin(Ctx& cx, const Stored& M1, void* out1, const Stored& M
         }
         tiles += P.job[i].col_tiles;
     }
-    colsum_partial_kernel<<<dim3(tiles, P.chunks), kThreads, 0, cx.stream>>>(P);
+    const cudaError_t e = launch_pdl(colsum_partial_kernel, dim3(tiles, P.chunks), cx.stream, P);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "colsum_partial_kernel launch");
+        cudaGetLastError();
+        cx.st = ECOSPA_ERR_CUDA;
+        return P;
+    }
     cx.st = check_launch("colsum_partial_kernel");
     return P;
 }
@@ -402,11 +445,15 @@ void finish(Ctx& cx, const PendingReduce* red, int n_red, const ColsumParams& cs
         blocks += J.n_blk;
     }
     P.red_blocks = blocks;
-    int64_t total_cols = 0;
-    for (int i = 0; i < cs.n_jobs; ++i) total_cols += cs.job[i].cols;
-    blocks += static_cast<int>(ceil_div(total_cols, kThreads));
+    for (int i = 0; i < cs.n_jobs; ++i) blocks += static_cast<int>(round_up32(cs.job[i].cols) / 32);
     if (blocks == 0) return;
-    post_kernel<<<blocks, kThreads, 0, cx.stream>>>(P);
+    const cudaError_t e = launch_pdl(post_kernel, dim3(blocks), cx.stream, P);
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "post_kernel launch");
+        cudaGetLastError();
+        cx.st = ECOSPA_ERR_CUDA;
+        return;
+    }
     cx.st = check_launch("post_kernel");
 }
 
