@@ -361,10 +361,11 @@ constexpr int64_t kWorkers = 74;                  // CTA pairs the engine keeps 
 // Cost of a product in k-blocks of 256x256 tiles (what one worker spends on it if it ran alone).
 int64_t gemm_cost(int64_t M, int64_t N, int64_t K) { return ceil_div(M, 256) * ceil_div(N, 256) * ceil_div(K, 64); }
 // `launch_cost` = cost of every product of the launch.  The scheduler hands tiles out longest first, so a
-// tile longer than a worker's fair share of the launch sets the duration: cut the tokens until it is not.
+// tile much longer than a worker's fair share of the launch sets the duration: cut the tokens until it is
+// not (a tile up to 1.3 shares is left whole: the partial sums and their reduction cost more than they save).
 int wgrad_splits(int64_t rows_out, int64_t cols_out, int64_t T, int64_t launch_cost) {
     const int64_t share = std::max<int64_t>(launch_cost / kWorkers, 1);
-    int64_t s = ceil_div(ceil_div(T, 64), share);
+    int64_t s = ceil_div(10 * ceil_div(T, 64), 13 * share);
     s = std::min<int64_t>(s, T / 1024);            // at least 16 k-blocks per range
     s = std::min<int64_t>(s, 6);
     return static_cast<int>(std::max<int64_t>(s, 1));
@@ -788,25 +789,31 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     Stored As;
     As.ptr = A; As.rows = T; As.cols = k; As.ld = ld_h;
 
-    // dH = (dY W_2^T) (.) act'(H): W_2 stored k x d_m = [N][K]; derivative fused into the epilogue
-    GemmOp da;
+    // Two launches of about equal length.  First: dH = (dY W_2^T) (.) act'(H) (W_2 stored k x d_m = [N][K], the
+    // derivative fused into the epilogue) together with dW_2 = A^T dY, which does not need dH.
+    const int nw = sw ? 2 : 1;
+    GemmOp ops[kMaxGemmOps];
+    PendingReduce red[3];
+    int n_ops = 0;
+    n_ops = add_wgrad(cx, ops, n_ops, As, dYs, k, d_m, T, dW2_c, ld_dw2, &red[0], 1,
+                      gemm_cost(k, d_m, T) + nw * gemm_cost(T, k, d_m));                                     // dW_2 (k x d_m)
+    if (cx.st != ECOSPA_OK) return cx.st;
+    GemmOp& da = ops[n_ops++];
     da.M = T; da.N = k; da.n_kseg = 1;
     da.seg[0].a = dYs; da.seg[0].b[0] = W2; da.seg[0].K = d_m;
     da.epi = sw ? EPI_DSWIGLU : (act == ECOSPA_ACT_GELU_ERF ? EPI_DGELU_ERF : EPI_DGELU_TANH);
     da.C = const_cast<void*>(dH.ptr); da.C2 = sw ? const_cast<void*>(dHb.ptr) : nullptr; da.ldc = dH.ld;
     da.H = H; da.Hb = Hb; da.ldh = ld_h;
-    if ((st = launch_grouped_gemm(&da, 1, cx.stream)) != ECOSPA_OK) return st;
+    if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
 
-    GemmOp ops[kMaxGemmOps];
-    PendingReduce red[3];
-    int n_ops = 0;
-    const int nw = sw ? 2 : 1;
-    const int64_t cost = gemm_cost(k, d_m, T) + nw * gemm_cost(d_m, k, T) + gemm_cost(T, d_m, nw * k);
-    n_ops = add_wgrad(cx, ops, n_ops, As, dYs, k, d_m, T, dW2_c, ld_dw2, &red[0], sw ? 3 : 2, cost);          // dW_2 (k x d_m) = A^T dY
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1, cost);           // dW_1 (d_m x k) = X^T dH
-    if (sw) n_ops = add_wgrad(cx, ops, n_ops, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1, cost); // dW_up = X^T dH_up
+    // Second: dW_1 = X^T dH (and dW_up = X^T dH_up), dX = dH W_1^T (+ dH_up W_up^T)
+    n_ops = 0;
+    const int64_t cost = nw * gemm_cost(d_m, k, T) + gemm_cost(T, d_m, nw * k);
+    n_ops = add_wgrad(cx, ops, n_ops, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1, cost);           // dW_1 (d_m x k)
+    if (sw) n_ops = add_wgrad(cx, ops, n_ops, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1, cost);           // dW_up
     if (cx.st != ECOSPA_OK) return cx.st;
-    GemmOp& dx = ops[n_ops++];                                                    // dX = dH W_1^T (+ dH_up W_up^T)
+    GemmOp& dx = ops[n_ops++];
+    dx = GemmOp();
     dx.M = T; dx.N = d_m; dx.n_kseg = sw ? 2 : 1;
     dx.seg[0].a = dH; dx.seg[0].b[0] = W1; dx.seg[0].K = k;
     if (sw) {
