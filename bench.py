@@ -27,6 +27,11 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (read + write) per gemm_kernel launch, averaged over the eight GEMM launches of a gpt2m layer:
+# `dram__bytes_read.sum + dram__bytes_write.sum` of one ncu capture of this build (profiles/gemm_kernel_gpt2m_layer.md).
+# Per-launch traffic does not depend on the number of layers captured.  Other workloads: not captured (None).
+NCU_GEMM_TRAFFIC_BYTES = {"gpt2m": 45.3e6}
+
 METRIC = "compacted-pair fwd/bwd TFLOP/s over the whole coupled-sparsity step (score+select+compact GB/s alongside)"
 
 
@@ -79,7 +84,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -356,7 +361,9 @@ def run_gpu(args):
         },
         "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": flops / ms_gemm / 1e9,
                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": flops / ms_gemm / 1e9 / peaks["bf16_tflops_sustained"], "traffic": None,
+                     "frac": flops / ms_gemm / 1e9 / peaks["bf16_tflops_sustained"],
+                     "traffic": NCU_GEMM_TRAFFIC_BYTES.get(wl.name) if (not args.layers and args.sparsity == 0.5) else None,
+                     "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
                      "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                      "launches_per_step": n_gemm_launches, "avg_launch_ms": ms_gemm / n_gemm_launches},
         "e2e": {"value": job_throughput(world, flops, ms_e2e) / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
@@ -458,7 +465,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=60)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="gpt2m")
