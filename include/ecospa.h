@@ -216,7 +216,10 @@ ecospa_status_t ecospa_coupled_qk_fwd(const void* X, int64_t ldx, int64_t T, int
                                       void* Qc, void* Kc, int64_t ld_out, void* workspace, size_t workspace_bytes,
                                       void* stream);
 /* Given dQc, dKc (T x n, pitch ld_dqk): dX = dQc W_Q^cT + dKc W_K^cT (added to dX if accumulate_dX),
- * dW_Q^c = X^T dQc, dW_K^c = X^T dKc (d_m x n, pitch ld_dw), db = column sums (may be NULL). */
+ * dW_Q^c = X^T dQc, dW_K^c = X^T dKc (d_m x n, pitch ld_dw), db = column sums (may be NULL).
+ * accumulate_dX, here and in the calls below: the product is rounded to the type of dX and then added to
+ * the stored dX by one reducing tile store per element (bf16 models: two roundings; fp32 models: exact
+ * fp32 addition); each element is added exactly once, so the result does not depend on timing. */
 ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int64_t T, int64_t d_m, const ecospa_mat_t* wq_c,
                                       const ecospa_mat_t* wk_c, int64_t n, const void* dQc, const void* dKc,
                                       int64_t ld_dqk, void* dX, int64_t ld_dx, int32_t accumulate_dX, void* dWq_c,
