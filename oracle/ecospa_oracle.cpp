@@ -13,6 +13,9 @@
 //   eco_fisher_pair              : Eq. "importance".
 //   eco_select_topk_*            : Definition 1 (aligned removal) applied to
 //                                  the (seg_len - k) lowest-scored indices.
+//   eco_threshold_counts_f32     : Algorithm 1, the "while sum of scores > theta: remove smallest" loop
+//                                  (how many aligned indices of each pair stay).
+//   eco_choose_pairs_f32         : Algorithm 1, the top-K pairs with the smallest importance.
 //   eco_compact_bytes            : Definition 1, the physical removal.
 //   eco_coupled_single / eco_individual_single / eco_frob_removed :
 //                                  Definitions 1 and 2, Propositions 1 and 2.
@@ -21,7 +24,9 @@
 //
 // Parity unpinned (conventions the paper does not fix, see the design notes):
 //   - the SwiGLU slot of eco_fisher_pair (W_1 = gate (.) up is not a parameter),
-//   - the choice between the erf and tanh GELU forms.
+//   - the choice between the erf and tanh GELU forms,
+//   - in eco_threshold_counts_f32, whether theta is a share of the score mass (l1 = 1) or is compared with the
+//     l2-normalised scores as stored (l1 = 0): the paper prints the l2 normaliser and thresholds of 85-95 %.
 //
 // Layout vocabulary: a matrix that owns a shared dimension D and another
 // dimension `other` is stored row-major either as  other x D  ("shared cols",
@@ -207,6 +212,54 @@ void eco_select_topk_f32(const float* upsilon, int n_seg, int seg_len, const int
     std::vector<double> tmp(static_cast<size_t>(n_seg) * seg_len);
     for (size_t i = 0; i < tmp.size(); ++i) tmp[i] = static_cast<double>(upsilon[i]);
     select_impl(tmp.data(), n_seg, seg_len, k, kept);
+}
+
+// ---------------------------------------------------------------------------
+// Algorithm 1, inner loop: "while the sum of the scores exceeds theta, remove the smallest score".
+// ---------------------------------------------------------------------------
+// Per segment (= per coupled pair): the scores that are still there are summed in fp64, largest first
+// (equal scores: lower index first); while that sum exceeds theta * total and more than k_min indices are
+// left, the smallest remaining score goes (among equal scores the higher index goes first, the same rule as
+// the top-k tie-break).  total = the sum of all scores of the segment when `l1` is set (theta is then the
+// fraction of the score mass that stays), 1 otherwise (the scores are compared with theta as stored).
+// chosen == nullptr: every segment is processed; otherwise segments with chosen[s] == 0 keep everything.
+// Output: how many indices stay per segment.  Scores are taken as stored fp32 values (exactly widened).
+void eco_threshold_counts_f32(const float* upsilon, int n_seg, int seg_len, double theta, int l1, int k_min,
+                              const int32_t* chosen, int32_t* k_out) {
+    for (int s = 0; s < n_seg; ++s) {
+        if (chosen && !chosen[s]) {
+            k_out[s] = seg_len;
+            continue;
+        }
+        const float* u = upsilon + static_cast<int64_t>(s) * seg_len;
+        std::vector<int32_t> order(seg_len);
+        std::iota(order.begin(), order.end(), 0);
+        std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return u[a] > u[b]; });
+        double total = 1.0;
+        if (l1) {
+            total = 0.0;
+            for (int i = 0; i < seg_len; ++i) total += static_cast<double>(u[order[i]]);
+        }
+        const double budget = theta * total;
+        int left = seg_len;
+        while (left > k_min) {
+            double sum = 0.0;                       // sum of what is left, largest first
+            for (int i = 0; i < left; ++i) sum += static_cast<double>(u[order[i]]);
+            if (!(sum > budget)) break;
+            --left;                                 // order[left] was the smallest one left
+        }
+        k_out[s] = left;
+    }
+}
+
+// Algorithm 1, "select the top-K coupled matrices with the smallest importance": the m smallest values of
+// `fisher` are marked (equal values: lower index first).
+void eco_choose_pairs_f32(const float* fisher, int n, int m, int32_t* chosen) {
+    std::vector<int32_t> order(n);
+    std::iota(order.begin(), order.end(), 0);
+    std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return fisher[a] < fisher[b]; });
+    for (int i = 0; i < n; ++i) chosen[i] = 0;
+    for (int i = 0; i < m && i < n; ++i) chosen[order[i]] = 1;
 }
 
 // ---------------------------------------------------------------------------

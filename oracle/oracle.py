@@ -153,6 +153,25 @@ def select_topk(ups, n_seg: int, seg_len: int, k: Sequence[int]) -> np.ndarray:
     return kept
 
 
+def threshold_counts(ups, n_seg: int, seg_len: int, theta: float, l1: bool = True, k_min: int = 1,
+                     chosen=None) -> np.ndarray:
+    """Kept count per segment after Algorithm 1's cumulative-threshold loop (fp32 scores as stored)."""
+    ups = np.ascontiguousarray(ups, dtype=np.float32)
+    assert ups.size == n_seg * seg_len
+    k = np.empty(n_seg, dtype=np.int32)
+    ch = _i32(chosen) if chosen is not None else None
+    lib().eco_threshold_counts_f32(_p(ups), n_seg, seg_len, C.c_double(theta), int(l1), int(k_min), _p(ch), _p(k))
+    return k
+
+
+def choose_pairs(fisher, m: int) -> np.ndarray:
+    """Flags of the m pairs with the smallest importance (ties: lower index first)."""
+    f = np.ascontiguousarray(fisher, dtype=np.float32)
+    out = np.empty(f.size, dtype=np.int32)
+    lib().eco_choose_pairs_f32(_p(f), f.size, int(m), _p(out))
+    return out
+
+
 def compact(t: torch.Tensor, layout: int, kept, ld_out: Optional[int] = None) -> torch.Tensor:
     """Gather the kept shared indices of `t` (2-D, or 1-D = a bias over the shared axis)."""
     kept = _i32(kept)

@@ -177,6 +177,16 @@ def test_ragged_kept_counts_gelu(k_ffn):
     run_block_full(wl, k_heads, k_ffn, B.ACT_GELU_ERF)
 
 
+def test_token_counts_that_end_inside_a_row_block():
+    """T = 333 and T = 77 end inside a 32-row warp block: the tile stores clip the rows past T, the saved
+    activations of the last block are fetched element by element, and accumulation must not touch them."""
+    wl = WL.WORKLOADS["tails768"]
+    k_heads = [WL.RAGGED_HEAD_KEPT[i % len(WL.RAGGED_HEAD_KEPT)] for i in range(wl.n_heads)]
+    run_block_full(wl, k_heads, 1073, B.ACT_GELU_ERF, T=333)
+    wl = WL.WORKLOADS["tiny_swiglu"]
+    run_block_full(wl, [13, 6], 77, B.ACT_SWIGLU, T=77, seed=2)
+
+
 def test_gelu_tanh_variant_small():
     wl = WL.WORKLOADS["tails768"]
     run_block_full(wl, [32] * wl.n_heads, 264, B.ACT_GELU_TANH, T=96)
