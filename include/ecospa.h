@@ -158,6 +158,37 @@ ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, const int32_t* 
                                            int32_t* seg_offsets, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Step 2, variable counts: the stopping rule of Algorithm 1 ("while the sum of the scores exceeds theta:
+ * remove the smallest score and its row/column") and its choice of pairs ("the top-K coupled matrices with
+ * the smallest importance").
+ *
+ * ecospa_choose_pairs: chosen[i] = 1 for the m smallest of the n importance values (Eq. "importance", as
+ *   written by ecospa_score_pairs), equal values: lower index first; 0 otherwise.  n <= 16384.
+ *   fisher DEVICE fp32 [n], chosen DEVICE out int32 [n].
+ *
+ * ecospa_select_aligned_threshold: for every segment, removes the lowest-scored indices one after the other
+ *   (equal scores: the higher index goes first) while the sum of the scores that are left exceeds
+ *   theta * total and more than k_min indices are left; total = the sum of all scores of the segment when
+ *   l1 != 0 (theta = share of the score mass that may stay), 1 when l1 == 0 (scores compared as stored).
+ *   Sums are taken in fp64.  Scores must be >= 0 (they are products of norms).  Segments with chosen[s] == 0
+ *   keep everything (chosen may be NULL: every segment is processed).
+ *   upsilon  DEVICE fp32, concatenated as written by ecospa_score_pairs
+ *   n_seg, seg_len HOST [n_pairs]
+ *   chosen   DEVICE int32 per segment (all pairs concatenated), may be NULL
+ *   kept     DEVICE out int32 with one slot per shared index (sum of n_seg * seg_len entries): segment s of
+ *            a pair writes its kept indices, ascending and relative to the pair group as in
+ *            ecospa_select_aligned_topk, at the position of its first shared index; the first k_out[s]
+ *            entries of the slot are valid, the rest is left untouched
+ *   k_out    DEVICE out int32 per segment: how many indices stay.  The caller reads it back to size the
+ *            compacted tensors (the counts are data dependent).
+ * Errors: theta < 0 or NaN, k_min < 0 -> ECOSPA_ERR_INVALID; seg_len > 2^20 -> ECOSPA_ERR_UNSUPPORTED.
+ */
+ecospa_status_t ecospa_choose_pairs(const float* fisher, int32_t n, int32_t m, int32_t* chosen, void* stream);
+ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon, const int32_t* n_seg, const int32_t* seg_len,
+                                                int32_t n_pairs, double theta, int32_t l1, int32_t k_min,
+                                                const int32_t* chosen, int32_t* kept, int32_t* k_out, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Step 3: physical removal.   Definition 1: drop column j of W_1 and row j of W_2 for every removed j
  * "keeping the original pairings"; Alg. 1 also drops the same rows/columns of the optimizer moments.
  *

@@ -170,6 +170,34 @@ def ecospa_select_aligned_topk(upsilon: torch.Tensor, n_seg: Sequence[int], seg_
         raise EcospaError(st, "ecospa_select_aligned_topk")
 
 
+def ecospa_choose_pairs(fisher: torch.Tensor, m: int, chosen: torch.Tensor, stream=None) -> None:
+    assert fisher.dtype == torch.float32 and chosen.dtype == torch.int32 and chosen.numel() >= fisher.numel()
+    fn = lib().ecospa_choose_pairs
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    st = fn(_ptr(fisher), fisher.numel(), int(m), _ptr(chosen), _stream(stream))
+    if st != 0:
+        raise EcospaError(st, "ecospa_choose_pairs")
+
+
+def ecospa_select_aligned_threshold(upsilon: torch.Tensor, n_seg: Sequence[int], seg_len: Sequence[int], theta: float,
+                                    kept: torch.Tensor, k_out: torch.Tensor, l1: bool = True, k_min: int = 1,
+                                    chosen: Optional[torch.Tensor] = None, stream=None) -> None:
+    n_pairs = len(n_seg)
+    a_nseg = (C.c_int32 * n_pairs)(*n_seg)
+    a_slen = (C.c_int32 * n_pairs)(*seg_len)
+    assert kept.dtype == torch.int32 and kept.numel() >= sum(a * b for a, b in zip(n_seg, seg_len))
+    assert k_out.dtype == torch.int32 and k_out.numel() >= sum(n_seg)
+    fn = lib().ecospa_select_aligned_threshold
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_int32, C.c_void_p,
+                   C.c_void_p, C.c_void_p, C.c_void_p]
+    st = fn(_ptr(upsilon), C.addressof(a_nseg), C.addressof(a_slen), n_pairs, float(theta), int(bool(l1)), int(k_min),
+            _ptr(chosen), _ptr(kept), _ptr(k_out), _stream(stream))
+    if st != 0:
+        raise EcospaError(st, "ecospa_select_aligned_threshold")
+
+
 def gather(inp: torch.Tensor, out: torch.Tensor, layout: int, kept: torch.Tensor, n_kept: int, shared_dim: int) -> Gather:
     g = Gather(mat(inp, layout), mat(out, layout), kept.data_ptr(), n_kept, shared_dim)
     g._keep = (inp, out, kept)

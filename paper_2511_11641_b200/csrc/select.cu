@@ -33,6 +33,8 @@ struct SelectParams {
     int32_t n_pairs, n_segs;
     int32_t seg_base;       // global index of this launch's first segment
     int32_t is_last;        // this launch writes the final seg_offsets entry
+    const int32_t* k_dev;   // non-null: kept counts are read from the device (indexed by global segment) and
+                            // segment s of a pair writes at the pair's score offset + s * seg_len
     SelPair pairs[kMaxPairs];
     int32_t out_off[kMaxSegs + 1];  // global offsets into kept
 };
@@ -60,8 +62,8 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     const int n = Q.seg_len;
     const int seg_in_pair = seg - Q.seg_start;
     const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg_in_pair) * n;
-    const int out0 = P.out_off[seg];
-    const int k = P.out_off[seg + 1] - out0;
+    const int out0 = P.k_dev ? Q.d_off + seg_in_pair * n : P.out_off[seg];
+    const int k = P.k_dev ? min(max(P.k_dev[P.seg_base + seg], 0), n) : P.out_off[seg + 1] - out0;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     if (P.seg_offsets && tid == 0) {
@@ -163,6 +165,155 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Algorithm 1's stopping rule: how many indices of a segment stay when the smallest scores are removed
+// while the sum of what is left exceeds theta * total.
+// ---------------------------------------------------------------------------------------------
+// Sum over the block in a fixed order (thread partial -> shuffle tree -> warps in order); all threads get it.
+__device__ __forceinline__ double block_sum_f64(double v, double* scratch) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) scratch[threadIdx.x >> 5] = v;
+    __syncthreads();
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < kWarps; ++w) t += scratch[w];
+    return t;
+}
+
+struct ThresholdParams {
+    const float* upsilon;
+    const int32_t* chosen;  // per global segment, may be null
+    int32_t* k_out;         // per global segment
+    double theta;
+    int32_t l1, k_min;
+    int32_t n_pairs, seg_base;
+    SelPair pairs[kMaxPairs];
+};
+
+// One CTA per segment.  The kept set is {key >= t} plus the first e elements of the tie group just below t,
+// where t is the smallest key threshold whose scores sum to at most the budget: found by bisection over
+// the 32-bit key space, every sum taken in fp64 over the whole segment.
+__global__ void __launch_bounds__(kThreads) threshold_count_kernel(const __grid_constant__ ThresholdParams P) {
+    __shared__ double scratch[kWarps];
+    __shared__ uint32_t sh_max[kWarps];
+    const int seg = blockIdx.x;
+    int lo_p = 0, hi_p = P.n_pairs - 1;
+    while (lo_p < hi_p) {
+        const int mid = (lo_p + hi_p + 1) >> 1;
+        if (P.pairs[mid].seg_start <= seg) lo_p = mid; else hi_p = mid - 1;
+    }
+    const SelPair& Q = P.pairs[lo_p];
+    const int n = Q.seg_len;
+    const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg - Q.seg_start) * n;
+    const int tid = threadIdx.x;
+    const int gseg = P.seg_base + seg;
+    if (P.chosen && P.chosen[gseg] == 0) {
+        if (tid == 0) P.k_out[gseg] = n;
+        return;
+    }
+    // sum of the scores whose key is at least t, and how many there are
+    auto mass_ge = [&](uint64_t t, int* count) -> double {
+        double s = 0.0;
+        int c = 0;
+        for (int j = tid; j < n; j += kThreads) {
+            const float f = __ldg(sc + j);
+            if (static_cast<uint64_t>(order_key(f)) >= t) {
+                s += static_cast<double>(f);
+                ++c;
+            }
+        }
+        if (count) *count = static_cast<int>(block_sum_f64(static_cast<double>(c), scratch));
+        return block_sum_f64(s, scratch);
+    };
+    const double all = mass_ge(0, nullptr);
+    const double budget = P.theta * (P.l1 ? all : 1.0);
+    int k = n;
+    if (all > budget) {
+        uint64_t lo = 0, hi = 1ull << 32;        // the empty set (t = 2^32) always fits
+        while (lo < hi) {
+            const uint64_t mid = (lo + hi) >> 1;
+            if (mass_ge(mid, nullptr) <= budget) hi = mid; else lo = mid + 1;
+        }
+        int cnt = 0;
+        double s = mass_ge(hi, &cnt);
+        // tie group just below the threshold: its largest key, its size and its (common) value
+        uint32_t below = 0;
+        bool any = false;
+        for (int j = tid; j < n; j += kThreads) {
+            const uint32_t key = order_key(__ldg(sc + j));
+            if (static_cast<uint64_t>(key) < hi) {
+                below = any ? max(below, key) : key;
+                any = true;
+            }
+        }
+        // block maximum of (any, below): encode "none" as 0 with a flag bit in 64 bits
+        unsigned long long enc = any ? (1ull << 32) | below : 0ull;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) enc = max(enc, __shfl_xor_sync(0xffffffffu, enc, o));
+        __syncthreads();
+        if ((tid & 31) == 0) {
+            sh_max[tid >> 5] = static_cast<uint32_t>(enc);
+            scratch[tid >> 5] = static_cast<double>(enc >> 32);
+        }
+        __syncthreads();
+        bool have = false;
+        uint32_t tkey = 0;
+        for (int w = 0; w < kWarps; ++w)
+            if (scratch[w] != 0.0) {
+                tkey = have ? max(tkey, sh_max[w]) : sh_max[w];
+                have = true;
+            }
+        __syncthreads();
+        int e = 0;
+        if (have) {
+            double val = 0.0;
+            int c = 0;
+            for (int j = tid; j < n; j += kThreads) {
+                const float f = __ldg(sc + j);
+                if (order_key(f) == tkey) {
+                    val = static_cast<double>(f);
+                    ++c;
+                }
+            }
+            const int ties = static_cast<int>(block_sum_f64(static_cast<double>(c), scratch));
+            // every thread that saw one holds the same value; take the maximum over the block
+            double vmax = val;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) vmax = fmax(vmax, __shfl_xor_sync(0xffffffffu, vmax, o));
+            __syncthreads();
+            if ((tid & 31) == 0) scratch[tid >> 5] = vmax;
+            __syncthreads();
+            double v = scratch[0];
+            for (int w = 1; w < kWarps; ++w) v = fmax(v, scratch[w]);
+            __syncthreads();
+            // (scores below zero do not occur: they are norms; a zero tie group adds nothing and always fits)
+            for (int j = 1; j <= ties; ++j) {
+                s += v;
+                if (s <= budget) e = j; else break;
+            }
+        }
+        k = cnt + e;
+    }
+    k = max(k, min(P.k_min, n));
+    if (tid == 0) P.k_out[gseg] = k;
+}
+
+// chosen[i] = 1 for the m smallest values (equal values: lower index first): rank by counting.
+__global__ void __launch_bounds__(1024) choose_pairs_kernel(const float* __restrict__ fisher, int n, int m,
+                                                            int32_t* __restrict__ chosen) {
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+        const float fi = fisher[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) {
+            const float fj = __ldg(fisher + j);
+            rank += (fj < fi || (fj == fi && j < i)) ? 1 : 0;
+        }
+        chosen[i] = rank < m ? 1 : 0;
+    }
+}
+
 }  // namespace
 
 }  // namespace ecospa
@@ -217,6 +368,7 @@ extern "C" ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, cons
         sp.out_off[ns] = out;
         sp.upsilon = upsilon;
         sp.kept = kept;
+        sp.k_dev = nullptr;
         sp.seg_offsets = seg_offsets;
         sp.n_pairs = np;
         sp.n_segs = ns;
@@ -226,4 +378,68 @@ extern "C" ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, cons
         if (st != ECOSPA_OK) return st;
     }
     return ECOSPA_OK;
+}
+
+extern "C" ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon, const int32_t* n_seg,
+                                                           const int32_t* seg_len, int32_t n_pairs, double theta,
+                                                           int32_t l1, int32_t k_min, const int32_t* chosen,
+                                                           int32_t* kept, int32_t* k_out, void* stream_) {
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    if (!upsilon || !n_seg || !seg_len || n_pairs < 1 || !kept || !k_out) return ECOSPA_ERR_INVALID;
+    if (!(theta >= 0.0) || k_min < 0) return ECOSPA_ERR_INVALID;
+    int64_t total_d = 0;
+    for (int p = 0; p < n_pairs; ++p) {
+        if (n_seg[p] < 1 || seg_len[p] < 1) return ECOSPA_ERR_INVALID;
+        if (seg_len[p] > (1 << 20)) return ECOSPA_ERR_UNSUPPORTED;
+        total_d += static_cast<int64_t>(n_seg[p]) * seg_len[p];
+    }
+    if (total_d > INT32_MAX) return ECOSPA_ERR_UNSUPPORTED;
+
+    static thread_local ThresholdParams tp;
+    static thread_local SelectParams sp;
+    int p = 0, s_in_p = 0;
+    int32_t d_off = 0, seg_global = 0;
+    while (p < n_pairs) {
+        int np = 0, ns = 0;
+        const int32_t seg_base = seg_global;
+        while (p < n_pairs && np < kMaxPairs && ns < kMaxSegs) {
+            const int take = std::min(n_seg[p] - s_in_p, kMaxSegs - ns);
+            SelPair& Q = sp.pairs[np];
+            Q.seg_start = ns - s_in_p;
+            Q.seg_len = seg_len[p];
+            Q.d_off = d_off;
+            Q.pad_ = 0;
+            tp.pairs[np] = Q;
+            ++np;
+            ns += take;
+            seg_global += take;
+            s_in_p += take;
+            if (s_in_p == n_seg[p]) {
+                d_off += n_seg[p] * seg_len[p];
+                ++p;
+                s_in_p = 0;
+            }
+        }
+        tp.upsilon = upsilon; tp.chosen = chosen; tp.k_out = k_out;
+        tp.theta = theta; tp.l1 = l1 ? 1 : 0; tp.k_min = k_min;
+        tp.n_pairs = np; tp.seg_base = seg_base;
+        threshold_count_kernel<<<ns, kThreads, 0, stream>>>(tp);
+        ecospa_status_t st = check_launch("threshold_count_kernel");
+        if (st != ECOSPA_OK) return st;
+        // the fixed-count selection, with the counts just written and one slot of seg_len entries per segment
+        sp.upsilon = upsilon; sp.kept = kept; sp.seg_offsets = nullptr;
+        sp.n_pairs = np; sp.n_segs = ns; sp.seg_base = seg_base; sp.is_last = 0;
+        sp.k_dev = k_out;
+        select_kernel<<<ns, kThreads, 0, stream>>>(sp);
+        if ((st = check_launch("select_kernel")) != ECOSPA_OK) return st;
+    }
+    return ECOSPA_OK;
+}
+
+extern "C" ecospa_status_t ecospa_choose_pairs(const float* fisher, int32_t n, int32_t m, int32_t* chosen, void* stream_) {
+    if (!fisher || !chosen || n < 1 || m < 0) return ECOSPA_ERR_INVALID;
+    if (n > 16384) return ECOSPA_ERR_UNSUPPORTED;
+    const int grid = (n + 1023) / 1024;
+    choose_pairs_kernel<<<grid, 1024, 0, static_cast<cudaStream_t>(stream_)>>>(fisher, n, m, chosen);
+    return check_launch("choose_pairs_kernel");
 }

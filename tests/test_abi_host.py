@@ -108,3 +108,29 @@ def test_compact_rejects_bad_arguments_without_launching(lib):
     g = B.Gather(m_in, _fake_mat(0x20000, other=8, ld=32), None, 32, 64)
     assert lib.ecospa_compact_tensors(C.addressof((B.Gather * 1)(g)), 1, None) == 1
     assert lib.ecospa_compact_tensors(None, 1, None) == 1
+
+
+def test_threshold_selection_rejects_bad_arguments_without_launching(lib):
+    fn = lib.ecospa_select_aligned_threshold
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_int32, C.c_void_p,
+                   C.c_void_p, C.c_void_p, C.c_void_p]
+    ups, kept, kout = C.c_void_p(0x1000), C.c_void_p(0x2000), C.c_void_p(0x3000)
+    one = (C.c_int32 * 1)(1)
+    slen = (C.c_int32 * 1)(64)
+    a = (C.addressof(one), C.addressof(slen), 1)
+    assert fn(None, *a, 0.9, 1, 1, None, kept, kout, None) == 1
+    assert fn(ups, *a, 0.9, 1, 1, None, None, kout, None) == 1
+    assert fn(ups, *a, 0.9, 1, 1, None, kept, None, None) == 1
+    assert fn(ups, *a, -0.1, 1, 1, None, kept, kout, None) == 1
+    assert fn(ups, *a, float("nan"), 1, 1, None, kept, kout, None) == 1
+    assert fn(ups, *a, 0.9, 1, -1, None, kept, kout, None) == 1
+    big = (C.c_int32 * 1)((1 << 20) + 1)
+    assert fn(ups, C.addressof(one), C.addressof(big), 1, 0.9, 1, 1, None, kept, kout, None) == 3
+    ch = lib.ecospa_choose_pairs
+    ch.restype = C.c_int
+    ch.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    assert ch(None, 4, 1, kept, None) == 1
+    assert ch(ups, 0, 1, kept, None) == 1
+    assert ch(ups, 4, -1, kept, None) == 1
+    assert ch(ups, 1 << 15, 1, kept, None) == 3
