@@ -333,3 +333,30 @@ def test_compaction_ragged_kept_counts_and_tensors_entry():
             ld = o.numel() if src.dim() == 1 else o.shape[1]
             ref = O.compact(src, layout, kd.cpu().numpy(), ld_out=ld)
             assert torch.equal(o.cpu().view(torch.int16), ref.view(torch.int16)), (nm, k_ffn)
+
+
+def test_fp32_optimizer_moments_follow_bf16_weights():
+    """Algorithm 1 removes the same rows/columns of the optimizer moments: fp32 first and second moments of a
+    bf16 FFN pair go through the same launch as the weights, with the same kept list, byte for byte."""
+    wl = WL.WORKLOADS["tails768"]
+    w = WL.layer_weights(wl, 0)
+    gen = torch.Generator().manual_seed(5)
+    mom = {"m1": torch.randn(w["w1"].shape, generator=gen), "v1": torch.rand(w["w1"].shape, generator=gen),
+           "m2": torch.randn(w["w2"].shape, generator=gen), "v2": torch.rand(w["w2"].shape, generator=gen)}
+    allt = {"w1": w["w1"], "w2": w["w2"], **mom}
+    d = to_dev(allt)
+    r = np.random.default_rng(4)
+    for k_ffn in (1337, 2044):
+        kept = np.sort(r.choice(wl.d_ffn, size=k_ffn, replace=False)).astype(np.int32)
+        kd = torch.from_numpy(kept).to(DEV)
+        jobs, outs = [], {}
+        for nm, layout in (("w1", 0), ("m1", 0), ("v1", 0), ("w2", 1), ("m2", 1), ("v2", 1)):
+            o = BL.alloc_compacted(d[nm], layout, k_ffn).fill_(7)
+            outs[nm] = (o, layout)
+            jobs.append(B.gather(d[nm], o, layout, kd, k_ffn, wl.d_ffn))
+        B.ecospa_compact_tensors(jobs)
+        torch.cuda.synchronize()
+        for nm, (o, layout) in outs.items():
+            ref = O.compact(allt[nm], layout, kept, ld_out=o.shape[1])
+            view = torch.int16 if allt[nm].element_size() == 2 else torch.int32
+            assert torch.equal(o.cpu().view(view), ref.view(view)), nm
