@@ -36,7 +36,8 @@ METRIC = "compacted-pair fwd/bwd TFLOP/s over the whole coupled-sparsity step (s
 
 
 # ---------------------------------------------------------------------------------------------
-# workload accounting (algorithmic bytes and flops; see the design doc for the derivation)
+# workload accounting: algorithmic bytes (every weight and gradient element read once for the scores, the
+# gather's reads and writes) and algorithmic flops (2*M*N*K of every product with the real kept counts)
 # ---------------------------------------------------------------------------------------------
 
 def step_flops(wl, n_attn: int, k_ffn: int) -> float:

@@ -22,7 +22,7 @@
 //   eco_proj_* / eco_ffn_*       : Eq. 2, 3 and 5 on the compacted matrices and
 //                                  their textbook reverse-mode derivatives.
 //
-// Parity unpinned (conventions the paper does not fix, see the design notes):
+// Parity unpinned (conventions the paper does not fix):
 //   - the SwiGLU slot of eco_fisher_pair (W_1 = gate (.) up is not a parameter),
 //   - the choice between the erf and tanh GELU forms,
 //   - in eco_threshold_counts_f32, whether theta is a share of the score mass (l1 = 1) or is compared with the

@@ -11,9 +11,13 @@
 // and activations are consumed in whatever row-major orientation they are stored).  Warp roles:
 //   warp 0      producer: one elected lane issues the TMA loads of a stage (two 64-deep k-blocks)
 //   warp 1      owns the 512 TMEM columns; one elected lane issues the MMAs and the commits
-//   warps 2..9  epilogue: two warps per TMEM lane quadrant, each takes half of the tile's columns
-// The tile list of all ops is walked with a static stride (tile = blockIdx.x + i * gridDim.x);
-// ops are ordered by decreasing contraction length so the long tiles start first.
+//   warps 2..9  epilogue: two warps per TMEM lane quadrant, each takes half of the tile's columns; a warp
+//               converts its rows, stages them in swizzled shared memory and one lane issues a TMA tile
+//               store (a reducing store when the output is added to what C holds)
+// Tiles are numbered op by op, longest contraction first; the host hands them out longest first to the
+// least-loaded worker and passes the lists as a table in the kernel parameters (a plain stride when
+// there are many tiles per worker).  The kernel is launched with programmatic stream serialization and
+// touches no global memory before griddepcontrol.wait, so its set-up overlaps the previous kernel's tail.
 // Every mbarrier wait is bounded in time; on expiry the CTA records an error code in a device
 // status word, waits for its copies in flight, frees its TMEM and returns.
 
