@@ -222,15 +222,17 @@ ecospa_status_t ecospa_compact_pair(const ecospa_pair_t* pair, const int32_t* ke
  *                 output below is bf16.  ECOSPA_F32: X, upstream gradients, biases, Y/Q/K/V/Out, dX and all
  *                 weight/bias gradients are fp32; operands are rounded to bf16 in the workspace first.
  *                 The saved FFN tensors H, Hb, A are bf16 in both cases.
- *   weights       compacted matrices as written by step 3: W_Q^c, W_K^c, W_V^c, W_1^c (W_gate^c, W_up^c)
- *                 are ECOSPA_SHARED_COLS (d_m x n, pitch ld); W_O^c, W_2^c are ECOSPA_SHARED_ROWS
- *                 (n x d_m).  other_dim must equal d_m.  The other storage orientation returns
- *                 ECOSPA_ERR_UNSUPPORTED.
+ *   weights       compacted matrices as written by step 3, each in either orientation (the descriptor's
+ *                 layout says which): ECOSPA_SHARED_COLS = d_m x n, ECOSPA_SHARED_ROWS = n x d_m, pitch ld.
+ *                 The equations' orientation is SHARED_COLS for W_Q^c, W_K^c, W_V^c, W_1^c (W_gate^c, W_up^c)
+ *                 and SHARED_ROWS for W_O^c, W_2^c; the transposed storage of each (what a framework's
+ *                 linear layer keeps) is consumed as it is, nothing is transposed in memory.  other_dim
+ *                 must equal d_m.  A weight gradient is written in the orientation of its weight
+ *                 (d_m x n with pitch >= n, or n x d_m with pitch >= d_m).
  *   pitches       all ld* in elements.  Every base pointer must be 16-byte aligned and every pitch a
  *                 multiple of 16 bytes (ECOSPA_ERR_ALIGNMENT otherwise); gradient outputs use the pitch
- *                 of a compacted weight (padded).  Outputs are written in 16-byte units: the pad columns
- *                 between n and the next multiple of 8 (bf16) elements may be overwritten (with what a zero
- *                 weight column yields); columns beyond that are left untouched.
+ *                 of a compacted weight (padded).  Only the real extent of an output is written (tile stores
+ *                 clipped at n, k, d_m and T); pad columns keep what the buffer held.
  *   workspace     DEVICE scratch, 16-byte aligned, at least ecospa_proj_workspace_bytes /
  *                 ecospa_ffn_workspace_bytes; may be NULL when that function returns 0.
  *   1/sqrt(d_h)   is not applied: Q^c and K^c are the plain projections.

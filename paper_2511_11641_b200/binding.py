@@ -307,11 +307,16 @@ def ecospa_ffn_workspace_bytes(T: int, d_m: int, k: int, act: int, dtype: int) -
     return int(_fn("ecospa_ffn_workspace_bytes")(T, d_m, k, act, dtype))
 
 
-def ecospa_coupled_qk_fwd(X, wq_c, wk_c, n: int, Qc, Kc, bq_c=None, bk_c=None, workspace=None, stream=None) -> None:
+# Layer calls.  Weights may be stored in either orientation: `w_in_layout` is the orientation of W_Q, W_K, W_V, W_1,
+# W_gate, W_up (default SHARED_COLS = d_m x n; SHARED_ROWS = n x d_m, the nn.Linear layout of those weights),
+# `w_out_layout` that of W_O, W_2, W_down (default SHARED_ROWS = n x d_m; SHARED_COLS = d_m x n, their nn.Linear
+# layout).  Weight gradients are written in the orientation of their weight.
+def ecospa_coupled_qk_fwd(X, wq_c, wk_c, n: int, Qc, Kc, bq_c=None, bk_c=None, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     """wq_c / wk_c: compacted weight buffers of shape (d_m, pitch); Qc / Kc: (T, pitch_out)."""
     T, d_m = X.shape
-    mq = mat(wq_c, SHARED_COLS)
-    mk = mat(wk_c, SHARED_COLS) if wk_c is not None else None
+    mq = mat(wq_c, w_in_layout)
+    mk = mat(wk_c, w_in_layout) if wk_c is not None else None
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_qk_fwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), n, _ptr(bq_c), _ptr(bk_c),
                                         Qc.data_ptr(), _ptr(Kc), Qc.stride(0), wp, wb, _stream(stream)),
@@ -319,10 +324,11 @@ def ecospa_coupled_qk_fwd(X, wq_c, wk_c, n: int, Qc, Kc, bq_c=None, bk_c=None, w
 
 
 def ecospa_coupled_qk_bwd(X, wq_c, wk_c, n: int, dQc, dKc, dX, dWq_c, dWk_c, dbq_c=None, dbk_c=None,
-                          accumulate_dX: bool = False, workspace=None, stream=None) -> None:
+                          accumulate_dX: bool = False, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    mq = mat(wq_c, SHARED_COLS)
-    mk = mat(wk_c, SHARED_COLS) if wk_c is not None else None
+    mq = mat(wq_c, w_in_layout)
+    mk = mat(wk_c, w_in_layout) if wk_c is not None else None
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_qk_bwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), n, dQc.data_ptr(), _ptr(dKc),
                                         dQc.stride(0), dX.data_ptr(), dX.stride(0), int(accumulate_dX), dWq_c.data_ptr(),
@@ -330,27 +336,30 @@ def ecospa_coupled_qk_bwd(X, wq_c, wk_c, n: int, dQc, dKc, dX, dWq_c, dWk_c, dbq
            "ecospa_coupled_qk_bwd")
 
 
-def ecospa_coupled_vo_fwd_v(X, wv_c, n: int, Vc, bv_c=None, workspace=None, stream=None) -> None:
+def ecospa_coupled_vo_fwd_v(X, wv_c, n: int, Vc, bv_c=None, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    mv = mat(wv_c, SHARED_COLS)
+    mv = mat(wv_c, w_in_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_vo_fwd_v")(X.data_ptr(), X.stride(0), T, d_m, _ref(mv), n, _ptr(bv_c), Vc.data_ptr(),
                                           Vc.stride(0), wp, wb, _stream(stream)), "ecospa_coupled_vo_fwd_v")
 
 
-def ecospa_coupled_vo_fwd_o(Ctx, wo_c, n: int, Out, bo=None, workspace=None, stream=None) -> None:
+def ecospa_coupled_vo_fwd_o(Ctx, wo_c, n: int, Out, bo=None, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T = Ctx.shape[0]
-    d_m = wo_c.shape[1]
-    mo = mat(wo_c, SHARED_ROWS)
+    d_m = wo_c.shape[1] if w_out_layout == SHARED_ROWS else wo_c.shape[0]
+    mo = mat(wo_c, w_out_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_vo_fwd_o")(Ctx.data_ptr(), Ctx.stride(0), T, d_m, _ref(mo), n, _ptr(bo), Out.data_ptr(),
                                           Out.stride(0), wp, wb, _stream(stream)), "ecospa_coupled_vo_fwd_o")
 
 
 def ecospa_coupled_vo_bwd(X, Ctx, wv_c, wo_c, n: int, dVc, dOut, dX, dCtx, dWv_c, dWo_c, dbv_c=None, dbo=None,
-                          accumulate_dX: bool = False, workspace=None, stream=None) -> None:
+                          accumulate_dX: bool = False, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    mv, mo = mat(wv_c, SHARED_COLS), mat(wo_c, SHARED_ROWS)
+    mv, mo = mat(wv_c, w_in_layout), mat(wo_c, w_out_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_vo_bwd")(X.data_ptr(), X.stride(0), Ctx.data_ptr(), Ctx.stride(0), T, d_m, _ref(mv), _ref(mo),
                                         n, dVc.data_ptr(), dVc.stride(0), dOut.data_ptr(), dOut.stride(0), dX.data_ptr(),
@@ -360,9 +369,10 @@ def ecospa_coupled_vo_bwd(X, Ctx, wv_c, wo_c, n: int, dVc, dOut, dX, dCtx, dWv_c
 
 
 def ecospa_coupled_qkv_fwd(X, wq_c, wk_c, wv_c, n_qk: int, n_vo: int, Qc, Kc, Vc, bq_c=None, bk_c=None, bv_c=None,
-                           workspace=None, stream=None) -> None:
+                           workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    mq, mk, mv = mat(wq_c, SHARED_COLS), mat(wk_c, SHARED_COLS), mat(wv_c, SHARED_COLS)
+    mq, mk, mv = mat(wq_c, w_in_layout), mat(wk_c, w_in_layout), mat(wv_c, w_in_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_qkv_fwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), _ref(mv), n_qk, n_vo,
                                          _ptr(bq_c), _ptr(bk_c), _ptr(bv_c), Qc.data_ptr(), Kc.data_ptr(), Vc.data_ptr(),
@@ -370,10 +380,10 @@ def ecospa_coupled_qkv_fwd(X, wq_c, wk_c, wv_c, n_qk: int, n_vo: int, Qc, Kc, Vc
 
 
 def ecospa_coupled_qkv_bwd(X, wq_c, wk_c, wv_c, n_qk: int, n_vo: int, dQc, dKc, dVc, dX, dWq_c, dWk_c, dWv_c,
-                           dbq_c=None, dbk_c=None, dbv_c=None, accumulate_dX: bool = False, workspace=None,
-                           stream=None) -> None:
+                           dbq_c=None, dbk_c=None, dbv_c=None, accumulate_dX: bool = False, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    mq, mk, mv = mat(wq_c, SHARED_COLS), mat(wk_c, SHARED_COLS), mat(wv_c, SHARED_COLS)
+    mq, mk, mv = mat(wq_c, w_in_layout), mat(wk_c, w_in_layout), mat(wv_c, w_in_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_qkv_bwd")(X.data_ptr(), X.stride(0), T, d_m, _ref(mq), _ref(mk), _ref(mv), n_qk, n_vo,
                                          dQc.data_ptr(), dKc.data_ptr(), dVc.data_ptr(), dQc.stride(0), dVc.stride(0),
@@ -383,20 +393,21 @@ def ecospa_coupled_qkv_bwd(X, wq_c, wk_c, wv_c, n_qk: int, n_vo: int, dQc, dKc, 
            "ecospa_coupled_qkv_bwd")
 
 
-def ecospa_coupled_vo_bwd_o(Ctx, wo_c, n: int, dOut, dCtx, dWo_c, dbo=None, workspace=None, stream=None) -> None:
+def ecospa_coupled_vo_bwd_o(Ctx, wo_c, n: int, dOut, dCtx, dWo_c, dbo=None, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T = Ctx.shape[0]
-    d_m = wo_c.shape[1]
-    mo = mat(wo_c, SHARED_ROWS)
+    d_m = wo_c.shape[1] if w_out_layout == SHARED_ROWS else wo_c.shape[0]
+    mo = mat(wo_c, w_out_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_vo_bwd_o")(Ctx.data_ptr(), Ctx.stride(0), T, d_m, _ref(mo), n, dOut.data_ptr(),
                                           dOut.stride(0), dCtx.data_ptr(), dCtx.stride(0), dWo_c.data_ptr(),
                                           dWo_c.stride(0), _ptr(dbo), wp, wb, _stream(stream)), "ecospa_coupled_vo_bwd_o")
 
 
-def ecospa_coupled_vo_bwd_v(X, wv_c, n: int, dVc, dX, dWv_c, dbv_c=None, accumulate_dX: bool = False, workspace=None,
-                            stream=None) -> None:
+def ecospa_coupled_vo_bwd_v(X, wv_c, n: int, dVc, dX, dWv_c, dbv_c=None, accumulate_dX: bool = False, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    mv = mat(wv_c, SHARED_COLS)
+    mv = mat(wv_c, w_in_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_vo_bwd_v")(X.data_ptr(), X.stride(0), T, d_m, _ref(mv), n, dVc.data_ptr(), dVc.stride(0),
                                           dX.data_ptr(), dX.stride(0), int(accumulate_dX), dWv_c.data_ptr(),
@@ -404,11 +415,12 @@ def ecospa_coupled_vo_bwd_v(X, wv_c, n: int, dVc, dX, dWv_c, dbv_c=None, accumul
 
 
 def ecospa_coupled_ffn_fwd(X, act: int, w1_c, w2_c, k: int, Y, H, A, w1b_c=None, Hb=None, b1_c=None, b2=None,
-                           workspace=None, stream=None) -> None:
+                           workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    m1 = mat(w1_c, SHARED_COLS)
-    m1b = mat(w1b_c, SHARED_COLS) if w1b_c is not None else None
-    m2 = mat(w2_c, SHARED_ROWS)
+    m1 = mat(w1_c, w_in_layout)
+    m1b = mat(w1b_c, w_in_layout) if w1b_c is not None else None
+    m2 = mat(w2_c, w_out_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_ffn_fwd")(X.data_ptr(), X.stride(0), T, d_m, act, _ref(m1), _ref(m1b), _ref(m2), k, _ptr(b1_c),
                                          _ptr(b2), Y.data_ptr(), Y.stride(0), H.data_ptr(), _ptr(Hb), A.data_ptr(),
@@ -416,11 +428,12 @@ def ecospa_coupled_ffn_fwd(X, act: int, w1_c, w2_c, k: int, Y, H, A, w1b_c=None,
 
 
 def ecospa_coupled_ffn_bwd(X, act: int, w1_c, w2_c, k: int, H, A, dY, dX, dW1_c, dW2_c, w1b_c=None, Hb=None,
-                           dW1b_c=None, db1_c=None, db2=None, workspace=None, stream=None) -> None:
+                           dW1b_c=None, db1_c=None, db2=None, workspace=None, stream=None,
+        w_in_layout: int = SHARED_COLS, w_out_layout: int = SHARED_ROWS) -> None:
     T, d_m = X.shape
-    m1 = mat(w1_c, SHARED_COLS)
-    m1b = mat(w1b_c, SHARED_COLS) if w1b_c is not None else None
-    m2 = mat(w2_c, SHARED_ROWS)
+    m1 = mat(w1_c, w_in_layout)
+    m1b = mat(w1b_c, w_in_layout) if w1b_c is not None else None
+    m2 = mat(w2_c, w_out_layout)
     wp, wb = _ws(workspace)
     _check(_fn("ecospa_coupled_ffn_bwd")(X.data_ptr(), X.stride(0), T, d_m, act, _ref(m1), _ref(m1b), _ref(m2), k, H.data_ptr(),
                                          _ptr(Hb), A.data_ptr(), H.stride(0), dY.data_ptr(), dY.stride(0), dX.data_ptr(),

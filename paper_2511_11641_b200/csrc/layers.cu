@@ -2,11 +2,11 @@
 // grouped launches of the tcgen05 GEMM engine plus two small helper kernels (fp32 -> bf16 staging for
 // fp32 models, and column sums for the bias gradients).
 //
-// Storage convention accepted here (the one the equations are written in):
-//   W_Q^c, W_K^c, W_V^c, W_1^c (gate/up): d_m x n row-major  (ECOSPA_SHARED_COLS, pitch ld >= n)
-//   W_O^c, W_2^c (down)                 : n x d_m row-major  (ECOSPA_SHARED_ROWS)
-// so every product below consumes its operands as stored (K-major or MN-major UMMA operands); nothing
-// is transposed in memory.
+// Storage: every compacted weight is accepted as d_m x n (ECOSPA_SHARED_COLS) or n x d_m (ECOSPA_SHARED_ROWS),
+// row-major; the equations' orientation is d_m x n for W_Q^c, W_K^c, W_V^c, W_1^c (gate/up) and n x d_m for
+// W_O^c, W_2^c (down).  Every product below consumes its operands as stored (K-major or MN-major UMMA
+// operands, chosen from the weight's layout); nothing is transposed in memory, and a weight gradient is
+// written in the orientation of its weight.
 
 #include <cuda_bf16.h>
 
@@ -312,14 +312,21 @@ ColsumParams colsum_begin(Ctx& cx, const Stored& M1, void* out1, const Stored& M
     return P;
 }
 
-// Compacted weight with n real shared indices, as stored: shared-cols d_m x n, or shared-rows n x d_m.
-ecospa_status_t check_weight(const ecospa_mat_t* w, int64_t d_m, int64_t n, int want_layout, int dtype) {
+// Compacted weight with n real shared indices, as stored: shared-cols d_m x n, or shared-rows n x d_m.  Either
+// orientation is accepted for every weight: the engine consumes K-major and MN-major operands alike, so a
+// stored orientation only decides which of the two a product sees (and in which orientation the weight
+// gradient is written: the same as the weight).
+ecospa_status_t check_weight(const ecospa_mat_t* w, int64_t d_m, int64_t n, int dtype) {
     if (!w || !w->ptr) return ECOSPA_ERR_INVALID;
     if (w->dtype != dtype || w->other_dim != d_m) return ECOSPA_ERR_INVALID;
-    if (w->layout != want_layout) return ECOSPA_ERR_UNSUPPORTED;
-    if (w->ld < (want_layout == ECOSPA_SHARED_COLS ? n : d_m)) return ECOSPA_ERR_INVALID;
+    if (w->layout != ECOSPA_SHARED_COLS && w->layout != ECOSPA_SHARED_ROWS) return ECOSPA_ERR_INVALID;
+    if (w->ld < (w->layout == ECOSPA_SHARED_COLS ? n : d_m)) return ECOSPA_ERR_INVALID;
     return ECOSPA_OK;
 }
+// Is the weight an MN-major B operand ([K][N] in memory) of a product that contracts over d_m (output = shared
+// index), respectively over the shared index (output = d_m)?
+bool mn_over_other(const ecospa_mat_t* w) { return w->layout == ECOSPA_SHARED_COLS; }
+bool mn_over_shared(const ecospa_mat_t* w) { return w->layout == ECOSPA_SHARED_ROWS; }
 Stored weight_bf16(Ctx& cx, const ecospa_mat_t* w, int64_t d_m, int64_t n) {
     if (w->layout == ECOSPA_SHARED_COLS) return as_bf16(cx, w->ptr, d_m, n, w->ld);
     return as_bf16(cx, w->ptr, n, d_m, w->ld);
@@ -342,12 +349,12 @@ size_t staged(int dtype, int64_t rows, int64_t cols) {  // bytes as_bf16 takes f
 size_t scratch(int64_t rows, int64_t cols) { return arena_need(static_cast<size_t>(rows) * round_up(cols, 8) * 2); }
 size_t colsum_need(int64_t rows, int64_t cols) { return arena_need(static_cast<size_t>(ceil_div(rows, kSumRows)) * cols * 4); }
 
-// C (T x n) = X (stored T x d_m, K-major) * W (shared-cols weight d_m x n, consumed MN-major) [+ bias]
-GemmOp proj_op(const Stored& X, const Stored& W, int64_t T, int64_t d_m, int64_t n, const void* bias, void* out, int64_t ld_out, int dtype) {
+// C (T x n) = X (stored T x d_m, K-major) * W (d_m x n consumed MN-major, or n x d_m consumed K-major) [+ bias]
+GemmOp proj_op(const Stored& X, const Stored& W, bool w_mn, int64_t T, int64_t d_m, int64_t n, const void* bias, void* out, int64_t ld_out, int dtype) {
     GemmOp op;
     op.M = T; op.N = n; op.n_kseg = 1;
     op.seg[0].a = X; op.seg[0].a_mn = false;
-    op.seg[0].b[0] = W; op.seg[0].b_mn = true;
+    op.seg[0].b[0] = W; op.seg[0].b_mn = w_mn;
     op.seg[0].K = d_m;
     op.epi = EPI_STORE;
     op.C = out; op.ldc = ld_out; op.out_f32 = dtype == ECOSPA_F32;
@@ -371,9 +378,13 @@ int wgrad_splits(int64_t rows_out, int64_t cols_out, int64_t T, int64_t launch_c
     return static_cast<int>(std::max<int64_t>(s, 1));
 }
 // Upper bound of the partial buffers over every launch this product can be part of (its own cost alone).
-size_t wgrad_need(int64_t rows_out, int64_t cols_out, int64_t T) {
+size_t wgrad_need_one(int64_t rows_out, int64_t cols_out, int64_t T) {
     const int S = wgrad_splits(rows_out, cols_out, T, gemm_cost(rows_out, cols_out, T));
     return S > 1 ? arena_need(static_cast<size_t>(S) * rows_out * round_up(cols_out, 4) * 4) : 0;
+}
+// the gradient is written in the weight's orientation, which the size query does not know
+size_t wgrad_need(int64_t rows_out, int64_t cols_out, int64_t T) {
+    return std::max(wgrad_need_one(rows_out, cols_out, T), wgrad_need_one(cols_out, rows_out, T));
 }
 struct PendingReduce {
     const float* partial = nullptr;
@@ -427,6 +438,16 @@ int add_wgrad(Ctx& cx, GemmOp* ops, int n_ops, const Stored& Xs, const Stored& d
     red->out = out; red->ld_out = ld_out;
     return n_ops;
 }
+// Gradient of a weight stored like `w`: d_m x n = other^T shared for a shared-cols weight, n x d_m = shared^T other
+// for a shared-rows one (other_act: T x d_m on the d_m side of the weight, shared_act: T x n on its shared side).
+int add_wgrad_w(Ctx& cx, GemmOp* ops, int n_ops, const ecospa_mat_t* w, const Stored& other_act, const Stored& shared_act,
+                int64_t d_m, int64_t n, int64_t T, void* out, int64_t ld_out, PendingReduce* red, int reserve,
+                int64_t launch_cost) {
+    if (w->layout == ECOSPA_SHARED_COLS)
+        return add_wgrad(cx, ops, n_ops, other_act, shared_act, d_m, n, T, out, ld_out, red, reserve, launch_cost);
+    return add_wgrad(cx, ops, n_ops, shared_act, other_act, n, d_m, T, out, ld_out, red, reserve, launch_cost);
+}
+
 // The finishing launch of a call: split-K reductions and column-sum finals together.
 void finish(Ctx& cx, const PendingReduce* red, int n_red, const ColsumParams& cs) {
     if (cx.st != ECOSPA_OK) return;
@@ -466,15 +487,16 @@ using namespace ecospa;
 
 extern "C" size_t ecospa_proj_workspace_bytes(int64_t T, int64_t d_m, int64_t n, int32_t dtype) {
     // worst case over the qk / vo calls: staged X, Ctx, upstream grads, weights, and the column-sum partials
-    return staged(dtype, T, d_m) * 2 + staged(dtype, d_m, n) * 2 + staged(dtype, n, d_m) + staged(dtype, T, n) * 3 +
-           colsum_need(T, n) * 3 + colsum_need(T, d_m) + wgrad_need(d_m, n, T) * 3 + wgrad_need(n, d_m, T) + staged(dtype, d_m, n) +
-           staged(dtype, T, n) + 1024;
+    const size_t w = std::max(staged(dtype, d_m, n), staged(dtype, n, d_m));   // a weight in either orientation
+    return staged(dtype, T, d_m) * 2 + w * 4 + staged(dtype, T, n) * 4 + colsum_need(T, n) * 3 + colsum_need(T, d_m) +
+           wgrad_need(d_m, n, T) * 4 + 1024;
 }
 
 extern "C" size_t ecospa_ffn_workspace_bytes(int64_t T, int64_t d_m, int64_t k, int32_t act, int32_t dtype) {
     const int nw = act == ECOSPA_ACT_SWIGLU ? 2 : 1;
-    return staged(dtype, T, d_m) * 2 + staged(dtype, d_m, k) * nw + staged(dtype, k, d_m) + scratch(T, k) * nw +
-           colsum_need(T, k) + colsum_need(T, d_m) + wgrad_need(d_m, k, T) * nw + wgrad_need(k, d_m, T) + 1024;
+    const size_t w = std::max(staged(dtype, d_m, k), staged(dtype, k, d_m));   // a weight in either orientation
+    return staged(dtype, T, d_m) * 2 + w * (nw + 1) + scratch(T, k) * nw + colsum_need(T, k) + colsum_need(T, d_m) +
+           wgrad_need(d_m, k, T) * (nw + 1) + 1024;
 }
 
 extern "C" ecospa_status_t ecospa_coupled_qk_fwd(const void* X, int64_t ldx, int64_t T, int64_t d_m,
@@ -485,14 +507,14 @@ extern "C" ecospa_status_t ecospa_coupled_qk_fwd(const void* X, int64_t ldx, int
     Ctx cx;
     ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(wq_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if (wk_c && (st = check_weight(wk_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
+    if (wk_c && (st = check_weight(wk_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
     if (wk_c && !Kc) return ECOSPA_ERR_INVALID;
     const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
     GemmOp ops[2];
     int n_ops = 0;
-    ops[n_ops++] = proj_op(Xs, weight_bf16(cx, wq_c, d_m, n), T, d_m, n, bq_c, Qc, ld_out, cx.dtype);
-    if (wk_c) ops[n_ops++] = proj_op(Xs, weight_bf16(cx, wk_c, d_m, n), T, d_m, n, bk_c, Kc, ld_out, cx.dtype);
+    ops[n_ops++] = proj_op(Xs, weight_bf16(cx, wq_c, d_m, n), mn_over_other(wq_c), T, d_m, n, bq_c, Qc, ld_out, cx.dtype);
+    if (wk_c) ops[n_ops++] = proj_op(Xs, weight_bf16(cx, wk_c, d_m, n), mn_over_other(wk_c), T, d_m, n, bk_c, Kc, ld_out, cx.dtype);
     if (cx.st != ECOSPA_OK) return cx.st;
     return launch_grouped_gemm(ops, n_ops, cx.stream);
 }
@@ -508,8 +530,8 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
     Ctx cx;
     ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(wq_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if (wk_c && (st = check_weight(wk_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
+    if (wk_c && (st = check_weight(wk_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
     const bool f32 = cx.dtype == ECOSPA_F32;
     const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
     const Stored dQs = as_bf16(cx, dQc, T, n, ld_dqk);
@@ -524,15 +546,15 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
     PendingReduce red[2];
     int n_ops = 0;
     const int64_t cost = (wk_c ? 2 : 1) * (gemm_cost(d_m, n, T) + gemm_cost(T, d_m, n));
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n, T, dWq_c, ld_dw, &red[0], wk_c ? 2 : 1, cost);
-    if (wk_c) n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n, T, dWk_c, ld_dw, &red[1], 1, cost);
+    n_ops = add_wgrad_w(cx, ops, n_ops, wq_c, Xs, dQs, d_m, n, T, dWq_c, ld_dw, &red[0], wk_c ? 2 : 1, cost);
+    if (wk_c) n_ops = add_wgrad_w(cx, ops, n_ops, wk_c, Xs, dKs, d_m, n, T, dWk_c, ld_dw, &red[1], 1, cost);
     if (cx.st != ECOSPA_OK) return cx.st;
     // dX = dQ W_Q^T (+ dK W_K^T): weights stored d_m x n are K-major B operands here
     GemmOp& dx = ops[n_ops++];
     dx.M = T; dx.N = d_m; dx.n_kseg = wk_c ? 2 : 1;
-    dx.seg[0].a = dQs; dx.seg[0].b[0] = Wq; dx.seg[0].K = n;
+    dx.seg[0].a = dQs; dx.seg[0].b[0] = Wq; dx.seg[0].b_mn = mn_over_shared(wq_c); dx.seg[0].K = n;
     if (wk_c) {
-        dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].K = n;
+        dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].b_mn = mn_over_shared(wk_c); dx.seg[1].K = n;
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
@@ -554,12 +576,12 @@ extern "C" ecospa_status_t ecospa_coupled_vo_fwd_o(const void* Ctxm, int64_t ld_
     Ctx cx;
     ecospa_status_t st = begin(cx, wo_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(wo_c, d_m, n, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wo_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
     GemmOp op;
     op.M = T; op.N = d_m; op.n_kseg = 1;
     op.seg[0].a = as_bf16(cx, Ctxm, T, n, ld_ctx);
-    op.seg[0].b[0] = weight_bf16(cx, wo_c, d_m, n);   // stored n x d_m = [K][N]
-    op.seg[0].b_mn = true;
+    op.seg[0].b[0] = weight_bf16(cx, wo_c, d_m, n);   // stored n x d_m = [K][N], or d_m x n = [N][K]
+    op.seg[0].b_mn = mn_over_shared(wo_c);
     op.seg[0].K = n;
     op.epi = EPI_STORE; op.C = Out; op.ldc = ld_out; op.out_f32 = cx.dtype == ECOSPA_F32;
     op.bias = bo; op.bias_f32 = cx.dtype == ECOSPA_F32;
@@ -577,8 +599,8 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     Ctx cx;
     ecospa_status_t st = begin(cx, wv_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(wv_c, d_m, n, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if ((st = check_weight(wo_c, d_m, n, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wv_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wo_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
     const bool f32 = cx.dtype == ECOSPA_F32;
     const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
     const Stored Cs = as_bf16(cx, Ctxm, T, n, ld_ctx);
@@ -592,18 +614,18 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     int n_ops = 0;
     // dW_O (n x d_m) = Ctx^T dOut ; dW_V (d_m x n) = X^T dV
     const int64_t cost = gemm_cost(n, d_m, T) + gemm_cost(d_m, n, T) + gemm_cost(T, n, d_m) + gemm_cost(T, d_m, n);
-    n_ops = add_wgrad(cx, ops, n_ops, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red[0], 3, cost);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n, T, dWv_c, ld_dwv, &red[1], 2, cost);
+    n_ops = add_wgrad_w(cx, ops, n_ops, wo_c, dOs, Cs, d_m, n, T, dWo_c, ld_dwo, &red[0], 3, cost);
+    n_ops = add_wgrad_w(cx, ops, n_ops, wv_c, Xs, dVs, d_m, n, T, dWv_c, ld_dwv, &red[1], 2, cost);
     if (cx.st != ECOSPA_OK) return cx.st;
     // dCtx (T x n) = dOut W_O^T : W_O stored n x d_m = [N][K]
     GemmOp& dc = ops[n_ops++];
     dc.M = T; dc.N = n; dc.n_kseg = 1;
-    dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].K = d_m;
+    dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].b_mn = mn_over_other(wo_c); dc.seg[0].K = d_m;
     dc.epi = EPI_STORE; dc.C = dCtx; dc.ldc = ld_dctx; dc.out_f32 = f32;
     // dX (T x d_m) = dV W_V^T : W_V stored d_m x n = [N][K]
     GemmOp& dx = ops[n_ops++];
     dx.M = T; dx.N = d_m; dx.n_kseg = 1;
-    dx.seg[0].a = dVs; dx.seg[0].b[0] = Wv; dx.seg[0].K = n;
+    dx.seg[0].a = dVs; dx.seg[0].b[0] = Wv; dx.seg[0].b_mn = mn_over_shared(wv_c); dx.seg[0].K = n;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
     finish(cx, red, 2, colsum_begin(cx, dVs, dbv_c, dOs, dbo));
@@ -621,14 +643,14 @@ extern "C" ecospa_status_t ecospa_coupled_qkv_fwd(const void* X, int64_t ldx, in
     Ctx cx;
     ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, std::min(n_qk, n_vo));
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(wq_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if ((st = check_weight(wk_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if ((st = check_weight(wv_c, d_m, n_vo, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n_qk, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wk_c, d_m, n_qk, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wv_c, d_m, n_vo, cx.dtype)) != ECOSPA_OK) return st;
     const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
     GemmOp ops[3];
-    ops[0] = proj_op(Xs, weight_bf16(cx, wq_c, d_m, n_qk), T, d_m, n_qk, bq_c, Qc, ld_qk, cx.dtype);
-    ops[1] = proj_op(Xs, weight_bf16(cx, wk_c, d_m, n_qk), T, d_m, n_qk, bk_c, Kc, ld_qk, cx.dtype);
-    ops[2] = proj_op(Xs, weight_bf16(cx, wv_c, d_m, n_vo), T, d_m, n_vo, bv_c, Vc, ld_v, cx.dtype);
+    ops[0] = proj_op(Xs, weight_bf16(cx, wq_c, d_m, n_qk), mn_over_other(wq_c), T, d_m, n_qk, bq_c, Qc, ld_qk, cx.dtype);
+    ops[1] = proj_op(Xs, weight_bf16(cx, wk_c, d_m, n_qk), mn_over_other(wk_c), T, d_m, n_qk, bk_c, Kc, ld_qk, cx.dtype);
+    ops[2] = proj_op(Xs, weight_bf16(cx, wv_c, d_m, n_vo), mn_over_other(wv_c), T, d_m, n_vo, bv_c, Vc, ld_v, cx.dtype);
     if (cx.st != ECOSPA_OK) return cx.st;
     return launch_grouped_gemm(ops, 3, cx.stream);
 }
@@ -647,9 +669,9 @@ extern "C" ecospa_status_t ecospa_coupled_qkv_bwd(const void* X, int64_t ldx, in
     Ctx cx;
     ecospa_status_t st = begin(cx, wq_c->dtype, workspace, workspace_bytes, stream, T, d_m, std::min(n_qk, n_vo));
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(wq_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if ((st = check_weight(wk_c, d_m, n_qk, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if ((st = check_weight(wv_c, d_m, n_vo, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wq_c, d_m, n_qk, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wk_c, d_m, n_qk, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wv_c, d_m, n_vo, cx.dtype)) != ECOSPA_OK) return st;
     const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
     const Stored dQs = as_bf16(cx, dQc, T, n_qk, ld_dqk);
     const Stored dKs = as_bf16(cx, dKc, T, n_qk, ld_dqk);
@@ -662,15 +684,15 @@ extern "C" ecospa_status_t ecospa_coupled_qkv_bwd(const void* X, int64_t ldx, in
     PendingReduce red[3];
     int n_ops = 0;
     const int64_t cost = 2 * gemm_cost(d_m, n_qk, T) + gemm_cost(d_m, n_vo, T) + gemm_cost(T, d_m, 2 * n_qk + n_vo);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dQs, d_m, n_qk, T, dWq_c, ld_dwqk, &red[0], 3, cost);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dKs, d_m, n_qk, T, dWk_c, ld_dwqk, &red[1], 2, cost);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dVs, d_m, n_vo, T, dWv_c, ld_dwv, &red[2], 1, cost);
+    n_ops = add_wgrad_w(cx, ops, n_ops, wq_c, Xs, dQs, d_m, n_qk, T, dWq_c, ld_dwqk, &red[0], 3, cost);
+    n_ops = add_wgrad_w(cx, ops, n_ops, wk_c, Xs, dKs, d_m, n_qk, T, dWk_c, ld_dwqk, &red[1], 2, cost);
+    n_ops = add_wgrad_w(cx, ops, n_ops, wv_c, Xs, dVs, d_m, n_vo, T, dWv_c, ld_dwv, &red[2], 1, cost);
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& dx = ops[n_ops++];
     dx.M = T; dx.N = d_m; dx.n_kseg = 3;
-    dx.seg[0].a = dQs; dx.seg[0].b[0] = Wq; dx.seg[0].K = n_qk;
-    dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].K = n_qk;
-    dx.seg[2].a = dVs; dx.seg[2].b[0] = Wv; dx.seg[2].K = n_vo;
+    dx.seg[0].a = dQs; dx.seg[0].b[0] = Wq; dx.seg[0].b_mn = mn_over_shared(wq_c); dx.seg[0].K = n_qk;
+    dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].b_mn = mn_over_shared(wk_c); dx.seg[1].K = n_qk;
+    dx.seg[2].a = dVs; dx.seg[2].b[0] = Wv; dx.seg[2].b_mn = mn_over_shared(wv_c); dx.seg[2].K = n_vo;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = cx.dtype == ECOSPA_F32; dx.accumulate = accumulate_dX != 0;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
     finish(cx, red, 3, colsum_begin(cx, dQs, dbq_c, dKs, dbk_c, dVs, dbv_c));
@@ -687,7 +709,7 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd_o(const void* Ctxm, int64_t ld_
     Ctx cx;
     ecospa_status_t st = begin(cx, wo_c->dtype, workspace, workspace_bytes, stream, T, d_m, n);
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(wo_c, d_m, n, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(wo_c, d_m, n, cx.dtype)) != ECOSPA_OK) return st;
     const Stored Cs = as_bf16(cx, Ctxm, T, n, ld_ctx);
     const Stored dOs = as_bf16(cx, dOut, T, d_m, ld_dout);
     const Stored Wo = weight_bf16(cx, wo_c, d_m, n);
@@ -695,11 +717,11 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd_o(const void* Ctxm, int64_t ld_
     GemmOp ops[kMaxGemmOps];
     PendingReduce red;
     const int64_t cost = gemm_cost(n, d_m, T) + gemm_cost(T, n, d_m);
-    int n_ops = add_wgrad(cx, ops, 0, Cs, dOs, n, d_m, T, dWo_c, ld_dwo, &red, 1, cost);   // dW_O (n x d_m) = Ctx^T dOut
+    int n_ops = add_wgrad_w(cx, ops, 0, wo_c, dOs, Cs, d_m, n, T, dWo_c, ld_dwo, &red, 1, cost);   // dW_O, stored like W_O
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& dc = ops[n_ops++];                                                        // dCtx = dOut W_O^T
     dc.M = T; dc.N = n; dc.n_kseg = 1;
-    dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].K = d_m;
+    dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].b_mn = mn_over_other(wo_c); dc.seg[0].K = d_m;
     dc.epi = EPI_STORE; dc.C = dCtx; dc.ldc = ld_dctx; dc.out_f32 = cx.dtype == ECOSPA_F32;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
     finish(cx, &red, 1, colsum_begin(cx, dOs, dbo));
@@ -728,9 +750,9 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_fwd(const void* X, int64_t ldx, in
     Ctx cx;
     ecospa_status_t st = begin(cx, w1_c->dtype, workspace, workspace_bytes, stream, T, d_m, k);
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(w1_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if (sw && (st = check_weight(w1b_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if ((st = check_weight(w2_c, d_m, k, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(w1_c, d_m, k, cx.dtype)) != ECOSPA_OK) return st;
+    if (sw && (st = check_weight(w1b_c, d_m, k, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(w2_c, d_m, k, cx.dtype)) != ECOSPA_OK) return st;
     if (ld_h < k || (ld_h * 2) % 16) return ld_h < k ? ECOSPA_ERR_INVALID : ECOSPA_ERR_ALIGNMENT;
     const bool f32 = cx.dtype == ECOSPA_F32;
     const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
@@ -739,7 +761,7 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_fwd(const void* X, int64_t ldx, in
     up.seg[0].a = Xs;
     up.seg[0].b[0] = weight_bf16(cx, w1_c, d_m, k);
     if (sw) up.seg[0].b[1] = weight_bf16(cx, w1b_c, d_m, k);
-    up.seg[0].b_mn = true;
+    up.seg[0].b_mn = mn_over_other(w1_c);
     up.seg[0].K = d_m;
     up.epi = sw ? EPI_SWIGLU : (act == ECOSPA_ACT_GELU_ERF ? EPI_GELU_ERF : EPI_GELU_TANH);
     up.C = H; up.C2 = sw ? Hb : A; up.C3 = sw ? A : nullptr; up.ldc = ld_h;
@@ -747,8 +769,8 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_fwd(const void* X, int64_t ldx, in
     GemmOp down;  // Y = A W_2 (+ b_2)
     down.M = T; down.N = d_m; down.n_kseg = 1;
     down.seg[0].a.ptr = A; down.seg[0].a.rows = T; down.seg[0].a.cols = k; down.seg[0].a.ld = ld_h;
-    down.seg[0].b[0] = weight_bf16(cx, w2_c, d_m, k);  // stored k x d_m = [K][N]
-    down.seg[0].b_mn = true;
+    down.seg[0].b[0] = weight_bf16(cx, w2_c, d_m, k);  // stored k x d_m = [K][N], or d_m x k = [N][K]
+    down.seg[0].b_mn = mn_over_shared(w2_c);
     down.seg[0].K = k;
     down.epi = EPI_STORE; down.C = Y; down.ldc = ld_y; down.out_f32 = f32;
     down.bias = b2; down.bias_f32 = f32;
@@ -771,9 +793,9 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     Ctx cx;
     ecospa_status_t st = begin(cx, w1_c->dtype, workspace, workspace_bytes, stream, T, d_m, k);
     if (st != ECOSPA_OK) return st;
-    if ((st = check_weight(w1_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if (sw && (st = check_weight(w1b_c, d_m, k, ECOSPA_SHARED_COLS, cx.dtype)) != ECOSPA_OK) return st;
-    if ((st = check_weight(w2_c, d_m, k, ECOSPA_SHARED_ROWS, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(w1_c, d_m, k, cx.dtype)) != ECOSPA_OK) return st;
+    if (sw && (st = check_weight(w1b_c, d_m, k, cx.dtype)) != ECOSPA_OK) return st;
+    if ((st = check_weight(w2_c, d_m, k, cx.dtype)) != ECOSPA_OK) return st;
     if (ld_h < k || (ld_h * 2) % 16) return ld_h < k ? ECOSPA_ERR_INVALID : ECOSPA_ERR_ALIGNMENT;
     const bool f32 = cx.dtype == ECOSPA_F32;
     const Stored Xs = as_bf16(cx, X, T, d_m, ldx);
@@ -795,12 +817,12 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     GemmOp ops[kMaxGemmOps];
     PendingReduce red[3];
     int n_ops = 0;
-    n_ops = add_wgrad(cx, ops, n_ops, As, dYs, k, d_m, T, dW2_c, ld_dw2, &red[0], 1,
-                      gemm_cost(k, d_m, T) + nw * gemm_cost(T, k, d_m));                                     // dW_2 (k x d_m)
+    n_ops = add_wgrad_w(cx, ops, n_ops, w2_c, dYs, As, d_m, k, T, dW2_c, ld_dw2, &red[0], 1,
+                        gemm_cost(k, d_m, T) + nw * gemm_cost(T, k, d_m));                                   // dW_2, stored like W_2
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& da = ops[n_ops++];
     da.M = T; da.N = k; da.n_kseg = 1;
-    da.seg[0].a = dYs; da.seg[0].b[0] = W2; da.seg[0].K = d_m;
+    da.seg[0].a = dYs; da.seg[0].b[0] = W2; da.seg[0].b_mn = mn_over_other(w2_c); da.seg[0].K = d_m;
     da.epi = sw ? EPI_DSWIGLU : (act == ECOSPA_ACT_GELU_ERF ? EPI_DGELU_ERF : EPI_DGELU_TANH);
     da.C = const_cast<void*>(dH.ptr); da.C2 = sw ? const_cast<void*>(dHb.ptr) : nullptr; da.ldc = dH.ld;
     da.H = H; da.Hb = Hb; da.ldh = ld_h;
@@ -809,15 +831,15 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     // Second: dW_1 = X^T dH (and dW_up = X^T dH_up), dX = dH W_1^T (+ dH_up W_up^T)
     n_ops = 0;
     const int64_t cost = nw * gemm_cost(d_m, k, T) + gemm_cost(T, d_m, nw * k);
-    n_ops = add_wgrad(cx, ops, n_ops, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1, cost);           // dW_1 (d_m x k)
-    if (sw) n_ops = add_wgrad(cx, ops, n_ops, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1, cost);           // dW_up
+    n_ops = add_wgrad_w(cx, ops, n_ops, w1_c, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1, cost);   // dW_1, stored like W_1
+    if (sw) n_ops = add_wgrad_w(cx, ops, n_ops, w1b_c, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1, cost); // dW_up
     if (cx.st != ECOSPA_OK) return cx.st;
     GemmOp& dx = ops[n_ops++];
     dx = GemmOp();
     dx.M = T; dx.N = d_m; dx.n_kseg = sw ? 2 : 1;
-    dx.seg[0].a = dH; dx.seg[0].b[0] = W1; dx.seg[0].K = k;
+    dx.seg[0].a = dH; dx.seg[0].b[0] = W1; dx.seg[0].b_mn = mn_over_shared(w1_c); dx.seg[0].K = k;
     if (sw) {
-        dx.seg[1].a = dHb; dx.seg[1].b[0] = W1b; dx.seg[1].K = k;
+        dx.seg[1].a = dHb; dx.seg[1].b[0] = W1b; dx.seg[1].b_mn = mn_over_shared(w1b_c); dx.seg[1].K = k;
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;

@@ -187,6 +187,104 @@ def test_token_counts_that_end_inside_a_row_block():
     run_block_full(wl, [13, 6], 77, B.ACT_SWIGLU, T=77, seed=2)
 
 
+def run_block_other_orientation(wl, k_heads, k_ffn, act, T=None, seed=0):
+    """The same products with every weight stored the other way round (W_Q, W_K, W_V, W_1 as n x d_m, i.e. the
+    nn.Linear layout; W_O, W_2 as d_m x n): outputs must not change and weight gradients come back in the
+    orientation of their weight."""
+    eb = wl.elem_bytes
+    w = WL.layer_weights(wl, 0)
+    kept = random_kept(wl, k_heads, k_ffn, seed)
+    n, k = len(kept["attn"]), len(kept["ffn"])
+    wc = compact_cpu(w, kept, lambda m: BL.pad8(m, eb))
+    T = T or wl.tokens
+    npad, kpad = BL.pad8(n, eb), BL.pad8(k, eb)
+    acts = WL.activations(wl, 0, tokens=T, kinds=["x", "dy", "dout", "dq", "dk", "dv", "ctx"],
+                          widths={"dq": npad, "dk": npad, "dv": npad, "ctx": npad})
+    a = {kk: v.to(DEV) for kk, v in acts.items()}
+    dt = wl.torch_dtype
+
+    def rows(t, m):            # d_m x pitch  ->  m x d_m
+        return t[:, :m].t().contiguous().to(DEV)
+
+    def cols(t, m, pad):       # m x d_m  ->  d_m x pitch, pad columns zero
+        o = torch.zeros((t.shape[1], pad), dtype=t.dtype)
+        o[:, :m] = t.t()
+        return o.to(DEV)
+
+    d = {"wq": rows(wc["wq"], n), "wk": rows(wc["wk"], n), "wv": rows(wc["wv"], n), "wo": cols(wc["wo"], n, npad),
+         "w1": rows(wc["w1"], k), "w2": cols(wc["w2"], k, kpad)}
+    if "w1b" in wc:
+        d["w1b"] = rows(wc["w1b"], k)
+    bias = {nm: wc[nm].to(DEV) for nm in ("bq", "bk", "bv", "b1", "b2") if nm in wc}
+    code = B.F32 if dt == torch.float32 else B.BF16
+    ws = torch.empty(B.ecospa_proj_workspace_bytes(T, wl.d_m, n, code) + 16, dtype=torch.uint8, device=DEV)
+    lay = dict(w_in_layout=B.SHARED_ROWS, w_out_layout=B.SHARED_COLS)
+    errs = {}
+    e = lambda *shape: torch.full(shape, 3.0, dtype=dt, device=DEV)
+
+    Q, K, V = e(T, npad), e(T, npad), e(T, npad)
+    B.ecospa_coupled_qkv_fwd(a["x"], d["wq"], d["wk"], d["wv"], n, n, Q, K, V, bq_c=bias.get("bq"), bk_c=bias.get("bk"),
+                             bv_c=bias.get("bv"), workspace=ws, **lay)
+    for nm, out in (("q", Q), ("k", K), ("v", V)):
+        errs[nm.upper()] = rel(out[:, :n], O.proj_fwd(acts["x"], wc["w" + nm], O.SHARED_COLS, n, bias=wc.get("b" + nm)))
+    Out = e(T, wl.d_m)
+    B.ecospa_coupled_vo_fwd_o(a["ctx"], d["wo"], n, Out, workspace=ws, **lay)
+    ctx_cpu = acts["ctx"][:, :n].contiguous()
+    errs["Out"] = rel(Out, O.outproj_fwd(ctx_cpu, wc["wo"], O.SHARED_ROWS, n, wl.d_m))
+
+    dCtx, dWo, dbo = e(T, npad), e(wl.d_m, npad), e(wl.d_m)
+    B.ecospa_coupled_vo_bwd_o(a["ctx"], d["wo"], n, a["dout"], dCtx, dWo, dbo, workspace=ws, **lay)
+    rdCtx, rdWo, rdbo = O.outproj_bwd(ctx_cpu, wc["wo"], O.SHARED_ROWS, n, wl.d_m, acts["dout"], want_db=True)
+    errs["dCtx"] = rel(dCtx[:, :n], rdCtx); errs["dWo"] = rel(dWo[:, :n], rdWo); errs["dbo"] = rel(dbo, rdbo)
+
+    dX = e(T, wl.d_m)
+    dWq, dWk, dWv = e(n, wl.d_m), e(n, wl.d_m), e(n, wl.d_m)
+    B.ecospa_coupled_qkv_bwd(a["x"], d["wq"], d["wk"], d["wv"], n, n, a["dq"], a["dk"], a["dv"], dX, dWq, dWk, dWv,
+                             workspace=ws, **lay)
+    ref_dx = None
+    for nm, dW in (("q", dWq), ("k", dWk), ("v", dWv)):
+        up = acts["d" + nm][:, :n].contiguous()
+        ref_dx, rdW, _ = O.proj_bwd(acts["x"], wc["w" + nm], O.SHARED_COLS, n, up, dX=ref_dx)
+        errs["dW" + nm] = rel(dW, rdW.T)
+    errs["dX"] = rel(dX, ref_dx)
+
+    sw = act == B.ACT_SWIGLU
+    buf = L.ffn_buffers(T, wl.d_m, k, act, dt, DEV)
+    buf["dW1"] = e(k, wl.d_m); buf["dW2"] = e(wl.d_m, kpad)
+    if sw:
+        buf["dW1b"] = e(k, wl.d_m)
+    B.ecospa_coupled_ffn_fwd(a["x"], act, d["w1"], d["w2"], k, buf["Y"], buf["H"], buf["A"], w1b_c=d.get("w1b"),
+                             Hb=buf.get("Hb"), b1_c=None if sw else bias.get("b1"), b2=None if sw else bias.get("b2"),
+                             workspace=buf["ws"], **lay)
+    B.ecospa_coupled_ffn_bwd(a["x"], act, d["w1"], d["w2"], k, buf["H"], buf["A"], a["dy"], buf["dX"], buf["dW1"],
+                             buf["dW2"], w1b_c=d.get("w1b"), Hb=buf.get("Hb"), dW1b_c=buf.get("dW1b"),
+                             db1_c=buf.get("db1"), db2=buf["db2"], workspace=buf["ws"], **lay)
+    B.ecospa_device_status()
+    b1 = None if sw else wc.get("b1")
+    b2 = None if sw else wc.get("b2")
+    rf = O.ffn_fwd(acts["x"], act, wc["w1"], wc["w2"], O.SHARED_COLS, O.SHARED_ROWS, k, W1b=wc.get("w1b"), b1=b1, b2=b2)
+    rb = O.ffn_bwd(acts["x"], act, wc["w1"], wc["w2"], O.SHARED_COLS, O.SHARED_ROWS, k, acts["dy"], W1b=wc.get("w1b"),
+                   b1=b1, want_bias=True)
+    errs["Y"] = rel(buf["Y"], rf["Y"]); errs["A"] = rel(buf["A"][:, :k], rf["A"])
+    errs["ffn.dX"] = rel(buf["dX"], rb["dX"]); errs["dW1"] = rel(buf["dW1"], rb["dW1"].T)
+    errs["dW2"] = rel(buf["dW2"][:, :k], rb["dW2"])
+    if sw:
+        errs["dW1b"] = rel(buf["dW1b"], rb["dW1b"].T)
+    else:
+        errs["db1"] = rel(buf["db1"], rb["db1"])
+    check(errs)
+
+
+def test_weights_stored_the_other_way_round():
+    wl = WL.WORKLOADS["tails768"]
+    k_heads = [WL.RAGGED_HEAD_KEPT[i % len(WL.RAGGED_HEAD_KEPT)] for i in range(wl.n_heads)]
+    run_block_other_orientation(wl, k_heads, 1337, B.ACT_GELU_ERF)
+    wl = WL.WORKLOADS["tiny_swiglu"]
+    run_block_other_orientation(wl, [13, 6], 77, B.ACT_SWIGLU, seed=1)
+    wl = WL.WORKLOADS["block_f32"]
+    run_block_other_orientation(wl, [32] * wl.n_heads, 512, B.ACT_GELU_ERF)
+
+
 def test_gelu_tanh_variant_small():
     wl = WL.WORKLOADS["tails768"]
     run_block_full(wl, [32] * wl.n_heads, 264, B.ACT_GELU_TANH, T=96)
