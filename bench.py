@@ -313,31 +313,61 @@ def run_gpu(args):
     ms_gemm = sum(b.elapsed_time(c) for _, b, c in marks) / args.steps
     ms_step = ms_total / args.steps
 
-    # ---- end to end: inputs start in pinned host memory, results are read back
+    # ---- end to end: every step's inputs start in pinned host memory and its results are read back.
+    # Two device-side copies of the model take turns, so the upload of step s + 1 (copy stream) runs while
+    # step s computes; every step still pays its own upload and read-back inside the timed region.
     host = m.host_copies()
     h2d = sum(h.numel() * h.element_size() for h, _ in host)
-    res_host = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (m.kept, m.fis, m.ups)]
-    chk_host = torch.empty(1, dtype=torch.float32, pin_memory=True)
-    d2h = sum(t.numel() * t.element_size() for t in res_host) + 4
+    m2 = Model(wl, args.sparsity, dev)
+    for _ in range(3):
+        m2.sparsify(); m2.layers()
+    if args.no_graph:
+        replay = [(sparsify, layers), (m2.sparsify, m2.layers)]
+    else:
+        g2_sp, g2_ly = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g2_sp):
+            m2.sparsify()
+        with torch.cuda.graph(g2_ly):
+            m2.layers()
+        replay = [(sparsify, layers), (g2_sp.replay, g2_ly.replay)]
+    models = [m, m2]
+    dev_in = [[d for _, d in host], [t for dd in m2.w + m2.g + m2.acts for t in dd.values()]]
+    host_in = [h for h, _ in host]
+    assert all(a.shape == b.shape and a.dtype == b.dtype for a, b in zip(dev_in[0], dev_in[1]))
+    res_host = [[torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in (mm.kept, mm.fis, mm.ups)] for mm in models]
+    chk_host = torch.empty(2, dtype=torch.float32, pin_memory=True)
+    d2h = sum(t.numel() * t.element_size() for t in res_host[0]) + 4
+    copy_stream = torch.cuda.Stream(device=dev)
+    copied = [torch.cuda.Event(), torch.cuda.Event()]
+    done = [torch.cuda.Event(), torch.cuda.Event()]
 
-    def e2e_step():
-        for h, d in host:
-            d.copy_(h, non_blocking=True)
-        sparsify(); layers()
-        for h, d in zip(res_host, (m.kept, m.fis, m.ups)):
-            h.copy_(d, non_blocking=True)
-        chk_host.copy_(m.o["dX"][0, :1].float(), non_blocking=True)
+    def e2e_steps_run(n):
+        cur = torch.cuda.current_stream()
+        for s_i in range(n):
+            b = s_i % 2
+            mm = models[b]
+            with torch.cuda.stream(copy_stream):
+                copy_stream.wait_event(done[b])               # the previous step on this copy of the model is over
+                for h, d in zip(host_in, dev_in[b]):
+                    d.copy_(h, non_blocking=True)
+                copied[b].record(copy_stream)
+            cur.wait_event(copied[b])
+            replay[b][0](); replay[b][1]()
+            for h, d in zip(res_host[b], (mm.kept, mm.fis, mm.ups)):
+                h.copy_(d, non_blocking=True)
+            chk_host[b:b + 1].copy_(mm.o["dX"][0, :1].float(), non_blocking=True)
+            done[b].record(cur)
 
-    e2e_steps = max(2, min(args.steps, 5))
-    e2e_step()
+    e2e_steps = max(4, min(args.steps, 8))
+    e2e_steps_run(2)
     barrier()
     e0, e1 = ev(), ev()
     e0.record()
-    for _ in range(e2e_steps):
-        e2e_step()
+    e2e_steps_run(e2e_steps)
     e1.record()
     barrier()
     ms_e2e = e0.elapsed_time(e1) / e2e_steps
+    B.ecospa_device_status()
 
     ms_step, ms_sp, ms_gemm, ms_e2e = max_over_ranks([ms_step, ms_sp, ms_gemm, ms_e2e], dev)
 
@@ -368,7 +398,8 @@ def run_gpu(args):
                      "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                      "launches_per_step": n_gemm_launches, "avg_launch_ms": ms_gemm / n_gemm_launches},
         "e2e": {"value": job_throughput(world, flops, ms_e2e) / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
-                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "pipeline": "two device copies of the model: the upload of step s+1 overlaps the compute of step s"},
         "gpu_launches": int(launches), "clocks": clocks,
     }
     if rank == 0:
