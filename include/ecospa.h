@@ -62,13 +62,23 @@ typedef struct {
     int64_t ld;        /* elements; >= D (SHARED_COLS) or >= other_dim (SHARED_ROWS) */
 } ecospa_mat_t;
 
+/* Rotary position embedding (Eq. "self-attention-rope"): W_Q P_t and W_K P_s rotate the shared index in 2 x 2
+ * blocks, so the unit that can be removed ("position matrices are then adjusted to match new dimensions",
+ * footnote to Eq. "l2norm") is a rotation pair of shared indices, and the rotations leave the Frobenius norm of a
+ * pair's two columns unchanged at every position.  Which two indices of a segment form pair b: */
+typedef enum {
+    ECOSPA_ROPE_NONE = 0,        /* no rotation: every shared index is scored and removed on its own */
+    ECOSPA_ROPE_INTERLEAVED = 1, /* (2b, 2b+1), the blocks as the paper prints them */
+    ECOSPA_ROPE_HALF = 2         /* (b, b + seg_len/2), the "rotate half" storage of the same blocks */
+} ecospa_rope_t;
+
 /* One stored group of coupled pairs.  w1b/g1b only for ECOSPA_PAIR_SWIGLU (w1 = gate, w1b = up).
  * g1/g1b/g2 are dL/dW of w1/w1b/w2 in the same shape and layout; ptr == NULL skips Fisher. */
 typedef struct {
     int32_t kind;    /* ecospa_pair_kind_t */
     int32_t n_seg;   /* pairs stored side by side (heads); 1 for an FFN */
     int32_t seg_len; /* shared indices per pair (d_h, or the FFN hidden width) */
-    int32_t reserved;
+    int32_t rope;    /* ecospa_rope_t: rotary position embedding acts on this pair group's shared index (Q/K pairs) */
     ecospa_mat_t w1, w1b, w2;
     ecospa_mat_t g1, g1b, g2;
 } ecospa_pair_t;
@@ -96,6 +106,11 @@ uint64_t ecospa_launch_count(void);
  *   upsilon[j] = raw[j] / ||raw[segment of j]||_2             (0 if the segment is all zero)
  *   fisher[s]  = 1/2 * ( SS(G_1, s)/|W_1,s| + SS(G_2, s)/|W_2,s| ) / n_samples
  *                (SwiGLU: the W_1 term is the mean of the gate and up terms)
+ *   pair.rope != ECOSPA_ROPE_NONE (plain pairs with an even seg_len only): the scored unit is a rotation pair
+ *   {j, j'} of shared indices,
+ *                raw[j] = raw[j'] = ||W_1[:, {j, j'}]||_F * ||W_2[{j, j'}, :]||_F,
+ *                upsilon[j] = upsilon[j'] = raw[j] / sqrt(sum over the segment's pairs of raw^2)
+ *                (both members carry the pair's value; select with ecospa_select_rotation_pairs)
  *
  * pairs      HOST  array of n_pairs descriptors (device tensors inside)
  * n_samples        |D| of Eq. "importance"; > 0
@@ -156,6 +171,17 @@ ecospa_status_t ecospa_score_pair_static(const ecospa_pair_t* pair, double n_sam
 ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, const int32_t* n_seg, const int32_t* seg_len,
                                            const int32_t* k_per_seg, int32_t n_pairs, int32_t* kept,
                                            int32_t* seg_offsets, void* stream);
+
+/* Step 2 with rotary position embedding: as ecospa_select_aligned_topk, but pair groups with rope[p] !=
+ * ECOSPA_ROPE_NONE keep whole rotation pairs (footnote to Eq. "l2norm": removal on W_Q / W_K, the position
+ * matrices shrink with them).  For such a group k_per_seg counts shared indices and must be even, seg_len must be
+ * even; the k/2 pairs with the largest score stay (the score is read at a pair's first member; equal scores: the
+ * lower pair first).  Kept indices are ascending; for ECOSPA_ROPE_HALF that puts the first members of the kept
+ * pairs before their second members, so the compacted matrix keeps the (u, u + k/2) pairing.
+ * rope HOST [n_pairs] of ecospa_rope_t.  Everything else as in ecospa_select_aligned_topk. */
+ecospa_status_t ecospa_select_rotation_pairs(const float* upsilon, const int32_t* n_seg, const int32_t* seg_len,
+                                             const int32_t* k_per_seg, const int32_t* rope, int32_t n_pairs,
+                                             int32_t* kept, int32_t* seg_offsets, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Step 2, variable counts: the stopping rule of Algorithm 1 ("while the sum of the scores exceeds theta:

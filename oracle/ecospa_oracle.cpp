@@ -10,6 +10,9 @@
 //                                  (numerator), SwiGLU W_1 = W_gate (.) W_up
 //                                  from the footnote to Eq. "importance".
 //   eco_upsilon                  : Eq. "l2norm" (per coupled pair = per segment).
+//   eco_upsilon_rope / eco_select_rotation_pairs_f32 : the same score and removal with rotary position
+//                                  embedding (Eq. "self-attention-rope", footnote to Eq. "l2norm"): rotation
+//                                  pairs of shared indices as the unit.
 //   eco_fisher_pair              : Eq. "importance".
 //   eco_select_topk_*            : Definition 1 (aligned removal) applied to
 //                                  the (seg_len - k) lowest-scored indices.
@@ -144,6 +147,50 @@ void eco_upsilon(const double* c1, const double* c2, int n_seg, int seg_len, dou
         }
         const double nrm = std::sqrt(nrm2);
         for (int j = 0; j < seg_len; ++j) upsilon[o + j] = nrm > 0.0 ? raw[o + j] / nrm : 0.0;
+    }
+}
+
+// With rotary position embedding (Eq. "self-attention-rope") W_Q P_t and W_K P_s rotate the shared index in
+// 2 x 2 blocks, and the footnote to Eq. "l2norm" removes on W_Q / W_K and shrinks the position matrices with them:
+// the removable unit is a rotation pair {a, b} of shared indices.  Its score is the Eq. "l2norm" score of the pair
+// taken as one unit: raw = ||W_1[:, {a,b}]||_F * ||W_2[{a,b}, :]||_F = sqrt(c1[a] + c1[b]) * sqrt(c2[a] + c2[b])
+// (a rotation of the two columns does not change it), normalised over the segment's seg_len/2 units.  Both
+// members of a pair carry the pair's value.  mode 1: pairs (2u, 2u+1); mode 2: pairs (u, u + seg_len/2).
+void eco_upsilon_rope(const double* c1, const double* c2, int n_seg, int seg_len, int mode, double* raw, double* upsilon) {
+    const int half = seg_len / 2;
+    for (int s = 0; s < n_seg; ++s) {
+        const int64_t o = static_cast<int64_t>(s) * seg_len;
+        double nrm2 = 0.0;
+        for (int u = 0; u < half; ++u) {
+            const int a = mode == 1 ? 2 * u : u, b = mode == 1 ? 2 * u + 1 : u + half;
+            const double r = std::sqrt(c1[o + a] + c1[o + b]) * std::sqrt(c2[o + a] + c2[o + b]);
+            raw[o + a] = raw[o + b] = r;
+            nrm2 += r * r;
+        }
+        const double nrm = std::sqrt(nrm2);
+        for (int j = 0; j < seg_len; ++j) upsilon[o + j] = nrm > 0.0 ? raw[o + j] / nrm : 0.0;
+    }
+}
+
+// Aligned removal of whole rotation pairs: per segment the k/2 units with the largest score stay (equal scores:
+// lower unit first; a unit's score is read at its first member); kept indices ascending.
+void eco_select_rotation_pairs_f32(const float* upsilon, int n_seg, int seg_len, const int32_t* k, int mode, int32_t* kept) {
+    const int half = seg_len / 2;
+    int64_t w = 0;
+    for (int s = 0; s < n_seg; ++s) {
+        const int64_t o = static_cast<int64_t>(s) * seg_len;
+        std::vector<int32_t> order(half);
+        std::iota(order.begin(), order.end(), 0);
+        auto unit_score = [&](int32_t u) { return upsilon[o + (mode == 1 ? 2 * u : u)]; };
+        std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return unit_score(a) > unit_score(b); });
+        std::vector<int32_t> idx;
+        for (int i = 0; i < k[s] / 2; ++i) {
+            const int32_t u = order[i];
+            idx.push_back(mode == 1 ? 2 * u : u);
+            idx.push_back(mode == 1 ? 2 * u + 1 : u + half);
+        }
+        std::sort(idx.begin(), idx.end());
+        for (int32_t c : idx) kept[w++] = static_cast<int32_t>(o) + c;
     }
 }
 

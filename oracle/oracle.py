@@ -109,21 +109,36 @@ def sumsq_shared_hadamard(gate, up, layout: int) -> np.ndarray:
     return out
 
 
-def upsilon(c1: np.ndarray, c2: np.ndarray, n_seg: int, seg_len: int):
+def upsilon(c1: np.ndarray, c2: np.ndarray, n_seg: int, seg_len: int, rope: int = 0):
     c1 = np.ascontiguousarray(c1, dtype=np.float64)
     c2 = np.ascontiguousarray(c2, dtype=np.float64)
     assert c1.size == c2.size == n_seg * seg_len
     raw = np.empty_like(c1)
     ups = np.empty_like(c1)
-    lib().eco_upsilon(_p(c1), _p(c2), n_seg, seg_len, _p(raw), _p(ups))
+    if rope:
+        assert seg_len % 2 == 0
+        lib().eco_upsilon_rope(_p(c1), _p(c2), n_seg, seg_len, int(rope), _p(raw), _p(ups))
+    else:
+        lib().eco_upsilon(_p(c1), _p(c2), n_seg, seg_len, _p(raw), _p(ups))
     return raw, ups
 
 
-def score_pair(w1, w2, layout1: int, layout2: int, n_seg: int, seg_len: int, w1b=None):
-    """(raw, upsilon) of a coupled pair; w1b given = SwiGLU pair with W_1 = w1 (.) w1b."""
+def score_pair(w1, w2, layout1: int, layout2: int, n_seg: int, seg_len: int, w1b=None, rope: int = 0):
+    """(raw, upsilon) of a coupled pair; w1b given = SwiGLU pair with W_1 = w1 (.) w1b; rope = 1 / 2: rotation
+    pairs (2u, 2u+1) / (u, u + seg_len/2) of shared indices are the scored unit."""
     c1 = sumsq_shared(w1, layout1) if w1b is None else sumsq_shared_hadamard(w1, w1b, layout1)
     c2 = sumsq_shared(w2, layout2)
-    return upsilon(c1, c2, n_seg, seg_len)
+    return upsilon(c1, c2, n_seg, seg_len, rope)
+
+
+def select_rotation_pairs(ups, n_seg: int, seg_len: int, k: Sequence[int], rope: int) -> np.ndarray:
+    """Ascending kept indices, whole rotation pairs only (k even), fp32 scores ranked as stored."""
+    k = _i32(k)
+    assert k.size == n_seg and (k % 2 == 0).all() and (k <= seg_len).all() and rope in (1, 2)
+    ups = np.ascontiguousarray(ups, dtype=np.float32)
+    kept = np.empty(int(k.sum()), dtype=np.int32)
+    lib().eco_select_rotation_pairs_f32(_p(ups), n_seg, seg_len, _p(k), int(rope), _p(kept))
+    return kept
 
 
 def fisher_pair(g1, g2, layout1: int, layout2: int, n_seg: int, seg_len: int, n_samples: float, g1b=None):

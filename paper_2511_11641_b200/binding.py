@@ -21,6 +21,7 @@ F32, BF16 = 0, 1
 SHARED_COLS, SHARED_ROWS = 0, 1
 PAIR_PLAIN, PAIR_SWIGLU = 0, 1
 ACT_NONE, ACT_GELU_ERF, ACT_GELU_TANH, ACT_SWIGLU = 0, 1, 2, 3
+ROPE_NONE, ROPE_INTERLEAVED, ROPE_HALF = 0, 1, 2
 
 
 class EcospaError(RuntimeError):
@@ -38,7 +39,7 @@ class Mat(C.Structure):
 
 
 class Pair(C.Structure):
-    _fields_ = [("kind", C.c_int32), ("n_seg", C.c_int32), ("seg_len", C.c_int32), ("reserved", C.c_int32),
+    _fields_ = [("kind", C.c_int32), ("n_seg", C.c_int32), ("seg_len", C.c_int32), ("rope", C.c_int32),
                 ("w1", Mat), ("w1b", Mat), ("w2", Mat), ("g1", Mat), ("g1b", Mat), ("g2", Mat)]
 
 
@@ -108,8 +109,8 @@ def mat(t: Optional[torch.Tensor], layout: int) -> Mat:
 
 
 def pair(kind: int, n_seg: int, seg_len: int, w1, w2, layout1: int, layout2: int, w1b=None,
-         g1=None, g2=None, g1b=None) -> Pair:
-    p = Pair(kind, n_seg, seg_len, 0, mat(w1, layout1), mat(w1b, layout1), mat(w2, layout2),
+         g1=None, g2=None, g1b=None, rope: int = 0) -> Pair:
+    p = Pair(kind, n_seg, seg_len, rope, mat(w1, layout1), mat(w1b, layout1), mat(w2, layout2),
              mat(g1, layout1), mat(g1b, layout1), mat(g2, layout2))
     p._keep = (w1, w2, w1b, g1, g2, g1b)   # keep the tensors alive as long as the descriptor
     return p
@@ -168,6 +169,25 @@ def ecospa_select_aligned_topk(upsilon: torch.Tensor, n_seg: Sequence[int], seg_
                                           n_pairs, _ptr(kept), _ptr(seg_offsets), _stream(stream))
     if st != 0:
         raise EcospaError(st, "ecospa_select_aligned_topk")
+
+
+def ecospa_select_rotation_pairs(upsilon: torch.Tensor, n_seg: Sequence[int], seg_len: Sequence[int],
+                                 k_per_seg: Sequence[int], rope: Sequence[int], kept: torch.Tensor,
+                                 seg_offsets: Optional[torch.Tensor] = None, stream=None) -> None:
+    n_pairs = len(n_seg)
+    a_nseg = (C.c_int32 * n_pairs)(*n_seg)
+    a_slen = (C.c_int32 * n_pairs)(*seg_len)
+    a_rope = (C.c_int32 * n_pairs)(*rope)
+    a_k = (C.c_int32 * len(k_per_seg))(*k_per_seg)
+    assert len(k_per_seg) == sum(n_seg) and len(rope) == n_pairs
+    assert kept.dtype == torch.int32 and kept.numel() >= sum(k_per_seg)
+    fn = lib().ecospa_select_rotation_pairs
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    st = fn(_ptr(upsilon), C.addressof(a_nseg), C.addressof(a_slen), C.addressof(a_k), C.addressof(a_rope), n_pairs,
+            _ptr(kept), _ptr(seg_offsets), _stream(stream))
+    if st != 0:
+        raise EcospaError(st, "ecospa_select_rotation_pairs")
 
 
 def ecospa_choose_pairs(fisher: torch.Tensor, m: int, chosen: torch.Tensor, stream=None) -> None:

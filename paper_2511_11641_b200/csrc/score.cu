@@ -58,8 +58,10 @@ struct PairDesc {
     int32_t d_off;      // offset of this pair in upsilon / raw
     int32_t seg_start;  // first global segment index (also offset into fisher)
     float inv_numel1, inv_numel2;
+    int32_t rope;       // ecospa_rope_t: the scored unit is a rotation pair of shared indices
+    int32_t pad_;
 };
-static_assert(sizeof(PairDesc) == 64, "pair descriptor size");
+static_assert(sizeof(PairDesc) == 72, "pair descriptor size");
 
 struct FinalizeParams {
     int32_t n_pairs;
@@ -257,14 +259,24 @@ __global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constan
     const float* c1 = Q.c1 + base;
     const float* c2 = Q.c2 + base;
 
+    // raw score of index j: its own column/row norms, or those of its rotation pair (both members get the
+    // pair's value; the pair is counted once in the normaliser)
+    const int half = Q.seg_len >> 1;
+    auto raw_of = [&](int j) -> float {
+        if (Q.rope == ECOSPA_ROPE_NONE) return sqrtf(c1[j]) * sqrtf(c2[j]);
+        const int a = Q.rope == ECOSPA_ROPE_INTERLEAVED ? (j & ~1) : (j < half ? j : j - half);
+        const int b = Q.rope == ECOSPA_ROPE_INTERLEAVED ? (a | 1) : a + half;
+        return sqrtf(c1[a] + c1[b]) * sqrtf(c2[a] + c2[b]);
+    };
     float ss = 0.f;
     for (int j = threadIdx.x; j < Q.seg_len; j += kThreads) {
-        const float r = sqrtf(c1[j]) * sqrtf(c2[j]);
+        const float r = raw_of(j);
         ss = fmaf(r, r, ss);
     }
-    const float nrm = sqrtf(block_sum<kWarps>(ss, scratch));
+    const float total = block_sum<kWarps>(ss, scratch);
+    const float nrm = sqrtf(Q.rope == ECOSPA_ROPE_NONE ? total : 0.5f * total);
     for (int j = threadIdx.x; j < Q.seg_len; j += kThreads) {
-        const float r = sqrtf(c1[j]) * sqrtf(c2[j]);
+        const float r = raw_of(j);
         if (P.raw) P.raw[Q.d_off + base + j] = r;
         P.upsilon[Q.d_off + base + j] = nrm > 0.f ? __fdiv_rn(r, nrm) : 0.f;
     }
@@ -320,6 +332,8 @@ ecospa_status_t validate_mat(const ecospa_mat_t& m, int64_t D, int want_dtype, i
 ecospa_status_t validate_pair(const ecospa_pair_t& p, bool need_grads) {
     if (p.kind != ECOSPA_PAIR_PLAIN && p.kind != ECOSPA_PAIR_SWIGLU) return ECOSPA_ERR_INVALID;
     if (p.n_seg < 1 || p.seg_len < 1) return ECOSPA_ERR_INVALID;
+    if (p.rope != ECOSPA_ROPE_NONE && p.rope != ECOSPA_ROPE_INTERLEAVED && p.rope != ECOSPA_ROPE_HALF) return ECOSPA_ERR_INVALID;
+    if (p.rope != ECOSPA_ROPE_NONE && (p.kind != ECOSPA_PAIR_PLAIN || (p.seg_len & 1))) return ECOSPA_ERR_INVALID;
     const int64_t D = static_cast<int64_t>(p.n_seg) * p.seg_len;
     if (D > (1 << 24)) return ECOSPA_ERR_UNSUPPORTED;
     ecospa_status_t st;
@@ -474,6 +488,7 @@ extern "C" ecospa_status_t ecospa_score_pairs(const ecospa_pair_t* pairs, int32_
             }
             Q.n_seg = pr.n_seg;
             Q.seg_len = pr.seg_len;
+            Q.rope = pr.rope;
             Q.d_off = d_off;
             Q.seg_start = segs;
             Q.inv_numel1 = static_cast<float>(1.0 / (static_cast<double>(pr.w1.other_dim) * pr.seg_len));

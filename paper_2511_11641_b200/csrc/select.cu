@@ -23,7 +23,7 @@ struct SelPair {
     int32_t seg_len;
     int32_t d_off;      // offset of the pair's scores in upsilon, and base added to nothing: kept
                         // indices are relative to the pair group (segment offset included)
-    int32_t pad_;
+    int32_t rope;       // ecospa_rope_t: units of two shared indices are ranked and kept together
 };
 
 struct SelectParams {
@@ -59,16 +59,22 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
         if (P.pairs[mid].seg_start <= seg) lo = mid; else hi = mid - 1;
     }
     const SelPair& Q = P.pairs[lo];
-    const int n = Q.seg_len;
+    const int seg_len = Q.seg_len;
     const int seg_in_pair = seg - Q.seg_start;
-    const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg_in_pair) * n;
-    const int out0 = P.k_dev ? Q.d_off + seg_in_pair * n : P.out_off[seg];
-    const int k = P.k_dev ? min(max(P.k_dev[P.seg_base + seg], 0), n) : P.out_off[seg + 1] - out0;
+    // With rotation pairs the ranked units are the seg_len/2 pairs; both members carry the pair's score, so
+    // unit u is read at index 2u (interleaved pairs) or u (pairs of the two halves).
+    const int rope = Q.rope;
+    const int n = rope ? seg_len >> 1 : seg_len;
+    const int stride = rope == ECOSPA_ROPE_INTERLEAVED ? 2 : 1;
+    const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg_in_pair) * seg_len;
+    const int out0 = P.k_dev ? Q.d_off + seg_in_pair * seg_len : P.out_off[seg];
+    const int k_idx = P.k_dev ? min(max(P.k_dev[P.seg_base + seg], 0), seg_len) : P.out_off[seg + 1] - out0;
+    const int k = rope ? k_idx >> 1 : k_idx;     // units to keep
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     if (P.seg_offsets && tid == 0) {
         P.seg_offsets[P.seg_base + seg] = out0;
-        if (P.is_last && seg == P.n_segs - 1) P.seg_offsets[P.seg_base + seg + 1] = out0 + k;
+        if (P.is_last && seg == P.n_segs - 1) P.seg_offsets[P.seg_base + seg + 1] = out0 + k_idx;
     }
     if (k <= 0) return;
 
@@ -79,7 +85,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
         hist[tid] = 0;
         __syncthreads();
         for (int j = tid; j < n; j += kThreads) {
-            const uint32_t key = order_key(__ldg(sc + j));
+            const uint32_t key = order_key(__ldg(sc + j * stride));
             if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255], 1);
         }
         __syncthreads();
@@ -122,13 +128,13 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     const bool all_eq = (want == cnt_eq);   // every element equal to the threshold is kept
 
     // ---- emit ascending: key > thr, plus the first `want` elements with key == thr
-    const int seg_first = seg_in_pair * n;  // kept indices are shared indices of the pair group
+    const int seg_first = seg_in_pair * seg_len;  // kept indices are shared indices of the pair group
     int run_eq = 0, run_out = 0;
     for (int base = 0; base < n; base += kThreads) {
         const int j = base + tid;
         uint32_t key = 0;
         bool valid = j < n;
-        if (valid) key = order_key(__ldg(sc + j));
+        if (valid) key = order_key(__ldg(sc + j * stride));
         const bool gt = valid && key > thr;
         const bool eq = valid && key == thr;
         bool sel;
@@ -160,7 +166,17 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
             tot += warp_tot[w];
         }
         run_out += tot;
-        if (sel && pos < k) P.kept[out0 + pos] = seg_first + j;
+        if (sel && pos < k) {
+            if (rope == ECOSPA_ROPE_NONE) {
+                P.kept[out0 + pos] = seg_first + j;
+            } else if (rope == ECOSPA_ROPE_INTERLEAVED) {           // members 2j, 2j + 1
+                P.kept[out0 + 2 * pos] = seg_first + 2 * j;
+                P.kept[out0 + 2 * pos + 1] = seg_first + 2 * j + 1;
+            } else {                                                // members j, j + seg_len/2: both halves ascending
+                P.kept[out0 + pos] = seg_first + j;
+                P.kept[out0 + k + pos] = seg_first + n + j;
+            }
+        }
         __syncthreads();
     }
 }
@@ -320,19 +336,22 @@ __global__ void __launch_bounds__(1024) choose_pairs_kernel(const float* __restr
 
 using namespace ecospa;
 
-extern "C" ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, const int32_t* n_seg,
-                                                      const int32_t* seg_len, const int32_t* k_per_seg,
-                                                      int32_t n_pairs, int32_t* kept, int32_t* seg_offsets,
-                                                      void* stream_) {
+static ecospa_status_t select_fixed_counts(const float* upsilon, const int32_t* n_seg, const int32_t* seg_len,
+                                           const int32_t* k_per_seg, const int32_t* rope, int32_t n_pairs,
+                                           int32_t* kept, int32_t* seg_offsets, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!upsilon || !n_seg || !seg_len || !k_per_seg || n_pairs < 1 || !kept) return ECOSPA_ERR_INVALID;
     int64_t total_segs = 0, total_d = 0, total_k = 0;
     for (int p = 0; p < n_pairs; ++p) {
         if (n_seg[p] < 1 || seg_len[p] < 1) return ECOSPA_ERR_INVALID;
         if (seg_len[p] > (1 << 20)) return ECOSPA_ERR_UNSUPPORTED;
+        const int32_t rp = rope ? rope[p] : ECOSPA_ROPE_NONE;
+        if (rp != ECOSPA_ROPE_NONE && rp != ECOSPA_ROPE_INTERLEAVED && rp != ECOSPA_ROPE_HALF) return ECOSPA_ERR_INVALID;
+        if (rp != ECOSPA_ROPE_NONE && (seg_len[p] & 1)) return ECOSPA_ERR_INVALID;
         for (int s = 0; s < n_seg[p]; ++s) {
             const int32_t k = k_per_seg[total_segs + s];
             if (k < 0 || k > seg_len[p]) return ECOSPA_ERR_INVALID;
+            if (rp != ECOSPA_ROPE_NONE && (k & 1)) return ECOSPA_ERR_INVALID;   // whole rotation pairs only
             total_k += k;
         }
         total_segs += n_seg[p];
@@ -353,7 +372,7 @@ extern "C" ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, cons
             Q.seg_start = ns - s_in_p;   // so that (seg - seg_start) is the segment index inside the pair
             Q.seg_len = seg_len[p];
             Q.d_off = d_off;
-            Q.pad_ = 0;
+            Q.rope = rope ? rope[p] : ECOSPA_ROPE_NONE;
             for (int s = 0; s < take; ++s) {
                 sp.out_off[ns++] = out;
                 out += k_per_seg[seg_global++];
@@ -378,6 +397,21 @@ extern "C" ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, cons
         if (st != ECOSPA_OK) return st;
     }
     return ECOSPA_OK;
+}
+
+extern "C" ecospa_status_t ecospa_select_aligned_topk(const float* upsilon, const int32_t* n_seg,
+                                                      const int32_t* seg_len, const int32_t* k_per_seg,
+                                                      int32_t n_pairs, int32_t* kept, int32_t* seg_offsets,
+                                                      void* stream) {
+    return select_fixed_counts(upsilon, n_seg, seg_len, k_per_seg, nullptr, n_pairs, kept, seg_offsets, stream);
+}
+
+extern "C" ecospa_status_t ecospa_select_rotation_pairs(const float* upsilon, const int32_t* n_seg,
+                                                        const int32_t* seg_len, const int32_t* k_per_seg,
+                                                        const int32_t* rope, int32_t n_pairs, int32_t* kept,
+                                                        int32_t* seg_offsets, void* stream) {
+    if (!rope) return ECOSPA_ERR_INVALID;
+    return select_fixed_counts(upsilon, n_seg, seg_len, k_per_seg, rope, n_pairs, kept, seg_offsets, stream);
 }
 
 extern "C" ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon, const int32_t* n_seg,
@@ -408,7 +442,7 @@ extern "C" ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon,
             Q.seg_start = ns - s_in_p;
             Q.seg_len = seg_len[p];
             Q.d_off = d_off;
-            Q.pad_ = 0;
+            Q.rope = ECOSPA_ROPE_NONE;
             tp.pairs[np] = Q;
             ++np;
             ns += take;

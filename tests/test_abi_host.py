@@ -134,3 +134,22 @@ def test_threshold_selection_rejects_bad_arguments_without_launching(lib):
     assert ch(ups, 0, 1, kept, None) == 1
     assert ch(ups, 4, -1, kept, None) == 1
     assert ch(ups, 1 << 15, 1, kept, None) == 3
+
+
+def test_rotation_pair_selection_rejects_bad_arguments_without_launching(lib):
+    fn = lib.ecospa_select_rotation_pairs
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    ups, kept = C.c_void_p(0x1000), C.c_void_p(0x2000)
+    one = (C.c_int32 * 1)(1)
+
+    def call(seg_len, k, mode, rope_null=False):
+        sl, kk, rp = (C.c_int32 * 1)(seg_len), (C.c_int32 * 1)(k), (C.c_int32 * 1)(mode)
+        return fn(ups, C.addressof(one), C.addressof(sl), C.addressof(kk), None if rope_null else C.addressof(rp), 1,
+                  kept, None, None)
+
+    assert call(64, 31, 1) == 1          # an odd count would split a rotation pair
+    assert call(63, 30, 2) == 1          # a segment of odd length has no pairing
+    assert call(64, 32, 3) == 1          # unknown pairing
+    assert call(64, 66, 1) == 1          # more than the segment holds
+    assert call(64, 32, 1, rope_null=True) == 1
