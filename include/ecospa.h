@@ -200,6 +200,9 @@ ecospa_status_t ecospa_select_rotation_pairs(const float* upsilon, const int32_t
  *   keep everything (chosen may be NULL: every segment is processed).
  *   upsilon  DEVICE fp32, concatenated as written by ecospa_score_pairs
  *   n_seg, seg_len HOST [n_pairs]
+ *   rope     HOST [n_pairs] of ecospa_rope_t, may be NULL (no rotation pairs).  A group with rotation pairs is
+ *            processed pair by pair: every pair's score counts once, pairs leave whole, k_out is even and at
+ *            least k_min rounded up to whole pairs (scores as written by ecospa_score_pairs for such a group)
  *   chosen   DEVICE int32 per segment (all pairs concatenated), may be NULL
  *   kept     DEVICE out int32 with one slot per shared index (sum of n_seg * seg_len entries): segment s of
  *            a pair writes its kept indices, ascending and relative to the pair group as in
@@ -211,8 +214,9 @@ ecospa_status_t ecospa_select_rotation_pairs(const float* upsilon, const int32_t
  */
 ecospa_status_t ecospa_choose_pairs(const float* fisher, int32_t n, int32_t m, int32_t* chosen, void* stream);
 ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon, const int32_t* n_seg, const int32_t* seg_len,
-                                                int32_t n_pairs, double theta, int32_t l1, int32_t k_min,
-                                                const int32_t* chosen, int32_t* kept, int32_t* k_out, void* stream);
+                                                const int32_t* rope, int32_t n_pairs, double theta, int32_t l1,
+                                                int32_t k_min, const int32_t* chosen, int32_t* kept, int32_t* k_out,
+                                                void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Step 3: physical removal.   Definition 1: drop column j of W_1 and row j of W_2 for every removed j

@@ -271,14 +271,22 @@ void eco_select_topk_f32(const float* upsilon, int n_seg, int seg_len, const int
 // fraction of the score mass that stays), 1 otherwise (the scores are compared with theta as stored).
 // chosen == nullptr: every segment is processed; otherwise segments with chosen[s] == 0 keep everything.
 // Output: how many indices stay per segment.  Scores are taken as stored fp32 values (exactly widened).
-void eco_threshold_counts_f32(const float* upsilon, int n_seg, int seg_len, double theta, int l1, int k_min,
+// rope != 0 (rotation pairs, see eco_upsilon_rope): the units are the seg_len/2 pairs, each with the score stored at
+// its first member and counted once; whole pairs leave; the result counts indices (even) and does not go below
+// k_min rounded up to whole pairs.
+void eco_threshold_counts_f32(const float* upsilon, int n_seg, int seg_len_idx, int rope, double theta, int l1, int k_min_idx,
                               const int32_t* chosen, int32_t* k_out) {
+    const int unit = rope ? 2 : 1;
+    const int seg_len = seg_len_idx / unit;
+    const int k_min = std::min((k_min_idx + unit - 1) / unit, seg_len);
+    std::vector<float> units(seg_len);
     for (int s = 0; s < n_seg; ++s) {
         if (chosen && !chosen[s]) {
-            k_out[s] = seg_len;
+            k_out[s] = seg_len_idx;
             continue;
         }
-        const float* u = upsilon + static_cast<int64_t>(s) * seg_len;
+        for (int j = 0; j < seg_len; ++j) units[j] = upsilon[static_cast<int64_t>(s) * seg_len_idx + (rope == 1 ? 2 * j : j)];
+        const float* u = units.data();
         std::vector<int32_t> order(seg_len);
         std::iota(order.begin(), order.end(), 0);
         std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return u[a] > u[b]; });
@@ -295,7 +303,7 @@ void eco_threshold_counts_f32(const float* upsilon, int n_seg, int seg_len, doub
             if (!(sum > budget)) break;
             --left;                                 // order[left] was the smallest one left
         }
-        k_out[s] = left;
+        k_out[s] = left * unit;
     }
 }
 

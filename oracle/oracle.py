@@ -169,13 +169,13 @@ def select_topk(ups, n_seg: int, seg_len: int, k: Sequence[int]) -> np.ndarray:
 
 
 def threshold_counts(ups, n_seg: int, seg_len: int, theta: float, l1: bool = True, k_min: int = 1,
-                     chosen=None) -> np.ndarray:
+                     chosen=None, rope: int = 0) -> np.ndarray:
     """Kept count per segment after Algorithm 1's cumulative-threshold loop (fp32 scores as stored)."""
     ups = np.ascontiguousarray(ups, dtype=np.float32)
     assert ups.size == n_seg * seg_len
     k = np.empty(n_seg, dtype=np.int32)
     ch = _i32(chosen) if chosen is not None else None
-    lib().eco_threshold_counts_f32(_p(ups), n_seg, seg_len, C.c_double(theta), int(l1), int(k_min), _p(ch), _p(k))
+    lib().eco_threshold_counts_f32(_p(ups), n_seg, seg_len, int(rope), C.c_double(theta), int(l1), int(k_min), _p(ch), _p(k))
     return k
 
 

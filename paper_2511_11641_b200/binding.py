@@ -202,18 +202,20 @@ def ecospa_choose_pairs(fisher: torch.Tensor, m: int, chosen: torch.Tensor, stre
 
 def ecospa_select_aligned_threshold(upsilon: torch.Tensor, n_seg: Sequence[int], seg_len: Sequence[int], theta: float,
                                     kept: torch.Tensor, k_out: torch.Tensor, l1: bool = True, k_min: int = 1,
-                                    chosen: Optional[torch.Tensor] = None, stream=None) -> None:
+                                    chosen: Optional[torch.Tensor] = None, rope: Optional[Sequence[int]] = None,
+                                    stream=None) -> None:
     n_pairs = len(n_seg)
     a_nseg = (C.c_int32 * n_pairs)(*n_seg)
     a_slen = (C.c_int32 * n_pairs)(*seg_len)
+    a_rope = (C.c_int32 * n_pairs)(*rope) if rope is not None else None
     assert kept.dtype == torch.int32 and kept.numel() >= sum(a * b for a, b in zip(n_seg, seg_len))
     assert k_out.dtype == torch.int32 and k_out.numel() >= sum(n_seg)
     fn = lib().ecospa_select_aligned_threshold
     fn.restype = C.c_int
-    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_int32, C.c_void_p,
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_int32, C.c_void_p,
                    C.c_void_p, C.c_void_p, C.c_void_p]
-    st = fn(_ptr(upsilon), C.addressof(a_nseg), C.addressof(a_slen), n_pairs, float(theta), int(bool(l1)), int(k_min),
-            _ptr(chosen), _ptr(kept), _ptr(k_out), _stream(stream))
+    st = fn(_ptr(upsilon), C.addressof(a_nseg), C.addressof(a_slen), C.addressof(a_rope) if a_rope is not None else None,
+            n_pairs, float(theta), int(bool(l1)), int(k_min), _ptr(chosen), _ptr(kept), _ptr(k_out), _stream(stream))
     if st != 0:
         raise EcospaError(st, "ecospa_select_aligned_threshold")
 

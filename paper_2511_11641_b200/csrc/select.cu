@@ -221,12 +221,15 @@ __global__ void __launch_bounds__(kThreads) threshold_count_kernel(const __grid_
         if (P.pairs[mid].seg_start <= seg) lo_p = mid; else hi_p = mid - 1;
     }
     const SelPair& Q = P.pairs[lo_p];
-    const int n = Q.seg_len;
-    const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg - Q.seg_start) * n;
+    // with rotation pairs the units are the seg_len/2 pairs, each counted once (its score sits at its first member)
+    const int unit = Q.rope ? 2 : 1;
+    const int n = Q.seg_len / unit;
+    const int stride = Q.rope == ECOSPA_ROPE_INTERLEAVED ? 2 : 1;
+    const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg - Q.seg_start) * Q.seg_len;
     const int tid = threadIdx.x;
     const int gseg = P.seg_base + seg;
     if (P.chosen && P.chosen[gseg] == 0) {
-        if (tid == 0) P.k_out[gseg] = n;
+        if (tid == 0) P.k_out[gseg] = Q.seg_len;
         return;
     }
     // sum of the scores whose key is at least t, and how many there are
@@ -234,7 +237,7 @@ __global__ void __launch_bounds__(kThreads) threshold_count_kernel(const __grid_
         double s = 0.0;
         int c = 0;
         for (int j = tid; j < n; j += kThreads) {
-            const float f = __ldg(sc + j);
+            const float f = __ldg(sc + j * stride);
             if (static_cast<uint64_t>(order_key(f)) >= t) {
                 s += static_cast<double>(f);
                 ++c;
@@ -258,7 +261,7 @@ __global__ void __launch_bounds__(kThreads) threshold_count_kernel(const __grid_
         uint32_t below = 0;
         bool any = false;
         for (int j = tid; j < n; j += kThreads) {
-            const uint32_t key = order_key(__ldg(sc + j));
+            const uint32_t key = order_key(__ldg(sc + j * stride));
             if (static_cast<uint64_t>(key) < hi) {
                 below = any ? max(below, key) : key;
                 any = true;
@@ -287,7 +290,7 @@ __global__ void __launch_bounds__(kThreads) threshold_count_kernel(const __grid_
             double val = 0.0;
             int c = 0;
             for (int j = tid; j < n; j += kThreads) {
-                const float f = __ldg(sc + j);
+                const float f = __ldg(sc + j * stride);
                 if (order_key(f) == tkey) {
                     val = static_cast<double>(f);
                     ++c;
@@ -312,8 +315,8 @@ __global__ void __launch_bounds__(kThreads) threshold_count_kernel(const __grid_
         }
         k = cnt + e;
     }
-    k = max(k, min(P.k_min, n));
-    if (tid == 0) P.k_out[gseg] = k;
+    k = max(k, min((P.k_min + unit - 1) / unit, n));
+    if (tid == 0) P.k_out[gseg] = k * unit;
 }
 
 // chosen[i] = 1 for the m smallest values (equal values: lower index first): rank by counting.
@@ -415,8 +418,8 @@ extern "C" ecospa_status_t ecospa_select_rotation_pairs(const float* upsilon, co
 }
 
 extern "C" ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon, const int32_t* n_seg,
-                                                           const int32_t* seg_len, int32_t n_pairs, double theta,
-                                                           int32_t l1, int32_t k_min, const int32_t* chosen,
+                                                           const int32_t* seg_len, const int32_t* rope, int32_t n_pairs,
+                                                           double theta, int32_t l1, int32_t k_min, const int32_t* chosen,
                                                            int32_t* kept, int32_t* k_out, void* stream_) {
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     if (!upsilon || !n_seg || !seg_len || n_pairs < 1 || !kept || !k_out) return ECOSPA_ERR_INVALID;
@@ -425,6 +428,9 @@ extern "C" ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon,
     for (int p = 0; p < n_pairs; ++p) {
         if (n_seg[p] < 1 || seg_len[p] < 1) return ECOSPA_ERR_INVALID;
         if (seg_len[p] > (1 << 20)) return ECOSPA_ERR_UNSUPPORTED;
+        const int32_t rp = rope ? rope[p] : ECOSPA_ROPE_NONE;
+        if (rp != ECOSPA_ROPE_NONE && rp != ECOSPA_ROPE_INTERLEAVED && rp != ECOSPA_ROPE_HALF) return ECOSPA_ERR_INVALID;
+        if (rp != ECOSPA_ROPE_NONE && (seg_len[p] & 1)) return ECOSPA_ERR_INVALID;
         total_d += static_cast<int64_t>(n_seg[p]) * seg_len[p];
     }
     if (total_d > INT32_MAX) return ECOSPA_ERR_UNSUPPORTED;
@@ -442,7 +448,7 @@ extern "C" ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon,
             Q.seg_start = ns - s_in_p;
             Q.seg_len = seg_len[p];
             Q.d_off = d_off;
-            Q.rope = ECOSPA_ROPE_NONE;
+            Q.rope = rope ? rope[p] : ECOSPA_ROPE_NONE;
             tp.pairs[np] = Q;
             ++np;
             ns += take;

@@ -113,12 +113,17 @@ def test_compact_rejects_bad_arguments_without_launching(lib):
 def test_threshold_selection_rejects_bad_arguments_without_launching(lib):
     fn = lib.ecospa_select_aligned_threshold
     fn.restype = C.c_int
-    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_int32, C.c_void_p,
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_int32, C.c_void_p,
                    C.c_void_p, C.c_void_p, C.c_void_p]
     ups, kept, kout = C.c_void_p(0x1000), C.c_void_p(0x2000), C.c_void_p(0x3000)
     one = (C.c_int32 * 1)(1)
     slen = (C.c_int32 * 1)(64)
-    a = (C.addressof(one), C.addressof(slen), 1)
+    a = (C.addressof(one), C.addressof(slen), None, 1)
+    odd = (C.c_int32 * 1)(63)
+    mode = (C.c_int32 * 1)(2)
+    assert fn(ups, C.addressof(one), C.addressof(odd), C.addressof(mode), 1, 0.9, 1, 1, None, kept, kout, None) == 1
+    bad = (C.c_int32 * 1)(5)
+    assert fn(ups, C.addressof(one), C.addressof(slen), C.addressof(bad), 1, 0.9, 1, 1, None, kept, kout, None) == 1
     assert fn(None, *a, 0.9, 1, 1, None, kept, kout, None) == 1
     assert fn(ups, *a, 0.9, 1, 1, None, None, kout, None) == 1
     assert fn(ups, *a, 0.9, 1, 1, None, kept, None, None) == 1
@@ -126,7 +131,7 @@ def test_threshold_selection_rejects_bad_arguments_without_launching(lib):
     assert fn(ups, *a, float("nan"), 1, 1, None, kept, kout, None) == 1
     assert fn(ups, *a, 0.9, 1, -1, None, kept, kout, None) == 1
     big = (C.c_int32 * 1)((1 << 20) + 1)
-    assert fn(ups, C.addressof(one), C.addressof(big), 1, 0.9, 1, 1, None, kept, kout, None) == 3
+    assert fn(ups, C.addressof(one), C.addressof(big), None, 1, 0.9, 1, 1, None, kept, kout, None) == 3
     ch = lib.ecospa_choose_pairs
     ch.restype = C.c_int
     ch.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]

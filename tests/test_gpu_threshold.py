@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def run_case(ups_np, n_seg, seg_len, theta, l1, k_min, chosen_np=None):
+def run_case(ups_np, n_seg, seg_len, theta, l1, k_min, chosen_np=None, rope=None):
     """ups_np: concatenated scores; n_seg / seg_len: per pair.  Returns nothing; asserts parity."""
     ups = torch.from_numpy(ups_np).to(DEV)
     total_segs = sum(n_seg)
@@ -26,24 +26,29 @@ def run_case(ups_np, n_seg, seg_len, theta, l1, k_min, chosen_np=None):
     kept = torch.full((D,), -7, dtype=torch.int32, device=DEV)
     k_out = torch.full((total_segs,), -1, dtype=torch.int32, device=DEV)
     chosen = torch.from_numpy(chosen_np).to(DEV) if chosen_np is not None else None
-    B.ecospa_select_aligned_threshold(ups, n_seg, seg_len, theta, kept, k_out, l1=l1, k_min=k_min, chosen=chosen)
+    B.ecospa_select_aligned_threshold(ups, n_seg, seg_len, theta, kept, k_out, l1=l1, k_min=k_min, chosen=chosen, rope=rope)
     torch.cuda.synchronize()
     k_gpu = k_out.cpu().numpy()
     kept_gpu = kept.cpu().numpy()
     off, seg = 0, 0
-    for ns, sl in zip(n_seg, seg_len):
+    for pi, (ns, sl) in enumerate(zip(n_seg, seg_len)):
         u = ups_np[off:off + ns * sl]
         ch = chosen_np[seg:seg + ns] if chosen_np is not None else None
-        k_ref = O.threshold_counts(u, ns, sl, theta, l1=l1, k_min=k_min, chosen=ch)
+        rp = rope[pi] if rope is not None else 0
+        k_ref = O.threshold_counts(u, ns, sl, theta, l1=l1, k_min=k_min, chosen=ch, rope=rp)
         for s in range(ns):
             kg, kr = int(k_gpu[seg + s]), int(k_ref[s])
             if kg != kr:
+                assert rp == 0, (seg + s, kg, kr)
                 v = np.sort(u[s * sl:(s + 1) * sl].astype(np.float64))[::-1]
                 total = v.sum() if l1 else 1.0
                 gap = min(abs(v[:kk].sum() - theta * total) for kk in (kg, kr))
                 assert abs(kg - kr) == 1 and gap <= 1e-9 * max(total, 1e-300), (seg + s, kg, kr, gap)
             # the kept indices are the top-k of the segment, ascending, relative to the pair group
-            want = O.select_topk(u[s * sl:(s + 1) * sl], 1, sl, [kg]) + s * sl
+            if rp:
+                want = O.select_rotation_pairs(u[s * sl:(s + 1) * sl], 1, sl, [kg], rp) + s * sl
+            else:
+                want = O.select_topk(u[s * sl:(s + 1) * sl], 1, sl, [kg]) + s * sl
             got = kept_gpu[off + s * sl: off + s * sl + kg]
             assert np.array_equal(got, want), (seg + s, kg)
             assert (kept_gpu[off + s * sl + kg: off + (s + 1) * sl] == -7).all()     # rest of the slot untouched
@@ -94,3 +99,18 @@ def test_choose_pairs_matches_oracle():
             ch = torch.full((n,), -1, dtype=torch.int32, device=DEV)
             B.ecospa_choose_pairs(fd, m, ch)
             assert np.array_equal(ch.cpu().numpy(), O.choose_pairs(f, m))
+
+
+@pytest.mark.parametrize("mode", [B.ROPE_INTERLEAVED, B.ROPE_HALF])
+def test_threshold_on_rotation_pairs(mode):
+    """Q/K group scored with rotation pairs, V/O group plain, in one call."""
+    wl = WL.WORKLOADS["llama1b"]
+    w = WL.layer_weights(wl, 0, device=DEV)
+    h, d_h = wl.n_heads, wl.d_h
+    pairs = [B.pair(B.PAIR_PLAIN, h, d_h, w["wq"], w["wk"], B.SHARED_COLS, B.SHARED_COLS, rope=mode),
+             B.pair(B.PAIR_PLAIN, h, d_h, w["wv"], w["wo"], B.SHARED_COLS, B.SHARED_ROWS)]
+    ups = torch.empty(2 * h * d_h, dtype=torch.float32, device=DEV)
+    B.ecospa_score_pairs(pairs, float(wl.tokens), ups, None, None)
+    u = ups.cpu().numpy()
+    for theta, k_min in ((0.9, 1), (0.6, 5), (1e-6, 3)):
+        run_case(u, [h, h], [d_h, d_h], theta, True, k_min, rope=[mode, B.ROPE_NONE])

@@ -107,3 +107,16 @@ def test_choose_pairs_against_a_stable_library_sort():
     g = np.array([3, 1, 1, 2], dtype=np.float32)
     assert O.choose_pairs(g, 1).tolist() == [0, 1, 0, 0]
     assert O.choose_pairs(g, 2).tolist() == [0, 1, 1, 0]
+
+
+def test_rotation_pairs_are_thresholded_as_units():
+    r = np.random.default_rng(17)
+    half = 24
+    unit = r.random(half).astype(np.float32)
+    inter = np.repeat(unit, 2)                       # members (2u, 2u+1) carry the pair's score
+    halves = np.concatenate([unit, unit])            # members (u, u + half)
+    for theta in (0.3, 0.8, 0.95):
+        k_units = int(O.threshold_counts(unit, 1, half, theta, l1=True, k_min=1)[0])
+        assert O.threshold_counts(inter, 1, 2 * half, theta, l1=True, k_min=1, rope=1)[0] == 2 * k_units
+        assert O.threshold_counts(halves, 1, 2 * half, theta, l1=True, k_min=2, rope=2)[0] == 2 * k_units
+    assert O.threshold_counts(inter, 1, 2 * half, 1e-9, l1=True, k_min=3, rope=1)[0] == 4      # k_min in whole pairs
