@@ -48,13 +48,16 @@ def step_flops(wl, n_attn: int, k_ffn: int) -> float:
     return 3.0 * fwd * wl.n_layers
 
 
-def sparsify_bytes(wl, rho: float, with_grads: bool = True) -> float:
+def sparsify_bytes(wl, rho: float, with_grads: bool = True, transposed: bool = False) -> float:
     """Weights (and gradients) read once for the scores; compaction reads a shared-cols tensor in
-    full and a shared-rows tensor at the kept fraction, and writes the kept fraction of both."""
+    full and a shared-rows tensor at the kept fraction, and writes the kept fraction of both.
+    transposed: every matrix is stored the other way round, which swaps the two kinds."""
     D = wl.n_heads * wl.d_h
     e = wl.elem_bytes
     cols = (3 * wl.d_m * D + (2 if wl.ffn == "swiglu" else 1) * wl.d_m * wl.d_ffn) * e * wl.n_layers
     rows = (wl.d_m * D + wl.d_m * wl.d_ffn) * e * wl.n_layers
+    if transposed:
+        cols, rows = rows, cols
     mult = 2 if with_grads else 1
     score = (cols + rows) * mult
     compact = (cols * (1 + rho) + rows * 2 * rho) * mult
@@ -127,17 +130,25 @@ class ClockSampler:
 class Model:
     """Device-resident synthetic model plus every buffer a step writes (allocated once)."""
 
-    def __init__(self, wl, sparsity: float, device, n_act_sets: int = 4):
+    def __init__(self, wl, sparsity: float, device, n_act_sets: int = 4, transposed: bool = False):
         import torch
         from paper_2511_11641_b200 import binding as B, block as BL, workloads as WL
         self.wl, self.dev, self.B, self.BL = wl, device, B, BL
         self.torch = torch
         self.w, self.g, self.pairs = [], [], []
+        # transposed: every weight matrix (and its gradient) stored the other way round, i.e. W_Q, W_K, W_V, W_1
+        # as D x d_m (what a framework's linear layer keeps) and W_O, W_2 as d_m x D
+        self.transposed = transposed
+        lin, lout = (B.SHARED_ROWS, B.SHARED_COLS) if transposed else (B.SHARED_COLS, B.SHARED_ROWS)
+        self.lay = dict(w_in_layout=lin, w_out_layout=lout)
         for l in range(wl.n_layers):
             w = WL.layer_weights(wl, l, device=device)
             g = WL.layer_grads(wl, l, device=device)
+            if transposed:
+                w = {k_: (v.t().contiguous() if v.dim() == 2 else v) for k_, v in w.items()}
+                g = {k_: (v.t().contiguous() if v.dim() == 2 else v) for k_, v in g.items()}
             self.w.append(w); self.g.append(g)
-            self.pairs += BL.block_pairs(w, wl.n_heads, wl.d_h, wl.d_ffn, g)
+            self.pairs += BL.block_pairs(w, wl.n_heads, wl.d_h, wl.d_ffn, g, layout_in=lin, layout_out=lout)
         plan = WL.kept_plan(wl, sparsity)
         self.n_attn, self.k_ffn = sum(plan["qk"]), plan["ffn"][0]
         self.k_per_seg = (plan["qk"] + plan["vo"] + plan["ffn"]) * wl.n_layers
@@ -156,8 +167,8 @@ class Model:
         groups = [(["wq", "wk", "bq", "bk"], ["gq", "gk"], self.n_attn, D_attn),
                   (["wv", "wo", "bv"], ["gv", "go"], self.n_attn, D_attn),
                   (["w1", "w1b", "w2", "b1"], ["g1", "g1b", "g2"], self.k_ffn, wl.d_ffn)]
-        layout = {"wq": 0, "wk": 0, "wv": 0, "wo": 1, "w1": 0, "w1b": 0, "w2": 1, "bq": 0, "bk": 0, "bv": 0, "b1": 0,
-                  "gq": 0, "gk": 0, "gv": 0, "go": 1, "g1": 0, "g1b": 0, "g2": 1}
+        layout = {"wq": lin, "wk": lin, "wv": lin, "wo": lout, "w1": lin, "w1b": lin, "w2": lout, "bq": 0, "bk": 0, "bv": 0,
+                  "b1": 0, "gq": lin, "gk": lin, "gv": lin, "go": lout, "g1": lin, "g1b": lin, "g2": lout}
         for l in range(wl.n_layers):
             c = {}
             for wn, gn, nk, D in groups:
@@ -181,13 +192,14 @@ class Model:
                                             widths={"dq": npad, "dk": npad, "dv": npad, "ctx": npad}, device=device))
         e = lambda *shape: torch.empty(shape, dtype=dt, device=device)
         self.o = {"Q": e(T, npad), "K": e(T, npad), "V": e(T, npad), "Out": e(T, d), "dX": e(T, d), "dCtx": e(T, npad),
-                  "dWq": e(d, npad), "dWk": e(d, npad), "dWv": e(d, npad), "dWo": e(n, d),
+                  "dWq": e(n, d) if transposed else e(d, npad), "dWk": e(n, d) if transposed else e(d, npad),
+                  "dWv": e(n, d) if transposed else e(d, npad), "dWo": e(d, npad) if transposed else e(n, d),
                   "dbq": e(n), "dbk": e(n), "dbv": e(n), "dbo": e(d)}
         self.o["dX"].zero_()
         from paper_2511_11641_b200 import layers as L
         self.L = L
         self.act = B.ACT_SWIGLU if wl.ffn == "swiglu" else B.ACT_GELU_ERF
-        self.ffn = L.ffn_buffers(T, d, k, self.act, dt, device)
+        self.ffn = L.ffn_buffers(T, d, k, self.act, dt, device, transposed=transposed)
         self.proj_ws = torch.empty(B.ecospa_proj_workspace_bytes(T, d, n, B.BF16 if dt == torch.bfloat16 else B.F32) + 16,
                                    dtype=torch.uint8, device=device)
 
@@ -204,17 +216,17 @@ class Model:
             c, a = self.c[l], self.acts[l % len(self.acts)]
             # forward: Q, K, V in one launch; (attention core is the caller's); output projection; FFN
             B.ecospa_coupled_qkv_fwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, o["Q"], o["K"], o["V"], bq_c=c.get("bq"),
-                                     bk_c=c.get("bk"), bv_c=c.get("bv"), workspace=self.proj_ws)
-            B.ecospa_coupled_vo_fwd_o(a["ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws)
+                                     bk_c=c.get("bk"), bv_c=c.get("bv"), workspace=self.proj_ws, **self.lay)
+            B.ecospa_coupled_vo_fwd_o(a["ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws, **self.lay)
             # FFN forward + backward
             self.L.ffn_fwd_bwd(a["x"], a["dy"], self.act, c["w1"], c["w2"], k, self.ffn, w1bc=c.get("w1b"),
-                               b1c=c.get("b1"), b2=self.w[l].get("b2"))
+                               b1c=c.get("b1"), b2=self.w[l].get("b2"), **self.lay)
             # backward: what dOut gives (dCtx, dW_O), then what dQ, dK, dV give (dW_Q, dW_K, dW_V, dX)
             B.ecospa_coupled_vo_bwd_o(a["ctx"], c["wo"], n, a["dout"], o["dCtx"], o["dWo"], o["dbo"] if bias else None,
-                                      workspace=self.proj_ws)
+                                      workspace=self.proj_ws, **self.lay)
             B.ecospa_coupled_qkv_bwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, a["dq"], a["dk"], a["dv"], o["dX"], o["dWq"],
                                      o["dWk"], o["dWv"], o["dbq"] if bias else None, o["dbk"] if bias else None,
-                                     o["dbv"] if bias else None, accumulate_dX=True, workspace=self.proj_ws)
+                                     o["dbv"] if bias else None, accumulate_dX=True, workspace=self.proj_ws, **self.lay)
 
     def host_copies(self):
         """Pinned host mirrors of every input of a step (weights, gradients, activations)."""
@@ -263,7 +275,7 @@ def run_gpu(args):
     if args.layers:
         import dataclasses
         wl = dataclasses.replace(wl, n_layers=args.layers)   # smaller model of the same shape (profiler captures)
-    m = Model(wl, args.sparsity, dev)
+    m = Model(wl, args.sparsity, dev, transposed=args.transposed)
     ev = lambda: torch.cuda.Event(enable_timing=True)
 
     def barrier():
@@ -318,7 +330,7 @@ def run_gpu(args):
     # step s computes; every step still pays its own upload and read-back inside the timed region.
     host = m.host_copies()
     h2d = sum(h.numel() * h.element_size() for h, _ in host)
-    m2 = Model(wl, args.sparsity, dev)
+    m2 = Model(wl, args.sparsity, dev, transposed=args.transposed)
     for _ in range(3):
         m2.sparsify(); m2.layers()
     if args.no_graph:
@@ -372,7 +384,7 @@ def run_gpu(args):
     ms_step, ms_sp, ms_gemm, ms_e2e = max_over_ranks([ms_step, ms_sp, ms_gemm, ms_e2e], dev)
 
     flops = step_flops(wl, m.n_attn, m.k_ffn)
-    sbytes = sparsify_bytes(wl, 1.0 - args.sparsity)
+    sbytes = sparsify_bytes(wl, 1.0 - args.sparsity, transposed=args.transposed)
     peaks = measured_peaks()
     n_gemm_launches = wl.n_layers * 8
     out = {
@@ -380,7 +392,8 @@ def run_gpu(args):
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic (seeded N(0,sigma) tensors)",
         "config": {"workload": f"{wl.name}: {wl.n_layers} layers d_model={wl.d_m} heads={wl.n_heads}x{wl.d_h} "
-                               f"ffn={wl.d_ffn} {wl.ffn} T={wl.tokens} sparsity={args.sparsity}",
+                               f"ffn={wl.d_ffn} {wl.ffn} T={wl.tokens} sparsity={args.sparsity}"
+                               + (" weights stored transposed" if args.transposed else ""),
                    "l2": "inputs larger than L2: 1.7 GB of weights/gradients per step, activations cycled over 4 sets",
                    "replicas": world, "launch": "eager" if args.no_graph else "cuda graph replay of the captured step"},
         "phases": {
@@ -393,7 +406,7 @@ def run_gpu(args):
         "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": flops / ms_gemm / 1e9,
                      "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": flops / ms_gemm / 1e9 / peaks["bf16_tflops_sustained"],
-                     "traffic": NCU_GEMM_TRAFFIC_BYTES.get(wl.name) if (not args.layers and args.sparsity == 0.5) else None,
+                     "traffic": NCU_GEMM_TRAFFIC_BYTES.get(wl.name) if (not args.layers and args.sparsity == 0.5 and not args.transposed) else None,
                      "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
                      "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                      "launches_per_step": n_gemm_launches, "avg_launch_ms": ms_gemm / n_gemm_launches},
@@ -504,6 +517,8 @@ def main():
     ap.add_argument("--sparsity", type=float, default=0.5)
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small cases for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--transposed", action="store_true",
+                    help="store every weight matrix the other way round (W_Q.. as D x d_m, W_O, W_2 as d_m x D)")
     ap.add_argument("--no-graph", action="store_true", help="issue every launch from the host instead of replaying a CUDA graph")
     args = ap.parse_args()
     if args.impl == "reference":

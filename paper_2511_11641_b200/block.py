@@ -15,21 +15,24 @@ GROUPS = ("qk", "vo", "ffn")
 
 
 def block_pairs(w: Dict[str, torch.Tensor], n_heads: int, d_h: int, d_ffn: int,
-                g: Optional[Dict[str, torch.Tensor]] = None) -> List[B.Pair]:
+                g: Optional[Dict[str, torch.Tensor]] = None, layout_in: int = B.SHARED_COLS,
+                layout_out: int = B.SHARED_ROWS) -> List[B.Pair]:
     """[QK, VO, FFN] pair groups of one block.
 
     QK: column j of head i of W^Q with column j of head i of W^K (W_1 = W_i^Q, W_2 = W_i^K^T).
     VO: column j of head i of W^V with row j of row-block i of W^O.
     FFN: column j of W_in (or of W_gate (.) W_up) with row j of W_out (W_down).
+    layout_in: storage of W^Q, W^K, W^V, W_in / W_gate / W_up (default: as the equations write them, d_m x D);
+    layout_out: storage of W^O, W_out / W_down (default D x d_m).
     """
     g = g or {}
     swiglu = "w1b" in w
     return [
-        B.pair(B.PAIR_PLAIN, n_heads, d_h, w["wq"], w["wk"], B.SHARED_COLS, B.SHARED_COLS,
+        B.pair(B.PAIR_PLAIN, n_heads, d_h, w["wq"], w["wk"], layout_in, layout_in,
                g1=g.get("gq"), g2=g.get("gk")),
-        B.pair(B.PAIR_PLAIN, n_heads, d_h, w["wv"], w["wo"], B.SHARED_COLS, B.SHARED_ROWS,
+        B.pair(B.PAIR_PLAIN, n_heads, d_h, w["wv"], w["wo"], layout_in, layout_out,
                g1=g.get("gv"), g2=g.get("go")),
-        B.pair(B.PAIR_SWIGLU if swiglu else B.PAIR_PLAIN, 1, d_ffn, w["w1"], w["w2"], B.SHARED_COLS, B.SHARED_ROWS,
+        B.pair(B.PAIR_SWIGLU if swiglu else B.PAIR_PLAIN, 1, d_ffn, w["w1"], w["w2"], layout_in, layout_out,
                w1b=w.get("w1b"), g1=g.get("g1"), g2=g.get("g2"), g1b=g.get("g1b")),
     ]
 

@@ -9,8 +9,9 @@ from . import binding as B
 from .block import pad8
 
 
-def ffn_buffers(T: int, d_m: int, k: int, act: int, dtype: torch.dtype, device) -> Dict[str, torch.Tensor]:
-    """Outputs and saved tensors of one FFN forward+backward (H, Hb, A are always bf16)."""
+def ffn_buffers(T: int, d_m: int, k: int, act: int, dtype: torch.dtype, device, transposed: bool = False) -> Dict[str, torch.Tensor]:
+    """Outputs and saved tensors of one FFN forward+backward (H, Hb, A are always bf16).  transposed: weights are
+    stored the other way round (W_1 as k x d_m, W_2 as d_m x k), and so are their gradients."""
     kp = pad8(k, 2)
     kpw = pad8(k, 2 if dtype == torch.bfloat16 else 4)
     sw = act == B.ACT_SWIGLU
@@ -19,13 +20,13 @@ def ffn_buffers(T: int, d_m: int, k: int, act: int, dtype: torch.dtype, device) 
         "H": torch.empty((T, kp), dtype=torch.bfloat16, device=device),
         "A": torch.empty((T, kp), dtype=torch.bfloat16, device=device),
         "dX": torch.empty((T, d_m), dtype=dtype, device=device),
-        "dW1": torch.zeros((d_m, kpw), dtype=dtype, device=device),
-        "dW2": torch.empty((k, d_m), dtype=dtype, device=device),
+        "dW1": torch.zeros((k, d_m) if transposed else (d_m, kpw), dtype=dtype, device=device),
+        "dW2": torch.zeros((d_m, kpw) if transposed else (k, d_m), dtype=dtype, device=device),
         "db2": torch.empty((d_m,), dtype=dtype, device=device),
     }
     if sw:
         d["Hb"] = torch.empty((T, kp), dtype=torch.bfloat16, device=device)
-        d["dW1b"] = torch.zeros((d_m, kpw), dtype=dtype, device=device)
+        d["dW1b"] = torch.zeros((k, d_m) if transposed else (d_m, kpw), dtype=dtype, device=device)
     else:
         d["db1"] = torch.empty((k,), dtype=dtype, device=device)
     code = B.F32 if dtype == torch.float32 else B.BF16
@@ -33,12 +34,13 @@ def ffn_buffers(T: int, d_m: int, k: int, act: int, dtype: torch.dtype, device) 
     return d
 
 
-def ffn_fwd_bwd(X, dY, act: int, w1c, w2c, k: int, buf: Dict[str, torch.Tensor], w1bc=None, b1c=None, b2=None) -> None:
+def ffn_fwd_bwd(X, dY, act: int, w1c, w2c, k: int, buf: Dict[str, torch.Tensor], w1bc=None, b1c=None, b2=None,
+                **layouts) -> None:
     B.ecospa_coupled_ffn_fwd(X, act, w1c, w2c, k, buf["Y"], buf["H"], buf["A"], w1b_c=w1bc, Hb=buf.get("Hb"),
-                             b1_c=b1c, b2=b2, workspace=buf["ws"])
+                             b1_c=b1c, b2=b2, workspace=buf["ws"], **layouts)
     B.ecospa_coupled_ffn_bwd(X, act, w1c, w2c, k, buf["H"], buf["A"], dY, buf["dX"], buf["dW1"], buf["dW2"],
                              w1b_c=w1bc, Hb=buf.get("Hb"), dW1b_c=buf.get("dW1b"), db1_c=buf.get("db1"),
-                             db2=buf["db2"], workspace=buf["ws"])
+                             db2=buf["db2"], workspace=buf["ws"], **layouts)
 
 
 def smoke_layer_check(wl, w1c, w1bc, w2c, k: int, dev) -> None:
