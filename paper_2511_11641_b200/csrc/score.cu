@@ -313,7 +313,7 @@ struct StatPlan {        // one per-index statistic of one pair
 
 int chunks_for(const ecospa_mat_t& m) {
     if (m.layout != ECOSPA_SHARED_COLS) return 1;
-    return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(8, m.other_dim / 64)));
+    return static_cast<int>(std::max<int64_t>(1, std::min<int64_t>(4, m.other_dim / 64)));
 }
 
 ecospa_status_t validate_mat(const ecospa_mat_t& m, int64_t D, int want_dtype, int want_layout, int64_t want_other) {

@@ -66,7 +66,7 @@ def test_static_scratch_scores_match_regular_call_twice_in_a_row(name):
 def test_static_scratch_rejects_oversized_pairs():
     limit = B.ecospa_score_pair_static_max_bytes()
     assert 0 < limit <= 16 << 20
-    D, other = 160 * 1024, 512          # 9 stat/partial vectors of 160 Ki floats need more than 4 MiB
+    D, other = 320 * 1024, 512          # the stat/partial vectors of 320 Ki floats need more than 4 MiB
     w1 = torch.zeros((other, D), dtype=torch.bfloat16, device=DEV)
     w2 = torch.zeros((D, 8), dtype=torch.bfloat16, device=DEV)
     p = B.pair(B.PAIR_PLAIN, 1, D, w1, w2, B.SHARED_COLS, B.SHARED_ROWS)
