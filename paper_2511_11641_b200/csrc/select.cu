@@ -46,6 +46,8 @@ __device__ __forceinline__ uint32_t order_key(float f) {
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// ROPE = false: no pair group of the launch has rotation pairs (the common case, compiled without the unit logic).
+template <bool ROPE>
 __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant__ SelectParams P) {
     __shared__ int hist[256];
     __shared__ int warp_tot[kWarps];
@@ -63,7 +65,7 @@ __global__ void __launch_bounds__(kThreads) select_kernel(const __grid_constant_
     const int seg_in_pair = seg - Q.seg_start;
     // With rotation pairs the ranked units are the seg_len/2 pairs; both members carry the pair's score, so
     // unit u is read at index 2u (interleaved pairs) or u (pairs of the two halves).
-    const int rope = Q.rope;
+    const int rope = ROPE ? Q.rope : ECOSPA_ROPE_NONE;
     const int n = rope ? seg_len >> 1 : seg_len;
     const int stride = rope == ECOSPA_ROPE_INTERLEAVED ? 2 : 1;
     const float* sc = P.upsilon + Q.d_off + static_cast<int64_t>(seg_in_pair) * seg_len;
@@ -395,7 +397,10 @@ static ecospa_status_t select_fixed_counts(const float* upsilon, const int32_t* 
         sp.n_pairs = np;
         sp.n_segs = ns;
         sp.is_last = (p >= n_pairs) ? 1 : 0;
-        select_kernel<<<ns, kThreads, 0, stream>>>(sp);
+        bool any_rope = false;
+        for (int i = 0; i < np; ++i) any_rope = any_rope || sp.pairs[i].rope != ECOSPA_ROPE_NONE;
+        if (any_rope) select_kernel<true><<<ns, kThreads, 0, stream>>>(sp);
+        else select_kernel<false><<<ns, kThreads, 0, stream>>>(sp);
         ecospa_status_t st = check_launch("select_kernel");
         if (st != ECOSPA_OK) return st;
     }
@@ -470,7 +475,10 @@ extern "C" ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon,
         sp.upsilon = upsilon; sp.kept = kept; sp.seg_offsets = nullptr;
         sp.n_pairs = np; sp.n_segs = ns; sp.seg_base = seg_base; sp.is_last = 0;
         sp.k_dev = k_out;
-        select_kernel<<<ns, kThreads, 0, stream>>>(sp);
+        bool any_rope = false;
+        for (int i = 0; i < np; ++i) any_rope = any_rope || sp.pairs[i].rope != ECOSPA_ROPE_NONE;
+        if (any_rope) select_kernel<true><<<ns, kThreads, 0, stream>>>(sp);
+        else select_kernel<false><<<ns, kThreads, 0, stream>>>(sp);
         if ((st = check_launch("select_kernel")) != ECOSPA_OK) return st;
     }
     return ECOSPA_OK;
