@@ -218,6 +218,14 @@ ecospa_status_t ecospa_select_aligned_threshold(const float* upsilon, const int3
                                                 int32_t k_min, const int32_t* chosen, int32_t* kept, int32_t* k_out,
                                                 void* stream);
 
+/* Turns the slots that ecospa_select_aligned_threshold wrote into the kept list of a whole tensor (the input of
+ * step 3): out[dst[s] + i] = slots[src[s] + i] + add[s] for i < k[s], segment by segment.  src, dst, k, add: HOST
+ * [n_segs] (k as read back from k_out; add = what turns a slot's indices into shared indices of the tensor being
+ * compacted, e.g. the column offset of a head that was scored as a group of its own).  slots, out: DEVICE.
+ * Index bookkeeping only; no counterpart in the paper beyond "remove the i-th row/column" of Algorithm 1. */
+ecospa_status_t ecospa_pack_kept(const int32_t* slots, const int32_t* src, const int32_t* dst, const int32_t* k,
+                                 const int32_t* add, int32_t n_segs, int32_t* out, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Step 3: physical removal.   Definition 1: drop column j of W_1 and row j of W_2 for every removed j
  * "keeping the original pairings"; Alg. 1 also drops the same rows/columns of the optimizer moments.

@@ -190,6 +190,21 @@ def ecospa_select_rotation_pairs(upsilon: torch.Tensor, n_seg: Sequence[int], se
         raise EcospaError(st, "ecospa_select_rotation_pairs")
 
 
+def ecospa_pack_kept(slots: torch.Tensor, src: Sequence[int], dst: Sequence[int], k: Sequence[int], add: Sequence[int],
+                     out: torch.Tensor, stream=None) -> None:
+    n = len(src)
+    assert len(dst) == n and len(k) == n and len(add) == n and slots.dtype == torch.int32 and out.dtype == torch.int32
+    arr = lambda v: (C.c_int32 * n)(*v)
+    a_src, a_dst, a_k, a_add = arr(src), arr(dst), arr(k), arr(add)
+    fn = lib().ecospa_pack_kept
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    st = fn(_ptr(slots), C.addressof(a_src), C.addressof(a_dst), C.addressof(a_k), C.addressof(a_add), n, _ptr(out),
+            _stream(stream))
+    if st != 0:
+        raise EcospaError(st, "ecospa_pack_kept")
+
+
 def ecospa_choose_pairs(fisher: torch.Tensor, m: int, chosen: torch.Tensor, stream=None) -> None:
     assert fisher.dtype == torch.float32 and chosen.dtype == torch.int32 and chosen.numel() >= fisher.numel()
     fn = lib().ecospa_choose_pairs

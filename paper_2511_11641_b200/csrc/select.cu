@@ -335,11 +335,44 @@ __global__ void __launch_bounds__(1024) choose_pairs_kernel(const float* __restr
     }
 }
 
+// Packs the per-segment slots of the variable-count selection into one ascending list per pair group:
+// out[dst[s] + i] = slots[src[s] + i] + add[s] for i < k[s].
+constexpr int kPackSegs = 512;
+struct PackParams {
+    const int32_t* slots;
+    int32_t* out;
+    int32_t n;
+    int32_t src[kPackSegs], dst[kPackSegs], k[kPackSegs], add[kPackSegs];
+};
+__global__ void __launch_bounds__(128) pack_kept_kernel(const __grid_constant__ PackParams P) {
+    const int s = blockIdx.x;
+    for (int i = threadIdx.x; i < P.k[s]; i += blockDim.x) P.out[P.dst[s] + i] = P.slots[P.src[s] + i] + P.add[s];
+}
+
 }  // namespace
 
 }  // namespace ecospa
 
 using namespace ecospa;
+
+extern "C" ecospa_status_t ecospa_pack_kept(const int32_t* slots, const int32_t* src, const int32_t* dst, const int32_t* k,
+                                            const int32_t* add, int32_t n_segs, int32_t* out, void* stream) {
+    if (!slots || !src || !dst || !k || !add || !out || n_segs < 1) return ECOSPA_ERR_INVALID;
+    for (int i = 0; i < n_segs; ++i)
+        if (src[i] < 0 || dst[i] < 0 || k[i] < 0) return ECOSPA_ERR_INVALID;
+    static thread_local PackParams pp;
+    for (int base = 0; base < n_segs; base += kPackSegs) {
+        const int n = std::min(kPackSegs, n_segs - base);
+        pp.slots = slots; pp.out = out; pp.n = n;
+        for (int i = 0; i < n; ++i) {
+            pp.src[i] = src[base + i]; pp.dst[i] = dst[base + i]; pp.k[i] = k[base + i]; pp.add[i] = add[base + i];
+        }
+        pack_kept_kernel<<<n, 128, 0, static_cast<cudaStream_t>(stream)>>>(pp);
+        const ecospa_status_t st = check_launch("pack_kept_kernel");
+        if (st != ECOSPA_OK) return st;
+    }
+    return ECOSPA_OK;
+}
 
 static ecospa_status_t select_fixed_counts(const float* upsilon, const int32_t* n_seg, const int32_t* seg_len,
                                            const int32_t* k_per_seg, const int32_t* rope, int32_t n_pairs,

@@ -158,3 +158,17 @@ def test_rotation_pair_selection_rejects_bad_arguments_without_launching(lib):
     assert call(64, 32, 3) == 1          # unknown pairing
     assert call(64, 66, 1) == 1          # more than the segment holds
     assert call(64, 32, 1, rope_null=True) == 1
+
+
+def test_pack_kept_rejects_bad_arguments_without_launching(lib):
+    fn = lib.ecospa_pack_kept
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    slots, out = C.c_void_p(0x1000), C.c_void_p(0x2000)
+    z, neg = (C.c_int32 * 1)(0), (C.c_int32 * 1)(-1)
+    a = C.addressof
+    assert fn(None, a(z), a(z), a(z), a(z), 1, out, None) == 1
+    assert fn(slots, a(z), a(z), a(z), a(z), 1, None, None) == 1
+    assert fn(slots, a(z), a(z), a(z), a(z), 0, out, None) == 1
+    assert fn(slots, a(neg), a(z), a(z), a(z), 1, out, None) == 1
+    assert fn(slots, a(z), a(z), a(neg), a(z), 1, out, None) == 1
