@@ -32,6 +32,7 @@ class Group:
     g2: Optional[torch.Tensor] = None
     g1b: Optional[torch.Tensor] = None
     aux: List[Tuple[torch.Tensor, int]] = field(default_factory=list)   # (tensor, layout): moments, biases (1-D)
+    rope: int = B.ROPE_NONE                                  # Q/K groups under rotary embedding: rotation pairs leave whole
 
     @property
     def D(self) -> int:
@@ -64,9 +65,9 @@ def describe(groups: Sequence[Group]):
     """Pair descriptors of all groups for the scoring call, with where each described pair sits.
 
     A group whose pairs all have the same width is one descriptor (n_seg pairs side by side); a ragged group is
-    one descriptor per pair, built on views of its tensors.  Returns (pairs, n_seg, seg_len, where) with
+    one descriptor per pair, built on views of its tensors.  Returns (pairs, n_seg, seg_len, where, rope) with
     where[i] = (group index, offset of descriptor i inside the group's shared axis)."""
-    pairs, n_seg, seg_len, where = [], [], [], []
+    pairs, n_seg, seg_len, where, rope = [], [], [], [], []
     for gi, g in enumerate(groups):
         kind = B.PAIR_SWIGLU if g.w1b is not None else B.PAIR_PLAIN
         D = g.D
@@ -84,9 +85,9 @@ def describe(groups: Sequence[Group]):
                 continue                                   # a pair that has lost every index takes no part any more
             v = {nm: _slice(t[nm], g.layout1 if nm in ("w1", "w1b", "g1", "g1b") else g.layout2, off, ext) for nm in t}
             pairs.append(B.pair(kind, ns, sl, v["w1"], v["w2"], g.layout1, g.layout2, w1b=v["w1b"],
-                                g1=v["g1"], g2=v["g2"], g1b=v["g1b"]))
-            n_seg.append(ns); seg_len.append(sl); where.append((gi, off))
-    return pairs, n_seg, seg_len, where
+                                g1=v["g1"], g2=v["g2"], g1b=v["g1b"], rope=g.rope))
+            n_seg.append(ns); seg_len.append(sl); where.append((gi, off)); rope.append(g.rope)
+    return pairs, n_seg, seg_len, where, rope
 
 
 def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: float, l1: bool = True,
@@ -96,7 +97,7 @@ def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: f
     the physical removal from every tensor of the group.  Returns (new groups, info)."""
     assert k_min >= 1 and all(w >= 1 for g in groups for w in g.widths)
     dev = groups[0].w1.device
-    pairs, n_seg, seg_len, where = describe(groups)
+    pairs, n_seg, seg_len, where, rope = describe(groups)
     total_segs = sum(n_seg)
     total_d = sum(a * b for a, b in zip(n_seg, seg_len))
     i32, f32 = torch.int32, torch.float32
@@ -110,7 +111,7 @@ def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: f
     slots = torch.empty(total_d, dtype=i32, device=dev)
     k_out = torch.empty(total_segs, dtype=i32, device=dev)
     B.ecospa_select_aligned_threshold(ups, n_seg, seg_len, theta, slots, k_out, l1=l1, k_min=k_min, chosen=chosen,
-                                      stream=stream)
+                                      rope=rope if any(rope) else None, stream=stream)
     k = k_out.cpu().tolist()                 # the one read-back: the counts size everything that follows
 
     # per group: the kept list of the whole shared axis, then one gather per tensor
@@ -144,7 +145,7 @@ def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: f
             return o
         ng = Group(shrink(g.w1, g.layout1), shrink(g.w2, g.layout2), g.layout1, g.layout2, new_widths[gi],
                    w1b=shrink(g.w1b, g.layout1), g1=shrink(g.g1, g.layout1), g2=shrink(g.g2, g.layout2),
-                   g1b=shrink(g.g1b, g.layout1), aux=[(shrink(t, lay), lay) for t, lay in g.aux])
+                   g1b=shrink(g.g1b, g.layout1), aux=[(shrink(t, lay), lay) for t, lay in g.aux], rope=g.rope)
         out_groups.append(ng)
     B.ecospa_compact_tensors(jobs, stream=stream)
     info = {"k": new_widths, "kept": kept_lists, "fisher": fis, "chosen": chosen, "upsilon": ups, "n_chosen": m}

@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def make_groups(wl, with_moments=True):
+def make_groups(wl, with_moments=True, rope=0):
     w = WL.layer_weights(wl, 0)
     g = WL.layer_grads(wl, 0)
     gen = torch.Generator().manual_seed(11)
@@ -27,7 +27,7 @@ def make_groups(wl, with_moments=True):
     def mom(t):
         return torch.rand(t.shape, generator=gen, dtype=torch.float32)
 
-    qk = dict(w1=w["wq"], w2=w["wk"], layout1=0, layout2=0, widths=[dh] * h, g1=g["gq"], g2=g["gk"], aux=[])
+    qk = dict(w1=w["wq"], w2=w["wk"], layout1=0, layout2=0, widths=[dh] * h, g1=g["gq"], g2=g["gk"], aux=[], rope=rope)
     vo = dict(w1=w["wv"], w2=w["wo"], layout1=0, layout2=1, widths=[dh] * h, g1=g["gv"], g2=g["go"], aux=[])
     ffn = dict(w1=w["w1"], w2=w["w2"], layout1=0, layout2=1, widths=[wl.d_ffn], g1=g["g1"], g2=g["g2"], aux=[])
     if "w1b" in w:
@@ -64,7 +64,7 @@ def oracle_pass(specs, info, n_samples, ratio, theta, k_min):
         for wd in sp["widths"]:
             s = lambda nm, lay: cut(sp[nm], lay, off, wd) if sp.get(nm) is not None else None
             _, u = O.score_pair(s("w1", sp["layout1"]), s("w2", sp["layout2"]), sp["layout1"], sp["layout2"], 1, wd,
-                                w1b=s("w1b", sp["layout1"]))
+                                w1b=s("w1b", sp["layout1"]), rope=sp.get("rope", 0))
             f = O.fisher_pair(s("g1", sp["layout1"]), s("g2", sp["layout2"]), sp["layout1"], sp["layout2"], 1, wd, n_samples,
                               g1b=s("g1b", sp["layout1"]))
             u_ref.append(u); f_ref.append(f)
@@ -86,8 +86,9 @@ def oracle_pass(specs, info, n_samples, ratio, theta, k_min):
         kept_g, new_w, off = [], [], 0
         for wd in sp["widths"]:
             u = ups[pos:pos + wd]
-            k = int(O.threshold_counts(u, 1, wd, theta, l1=True, k_min=k_min, chosen=[int(chosen[seg])])[0])
-            kept_g.append(O.select_topk(u, 1, wd, [k]) + off)
+            rp = sp.get("rope", 0)
+            k = int(O.threshold_counts(u, 1, wd, theta, l1=True, k_min=k_min, chosen=[int(chosen[seg])], rope=rp)[0])
+            kept_g.append((O.select_rotation_pairs(u, 1, wd, [k], rp) if rp else O.select_topk(u, 1, wd, [k])) + off)
             new_w.append(k)
             pos += wd; off += wd; seg += 1
         kept_g = np.concatenate(kept_g).astype(np.int32)
@@ -110,10 +111,11 @@ def same_bytes(gpu_t, ref, layout, D):
     return torch.equal(g.view(view), ref.contiguous().view(view))
 
 
-@pytest.mark.parametrize("name", ["tails768", "tiny_swiglu"])
-def test_two_passes_match_the_oracle(name):
+@pytest.mark.parametrize("name,rope", [("tails768", 0), ("tiny_swiglu", 0), ("tails768", B.ROPE_HALF),
+                                       ("tiny_swiglu", B.ROPE_INTERLEAVED)])
+def test_two_passes_match_the_oracle(name, rope):
     wl = WL.WORKLOADS[name]
-    specs = make_groups(wl)
+    specs = make_groups(wl, rope=rope)
     groups = [to_gpu(sp) for sp in specs]
     n_samples = float(wl.tokens)
     for ratio, theta in ((0.5, 0.9), (0.6, 0.8)):
