@@ -4,4 +4,4 @@ The work is done by CUDA kernels in libecospa.so behind a C ABI (include/ecospa.
 `binding` marshals torch tensors into it.  Importing this package does not load the
 library; the first call does, and raises if it has not been built.
 """
-from . import binding, block, layers, workloads  # noqa: F401
+from . import algorithm1, binding, block, layers, workloads  # noqa: F401
