@@ -410,6 +410,16 @@ def run_gpu(args):
                      "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
                      "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                      "launches_per_step": n_gemm_launches, "avg_launch_ms": ms_gemm / n_gemm_launches},
+        # the memory-bound part of the step against the measured copy bandwidth: score + select + compact as one unit
+        # (sumsq_kernel and gather_kernel move all of its bytes; traffic = their DRAM bytes under ncu on 8 layers of
+        # gpt2m, which grow in proportion to the layer count: 889.3 MB per 8 layers, profiles/sparsify_kernels_*.md)
+        "roofline_hbm": {"bound": "hbm", "kernel": "sumsq_kernel + gather_kernel (+ finalize, select)",
+                         "achieved": sbytes / ms_sp / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": sbytes / ms_sp / 1e6 / peaks["hbm_gbs"],
+                         "traffic": (889.3e6 * wl.n_layers / 8 if (wl.name == "gpt2m" and args.sparsity == 0.5
+                                                                   and not args.transposed) else None),
+                         "traffic_unit": "bytes per step (DRAM read + write, ncu, scaled by layers)",
+                         "peak_source": peaks["source"] + " (copy bandwidth)"},
         "e2e": {"value": job_throughput(world, flops, ms_e2e) / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "pipeline": "two device copies of the model: the upload of step s+1 overlaps the compute of step s"},
