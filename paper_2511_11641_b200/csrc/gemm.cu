@@ -3,7 +3,7 @@
 //   single  cta_group::1, one CTA per SM computes 128x256 tiles (2 stages of 2 x (16 KB A + 32 KB B))
 //   pair    cta_group::2, a cluster of two CTAs computes 256x256 tiles: each CTA loads its 128 rows of A
 //           and its half of B (3 stages of 2 x (16 KB + 16 KB)), the leader CTA issues the MMAs for both,
-//           so every SM fetches a third less operand data per flop.  No cluster multicast is used: the
+//           so every SM fetches a third less operand data per flop.  Every CTA issues its own loads: the
 //           peer's loads signal the leader's barrier, and completion is committed to each CTA's barrier.
 //
 // One launch computes up to kMaxGemmOps independent products ("ops"), each C = sum over one to three
