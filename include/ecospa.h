@@ -63,9 +63,9 @@ typedef struct {
 } ecospa_mat_t;
 
 /* Rotary position embedding (Eq. "self-attention-rope"): W_Q P_t and W_K P_s rotate the shared index in 2 x 2
- * blocks, so the unit that can be removed ("position matrices are then adjusted to match new dimensions",
- * footnote to Eq. "l2norm") is a rotation pair of shared indices, and the rotations leave the Frobenius norm of a
- * pair's two columns unchanged at every position.  Which two indices of a segment form pair b: */
+ * blocks.  The footnote to Eq. "l2norm" removes on W_Q / W_K and has the position matrices shrink to the new
+ * width, so the unit that can be removed is a rotation pair of shared indices; the rotations leave the Frobenius
+ * norm of a pair's two columns unchanged at every position.  Which two indices of a segment form pair b: */
 typedef enum {
     ECOSPA_ROPE_NONE = 0,        /* no rotation: every shared index is scored and removed on its own */
     ECOSPA_ROPE_INTERLEAVED = 1, /* (2b, 2b+1), the blocks as the paper prints them */
@@ -123,6 +123,7 @@ uint64_t ecospa_launch_count(void);
  * Results are bit-identical from run to run (no floating-point atomics).
  * NaN/Inf inputs: unspecified.  Tensors with 16-byte aligned base and ld*sizeof(elem) % 16 == 0
  * take the vector path; others are read element-wise (slower, same results).
+ * D = n_seg * seg_len up to 2^22 per pair group (ECOSPA_ERR_UNSUPPORTED beyond).
  */
 size_t ecospa_score_workspace_bytes(const ecospa_pair_t* pairs, int32_t n_pairs);
 ecospa_status_t ecospa_score_pairs(const ecospa_pair_t* pairs, int32_t n_pairs, double n_samples, float* upsilon,
@@ -365,10 +366,17 @@ ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, int64_t T, in
  * pair mode is off (environment ECOSPA_GEMM_PAIR=0), -1 on a CUDA error.  Informational. */
 int32_t ecospa_gemm_resident_pairs(void);
 
-/* Synchronises `stream` and reports the device status word: ECOSPA_OK and *code = 0, or
+/* Synchronises `stream` and reports the status word of the current device: ECOSPA_OK and *code = 0, or
  * ECOSPA_ERR_TIMEOUT and *code = which bounded wait expired (1 producer, 2 accumulator-free,
- * 3 operands-ready, 4 accumulator-ready); the word is cleared.  This is the one call that blocks. */
+ * 3 operands-ready, 4 accumulator-ready); the word is cleared.  This is the one call that blocks.
+ * Every device the library is used on has its own status word. */
 ecospa_status_t ecospa_device_status(void* stream, int32_t* code);
+
+/* How long a device-side wait of the step-4 kernels (on an operand copy, a free pipeline stage or an
+ * accumulator) may last before the kernel gives up, records its code and returns; nanoseconds, default
+ * 2 s, process-wide, read when a call enqueues its launches.  ns == 0 -> ECOSPA_ERR_INVALID.  (No counterpart in
+ * the paper: failure reporting of this library.) */
+ecospa_status_t ecospa_set_device_wait_limit_ns(uint64_t ns);
 
 #ifdef __cplusplus
 }

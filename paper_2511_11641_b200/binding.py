@@ -485,6 +485,20 @@ def ecospa_launch_count() -> int:
     return int(f())
 
 
+def ecospa_set_device_wait_limit_ns(ns: int) -> None:
+    """How long a device-side wait of the layer kernels may last before the kernel gives up (default 2 s)."""
+    f = lib().ecospa_set_device_wait_limit_ns
+    f.restype = C.c_int
+    f.argtypes = [C.c_uint64]
+    _check(f(int(ns)), "ecospa_set_device_wait_limit_ns")
+
+
+def ecospa_gemm_resident_pairs() -> int:
+    f = lib().ecospa_gemm_resident_pairs
+    f.restype = C.c_int32
+    return int(f())
+
+
 def ecospa_device_status(stream=None) -> int:
     """Synchronises the stream; returns 0 or raises EcospaError(ERR_TIMEOUT) carrying the wait code."""
     code = C.c_int32(0)

@@ -160,6 +160,7 @@ ecospa_status_t validate_job(const ecospa_gather_t& g) {
     if (in.layout != ECOSPA_SHARED_COLS && in.layout != ECOSPA_SHARED_ROWS) return ECOSPA_ERR_INVALID;
     if (in.other_dim < 1 || in.other_dim > INT32_MAX || in.ld > INT32_MAX || out.ld > INT32_MAX) return ECOSPA_ERR_INVALID;
     if (g.n_kept < 0 || g.shared_dim < 1 || g.n_kept > g.shared_dim) return ECOSPA_ERR_INVALID;
+    if (g.shared_dim > (1 << 22)) return ECOSPA_ERR_UNSUPPORTED;   // tile counts along the shared axis are 16-bit
     const int eb = elem_bytes(in.dtype);
     if (reinterpret_cast<uintptr_t>(in.ptr) % eb || reinterpret_cast<uintptr_t>(out.ptr) % eb) return ECOSPA_ERR_ALIGNMENT;
     int64_t in_bytes, out_bytes;

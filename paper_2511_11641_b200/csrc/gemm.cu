@@ -25,6 +25,7 @@
 #include <cuda_bf16.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <mutex>
@@ -52,7 +53,7 @@ constexpr int kMapsPerOp = kOperandMaps + 3; // + one store map per output (C, C
 constexpr int kEpiSlotBytes = 32 * 32 * 2;  // one 32-row x 64-byte staging image; a warp owns two (= one 32 x 128-byte image)
 constexpr int kEpiBytes = kEpiWarps * 2 * kEpiSlotBytes;
 constexpr int kSmemBytes = kRingBytes + kEpiBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr unsigned long long kDefaultWaitLimitNs = 2000000000ull;  // 2 s
 
 struct DevProblem {
     int32_t M, N;
@@ -89,6 +90,7 @@ struct GemmParams {
     uint16_t order[kMaxOrder];
     int32_t n_problems, total_tiles, rounds, use_order;
     int* status;
+    unsigned long long wait_limit_ns;   // every mbarrier wait of the launch gives up after this long
 };
 
 __device__ int g_gemm_status = 0;
@@ -126,18 +128,21 @@ __device__ __forceinline__ unsigned long long global_ns() {
 
 // Bounded wait.  Returns false if the wait gave up (or another thread of the CTA already did).
 template <bool CLUSTER>
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code, int* status) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int code, int* status,
+                                          unsigned long long limit_ns) {
     // Fast path: plain polling.  The (slow) global timer is only consulted every 1024 failed polls,
-    // so a wait that completes normally never touches it.
+    // so a wait that completes normally never touches it (limits under a millisecond look at it on
+    // every failed poll, so that they are kept to within a poll).
     unsigned long long t0 = 0;
     uint32_t spins = 0;
+    const uint32_t mask = limit_ns < 1000000ull ? 0u : 1023u;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
-        if ((++spins & 1023u) == 0) {
+        if ((++spins & mask) == 0) {
             if (*abort_flag) return false;
             const unsigned long long now = global_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicCAS(status, 0, code);
                 return false;
@@ -603,7 +608,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 const int kb_lo = seg ? Q.kb_end[seg - 1] : 0, kb_hi = Q.kb_end[seg];
                 for (int kb0 = kb_lo; kb0 < kb_hi; kb0 += kSub) {
                     const int nsub = min(kSub, kb_hi - kb0);
-                    if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status))) break;
+                    if (!(ok = mbar_wait<PAIR>(empty_bar(stage), phase ^ 1u, abort_flag, 1, P.status, P.wait_limit_ns))) break;
                     // "big" operands arrive as one box holding both k-blocks (zero-filled past the end of K)
                     const bool a_big = PAIR && Q.a_big[seg], b_big = PAIR && Q.b_big[seg];
                     const uint32_t tx = (a_big ? kSub : nsub) * kAStage + (b_big ? kSub : nsub) * kBLocal;
@@ -722,14 +727,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                 const DevProblem& Q = find_problem(P, tile);
                 const int acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1u;
-                if (!(ok = mbar_wait<PAIR>(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 2, P.status))) break;
+                if (!(ok = mbar_wait<PAIR>(tempty_bar(acc), acc_phase ^ 1u, abort_flag, 2, P.status, P.wait_limit_ns))) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int seg = 0; ok && seg < kMaxSeg; ++seg) {
                 const int kb_lo = seg ? Q.kb_end[seg - 1] : 0, kb_hi = Q.kb_end[seg];
                 for (int kb0 = kb_lo; kb0 < kb_hi; kb0 += kSub) {
                     const int nsub = min(kSub, kb_hi - kb0);
-                    if (!(ok = mbar_wait<PAIR>(full_bar(stage), phase, abort_flag, 3, P.status))) break;
+                    if (!(ok = mbar_wait<PAIR>(full_bar(stage), phase, abort_flag, 3, P.status, P.wait_limit_ns))) break;
                     tc_fence_after();
 #pragma unroll
                     for (int sub = 0; sub < kSub; ++sub) {
@@ -813,7 +818,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_kernel(const __grid_constant
                                              : __uint_as_float(static_cast<uint32_t>(static_cast<const unsigned short*>(Q.bias)[col]) << 16);
                 }
             }
-            if (!(ok = mbar_wait<PAIR>(tfull_bar(acc), acc_phase, abort_flag, 4, P.status))) break;
+            if (!(ok = mbar_wait<PAIR>(tfull_bar(acc), acc_phase, abort_flag, 4, P.status, P.wait_limit_ns))) break;
             tc_fence_after();
             const uint32_t t_row = tmem_base + acc * BN + (static_cast<uint32_t>(quad * 32) << 16);
             const bool warp_rows = m_warp < QM;          // any row of this warp inside the output
@@ -1109,25 +1114,41 @@ ecospa_status_t encode_out_map(CUtensorMap* out, void* ptr, int64_t rows, int64_
     return ECOSPA_OK;
 }
 
-int g_num_sms = 0;
-int* g_status_ptr = nullptr;
-int g_max_pairs = 0;   // CTA pairs that can be resident at once (clusters must fit inside a GPC)
+// Per-device facts of the engine, looked up the first time a device is used (with that device current).
+constexpr int kMaxDevices = 64;
+struct DeviceState {
+    std::once_flag once;
+    ecospa_status_t st = ECOSPA_OK;
+    int num_sms = 0;
+    int max_pairs = 0;      // CTA pairs that can be resident at once (clusters must fit inside a GPC)
+    int* status_ptr = nullptr;   // this device's copy of g_gemm_status
+};
+DeviceState g_dev[kMaxDevices];
 int g_pair_mode = 1;   // 1: CTA pairs (cta_group::2) whenever an op has more than one 128-row tile; 0: never
+std::atomic<unsigned long long> g_wait_limit_ns{kDefaultWaitLimitNs};
 
-ecospa_status_t gemm_setup() {
-    static std::once_flag once;
-    static ecospa_status_t st = ECOSPA_OK;
-    std::call_once(once, [] {
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+// State of the current device (set up on first use), or nullptr with *st set.
+DeviceState* gemm_setup(ecospa_status_t* st_out) {
+    int dev = 0;
+    cudaError_t e0 = cudaGetDevice(&dev);
+    if (e0 != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+        if (e0 != cudaSuccess) {
+            set_cuda_error(e0, "gemm setup (cudaGetDevice)");
+            cudaGetLastError();
+        }
+        *st_out = e0 != cudaSuccess ? ECOSPA_ERR_CUDA : ECOSPA_ERR_UNSUPPORTED;
+        return nullptr;
+    }
+    DeviceState& D = g_dev[dev];
+    std::call_once(D.once, [&D, dev] {
+        cudaError_t e = cudaDeviceGetAttribute(&D.num_sms, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (const char* v = std::getenv("ECOSPA_GEMM_PAIR")) g_pair_mode = std::atoi(v);
         if (e == cudaSuccess) {
             // the tile schedule is static, so only as many pairs as can run at the same time are launched
             cudaLaunchConfig_t cfg = {};
-            cfg.gridDim = dim3(2 * (g_num_sms / 2));
+            cfg.gridDim = dim3(2 * (D.num_sms / 2));
             cfg.blockDim = dim3(kThreads);
             cfg.dynamicSmemBytes = kSmemBytes;
             cudaLaunchAttribute attr[1];
@@ -1138,17 +1159,18 @@ ecospa_status_t gemm_setup() {
             cfg.attrs = attr;
             cfg.numAttrs = 1;
             int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true>, &cfg) == cudaSuccess && n > 0) g_max_pairs = n;
+            if (cudaOccupancyMaxActiveClusters(&n, gemm_kernel<true>, &cfg) == cudaSuccess && n > 0) D.max_pairs = n;
             else cudaGetLastError();
-            if (g_max_pairs < 1) g_pair_mode = 0;
         }
-        if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&g_status_ptr), g_gemm_status);
+        if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&D.status_ptr), g_gemm_status);
         if (e != cudaSuccess) {
             set_cuda_error(e, "gemm setup");
-            st = ECOSPA_ERR_CUDA;
+            cudaGetLastError();
+            D.st = ECOSPA_ERR_CUDA;
         }
     });
-    return st;
+    *st_out = D.st;
+    return D.st == ECOSPA_OK ? &D : nullptr;
 }
 
 // Tile schedule.  Tiles are numbered op by op, longest contraction first.  With few tiles per worker the
@@ -1189,10 +1211,38 @@ void build_schedule(GemmParams& gp, int workers) {
 
 }  // namespace
 
-ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t stream) {
+// Host-only checks of a launch (no CUDA call): shapes, pointers, 16-byte alignment of every base and pitch.
+ecospa_status_t validate_gemm_ops(const GemmOp* ops, int n_ops) {
     if (!ops || n_ops < 1 || n_ops > kMaxGemmOps) return ECOSPA_ERR_INVALID;
-    ecospa_status_t st = gemm_setup();
+    for (int i = 0; i < n_ops; ++i) {
+        const GemmOp& op = ops[i];
+        if (op.M < 1 || op.N < 1 || op.n_kseg < 1 || op.n_kseg > kMaxSeg || !op.C || op.ldc < 1) return ECOSPA_ERR_INVALID;
+        if (op.M > INT32_MAX || op.N > INT32_MAX) return ECOSPA_ERR_INVALID;
+        if (op.epi < EPI_STORE || op.epi > EPI_DSWIGLU) return ECOSPA_ERR_INVALID;
+        const int out_eb = op.out_f32 ? 4 : 2;
+        if (!aligned16(op.C) || (op.ldc * out_eb) % 16) return ECOSPA_ERR_ALIGNMENT;
+        if (op.ldc < op.N) return ECOSPA_ERR_INVALID;
+        if (op.bias && !aligned16(op.bias)) return ECOSPA_ERR_ALIGNMENT;
+        for (int s = 0; s < op.n_kseg; ++s) {
+            const KSegment& ks = op.seg[s];
+            if (ks.K < 1 || ks.k_begin < 0 || ks.k_begin % BK) return ECOSPA_ERR_INVALID;
+            const Stored* mats[3] = {&ks.a, &ks.b[0], op.epi == EPI_SWIGLU ? &ks.b[1] : nullptr};
+            for (const Stored* m : mats) {
+                if (!m) continue;
+                if (!m->ptr || m->rows < 1 || m->cols < 1 || m->ld < m->cols) return ECOSPA_ERR_INVALID;
+                if (!aligned16(m->ptr) || (m->ld * 2) % 16) return ECOSPA_ERR_ALIGNMENT;
+            }
+        }
+    }
+    return ECOSPA_OK;
+}
+
+ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t stream) {
+    ecospa_status_t st = validate_gemm_ops(ops, n_ops);
     if (st != ECOSPA_OK) return st;
+    DeviceState* dev = gemm_setup(&st);
+    if (!dev) return st;
+    const int g_max_pairs = dev->max_pairs, g_num_sms = dev->num_sms;
 
     // longest contraction first
     int order[kMaxGemmOps];
@@ -1296,7 +1346,8 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
     }
     gp.n_problems = n_ops;
     gp.total_tiles = tiles;
-    gp.status = g_status_ptr;
+    gp.status = dev->status_ptr;
+    gp.wait_limit_ns = g_wait_limit_ns.load(std::memory_order_relaxed);
     const int workers = pair ? std::min(tiles, g_max_pairs) : std::min(tiles, g_num_sms);
     build_schedule(gp, workers);
     cudaLaunchConfig_t cfg = {};
@@ -1322,29 +1373,40 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
     return check_launch("gemm_kernel");
 }
 
+int gemm_resident_pairs() {
+    ecospa_status_t st;
+    DeviceState* dev = gemm_setup(&st);
+    if (!dev) return -1;
+    return g_pair_mode ? dev->max_pairs : 0;
+}
+
 }  // namespace ecospa
 
 extern "C" ecospa_status_t ecospa_device_status(void* stream, int32_t* code) {
     if (!code) return ECOSPA_ERR_INVALID;
-    ecospa_status_t st = ecospa::gemm_setup();
-    if (st != ECOSPA_OK) return st;
+    ecospa_status_t st;
+    ecospa::DeviceState* dev = ecospa::gemm_setup(&st);
+    if (!dev) return st;
     cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
     int v = 0;
-    if (e == cudaSuccess) e = cudaMemcpy(&v, ecospa::g_status_ptr, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(&v, dev->status_ptr, sizeof(int), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) {
         ecospa::set_cuda_error(e, "ecospa_device_status");
         return ECOSPA_ERR_CUDA;
     }
     *code = v;
     if (v != 0) {
-        cudaMemset(ecospa::g_status_ptr, 0, sizeof(int));
+        cudaMemset(dev->status_ptr, 0, sizeof(int));
         return ECOSPA_ERR_TIMEOUT;
     }
     return ECOSPA_OK;
 }
 
 // Number of CTA pairs the GEMM engine runs at once on the current device (0 = pair mode off).
-extern "C" int32_t ecospa_gemm_resident_pairs(void) {
-    if (ecospa::gemm_setup() != ECOSPA_OK) return -1;
-    return ecospa::g_pair_mode ? ecospa::g_max_pairs : 0;
+extern "C" int32_t ecospa_gemm_resident_pairs(void) { return ecospa::gemm_resident_pairs(); }
+
+extern "C" ecospa_status_t ecospa_set_device_wait_limit_ns(uint64_t ns) {
+    if (ns == 0) return ECOSPA_ERR_INVALID;
+    ecospa::g_wait_limit_ns.store(ns, std::memory_order_relaxed);
+    return ECOSPA_OK;
 }

@@ -60,4 +60,11 @@ constexpr int kMaxGemmOps = 16;
 // contraction are scheduled first).  Operands must be 16-byte aligned with 16-byte pitches.
 ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t stream);
 
+// The host-only checks launch_grouped_gemm starts with (shapes, null pointers, 16-byte alignment of every base and
+// pitch); makes no CUDA call.  Calls that enqueue several launches check all of them before the first.
+ecospa_status_t validate_gemm_ops(const GemmOp* ops, int n_ops);
+
+// CTA pairs the engine keeps resident on the current device (0: pair mode off, -1: no usable device).
+int gemm_resident_pairs();
+
 }  // namespace ecospa

@@ -269,10 +269,12 @@ Stored scratch_bf16(Ctx& cx, int64_t rows, int64_t cols) {
     return s;
 }
 
-// Column sums of up to three bf16 matrices with the same row count: launches the chunk-partial kernel and
-// returns the description the finishing launch needs.  A null output skips that matrix.
-ColsumParams colsum_begin(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), void* out2 = nullptr,
-                          const Stored& M3 = Stored(), void* out3 = nullptr) {
+// Column sums of up to three bf16 matrices with the same row count.  colsum_plan takes the scratch of the chunk
+// partials from the workspace (so that a short workspace is reported before anything is launched) and returns the
+// description that colsum_begin (launch of the chunk-partial kernel) and the finishing launch need.  A null output
+// skips that matrix.
+ColsumParams colsum_plan(Ctx& cx, const Stored& M1, void* out1, const Stored& M2 = Stored(), void* out2 = nullptr,
+                         const Stored& M3 = Stored(), void* out3 = nullptr) {
     ColsumParams P = {};
     if (cx.st != ECOSPA_OK) return P;
     const Stored* mats[3] = {&M1, &M2, &M3};
@@ -291,7 +293,6 @@ ColsumParams colsum_begin(Ctx& cx, const Stored& M1, void* out1, const Stored& M
     if (P.n_jobs == 0) return P;
     P.chunks = static_cast<int32_t>(ceil_div(P.rows, kSumRows));
     P.out_f32 = cx.dtype == ECOSPA_F32;
-    int tiles = 0;
     for (int i = 0; i < P.n_jobs; ++i) {
         P.job[i].partial = static_cast<float*>(cx.arena.take(static_cast<size_t>(P.chunks) * P.job[i].cols * 4));
         if (!P.job[i].partial) {
@@ -299,8 +300,13 @@ ColsumParams colsum_begin(Ctx& cx, const Stored& M1, void* out1, const Stored& M
             P.n_jobs = 0;
             return P;
         }
-        tiles += P.job[i].col_tiles;
     }
+    return P;
+}
+const ColsumParams& colsum_begin(Ctx& cx, const ColsumParams& P) {
+    if (cx.st != ECOSPA_OK || P.n_jobs == 0) return P;
+    int tiles = 0;
+    for (int i = 0; i < P.n_jobs; ++i) tiles += P.job[i].col_tiles;
     const cudaError_t e = launch_pdl(colsum_partial_kernel, dim3(tiles, P.chunks), cx.stream, P);
     if (e != cudaSuccess) {
         set_cuda_error(e, "colsum_partial_kernel launch");
@@ -364,14 +370,24 @@ GemmOp proj_op(const Stored& X, const Stored& W, bool w_mn, int64_t T, int64_t d
 // Weight gradients contract over the T tokens and have few output tiles, so on their own they would keep
 // most SMs idle behind one long tile.  The token range is therefore cut into `splits` ranges computed as
 // separate ops of the same launch into fp32 partial buffers, which the finishing launch (post_kernel) adds up in split order.
-constexpr int64_t kWorkers = 74;                  // CTA pairs the engine keeps resident
+// Workers of a launch: the CTA pairs the engine keeps resident on the current device (74 on a 148-SM part, which is
+// also what the size queries assume when no device can be asked).
+int64_t engine_workers() {
+    static thread_local int cached = 0;
+    if (cached <= 0) {
+        const int n = gemm_resident_pairs();
+        if (n <= 0) return 74;
+        cached = n;
+    }
+    return cached;
+}
 // Cost of a product in k-blocks of 256x256 tiles (what one worker spends on it if it ran alone).
 int64_t gemm_cost(int64_t M, int64_t N, int64_t K) { return ceil_div(M, 256) * ceil_div(N, 256) * ceil_div(K, 64); }
 // `launch_cost` = cost of every product of the launch.  The scheduler hands tiles out longest first, so a
 // tile much longer than a worker's fair share of the launch sets the duration: cut the tokens until it is
 // not (a tile up to 1.3 shares is left whole: the partial sums and their reduction cost more than they save).
 int wgrad_splits(int64_t rows_out, int64_t cols_out, int64_t T, int64_t launch_cost) {
-    const int64_t share = std::max<int64_t>(launch_cost / kWorkers, 1);
+    const int64_t share = std::max<int64_t>(launch_cost / engine_workers(), 1);
     int64_t s = ceil_div(10 * ceil_div(T, 64), 13 * share);
     s = std::min<int64_t>(s, T / 1024);            // at least 16 k-blocks per range
     s = std::min<int64_t>(s, 6);
@@ -557,8 +573,10 @@ extern "C" ecospa_status_t ecospa_coupled_qk_bwd(const void* X, int64_t ldx, int
         dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].b_mn = mn_over_shared(wk_c); dx.seg[1].K = n;
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
+    const ColsumParams cs = colsum_plan(cx, dQs, dbq_c, dKs, wk_c ? dbk_c : nullptr);
+    if (cx.st != ECOSPA_OK) return cx.st;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    finish(cx, red, 2, colsum_begin(cx, dQs, dbq_c, dKs, wk_c ? dbk_c : nullptr));
+    finish(cx, red, 2, colsum_begin(cx, cs));
     return cx.st;
 }
 
@@ -627,8 +645,10 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd(const void* X, int64_t ldx, con
     dx.M = T; dx.N = d_m; dx.n_kseg = 1;
     dx.seg[0].a = dVs; dx.seg[0].b[0] = Wv; dx.seg[0].b_mn = mn_over_shared(wv_c); dx.seg[0].K = n;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32; dx.accumulate = accumulate_dX != 0;
+    const ColsumParams cs = colsum_plan(cx, dVs, dbv_c, dOs, dbo);
+    if (cx.st != ECOSPA_OK) return cx.st;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    finish(cx, red, 2, colsum_begin(cx, dVs, dbv_c, dOs, dbo));
+    finish(cx, red, 2, colsum_begin(cx, cs));
     return cx.st;
 }
 
@@ -694,8 +714,10 @@ extern "C" ecospa_status_t ecospa_coupled_qkv_bwd(const void* X, int64_t ldx, in
     dx.seg[1].a = dKs; dx.seg[1].b[0] = Wk; dx.seg[1].b_mn = mn_over_shared(wk_c); dx.seg[1].K = n_qk;
     dx.seg[2].a = dVs; dx.seg[2].b[0] = Wv; dx.seg[2].b_mn = mn_over_shared(wv_c); dx.seg[2].K = n_vo;
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = cx.dtype == ECOSPA_F32; dx.accumulate = accumulate_dX != 0;
+    const ColsumParams cs = colsum_plan(cx, dQs, dbq_c, dKs, dbk_c, dVs, dbv_c);
+    if (cx.st != ECOSPA_OK) return cx.st;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    finish(cx, red, 3, colsum_begin(cx, dQs, dbq_c, dKs, dbk_c, dVs, dbv_c));
+    finish(cx, red, 3, colsum_begin(cx, cs));
     return cx.st;
 }
 
@@ -723,8 +745,10 @@ extern "C" ecospa_status_t ecospa_coupled_vo_bwd_o(const void* Ctxm, int64_t ld_
     dc.M = T; dc.N = n; dc.n_kseg = 1;
     dc.seg[0].a = dOs; dc.seg[0].b[0] = Wo; dc.seg[0].b_mn = mn_over_other(wo_c); dc.seg[0].K = d_m;
     dc.epi = EPI_STORE; dc.C = dCtx; dc.ldc = ld_dctx; dc.out_f32 = cx.dtype == ECOSPA_F32;
+    const ColsumParams cs = colsum_plan(cx, dOs, dbo);
+    if (cx.st != ECOSPA_OK) return cx.st;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    finish(cx, &red, 1, colsum_begin(cx, dOs, dbo));
+    finish(cx, &red, 1, colsum_begin(cx, cs));
     return cx.st;
 }
 
@@ -775,6 +799,7 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_fwd(const void* X, int64_t ldx, in
     down.epi = EPI_STORE; down.C = Y; down.ldc = ld_y; down.out_f32 = f32;
     down.bias = b2; down.bias_f32 = f32;
     if (cx.st != ECOSPA_OK) return cx.st;
+    if ((st = validate_gemm_ops(&up, 1)) != ECOSPA_OK || (st = validate_gemm_ops(&down, 1)) != ECOSPA_OK) return st;
     if ((st = launch_grouped_gemm(&up, 1, cx.stream)) != ECOSPA_OK) return st;
     return launch_grouped_gemm(&down, 1, cx.stream);
 }
@@ -812,9 +837,10 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     As.ptr = A; As.rows = T; As.cols = k; As.ld = ld_h;
 
     // Two launches of about equal length.  First: dH = (dY W_2^T) (.) act'(H) (W_2 stored k x d_m = [N][K], the
-    // derivative fused into the epilogue) together with dW_2 = A^T dY, which does not need dH.
+    // derivative fused into the epilogue) together with dW_2 = A^T dY, which does not need dH.  Both launches are
+    // described (and all their scratch is taken from the workspace) before the first one is enqueued.
     const int nw = sw ? 2 : 1;
-    GemmOp ops[kMaxGemmOps];
+    GemmOp ops[kMaxGemmOps], ops2[kMaxGemmOps];
     PendingReduce red[3];
     int n_ops = 0;
     n_ops = add_wgrad_w(cx, ops, n_ops, w2_c, dYs, As, d_m, k, T, dW2_c, ld_dw2, &red[0], 1,
@@ -826,15 +852,14 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
     da.epi = sw ? EPI_DSWIGLU : (act == ECOSPA_ACT_GELU_ERF ? EPI_DGELU_ERF : EPI_DGELU_TANH);
     da.C = const_cast<void*>(dH.ptr); da.C2 = sw ? const_cast<void*>(dHb.ptr) : nullptr; da.ldc = dH.ld;
     da.H = H; da.Hb = Hb; da.ldh = ld_h;
-    if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
 
     // Second: dW_1 = X^T dH (and dW_up = X^T dH_up), dX = dH W_1^T (+ dH_up W_up^T)
-    n_ops = 0;
+    int n_ops2 = 0;
     const int64_t cost = nw * gemm_cost(d_m, k, T) + gemm_cost(T, d_m, nw * k);
-    n_ops = add_wgrad_w(cx, ops, n_ops, w1_c, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1, cost);   // dW_1, stored like W_1
-    if (sw) n_ops = add_wgrad_w(cx, ops, n_ops, w1b_c, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1, cost); // dW_up
+    n_ops2 = add_wgrad_w(cx, ops2, n_ops2, w1_c, Xs, dH, d_m, k, T, dW1_c, ld_dw1, &red[1], sw ? 2 : 1, cost);   // dW_1, stored like W_1
+    if (sw) n_ops2 = add_wgrad_w(cx, ops2, n_ops2, w1b_c, Xs, dHb, d_m, k, T, dW1b_c, ld_dw1, &red[2], 1, cost); // dW_up
     if (cx.st != ECOSPA_OK) return cx.st;
-    GemmOp& dx = ops[n_ops++];
+    GemmOp& dx = ops2[n_ops2++];
     dx = GemmOp();
     dx.M = T; dx.N = d_m; dx.n_kseg = sw ? 2 : 1;
     dx.seg[0].a = dH; dx.seg[0].b[0] = W1; dx.seg[0].b_mn = mn_over_shared(w1_c); dx.seg[0].K = k;
@@ -842,7 +867,11 @@ extern "C" ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, in
         dx.seg[1].a = dHb; dx.seg[1].b[0] = W1b; dx.seg[1].b_mn = mn_over_shared(w1b_c); dx.seg[1].K = k;
     }
     dx.epi = EPI_STORE; dx.C = dX; dx.ldc = ld_dx; dx.out_f32 = f32;
+    const ColsumParams cs = colsum_plan(cx, dYs, db2, dH, sw ? nullptr : db1_c);
+    if (cx.st != ECOSPA_OK) return cx.st;
+    if ((st = validate_gemm_ops(ops, n_ops)) != ECOSPA_OK || (st = validate_gemm_ops(ops2, n_ops2)) != ECOSPA_OK) return st;
     if ((st = launch_grouped_gemm(ops, n_ops, cx.stream)) != ECOSPA_OK) return st;
-    finish(cx, red, 3, colsum_begin(cx, dYs, db2, dH, sw ? nullptr : db1_c));
+    if ((st = launch_grouped_gemm(ops2, n_ops2, cx.stream)) != ECOSPA_OK) return st;
+    finish(cx, red, 3, colsum_begin(cx, cs));
     return cx.st;
 }

@@ -335,7 +335,7 @@ ecospa_status_t validate_pair(const ecospa_pair_t& p, bool need_grads) {
     if (p.rope != ECOSPA_ROPE_NONE && p.rope != ECOSPA_ROPE_INTERLEAVED && p.rope != ECOSPA_ROPE_HALF) return ECOSPA_ERR_INVALID;
     if (p.rope != ECOSPA_ROPE_NONE && (p.kind != ECOSPA_PAIR_PLAIN || (p.seg_len & 1))) return ECOSPA_ERR_INVALID;
     const int64_t D = static_cast<int64_t>(p.n_seg) * p.seg_len;
-    if (D > (1 << 24)) return ECOSPA_ERR_UNSUPPORTED;
+    if (D > (1 << 22)) return ECOSPA_ERR_UNSUPPORTED;   // tile counts along D are 16-bit
     ecospa_status_t st;
     if ((st = validate_mat(p.w1, D, -1, -1, -1)) != ECOSPA_OK) return st;
     if ((st = validate_mat(p.w2, D, p.w1.dtype, -1, -1)) != ECOSPA_OK) return st;

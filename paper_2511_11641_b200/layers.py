@@ -41,32 +41,3 @@ def ffn_fwd_bwd(X, dY, act: int, w1c, w2c, k: int, buf: Dict[str, torch.Tensor],
     B.ecospa_coupled_ffn_bwd(X, act, w1c, w2c, k, buf["H"], buf["A"], dY, buf["dX"], buf["dW1"], buf["dW2"],
                              w1b_c=w1bc, Hb=buf.get("Hb"), dW1b_c=buf.get("dW1b"), db1_c=buf.get("db1"),
                              db2=buf["db2"], workspace=buf["ws"], **layouts)
-
-
-def smoke_layer_check(wl, w1c, w1bc, w2c, k: int, dev) -> None:
-    """One tiny compacted SwiGLU FFN forward/backward on the GPU against the fp64 oracle."""
-    import numpy as np
-    from oracle import oracle as O
-    from . import workloads as WL
-
-    acts = WL.activations(wl, 0, kinds=["x", "dy"])
-    X, dY = acts["x"].to(dev), acts["dy"].to(dev)
-    T = X.shape[0]
-    buf = ffn_buffers(T, wl.d_m, k, B.ACT_SWIGLU, torch.bfloat16, dev)
-    ffn_fwd_bwd(X, dY, B.ACT_SWIGLU, w1c, w2c, k, buf, w1bc=w1bc)
-    B.ecospa_device_status()
-    ref_f = O.ffn_fwd(acts["x"], O.ACT_SWIGLU, w1c.cpu(), w2c.cpu(), O.SHARED_COLS, O.SHARED_ROWS, k, W1b=w1bc.cpu())
-    ref_b = O.ffn_bwd(acts["x"], O.ACT_SWIGLU, w1c.cpu(), w2c.cpu(), O.SHARED_COLS, O.SHARED_ROWS, k, acts["dy"],
-                      W1b=w1bc.cpu())
-
-    def rel(a, b):
-        return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30))
-
-    errs = {
-        "Y": rel(buf["Y"].double().cpu().numpy(), ref_f["Y"]),
-        "dX": rel(buf["dX"].double().cpu().numpy(), ref_b["dX"]),
-        "dW1": rel(buf["dW1"][:, :k].double().cpu().numpy(), ref_b["dW1"]),
-        "dW2": rel(buf["dW2"].double().cpu().numpy(), ref_b["dW2"].T),
-    }
-    bad = {n: e for n, e in errs.items() if not e <= 2e-2}
-    assert not bad, f"layer mismatch vs oracle: {bad}"

@@ -172,3 +172,138 @@ def test_pack_kept_rejects_bad_arguments_without_launching(lib):
     assert fn(slots, a(z), a(z), a(z), a(z), 0, out, None) == 1
     assert fn(slots, a(neg), a(z), a(z), a(z), 1, out, None) == 1
     assert fn(slots, a(z), a(z), a(neg), a(z), 1, out, None) == 1
+
+
+# ---------------------------------------------------------------------------------------------
+# step 4 (compacted-pair forward/backward): everything below is rejected on the host, before any
+# CUDA call, so it runs without a GPU.  Pointers are fake addresses that are never dereferenced.
+# ---------------------------------------------------------------------------------------------
+
+def _w(ptr, layout=B.SHARED_COLS, d_m=64, ld=64, dtype=B.BF16):
+    return B.Mat(ptr, dtype, layout, d_m, ld)
+
+
+def test_layer_calls_reject_bad_arguments_without_launching(lib):
+    f = B._fn
+    a = C.addressof
+    X, Q, K, V, ws = 0x10000, 0x20000, 0x30000, 0x40000, 0x50000
+    T, d_m, n = 128, 64, 32
+    wq, wk, wv = _w(0x1000), _w(0x2000), _w(0x3000)
+    wo = _w(0x4000, layout=B.SHARED_ROWS)
+    big = 1 << 24
+    qk_fwd = f("ecospa_coupled_qk_fwd")
+    # null weight descriptor / null output / null weight pointer
+    assert qk_fwd(X, d_m, T, d_m, None, a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(wk), n, None, None, None, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, T, d_m, a(_w(None)), a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    # K requested (weight given) without an output for it; sizes < 1; weight of another width or dtype
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(wk), n, None, None, Q, None, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, 0, d_m, a(wq), a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(wk), 0, None, None, Q, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, T, d_m, a(_w(0x1000, d_m=128)), a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(_w(0x2000, dtype=B.F32)), n, None, None, Q, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, T, d_m, a(_w(0x1000, ld=16)), a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, d_m, T, d_m, a(_w(0x1000, layout=7)), a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    # X missing; X narrower than d_m
+    assert qk_fwd(None, d_m, T, d_m, a(wq), a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    assert qk_fwd(X, 32, T, d_m, a(wq), a(wk), n, None, None, Q, K, 32, ws, big, None) == 1
+    # alignment: workspace, output pointer, output pitch, X pitch, weight pointer, weight pitch, bias pointer
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(wk), n, None, None, Q, K, 32, ws + 4, big, None) == 2
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(wk), n, None, None, Q + 2, K, 32, ws, big, None) == 2
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(wk), n, None, None, Q, K, 36, ws, big, None) == 2
+    assert qk_fwd(X, d_m + 4, T, d_m, a(wq), a(wk), n, None, None, Q, K, 32, ws, big, None) == 2
+    assert qk_fwd(X, d_m, T, d_m, a(_w(0x1008)), a(wk), n, None, None, Q, K, 32, ws, big, None) == 2
+    assert qk_fwd(X, d_m, T, d_m, a(_w(0x1000, ld=68)), a(wk), n, None, None, Q, K, 32, ws, big, None) == 2
+    assert qk_fwd(X, d_m, T, d_m, a(wq), a(wk), n, 0x7002, None, Q, K, 32, ws, big, None) == 2
+    # the other forward calls share the checks
+    assert f("ecospa_coupled_vo_fwd_v")(X, d_m, T, d_m, None, n, None, V, 32, ws, big, None) == 1
+    assert f("ecospa_coupled_vo_fwd_o")(X, 32, T, d_m, a(wo), n, None, None, d_m, ws, big, None) == 1
+    assert f("ecospa_coupled_vo_fwd_o")(X, 32, T, d_m, a(_w(0x4000, layout=B.SHARED_ROWS, ld=32)), n, None, Q, d_m, ws, big, None) == 1
+    assert f("ecospa_coupled_qkv_fwd")(X, d_m, T, d_m, a(wq), a(wk), None, n, n, None, None, None, Q, K, V, 32, 32, ws, big,
+                                       None) == 1
+    assert f("ecospa_coupled_qkv_fwd")(X, d_m, T, d_m, a(wq), a(wk), a(wv), n, n, None, None, None, Q, K, V, 32, 36, ws, big,
+                                       None) == 2
+
+    # backward calls: missing gradient inputs / outputs, short or missing workspace
+    dQ, dK, dX, dWq, dWk, db = 0x60000, 0x70000, 0x80000, 0x90000, 0xA0000, 0xB0000
+    qk_bwd = f("ecospa_coupled_qk_bwd")
+    assert qk_bwd(X, d_m, T, d_m, a(wq), a(wk), n, None, dK, 32, dX, d_m, 0, dWq, dWk, 32, None, None, ws, big, None) == 1
+    assert qk_bwd(X, d_m, T, d_m, a(wq), a(wk), n, dQ, dK, 32, None, d_m, 0, dWq, dWk, 32, None, None, ws, big, None) == 1
+    assert qk_bwd(X, d_m, T, d_m, a(wq), a(wk), n, dQ, dK, 32, dX, d_m, 0, dWq, None, 32, None, None, ws, big, None) == 1
+    # bias gradients need column-sum scratch: no workspace, or one that is too small -> nothing is launched
+    assert qk_bwd(X, d_m, T, d_m, a(wq), a(wk), n, dQ, dK, 32, dX, d_m, 0, dWq, dWk, 32, db, db + 256, None, 0, None) == 6
+    assert qk_bwd(X, d_m, T, d_m, a(wq), a(wk), n, dQ, dK, 32, dX, d_m, 0, dWq, dWk, 32, db, db + 256, ws, 64, None) == 6
+    need = lib.ecospa_proj_workspace_bytes(T, d_m, n, B.BF16)
+    assert need > 0
+    # misaligned gradient pitch
+    assert qk_bwd(X, d_m, T, d_m, a(wq), a(wk), n, dQ, dK, 36, dX, d_m, 0, dWq, dWk, 32, None, None, ws, big, None) == 2
+    vo_bwd_o = f("ecospa_coupled_vo_bwd_o")
+    assert vo_bwd_o(None, 32, T, d_m, a(wo), n, dQ, d_m, dK, 32, dWq, d_m, None, ws, big, None) == 1
+    assert vo_bwd_o(X, 32, T, d_m, a(wo), n, dQ, d_m, dK, 32, dWq, d_m, db, None, 0, None) == 6
+    qkv_bwd = f("ecospa_coupled_qkv_bwd")
+    assert qkv_bwd(X, d_m, T, d_m, a(wq), a(wk), a(wv), n, n, dQ, dK, None, 32, 32, dX, d_m, 1, dWq, dWk, dWk + 0x8000, 32,
+                   32, None, None, None, ws, big, None) == 1
+    assert qkv_bwd(X, d_m, T, d_m, a(wq), a(wk), a(wv), n, n, dQ, dK, dK + 0x8000, 32, 32, dX, d_m, 1, dWq, dWk,
+                   dWk + 0x8000, 32, 32, db, db + 256, db + 512, ws, 128, None) == 6
+
+    # fp32 models stage their operands in the workspace: without one the call stops before the first launch
+    wq32 = _w(0x1000, dtype=B.F32)
+    assert qk_fwd(X, d_m, T, d_m, a(wq32), None, n, None, None, Q, None, 32, None, 0, None) == 6
+    assert lib.ecospa_proj_workspace_bytes(T, d_m, n, B.F32) > need
+
+
+def test_ffn_calls_reject_bad_arguments_without_launching(lib):
+    f = B._fn
+    a = C.addressof
+    X, Y, H, Hb, A, ws = 0x10000, 0x20000, 0x30000, 0x40000, 0x50000, 0x60000
+    T, d_m, k = 128, 64, 48
+    w1, w1b = _w(0x1000), _w(0x2000)
+    w2 = _w(0x3000, layout=B.SHARED_ROWS)
+    big = 1 << 24
+    fwd = f("ecospa_coupled_ffn_fwd")
+    ok_args = lambda act, w1b_, Hb_: (X, d_m, T, d_m, act, a(w1), w1b_, a(w2), k, None, None, Y, d_m, H, Hb_, A, 48, ws, big, None)
+    # unknown activation; ACT_NONE is not an FFN; SwiGLU without the up matrix or without its saved tensor
+    assert fwd(*ok_args(9, None, None)) == 1
+    assert fwd(*ok_args(B.ACT_NONE, None, None)) == 1
+    assert fwd(*ok_args(B.ACT_SWIGLU, None, Hb)) == 1
+    assert fwd(*ok_args(B.ACT_SWIGLU, a(w1b), None)) == 1
+    # saved-activation pitch: smaller than k, or not a multiple of 16 bytes
+    assert fwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, None, None, Y, d_m, H, None, A, 40, ws, big, None) == 1
+    assert fwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, None, None, Y, d_m, H, None, A, 50, ws, big, None) == 2
+    # null outputs
+    assert fwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, None, None, None, d_m, H, None, A, 48, ws, big, None) == 1
+    assert fwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, None, None, Y, d_m, None, None, A, 48, ws, big, None) == 1
+    # misaligned output
+    assert fwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, None, None, Y + 8, d_m, H, None, A, 48, ws, big, None) == 2
+    bwd = f("ecospa_coupled_ffn_bwd")
+    dY, dX, dW1, dW2, db = 0x70000, 0x80000, 0x90000, 0xA0000, 0xB0000
+    # the backward pass always needs scratch for dH: none, or too little
+    assert bwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, H, None, A, 48, dY, d_m, dX, d_m, dW1, None, 48, dW2,
+               d_m, None, None, None, 0, None) == 6
+    assert bwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, H, None, A, 48, dY, d_m, dX, d_m, dW1, None, 48, dW2,
+               d_m, db, db + 256, ws, 1024, None) == 6
+    assert bwd(X, d_m, T, d_m, B.ACT_SWIGLU, a(w1), a(w1b), a(w2), k, H, Hb, A, 48, dY, d_m, dX, d_m, dW1, None, 48, dW2,
+               d_m, None, None, ws, big, None) == 1          # SwiGLU without an output for dW_up
+    assert bwd(X, d_m, T, d_m, B.ACT_GELU_ERF, a(w1), None, a(w2), k, H, None, A, 48, None, d_m, dX, d_m, dW1, None, 48, dW2,
+               d_m, None, None, ws, big, None) == 1
+    assert lib.ecospa_ffn_workspace_bytes(T, d_m, k, B.ACT_SWIGLU, B.BF16) > lib.ecospa_ffn_workspace_bytes(
+        T, d_m, k, B.ACT_GELU_ERF, B.BF16) > 0
+
+
+def test_wait_limit_setter(lib):
+    fn = lib.ecospa_set_device_wait_limit_ns
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_uint64]
+    assert fn(0) == 1
+    assert fn(2_000_000_000) == 0
+
+
+def test_shared_dimension_limit(lib):
+    null = B.Mat(None, 0, 0, 0, 0)
+    D = (1 << 22) + 64
+    p = B.Pair(B.PAIR_PLAIN, 1, D, 0, _fake_mat(0x1000, dtype=B.F32, other=4, ld=D), null,
+               _fake_mat(0x40000000, dtype=B.F32, layout=B.SHARED_ROWS, other=4, ld=4), null, null, null)
+    assert lib.ecospa_score_pairs(C.addressof((B.Pair * 1)(p)), 1, 1.0, C.c_void_p(0x3000), None, None,
+                                  C.c_void_p(0x4000), 1 << 30, None) == 3
+    g = B.Gather(_fake_mat(0x10000, other=2, ld=D), _fake_mat(0x80000000, other=2, ld=64), 0x9000, 32, D)
+    assert lib.ecospa_compact_tensors(C.addressof((B.Gather * 1)(g)), 1, None) == 3

@@ -21,9 +21,24 @@ DEV = "cuda"
 TOL = 2e-2
 
 
-def rel(got, ref):
+def rel(got, ref, th=32, tw=64):
+    """Relative Frobenius error of the whole tensor, and for 2-D outputs also of every th x tw tile (the unit one
+    epilogue warp stores), so that a single wrong tile cannot hide in the norm of a large tensor; returns the larger.
+    A tile's denominator is floored at half of what a tile of average magnitude would have (edge tiles with a few
+    columns, tiles that happen to be small)."""
     got = got.double().cpu().numpy() if isinstance(got, torch.Tensor) else got
-    return float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
+    whole = float(np.linalg.norm(got - ref) / max(np.linalg.norm(ref), 1e-300))
+    if got.ndim != 2:
+        return whole
+    R, Cn = ref.shape
+    rp, cp = -(-R // th) * th, -(-Cn // tw) * tw
+    d2 = np.zeros((rp, cp)); d2[:R, :Cn] = (got - ref) ** 2
+    r2 = np.zeros((rp, cp)); r2[:R, :Cn] = ref ** 2
+    num = np.sqrt(d2.reshape(rp // th, th, cp // tw, tw).sum(axis=(1, 3)))
+    den = np.sqrt(r2.reshape(rp // th, th, cp // tw, tw).sum(axis=(1, 3)))
+    floor = 0.5 * np.sqrt(r2.sum() / max(R * Cn, 1) * th * tw)
+    tiles = float((num / np.maximum(den, max(floor, 1e-300))).max())
+    return max(whole, tiles)
 
 
 def check(errs):

@@ -360,3 +360,98 @@ def test_fp32_optimizer_moments_follow_bf16_weights():
             ref = O.compact(allt[nm], layout, kept, ld_out=o.shape[1])
             view = torch.int16 if allt[nm].element_size() == 2 else torch.int32
             assert torch.equal(o.cpu().view(view), ref.view(view)), nm
+
+
+# ---------------------------------------------------------------------------
+# heavy-tailed single layer (LLaMA-7B shape) and the re-estimation sweep (LLaMA-1B shape)
+# ---------------------------------------------------------------------------
+
+_LAYOUTS = {"wq": 0, "wk": 0, "wv": 0, "wo": 1, "w1": 0, "w1b": 0, "w2": 1,
+            "gq": 0, "gk": 0, "gv": 0, "go": 1, "g1": 0, "g1b": 0, "g2": 1, "bq": 0, "bk": 0, "bv": 0, "b1": 0}
+_GROUP_OF = {"wq": 0, "wk": 0, "gq": 0, "gk": 0, "bq": 0, "bk": 0, "wv": 1, "wo": 1, "gv": 1, "go": 1, "bv": 1,
+             "w1": 2, "w1b": 2, "w2": 2, "g1": 2, "g1b": 2, "g2": 2, "b1": 2}
+
+
+def select_and_compact_vs_oracle(wl, allt, w_d, ups, sparsity, names):
+    """Selection on the GPU's own fp32 scores vs the oracle's ranking of the same vector (bit-exact), then
+    compaction of `names` by the library vs the oracle's byte copy with that kept list."""
+    plan = WL.kept_plan(wl, sparsity)
+    n_seg = [wl.n_heads, wl.n_heads, 1]; seg_len = [wl.d_h, wl.d_h, wl.d_ffn]
+    k = plan["qk"] + plan["vo"] + plan["ffn"]
+    ks = [sum(plan["qk"]), sum(plan["vo"]), sum(plan["ffn"])]
+    kept_d = torch.empty(sum(k), dtype=torch.int32, device=DEV)
+    B.ecospa_select_aligned_topk(ups, n_seg, seg_len, k, kept_d)
+    kept = kept_d.cpu().numpy()
+    np.testing.assert_array_equal(kept, oracle_select(ups.cpu().numpy(), n_seg, seg_len, k))
+    if not names:
+        return kept
+    starts = [0, ks[0], ks[0] + ks[1]]
+    dims = [wl.n_heads * wl.d_h, wl.n_heads * wl.d_h, wl.d_ffn]
+    jobs, outs = [], {}
+    for nm in names:
+        gi = _GROUP_OF[nm]
+        o = BL.alloc_compacted(w_d[nm], _LAYOUTS[nm], ks[gi]).fill_(7)
+        outs[nm] = o
+        jobs.append(B.gather(w_d[nm], o, _LAYOUTS[nm], kept_d[starts[gi]: starts[gi] + ks[gi]], ks[gi], dims[gi]))
+    B.ecospa_compact_tensors(jobs)
+    torch.cuda.synchronize()
+    for nm, o in outs.items():
+        gi = _GROUP_OF[nm]
+        kk = kept[starts[gi]: starts[gi] + ks[gi]]
+        ref = O.compact(allt[nm], _LAYOUTS[nm], kk, ld_out=o.shape[1] if o.dim() == 2 else o.numel())
+        assert torch.equal(o.cpu().view(torch.int16), ref.view(torch.int16)), (nm, sparsity)
+    return kept
+
+
+def test_heavy_tailed_layer_scores_selection_compaction():
+    """The LLaMA-7B-shaped layer whose shared-index vectors carry a x10 tail: scores and pair-level importance
+    against the oracle, then kept sets and compacted tensors at 25 / 50 / 75 %."""
+    wl = WL.WORKLOADS["llama7b_layer"]
+    w = WL.layer_weights(wl, 0); g = WL.layer_grads(wl, 0)
+    raw_o, ups_o, fis_o = oracle_block_scores(w, g, wl, wl.tokens)
+    allt = dict(w); allt.update(g)
+    w_d = to_dev(allt)
+    _, ups, raw, fis = gpu_block_scores(w_d, w_d, wl, wl.tokens)
+    sb = seg_bounds_of(wl)
+    assert_close_per_segment(ups, ups_o, sb)
+    assert_close_per_segment(raw, raw_o, sb)
+    np.testing.assert_allclose(fis.double().cpu().numpy(), fis_o, rtol=REL)
+    # the tail is what decides: the scores of a head span more than an order of magnitude
+    head0 = ups_o[: wl.d_h]
+    assert head0.max() > 10 * np.median(head0)
+    for s in (0.25, 0.5, 0.75):
+        select_and_compact_vs_oracle(wl, allt, w_d, ups, s, ["wq", "wk", "wv", "wo", "w1", "w1b", "w2"])
+
+
+def test_reestimation_sweep_one_layer():
+    """Re-estimation as Algorithm 1 repeats it: weights fixed, gradients redrawn per step.  One LLaMA-1B-shaped layer,
+    three of the ten gradient draws: importance vs the oracle for every draw; kept sets at all nine sparsities
+    (10 ... 90 %) bit-exact on the same fp32 scores; compaction of weights and of the redrawn gradients byte-exact
+    at 10 / 50 / 90 %."""
+    wl = WL.WORKLOADS["llama1b"]
+    layer = 5
+    w = WL.layer_weights(wl, layer)
+    w_d = to_dev(w)
+    _, ups_o, _ = oracle_block_scores(w, None, wl, wl.tokens)
+    ups_first = None
+    for seed in (0, 4, 9):
+        g = WL.layer_grads(wl, layer, step=seed)
+        g_d = to_dev(g)
+        _, ups, _, fis = gpu_block_scores(w_d, g_d, wl, wl.tokens)
+        fis_o = np.concatenate([
+            O.fisher_pair(g["gq"], g["gk"], 0, 0, wl.n_heads, wl.d_h, wl.tokens),
+            O.fisher_pair(g["gv"], g["go"], 0, 1, wl.n_heads, wl.d_h, wl.tokens),
+            O.fisher_pair(g["g1"], g["g2"], 0, 1, 1, wl.d_ffn, wl.tokens, g1b=g["g1b"])])
+        np.testing.assert_allclose(fis.double().cpu().numpy(), fis_o, rtol=REL)
+        assert_close_per_segment(ups, ups_o, seg_bounds_of(wl))
+        if ups_first is None:
+            ups_first = ups.clone()
+        else:
+            assert torch.equal(ups, ups_first)          # the scores do not depend on the gradients
+        allt = dict(w); allt.update(g)
+        d_all = dict(w_d); d_all.update(g_d)
+        for s10 in range(1, 10):
+            s = s10 / 10.0
+            names = ["wq", "wk", "wo", "w1", "w1b", "w2", "gq", "go", "g1", "g1b", "g2"] if s10 in (1, 5, 9) else []
+            kept = select_and_compact_vs_oracle(wl, allt, d_all, ups, s, names)
+            assert len(kept) == 2 * wl.n_heads * WL.kept_count(wl.d_h, s) + WL.kept_count(wl.d_ffn, s)
