@@ -1,4 +1,4 @@
-"""Benchmark of the coupled-sparsity hot path on a GPT-2-Medium-shaped model (or another workload).
+"""Benchmark of the coupled-sparsity hot path on a LLaMA-1B-shaped model (or another workload).
 
 One step = one pass of the whole hot path over every layer of the model:
   score (+ Fisher) of all coupled pairs -> aligned top-k -> compaction of weights, biases and
@@ -27,10 +27,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (read + write) per gemm_kernel launch, averaged over the eight GEMM launches of a gpt2m layer:
-# `dram__bytes_read.sum + dram__bytes_write.sum` of one ncu capture of this build (profiles/gemm_kernel_gpt2m_layer.md).
-# Per-launch traffic does not depend on the number of layers captured.  Other workloads: not captured (None).
-NCU_GEMM_TRAFFIC_BYTES = {"gpt2m": 45.3e6}
+# DRAM bytes (read + write) per gemm_kernel launch, averaged over the eight GEMM launches of a layer:
+# `dram__bytes_read.sum + dram__bytes_write.sum` of one ncu capture of this build per workload (one layer captured;
+# per-launch traffic does not depend on the number of layers).  Workloads without a capture: None.
+NCU_GEMM_TRAFFIC_BYTES = {"gpt2m": 45.3e6, "llama1b": 213.7e6}
+# DRAM bytes per step of sumsq_kernel + gather_kernel on 8 gpt2m layers under ncu (grow in proportion to the layers)
+NCU_SPARSIFY_TRAFFIC_BYTES_PER_LAYER = {"gpt2m": 889.3e6 / 8}
 
 METRIC = "compacted-pair fwd/bwd TFLOP/s over the whole coupled-sparsity step (score+select+compact GB/s alongside)"
 
@@ -150,6 +152,7 @@ class Model:
             self.w.append(w); self.g.append(g)
             self.pairs += BL.block_pairs(w, wl.n_heads, wl.d_h, wl.d_ffn, g, layout_in=lin, layout_out=lout)
         plan = WL.kept_plan(wl, sparsity)
+        self.plan = plan
         self.n_attn, self.k_ffn = sum(plan["qk"]), plan["ffn"][0]
         self.k_per_seg = (plan["qk"] + plan["vo"] + plan["ffn"]) * wl.n_layers
         self.n_seg = [wl.n_heads, wl.n_heads, 1] * wl.n_layers
@@ -169,6 +172,7 @@ class Model:
                   (["w1", "w1b", "w2", "b1"], ["g1", "g1b", "g2"], self.k_ffn, wl.d_ffn)]
         layout = {"wq": lin, "wk": lin, "wv": lin, "wo": lout, "w1": lin, "w1b": lin, "w2": lout, "bq": 0, "bk": 0, "bv": 0,
                   "b1": 0, "gq": lin, "gk": lin, "gv": lin, "go": lout, "g1": lin, "g1b": lin, "g2": lout}
+        self.layout = layout
         for l in range(wl.n_layers):
             c = {}
             for wn, gn, nk, D in groups:
@@ -209,24 +213,28 @@ class Model:
         B.ecospa_select_aligned_topk(self.ups, self.n_seg, self.seg_len, self.k_per_seg, self.kept)
         B.ecospa_compact_tensors(self.jobs)
 
-    def layers(self):
+    def layer(self, l: int):
+        """Forward and backward of the compacted QK / VO / FFN pairs of layer l."""
         B, o, n, k = self.B, self.o, self.n_attn, self.k_ffn
         bias = self.wl.bias
+        c, a = self.c[l], self.acts[l % len(self.acts)]
+        # forward: Q, K, V in one launch; (attention core is the caller's); output projection; FFN
+        B.ecospa_coupled_qkv_fwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, o["Q"], o["K"], o["V"], bq_c=c.get("bq"),
+                                 bk_c=c.get("bk"), bv_c=c.get("bv"), workspace=self.proj_ws, **self.lay)
+        B.ecospa_coupled_vo_fwd_o(a["ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws, **self.lay)
+        # FFN forward + backward
+        self.L.ffn_fwd_bwd(a["x"], a["dy"], self.act, c["w1"], c["w2"], k, self.ffn, w1bc=c.get("w1b"),
+                           b1c=c.get("b1"), b2=self.w[l].get("b2"), **self.lay)
+        # backward: what dOut gives (dCtx, dW_O), then what dQ, dK, dV give (dW_Q, dW_K, dW_V, dX)
+        B.ecospa_coupled_vo_bwd_o(a["ctx"], c["wo"], n, a["dout"], o["dCtx"], o["dWo"], o["dbo"] if bias else None,
+                                  workspace=self.proj_ws, **self.lay)
+        B.ecospa_coupled_qkv_bwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, a["dq"], a["dk"], a["dv"], o["dX"], o["dWq"],
+                                 o["dWk"], o["dWv"], o["dbq"] if bias else None, o["dbk"] if bias else None,
+                                 o["dbv"] if bias else None, accumulate_dX=True, workspace=self.proj_ws, **self.lay)
+
+    def layers(self):
         for l in range(self.wl.n_layers):
-            c, a = self.c[l], self.acts[l % len(self.acts)]
-            # forward: Q, K, V in one launch; (attention core is the caller's); output projection; FFN
-            B.ecospa_coupled_qkv_fwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, o["Q"], o["K"], o["V"], bq_c=c.get("bq"),
-                                     bk_c=c.get("bk"), bv_c=c.get("bv"), workspace=self.proj_ws, **self.lay)
-            B.ecospa_coupled_vo_fwd_o(a["ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws, **self.lay)
-            # FFN forward + backward
-            self.L.ffn_fwd_bwd(a["x"], a["dy"], self.act, c["w1"], c["w2"], k, self.ffn, w1bc=c.get("w1b"),
-                               b1c=c.get("b1"), b2=self.w[l].get("b2"), **self.lay)
-            # backward: what dOut gives (dCtx, dW_O), then what dQ, dK, dV give (dW_Q, dW_K, dW_V, dX)
-            B.ecospa_coupled_vo_bwd_o(a["ctx"], c["wo"], n, a["dout"], o["dCtx"], o["dWo"], o["dbo"] if bias else None,
-                                      workspace=self.proj_ws, **self.lay)
-            B.ecospa_coupled_qkv_bwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, a["dq"], a["dk"], a["dv"], o["dX"], o["dWq"],
-                                     o["dWk"], o["dWv"], o["dbq"] if bias else None, o["dbk"] if bias else None,
-                                     o["dbv"] if bias else None, accumulate_dX=True, workspace=self.proj_ws, **self.lay)
+            self.layer(l)
 
     def host_copies(self):
         """Pinned host mirrors of every input of a step (weights, gradients, activations)."""
@@ -256,7 +264,278 @@ def job_throughput(world: int, units_per_rank: float, ms: float) -> float:
     return world * units_per_rank / ms
 
 
+def tensor_peak(peaks, timed_ms: float, clocks) -> dict:
+    """Which measured cuBLAS bf16 figure a tensor-bound number is compared with: the burst figure when the timed
+    region is short (under about 2 s) or the SM clock stayed at its maximum, the sustained (power-capped) one
+    otherwise."""
+    sm, mx = (clocks or {}).get("sm_mhz"), (clocks or {}).get("sm_max_mhz")
+    at_max = bool(sm and mx and sm >= 0.97 * mx)
+    burst = timed_ms < 2000.0 or at_max
+    return {"peak": peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"],
+            "which": "burst" if burst else "sustained"}
+
+
+def measure_step(m, args, world, rank, local, steps: int, graph: bool = True):
+    """Times `steps` passes of the whole hot path of model `m` (device-resident inputs): returns per-step
+    milliseconds of the whole step, the sparsify phase and the layer phase (CUDA events on the launching stream),
+    the clock record of the timed region, and the launches of one step."""
+    import torch
+    import torch.distributed as dist
+    B = m.B
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(3, args.warmup)):
+        m.sparsify(); m.layers()
+    B.ecospa_device_status()
+    # The calls are stateless and asynchronous, so a step can be captured once into CUDA graphs and
+    # replayed: the launches of a step then cost no host time.  --no-graph issues them one by one.
+    l0 = B.ecospa_launch_count()
+    if not graph:
+        sparsify, layers = m.sparsify, m.layers
+        m.sparsify(); m.layers()
+    else:
+        g_sp, g_ly = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g_sp):
+            m.sparsify()
+        with torch.cuda.graph(g_ly):
+            m.layers()
+        sparsify, layers = g_sp.replay, g_ly.replay
+        m._graphs = (g_sp, g_ly)
+    launches = B.ecospa_launch_count() - l0
+    for _ in range(2):
+        sparsify(); layers()
+    B.ecospa_device_status()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    marks = []
+    barrier()
+    t_all0, t_all1 = ev(), ev()
+    t_all0.record()
+    for _ in range(steps):
+        e0, e1, e2 = ev(), ev(), ev()
+        e0.record(); sparsify(); e1.record(); layers(); e2.record()
+        marks.append((e0, e1, e2))
+    t_all1.record()
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    B.ecospa_device_status()
+    ms_total = t_all0.elapsed_time(t_all1)
+    ms_sp = sum(a.elapsed_time(b) for a, b, _ in marks) / steps
+    ms_gemm = sum(b.elapsed_time(c) for _, b, c in marks) / steps
+    return {"ms_step": ms_total / steps, "ms_sp": ms_sp, "ms_gemm": ms_gemm, "clocks": clocks, "launches": int(launches),
+            "replay": (sparsify, layers), "timed_ms": ms_total}
+
+
+def phase_report(wl, m, r, peaks, sparsity, transposed=False):
+    """The figures of one measured workload: both phases against the measured and the nominal peaks."""
+    flops = step_flops(wl, m.n_attn, m.k_ffn)
+    sbytes = sparsify_bytes(wl, 1.0 - sparsity, transposed=transposed)
+    tf = flops / r["ms_gemm"] / 1e9
+    gbs = sbytes / r["ms_sp"] / 1e6
+    tp = tensor_peak(peaks, r["timed_ms"], r["clocks"])
+    sm = (r["clocks"] or {}).get("sm_mhz")
+    return {
+        "workload": wl.name, "sparsity": sparsity, "ms_per_step": r["ms_step"],
+        "gemm_ms": r["ms_gemm"], "gemm_TFLOP/s": tf, "gemm_flops_per_step": flops,
+        "gemm_frac_of_measured_burst": tf / peaks["bf16_tflops"],
+        "gemm_frac_of_measured_sustained": tf / peaks["bf16_tflops_sustained"],
+        "gemm_frac_of_nominal_2250": tf / 2250.0, "gemm_denominator_for_this_run": tp["which"],
+        "gemm_ms_x_sm_mhz": (r["ms_gemm"] * sm) if sm else None,
+        "sparsify_ms": r["ms_sp"], "sparsify_GB/s": gbs, "sparsify_bytes_per_step": sbytes,
+        "sparsify_byte_accounting": "per tensor: every weight and gradient read once for the scores; compaction reads a "
+                                    "shared-cols tensor in full and a shared-rows tensor at the kept fraction, writes the kept fraction",
+        "sparsify_GB/s_if_every_tensor_counted_as_shared_rows": (2.0 + 4.0 * (1.0 - sparsity)) * WL_model_bytes(wl) / r["ms_sp"] / 1e6,
+        "sparsify_frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "sparsify_frac_of_nominal_8TBs": gbs / 8000.0,
+        "clocks": r["clocks"], "gpu_launches": r["launches"],
+    }
+
+
+def WL_model_bytes(wl):
+    from paper_2511_11641_b200 import workloads as WL
+    return WL.model_bytes(wl)
+
+
+# ---------------------------------------------------------------------------------------------
+# the re-estimation sweep: score + select + compact over all layers at sparsity 10 ... 90 %, gradients redrawn
+# per step with seeds 0 ... 9 (the per-epoch re-estimation of Algorithm 1); GB/s per sparsity, median over seeds
+# ---------------------------------------------------------------------------------------------
+
+def reestimation_sweep(wl, dev, local, rank, seeds=range(10), sparsities=tuple(s / 10 for s in range(1, 10)), reps=3):
+    import torch
+    from paper_2511_11641_b200 import binding as B, block as BL, workloads as WL
+    w, g, pairs = [], [], []
+    for l in range(wl.n_layers):
+        w.append(WL.layer_weights(wl, l, device=dev))
+        g.append(WL.layer_grads(wl, l, device=dev))
+        pairs += BL.block_pairs(w[l], wl.n_heads, wl.d_h, wl.d_ffn, g[l])
+    D_layer = 2 * wl.n_heads * wl.d_h + wl.d_ffn
+    ups = torch.empty(D_layer * wl.n_layers, dtype=torch.float32, device=dev)
+    fis = torch.empty((2 * wl.n_heads + 1) * wl.n_layers, dtype=torch.float32, device=dev)
+    score_ws = torch.empty(B.ecospa_score_workspace_bytes(pairs), dtype=torch.uint8, device=dev)
+    n_seg = [wl.n_heads, wl.n_heads, 1] * wl.n_layers
+    seg_len = [wl.d_h, wl.d_h, wl.d_ffn] * wl.n_layers
+    D_attn = wl.n_heads * wl.d_h
+    layout = {"wq": 0, "wk": 0, "wv": 0, "wo": 1, "w1": 0, "w1b": 0, "w2": 1, "gq": 0, "gk": 0, "gv": 0, "go": 1, "g1": 0,
+              "g1b": 0, "g2": 1}
+    setups = {}
+    for s in sparsities:
+        plan = WL.kept_plan(wl, s)
+        n_attn, k_ffn = sum(plan["qk"]), plan["ffn"][0]
+        k_per_seg = (plan["qk"] + plan["vo"] + plan["ffn"]) * wl.n_layers
+        kept = torch.empty(sum(k_per_seg), dtype=torch.int32, device=dev)
+        jobs, outs, off = [], [], 0
+        for l in range(wl.n_layers):
+            for names, nk, D in ((("wq", "wk", "gq", "gk"), n_attn, D_attn), (("wv", "wo", "gv", "go"), n_attn, D_attn),
+                                 (("w1", "w1b", "w2", "g1", "g1b", "g2"), k_ffn, wl.d_ffn)):
+                kd = kept[off:off + nk]
+                for nm in names:
+                    src = w[l].get(nm) if nm in w[l] else g[l].get(nm)
+                    if src is None:
+                        continue
+                    o = BL.alloc_compacted(src, layout[nm], nk)
+                    outs.append(o)
+                    jobs.append(B.gather(src, o, layout[nm], kd, nk, D))
+                off += nk
+        setups[s] = (k_per_seg, kept, jobs, outs)
+
+    def run(s):
+        k_per_seg, kept, jobs, _ = setups[s]
+        B.ecospa_score_pairs(pairs, float(wl.tokens), ups, None, fis, score_ws)
+        B.ecospa_select_aligned_topk(ups, n_seg, seg_len, k_per_seg, kept)
+        B.ecospa_compact_tensors(jobs)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    times = {s: [] for s in sparsities}
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for s in sparsities:
+        run(s)                                                       # warm-up of every configuration
+    torch.cuda.synchronize()
+    fisher_by_seed = []
+    for seed in seeds:
+        for l in range(wl.n_layers):                                 # redraw the gradients of this step, in place
+            fresh = WL.layer_grads(wl, l, step=seed, device=dev)
+            for nm, t in fresh.items():
+                g[l][nm].copy_(t)
+            del fresh
+        for s in sparsities:
+            run(s)
+            e0, e1 = ev(), ev()
+            e0.record()
+            for _ in range(reps):
+                run(s)
+            e1.record()
+            torch.cuda.synchronize()
+            times[s].append(e0.elapsed_time(e1) / reps)
+        fisher_by_seed.append(float(fis.double().mean().item()))
+    clocks = sampler.stop() if rank == 0 else None
+    B.ecospa_device_status()
+    peaks = measured_peaks()
+    out = {"workload": wl.name, "seeds": len(list(seeds)), "reps_per_seed": reps, "clocks": clocks, "per_sparsity": {}}
+    for s in sparsities:
+        ms = statistics.median(times[s])
+        by = sparsify_bytes(wl, 1.0 - s)
+        out["per_sparsity"][f"{s:.1f}"] = {"ms_median": ms, "GB/s": by / ms / 1e6, "bytes": by,
+                                          "frac_of_measured_hbm": by / ms / 1e6 / peaks["hbm_gbs"],
+                                          "frac_of_nominal_8TBs": by / ms / 1e6 / 8000.0}
+    # the importance values do change from draw to draw (the scores do not depend on the gradients)
+    out["mean_importance_by_seed_distinct"] = len(set(fisher_by_seed)) == len(fisher_by_seed)
+    return out
+
+
+# ---------------------------------------------------------------------------------------------
+# parity of what was timed: layer 0 of the benchmarked model against the oracle
+# ---------------------------------------------------------------------------------------------
+
+def parity_check(m, n_rows: int = 8):
+    """Re-runs the step's calls on layer 0 of the benchmarked model and compares them with the CPU oracle: scores,
+    kept sets (oracle ranking of the same fp32 scores), compacted weights (bytes), and the layer outputs and input
+    gradients on sampled token rows (relative l2 per row, fp64 oracle)."""
+    import numpy as np
+    import torch
+    from oracle import oracle as O
+    wl, B = m.wl, m.B
+    if m.transposed:
+        return {"skipped": "weights stored transposed: the tests cover this orientation"}
+    m.sparsify()
+    m.o["dX"].zero_()
+    m.layer(0)
+    B.ecospa_device_status()
+    w = {k: v.cpu() for k, v in m.w[0].items()}
+    D_attn = wl.n_heads * wl.d_h
+    D_layer = 2 * D_attn + wl.d_ffn
+    ups = m.ups[:D_layer].cpu().numpy()
+    sw = wl.ffn == "swiglu"
+    groups = [("wq", "wk", None, 0, 0, wl.n_heads, wl.d_h, m.plan["qk"]), ("wv", "wo", None, 0, 1, wl.n_heads, wl.d_h, m.plan["vo"]),
+              ("w1", "w2", "w1b" if sw else None, 0, 1, 1, wl.d_ffn, m.plan["ffn"])]
+    res = {"tolerance_rows": 2e-2, "tolerance_scores": 1e-5}
+    off_d, off_k, score_err, kept_equal, bytes_equal = 0, 0, 0.0, True, True
+    kept_all = m.kept.cpu().numpy()
+    kept_of = {}
+    for n1, n2, n1b, l1, l2, n_seg, seg_len, k in groups:
+        _, ups_o = O.score_pair(w[n1], w[n2], l1, l2, n_seg, seg_len, w1b=w.get(n1b) if n1b else None)
+        got = ups[off_d:off_d + n_seg * seg_len].astype(np.float64)
+        for sgm in range(n_seg):
+            a, b = sgm * seg_len, (sgm + 1) * seg_len
+            score_err = max(score_err, float(np.max(np.abs(got[a:b] - ups_o[a:b]) / (np.abs(ups_o[a:b]) + ups_o[a:b].max()))))
+        kept_o = O.select_topk(ups[off_d:off_d + n_seg * seg_len], n_seg, seg_len, k)
+        kept_g = kept_all[off_k:off_k + sum(k)]
+        kept_equal = kept_equal and bool(np.array_equal(kept_o, kept_g))
+        kept_of[n1] = kept_g
+        for nm, lay in ((n1, l1), (n2, l2), (n1b, l1)):
+            if nm:
+                o = m.c[0][nm]
+                ref = O.compact(w[nm], lay, kept_g, ld_out=o.shape[1])
+                bytes_equal = bytes_equal and bool(torch.equal(o.cpu().view(torch.int16), ref.view(torch.int16)))
+        off_d += n_seg * seg_len; off_k += sum(k)
+    res.update({"score_max_rel_err": score_err, "kept_sets_equal": kept_equal, "compacted_bytes_equal": bytes_equal})
+    # layer math on sampled token rows
+    r = np.random.default_rng(0)
+    rows = np.sort(r.choice(wl.tokens, size=n_rows, replace=False))
+    rt = torch.from_numpy(rows); rd = rt.to(m.dev)
+    a = m.acts[0]
+    c = {k: v.cpu() for k, v in m.c[0].items() if k in ("wq", "wk", "wv", "wo", "w1", "w1b", "w2", "bq", "bk", "bv", "b1")}
+    n, k = m.n_attn, m.k_ffn
+    X = a["x"][rd].cpu().contiguous()
+
+    def row_err(got, ref):
+        got = got.double().cpu().numpy()
+        return float(np.max(np.linalg.norm(got - ref, axis=1) / np.maximum(np.linalg.norm(ref, axis=1), 1e-300)))
+
+    errs = {}
+    for nm, out in (("q", "Q"), ("k", "K"), ("v", "V")):
+        errs[out] = row_err(m.o[out][rd][:, :n], O.proj_fwd(X, c["w" + nm], 0, n, bias=c.get("b" + nm)))
+    ctx = a["ctx"][rd].cpu()[:, :n].contiguous()
+    errs["Out"] = row_err(m.o["Out"][rd], O.outproj_fwd(ctx, c["wo"], 1, n, wl.d_m))
+    rdCtx, _, _ = O.outproj_bwd(ctx, c["wo"], 1, n, wl.d_m, a["dout"][rd].cpu().contiguous())
+    errs["dCtx"] = row_err(m.o["dCtx"][rd][:, :n], rdCtx)
+    rdX = None
+    for nm in ("q", "k", "v"):
+        rdX, _, _ = O.proj_bwd(X, c["w" + nm], 0, n, a["d" + nm][rd].cpu()[:, :n].contiguous(), dX=rdX)
+    errs["dX(attention)"] = row_err(m.o["dX"][rd], rdX)
+    act = O.ACT_SWIGLU if sw else O.ACT_GELU_ERF
+    b2 = w.get("b2")
+    rf = O.ffn_fwd(X, act, c["w1"], c["w2"], 0, 1, k, W1b=c.get("w1b"), b1=c.get("b1"), b2=b2)
+    rb = O.ffn_bwd(X, act, c["w1"], c["w2"], 0, 1, k, a["dy"][rd].cpu().contiguous(), W1b=c.get("w1b"), b1=c.get("b1"))
+    errs["Y"] = row_err(m.ffn["Y"][rd], rf["Y"])
+    errs["A"] = row_err(m.ffn["A"][rd][:, :k], rf["A"])
+    errs["dX(ffn)"] = row_err(m.ffn["dX"][rd], rb["dX"])
+    res["max_row_rel_err"] = errs
+    res["rows_sampled"] = int(n_rows)
+    res["ok"] = bool(kept_equal and bytes_equal and score_err <= 1e-5 and all(v <= 2e-2 for v in errs.values()))
+    return res
+
+
 def run_gpu(args):
+    import dataclasses
     import torch
     import torch.distributed as dist
     from paper_2511_11641_b200 import binding as B, workloads as WL
@@ -273,7 +552,6 @@ def run_gpu(args):
     dev = torch.device("cuda", local)
     wl = WL.WORKLOADS[args.workload]
     if args.layers:
-        import dataclasses
         wl = dataclasses.replace(wl, n_layers=args.layers)   # smaller model of the same shape (profiler captures)
     m = Model(wl, args.sparsity, dev, transposed=args.transposed)
     ev = lambda: torch.cuda.Event(enable_timing=True)
@@ -284,46 +562,9 @@ def run_gpu(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(3, args.warmup)):
-        m.sparsify(); m.layers()
-    B.ecospa_device_status()
-    # The calls are stateless and asynchronous, so a step can be captured once into CUDA graphs and
-    # replayed: the ~500 launches of a step then cost no host time.  --no-graph issues them one by one.
-    l0 = B.ecospa_launch_count()
-    if args.no_graph:
-        sparsify, layers = m.sparsify, m.layers
-        m.sparsify(); m.layers()
-    else:
-        g_sp, g_ly = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_sp):
-            m.sparsify()
-        with torch.cuda.graph(g_ly):
-            m.layers()
-        sparsify, layers = g_sp.replay, g_ly.replay
-    launches = B.ecospa_launch_count() - l0
-    for _ in range(2):
-        sparsify(); layers()
-    B.ecospa_device_status()
-    # ---- device-resident timing
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    marks = []
-    barrier()
-    t_all0, t_all1 = ev(), ev()
-    t_all0.record()
-    for _ in range(args.steps):
-        e0, e1, e2 = ev(), ev(), ev()
-        e0.record(); sparsify(); e1.record(); layers(); e2.record()
-        marks.append((e0, e1, e2))
-    t_all1.record()
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    B.ecospa_device_status()
-    ms_total = t_all0.elapsed_time(t_all1)
-    ms_sp = sum(a.elapsed_time(b) for a, b, _ in marks) / args.steps
-    ms_gemm = sum(b.elapsed_time(c) for _, b, c in marks) / args.steps
-    ms_step = ms_total / args.steps
+    r = measure_step(m, args, world, rank, local, args.steps, graph=not args.no_graph)
+    sparsify, layers = r["replay"]
+    ms_step, ms_sp, ms_gemm, clocks, launches = r["ms_step"], r["ms_sp"], r["ms_gemm"], r["clocks"], r["launches"]
 
     # ---- end to end: every step's inputs start in pinned host memory and its results are read back.
     # Two device-side copies of the model take turns, so the upload of step s + 1 (copy stream) runs while
@@ -380,6 +621,9 @@ def run_gpu(args):
     barrier()
     ms_e2e = e0.elapsed_time(e1) / e2e_steps
     B.ecospa_device_status()
+    del m2, host, host_in, dev_in, res_host, replay
+    if not args.no_graph:
+        del g2_sp, g2_ly
 
     ms_step, ms_sp, ms_gemm, ms_e2e = max_over_ranks([ms_step, ms_sp, ms_gemm, ms_e2e], dev)
 
@@ -387,6 +631,11 @@ def run_gpu(args):
     sbytes = sparsify_bytes(wl, 1.0 - args.sparsity, transposed=args.transposed)
     peaks = measured_peaks()
     n_gemm_launches = wl.n_layers * 8
+    tf = flops / ms_gemm / 1e9
+    tp = tensor_peak(peaks, r["timed_ms"], clocks)
+    sm_mhz = (clocks or {}).get("sm_mhz")
+    plain = not args.layers and args.sparsity == 0.5 and not args.transposed
+    sp_traffic = NCU_SPARSIFY_TRAFFIC_BYTES_PER_LAYER.get(wl.name)
     out = {
         "metric": METRIC, "value": job_throughput(world, flops, ms_step) / 1e9, "unit": "TFLOP/s", "n_gpus": world,
         "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step, "higher_is_better": True,
@@ -394,30 +643,42 @@ def run_gpu(args):
         "config": {"workload": f"{wl.name}: {wl.n_layers} layers d_model={wl.d_m} heads={wl.n_heads}x{wl.d_h} "
                                f"ffn={wl.d_ffn} {wl.ffn} T={wl.tokens} sparsity={args.sparsity}"
                                + (" weights stored transposed" if args.transposed else ""),
-                   "l2": "inputs larger than L2: 1.7 GB of weights/gradients per step, activations cycled over 4 sets",
+                   "l2": f"inputs larger than L2: {2 * WL.model_bytes(wl) / 1e9:.1f} GB of weights/gradients per step, "
+                         "activations cycled over 4 sets",
                    "replicas": world, "launch": "eager" if args.no_graph else "cuda graph replay of the captured step"},
         "phases": {
             "sparsify": {"ms": ms_sp, "GB/s": sbytes / ms_sp / 1e6, "bytes": sbytes,
+                         "byte_accounting": "per tensor (scores: every weight and gradient once; compaction: shared-cols "
+                                            "tensors read in full, shared-rows at the kept fraction, kept fraction written)",
+                         "GB/s_if_every_tensor_counted_as_shared_rows": (2.0 + 4.0 * (1.0 - args.sparsity)) * WL.model_bytes(wl) / ms_sp / 1e6,
                          "frac_of_measured_hbm": sbytes / ms_sp / 1e6 / peaks["hbm_gbs"],
                          "frac_of_nominal_8TBs": sbytes / ms_sp / 1e6 / 8000.0},
-            "gemm": {"ms": ms_gemm, "TFLOP/s": flops / ms_gemm / 1e9, "flops": flops,
-                     "frac_of_nominal_2250": flops / ms_gemm / 1e9 / 2250.0},
+            "gemm": {"ms": ms_gemm, "TFLOP/s": tf, "flops": flops,
+                     "frac_of_measured_burst": tf / peaks["bf16_tflops"],
+                     "frac_of_measured_sustained": tf / peaks["bf16_tflops_sustained"],
+                     "frac_of_nominal_2250": tf / 2250.0,
+                     "ms_x_sm_mhz": ms_gemm * sm_mhz if sm_mhz else None},
         },
-        "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": flops / ms_gemm / 1e9,
-                     "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                     "frac": flops / ms_gemm / 1e9 / peaks["bf16_tflops_sustained"],
-                     "traffic": NCU_GEMM_TRAFFIC_BYTES.get(wl.name) if (not args.layers and args.sparsity == 0.5 and not args.transposed) else None,
+        # the layer phase = 8 gemm_kernel launches per layer plus the small bias-gradient / split-K finishing launches,
+        # so `achieved` slightly understates the kernel itself
+        "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": tf,
+                     "peak": tp["peak"], "unit": "TFLOP/s", "frac": tf / tp["peak"],
+                     "peak_source": f"{peaks['source']} cuBLAS bf16, {tp['which']} figure (timed region "
+                                    f"{r['timed_ms'] / 1e3:.2f} s, median SM clock {sm_mhz} MHz)",
+                     "frac_of_measured_burst": tf / peaks["bf16_tflops"],
+                     "frac_of_measured_sustained": tf / peaks["bf16_tflops_sustained"],
+                     "frac_of_nominal_2250": tf / 2250.0,
+                     "traffic": NCU_GEMM_TRAFFIC_BYTES.get(wl.name) if plain else None,
                      "traffic_unit": "bytes per launch (DRAM read + write, ncu)",
-                     "peak_source": peaks["source"] + " (sustained cuBLAS bf16)",
                      "launches_per_step": n_gemm_launches, "avg_launch_ms": ms_gemm / n_gemm_launches},
         # the memory-bound part of the step against the measured copy bandwidth: score + select + compact as one unit
-        # (sumsq_kernel and gather_kernel move all of its bytes; traffic = their DRAM bytes under ncu on 8 layers of
-        # gpt2m, which grow in proportion to the layer count: 889.3 MB per 8 layers, profiles/sparsify_kernels_*.md)
+        # (sumsq_kernel and gather_kernel move all of its bytes; traffic = their DRAM bytes under ncu, which grow in
+        # proportion to the layer count)
         "roofline_hbm": {"bound": "hbm", "kernel": "sumsq_kernel + gather_kernel (+ finalize, select)",
                          "achieved": sbytes / ms_sp / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                          "frac": sbytes / ms_sp / 1e6 / peaks["hbm_gbs"],
-                         "traffic": (889.3e6 * wl.n_layers / 8 if (wl.name == "gpt2m" and args.sparsity == 0.5
-                                                                   and not args.transposed) else None),
+                         "frac_of_nominal_8TBs": sbytes / ms_sp / 1e6 / 8000.0,
+                         "traffic": sp_traffic * wl.n_layers if (sp_traffic and plain) else None,
                          "traffic_unit": "bytes per step (DRAM read + write, ncu, scaled by layers)",
                          "peak_source": peaks["source"] + " (copy bandwidth)"},
         "e2e": {"value": job_throughput(world, flops, ms_e2e) / 1e9, "unit": "TFLOP/s", "ms_per_step": ms_e2e,
@@ -425,9 +686,32 @@ def run_gpu(args):
                 "pipeline": "two device copies of the model: the upload of step s+1 overlaps the compute of step s"},
         "gpu_launches": int(launches), "clocks": clocks,
     }
+    if rank == 0 and world == 1:
+        out["parity_check"] = parity_check(m)
+    # ---- the other configurations (1 GPU runs only): each with its own clock record
+    if world == 1 and not args.no_configs and not args.layers:
+        cfgs = {}
+        cfgs["cfg3_llama1b" if wl.name == "llama1b" else "main"] = phase_report(wl, m, r, peaks, args.sparsity, args.transposed)
+        del m, sparsify, layers, r
+        torch.cuda.empty_cache()
+        cfg_steps = {"gpt2m": 40, "llama1b": 20, "llama7b_layer": 60}
+        plan = [("cfg2_gpt2m", "gpt2m", 0.5), ("cfg3_llama1b", "llama1b", 0.5), ("cfg4_llama7b_layer_s0.25", "llama7b_layer", 0.25),
+                ("cfg4_llama7b_layer_s0.50", "llama7b_layer", 0.5), ("cfg4_llama7b_layer_s0.75", "llama7b_layer", 0.75)]
+        for key, name, sp in plan:
+            if key in cfgs:
+                continue
+            w2 = WL.WORKLOADS[name]
+            mm = Model(w2, sp, dev)
+            rr = measure_step(mm, args, world, rank, local, cfg_steps[name], graph=not args.no_graph)
+            cfgs[key] = phase_report(w2, mm, rr, peaks, sp)
+            del mm, rr
+            torch.cuda.empty_cache()
+        cfgs["cfg5_reestimation_sweep"] = reestimation_sweep(WL.WORKLOADS["llama1b"], dev, local, rank)
+        torch.cuda.empty_cache()
+        out["configs"] = cfgs
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = cpu_sample(wl, args.sparsity)
+            out["cpu_baseline"] = cpu_baseline(wl, args.sparsity)
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
@@ -437,11 +721,21 @@ def run_gpu(args):
 # the CPU oracle on a bounded sample of the same step
 # ---------------------------------------------------------------------------------------------
 
-def cpu_sample(wl, sparsity: float, tokens: int = 256):
-    """Layer 0 of the workload through the oracle: score + Fisher + select + compact at full size,
-    then forward/backward of the compacted pairs on `tokens` token rows.  Returns the metric
-    (algorithmic flops / wall time) for that sample."""
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def cpu_sample(wl, sparsity: float, tokens: int = 256, threads: int = 1):
+    """Layer 0 of the workload through the oracle, as it stands: score + Fisher + select + compact at full size,
+    then forward/backward of the compacted pairs on `tokens` token rows.  With threads > 1 the pair groups (and their
+    tensors) of the first part, and equal chunks of the token rows of the second, are handed to a thread pool (the
+    oracle's C routines release the interpreter lock); every thread runs the same plain code on its share.  Returns
+    the metric (algorithmic flops / wall time) for that sample."""
     import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import oracle as O
     from paper_2511_11641_b200 import workloads as WL
     from paper_2511_11641_b200.block import pad8
@@ -453,37 +747,82 @@ def cpu_sample(wl, sparsity: float, tokens: int = 256):
                           widths={kk: n_attn for kk in ("dq", "dk", "dv", "ctx")})
     sw = wl.ffn == "swiglu"
     act = O.ACT_SWIGLU if sw else O.ACT_GELU_ERF
+    pool = ThreadPoolExecutor(max_workers=threads) if threads > 1 else None
+
+    def run_all(fns):
+        if pool is None:
+            return [f() for f in fns]
+        return [fu.result() for fu in [pool.submit(f) for f in fns]]
+
     t0 = time.perf_counter()
     groups = [("wq", "wk", None, "gq", "gk", None, 0, 0, wl.n_heads, wl.d_h, plan["qk"]),
               ("wv", "wo", None, "gv", "go", None, 0, 1, wl.n_heads, wl.d_h, plan["vo"]),
               ("w1", "w2", "w1b" if sw else None, "g1", "g2", "g1b" if sw else None, 0, 1, 1, wl.d_ffn, plan["ffn"])]
     c = {}
-    for n1, n2, n1b, g1, g2, g1b, l1, l2, n_seg, seg_len, k in groups:
+
+    def do_group(grp):
+        n1, n2, n1b, g1, g2, g1b, l1, l2, n_seg, seg_len, k = grp
         _, ups = O.score_pair(w[n1], w[n2], l1, l2, n_seg, seg_len, w1b=w.get(n1b) if n1b else None)
         O.fisher_pair(g[g1], g[g2], l1, l2, n_seg, seg_len, float(wl.tokens), g1b=g.get(g1b) if g1b else None)
         kept = O.select_topk(ups.astype(np.float32), n_seg, seg_len, k)
+        out = {}
         for nm, lay in ((n1, l1), (n2, l2), (n1b, l1), (g1, l1), (g2, l2), (g1b, l1)):
             if nm:
                 src = w[nm] if nm in w else g[nm]
-                c[nm] = O.compact(src, lay, kept, ld_out=pad8(len(kept), wl.elem_bytes) if lay == 0 else None)
+                out[nm] = O.compact(src, lay, kept, ld_out=pad8(len(kept), wl.elem_bytes) if lay == 0 else None)
+        return out
+
+    for d in run_all([(lambda grp=grp: do_group(grp)) for grp in groups]):
+        c.update(d)
     t1 = time.perf_counter()
-    x = acts["x"]
-    O.proj_fwd(x, c["wq"], 0, n_attn); O.proj_fwd(x, c["wk"], 0, n_attn); O.proj_fwd(x, c["wv"], 0, n_attn)
-    O.outproj_fwd(acts["ctx"], c["wo"], 1, n_attn, wl.d_m)
-    dX, _, _ = O.proj_bwd(x, c["wq"], 0, n_attn, acts["dq"])
-    O.proj_bwd(x, c["wk"], 0, n_attn, acts["dk"], dX=dX)
-    O.proj_bwd(x, c["wv"], 0, n_attn, acts["dv"])
-    O.outproj_bwd(acts["ctx"], c["wo"], 1, n_attn, wl.d_m, acts["dout"])
-    O.ffn_fwd(x, act, c["w1"], c["w2"], 0, 1, k_ffn, W1b=c.get("w1b"))
-    O.ffn_bwd(x, act, c["w1"], c["w2"], 0, 1, k_ffn, acts["dy"], W1b=c.get("w1b"))
+
+    def do_rows(lo, hi):
+        x = acts["x"][lo:hi].contiguous()
+        sl = lambda nm: acts[nm][lo:hi].contiguous()
+        O.proj_fwd(x, c["wq"], 0, n_attn); O.proj_fwd(x, c["wk"], 0, n_attn); O.proj_fwd(x, c["wv"], 0, n_attn)
+        O.outproj_fwd(sl("ctx"), c["wo"], 1, n_attn, wl.d_m)
+        dX, _, _ = O.proj_bwd(x, c["wq"], 0, n_attn, sl("dq"))
+        O.proj_bwd(x, c["wk"], 0, n_attn, sl("dk"), dX=dX)
+        O.proj_bwd(x, c["wv"], 0, n_attn, sl("dv"))
+        O.outproj_bwd(sl("ctx"), c["wo"], 1, n_attn, wl.d_m, sl("dout"))
+        O.ffn_fwd(x, act, c["w1"], c["w2"], 0, 1, k_ffn, W1b=c.get("w1b"))
+        O.ffn_bwd(x, act, c["w1"], c["w2"], 0, 1, k_ffn, sl("dy"), W1b=c.get("w1b"))
+
+    chunks = max(1, min(threads, tokens))
+    bounds = [(i * tokens // chunks, (i + 1) * tokens // chunks) for i in range(chunks)]
+    run_all([(lambda lo=lo, hi=hi: do_rows(lo, hi)) for lo, hi in bounds if hi > lo])
     t2 = time.perf_counter()
+    if pool is not None:
+        pool.shutdown()
     flops = step_flops(wl, n_attn, k_ffn) / wl.n_layers * tokens / wl.tokens
     sbytes = sparsify_bytes(wl, 1.0 - sparsity) / wl.n_layers
-    return {"value": flops / (t2 - t0) / 1e12, "unit": "TFLOP/s", "cores": 1, "kind": "oracle",
+    return {"value": flops / (t2 - t0) / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
             "sample": f"layer 0 of {wl.name}: score+Fisher+select+compact at full size ({t1 - t0:.2f} s, "
                       f"{sbytes / (t1 - t0) / 1e9:.3f} GB/s), then fwd+bwd of the compacted QK/VO/FFN pairs on "
-                      f"{tokens} of {wl.tokens} tokens ({t2 - t1:.2f} s)",
+                      f"{tokens} of {wl.tokens} tokens ({t2 - t1:.2f} s), {threads} thread(s)",
             "seconds": t2 - t0, "gemm_tflops": flops / (t2 - t1) / 1e12, "sparsify_GB/s": sbytes / (t1 - t0) / 1e9}
+
+
+def sample_tokens(wl, seconds: float = 12.0) -> int:
+    """Token rows whose fp64 triple-loop forward/backward takes about `seconds` on one core (~1.5 GFLOP/s)."""
+    per_token = step_flops(wl, wl.n_heads * wl.d_h // 2, wl.d_ffn // 2) / wl.n_layers / wl.tokens
+    return int(max(16, min(256, seconds * 1.5e9 / per_token)))
+
+
+def cpu_baseline(wl, sparsity: float):
+    """The oracle timed on this machine's host cores: once on one thread, once on every core of the affinity mask
+    (capped at 32) on a sample of `cores` times as many token rows.  `value` / `cores` are the threaded run."""
+    tokens = sample_tokens(wl)
+    one = cpu_sample(wl, sparsity, tokens, threads=1)
+    cores = min(32, host_cores())
+    if cores == 1:
+        one["single_thread"] = {"value": one["value"], "sample": one["sample"]}
+        return one
+    many = cpu_sample(wl, sparsity, min(wl.tokens, tokens * min(cores, 8)), threads=cores)
+    many["single_thread"] = {"value": one["value"], "gemm_tflops": one["gemm_tflops"], "sparsify_GB/s": one["sparsify_GB/s"],
+                             "sample": one["sample"]}
+    many["host_cores_in_affinity_mask"] = host_cores()
+    return many
 
 
 def run_reference(args):
@@ -520,13 +859,16 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gpt2m")
+    ap.add_argument("--workload", default="llama1b")
     ap.add_argument("--sparsity", type=float, default=0.5)
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (small cases for profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the other configurations (GPT-2-Medium shape, LLaMA-7B layer at three sparsities, "
+                         "re-estimation sweep) that a 1-GPU run reports beside the main workload")
     ap.add_argument("--transposed", action="store_true",
                     help="store every weight matrix the other way round (W_Q.. as D x d_m, W_O, W_2 as d_m x D)")
     ap.add_argument("--no-graph", action="store_true", help="issue every launch from the host instead of replaying a CUDA graph")
