@@ -24,12 +24,18 @@
 //                                  Definitions 1 and 2, Propositions 1 and 2.
 //   eco_proj_* / eco_ffn_*       : Eq. 2, 3 and 5 on the compacted matrices and
 //                                  their textbook reverse-mode derivatives.
+//   eco_attn_fwd / eco_attn_bwd  : the head of Eq. 2, phi(Q_i K_i^T / sqrt(d_h)) V_i, on compacted heads whose
+//                                  Q/K width and V width differ from head to head (the "Coupled Weight Matrix in
+//                                  MHA" reformulation with W_i^QK, W_i^VO restricted to the kept indices), and its
+//                                  textbook reverse mode.
 //
 // Parity unpinned (conventions the paper does not fix):
 //   - the SwiGLU slot of eco_fisher_pair (W_1 = gate (.) up is not a parameter),
 //   - the choice between the erf and tanh GELU forms,
 //   - in eco_threshold_counts_f32, whether theta is a share of the score mass (l1 = 1) or is compared with the
-//     l2-normalised scores as stored (l1 = 0): the paper prints the l2 normaliser and thresholds of 85-95 %.
+//     l2-normalised scores as stored (l1 = 0): the paper prints the l2 normaliser and thresholds of 85-95 %;
+//   - the causal flag of eco_attn_*: Eq. 2 prints no mask (causal = 0 is the equation as printed); the decoder
+//     models of the experiments mask keys after the query, which causal = 1 restates.
 //
 // Layout vocabulary: a matrix that owns a shared dimension D and another
 // dimension `other` is stored row-major either as  other x D  ("shared cols",
@@ -324,18 +330,23 @@ void eco_choose_pairs_f32(const float* fisher, int n, int m, int32_t* chosen) {
 //                       columns [n_kept, ld_out) are written as zero bytes.
 // layout 1 (D x other): out is n_kept x other with leading dimension ld_out >= other,
 //                       columns [other, ld_out) are written as zero bytes.
+// A kept entry of -1 stands for "no index": the output gets a zero column (row) there.  It lets a caller give
+// every head's block of a compacted tensor a padded width; zero columns add nothing to any product they enter.
 void eco_compact_bytes(const uint8_t* in, int elem_bytes, int layout, int64_t other, int64_t ld_in,
                        const int32_t* kept, int64_t n_kept, uint8_t* out, int64_t ld_out) {
     if (layout == 0) {
         for (int64_t i = 0; i < other; ++i) {
-            for (int64_t c = 0; c < n_kept; ++c)
-                std::memcpy(out + (i * ld_out + c) * elem_bytes, in + (i * ld_in + kept[c]) * elem_bytes, elem_bytes);
+            for (int64_t c = 0; c < n_kept; ++c) {
+                if (kept[c] < 0) std::memset(out + (i * ld_out + c) * elem_bytes, 0, elem_bytes);
+                else std::memcpy(out + (i * ld_out + c) * elem_bytes, in + (i * ld_in + kept[c]) * elem_bytes, elem_bytes);
+            }
             std::memset(out + (i * ld_out + n_kept) * elem_bytes, 0, (ld_out - n_kept) * elem_bytes);
         }
     } else {
         for (int64_t r = 0; r < n_kept; ++r) {
-            std::memcpy(out + r * ld_out * elem_bytes, in + static_cast<int64_t>(kept[r]) * ld_in * elem_bytes,
-                        other * elem_bytes);
+            if (kept[r] < 0) std::memset(out + r * ld_out * elem_bytes, 0, other * elem_bytes);
+            else std::memcpy(out + r * ld_out * elem_bytes, in + static_cast<int64_t>(kept[r]) * ld_in * elem_bytes,
+                             other * elem_bytes);
             std::memset(out + (r * ld_out + other) * elem_bytes, 0, (ld_out - other) * elem_bytes);
         }
     }
@@ -600,6 +611,103 @@ void eco_ffn_bwd(const void* X, int xdtype, int64_t T, int64_t d_m, int64_t ldx,
                 if (act == 3) s += dHb[t * k + j] * w1b.at(i, j);
             }
             dX[t * d_m + i] = s;
+        }
+}
+
+// ---------------------------------------------------------------------------
+// Attention on compacted heads.  Q, K (T x ..., pitch ldq / ldk) hold head h in columns [qk_off[h], qk_off[h] +
+// qk_w[h]); V (pitch ldv) holds it in columns [vo_off[h], vo_off[h] + vo_w[h]).  T = batch * seq: sequence b is
+// rows [b*seq, (b+1)*seq).  For every sequence and head, Eq. 2:
+//     S = scale * Q_h K_h^T,   P = phi(S) (softmax over the keys of each query row),   Ctx_h = P V_h
+// `scale` is the caller's 1/sqrt(d_h) with the architectural d_h of Eq. 2 (removal does not change it: the logits of
+// the compacted head are the full head's logits restricted to the kept indices).  causal != 0: query i sees keys
+// j <= i only.  Outputs in fp64: Ctx (T x ldc, head h in the V columns of head h), lse[h*T + t] = log sum_j exp(S_tj)
+// (may be NULL), P (n_heads x batch x seq x seq, may be NULL: for the tests on small sizes).
+// ---------------------------------------------------------------------------
+void eco_attn_fwd(const void* Q, const void* K, const void* V, int dtype, int64_t batch, int64_t seq, int n_heads,
+                  const int32_t* qk_off, const int32_t* qk_w, const int32_t* vo_off, const int32_t* vo_w, int64_t ldq,
+                  int64_t ldk, int64_t ldv, double scale, int causal, double* Ctx, int64_t ldc, double* lse, double* P) {
+    const int64_t T = batch * seq;
+    std::vector<double> srow(seq);
+    for (int h = 0; h < n_heads; ++h)
+        for (int64_t b = 0; b < batch; ++b)
+            for (int64_t i = 0; i < seq; ++i) {
+                const int64_t ti = b * seq + i;
+                const int64_t n_keys = causal ? i + 1 : seq;
+                double mx = -INFINITY;
+                for (int64_t j = 0; j < n_keys; ++j) {
+                    const int64_t tj = b * seq + j;
+                    double s = 0.0;
+                    for (int c = 0; c < qk_w[h]; ++c)
+                        s += load_elem(Q, dtype, ti * ldq + qk_off[h] + c) * load_elem(K, dtype, tj * ldk + qk_off[h] + c);
+                    srow[j] = s * scale;
+                    mx = std::max(mx, srow[j]);
+                }
+                double z = 0.0;
+                for (int64_t j = 0; j < n_keys; ++j) z += std::exp(srow[j] - mx);
+                if (lse) lse[static_cast<int64_t>(h) * T + ti] = mx + std::log(z);
+                for (int64_t j = 0; j < seq; ++j) {
+                    const double p = j < n_keys ? std::exp(srow[j] - mx) / z : 0.0;
+                    srow[j] = p;
+                    if (P) P[((static_cast<int64_t>(h) * batch + b) * seq + i) * seq + j] = p;
+                }
+                for (int c = 0; c < vo_w[h]; ++c) {
+                    double o = 0.0;
+                    for (int64_t j = 0; j < n_keys; ++j) o += srow[j] * load_elem(V, dtype, (b * seq + j) * ldv + vo_off[h] + c);
+                    Ctx[ti * ldc + vo_off[h] + c] = o;
+                }
+            }
+}
+
+// Reverse mode of eco_attn_fwd for L = <Ctx, dCtx>.  With P recomputed as above, per sequence and head:
+//     dV = P^T dCtx_h,   dP = dCtx_h V_h^T,   dS_ij = P_ij (dP_ij - sum_j' P_ij' dP_ij'),
+//     dQ_h = scale * dS K_h,   dK_h = scale * dS^T Q_h.
+// dCtx has the dtype and column layout of V (pitch lddc).  dQ, dK (T x ldq_out), dV (T x ldv_out) in fp64, same
+// column layout as Q, K, V; only the heads' columns are written.
+void eco_attn_bwd(const void* Q, const void* K, const void* V, const void* dCtx, int dtype, int64_t batch, int64_t seq,
+                  int n_heads, const int32_t* qk_off, const int32_t* qk_w, const int32_t* vo_off, const int32_t* vo_w,
+                  int64_t ldq, int64_t ldk, int64_t ldv, int64_t lddc, double scale, int causal, double* dQ, double* dK,
+                  int64_t ldq_out, double* dV, int64_t ldv_out) {
+    std::vector<double> p(seq), dp(seq);
+    for (int h = 0; h < n_heads; ++h)
+        for (int64_t b = 0; b < batch; ++b) {
+            for (int64_t t = b * seq; t < (b + 1) * seq; ++t) {
+                for (int c = 0; c < qk_w[h]; ++c) dQ[t * ldq_out + qk_off[h] + c] = dK[t * ldq_out + qk_off[h] + c] = 0.0;
+                for (int c = 0; c < vo_w[h]; ++c) dV[t * ldv_out + vo_off[h] + c] = 0.0;
+            }
+            for (int64_t i = 0; i < seq; ++i) {
+                const int64_t ti = b * seq + i;
+                const int64_t n_keys = causal ? i + 1 : seq;
+                double mx = -INFINITY;
+                for (int64_t j = 0; j < n_keys; ++j) {
+                    double s = 0.0;
+                    for (int c = 0; c < qk_w[h]; ++c)
+                        s += load_elem(Q, dtype, ti * ldq + qk_off[h] + c) * load_elem(K, dtype, (b * seq + j) * ldk + qk_off[h] + c);
+                    p[j] = s * scale;
+                    mx = std::max(mx, p[j]);
+                }
+                double z = 0.0;
+                for (int64_t j = 0; j < n_keys; ++j) z += std::exp(p[j] - mx);
+                double dot = 0.0;
+                for (int64_t j = 0; j < n_keys; ++j) {
+                    p[j] = std::exp(p[j] - mx) / z;
+                    double d = 0.0;
+                    for (int c = 0; c < vo_w[h]; ++c)
+                        d += load_elem(dCtx, dtype, ti * lddc + vo_off[h] + c) * load_elem(V, dtype, (b * seq + j) * ldv + vo_off[h] + c);
+                    dp[j] = d;
+                    dot += p[j] * d;
+                }
+                for (int64_t j = 0; j < n_keys; ++j) {
+                    const int64_t tj = b * seq + j;
+                    for (int c = 0; c < vo_w[h]; ++c)
+                        dV[tj * ldv_out + vo_off[h] + c] += p[j] * load_elem(dCtx, dtype, ti * lddc + vo_off[h] + c);
+                    const double ds = p[j] * (dp[j] - dot) * scale;
+                    for (int c = 0; c < qk_w[h]; ++c) {
+                        dQ[ti * ldq_out + qk_off[h] + c] += ds * load_elem(K, dtype, tj * ldk + qk_off[h] + c);
+                        dK[tj * ldq_out + qk_off[h] + c] += ds * load_elem(Q, dtype, ti * ldq + qk_off[h] + c);
+                    }
+                }
+            }
         }
 }
 

@@ -327,3 +327,42 @@ def ffn_bwd(X, act: int, W1, W2, layout1: int, layout2: int, k: int, dY, W1b=Non
                       C.c_int64(w2.ld), bb1.ptr, dy.ptr, C.c_int64(dy.ld), _p(dX), _p(dW1), _p(dW1b), _p(dW2),
                       _p(db1), _p(db2))
     return {"dX": dX, "dW1": dW1, "dW1b": dW1b, "dW2": dW2, "db1": db1, "db2": db2}
+
+
+# ---------------------------------------------------------------------------
+# attention on compacted heads
+# ---------------------------------------------------------------------------
+
+def attn_fwd(Q, K, V, batch: int, seq: int, qk_off, qk_w, vo_off, vo_w, scale: float, causal: bool = False,
+             want_p: bool = False):
+    """Returns dict(Ctx (T x V.shape[1], fp64; columns outside the heads are zero), lse (n_heads x T), P or None)."""
+    q, k, v = _Buf(Q), _Buf(K), _Buf(V)
+    assert q.dtype == k.dtype == v.dtype
+    T = batch * seq
+    assert Q.shape[0] == T and K.shape[0] == T and V.shape[0] == T
+    qo, qw, vo, vw = _i32(qk_off), _i32(qk_w), _i32(vo_off), _i32(vo_w)
+    H = qo.size
+    assert qw.size == H and vo.size == H and vw.size == H
+    Ctx = np.zeros((T, V.shape[1]), dtype=np.float64)
+    lse = np.empty((H, T), dtype=np.float64)
+    P = np.empty((H, batch, seq, seq), dtype=np.float64) if want_p else None
+    lib().eco_attn_fwd(q.ptr, k.ptr, v.ptr, q.dtype, C.c_int64(batch), C.c_int64(seq), H, _p(qo), _p(qw), _p(vo), _p(vw),
+                       C.c_int64(q.ld), C.c_int64(k.ld), C.c_int64(v.ld), C.c_double(scale), int(causal), _p(Ctx),
+                       C.c_int64(Ctx.shape[1]), _p(lse), _p(P))
+    return {"Ctx": Ctx, "lse": lse, "P": P}
+
+
+def attn_bwd(Q, K, V, dCtx, batch: int, seq: int, qk_off, qk_w, vo_off, vo_w, scale: float, causal: bool = False):
+    """Returns dict(dQ, dK (T x Q.shape[1]), dV (T x V.shape[1])) in fp64, zero outside the heads' columns."""
+    q, k, v, dc = _Buf(Q), _Buf(K), _Buf(V), _Buf(dCtx)
+    assert q.dtype == k.dtype == v.dtype == dc.dtype
+    T = batch * seq
+    qo, qw, vo, vw = _i32(qk_off), _i32(qk_w), _i32(vo_off), _i32(vo_w)
+    H = qo.size
+    dQ = np.zeros((T, Q.shape[1]), dtype=np.float64)
+    dK = np.zeros((T, Q.shape[1]), dtype=np.float64)
+    dV = np.zeros((T, V.shape[1]), dtype=np.float64)
+    lib().eco_attn_bwd(q.ptr, k.ptr, v.ptr, dc.ptr, q.dtype, C.c_int64(batch), C.c_int64(seq), H, _p(qo), _p(qw), _p(vo),
+                       _p(vw), C.c_int64(q.ld), C.c_int64(k.ld), C.c_int64(v.ld), C.c_int64(dc.ld), C.c_double(scale),
+                       int(causal), _p(dQ), _p(dK), C.c_int64(dQ.shape[1]), _p(dV), C.c_int64(dV.shape[1]))
+    return {"dQ": dQ, "dK": dK, "dV": dV}
