@@ -238,7 +238,8 @@ ecospa_status_t ecospa_pack_kept(const int32_t* slots, const int32_t* src, const
  * [n_kept, round_up(n_kept, 16 bytes)) for SHARED_COLS, [other_dim, round_up(other_dim, 16 bytes)) for
  * SHARED_ROWS, never beyond ld) are zero-filled.  out must not overlap in.
  * kept indices must be ascending and < D (not checked on the device beyond a clamp that keeps every
- * access inside `in`).
+ * access inside `in`).  An entry of -1 stands for "no index": the output gets a zero column (row) at that position
+ * (used to pad every head's block of a compacted tensor to the width the attention kernels need).
  */
 ecospa_status_t ecospa_compact_tensors(const ecospa_gather_t* jobs, int32_t n_jobs, void* stream);
 ecospa_status_t ecospa_compact_pair(const ecospa_pair_t* pair, const int32_t* kept, int32_t n_kept,
@@ -362,13 +363,63 @@ ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, int64_t T, in
                                        void* dW1b_c, int64_t ld_dw1, void* dW2_c, int64_t ld_dw2, void* db1_c,
                                        void* db2, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Attention core on the compacted heads: the head of Eq. 2,
+ *     head_i = phi( Q_i K_i^T / sqrt(d_h) ) V_i ,
+ * evaluated on the matrices that aligned removal leaves (Sec. 3.1, "Coupled Weight Matrix in MHA": the pair
+ * W_i^Q W_i^KT restricted to the kept indices of the QK pair, W_i^V W_i^O to those of the VO pair), so the Q/K width
+ * and the V width differ from each other and from head to head.  It sits between ecospa_coupled_qkv_fwd and
+ * ecospa_coupled_vo_fwd_o (and, in the backward pass, between ecospa_coupled_vo_bwd_o and ecospa_coupled_qkv_bwd).
+ *
+ * Layout: Qc, Kc (T x n_qk, pitch ld_qk) hold head h in columns [qk_off[h], qk_off[h] + qk_w[h]); Vc, Ctx and dCtx
+ * hold it in columns [vo_off[h], vo_off[h] + vo_w[h]).  T = batch * seq, sequence b = rows [b*seq, (b+1)*seq).
+ * Every width must be a multiple of 16 (at most 128) and every offset a multiple of 8: give the compaction step a
+ * kept list in which every head's block is padded with -1 entries (ecospa_pad_kept) -- a zero column of Q^c / K^c adds
+ * nothing to Q K^T and a zero column of V^c yields a zero column of Ctx, so results on the real columns do not
+ * change.  bf16 tensors only; at most 128 heads.
+ *   scale   the caller's 1/sqrt(d_h) with the architectural d_h of Eq. 2 (removal does not change it); > 0
+ *   causal  != 0: query i attends to keys j <= i of its sequence (Eq. 2 prints no mask: causal == 0 is the equation
+ *           as printed; decoder models mask)
+ *   lse     DEVICE fp32 [n_heads * T]: lse[h*T + t] = log sum_j exp(scale * q_t . k_j), written by the forward call
+ *           and read by the backward call
+ * Forward: Ctx (T x n_vo, pitch ld_ctx); only the heads' columns of rows < T are written.
+ * Backward (reverse mode of the same expression): given dCtx, writes dQc, dKc (pitch ld_dqk) and dVc (pitch ld_dv) in
+ * the layout of Qc, Kc, Vc.  workspace: DEVICE, at least ecospa_attn_workspace_bytes, 16-byte aligned.
+ * Results are deterministic (no atomics: dK and dV are accumulated by the CTA that owns the key block, dQ by the CTA
+ * that owns the query block).  A device-side wait that expires records codes 11-13 (forward), 14-19 (backward).
+ */
+typedef struct {
+    int32_t n_heads;
+    const int32_t* qk_off; /* HOST [n_heads] first column of head h in Qc / Kc */
+    const int32_t* qk_w;   /* HOST [n_heads] its (padded) width */
+    const int32_t* vo_off; /* HOST [n_heads] first column of head h in Vc / Ctx */
+    const int32_t* vo_w;   /* HOST [n_heads] its (padded) width */
+} ecospa_heads_t;
+
+size_t ecospa_attn_workspace_bytes(int64_t batch, int64_t seq, int32_t n_heads);
+ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* Kc, int64_t ld_qk, const void* Vc, int64_t ld_v,
+                                        int64_t batch, int64_t seq, const ecospa_heads_t* heads, float scale,
+                                        int32_t causal, void* Ctx, int64_t ld_ctx, float* lse, void* stream);
+ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* Kc, int64_t ld_qk, const void* Vc, int64_t ld_v,
+                                        const void* Ctx, int64_t ld_ctx, const void* dCtx, int64_t ld_dctx,
+                                        const float* lse, int64_t batch, int64_t seq, const ecospa_heads_t* heads,
+                                        float scale, int32_t causal, void* dQc, void* dKc, int64_t ld_dqk, void* dVc,
+                                        int64_t ld_dv, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Kept list with padded segments: for every segment s (HOST arrays of n_segs entries), out[dst[s] + i] =
+ * kept[src[s] + i] for i < k[s] and -1 for k[s] <= i < k_padded[s].  A -1 entry makes the compaction step write a
+ * zero column (row) at that position.  kept, out: DEVICE int32.  Index bookkeeping only (no counterpart in the paper). */
+ecospa_status_t ecospa_pad_kept(const int32_t* kept, const int32_t* src, const int32_t* dst, const int32_t* k,
+                                const int32_t* k_padded, int32_t n_segs, int32_t* out, void* stream);
+
 /* How many CTA pairs (2-SM clusters) of the GEMM engine are resident at once on the current device; 0 when
  * pair mode is off (environment ECOSPA_GEMM_PAIR=0), -1 on a CUDA error.  Informational. */
 int32_t ecospa_gemm_resident_pairs(void);
 
 /* Synchronises `stream` and reports the status word of the current device: ECOSPA_OK and *code = 0, or
  * ECOSPA_ERR_TIMEOUT and *code = which bounded wait expired (1 producer, 2 accumulator-free,
- * 3 operands-ready, 4 accumulator-ready); the word is cleared.  This is the one call that blocks.
+ * 3 operands-ready, 4 accumulator-ready; 11-19: the attention kernels); the word is cleared.  This is the one call
+ * that blocks.
  * Every device the library is used on has its own status word. */
 ecospa_status_t ecospa_device_status(void* stream, int32_t* code);
 

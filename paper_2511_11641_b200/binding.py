@@ -479,6 +479,73 @@ def ecospa_coupled_ffn_bwd(X, act: int, w1_c, w2_c, k: int, H, A, dY, dX, dW1_c,
            "ecospa_coupled_ffn_bwd")
 
 
+# ---------------------------------------------------------------------------------------------
+# attention core on compacted heads
+# ---------------------------------------------------------------------------------------------
+
+class Heads(C.Structure):
+    _fields_ = [("n_heads", C.c_int32), ("qk_off", C.c_void_p), ("qk_w", C.c_void_p), ("vo_off", C.c_void_p),
+                ("vo_w", C.c_void_p)]
+
+
+def heads(qk_off: Sequence[int], qk_w: Sequence[int], vo_off: Sequence[int], vo_w: Sequence[int]) -> Heads:
+    """Descriptor of the per-head column blocks of Qc / Kc (qk_*) and of Vc / Ctx (vo_*)."""
+    n = len(qk_off)
+    assert len(qk_w) == n and len(vo_off) == n and len(vo_w) == n
+    arrs = [(C.c_int32 * n)(*[int(x) for x in v]) for v in (qk_off, qk_w, vo_off, vo_w)]
+    h = Heads(n, *[C.addressof(a) for a in arrs])
+    h._keep = arrs
+    return h
+
+
+def ecospa_attn_workspace_bytes(batch: int, seq: int, n_heads: int) -> int:
+    f = lib().ecospa_attn_workspace_bytes
+    f.restype = C.c_size_t
+    f.argtypes = [C.c_int64, C.c_int64, C.c_int32]
+    return int(f(batch, seq, n_heads))
+
+
+def ecospa_coupled_attn_fwd(Qc, Kc, Vc, batch: int, seq: int, hd: Heads, scale: float, causal: bool, Ctx, lse,
+                            stream=None) -> None:
+    """Ctx_h = softmax(scale * Q_h K_h^T) V_h per sequence and head; lse: fp32 [n_heads * T]."""
+    f = lib().ecospa_coupled_attn_fwd
+    f.restype = C.c_int
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_float,
+                  C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+    assert Qc.stride(0) == Kc.stride(0)
+    _check(f(Qc.data_ptr(), Kc.data_ptr(), Qc.stride(0), Vc.data_ptr(), Vc.stride(0), batch, seq, C.addressof(hd),
+             float(scale), int(bool(causal)), Ctx.data_ptr(), Ctx.stride(0), lse.data_ptr(), _stream(stream)),
+           "ecospa_coupled_attn_fwd")
+
+
+def ecospa_coupled_attn_bwd(Qc, Kc, Vc, Ctx, dCtx, lse, batch: int, seq: int, hd: Heads, scale: float, causal: bool,
+                            dQc, dKc, dVc, workspace, stream=None) -> None:
+    f = lib().ecospa_coupled_attn_bwd
+    f.restype = C.c_int
+    f.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                  C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_float, C.c_int32, C.c_void_p, C.c_void_p, C.c_int64,
+                  C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+    assert Qc.stride(0) == Kc.stride(0) and dQc.stride(0) == dKc.stride(0)
+    wp, wb = _ws(workspace)
+    _check(f(Qc.data_ptr(), Kc.data_ptr(), Qc.stride(0), Vc.data_ptr(), Vc.stride(0), Ctx.data_ptr(), Ctx.stride(0),
+             dCtx.data_ptr(), dCtx.stride(0), lse.data_ptr(), batch, seq, C.addressof(hd), float(scale),
+             int(bool(causal)), dQc.data_ptr(), dKc.data_ptr(), dQc.stride(0), dVc.data_ptr(), dVc.stride(0), wp, wb,
+             _stream(stream)), "ecospa_coupled_attn_bwd")
+
+
+def ecospa_pad_kept(kept: torch.Tensor, src: Sequence[int], dst: Sequence[int], k: Sequence[int],
+                    k_padded: Sequence[int], out: torch.Tensor, stream=None) -> None:
+    n = len(src)
+    assert len(dst) == n and len(k) == n and len(k_padded) == n and kept.dtype == torch.int32 and out.dtype == torch.int32
+    arr = lambda v: (C.c_int32 * n)(*[int(x) for x in v])
+    a_src, a_dst, a_k, a_kp = arr(src), arr(dst), arr(k), arr(k_padded)
+    fn = lib().ecospa_pad_kept
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+    _check(fn(_ptr(kept), C.addressof(a_src), C.addressof(a_dst), C.addressof(a_k), C.addressof(a_kp), n, _ptr(out),
+              _stream(stream)), "ecospa_pad_kept")
+
+
 def ecospa_launch_count() -> int:
     f = lib().ecospa_launch_count
     f.restype = C.c_uint64

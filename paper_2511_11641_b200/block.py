@@ -51,3 +51,14 @@ def alloc_compacted(t: torch.Tensor, layout: int, n_kept: int) -> torch.Tensor:
     if layout == B.SHARED_COLS:
         return torch.empty((t.shape[0], pad8(n_kept, t.element_size())), dtype=t.dtype, device=t.device)
     return torch.empty((n_kept, t.shape[1]), dtype=t.dtype, device=t.device)
+
+
+def padded_head_layout(k_heads: Sequence[int], multiple: int = 16) -> Tuple[List[int], List[int], int]:
+    """Column blocks of compacted heads padded to the width granularity of the attention kernels:
+    (first column of every head, its padded width, total padded width)."""
+    off, w, o = [], [], 0
+    for k in k_heads:
+        kp = (int(k) + multiple - 1) // multiple * multiple
+        off.append(o); w.append(kp)
+        o += kp
+    return off, w, o

@@ -1,0 +1,949 @@
+// Attention core on compacted heads (Eq. 2 per head, with the heads of the coupled-matrix reformulation of Sec. 3.1
+// restricted to their kept indices): Ctx_h = softmax(scale * Q_h K_h^T) V_h for heads whose Q/K width and V width
+// differ from head to head, forward and backward.  sm_100a: TMA tile loads -> shared memory -> tcgen05.mma with the
+// score tiles and the output tile in TMEM; the softmax runs in registers, one thread per query row.
+//
+// Layout: Q^c, K^c (T x n_qk) and V^c, Ctx (T x n_vo) hold head h in columns [off_h, off_h + w_h) with w_h a multiple of
+// 16 (the compaction step pads every head's block with zero columns: a zero column of Q^c / K^c adds nothing to
+// Q K^T, and a zero column of V^c gives a zero column of Ctx) and off_h a multiple of 8, so that every tile load starts
+// on a 16-byte boundary and every contraction is a whole number of 16-deep MMA steps.
+//
+// Forward kernel, one CTA per SM, 192 threads.  A work item is (sequence b, head h, 128 query rows); a CTA walks a
+// static list of items (for causal attention the long ones first).
+//   warp 0      producer: one lane issues the TMA loads of the item's Q tile (2 buffers) and of every K / V tile
+//               (2 stages); a tile is one or two 64-column blocks of 128 rows x 128 bytes, 128-byte swizzle
+//   warp 1      owns TMEM (512 columns: two 128-column score buffers, one output tile of up to 128 columns); one lane
+//               issues S = Q K^T (K-major operands) and O_tile = P V (P from shared memory, V as stored = MN-major)
+//   warps 2..5  softmax, thread = query row (= TMEM lane): row maximum over the score tile, p = 2^(s*c - m) with the
+//               running maximum m, P as bf16 into shared memory (K-major, swizzled) for the second product, and the
+//               running output O = O * 2^(m_old - m_new) + O_tile in registers; at the end O / l and the row's
+//               log-sum-exp are written
+// The score tile of key block j+1 is issued before P V of block j, so the tensor pipe works while the softmax of the
+// next block runs.  Every mbarrier wait is bounded; on expiry the CTA records a code (11 producer, 12 MMA issuer,
+// 13 softmax) in the device status word, lets copies land, frees TMEM and returns.
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include "common.cuh"
+#include "gemm.cuh"
+#include "tc.cuh"
+
+namespace ecospa {
+
+namespace {
+
+using namespace tc;
+
+constexpr int kTile = 128;                  // query rows and key rows per tile
+constexpr int kBlockBytes = kTile * 128;    // one 64-column block of a 128-row tile
+constexpr int kMaxHeads = 128;
+constexpr int kFwdThreads = 192;
+constexpr int kTmemCols = 512;
+constexpr uint32_t kColS = 0, kColO = 256;  // TMEM columns: score buffers at 0 and 128, output tile at 256
+
+struct HeadLayout {
+    int32_t qk_off[kMaxHeads], qk_w[kMaxHeads], vo_off[kMaxHeads], vo_w[kMaxHeads];
+};
+
+struct AttnFwdParams {
+    alignas(64) CUtensorMap map_q, map_k, map_v;
+    HeadLayout heads;
+    int32_t batch, seq, n_heads, n_qt, causal, n_items;
+    float scale_log2e;                      // scale * log2(e): scores are exponentiated in base 2
+    uint16_t* ctx;
+    int64_t ld_ctx;
+    float* lse;                             // [n_heads][T], natural logarithm
+    int* status;
+    unsigned long long wait_limit_ns;
+};
+
+struct Item {
+    int b, h, qt, n_kv;
+};
+__device__ __forceinline__ Item decode_item(int it, int n_qt, int n_heads, int batch, int n_kt, int causal) {
+    Item I;
+    const int per = n_heads * batch;
+    I.qt = n_qt - 1 - it / per;             // long (late) query tiles first
+    const int rem = it % per;
+    I.h = rem / batch;
+    I.b = rem % batch;
+    I.n_kv = causal ? min(n_kt, I.qt + 1) : n_kt;
+    return I;
+}
+
+template <int NB>   // 64-column blocks per tile: 1 (every head at most 64 wide) or 2
+__global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_constant__ AttnFwdParams P) {
+    constexpr int kTileBytes = NB * kBlockBytes;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw_addr);
+    const uint32_t sQ = base, sK = sQ + 2 * kTileBytes, sV = sK + 2 * kTileBytes, sP = sV + 2 * kTileBytes;
+    uint8_t* tail = smem + 6 * kTileBytes + 2 * kBlockBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 16 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto q_full = [&](uint32_t s) { return bar0 + 8u * s; };
+    auto q_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };
+    auto kv_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
+    auto kv_empty = [&](uint32_t s) { return bar0 + 8u * (6 + s); };
+    auto s_full = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
+    const uint32_t p_full = bar0 + 8u * 10, o_full = bar0 + 8u * 11;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int n_kt = (P.seq + kTile - 1) / kTile;
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < 2; ++s) {
+            mbar_init(q_full(s), 1);
+            mbar_init(q_empty(s), 1);
+            mbar_init(kv_full(s), 1);
+            mbar_init(kv_empty(s), 1);
+            mbar_init(s_full(s), 1);
+        }
+        mbar_init(p_full, 128);
+        mbar_init(o_full, 1);
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&P.map_q);
+        prefetch_tensormap(&P.map_k);
+        prefetch_tensormap(&P.map_v);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_holder), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t g = 0, qi = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++qi) {
+                const Item I = decode_item(it, P.n_qt, P.n_heads, P.batch, n_kt, P.causal);
+                const int qoff = P.heads.qk_off[I.h], voff = P.heads.vo_off[I.h];
+                const int nbq = (P.heads.qk_w[I.h] + 63) >> 6, nbv = (P.heads.vo_w[I.h] + 63) >> 6;
+                const int row0 = I.b * P.seq;
+                const uint32_t qs = qi & 1;
+                if (!(ok = mbar_wait(q_empty(qs), ((qi >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
+                mbar_expect_tx(q_full(qs), nbq * kBlockBytes);
+                for (int blk = 0; blk < nbq; ++blk)
+                    tma_load_2d(sQ + qs * kTileBytes + blk * kBlockBytes, &P.map_q, qoff + 64 * blk, row0 + I.qt * kTile, q_full(qs));
+                for (int j = 0; j < I.n_kv; ++j, ++g) {
+                    const uint32_t st = g & 1;
+                    if (!(ok = mbar_wait(kv_empty(st), ((g >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
+                    mbar_expect_tx(kv_full(st), (nbq + nbv) * kBlockBytes);
+                    for (int blk = 0; blk < nbq; ++blk)
+                        tma_load_2d(sK + st * kTileBytes + blk * kBlockBytes, &P.map_k, qoff + 64 * blk, row0 + j * kTile, kv_full(st));
+                    for (int blk = 0; blk < nbv; ++blk)
+                        tma_load_2d(sV + st * kTileBytes + blk * kBlockBytes, &P.map_v, voff + 64 * blk, row0 + j * kTile, kv_full(st));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t g = 0, qi = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++qi) {
+                const Item I = decode_item(it, P.n_qt, P.n_heads, P.batch, n_kt, P.causal);
+                const int wq = P.heads.qk_w[I.h], wv = P.heads.vo_w[I.h];
+                const uint32_t qs = qi & 1;
+                if (!(ok = mbar_wait(q_full(qs), (qi >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                const uint32_t idesc_s = make_idesc(kTile, kTile, 0, 0);
+                const uint32_t idesc_o = make_idesc(kTile, wv, 0, 1);
+                // S = Q K^T of key block gg into score buffer gg & 1
+                auto issue_scores = [&](uint32_t gg) -> bool {
+                    const uint32_t st = gg & 1;
+                    if (!mbar_wait(kv_full(st), (gg >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns)) return false;
+                    tc_fence_after();
+                    for (int ks = 0; ks < (wq >> 4); ++ks) {
+                        const uint32_t o = (ks >> 2) * kBlockBytes + (ks & 3) * 32;
+                        tc_mma_bf16(tmem_base + kColS + st * kTile, make_smem_desc(sQ + qs * kTileBytes + o, 16, 1024),
+                                    make_smem_desc(sK + st * kTileBytes + o, 16, 1024), idesc_s, ks != 0 ? 1u : 0u);
+                    }
+                    tc_commit(s_full(st));
+                    return true;
+                };
+                if (!(ok = issue_scores(g))) break;
+                for (int j = 0; j < I.n_kv; ++j, ++g) {
+                    if (j + 1 < I.n_kv && !(ok = issue_scores(g + 1))) break;
+                    if (!(ok = mbar_wait(p_full, g & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                    tc_fence_after();
+                    const uint32_t st = g & 1;
+                    for (int ks = 0; ks < kTile / 16; ++ks)   // O_tile = P V over the 128 keys of the block
+                        tc_mma_bf16(tmem_base + kColO, make_smem_desc(sP + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
+                                    make_smem_desc(sV + st * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc_o, ks != 0 ? 1u : 0u);
+                    tc_commit(o_full);
+                    tc_commit(kv_empty(st));
+                }
+                if (ok) tc_commit(q_empty(qs));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax, thread = query row
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const uint32_t p_row = sP + row * 128;
+        const int swz = row & 7;
+        uint32_t g = 0;
+        bool ok = true;
+        const int64_t T = static_cast<int64_t>(P.batch) * P.seq;
+        for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x) {
+            const Item I = decode_item(it, P.n_qt, P.n_heads, P.batch, n_kt, P.causal);
+            const int wv = P.heads.vo_w[I.h];
+            const int q_pos = I.qt * kTile + row;                     // position of this row in its sequence
+            const int limit = P.causal ? min(P.seq, q_pos + 1) : P.seq;   // keys [0, limit) are visible
+            float m = -INFINITY, l = 0.f, alpha_prev = 0.f;
+            float o[NB * 64];
+#pragma unroll
+            for (int i = 0; i < NB * 64; ++i) o[i] = 0.f;
+            // O = O * a + O_tile (the output tile of the previous key block)
+            auto fold_output = [&](float a) {
+#pragma unroll
+                for (int c = 0; c < NB * 4; ++c) {
+                    if (c * 16 < wv) {
+                        uint32_t r[16];
+                        tc_ld16(t_lane + kColO + c * 16, r);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) o[c * 16 + i] = fmaf(o[c * 16 + i], a, __uint_as_float(r[i]));
+                    }
+                }
+            };
+            for (int j = 0; j < I.n_kv; ++j, ++g) {
+                const uint32_t sb = g & 1;
+                if (!(ok = mbar_wait(s_full(sb), (g >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                const uint32_t t_s = t_lane + kColS + sb * kTile;
+                const int kv0 = j * kTile;
+                const bool masked = kv0 + kTile > limit;
+                // pass 1: row maximum of this block
+                float mx = -INFINITY;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tc_ld32(t_s + c * 32, r);
+                    tc_wait_ld();
+                    if (masked) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (kv0 + c * 32 + i < limit) mx = fmaxf(mx, __uint_as_float(r[i]));
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
+                    }
+                }
+                const float m_new = fmaxf(m, mx * P.scale_log2e);
+                const float alpha = ex2(m - m_new);
+                if (j > 0) {
+                    if (!(ok = mbar_wait(o_full, (g - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                    tc_fence_after();
+                    fold_output(alpha_prev);
+                }
+                // pass 2: p = 2^(s * c - m_new), row sum, P as bf16 into shared memory
+                float rs = 0.f;
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t r[32];
+                    tc_ld32(t_s + c * 32, r);
+                    tc_wait_ld();
+                    float p[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const float e = ex2(fmaf(__uint_as_float(r[i]), P.scale_log2e, -m_new));
+                        p[i] = (masked && kv0 + c * 32 + i >= limit) ? 0.f : e;
+                        rs += p[i];
+                    }
+                    // 32 columns = four 16-byte chunks of block c / 2; chunk q of a row sits at (q ^ (row & 7))
+                    const uint32_t blk = p_row + (c >> 1) * kBlockBytes;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int chunk = (c & 1) * 4 + q;
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(blk + ((chunk ^ swz) << 4)),
+                                     "r"(pack_bf16(p[8 * q + 0], p[8 * q + 1])), "r"(pack_bf16(p[8 * q + 2], p[8 * q + 3])),
+                                     "r"(pack_bf16(p[8 * q + 4], p[8 * q + 5])), "r"(pack_bf16(p[8 * q + 6], p[8 * q + 7]))
+                                     : "memory");
+                    }
+                }
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(p_full);
+                l = fmaf(l, alpha, rs);
+                m = m_new;
+                alpha_prev = alpha;
+            }
+            if (!ok) break;
+            if (!(ok = mbar_wait(o_full, (g - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+            tc_fence_after();
+            fold_output(alpha_prev);
+            if (q_pos < P.seq) {
+                const int64_t t = static_cast<int64_t>(I.b) * P.seq + q_pos;
+                const float inv = 1.f / l;
+                uint16_t* dst = P.ctx + t * P.ld_ctx + P.heads.vo_off[I.h];
+#pragma unroll
+                for (int c = 0; c < NB * 8; ++c) {
+                    if (c * 8 < wv) {
+                        uint4 v;
+                        v.x = pack_bf16(o[c * 8 + 0] * inv, o[c * 8 + 1] * inv);
+                        v.y = pack_bf16(o[c * 8 + 2] * inv, o[c * 8 + 3] * inv);
+                        v.z = pack_bf16(o[c * 8 + 4] * inv, o[c * 8 + 5] * inv);
+                        v.w = pack_bf16(o[c * 8 + 6] * inv, o[c * 8 + 7] * inv);
+                        *reinterpret_cast<uint4*>(dst + c * 8) = v;
+                    }
+                }
+                P.lse[static_cast<int64_t>(I.h) * T + t] = m * 0.6931471805599453f + logf(l);
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);   // copies still in flight land before the memory is released
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// backward
+// ------------------------------------------------------------------------------------------------
+// Reverse mode of Ctx_h = P V_h, P = softmax(scale * Q_h K_h^T), with P recomputed from the saved log-sum-exp:
+//     dV = P^T dCtx,  dP = dCtx V^T,  dS = P (.) (dP - D),  D_t = sum_c dCtx[t, c] Ctx[t, c],
+//     dQ = scale * dS K,  dK = scale * dS^T Q.
+// Three launches: the row dots D (memory-bound), then one launch that owns key blocks (dK and dV accumulate in TMEM
+// over the query blocks) and one that owns query blocks (dQ accumulates over the key blocks).  Nothing is added
+// across CTAs, so the results do not depend on timing.
+
+// D[h][t] for every head: a warp takes a row, every lane multiplies 16-byte vectors (8 columns, which never straddle a
+// head because offsets and widths are multiples of 8), and the per-vector partial sums are added per head in order.
+constexpr int kDotWarps = 4;
+constexpr int kDotMaxVecs = 2048;      // 16384 columns
+struct DotParams {
+    HeadLayout heads;
+    const uint16_t* ctx;
+    const uint16_t* dctx;
+    float* out;                        // [n_heads][T]
+    int64_t ld_ctx, ld_dctx, T;
+    int32_t n_heads, n_vecs;
+};
+__global__ void __launch_bounds__(32 * kDotWarps) attn_rowdot_kernel(const __grid_constant__ DotParams P) {
+    __shared__ float part[kDotWarps][kDotMaxVecs];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t t = static_cast<int64_t>(blockIdx.x) * kDotWarps + warp;
+    if (t >= P.T) return;
+    const uint16_t* a = P.ctx + t * P.ld_ctx;
+    const uint16_t* b = P.dctx + t * P.ld_dctx;
+    for (int v = lane; v < P.n_vecs; v += 32) {
+        const uint4 x = *reinterpret_cast<const uint4*>(a + 8 * v);
+        const uint4 y = *reinterpret_cast<const uint4*>(b + 8 * v);
+        float s = bf16_lo(x.x) * bf16_lo(y.x);
+        s = fmaf(bf16_hi(x.x), bf16_hi(y.x), s);
+        s = fmaf(bf16_lo(x.y), bf16_lo(y.y), s);
+        s = fmaf(bf16_hi(x.y), bf16_hi(y.y), s);
+        s = fmaf(bf16_lo(x.z), bf16_lo(y.z), s);
+        s = fmaf(bf16_hi(x.z), bf16_hi(y.z), s);
+        s = fmaf(bf16_lo(x.w), bf16_lo(y.w), s);
+        s = fmaf(bf16_hi(x.w), bf16_hi(y.w), s);
+        part[warp][v] = s;
+    }
+    __syncwarp();
+    for (int h = lane; h < P.n_heads; h += 32) {
+        const int v0 = P.heads.vo_off[h] >> 3, nv = P.heads.vo_w[h] >> 3;
+        float s = 0.f;
+        for (int i = 0; i < nv; ++i) s += part[warp][v0 + i];
+        P.out[static_cast<int64_t>(h) * P.T + t] = s;
+    }
+}
+
+struct AttnBwdParams {
+    alignas(64) CUtensorMap map_q, map_k, map_v, map_do;
+    HeadLayout heads;
+    int32_t batch, seq, n_heads, n_t, causal, n_items;
+    float scale_log2e, scale;
+    const float* lse;                  // [n_heads][T], natural logarithm
+    const float* dvec;                 // [n_heads][T] row dots D
+    uint16_t* dq;
+    uint16_t* dk;
+    uint16_t* dv;
+    int64_t ld_dqk, ld_dv;
+    int* status;
+    unsigned long long wait_limit_ns;
+};
+
+// MODE 0: a CTA owns a key block of a (sequence, head) and walks the query blocks: K, V resident, Q_i and dCtx_i
+//         streamed; X = S^T = K Q_i^T and Y = dP^T = V dCtx_i^T (thread = key row, columns = queries); P^T and dS^T go to
+//         shared memory; dV += P^T dCtx_i and dK += dS^T Q_i accumulate in TMEM.
+// MODE 1: a CTA owns a query block and walks the key blocks: Q, dCtx resident, K_j and V_j streamed; X = S = Q K_j^T and
+//         Y = dP = dCtx V_j^T (thread = query row); dS goes to shared memory; dQ += dS K_j accumulates in TMEM.
+// Streamed tiles serve twice: as K-major B operands of the score products and as MN-major B operands of the
+// accumulating ones (same bytes, other descriptor).  Warp roles as in the forward kernel.  The score products of
+// step i+1 are issued before the accumulating products of step i.  Wait codes: 14 / 15 / 16 (MODE 0 producer, issuer,
+// compute) and 17 / 18 / 19 (MODE 1).
+template <int NB, int MODE>
+struct BwdCfg {
+    static constexpr int kTileBytes = NB * kBlockBytes;
+    static constexpr int kResStages = NB == 1 ? 2 : 1;                         // buffers of the resident pair of tiles
+    static constexpr int kStrStages = (NB == 1 || MODE == 1) ? 2 : 1;          // stages of the streamed pair of tiles
+    static constexpr int kOutTiles = MODE == 0 ? 2 : 1;                        // P^T and dS^T, or dS
+    static constexpr int kVecBytes = MODE == 0 ? 2 * 2 * kTile * 4 : 0;        // lse and D of a query block, two buffers
+    static constexpr int kSmem = 2 * kTileBytes * (kResStages + kStrStages) + kOutTiles * 2 * kBlockBytes + kVecBytes + 1024 + 256;
+};
+
+template <int NB, int MODE>
+__global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_constant__ AttnBwdParams P) {
+    using Cfg = BwdCfg<NB, MODE>;
+    constexpr int kTileBytes = Cfg::kTileBytes;
+    constexpr int RS = Cfg::kResStages, SS = Cfg::kStrStages;
+    constexpr uint32_t kColX = 0, kColY = 128, kColAcc1 = 256, kColAcc2 = 384;
+    constexpr int kCodeBase = MODE == 0 ? 14 : 17;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw_addr);
+    // resident: [stage][a | b], streamed: [stage][a | b], out tiles, vectors, barriers
+    const uint32_t sRes = base, sStr = sRes + 2 * kTileBytes * RS, sOut = sStr + 2 * kTileBytes * SS;
+    uint8_t* vec_raw = smem + 2 * kTileBytes * (RS + SS) + Cfg::kOutTiles * 2 * kBlockBytes;
+    float* vec = reinterpret_cast<float*>(vec_raw);                               // [2 buffers][lse2 | D][128]
+    uint8_t* tail = vec_raw + Cfg::kVecBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 16 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto r_full = [&](uint32_t s) { return bar0 + 8u * s; };
+    auto r_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };
+    auto t_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
+    auto t_empty = [&](uint32_t s) { return bar0 + 8u * (6 + s); };
+    const uint32_t x_full = bar0 + 8u * 8, out_full = bar0 + 8u * 9, out_empty = bar0 + 8u * 10, acc_full = bar0 + 8u * 11,
+                   acc_empty = bar0 + 8u * 12, vec_ready = bar0 + 8u * 13;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < 2; ++s) {
+            mbar_init(r_full(s), 1);
+            mbar_init(r_empty(s), 1);
+            mbar_init(t_full(s), 1);
+            mbar_init(t_empty(s), 1);
+        }
+        mbar_init(x_full, 1);
+        mbar_init(out_full, 128);
+        mbar_init(out_empty, 1);
+        mbar_init(acc_full, 1);
+        mbar_init(acc_empty, 128);
+        mbar_init(vec_ready, 128);
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&P.map_q);
+        prefetch_tensormap(&P.map_k);
+        prefetch_tensormap(&P.map_v);
+        prefetch_tensormap(&P.map_do);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_holder), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    // item -> (sequence, head, owned block, number of steps, first streamed block)
+    struct BItem {
+        int b, h, own, n_steps, first;
+    };
+    auto decode = [&](int it) {
+        BItem I;
+        const int per = P.n_heads * P.batch;
+        const int a = it / per;
+        I.own = MODE == 0 ? a : P.n_t - 1 - a;                 // causal: the blocks with the most steps first
+        const int rem = it % per;
+        I.h = rem / P.batch;
+        I.b = rem % P.batch;
+        if (MODE == 0) {
+            I.first = P.causal ? I.own : 0;                    // query blocks at or after the key block
+            I.n_steps = P.n_t - I.first;
+        } else {
+            I.first = 0;
+            I.n_steps = P.causal ? I.own + 1 : P.n_t;          // key blocks up to the query block
+        }
+        return I;
+    };
+    // which tensor maps / head columns the resident and streamed "a" (Q/K side) and "b" (V/dCtx side) tiles use
+    const CUtensorMap* map_ra = MODE == 0 ? &P.map_k : &P.map_q;
+    const CUtensorMap* map_rb = MODE == 0 ? &P.map_v : &P.map_do;
+    const CUtensorMap* map_sa = MODE == 0 ? &P.map_q : &P.map_k;
+    const CUtensorMap* map_sb = MODE == 0 ? &P.map_do : &P.map_v;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t g = 0, ri = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
+                const BItem I = decode(it);
+                const int qoff = P.heads.qk_off[I.h], voff = P.heads.vo_off[I.h];
+                const int nba = (P.heads.qk_w[I.h] + 63) >> 6, nbb = (P.heads.vo_w[I.h] + 63) >> 6;
+                const int row0 = I.b * P.seq;
+                const uint32_t rs = ri % RS;
+                if (!(ok = mbar_wait(r_empty(rs), ((ri / RS) & 1u) ^ 1u, abort_flag, kCodeBase, P.status, P.wait_limit_ns))) break;
+                mbar_expect_tx(r_full(rs), (nba + nbb) * kBlockBytes);
+                for (int blk = 0; blk < nba; ++blk)
+                    tma_load_2d(sRes + (2 * rs) * kTileBytes + blk * kBlockBytes, map_ra, qoff + 64 * blk, row0 + I.own * kTile, r_full(rs));
+                for (int blk = 0; blk < nbb; ++blk)
+                    tma_load_2d(sRes + (2 * rs + 1) * kTileBytes + blk * kBlockBytes, map_rb, voff + 64 * blk, row0 + I.own * kTile, r_full(rs));
+                for (int i = 0; i < I.n_steps; ++i, ++g) {
+                    const uint32_t st = g % SS;
+                    if (!(ok = mbar_wait(t_empty(st), ((g / SS) & 1u) ^ 1u, abort_flag, kCodeBase, P.status, P.wait_limit_ns))) break;
+                    mbar_expect_tx(t_full(st), (nba + nbb) * kBlockBytes);
+                    const int y = row0 + (I.first + i) * kTile;
+                    for (int blk = 0; blk < nba; ++blk)
+                        tma_load_2d(sStr + (2 * st) * kTileBytes + blk * kBlockBytes, map_sa, qoff + 64 * blk, y, t_full(st));
+                    for (int blk = 0; blk < nbb; ++blk)
+                        tma_load_2d(sStr + (2 * st + 1) * kTileBytes + blk * kBlockBytes, map_sb, voff + 64 * blk, y, t_full(st));
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t g = 0, ri = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
+                const BItem I = decode(it);
+                const int wa = P.heads.qk_w[I.h], wb = P.heads.vo_w[I.h];
+                const uint32_t rs = ri % RS;
+                if (!(ok = mbar_wait(r_full(rs), (ri / RS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                const uint32_t idesc_x = make_idesc(kTile, kTile, 0, 0);
+                // X = Ra Sa^T (contraction over the Q/K width), Y = Rb Sb^T (over the V width) of step gg
+                auto issue_scores = [&](uint32_t gg) -> bool {
+                    const uint32_t st = gg % SS;
+                    if (!mbar_wait(t_full(st), (gg / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns)) return false;
+                    tc_fence_after();
+                    for (int ks = 0; ks < (wa >> 4); ++ks) {
+                        const uint32_t o = (ks >> 2) * kBlockBytes + (ks & 3) * 32;
+                        tc_mma_bf16(tmem_base + kColX, make_smem_desc(sRes + (2 * rs) * kTileBytes + o, 16, 1024),
+                                    make_smem_desc(sStr + (2 * st) * kTileBytes + o, 16, 1024), idesc_x, ks != 0 ? 1u : 0u);
+                    }
+                    for (int ks = 0; ks < (wb >> 4); ++ks) {
+                        const uint32_t o = (ks >> 2) * kBlockBytes + (ks & 3) * 32;
+                        tc_mma_bf16(tmem_base + kColY, make_smem_desc(sRes + (2 * rs + 1) * kTileBytes + o, 16, 1024),
+                                    make_smem_desc(sStr + (2 * st + 1) * kTileBytes + o, 16, 1024), idesc_x, ks != 0 ? 1u : 0u);
+                    }
+                    tc_commit(x_full);
+                    return true;
+                };
+                if (!(ok = issue_scores(g))) break;
+                for (int i = 0; i < I.n_steps; ++i, ++g) {
+                    if (!(ok = mbar_wait(out_full, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                    tc_fence_after();
+                    // with two stages the next step's score products go first, so that the compute warps can start on them
+                    // while the accumulating products of this step run
+                    if (SS > 1 && i + 1 < I.n_steps && !(ok = issue_scores(g + 1))) break;
+                    if (i == 0) {   // the accumulators of the previous item have been read out
+                        if (!(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                        tc_fence_after();
+                    }
+                    const uint32_t st = g % SS;
+                    if (MODE == 0) {   // dV += P^T dCtx_i : B = streamed b tile, MN-major, N = V width
+                        const uint32_t idesc = make_idesc(kTile, wb, 0, 1);
+                        for (int ks = 0; ks < kTile / 16; ++ks)
+                            tc_mma_bf16(tmem_base + kColAcc1, make_smem_desc(sOut + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
+                                        make_smem_desc(sStr + (2 * st + 1) * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc,
+                                        (i | ks) != 0 ? 1u : 0u);
+                    }
+                    {   // dK += dS^T Q_i  (MODE 1: dQ += dS K_j): B = streamed a tile, MN-major, N = Q/K width
+                        const uint32_t idesc = make_idesc(kTile, wa, 0, 1);
+                        const uint32_t sA = sOut + (MODE == 0 ? 2 * kBlockBytes : 0);
+                        for (int ks = 0; ks < kTile / 16; ++ks)
+                            tc_mma_bf16(tmem_base + kColAcc2, make_smem_desc(sA + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
+                                        make_smem_desc(sStr + (2 * st) * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc,
+                                        (i | ks) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(out_empty);
+                    tc_commit(t_empty(st));
+                    // with one stage the next step's tiles can only be loaded once these products have released it
+                    if (SS == 1 && i + 1 < I.n_steps && !(ok = issue_scores(g + 1))) break;
+                }
+                if (ok) {
+                    tc_commit(acc_full);
+                    tc_commit(r_empty(rs));
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ compute, thread = row of the owned block
+        const int tid = threadIdx.x - 64;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const uint32_t out_row = sOut + row * 128;
+        const int swz = row & 7;
+        uint32_t g = 0, ri = 0;
+        bool ok = true;
+        const int64_t T = static_cast<int64_t>(P.batch) * P.seq;
+        constexpr float kLog2e = 1.4426950408889634f;
+        for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
+            const BItem I = decode(it);
+            const int own_pos = I.own * kTile + row;                 // position of this thread's row in the sequence
+            const float* lse_h = P.lse + static_cast<int64_t>(I.h) * T + static_cast<int64_t>(I.b) * P.seq;
+            const float* d_h = P.dvec + static_cast<int64_t>(I.h) * T + static_cast<int64_t>(I.b) * P.seq;
+            float lse_r = 0.f, d_r = 0.f;       // MODE 1: this row's values.  MODE 0: the next query block's value of column tid
+            if (MODE == 1) {
+                if (own_pos < P.seq) {
+                    lse_r = lse_h[own_pos] * kLog2e;
+                    d_r = d_h[own_pos];
+                }
+            } else {
+                const int qp = I.first * kTile + tid;
+                if (qp < P.seq) {
+                    lse_r = lse_h[qp] * kLog2e;
+                    d_r = d_h[qp];
+                }
+            }
+            for (int i = 0; i < I.n_steps; ++i, ++g) {
+                const int other0 = (I.first + i) * kTile;            // first position of the streamed block
+                float* vb = vec + (g & 1) * 2 * kTile;
+                if (MODE == 0) {
+                    vb[tid] = lse_r;
+                    vb[kTile + tid] = d_r;
+                    mbar_arrive(vec_ready);     // (a bounded wait instead of a block barrier: a thread that gave up is not waited for)
+                    if (!(ok = mbar_wait(vec_ready, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+                    lse_r = d_r = 0.f;
+                    const int qp = other0 + kTile + tid;             // prefetch for the next query block
+                    if (i + 1 < I.n_steps && qp < P.seq) {
+                        lse_r = lse_h[qp] * kLog2e;
+                        d_r = d_h[qp];
+                    }
+                }
+                if (!(ok = mbar_wait(x_full, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                // (query position, key position) of element (row, column c): MODE 0 rows are keys, MODE 1 rows are queries
+                const int q0 = MODE == 0 ? other0 : I.own * kTile, k0 = MODE == 0 ? I.own * kTile : other0;
+                const bool masked = q0 + kTile > P.seq || k0 + kTile > P.seq || (P.causal && q0 < k0 + kTile);
+#pragma unroll 1
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t rx[32], ry[32];
+                    tc_ld32(t_lane + kColX + c * 32, rx);
+                    tc_ld32(t_lane + kColY + c * 32, ry);
+                    tc_wait_ld();
+                    float p[32], ds[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const int col = c * 32 + e;
+                        const float l2 = MODE == 0 ? vb[col] : lse_r;
+                        const float dd = MODE == 0 ? vb[kTile + col] : d_r;
+                        float pe = ex2(fmaf(__uint_as_float(rx[e]), P.scale_log2e, -l2));
+                        if (masked) {
+                            const int qp = MODE == 0 ? q0 + col : own_pos;
+                            const int kp = MODE == 0 ? own_pos : k0 + col;
+                            const bool valid = qp < P.seq && kp < P.seq && (!P.causal || kp <= qp);
+                            pe = valid ? pe : 0.f;
+                        }
+                        p[e] = pe;
+                        ds[e] = pe * (__uint_as_float(ry[e]) - dd);
+                    }
+                    if (c == 0) {   // the products that read the previous step's tiles from shared memory are done
+                        if (!(ok = mbar_wait(out_empty, (g & 1u) ^ 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+                    }
+                    const uint32_t blk = out_row + (c >> 1) * kBlockBytes;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const int chunk = (c & 1) * 4 + q;
+                        if (MODE == 0)
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(blk + ((chunk ^ swz) << 4)),
+                                         "r"(pack_bf16(p[8 * q + 0], p[8 * q + 1])), "r"(pack_bf16(p[8 * q + 2], p[8 * q + 3])),
+                                         "r"(pack_bf16(p[8 * q + 4], p[8 * q + 5])), "r"(pack_bf16(p[8 * q + 6], p[8 * q + 7]))
+                                         : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(blk + (MODE == 0 ? 2 * kBlockBytes : 0) + ((chunk ^ swz) << 4)),
+                                     "r"(pack_bf16(ds[8 * q + 0], ds[8 * q + 1])), "r"(pack_bf16(ds[8 * q + 2], ds[8 * q + 3])),
+                                     "r"(pack_bf16(ds[8 * q + 4], ds[8 * q + 5])), "r"(pack_bf16(ds[8 * q + 6], ds[8 * q + 7]))
+                                     : "memory");
+                    }
+                }
+                if (!ok) break;
+                fence_async_smem();
+                tc_fence_before();
+                mbar_arrive(out_full);
+            }
+            if (!ok) break;
+            // the accumulators of this item are complete: write them out
+            if (!(ok = mbar_wait(acc_full, ri & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+            tc_fence_after();
+            const bool live = own_pos < P.seq;
+            const int64_t t = static_cast<int64_t>(I.b) * P.seq + own_pos;
+            auto write_acc = [&](uint32_t col0, int w, uint16_t* dst, float mul) {
+#pragma unroll
+                for (int c = 0; c < NB * 4; ++c) {
+                    if (c * 16 < w) {
+                        uint32_t r[16];
+                        tc_ld16(t_lane + col0 + c * 16, r);
+                        tc_wait_ld();
+                        if (live) {
+                            uint4 v0, v1;
+                            v0.x = pack_bf16(__uint_as_float(r[0]) * mul, __uint_as_float(r[1]) * mul);
+                            v0.y = pack_bf16(__uint_as_float(r[2]) * mul, __uint_as_float(r[3]) * mul);
+                            v0.z = pack_bf16(__uint_as_float(r[4]) * mul, __uint_as_float(r[5]) * mul);
+                            v0.w = pack_bf16(__uint_as_float(r[6]) * mul, __uint_as_float(r[7]) * mul);
+                            v1.x = pack_bf16(__uint_as_float(r[8]) * mul, __uint_as_float(r[9]) * mul);
+                            v1.y = pack_bf16(__uint_as_float(r[10]) * mul, __uint_as_float(r[11]) * mul);
+                            v1.z = pack_bf16(__uint_as_float(r[12]) * mul, __uint_as_float(r[13]) * mul);
+                            v1.w = pack_bf16(__uint_as_float(r[14]) * mul, __uint_as_float(r[15]) * mul);
+                            *reinterpret_cast<uint4*>(dst + c * 16) = v0;
+                            *reinterpret_cast<uint4*>(dst + c * 16 + 8) = v1;
+                        }
+                    }
+                }
+            };
+            if (MODE == 0) {
+                write_acc(kColAcc1, P.heads.vo_w[I.h], P.dv + t * P.ld_dv + P.heads.vo_off[I.h], 1.f);
+                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dk + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale);
+            } else {
+                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale);
+            }
+            tc_fence_before();
+            mbar_arrive(acc_empty);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                              const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                              CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeFn attn_encode_fn() {
+    static EncodeFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeFn>(p);
+    });
+    return fn;
+}
+// bf16 row-major (rows x cols, pitch ld) as tiles of 64 columns x 128 rows, 128-byte swizzle, zero fill outside
+ecospa_status_t encode_tile_map(CUtensorMap* out, const void* ptr, int64_t rows, int64_t cols, int64_t ld) {
+    EncodeFn enc = attn_encode_fn();
+    if (!enc) {
+        set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
+        return ECOSPA_ERR_CUDA;
+    }
+    const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+    const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(kTile)};
+    const cuuint32_t estr[2] = {1, 1};
+    if (enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+        set_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled (attention)");
+        return ECOSPA_ERR_CUDA;
+    }
+    return ECOSPA_OK;
+}
+
+// Host-only checks shared by the forward and the backward call; fills the layout and the total widths.
+ecospa_status_t check_heads(const ecospa_heads_t* heads, HeadLayout& L, int64_t& n_qk, int64_t& n_vo, int& max_w) {
+    if (!heads || !heads->qk_off || !heads->qk_w || !heads->vo_off || !heads->vo_w) return ECOSPA_ERR_INVALID;
+    if (heads->n_heads < 1) return ECOSPA_ERR_INVALID;
+    if (heads->n_heads > kMaxHeads) return ECOSPA_ERR_UNSUPPORTED;
+    n_qk = n_vo = 0;
+    max_w = 0;
+    for (int h = 0; h < heads->n_heads; ++h) {
+        const int32_t qo = heads->qk_off[h], qw = heads->qk_w[h], vo = heads->vo_off[h], vw = heads->vo_w[h];
+        if (qo < 0 || vo < 0 || qw < 1 || vw < 1) return ECOSPA_ERR_INVALID;
+        if (qw > 128 || vw > 128) return ECOSPA_ERR_UNSUPPORTED;
+        if ((qw & 15) || (vw & 15) || (qo & 7) || (vo & 7)) return ECOSPA_ERR_ALIGNMENT;
+        L.qk_off[h] = qo; L.qk_w[h] = qw; L.vo_off[h] = vo; L.vo_w[h] = vw;
+        n_qk = std::max<int64_t>(n_qk, qo + qw);
+        n_vo = std::max<int64_t>(n_vo, vo + vw);
+        max_w = std::max(max_w, std::max(qw, vw));
+    }
+    return ECOSPA_OK;
+}
+ecospa_status_t check_mat(const void* p, int64_t ld, int64_t cols) {
+    if (!p || ld < cols) return ECOSPA_ERR_INVALID;
+    if (!aligned16(p) || (ld * 2) % 16) return ECOSPA_ERR_ALIGNMENT;
+    return ECOSPA_OK;
+}
+
+template <typename Params>
+size_t fwd_smem_bytes(int nb) { return static_cast<size_t>(6 * nb + 2) * kBlockBytes + 1024 + 256; }
+
+}  // namespace
+
+}  // namespace ecospa
+
+using namespace ecospa;
+
+extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* Kc, int64_t ld_qk, const void* Vc, int64_t ld_v,
+                                                   int64_t batch, int64_t seq, const ecospa_heads_t* heads, float scale,
+                                                   int32_t causal, void* Ctx, int64_t ld_ctx, float* lse, void* stream) {
+    static thread_local AttnFwdParams P;
+    int64_t n_qk = 0, n_vo = 0;
+    int max_w = 0;
+    ecospa_status_t st = check_heads(heads, P.heads, n_qk, n_vo, max_w);
+    if (st != ECOSPA_OK) return st;
+    if (batch < 1 || seq < 1 || batch * seq > INT32_MAX || !lse) return ECOSPA_ERR_INVALID;
+    if (!(scale > 0.f) || !std::isfinite(scale)) return ECOSPA_ERR_INVALID;
+    if ((st = check_mat(Qc, ld_qk, n_qk)) != ECOSPA_OK || (st = check_mat(Kc, ld_qk, n_qk)) != ECOSPA_OK ||
+        (st = check_mat(Vc, ld_v, n_vo)) != ECOSPA_OK || (st = check_mat(Ctx, ld_ctx, n_vo)) != ECOSPA_OK)
+        return st;
+    if (reinterpret_cast<uintptr_t>(lse) & 3u) return ECOSPA_ERR_ALIGNMENT;
+    int* status = engine_status_ptr(&st);
+    if (!status) return st;
+    const int64_t T = batch * seq;
+    if ((st = encode_tile_map(&P.map_q, Qc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_k, Kc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_v, Vc, T, n_vo, ld_v)) != ECOSPA_OK) return st;
+    P.batch = static_cast<int32_t>(batch);
+    P.seq = static_cast<int32_t>(seq);
+    P.n_heads = heads->n_heads;
+    P.n_qt = static_cast<int32_t>(ceil_div(seq, kTile));
+    P.causal = causal != 0;
+    const int64_t items = static_cast<int64_t>(P.n_qt) * P.n_heads * batch;
+    if (items > INT32_MAX) return ECOSPA_ERR_UNSUPPORTED;
+    P.n_items = static_cast<int32_t>(items);
+    P.scale_log2e = scale * 1.4426950408889634f;
+    P.ctx = static_cast<uint16_t*>(Ctx);
+    P.ld_ctx = ld_ctx;
+    P.lse = lse;
+    P.status = status;
+    P.wait_limit_ns = engine_wait_limit_ns();
+    const int nb = max_w > 64 ? 2 : 1;
+    const size_t smem = fwd_smem_bytes<AttnFwdParams>(nb);
+    static std::once_flag once[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaError_t e = cudaSuccess;
+    std::call_once(once[dev & 63], [&] {
+        e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fwd_smem_bytes<AttnFwdParams>(1)));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fwd_smem_bytes<AttnFwdParams>(2)));
+    });
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "attention setup");
+        cudaGetLastError();
+        return ECOSPA_ERR_CUDA;
+    }
+    const int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
+    if (nb == 1) attn_fwd_kernel<1><<<grid, kFwdThreads, smem, static_cast<cudaStream_t>(stream)>>>(P);
+    else attn_fwd_kernel<2><<<grid, kFwdThreads, smem, static_cast<cudaStream_t>(stream)>>>(P);
+    return check_launch("attn_fwd_kernel");
+}
+
+extern "C" size_t ecospa_attn_workspace_bytes(int64_t batch, int64_t seq, int32_t n_heads) {
+    if (batch < 1 || seq < 1 || n_heads < 1) return 0;
+    return static_cast<size_t>(batch) * seq * n_heads * 4 + 256;      // the row dots D, one fp32 per (head, token)
+}
+
+extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* Kc, int64_t ld_qk, const void* Vc, int64_t ld_v,
+                                                   const void* Ctx, int64_t ld_ctx, const void* dCtx, int64_t ld_dctx,
+                                                   const float* lse, int64_t batch, int64_t seq, const ecospa_heads_t* heads,
+                                                   float scale, int32_t causal, void* dQc, void* dKc, int64_t ld_dqk,
+                                                   void* dVc, int64_t ld_dv, void* workspace, size_t workspace_bytes,
+                                                   void* stream_) {
+    static thread_local AttnBwdParams P;
+    static thread_local DotParams D;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    int64_t n_qk = 0, n_vo = 0;
+    int max_w = 0;
+    ecospa_status_t st = check_heads(heads, P.heads, n_qk, n_vo, max_w);
+    if (st != ECOSPA_OK) return st;
+    if (batch < 1 || seq < 1 || batch * seq > INT32_MAX || !lse) return ECOSPA_ERR_INVALID;
+    if (!(scale > 0.f) || !std::isfinite(scale)) return ECOSPA_ERR_INVALID;
+    if ((st = check_mat(Qc, ld_qk, n_qk)) != ECOSPA_OK || (st = check_mat(Kc, ld_qk, n_qk)) != ECOSPA_OK ||
+        (st = check_mat(Vc, ld_v, n_vo)) != ECOSPA_OK || (st = check_mat(Ctx, ld_ctx, n_vo)) != ECOSPA_OK ||
+        (st = check_mat(dCtx, ld_dctx, n_vo)) != ECOSPA_OK || (st = check_mat(dQc, ld_dqk, n_qk)) != ECOSPA_OK ||
+        (st = check_mat(dKc, ld_dqk, n_qk)) != ECOSPA_OK || (st = check_mat(dVc, ld_dv, n_vo)) != ECOSPA_OK)
+        return st;
+    if (reinterpret_cast<uintptr_t>(lse) & 3u) return ECOSPA_ERR_ALIGNMENT;
+    if (n_vo / 8 > kDotMaxVecs) return ECOSPA_ERR_UNSUPPORTED;
+    if (!workspace || workspace_bytes < ecospa_attn_workspace_bytes(batch, seq, heads->n_heads)) return ECOSPA_ERR_WORKSPACE;
+    if (!aligned16(workspace)) return ECOSPA_ERR_ALIGNMENT;
+    int* status = engine_status_ptr(&st);
+    if (!status) return st;
+    const int64_t T = batch * seq;
+    if ((st = encode_tile_map(&P.map_q, Qc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_k, Kc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_v, Vc, T, n_vo, ld_v)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_do, dCtx, T, n_vo, ld_dctx)) != ECOSPA_OK) return st;
+    float* dvec = static_cast<float*>(workspace);
+    P.batch = static_cast<int32_t>(batch);
+    P.seq = static_cast<int32_t>(seq);
+    P.n_heads = heads->n_heads;
+    P.n_t = static_cast<int32_t>(ceil_div(seq, kTile));
+    P.causal = causal != 0;
+    const int64_t items = static_cast<int64_t>(P.n_t) * P.n_heads * batch;
+    if (items > INT32_MAX) return ECOSPA_ERR_UNSUPPORTED;
+    P.n_items = static_cast<int32_t>(items);
+    P.scale = scale;
+    P.scale_log2e = scale * 1.4426950408889634f;
+    P.lse = lse;
+    P.dvec = dvec;
+    P.dq = static_cast<uint16_t*>(dQc);
+    P.dk = static_cast<uint16_t*>(dKc);
+    P.dv = static_cast<uint16_t*>(dVc);
+    P.ld_dqk = ld_dqk;
+    P.ld_dv = ld_dv;
+    P.status = status;
+    P.wait_limit_ns = engine_wait_limit_ns();
+    static std::once_flag once[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaError_t e = cudaSuccess;
+    std::call_once(once[dev & 63], [&] {
+        e = cudaFuncSetAttribute(attn_bwd_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<1, 0>::kSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<2, 0>::kSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<1, 1>::kSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<2, 1>::kSmem);
+    });
+    if (e != cudaSuccess) {
+        set_cuda_error(e, "attention backward setup");
+        cudaGetLastError();
+        return ECOSPA_ERR_CUDA;
+    }
+    // row dots D
+    D.heads = P.heads;
+    D.ctx = static_cast<const uint16_t*>(Ctx);
+    D.dctx = static_cast<const uint16_t*>(dCtx);
+    D.out = dvec;
+    D.ld_ctx = ld_ctx;
+    D.ld_dctx = ld_dctx;
+    D.T = T;
+    D.n_heads = heads->n_heads;
+    D.n_vecs = static_cast<int32_t>(n_vo / 8);
+    attn_rowdot_kernel<<<static_cast<unsigned>(ceil_div(T, kDotWarps)), 32 * kDotWarps, 0, stream>>>(D);
+    if ((st = check_launch("attn_rowdot_kernel")) != ECOSPA_OK) return st;
+    const int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
+    const int nb = max_w > 64 ? 2 : 1;
+    if (nb == 1) attn_bwd_kernel<1, 0><<<grid, kFwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
+    else attn_bwd_kernel<2, 0><<<grid, kFwdThreads, BwdCfg<2, 0>::kSmem, stream>>>(P);
+    if ((st = check_launch("attn_bwd_kernel (dK, dV)")) != ECOSPA_OK) return st;
+    if (nb == 1) attn_bwd_kernel<1, 1><<<grid, kFwdThreads, BwdCfg<1, 1>::kSmem, stream>>>(P);
+    else attn_bwd_kernel<2, 1><<<grid, kFwdThreads, BwdCfg<2, 1>::kSmem, stream>>>(P);
+    return check_launch("attn_bwd_kernel (dQ)");
+}

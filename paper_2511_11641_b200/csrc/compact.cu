@@ -54,7 +54,8 @@ __device__ __forceinline__ void cols_tile(const GatherJob& J, int local) {
 #pragma unroll
     for (int e = 0; e < V; ++e) {
         const int c = c0 + e;
-        idx[e] = c < J.n_kept ? min(max(__ldg(J.kept + c), 0), J.D - 1) : -1;
+        const int kc = c < J.n_kept ? __ldg(J.kept + c) : -1;      // -1 = no index: a zero column
+        idx[e] = kc < 0 ? -1 : min(kc, J.D - 1);
     }
     const E* in = static_cast<const E*>(J.in);
     E* out = static_cast<E*>(J.out);
@@ -105,9 +106,14 @@ __device__ __forceinline__ void rows_tile(const GatherJob& J, int local) {
     for (int rr = warp; rr < kRowTile; rr += kWarps) {
         const int r = local * kRowTile + rr;
         if (r >= J.n_kept) break;
-        const int src_row = min(max(__ldg(J.kept + r), 0), J.D - 1);
-        const char* src = static_cast<const char*>(J.in) + src_row * pitch_in;
+        const int kr = __ldg(J.kept + r);
         char* dst = static_cast<char*>(J.out) + r * pitch_out;
+        if (kr < 0) {                                              // no index: a zero row
+            for (int64_t b = 2 * lane; b < row_bytes + pad_bytes; b += 64) *reinterpret_cast<uint16_t*>(dst + b) = 0;
+            continue;
+        }
+        const int src_row = min(kr, J.D - 1);
+        const char* src = static_cast<const char*>(J.in) + src_row * pitch_in;
         int64_t done = 0;
         if (J.aligned) {
             const int nvec = static_cast<int>(row_bytes / 16);

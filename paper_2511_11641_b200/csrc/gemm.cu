@@ -1373,6 +1373,17 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
     return check_launch("gemm_kernel");
 }
 
+int* engine_status_ptr(ecospa_status_t* st) {
+    DeviceState* dev = gemm_setup(st);
+    return dev ? dev->status_ptr : nullptr;
+}
+int engine_num_sms() {
+    ecospa_status_t st;
+    DeviceState* dev = gemm_setup(&st);
+    return dev ? dev->num_sms : 0;
+}
+unsigned long long engine_wait_limit_ns() { return g_wait_limit_ns.load(std::memory_order_relaxed); }
+
 int gemm_resident_pairs() {
     ecospa_status_t st;
     DeviceState* dev = gemm_setup(&st);

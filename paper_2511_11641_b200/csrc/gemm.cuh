@@ -64,6 +64,12 @@ ecospa_status_t launch_grouped_gemm(const GemmOp* ops, int n_ops, cudaStream_t s
 // pitch); makes no CUDA call.  Calls that enqueue several launches check all of them before the first.
 ecospa_status_t validate_gemm_ops(const GemmOp* ops, int n_ops);
 
+// What the other tensor-core kernels of the library share with the engine: the current device's status word (device
+// pointer; nullptr with *st set when no device can be used), its SM count, and the limit of device-side waits.
+int* engine_status_ptr(ecospa_status_t* st);
+int engine_num_sms();
+unsigned long long engine_wait_limit_ns();
+
 // CTA pairs the engine keeps resident on the current device (0: pair mode off, -1: no usable device).
 int gemm_resident_pairs();
 

@@ -349,11 +349,37 @@ __global__ void __launch_bounds__(128) pack_kept_kernel(const __grid_constant__ 
     for (int i = threadIdx.x; i < P.k[s]; i += blockDim.x) P.out[P.dst[s] + i] = P.slots[P.src[s] + i] + P.add[s];
 }
 
+// Kept list with padded segments: the k[s] entries of segment s, then -1 ("no index") up to its padded count
+// (carried in the `add` slot of the parameters).
+__global__ void __launch_bounds__(128) pad_kept_kernel(const __grid_constant__ PackParams P) {
+    const int s = blockIdx.x;
+    for (int i = threadIdx.x; i < P.add[s]; i += blockDim.x) P.out[P.dst[s] + i] = i < P.k[s] ? P.slots[P.src[s] + i] : -1;
+}
+
 }  // namespace
 
 }  // namespace ecospa
 
 using namespace ecospa;
+
+extern "C" ecospa_status_t ecospa_pad_kept(const int32_t* kept, const int32_t* src, const int32_t* dst, const int32_t* k,
+                                           const int32_t* k_padded, int32_t n_segs, int32_t* out, void* stream) {
+    if (!kept || !src || !dst || !k || !k_padded || !out || n_segs < 1) return ECOSPA_ERR_INVALID;
+    for (int i = 0; i < n_segs; ++i)
+        if (src[i] < 0 || dst[i] < 0 || k[i] < 0 || k_padded[i] < k[i]) return ECOSPA_ERR_INVALID;
+    static thread_local PackParams pp;
+    for (int base = 0; base < n_segs; base += kPackSegs) {
+        const int n = std::min(kPackSegs, n_segs - base);
+        pp.slots = kept; pp.out = out; pp.n = n;
+        for (int i = 0; i < n; ++i) {
+            pp.src[i] = src[base + i]; pp.dst[i] = dst[base + i]; pp.k[i] = k[base + i]; pp.add[i] = k_padded[base + i];
+        }
+        pad_kept_kernel<<<n, 128, 0, static_cast<cudaStream_t>(stream)>>>(pp);
+        const ecospa_status_t st = check_launch("pad_kept_kernel");
+        if (st != ECOSPA_OK) return st;
+    }
+    return ECOSPA_OK;
+}
 
 extern "C" ecospa_status_t ecospa_pack_kept(const int32_t* slots, const int32_t* src, const int32_t* dst, const int32_t* k,
                                             const int32_t* add, int32_t n_segs, int32_t* out, void* stream) {

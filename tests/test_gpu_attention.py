@@ -1,0 +1,205 @@
+"""GPU parity of the attention core on compacted heads (through the C ABI) vs the fp64 oracle.
+
+Tolerance: relative Frobenius error <= 2e-2 per head and sequence for Ctx and for dQ, dK, dV (bf16 operands and bf16
+probabilities on the tensor cores, fp32 accumulation and softmax; the oracle works in fp64 on the same bf16 inputs);
+the log-sum-exp within 2e-3 absolute.  Small cases are compared in full; the LLaMA-1B-sized case on sampled
+(sequence, head) pairs, each of which is an independent sub-problem.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2511_11641_b200 import binding as B
+from paper_2511_11641_b200 import block as BL
+from paper_2511_11641_b200 import workloads as WL
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+TOL = 2e-2
+
+
+def make_inputs(batch, seq, k_qk, k_vo, seed=0, with_grad=False):
+    """bf16 Q, K, V (and dCtx) in the padded layout: head h has k real columns followed by zero columns up to the
+    next multiple of 16; a few extra columns of pitch beyond the last head hold a canary value."""
+    qo, qw, nq = BL.padded_head_layout(k_qk)
+    vo, vw, nv = BL.padded_head_layout(k_vo)
+    T = batch * seq
+    g = torch.Generator().manual_seed(seed)
+
+    def fill(n, off, k):
+        t = torch.zeros((T, n + 8), dtype=torch.bfloat16)
+        for h in range(len(k)):
+            t[:, off[h]: off[h] + k[h]] = torch.randn((T, k[h]), generator=g).to(torch.bfloat16)
+        return t
+
+    d = {"Q": fill(nq, qo, k_qk), "K": fill(nq, qo, k_qk), "V": fill(nv, vo, k_vo)}
+    if with_grad:
+        d["dCtx"] = fill(nv, vo, k_vo)
+    return d, (qo, qw, nq), (vo, vw, nv)
+
+
+def rel(a, b):
+    return float(np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-300))
+
+
+def run_forward(batch, seq, k_qk, k_vo, causal, seed=0, d_h=64):
+    d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, k_qk, k_vo, seed)
+    T = batch * seq
+    dd = {k: v.to(DEV) for k, v in d.items()}
+    Ctx = torch.full((T, nv + 8), 7.0, dtype=torch.bfloat16, device=DEV)
+    lse = torch.full((len(k_qk) * T + 16,), -3.0, dtype=torch.float32, device=DEV)
+    hd = B.heads(qo, qw, vo, vw)
+    scale = 1.0 / np.sqrt(d_h)
+    B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, hd, scale, causal, Ctx, lse)
+    B.ecospa_device_status()
+    ref = O.attn_fwd(d["Q"], d["K"], d["V"], batch, seq, qo, k_qk, vo, k_vo, scale, causal)
+    got = Ctx.double().cpu().numpy()
+    for h in range(len(k_qk)):
+        for b in range(batch):
+            rows = slice(b * seq, (b + 1) * seq)
+            cols = slice(vo[h], vo[h] + k_vo[h])
+            e = rel(got[rows, cols], ref["Ctx"][rows, cols])
+            assert e <= TOL, f"Ctx head {h} sequence {b}: {e}"
+            per_row = np.linalg.norm(got[rows, cols] - ref["Ctx"][rows, cols], axis=1) / np.linalg.norm(ref["Ctx"][rows, cols], axis=1)
+            assert per_row.max() <= 3 * TOL, f"Ctx head {h} sequence {b}: worst row {per_row.argmax()} {per_row.max()}"
+        # pad columns of the head come out as zeros (zero V columns), nothing else is written
+        assert np.all(got[:, vo[h] + k_vo[h]: vo[h] + vw[h]] == 0)
+    assert torch.all(Ctx[:, nv:] == 7.0), "columns past the last head must stay untouched"
+    got_lse = lse[: len(k_qk) * T].double().cpu().numpy().reshape(len(k_qk), T)
+    np.testing.assert_allclose(got_lse, ref["lse"], rtol=0, atol=2e-3)
+    assert torch.all(lse[len(k_qk) * T:] == -3.0)
+    return dd, d, Ctx, lse, hd, scale
+
+
+RAGGED = WL.RAGGED_HEAD_KEPT      # 20, 21, 25, 26, 30, 37, 64: widths the paper's compressed GPT-2-Small shows
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("seq", [77, 128, 300])
+def test_forward_ragged_heads_small(seq, causal):
+    k_qk = [RAGGED[i % len(RAGGED)] for i in range(9)]
+    k_vo = [RAGGED[(i + 3) % len(RAGGED)] for i in range(9)]
+    run_forward(2, seq, k_qk, k_vo, causal, seed=seq)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_wide_heads(causal):
+    """Heads of a 128-wide architecture (LLaMA-7B shape): widths above 64 take two column blocks per tile."""
+    run_forward(2, 200, [96, 128, 72, 33, 64], [128, 17, 100, 64, 80], causal, seed=5, d_h=128)
+
+
+def test_forward_block_config_in_full():
+    """The one-block configuration (4 heads x 64, batch 4 x seq 128, 50 %: 32 of 64 kept) in full."""
+    for causal in (False, True):
+        run_forward(4, 128, [32] * 4, [32] * 4, causal, seed=1)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_llama1b_sized_sampled_heads(causal):
+    """batch 4 x seq 2048, 32 heads with the paper's ragged widths: sampled (sequence, head) pairs in full."""
+    batch, seq, H = 4, 2048, 32
+    k_qk = [RAGGED[i % len(RAGGED)] for i in range(H)]
+    k_vo = [RAGGED[(i + 2) % len(RAGGED)] for i in range(H)]
+    d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, k_qk, k_vo, seed=11)
+    T = batch * seq
+    dd = {k: v.to(DEV) for k, v in d.items()}
+    Ctx = torch.zeros((T, nv + 8), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+    scale = 0.125
+    B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, B.heads(qo, qw, vo, vw), scale, causal, Ctx, lse)
+    B.ecospa_device_status()
+    got = Ctx.double().cpu().numpy()
+    got_lse = lse.double().cpu().numpy().reshape(H, T)
+    for b, h in ((0, 0), (3, 6), (1, 17), (2, 31)):
+        rows = slice(b * seq, (b + 1) * seq)
+        q = d["Q"][rows, qo[h]: qo[h] + k_qk[h]].contiguous()
+        k = d["K"][rows, qo[h]: qo[h] + k_qk[h]].contiguous()
+        v = d["V"][rows, vo[h]: vo[h] + k_vo[h]].contiguous()
+        ref = O.attn_fwd(q, k, v, 1, seq, [0], [k_qk[h]], [0], [k_vo[h]], scale, causal)
+        e = rel(got[rows, vo[h]: vo[h] + k_vo[h]], ref["Ctx"])
+        assert e <= TOL, (b, h, e)
+        np.testing.assert_allclose(got_lse[h, rows], ref["lse"][0], rtol=0, atol=2e-3)
+
+
+# ---------------------------------------------------------------------------------------------
+# backward
+# ---------------------------------------------------------------------------------------------
+
+def run_backward(batch, seq, k_qk, k_vo, causal, seed=0, d_h=64):
+    d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, k_qk, k_vo, seed, with_grad=True)
+    T, H = batch * seq, len(k_qk)
+    dd = {k: v.to(DEV) for k, v in d.items()}
+    Ctx = torch.zeros((T, nv + 8), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+    hd = B.heads(qo, qw, vo, vw)
+    scale = 1.0 / np.sqrt(d_h)
+    B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, hd, scale, causal, Ctx, lse)
+    full = lambda n: torch.full((T, n + 8), 7.0, dtype=torch.bfloat16, device=DEV)
+    dQ, dK, dV = full(nq), full(nq), full(nv)
+    ws = torch.empty(B.ecospa_attn_workspace_bytes(batch, seq, H), dtype=torch.uint8, device=DEV)
+    B.ecospa_coupled_attn_bwd(dd["Q"], dd["K"], dd["V"], Ctx, dd["dCtx"], lse, batch, seq, hd, scale, causal, dQ, dK, dV, ws)
+    B.ecospa_device_status()
+    ref = O.attn_bwd(d["Q"], d["K"], d["V"], d["dCtx"], batch, seq, qo, k_qk, vo, k_vo, scale, causal)
+    for name, got_t, off, k, wpad, n in (("dQ", dQ, qo, k_qk, qw, nq), ("dK", dK, qo, k_qk, qw, nq), ("dV", dV, vo, k_vo, vw, nv)):
+        got = got_t.double().cpu().numpy()
+        for h in range(H):
+            for b in range(batch):
+                rows = slice(b * seq, (b + 1) * seq)
+                cols = slice(off[h], off[h] + k[h])
+                e = rel(got[rows, cols], ref[name][rows, cols])
+                assert e <= TOL, f"{name} head {h} sequence {b}: {e}"
+            assert np.all(got[:, off[h] + k[h]: off[h] + wpad[h]] == 0), f"{name}: pad columns of head {h}"
+        assert torch.all(got_t[:, n:] == 7.0), f"{name}: columns past the last head must stay untouched"
+    return dQ, dK, dV
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("seq", [77, 128, 300])
+def test_backward_ragged_heads_small(seq, causal):
+    k_qk = [RAGGED[i % len(RAGGED)] for i in range(9)]
+    k_vo = [RAGGED[(i + 3) % len(RAGGED)] for i in range(9)]
+    run_backward(2, seq, k_qk, k_vo, causal, seed=seq + 1)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_wide_heads(causal):
+    run_backward(2, 200, [96, 128, 72, 33, 64], [128, 17, 100, 64, 80], causal, seed=6, d_h=128)
+
+
+def test_backward_block_config_in_full_and_bit_identical_reruns():
+    for causal in (False, True):
+        a = run_backward(4, 128, [32] * 4, [32] * 4, causal, seed=2)
+        b = run_backward(4, 128, [32] * 4, [32] * 4, causal, seed=2)
+        for x, y in zip(a, b):
+            assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_llama1b_sized_sampled_heads(causal):
+    batch, seq, H = 4, 2048, 32
+    k_qk = [RAGGED[i % len(RAGGED)] for i in range(H)]
+    k_vo = [RAGGED[(i + 2) % len(RAGGED)] for i in range(H)]
+    d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, k_qk, k_vo, seed=12, with_grad=True)
+    T = batch * seq
+    dd = {k: v.to(DEV) for k, v in d.items()}
+    Ctx = torch.zeros((T, nv + 8), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+    hd = B.heads(qo, qw, vo, vw)
+    scale = 0.125
+    B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, hd, scale, causal, Ctx, lse)
+    z = lambda n: torch.zeros((T, n + 8), dtype=torch.bfloat16, device=DEV)
+    dQ, dK, dV = z(nq), z(nq), z(nv)
+    ws = torch.empty(B.ecospa_attn_workspace_bytes(batch, seq, H), dtype=torch.uint8, device=DEV)
+    B.ecospa_coupled_attn_bwd(dd["Q"], dd["K"], dd["V"], Ctx, dd["dCtx"], lse, batch, seq, hd, scale, causal, dQ, dK, dV, ws)
+    B.ecospa_device_status()
+    g = {"dQ": dQ.double().cpu().numpy(), "dK": dK.double().cpu().numpy(), "dV": dV.double().cpu().numpy()}
+    for b, h in ((0, 1), (3, 13), (2, 31)):
+        rows = slice(b * seq, (b + 1) * seq)
+        cq, cv = slice(qo[h], qo[h] + k_qk[h]), slice(vo[h], vo[h] + k_vo[h])
+        sub = lambda t, c: t[rows, c].contiguous()
+        ref = O.attn_bwd(sub(d["Q"], cq), sub(d["K"], cq), sub(d["V"], cv), sub(d["dCtx"], cv), 1, seq, [0], [k_qk[h]], [0],
+                         [k_vo[h]], scale, causal)
+        for name, c in (("dQ", cq), ("dK", cq), ("dV", cv)):
+            e = rel(g[name][rows, c], ref[name])
+            assert e <= TOL, (name, b, h, e)
