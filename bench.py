@@ -2,14 +2,16 @@
 
 One step = one pass of the whole hot path over every layer of the model:
   score (+ Fisher) of all coupled pairs -> aligned top-k -> compaction of weights, biases and
-  gradients -> forward and backward of every compacted QK / VO / FFN pair.
+  gradients -> forward and backward of every compacted block (Q/K/V projections, attention core on the
+  compacted heads, output projection, FFN).
 
     python bench.py --gpus 1 --steps 10 --warmup 3
     python bench.py --impl reference            # the CPU oracle on a bounded sample of the same step
 
 Prints one JSON line (rank 0).  `value` is the tensor-core throughput of the step (algorithmic
-flops of the compacted-pair GEMMs / whole step time); the memory-bound phase is reported
-alongside as GB/s.  With N > 1 every rank runs an independent replica (the path has no exchange
+flops of every product of the step / whole step time); the memory-bound phase is reported
+alongside as GB/s, and the projection / FFN products and the attention core are also replayed
+on their own for their rooflines.  With N > 1 every rank runs an independent replica (the path has no exchange
 step); times are the maximum over ranks.
 """
 from __future__ import annotations
@@ -48,6 +50,16 @@ def step_flops(wl, n_attn: int, k_ffn: int) -> float:
     ffn_mats = 3 if wl.ffn == "swiglu" else 2
     fwd = 2.0 * T * d * (2 * n_attn) + 2.0 * T * d * (2 * n_attn) + 2.0 * T * d * k_ffn * ffn_mats
     return 3.0 * fwd * wl.n_layers
+
+
+def attention_flops(wl, k_qk: int, k_vo: int, causal: bool) -> float:
+    """Products of the attention core on the compacted heads, all layers: forward S = Q K^T and P V (2 products),
+    backward S again, dP, dV, dQ, dK (5 products), 2*seq*seq*width flops each per sequence and head with the real
+    kept widths; a causal mask halves the pairs."""
+    pairs = wl.batch * wl.n_heads * float(wl.seq) * wl.seq * (0.5 if causal else 1.0)
+    fwd = 2.0 * pairs * (k_qk + k_vo)
+    bwd = 2.0 * pairs * (3 * k_qk + 2 * k_vo)
+    return (fwd + bwd) * wl.n_layers
 
 
 def sparsify_bytes(wl, rho: float, with_grads: bool = True, transposed: bool = False) -> float:
@@ -154,6 +166,15 @@ class Model:
         plan = WL.kept_plan(wl, sparsity)
         self.plan = plan
         self.n_attn, self.k_ffn = sum(plan["qk"]), plan["ffn"][0]
+        # The attention kernels want every head's block of Q^c, K^c, V^c padded to a multiple of 16 columns: the kept
+        # lists of the two attention groups are padded with "no index" entries (zero columns) before compaction.
+        self.qk_off, self.qk_w, self.n_qk_p = BL.padded_head_layout(plan["qk"])
+        self.vo_off, self.vo_w, self.n_vo_p = BL.padded_head_layout(plan["vo"])
+        assert self.n_qk_p == self.n_vo_p, "the benchmark keeps the same count in the QK and VO pair of a head"
+        self.n_attn_p = self.n_qk_p
+        self.padded = self.n_attn_p != self.n_attn
+        self.causal = True     # GPT-2- and LLaMA-shaped decoders mask keys after the query
+        self.scale = 1.0 / (wl.d_h ** 0.5)
         self.k_per_seg = (plan["qk"] + plan["vo"] + plan["ffn"]) * wl.n_layers
         self.n_seg = [wl.n_heads, wl.n_heads, 1] * wl.n_layers
         self.seg_len = [wl.d_h, wl.d_h, wl.d_ffn] * wl.n_layers
@@ -162,6 +183,8 @@ class Model:
         self.ups = torch.empty(D_layer * wl.n_layers, dtype=f32, device=device)
         self.fis = torch.empty((2 * wl.n_heads + 1) * wl.n_layers, dtype=f32, device=device)
         self.kept = torch.empty(sum(self.k_per_seg), dtype=i32, device=device)
+        # padded kept lists of the attention groups, layer after layer: [QK | VO]
+        self.kept_p = torch.empty(2 * self.n_attn_p * wl.n_layers, dtype=i32, device=device) if self.padded else None
         self.score_ws = torch.empty(B.ecospa_score_workspace_bytes(self.pairs), dtype=torch.uint8, device=device)
         # compaction jobs: weights, biases and gradients of every pair group
         self.c, self.jobs = [], []
@@ -173,21 +196,36 @@ class Model:
         layout = {"wq": lin, "wk": lin, "wv": lin, "wo": lout, "w1": lin, "w1b": lin, "w2": lout, "bq": 0, "bk": 0, "bv": 0,
                   "b1": 0, "gq": lin, "gk": lin, "gv": lin, "go": lout, "g1": lin, "g1b": lin, "g2": lout}
         self.layout = layout
+        self.pad_args = None
+        if self.padded:
+            src, dst, kk, kp = [], [], [], []
+            o_src, o_dst = 0, 0
+            for l in range(wl.n_layers):
+                for grp, widths in (("qk", self.qk_w), ("vo", self.vo_w)):
+                    for h in range(wl.n_heads):
+                        src.append(o_src); dst.append(o_dst); kk.append(plan[grp][h]); kp.append(widths[h])
+                        o_src += plan[grp][h]; o_dst += widths[h]
+                o_src += self.k_ffn
+            self.pad_args = (src, dst, kk, kp)
         for l in range(wl.n_layers):
             c = {}
-            for wn, gn, nk, D in groups:
+            for gi, (wn, gn, nk, D) in enumerate(groups):
                 kd = self.kept[off:off + nk]
+                nk_out = nk
+                if self.padded and gi < 2:
+                    nk_out = self.n_attn_p
+                    kd = self.kept_p[(2 * l + gi) * nk_out:(2 * l + gi + 1) * nk_out]
                 for nm in wn + gn:
                     src = self.w[l].get(nm) if nm in self.w[l] else self.g[l].get(nm)
                     if src is None:
                         continue
-                    o = BL.alloc_compacted(src, layout[nm], nk)
+                    o = BL.alloc_compacted(src, layout[nm], nk_out)
                     c[nm] = o
-                    self.jobs.append(B.gather(src, o, layout[nm], kd, nk, D))
+                    self.jobs.append(B.gather(src, o, layout[nm], kd, nk_out, D))
                 off += nk
             self.c.append(c)
         # activations and upstream gradients: a small pool of distinct sets cycled over the layers
-        T, d, n, k = wl.tokens, wl.d_m, self.n_attn, self.k_ffn
+        T, d, n, k = wl.tokens, wl.d_m, self.n_attn_p, self.k_ffn
         npad = BL.pad8(n)
         dt = wl.torch_dtype
         self.acts = []
@@ -200,6 +238,12 @@ class Model:
                   "dWv": e(n, d) if transposed else e(d, npad), "dWo": e(d, npad) if transposed else e(n, d),
                   "dbq": e(n), "dbk": e(n), "dbv": e(n), "dbo": e(d)}
         self.o["dX"].zero_()
+        # attention core: mixed values, their gradient, and the gradients it hands to the projections' backward
+        self.o.update({"Ctx": e(T, npad), "dQ": e(T, npad), "dK": e(T, npad), "dV": e(T, npad)})
+        self.lse = torch.empty(wl.n_heads * T, dtype=f32, device=device)
+        self.heads = B.heads(self.qk_off, self.qk_w, self.vo_off, self.vo_w)
+        self.attn_ws = torch.empty(B.ecospa_attn_workspace_bytes(wl.batch, wl.seq, wl.n_heads), dtype=torch.uint8, device=device)
+        self.has_attention = wl.torch_dtype == torch.bfloat16 and not transposed
         from paper_2511_11641_b200 import layers as L
         self.L = L
         self.act = B.ACT_SWIGLU if wl.ffn == "swiglu" else B.ACT_GELU_ERF
@@ -211,11 +255,54 @@ class Model:
         B = self.B
         B.ecospa_score_pairs(self.pairs, float(self.wl.tokens), self.ups, None, self.fis, self.score_ws)
         B.ecospa_select_aligned_topk(self.ups, self.n_seg, self.seg_len, self.k_per_seg, self.kept)
+        if self.padded:
+            B.ecospa_pad_kept(self.kept, *self.pad_args, self.kept_p)
         B.ecospa_compact_tensors(self.jobs)
 
+    def attention_fwd(self):
+        o, wl = self.o, self.wl
+        self.B.ecospa_coupled_attn_fwd(o["Q"], o["K"], o["V"], wl.batch, wl.seq, self.heads, self.scale, self.causal, o["Ctx"],
+                                       self.lse)
+
+    def attention_bwd(self):
+        o, wl = self.o, self.wl
+        self.B.ecospa_coupled_attn_bwd(o["Q"], o["K"], o["V"], o["Ctx"], o["dCtx"], self.lse, wl.batch, wl.seq, self.heads,
+                                       self.scale, self.causal, o["dQ"], o["dK"], o["dV"], self.attn_ws)
+
+    def block(self, l: int):
+        """Forward and backward of layer l as a training step meets them: Q, K, V projections -> attention core ->
+        output projection -> FFN forward and backward -> output projection backward -> attention backward ->
+        backward of the three projections.  Every call consumes what the previous one produced."""
+        B, o, n, k = self.B, self.o, self.n_attn_p, self.k_ffn
+        bias = self.wl.bias
+        c, a = self.c[l], self.acts[l % len(self.acts)]
+        B.ecospa_coupled_qkv_fwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, o["Q"], o["K"], o["V"], bq_c=c.get("bq"),
+                                 bk_c=c.get("bk"), bv_c=c.get("bv"), workspace=self.proj_ws, **self.lay)
+        self.attention_fwd()
+        B.ecospa_coupled_vo_fwd_o(o["Ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws, **self.lay)
+        self.L.ffn_fwd_bwd(a["x"], a["dy"], self.act, c["w1"], c["w2"], k, self.ffn, w1bc=c.get("w1b"),
+                           b1c=c.get("b1"), b2=self.w[l].get("b2"), **self.lay)
+        B.ecospa_coupled_vo_bwd_o(o["Ctx"], c["wo"], n, a["dout"], o["dCtx"], o["dWo"], o["dbo"] if bias else None,
+                                  workspace=self.proj_ws, **self.lay)
+        self.attention_bwd()
+        B.ecospa_coupled_qkv_bwd(a["x"], c["wq"], c["wk"], c["wv"], n, n, o["dQ"], o["dK"], o["dV"], o["dX"], o["dWq"],
+                                 o["dWk"], o["dWv"], o["dbq"] if bias else None, o["dbk"] if bias else None,
+                                 o["dbv"] if bias else None, accumulate_dX=True, workspace=self.proj_ws, **self.lay)
+
+    def blocks(self):
+        for l in range(self.wl.n_layers):
+            self.block(l)
+
+    def attention_only(self):
+        """The attention calls of a step on their own (for their share of the step time)."""
+        for l in range(self.wl.n_layers):
+            self.attention_fwd()
+            self.attention_bwd()
+
     def layer(self, l: int):
-        """Forward and backward of the compacted QK / VO / FFN pairs of layer l."""
-        B, o, n, k = self.B, self.o, self.n_attn, self.k_ffn
+        """Forward and backward of the compacted QK / VO / FFN pairs of layer l (the projections and the FFN only:
+        the attention-mixed values and the gradients of Q^c, K^c, V^c come from the input pool)."""
+        B, o, n, k = self.B, self.o, self.n_attn_p, self.k_ffn
         bias = self.wl.bias
         c, a = self.c[l], self.acts[l % len(self.acts)]
         # forward: Q, K, V in one launch; (attention core is the caller's); output projection; FFN
@@ -276,9 +363,13 @@ def tensor_peak(peaks, timed_ms: float, clocks) -> dict:
 
 
 def measure_step(m, args, world, rank, local, steps: int, graph: bool = True):
-    """Times `steps` passes of the whole hot path of model `m` (device-resident inputs): returns per-step
-    milliseconds of the whole step, the sparsify phase and the layer phase (CUDA events on the launching stream),
-    the clock record of the timed region, and the launches of one step."""
+    """Times `steps` passes of the whole hot path of model `m` (device-resident inputs), CUDA events on the launching
+    stream, barrier and synchronize on both sides of every timed region.
+    Region 1 (the step): score + select + compact, then every layer's block (projections, attention core, FFN, and
+      their backward) -> ms_step, ms_sp (the sparsify phase), ms_blocks.
+    Region 2: the projection / FFN products of every layer on their own (the launches of gemm_kernel) -> ms_gemm.
+    Region 3: the attention calls of every layer on their own -> ms_attn.
+    Each region has its own clock record; `launches` counts the library's launches of one step of region 1."""
     import torch
     import torch.distributed as dist
     B = m.B
@@ -290,47 +381,86 @@ def measure_step(m, args, world, rank, local, steps: int, graph: bool = True):
             dist.barrier()
             torch.cuda.synchronize()
 
+    full = m.blocks if m.has_attention else m.layers
     for _ in range(max(3, args.warmup)):
-        m.sparsify(); m.layers()
+        m.sparsify(); full(); m.layers()
     B.ecospa_device_status()
     # The calls are stateless and asynchronous, so a step can be captured once into CUDA graphs and
     # replayed: the launches of a step then cost no host time.  --no-graph issues them one by one.
     l0 = B.ecospa_launch_count()
+    fns = {"sparsify": m.sparsify, "blocks": full, "gemm": m.layers}
+    if m.has_attention:
+        fns["attn"] = m.attention_only
     if not graph:
-        sparsify, layers = m.sparsify, m.layers
-        m.sparsify(); m.layers()
+        m.sparsify(); full()
+        launches = B.ecospa_launch_count() - l0
     else:
-        g_sp, g_ly = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g_sp):
-            m.sparsify()
-        with torch.cuda.graph(g_ly):
-            m.layers()
-        sparsify, layers = g_sp.replay, g_ly.replay
-        m._graphs = (g_sp, g_ly)
-    launches = B.ecospa_launch_count() - l0
+        graphs = {}
+        for nm in ("sparsify", "blocks"):
+            graphs[nm] = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graphs[nm]):
+                fns[nm]()
+        launches = B.ecospa_launch_count() - l0
+        for nm in fns:
+            if nm not in graphs:
+                graphs[nm] = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graphs[nm]):
+                    fns[nm]()
+        fns = {nm: g.replay for nm, g in graphs.items()}
+        m._graphs = graphs
     for _ in range(2):
-        sparsify(); layers()
+        fns["sparsify"](); fns["blocks"]()
     B.ecospa_device_status()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
-    marks = []
-    barrier()
-    t_all0, t_all1 = ev(), ev()
-    t_all0.record()
-    for _ in range(steps):
-        e0, e1, e2 = ev(), ev(), ev()
-        e0.record(); sparsify(); e1.record(); layers(); e2.record()
-        marks.append((e0, e1, e2))
-    t_all1.record()
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
-    B.ecospa_device_status()
-    ms_total = t_all0.elapsed_time(t_all1)
-    ms_sp = sum(a.elapsed_time(b) for a, b, _ in marks) / steps
-    ms_gemm = sum(b.elapsed_time(c) for _, b, c in marks) / steps
-    return {"ms_step": ms_total / steps, "ms_sp": ms_sp, "ms_gemm": ms_gemm, "clocks": clocks, "launches": int(launches),
-            "replay": (sparsify, layers), "timed_ms": ms_total}
+
+    def region(seq_of_fns):
+        """steps x the given calls; returns (ms per step of the whole, ms per step of each call, clock record)."""
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        marks = []
+        barrier()
+        t0, t1 = ev(), ev()
+        t0.record()
+        for _ in range(steps):
+            es = [ev()]
+            es[0].record()
+            for f in seq_of_fns:
+                f()
+                es.append(ev()); es[-1].record()
+            marks.append(es)
+        t1.record()
+        barrier()
+        clocks = sampler.stop() if rank == 0 else None
+        B.ecospa_device_status()
+        parts = [sum(es[i].elapsed_time(es[i + 1]) for es in marks) / steps for i in range(len(seq_of_fns))]
+        return t0.elapsed_time(t1) / steps, parts, clocks, t0.elapsed_time(t1)
+
+    ms_step, (ms_sp, ms_blocks), clocks, timed_ms = region([fns["sparsify"], fns["blocks"]])
+    ms_gemm, _, clocks_gemm, timed_gemm = region([fns["gemm"]])
+    ms_attn, clocks_attn = None, None
+    if "attn" in fns:
+        ms_attn, _, clocks_attn, _ = region([fns["attn"]])
+    return {"ms_step": ms_step, "ms_sp": ms_sp, "ms_blocks": ms_blocks, "ms_gemm": ms_gemm, "ms_attn": ms_attn,
+            "clocks": clocks, "clocks_gemm": clocks_gemm, "clocks_attn": clocks_attn, "launches": int(launches),
+            "replay": (fns["sparsify"], fns["blocks"]), "timed_ms": timed_ms, "timed_gemm_ms": timed_gemm}
+
+
+def attention_report(wl, m, r):
+    """The attention core's share: algorithmic flops / its own replay time, and its exponentials against the
+    special-function rate of the part (one 2^x per query-key pair in the forward pass and in each of the two backward
+    kernels; 16 per clock per SM, 148 SMs, at the SM clock sampled during the region)."""
+    if r["ms_attn"] is None:
+        return None
+    fl = attention_flops(wl, m.plan["qk"][0], m.plan["vo"][0], m.causal)
+    pairs = wl.batch * wl.n_heads * float(wl.seq) * wl.seq * (0.5 if m.causal else 1.0) * wl.n_layers
+    sm = (r["clocks_attn"] or {}).get("sm_mhz") or 1965.0
+    exp_peak = 148 * 16 * sm * 1e6          # exponentials per second
+    return {"ms": r["ms_attn"], "TFLOP/s": fl / r["ms_attn"] / 1e9, "flops": fl, "frac_of_nominal_2250": fl / r["ms_attn"] / 1e9 / 2250.0,
+            "causal": m.causal, "head_widths": f"{m.plan['qk'][0]} of {wl.d_h} (padded to {m.qk_w[0]})",
+            "roofline": {"bound": "alu", "kernel": "attn_fwd_kernel + attn_bwd_kernel x2", "achieved": 3 * pairs / (r["ms_attn"] * 1e-3) / 1e12,
+                         "peak": exp_peak / 1e12, "unit": "T exp/s", "frac": 3 * pairs / (r["ms_attn"] * 1e-3) / exp_peak,
+                         "peak_source": f"16 ex2/clk/SM x 148 SMs x {sm:.0f} MHz (sampled)"},
+            "clocks": r["clocks_attn"]}
 
 
 def phase_report(wl, m, r, peaks, sparsity, transposed=False):
@@ -339,10 +469,13 @@ def phase_report(wl, m, r, peaks, sparsity, transposed=False):
     sbytes = sparsify_bytes(wl, 1.0 - sparsity, transposed=transposed)
     tf = flops / r["ms_gemm"] / 1e9
     gbs = sbytes / r["ms_sp"] / 1e6
-    tp = tensor_peak(peaks, r["timed_ms"], r["clocks"])
-    sm = (r["clocks"] or {}).get("sm_mhz")
+    tp = tensor_peak(peaks, r["timed_gemm_ms"], r["clocks_gemm"])
+    sm = (r["clocks_gemm"] or {}).get("sm_mhz")
+    afl = attention_flops(wl, m.plan["qk"][0], m.plan["vo"][0], m.causal) if m.has_attention else 0.0
     return {
         "workload": wl.name, "sparsity": sparsity, "ms_per_step": r["ms_step"],
+        "step_TFLOP/s": (flops + afl) / r["ms_step"] / 1e9, "blocks_ms": r["ms_blocks"],
+        "attention": attention_report(wl, m, r), "clocks_gemm": r["clocks_gemm"],
         "gemm_ms": r["ms_gemm"], "gemm_TFLOP/s": tf, "gemm_flops_per_step": flops,
         "gemm_frac_of_measured_burst": tf / peaks["bf16_tflops"],
         "gemm_frac_of_measured_sustained": tf / peaks["bf16_tflops_sustained"],
@@ -469,6 +602,7 @@ def parity_check(m, n_rows: int = 8):
     m.o["dX"].zero_()
     m.layer(0)
     B.ecospa_device_status()
+    kept_p_all = m.kept_p.cpu().numpy() if m.padded else None
     w = {k: v.cpu() for k, v in m.w[0].items()}
     D_attn = wl.n_heads * wl.d_h
     D_layer = 2 * D_attn + wl.d_ffn
@@ -489,6 +623,14 @@ def parity_check(m, n_rows: int = 8):
         kept_o = O.select_topk(ups[off_d:off_d + n_seg * seg_len], n_seg, seg_len, k)
         kept_g = kept_all[off_k:off_k + sum(k)]
         kept_equal = kept_equal and bool(np.array_equal(kept_o, kept_g))
+        if m.padded and n_seg > 1:
+            # the list the compaction used: every head's kept indices followed by "no index" entries up to its padded width
+            gi = 0 if n1 == "wq" else 1
+            kept_g = kept_p_all[gi * m.n_attn_p:(gi + 1) * m.n_attn_p]
+            widths = m.qk_w if gi == 0 else m.vo_w
+            exp = np.concatenate([np.concatenate([kept_o[sum(k[:h]):sum(k[:h + 1])], -np.ones(widths[h] - k[h], dtype=np.int32)])
+                                  for h in range(n_seg)])
+            kept_equal = kept_equal and bool(np.array_equal(exp, kept_g))
         kept_of[n1] = kept_g
         for nm, lay in ((n1, l1), (n2, l2), (n1b, l1)):
             if nm:
@@ -503,7 +645,7 @@ def parity_check(m, n_rows: int = 8):
     rt = torch.from_numpy(rows); rd = rt.to(m.dev)
     a = m.acts[0]
     c = {k: v.cpu() for k, v in m.c[0].items() if k in ("wq", "wk", "wv", "wo", "w1", "w1b", "w2", "bq", "bk", "bv", "b1")}
-    n, k = m.n_attn, m.k_ffn
+    n, k = m.n_attn_p, m.k_ffn
     X = a["x"][rd].cpu().contiguous()
 
     def row_err(got, ref):
@@ -530,7 +672,27 @@ def parity_check(m, n_rows: int = 8):
     errs["dX(ffn)"] = row_err(m.ffn["dX"][rd], rb["dX"])
     res["max_row_rel_err"] = errs
     res["rows_sampled"] = int(n_rows)
-    res["ok"] = bool(kept_equal and bytes_equal and score_err <= 1e-5 and all(v <= 2e-2 for v in errs.values()))
+    aerrs = {}
+    if m.has_attention:
+        # the chained block of layer 0, then one (sequence, head) pair of its attention core against the oracle
+        m.block(0)
+        B.ecospa_device_status()
+        b_s, h_s = wl.batch - 1, min(3, wl.n_heads - 1)
+        rows_s = slice(b_s * wl.seq, (b_s + 1) * wl.seq)
+        kq, kv = m.plan["qk"][h_s], m.plan["vo"][h_s]
+        cq = slice(m.qk_off[h_s], m.qk_off[h_s] + kq)
+        cv = slice(m.vo_off[h_s], m.vo_off[h_s] + kv)
+        sub = lambda t, c: t[rows_s, c].cpu().contiguous()
+        q, kk_, v, dc = sub(m.o["Q"], cq), sub(m.o["K"], cq), sub(m.o["V"], cv), sub(m.o["dCtx"], cv)
+        rf = O.attn_fwd(q, kk_, v, 1, wl.seq, [0], [kq], [0], [kv], m.scale, m.causal)
+        rb = O.attn_bwd(q, kk_, v, dc, 1, wl.seq, [0], [kq], [0], [kv], m.scale, m.causal)
+        fro = lambda got, ref: float(np.linalg.norm(got.double().cpu().numpy() - ref) / max(np.linalg.norm(ref), 1e-300))
+        aerrs = {"Ctx": fro(m.o["Ctx"][rows_s, cv], rf["Ctx"]), "dQ": fro(m.o["dQ"][rows_s, cq], rb["dQ"]),
+                 "dK": fro(m.o["dK"][rows_s, cq], rb["dK"]), "dV": fro(m.o["dV"][rows_s, cv], rb["dV"])}
+        res["attention_rel_frobenius"] = aerrs
+        res["attention_sample"] = f"sequence {b_s}, head {h_s} of layer 0, in full"
+    res["ok"] = bool(kept_equal and bytes_equal and score_err <= 1e-5 and all(v <= 2e-2 for v in errs.values())
+                     and all(v <= 2e-2 for v in aerrs.values()))
     return res
 
 
@@ -572,16 +734,17 @@ def run_gpu(args):
     host = m.host_copies()
     h2d = sum(h.numel() * h.element_size() for h, _ in host)
     m2 = Model(wl, args.sparsity, dev, transposed=args.transposed)
+    full2 = m2.blocks if m2.has_attention else m2.layers
     for _ in range(3):
-        m2.sparsify(); m2.layers()
+        m2.sparsify(); full2()
     if args.no_graph:
-        replay = [(sparsify, layers), (m2.sparsify, m2.layers)]
+        replay = [(sparsify, layers), (m2.sparsify, full2)]
     else:
         g2_sp, g2_ly = torch.cuda.CUDAGraph(), torch.cuda.CUDAGraph()
         with torch.cuda.graph(g2_sp):
             m2.sparsify()
         with torch.cuda.graph(g2_ly):
-            m2.layers()
+            full2()
         replay = [(sparsify, layers), (g2_sp.replay, g2_ly.replay)]
     models = [m, m2]
     dev_in = [[d for _, d in host], [t for dd in m2.w + m2.g + m2.acts for t in dd.values()]]
@@ -625,15 +788,21 @@ def run_gpu(args):
     if not args.no_graph:
         del g2_sp, g2_ly
 
-    ms_step, ms_sp, ms_gemm, ms_e2e = max_over_ranks([ms_step, ms_sp, ms_gemm, ms_e2e], dev)
+    ms_attn = r["ms_attn"] if r["ms_attn"] is not None else 0.0
+    ms_step, ms_sp, ms_gemm, ms_e2e, ms_attn, ms_blocks = max_over_ranks([ms_step, ms_sp, ms_gemm, ms_e2e, ms_attn, r["ms_blocks"]], dev)
+    r["ms_gemm"], r["ms_sp"], r["ms_step"], r["ms_blocks"] = ms_gemm, ms_sp, ms_step, ms_blocks
+    if r["ms_attn"] is not None:
+        r["ms_attn"] = ms_attn
 
-    flops = step_flops(wl, m.n_attn, m.k_ffn)
+    gemm_flops = step_flops(wl, m.n_attn, m.k_ffn)
+    attn_flops = attention_flops(wl, m.plan["qk"][0], m.plan["vo"][0], m.causal) if m.has_attention else 0.0
+    flops = gemm_flops + attn_flops            # every product of a step: projections, FFN, attention core
     sbytes = sparsify_bytes(wl, 1.0 - args.sparsity, transposed=args.transposed)
     peaks = measured_peaks()
     n_gemm_launches = wl.n_layers * 8
-    tf = flops / ms_gemm / 1e9
-    tp = tensor_peak(peaks, r["timed_ms"], clocks)
-    sm_mhz = (clocks or {}).get("sm_mhz")
+    tf = gemm_flops / ms_gemm / 1e9
+    tp = tensor_peak(peaks, r["timed_gemm_ms"], r["clocks_gemm"])
+    sm_mhz = (r["clocks_gemm"] or {}).get("sm_mhz")
     plain = not args.layers and args.sparsity == 0.5 and not args.transposed
     sp_traffic = NCU_SPARSIFY_TRAFFIC_BYTES_PER_LAYER.get(wl.name)
     out = {
@@ -653,7 +822,11 @@ def run_gpu(args):
                          "GB/s_if_every_tensor_counted_as_shared_rows": (2.0 + 4.0 * (1.0 - args.sparsity)) * WL.model_bytes(wl) / ms_sp / 1e6,
                          "frac_of_measured_hbm": sbytes / ms_sp / 1e6 / peaks["hbm_gbs"],
                          "frac_of_nominal_8TBs": sbytes / ms_sp / 1e6 / 8000.0},
-            "gemm": {"ms": ms_gemm, "TFLOP/s": tf, "flops": flops,
+            "blocks": {"ms": ms_blocks, "what": "every layer's projections, attention core, FFN and their backward, chained",
+                       "TFLOP/s": flops / ms_blocks / 1e9},
+            "attention": attention_report(wl, m, r),
+            "gemm": {"ms": ms_gemm, "TFLOP/s": tf, "flops": gemm_flops, "clocks": r["clocks_gemm"],
+                     "what": "the projection and FFN products of every layer replayed on their own (gemm_kernel launches)",
                      "frac_of_measured_burst": tf / peaks["bf16_tflops"],
                      "frac_of_measured_sustained": tf / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": tf / 2250.0,
@@ -664,7 +837,7 @@ def run_gpu(args):
         "roofline": {"bound": "tensor", "kernel": "gemm_kernel", "achieved": tf,
                      "peak": tp["peak"], "unit": "TFLOP/s", "frac": tf / tp["peak"],
                      "peak_source": f"{peaks['source']} cuBLAS bf16, {tp['which']} figure (timed region "
-                                    f"{r['timed_ms'] / 1e3:.2f} s, median SM clock {sm_mhz} MHz)",
+                                    f"{r['timed_gemm_ms'] / 1e3:.2f} s, median SM clock {sm_mhz} MHz)",
                      "frac_of_measured_burst": tf / peaks["bf16_tflops"],
                      "frac_of_measured_sustained": tf / peaks["bf16_tflops_sustained"],
                      "frac_of_nominal_2250": tf / 2250.0,
@@ -791,15 +964,28 @@ def cpu_sample(wl, sparsity: float, tokens: int = 256, threads: int = 1):
     chunks = max(1, min(threads, tokens))
     bounds = [(i * tokens // chunks, (i + 1) * tokens // chunks) for i in range(chunks)]
     run_all([(lambda lo=lo, hi=hi: do_rows(lo, hi)) for lo, hi in bounds if hi > lo])
+    # attention core: `threads` heads of one sequence truncated to s_a positions (causal), forward and backward
+    s_a = min(wl.seq, 256)
+    kq, kv = plan["qk"][0], plan["vo"][0]
+    aw = WL.activations(wl, 1, tokens=s_a, kinds=["dq", "dk", "dv", "ctx"], widths={kk: kq for kk in ("dq", "dk")} | {"dv": kv, "ctx": kv})
+
+    def do_head():
+        O.attn_fwd(aw["dq"], aw["dk"], aw["dv"], 1, s_a, [0], [kq], [0], [kv], 1.0 / wl.d_h ** 0.5, True)
+        O.attn_bwd(aw["dq"], aw["dk"], aw["dv"], aw["ctx"], 1, s_a, [0], [kq], [0], [kv], 1.0 / wl.d_h ** 0.5, True)
+
+    n_heads_a = max(1, threads)
+    run_all([do_head for _ in range(n_heads_a)])
     t2 = time.perf_counter()
     if pool is not None:
         pool.shutdown()
-    flops = step_flops(wl, n_attn, k_ffn) / wl.n_layers * tokens / wl.tokens
+    attn_fl = n_heads_a * 0.5 * s_a * s_a * 2.0 * ((kq + kv) + (3 * kq + 2 * kv))
+    flops = step_flops(wl, n_attn, k_ffn) / wl.n_layers * tokens / wl.tokens + attn_fl
     sbytes = sparsify_bytes(wl, 1.0 - sparsity) / wl.n_layers
     return {"value": flops / (t2 - t0) / 1e12, "unit": "TFLOP/s", "cores": threads, "kind": "oracle",
             "sample": f"layer 0 of {wl.name}: score+Fisher+select+compact at full size ({t1 - t0:.2f} s, "
                       f"{sbytes / (t1 - t0) / 1e9:.3f} GB/s), then fwd+bwd of the compacted QK/VO/FFN pairs on "
-                      f"{tokens} of {wl.tokens} tokens ({t2 - t1:.2f} s), {threads} thread(s)",
+                      f"{tokens} of {wl.tokens} tokens and of the attention core on {n_heads_a} head(s) x {s_a} positions "
+                      f"({t2 - t1:.2f} s), {threads} thread(s)",
             "seconds": t2 - t0, "gemm_tflops": flops / (t2 - t1) / 1e12, "sparsify_GB/s": sbytes / (t1 - t0) / 1e9}
 
 
@@ -842,9 +1028,7 @@ def run_reference(args):
     for _ in range(steps):
         last = cpu_sample(wl, args.sparsity, tokens)
     dt = (time.perf_counter() - t0) / steps
-    plan = WL.kept_plan(wl, args.sparsity)
-    flops = step_flops(wl, sum(plan["qk"]), plan["ffn"][0]) / wl.n_layers * tokens / wl.tokens
-    v = flops / dt / 1e12
+    v = last["value"] * last["seconds"] / dt     # the sample's flops over the mean step time
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": steps,
         "warmup": warm, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,

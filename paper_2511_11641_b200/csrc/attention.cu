@@ -8,16 +8,17 @@
 // Q K^T, and a zero column of V^c gives a zero column of Ctx) and off_h a multiple of 8, so that every tile load starts
 // on a 16-byte boundary and every contraction is a whole number of 16-deep MMA steps.
 //
-// Forward kernel, one CTA per SM, 192 threads.  A work item is (sequence b, head h, 128 query rows); a CTA walks a
+// Forward kernel, one CTA per SM, 576 threads.  A work item is (sequence b, head h, 128 query rows); a CTA walks a
 // static list of items (for causal attention the long ones first).
 //   warp 0      producer: one lane issues the TMA loads of the item's Q tile (2 buffers) and of every K / V tile
 //               (2 stages); a tile is one or two 64-column blocks of 128 rows x 128 bytes, 128-byte swizzle
 //   warp 1      owns TMEM (512 columns: two 128-column score buffers, one output tile of up to 128 columns); one lane
 //               issues S = Q K^T (K-major operands) and O_tile = P V (P from shared memory, V as stored = MN-major)
-//   warps 2..5  softmax, thread = query row (= TMEM lane): row maximum over the score tile, p = 2^(s*c - m) with the
+//   warps 2..17 softmax, thread = (query row = TMEM lane, quarter of the 128 key columns): row maximum over the score
+//               tile (the four threads of a row exchange their maxima through shared memory), p = 2^(s*c - m) with the
 //               running maximum m, P as bf16 into shared memory (K-major, swizzled) for the second product, and the
-//               running output O = O * 2^(m_old - m_new) + O_tile in registers; at the end O / l and the row's
-//               log-sum-exp are written
+//               running output O = O * 2^(m_old - m_new) + O_tile in registers (each thread its quarter of the columns);
+//               at the end O / l and the row's log-sum-exp are written
 // The score tile of key block j+1 is issued before P V of block j, so the tensor pipe works while the softmax of the
 // next block runs.  Every mbarrier wait is bounded; on expiry the CTA records a code (11 producer, 12 MMA issuer,
 // 13 softmax) in the device status word, lets copies land, frees TMEM and returns.
@@ -43,7 +44,9 @@ using namespace tc;
 constexpr int kTile = 128;                  // query rows and key rows per tile
 constexpr int kBlockBytes = kTile * 128;    // one 64-column block of a 128-row tile
 constexpr int kMaxHeads = 128;
-constexpr int kFwdThreads = 192;
+constexpr int kFwdParts = 4;
+constexpr int kFwdThreads = 64 + kFwdParts * 128;   // producer warp, MMA warp, four sets of four softmax warps
+constexpr int kBwdThreads = 64 + 4 * 128;   // producer warp, MMA warp, four sets of four compute warps
 constexpr int kTmemCols = 512;
 constexpr uint32_t kColS = 0, kColO = 256;  // TMEM columns: score buffers at 0 and 128, output tile at 256
 
@@ -80,22 +83,28 @@ __device__ __forceinline__ Item decode_item(int it, int n_qt, int n_heads, int b
 template <int NB>   // 64-column blocks per tile: 1 (every head at most 64 wide) or 2
 __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_constant__ AttnFwdParams P) {
     constexpr int kTileBytes = NB * kBlockBytes;
+    constexpr int QS = NB == 1 ? 2 : 1;                      // buffers of the Q tile (wide heads: one, to fit shared memory)
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw_addr);
-    const uint32_t sQ = base, sK = sQ + 2 * kTileBytes, sV = sK + 2 * kTileBytes, sP = sV + 2 * kTileBytes;
-    uint8_t* tail = smem + 6 * kTileBytes + 2 * kBlockBytes;
+    const uint32_t sQ = base, sK = sQ + QS * kTileBytes, sV = sK + 2 * kTileBytes, sP = sV + 2 * kTileBytes;
+    float* xchg = reinterpret_cast<float*>(smem + (QS + 4) * kTileBytes + 2 * kBlockBytes);   // [2 phases][4 parts][128 rows]
+    uint8_t* tail = smem + (QS + 4) * kTileBytes + 2 * kBlockBytes + 2 * kFwdParts * kTile * 4;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 16 * 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * 8 + 8);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 20 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 20 * 8 + 8);
     const uint32_t bar0 = smem_u32(bars);
     auto q_full = [&](uint32_t s) { return bar0 + 8u * s; };
     auto q_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };
-    auto kv_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
-    auto kv_empty = [&](uint32_t s) { return bar0 + 8u * (6 + s); };
+    // K and V tiles have rings of their own: a K stage is free as soon as the score product that read it is done (one
+    // step earlier than the V stage), so the load of the next K tile is not held up by the second product
+    auto k_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
+    auto k_empty = [&](uint32_t s) { return bar0 + 8u * (6 + s); };
     auto s_full = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
-    const uint32_t p_full = bar0 + 8u * 10, o_full = bar0 + 8u * 11;
+    const uint32_t p_full = bar0 + 8u * 10, o_full = bar0 + 8u * 11, x_ready = bar0 + 8u * 12;
+    auto v_full = [&](uint32_t s) { return bar0 + 8u * (13 + s); };
+    auto v_empty = [&](uint32_t s) { return bar0 + 8u * (15 + s); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_kt = (P.seq + kTile - 1) / kTile;
@@ -103,12 +112,15 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
         for (uint32_t s = 0; s < 2; ++s) {
             mbar_init(q_full(s), 1);
             mbar_init(q_empty(s), 1);
-            mbar_init(kv_full(s), 1);
-            mbar_init(kv_empty(s), 1);
+            mbar_init(k_full(s), 1);
+            mbar_init(k_empty(s), 1);
+            mbar_init(v_full(s), 1);
+            mbar_init(v_empty(s), 1);
             mbar_init(s_full(s), 1);
         }
-        mbar_init(p_full, 128);
+        mbar_init(p_full, kFwdThreads - 64);
         mbar_init(o_full, 1);
+        mbar_init(x_ready, kFwdThreads - 64);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.map_q);
@@ -131,19 +143,21 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                 const int qoff = P.heads.qk_off[I.h], voff = P.heads.vo_off[I.h];
                 const int nbq = (P.heads.qk_w[I.h] + 63) >> 6, nbv = (P.heads.vo_w[I.h] + 63) >> 6;
                 const int row0 = I.b * P.seq;
-                const uint32_t qs = qi & 1;
-                if (!(ok = mbar_wait(q_empty(qs), ((qi >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
+                const uint32_t qs = qi % QS;
+                if (!(ok = mbar_wait(q_empty(qs), ((qi / QS) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
                 mbar_expect_tx(q_full(qs), nbq * kBlockBytes);
                 for (int blk = 0; blk < nbq; ++blk)
                     tma_load_2d(sQ + qs * kTileBytes + blk * kBlockBytes, &P.map_q, qoff + 64 * blk, row0 + I.qt * kTile, q_full(qs));
                 for (int j = 0; j < I.n_kv; ++j, ++g) {
                     const uint32_t st = g & 1;
-                    if (!(ok = mbar_wait(kv_empty(st), ((g >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
-                    mbar_expect_tx(kv_full(st), (nbq + nbv) * kBlockBytes);
+                    if (!(ok = mbar_wait(k_empty(st), ((g >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
+                    mbar_expect_tx(k_full(st), nbq * kBlockBytes);
                     for (int blk = 0; blk < nbq; ++blk)
-                        tma_load_2d(sK + st * kTileBytes + blk * kBlockBytes, &P.map_k, qoff + 64 * blk, row0 + j * kTile, kv_full(st));
+                        tma_load_2d(sK + st * kTileBytes + blk * kBlockBytes, &P.map_k, qoff + 64 * blk, row0 + j * kTile, k_full(st));
+                    if (!(ok = mbar_wait(v_empty(st), ((g >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
+                    mbar_expect_tx(v_full(st), nbv * kBlockBytes);
                     for (int blk = 0; blk < nbv; ++blk)
-                        tma_load_2d(sV + st * kTileBytes + blk * kBlockBytes, &P.map_v, voff + 64 * blk, row0 + j * kTile, kv_full(st));
+                        tma_load_2d(sV + st * kTileBytes + blk * kBlockBytes, &P.map_v, voff + 64 * blk, row0 + j * kTile, v_full(st));
                 }
             }
         }
@@ -155,14 +169,14 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++qi) {
                 const Item I = decode_item(it, P.n_qt, P.n_heads, P.batch, n_kt, P.causal);
                 const int wq = P.heads.qk_w[I.h], wv = P.heads.vo_w[I.h];
-                const uint32_t qs = qi & 1;
-                if (!(ok = mbar_wait(q_full(qs), (qi >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                const uint32_t qs = qi % QS;
+                if (!(ok = mbar_wait(q_full(qs), (qi / QS) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
                 const uint32_t idesc_s = make_idesc(kTile, kTile, 0, 0);
                 const uint32_t idesc_o = make_idesc(kTile, wv, 0, 1);
                 // S = Q K^T of key block gg into score buffer gg & 1
                 auto issue_scores = [&](uint32_t gg) -> bool {
                     const uint32_t st = gg & 1;
-                    if (!mbar_wait(kv_full(st), (gg >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns)) return false;
+                    if (!mbar_wait(k_full(st), (gg >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns)) return false;
                     tc_fence_after();
                     for (int ks = 0; ks < (wq >> 4); ++ks) {
                         const uint32_t o = (ks >> 2) * kBlockBytes + (ks & 3) * 32;
@@ -170,30 +184,41 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                                     make_smem_desc(sK + st * kTileBytes + o, 16, 1024), idesc_s, ks != 0 ? 1u : 0u);
                     }
                     tc_commit(s_full(st));
+                    tc_commit(k_empty(st));
                     return true;
                 };
                 if (!(ok = issue_scores(g))) break;
                 for (int j = 0; j < I.n_kv; ++j, ++g) {
                     if (j + 1 < I.n_kv && !(ok = issue_scores(g + 1))) break;
                     if (!(ok = mbar_wait(p_full, g & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
-                    tc_fence_after();
                     const uint32_t st = g & 1;
+                    if (!(ok = mbar_wait(v_full(st), (g >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                    tc_fence_after();
                     for (int ks = 0; ks < kTile / 16; ++ks)   // O_tile = P V over the 128 keys of the block
                         tc_mma_bf16(tmem_base + kColO, make_smem_desc(sP + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
                                     make_smem_desc(sV + st * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc_o, ks != 0 ? 1u : 0u);
                     tc_commit(o_full);
-                    tc_commit(kv_empty(st));
+                    tc_commit(v_empty(st));
                 }
                 if (ok) tc_commit(q_empty(qs));
             }
         }
     } else {
-        // ------------------------------------------------------------------ softmax, thread = query row
+        // ------------------------------------------------------------------ softmax
+        // Thread = (query row, quarter of the key block's columns): warps 2..5 take columns [0, 32) of the 128 keys,
+        // warps 6..9 [32, 64), and so on, so every scheduler has four softmax warps to interleave.  A thread keeps its
+        // 32 scores in registers (one TMEM read per block).  The four threads of a row agree on the row maximum
+        // through shared memory once per key block; each keeps the sum of its own probabilities (added once, at the
+        // end) and folds its own quarter of the output columns.
+        const int part = (warp - 2) >> 2;
         const int row = (warp & 3) * 32 + lane;
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        const uint32_t p_row = sP + row * 128;
+        // this thread's 32 columns = four 16-byte chunks of block part / 2 of the row's image
+        const uint32_t p_row = sP + (part >> 1) * kBlockBytes + row * 128;
+        const int chunk0 = (part & 1) * 4;
         const int swz = row & 7;
-        uint32_t g = 0;
+        constexpr int kOwn = NB * 16;                                   // output columns this thread folds
+        uint32_t g = 0, xph = 0;
         bool ok = true;
         const int64_t T = static_cast<int64_t>(P.batch) * P.seq;
         for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x) {
@@ -202,45 +227,54 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             const int q_pos = I.qt * kTile + row;                     // position of this row in its sequence
             const int limit = P.causal ? min(P.seq, q_pos + 1) : P.seq;   // keys [0, limit) are visible
             float m = -INFINITY, l = 0.f, alpha_prev = 0.f;
-            float o[NB * 64];
+            float o[kOwn];
 #pragma unroll
-            for (int i = 0; i < NB * 64; ++i) o[i] = 0.f;
-            // O = O * a + O_tile (the output tile of the previous key block)
+            for (int i = 0; i < kOwn; ++i) o[i] = 0.f;
+            // O = O * a + O_tile (the output tile of the previous key block), this thread's columns
             auto fold_output = [&](float a) {
 #pragma unroll
-                for (int c = 0; c < NB * 4; ++c) {
-                    if (c * 16 < wv) {
+                for (int c = 0; c < NB; ++c) {
+                    const int col = part * kOwn + c * 16;
+                    if (col < wv) {
                         uint32_t r[16];
-                        tc_ld16(t_lane + kColO + c * 16, r);
+                        tc_ld16(t_lane + kColO + col, r);
                         tc_wait_ld();
 #pragma unroll
                         for (int i = 0; i < 16; ++i) o[c * 16 + i] = fmaf(o[c * 16 + i], a, __uint_as_float(r[i]));
                     }
                 }
             };
+            // values of the row's other threads: through xchg[phase & 1][part][row], one mbarrier phase per exchange
+            auto exchange = [&](float v, float (&others)[3]) -> bool {
+                float* buf = xchg + (xph & 1) * kFwdParts * kTile;
+                buf[part * kTile + row] = v;
+                mbar_arrive(x_ready);
+                if (!mbar_wait(x_ready, xph & 1u, abort_flag, 13, P.status, P.wait_limit_ns)) return false;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) others[k] = buf[((part + 1 + k) & 3) * kTile + row];
+                ++xph;
+                return true;
+            };
             for (int j = 0; j < I.n_kv; ++j, ++g) {
                 const uint32_t sb = g & 1;
                 if (!(ok = mbar_wait(s_full(sb), (g >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
                 tc_fence_after();
-                const uint32_t t_s = t_lane + kColS + sb * kTile;
-                const int kv0 = j * kTile;
-                const bool masked = kv0 + kTile > limit;
-                // pass 1: row maximum of this block
-                float mx = -INFINITY;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tc_ld32(t_s + c * 32, r);
-                    tc_wait_ld();
-                    if (masked) {
+                const int kv0 = j * kTile + part * 32;                // first key of this thread's columns
+                uint32_t r[32];
+                tc_ld32(t_lane + kColS + sb * kTile + part * 32, r);
+                tc_wait_ld();
+                if (kv0 + 32 > limit) {                               // keys past the limit count as -inf
 #pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (kv0 + c * 32 + i < limit) mx = fmaxf(mx, __uint_as_float(r[i]));
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(r[i]));
-                    }
+                    for (int i = 0; i < 32; ++i)
+                        if (kv0 + i >= limit) r[i] = 0xff800000u;
                 }
+                // maximum over this thread's columns (four independent chains), then over the row
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), mo[3];
+                if (!(ok = exchange(mx, mo))) break;
+                mx = fmaxf(fmaxf(mx, mo[0]), fmaxf(mo[1], mo[2]));
                 const float m_new = fmaxf(m, mx * P.scale_log2e);
                 const float alpha = ex2(m - m_new);
                 if (j > 0) {
@@ -248,35 +282,25 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                     tc_fence_after();
                     fold_output(alpha_prev);
                 }
-                // pass 2: p = 2^(s * c - m_new), row sum, P as bf16 into shared memory
-                float rs = 0.f;
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tc_ld32(t_s + c * 32, r);
-                    tc_wait_ld();
-                    float p[32];
+                // p = 2^(s * c - m_new) (2^-inf = 0 for the masked keys), row sum, P as bf16 into shared memory
+                float rs4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) {
-                        const float e = ex2(fmaf(__uint_as_float(r[i]), P.scale_log2e, -m_new));
-                        p[i] = (masked && kv0 + c * 32 + i >= limit) ? 0.f : e;
-                        rs += p[i];
-                    }
-                    // 32 columns = four 16-byte chunks of block c / 2; chunk q of a row sits at (q ^ (row & 7))
-                    const uint32_t blk = p_row + (c >> 1) * kBlockBytes;
+                for (int q = 0; q < 4; ++q) {
+                    float p[8];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int chunk = (c & 1) * 4 + q;
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(blk + ((chunk ^ swz) << 4)),
-                                     "r"(pack_bf16(p[8 * q + 0], p[8 * q + 1])), "r"(pack_bf16(p[8 * q + 2], p[8 * q + 3])),
-                                     "r"(pack_bf16(p[8 * q + 4], p[8 * q + 5])), "r"(pack_bf16(p[8 * q + 6], p[8 * q + 7]))
-                                     : "memory");
+                    for (int i = 0; i < 8; ++i) {
+                        p[i] = ex2(fmaf(__uint_as_float(r[8 * q + i]), P.scale_log2e, -m_new));
+                        rs4[i & 3] += p[i];
                     }
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_row + (((chunk0 + q) ^ swz) << 4)),
+                                 "r"(pack_bf16(p[0], p[1])), "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])),
+                                 "r"(pack_bf16(p[6], p[7]))
+                                 : "memory");
                 }
                 fence_async_smem();
                 tc_fence_before();
                 mbar_arrive(p_full);
-                l = fmaf(l, alpha, rs);
+                l = fmaf(l, alpha, (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
                 m = m_new;
                 alpha_prev = alpha;
             }
@@ -284,13 +308,22 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             if (!(ok = mbar_wait(o_full, (g - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
             tc_fence_after();
             fold_output(alpha_prev);
+            float lo[3];
+            if (!(ok = exchange(l, lo))) break;
+            {   // every thread of the row adds the four partial sums in the order of the parts
+                float lp[4];
+                lp[part] = l;
+#pragma unroll
+                for (int k = 0; k < 3; ++k) lp[(part + 1 + k) & 3] = lo[k];
+                l = (lp[0] + lp[1]) + (lp[2] + lp[3]);
+            }
             if (q_pos < P.seq) {
                 const int64_t t = static_cast<int64_t>(I.b) * P.seq + q_pos;
                 const float inv = 1.f / l;
-                uint16_t* dst = P.ctx + t * P.ld_ctx + P.heads.vo_off[I.h];
+                uint16_t* dst = P.ctx + t * P.ld_ctx + P.heads.vo_off[I.h] + part * kOwn;
 #pragma unroll
-                for (int c = 0; c < NB * 8; ++c) {
-                    if (c * 8 < wv) {
+                for (int c = 0; c < NB * 2; ++c) {
+                    if (part * kOwn + c * 8 < wv) {
                         uint4 v;
                         v.x = pack_bf16(o[c * 8 + 0] * inv, o[c * 8 + 1] * inv);
                         v.y = pack_bf16(o[c * 8 + 2] * inv, o[c * 8 + 3] * inv);
@@ -299,7 +332,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                         *reinterpret_cast<uint4*>(dst + c * 8) = v;
                     }
                 }
-                P.lse[static_cast<int64_t>(I.h) * T + t] = m * 0.6931471805599453f + logf(l);
+                if (part == 0) P.lse[static_cast<int64_t>(I.h) * T + t] = m * 0.6931471805599453f + logf(l);
             }
         }
     }
@@ -390,7 +423,8 @@ struct AttnBwdParams {
 // MODE 1: a CTA owns a query block and walks the key blocks: Q, dCtx resident, K_j and V_j streamed; X = S = Q K_j^T and
 //         Y = dP = dCtx V_j^T (thread = query row); dS goes to shared memory; dQ += dS K_j accumulates in TMEM.
 // Streamed tiles serve twice: as K-major B operands of the score products and as MN-major B operands of the
-// accumulating ones (same bytes, other descriptor).  Warp roles as in the forward kernel.  The score products of
+// accumulating ones (same bytes, other descriptor).  Warp roles as in the forward kernel, with sixteen compute warps
+// (thread = row, quarter of the columns).  The score products of
 // step i+1 are issued before the accumulating products of step i.  Wait codes: 14 / 15 / 16 (MODE 0 producer, issuer,
 // compute) and 17 / 18 / 19 (MODE 1).
 template <int NB, int MODE>
@@ -404,7 +438,7 @@ struct BwdCfg {
 };
 
 template <int NB, int MODE>
-__global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_constant__ AttnBwdParams P) {
+__global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ AttnBwdParams P) {
     using Cfg = BwdCfg<NB, MODE>;
     constexpr int kTileBytes = Cfg::kTileBytes;
     constexpr int RS = Cfg::kResStages, SS = Cfg::kStrStages;
@@ -439,11 +473,11 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_c
             mbar_init(t_empty(s), 1);
         }
         mbar_init(x_full, 1);
-        mbar_init(out_full, 128);
+        mbar_init(out_full, kBwdThreads - 64);
         mbar_init(out_empty, 1);
         mbar_init(acc_full, 1);
-        mbar_init(acc_empty, 128);
-        mbar_init(vec_ready, 128);
+        mbar_init(acc_empty, kBwdThreads - 64);
+        mbar_init(vec_ready, kBwdThreads - 64);   // every compute thread arrives: no waiter can fall two phases behind
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.map_q);
@@ -581,11 +615,16 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_c
             }
         }
     } else {
-        // ------------------------------------------------------------------ compute, thread = row of the owned block
-        const int tid = threadIdx.x - 64;
+        // ------------------------------------------------------------------ compute
+        // Thread = (row of the owned block = TMEM lane, quarter of the streamed block's 128 columns): warps 2..5 take
+        // columns [0, 32), warps 6..9 [32, 64), and so on, so every scheduler has four compute warps to interleave.
+        const int part = (warp - 2) >> 2;
         const int row = (warp & 3) * 32 + lane;
+        const int col0 = part * 32;                                    // this thread's columns of the streamed block
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        const uint32_t out_row = sOut + row * 128;
+        // 32 columns = four 16-byte chunks of block col0 / 64 of the row's image
+        const uint32_t out_row = sOut + (col0 >> 6) * kBlockBytes + row * 128;
+        const int chunk0 = (col0 & 63) >> 3;
         const int swz = row & 7;
         uint32_t g = 0, ri = 0;
         bool ok = true;
@@ -596,14 +635,16 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_c
             const int own_pos = I.own * kTile + row;                 // position of this thread's row in the sequence
             const float* lse_h = P.lse + static_cast<int64_t>(I.h) * T + static_cast<int64_t>(I.b) * P.seq;
             const float* d_h = P.dvec + static_cast<int64_t>(I.h) * T + static_cast<int64_t>(I.b) * P.seq;
-            float lse_r = 0.f, d_r = 0.f;       // MODE 1: this row's values.  MODE 0: the next query block's value of column tid
+            // MODE 1: this row's log-sum-exp (base 2) and row dot.  MODE 0 (threads of part 0 only): the values of
+            // query `row` of the next query block, fetched one step ahead and staged in shared memory for all rows.
+            float lse_r = 0.f, d_r = 0.f;
             if (MODE == 1) {
                 if (own_pos < P.seq) {
                     lse_r = lse_h[own_pos] * kLog2e;
                     d_r = d_h[own_pos];
                 }
-            } else {
-                const int qp = I.first * kTile + tid;
+            } else if (part == 0) {
+                const int qp = I.first * kTile + row;
                 if (qp < P.seq) {
                     lse_r = lse_h[qp] * kLog2e;
                     d_r = d_h[qp];
@@ -613,15 +654,20 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_c
                 const int other0 = (I.first + i) * kTile;            // first position of the streamed block
                 float* vb = vec + (g & 1) * 2 * kTile;
                 if (MODE == 0) {
-                    vb[tid] = lse_r;
-                    vb[kTile + tid] = d_r;
-                    mbar_arrive(vec_ready);     // (a bounded wait instead of a block barrier: a thread that gave up is not waited for)
+                    if (part == 0) {
+                        vb[row] = lse_r;
+                        vb[kTile + row] = d_r;
+                    }
+                    mbar_arrive(vec_ready);
+                    // (a bounded wait instead of a block barrier: a thread that gave up is not waited for)
                     if (!(ok = mbar_wait(vec_ready, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
-                    lse_r = d_r = 0.f;
-                    const int qp = other0 + kTile + tid;             // prefetch for the next query block
-                    if (i + 1 < I.n_steps && qp < P.seq) {
-                        lse_r = lse_h[qp] * kLog2e;
-                        d_r = d_h[qp];
+                    if (part == 0) {
+                        lse_r = d_r = 0.f;
+                        const int qp = other0 + kTile + row;         // prefetch for the next query block
+                        if (i + 1 < I.n_steps && qp < P.seq) {
+                            lse_r = lse_h[qp] * kLog2e;
+                            d_r = d_h[qp];
+                        }
                     }
                 }
                 if (!(ok = mbar_wait(x_full, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
@@ -629,63 +675,72 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_c
                 // (query position, key position) of element (row, column c): MODE 0 rows are keys, MODE 1 rows are queries
                 const int q0 = MODE == 0 ? other0 : I.own * kTile, k0 = MODE == 0 ? I.own * kTile : other0;
                 const bool masked = q0 + kTile > P.seq || k0 + kTile > P.seq || (P.causal && q0 < k0 + kTile);
-#pragma unroll 1
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t rx[32], ry[32];
-                    tc_ld32(t_lane + kColX + c * 32, rx);
-                    tc_ld32(t_lane + kColY + c * 32, ry);
+                // two halves of 16 columns: probabilities and dS are packed to bf16 pairs as soon as they exist
+                uint32_t pk_p[16], pk_ds[16];
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    uint32_t rx[16], ry[16];
+                    tc_ld16(t_lane + kColX + col0 + 16 * hh, rx);
+                    tc_ld16(t_lane + kColY + col0 + 16 * hh, ry);
                     tc_wait_ld();
-                    float p[32], ds[32];
+                    if (masked) {                                     // pairs outside the mask count as -inf (p = 0)
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int col = c * 32 + e;
-                        const float l2 = MODE == 0 ? vb[col] : lse_r;
-                        const float dd = MODE == 0 ? vb[kTile + col] : d_r;
-                        float pe = ex2(fmaf(__uint_as_float(rx[e]), P.scale_log2e, -l2));
-                        if (masked) {
-                            const int qp = MODE == 0 ? q0 + col : own_pos;
-                            const int kp = MODE == 0 ? own_pos : k0 + col;
-                            const bool valid = qp < P.seq && kp < P.seq && (!P.causal || kp <= qp);
-                            pe = valid ? pe : 0.f;
+                        for (int e = 0; e < 16; ++e) {
+                            const int c = col0 + 16 * hh + e;
+                            const int qp = MODE == 0 ? q0 + c : own_pos;
+                            const int kp = MODE == 0 ? own_pos : k0 + c;
+                            if (!(qp < P.seq && kp < P.seq && (!P.causal || kp <= qp))) rx[e] = 0xff800000u;
                         }
-                        p[e] = pe;
-                        ds[e] = pe * (__uint_as_float(ry[e]) - dd);
                     }
-                    if (c == 0) {   // the products that read the previous step's tiles from shared memory are done
-                        if (!(ok = mbar_wait(out_empty, (g & 1u) ^ 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
-                    }
-                    const uint32_t blk = out_row + (c >> 1) * kBlockBytes;
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const int chunk = (c & 1) * 4 + q;
-                        if (MODE == 0)
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(blk + ((chunk ^ swz) << 4)),
-                                         "r"(pack_bf16(p[8 * q + 0], p[8 * q + 1])), "r"(pack_bf16(p[8 * q + 2], p[8 * q + 3])),
-                                         "r"(pack_bf16(p[8 * q + 4], p[8 * q + 5])), "r"(pack_bf16(p[8 * q + 6], p[8 * q + 7]))
-                                         : "memory");
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(blk + (MODE == 0 ? 2 * kBlockBytes : 0) + ((chunk ^ swz) << 4)),
-                                     "r"(pack_bf16(ds[8 * q + 0], ds[8 * q + 1])), "r"(pack_bf16(ds[8 * q + 2], ds[8 * q + 3])),
-                                     "r"(pack_bf16(ds[8 * q + 4], ds[8 * q + 5])), "r"(pack_bf16(ds[8 * q + 6], ds[8 * q + 7]))
-                                     : "memory");
+                    for (int e = 0; e < 16; e += 4) {
+                        float l2[4] = {lse_r, lse_r, lse_r, lse_r}, dd[4] = {d_r, d_r, d_r, d_r};
+                        if (MODE == 0) {
+                            const float4 a4 = *reinterpret_cast<const float4*>(vb + col0 + 16 * hh + e);
+                            const float4 b4 = *reinterpret_cast<const float4*>(vb + kTile + col0 + 16 * hh + e);
+                            l2[0] = a4.x; l2[1] = a4.y; l2[2] = a4.z; l2[3] = a4.w;
+                            dd[0] = b4.x; dd[1] = b4.y; dd[2] = b4.z; dd[3] = b4.w;
+                        }
+                        float pe[4], de[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            pe[u] = ex2(fmaf(__uint_as_float(rx[e + u]), P.scale_log2e, -l2[u]));
+                            de[u] = pe[u] * (__uint_as_float(ry[e + u]) - dd[u]);
+                        }
+                        pk_p[8 * hh + (e >> 1)] = pack_bf16(pe[0], pe[1]);
+                        pk_p[8 * hh + (e >> 1) + 1] = pack_bf16(pe[2], pe[3]);
+                        pk_ds[8 * hh + (e >> 1)] = pack_bf16(de[0], de[1]);
+                        pk_ds[8 * hh + (e >> 1) + 1] = pack_bf16(de[2], de[3]);
                     }
                 }
-                if (!ok) break;
+                // the products that read the previous step's tiles from shared memory are done
+                if (!(ok = mbar_wait(out_empty, (g & 1u) ^ 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const int chunk = chunk0 + q;
+                    if (MODE == 0)
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + ((chunk ^ swz) << 4)),
+                                     "r"(pk_p[4 * q + 0]), "r"(pk_p[4 * q + 1]), "r"(pk_p[4 * q + 2]), "r"(pk_p[4 * q + 3]) : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + (MODE == 0 ? 2 * kBlockBytes : 0) + ((chunk ^ swz) << 4)),
+                                 "r"(pk_ds[4 * q + 0]), "r"(pk_ds[4 * q + 1]), "r"(pk_ds[4 * q + 2]), "r"(pk_ds[4 * q + 3]) : "memory");
+                }
                 fence_async_smem();
                 tc_fence_before();
                 mbar_arrive(out_full);
             }
             if (!ok) break;
-            // the accumulators of this item are complete: write them out
+            // the accumulators of this item are complete: write them out (every thread its quarter of the columns)
             if (!(ok = mbar_wait(acc_full, ri & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
             tc_fence_after();
             const bool live = own_pos < P.seq;
             const int64_t t = static_cast<int64_t>(I.b) * P.seq + own_pos;
-            auto write_acc = [&](uint32_t col0, int w, uint16_t* dst, float mul) {
+            auto write_acc = [&](uint32_t colbase, int w, uint16_t* dst, float mul) {
 #pragma unroll
-                for (int c = 0; c < NB * 4; ++c) {
-                    if (c * 16 < w) {
+                for (int c = 0; c < NB; ++c) {
+                    const int col = part * (NB * 16) + c * 16;
+                    if (col < w) {
                         uint32_t r[16];
-                        tc_ld16(t_lane + col0 + c * 16, r);
+                        tc_ld16(t_lane + colbase + col, r);
                         tc_wait_ld();
                         if (live) {
                             uint4 v0, v1;
@@ -697,8 +752,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_bwd_kernel(const __grid_c
                             v1.y = pack_bf16(__uint_as_float(r[10]) * mul, __uint_as_float(r[11]) * mul);
                             v1.z = pack_bf16(__uint_as_float(r[12]) * mul, __uint_as_float(r[13]) * mul);
                             v1.w = pack_bf16(__uint_as_float(r[14]) * mul, __uint_as_float(r[15]) * mul);
-                            *reinterpret_cast<uint4*>(dst + c * 16) = v0;
-                            *reinterpret_cast<uint4*>(dst + c * 16 + 8) = v1;
+                            *reinterpret_cast<uint4*>(dst + col) = v0;
+                            *reinterpret_cast<uint4*>(dst + col + 8) = v1;
                         }
                     }
                 }
@@ -791,7 +846,7 @@ ecospa_status_t check_mat(const void* p, int64_t ld, int64_t cols) {
 }
 
 template <typename Params>
-size_t fwd_smem_bytes(int nb) { return static_cast<size_t>(6 * nb + 2) * kBlockBytes + 1024 + 256; }
+size_t fwd_smem_bytes(int nb) { return static_cast<size_t>((nb == 1 ? 6 : 5) * nb + 2) * kBlockBytes + 2 * kFwdParts * kTile * 4 + 1024 + 256; }
 
 }  // namespace
 
@@ -940,10 +995,10 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     if ((st = check_launch("attn_rowdot_kernel")) != ECOSPA_OK) return st;
     const int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
     const int nb = max_w > 64 ? 2 : 1;
-    if (nb == 1) attn_bwd_kernel<1, 0><<<grid, kFwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
-    else attn_bwd_kernel<2, 0><<<grid, kFwdThreads, BwdCfg<2, 0>::kSmem, stream>>>(P);
+    if (nb == 1) attn_bwd_kernel<1, 0><<<grid, kBwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
+    else attn_bwd_kernel<2, 0><<<grid, kBwdThreads, BwdCfg<2, 0>::kSmem, stream>>>(P);
     if ((st = check_launch("attn_bwd_kernel (dK, dV)")) != ECOSPA_OK) return st;
-    if (nb == 1) attn_bwd_kernel<1, 1><<<grid, kFwdThreads, BwdCfg<1, 1>::kSmem, stream>>>(P);
-    else attn_bwd_kernel<2, 1><<<grid, kFwdThreads, BwdCfg<2, 1>::kSmem, stream>>>(P);
+    if (nb == 1) attn_bwd_kernel<1, 1><<<grid, kBwdThreads, BwdCfg<1, 1>::kSmem, stream>>>(P);
+    else attn_bwd_kernel<2, 1><<<grid, kBwdThreads, BwdCfg<2, 1>::kSmem, stream>>>(P);
     return check_launch("attn_bwd_kernel (dQ)");
 }
