@@ -366,3 +366,35 @@ def attn_bwd(Q, K, V, dCtx, batch: int, seq: int, qk_off, qk_w, vo_off, vo_w, sc
                        _p(vw), C.c_int64(q.ld), C.c_int64(k.ld), C.c_int64(v.ld), C.c_int64(dc.ld), C.c_double(scale),
                        int(causal), _p(dQ), _p(dK), C.c_int64(dQ.shape[1]), _p(dV), C.c_int64(dV.shape[1]))
     return {"dQ": dQ, "dK": dK, "dV": dV}
+
+
+# ---------------------------------------------------------------------------
+# grouped-query attention: the pairs W_i^Q W_g(i)^K^T and W_g(i)^V W_i^O of "Extension to GQA"
+# ---------------------------------------------------------------------------
+
+def group_sum(c: np.ndarray, n_groups: int, rep: int, seg_len: int) -> np.ndarray:
+    """c holds one value per shared index of `n_groups * rep` heads stored side by side, the heads of a group next to
+    each other; returns, per group and index, the sum over the group's heads (length n_groups * seg_len)."""
+    c = np.asarray(c, dtype=np.float64)
+    assert c.size == n_groups * rep * seg_len
+    return c.reshape(n_groups, rep, seg_len).sum(axis=1).reshape(-1)
+
+
+def score_pair_gqa(w1, w2, layout1: int, layout2: int, n_groups: int, seg_len: int, rep1: int = 1, rep2: int = 1):
+    """(raw, upsilon) per K/V group.  The heads that share a K (or V) head share its removable index: removing index
+    j of group g removes it from every pair of the group at once, so the group is scored as ONE coupled pair whose
+    W_1 (rep1 > 1: the group's query heads, stacked) or W_2 (rep2 > 1: the group's W^O row blocks, side by side) is
+    the stack of the group's heads: the norm of index j on that side is the l2 norm over the whole stack."""
+    c1 = group_sum(sumsq_shared(w1, layout1), n_groups, rep1, seg_len)
+    c2 = group_sum(sumsq_shared(w2, layout2), n_groups, rep2, seg_len)
+    return upsilon(c1, c2, n_groups, seg_len)
+
+
+def fisher_pair_gqa(g1, g2, layout1: int, layout2: int, n_groups: int, seg_len: int, n_samples: float, rep1: int = 1,
+                    rep2: int = 1) -> np.ndarray:
+    """Eq. "importance" of the group's stacked pair: each side's mean squared gradient is taken over the whole stack."""
+    s1 = group_sum(sumsq_shared(g1, layout1), n_groups, rep1, seg_len).reshape(n_groups, seg_len).sum(axis=1)
+    s2 = group_sum(sumsq_shared(g2, layout2), n_groups, rep2, seg_len).reshape(n_groups, seg_len).sum(axis=1)
+    other1, _ = _shared_dims(g1, layout1)
+    other2, _ = _shared_dims(g2, layout2)
+    return 0.5 * (s1 / (other1 * rep1 * seg_len) + s2 / (other2 * rep2 * seg_len)) / n_samples
