@@ -81,6 +81,13 @@ typedef struct {
     int32_t rope;    /* ecospa_rope_t: rotary position embedding acts on this pair group's shared index (Q/K pairs) */
     ecospa_mat_t w1, w1b, w2;
     ecospa_mat_t g1, g1b, g2;
+    /* Grouped-query attention ("Extension to GQA": pairs W_i^Q W_g(i)^KT and W_g(i)^V W_i^O).  w1_rep > 1: w1 (and g1)
+     * hold w1_rep heads per segment, the heads of a group side by side -- shared extent w1_rep * n_seg * seg_len, head
+     * (s, r) in shared indices [(s*w1_rep + r)*seg_len, +seg_len) -- and the segment is scored as ONE pair whose W_1 is
+     * the stack of those heads: the norm of index j on that side is taken over all of them (removing index j removes
+     * it from every head of the group).  w2_rep likewise for w2 / g2 (the W^O row blocks of a V group).  0 and 1 both
+     * mean an ordinary pair.  Plain pairs without rotation pairs only. */
+    int32_t w1_rep, w2_rep;
 } ecospa_pair_t;
 
 /* One gather job of the compaction step: out = in restricted to the kept shared indices. */

@@ -40,7 +40,8 @@ class Mat(C.Structure):
 
 class Pair(C.Structure):
     _fields_ = [("kind", C.c_int32), ("n_seg", C.c_int32), ("seg_len", C.c_int32), ("rope", C.c_int32),
-                ("w1", Mat), ("w1b", Mat), ("w2", Mat), ("g1", Mat), ("g1b", Mat), ("g2", Mat)]
+                ("w1", Mat), ("w1b", Mat), ("w2", Mat), ("g1", Mat), ("g1b", Mat), ("g2", Mat),
+                ("w1_rep", C.c_int32), ("w2_rep", C.c_int32)]
 
 
 class Gather(C.Structure):
@@ -109,9 +110,10 @@ def mat(t: Optional[torch.Tensor], layout: int) -> Mat:
 
 
 def pair(kind: int, n_seg: int, seg_len: int, w1, w2, layout1: int, layout2: int, w1b=None,
-         g1=None, g2=None, g1b=None, rope: int = 0) -> Pair:
+         g1=None, g2=None, g1b=None, rope: int = 0, w1_rep: int = 1, w2_rep: int = 1) -> Pair:
+    """w1_rep / w2_rep > 1: grouped-query attention, that many heads per segment stacked on the W_1 / W_2 side."""
     p = Pair(kind, n_seg, seg_len, rope, mat(w1, layout1), mat(w1b, layout1), mat(w2, layout2),
-             mat(g1, layout1), mat(g1b, layout1), mat(g2, layout2))
+             mat(g1, layout1), mat(g1b, layout1), mat(g2, layout2), w1_rep, w2_rep)
     p._keep = (w1, w2, w1b, g1, g2, g1b)   # keep the tensors alive as long as the descriptor
     return p
 

@@ -250,6 +250,8 @@ extern "C" ecospa_status_t ecospa_compact_pair(const ecospa_pair_t* pair, const 
     const bool sw = pair->kind == ECOSPA_PAIR_SWIGLU;
     if (sw && !w1b_out) return ECOSPA_ERR_INVALID;
     if (pair->n_seg < 1 || pair->seg_len < 1) return ECOSPA_ERR_INVALID;
+    // grouped heads: the two sides have different shared extents and kept lists; use ecospa_compact_tensors
+    if (pair->w1_rep > 1 || pair->w2_rep > 1) return ECOSPA_ERR_UNSUPPORTED;
     const int64_t D = static_cast<int64_t>(pair->n_seg) * pair->seg_len;
     if (n_kept > D) return ECOSPA_ERR_INVALID;
     std::vector<ecospa_gather_t> jobs;

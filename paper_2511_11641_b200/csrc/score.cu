@@ -59,7 +59,7 @@ struct PairDesc {
     int32_t seg_start;  // first global segment index (also offset into fisher)
     float inv_numel1, inv_numel2;
     int32_t rope;       // ecospa_rope_t: the scored unit is a rotation pair of shared indices
-    int32_t pad_;
+    int16_t rep1, rep2; // heads stacked per segment on the W_1 / W_2 side (grouped-query attention); 1 = ordinary pair
 };
 static_assert(sizeof(PairDesc) == 72, "pair descriptor size");
 
@@ -256,6 +256,38 @@ __global__ void __launch_bounds__(kThreads) finalize_kernel(const __grid_constan
     const PairDesc& Q = P.pairs[pi];
     const int s = seg - Q.seg_start;
     const int base = s * Q.seg_len;
+    if (Q.rep1 > 1 || Q.rep2 > 1) {
+        // Grouped heads: the statistic of index j on a stacked side is the sum over the group's heads, in head order.
+        auto stacked = [&](const float* v, int rep, int j) {
+            float t = 0.f;
+            for (int r = 0; r < rep; ++r) t += v[(s * rep + r) * Q.seg_len + j];
+            return t;
+        };
+        float ss = 0.f;
+        for (int j = threadIdx.x; j < Q.seg_len; j += kThreads) {
+            const float r = sqrtf(stacked(Q.c1, Q.rep1, j)) * sqrtf(stacked(Q.c2, Q.rep2, j));
+            ss = fmaf(r, r, ss);
+        }
+        const float nrm = sqrtf(block_sum<kWarps>(ss, scratch));
+        for (int j = threadIdx.x; j < Q.seg_len; j += kThreads) {
+            const float r = sqrtf(stacked(Q.c1, Q.rep1, j)) * sqrtf(stacked(Q.c2, Q.rep2, j));
+            if (P.raw) P.raw[Q.d_off + base + j] = r;
+            P.upsilon[Q.d_off + base + j] = nrm > 0.f ? __fdiv_rn(r, nrm) : 0.f;
+        }
+        if (P.fisher) {
+            float a = 0.f, b = 0.f;
+            for (int j = threadIdx.x; j < Q.seg_len; j += kThreads) {
+                a += stacked(Q.gs1, Q.rep1, j);
+                b += stacked(Q.gs2, Q.rep2, j);
+            }
+            a = block_sum<kWarps>(a, scratch);
+            b = block_sum<kWarps>(b, scratch);
+            if (threadIdx.x == 0)
+                P.fisher[seg] = static_cast<float>(0.5 * (static_cast<double>(a) * Q.inv_numel1 + static_cast<double>(b) * Q.inv_numel2) *
+                                                   P.inv_n_samples);
+        }
+        return;
+    }
     const float* c1 = Q.c1 + base;
     const float* c2 = Q.c2 + base;
 
@@ -335,15 +367,18 @@ ecospa_status_t validate_pair(const ecospa_pair_t& p, bool need_grads) {
     if (p.rope != ECOSPA_ROPE_NONE && p.rope != ECOSPA_ROPE_INTERLEAVED && p.rope != ECOSPA_ROPE_HALF) return ECOSPA_ERR_INVALID;
     if (p.rope != ECOSPA_ROPE_NONE && (p.kind != ECOSPA_PAIR_PLAIN || (p.seg_len & 1))) return ECOSPA_ERR_INVALID;
     const int64_t D = static_cast<int64_t>(p.n_seg) * p.seg_len;
-    if (D > (1 << 22)) return ECOSPA_ERR_UNSUPPORTED;   // tile counts along D are 16-bit
+    if (p.w1_rep < 0 || p.w2_rep < 0 || p.w1_rep > 1024 || p.w2_rep > 1024) return ECOSPA_ERR_INVALID;
+    const int64_t r1 = std::max(1, p.w1_rep), r2 = std::max(1, p.w2_rep);
+    if ((r1 > 1 || r2 > 1) && (p.kind != ECOSPA_PAIR_PLAIN || p.rope != ECOSPA_ROPE_NONE)) return ECOSPA_ERR_INVALID;
+    if (D * std::max(r1, r2) > (1 << 22)) return ECOSPA_ERR_UNSUPPORTED;   // tile counts along D are 16-bit
     ecospa_status_t st;
-    if ((st = validate_mat(p.w1, D, -1, -1, -1)) != ECOSPA_OK) return st;
-    if ((st = validate_mat(p.w2, D, p.w1.dtype, -1, -1)) != ECOSPA_OK) return st;
+    if ((st = validate_mat(p.w1, D * r1, -1, -1, -1)) != ECOSPA_OK) return st;
+    if ((st = validate_mat(p.w2, D * r2, p.w1.dtype, -1, -1)) != ECOSPA_OK) return st;
     if (p.kind == ECOSPA_PAIR_SWIGLU &&
         (st = validate_mat(p.w1b, D, p.w1.dtype, p.w1.layout, p.w1.other_dim)) != ECOSPA_OK) return st;
     if (need_grads) {
-        if ((st = validate_mat(p.g1, D, -1, p.w1.layout, p.w1.other_dim)) != ECOSPA_OK) return st;
-        if ((st = validate_mat(p.g2, D, -1, p.w2.layout, p.w2.other_dim)) != ECOSPA_OK) return st;
+        if ((st = validate_mat(p.g1, D * r1, -1, p.w1.layout, p.w1.other_dim)) != ECOSPA_OK) return st;
+        if ((st = validate_mat(p.g2, D * r2, -1, p.w2.layout, p.w2.other_dim)) != ECOSPA_OK) return st;
         if (p.kind == ECOSPA_PAIR_SWIGLU &&
             (st = validate_mat(p.g1b, D, -1, p.w1.layout, p.w1.other_dim)) != ECOSPA_OK) return st;
     }
@@ -374,13 +409,14 @@ size_t plan_stats(const ecospa_pair_t* pairs, int n_pairs, bool grads, std::vect
     for (int i = 0; i < n_pairs; ++i) {
         const ecospa_pair_t& p = pairs[i];
         const int64_t D = static_cast<int64_t>(p.n_seg) * p.seg_len;
+        const int64_t D1 = D * std::max(1, p.w1_rep), D2 = D * std::max(1, p.w2_rep);   // grouped heads: the stacked extent
         const bool sw = p.kind == ECOSPA_PAIR_SWIGLU;
-        add(&p.w1, sw ? &p.w1b : nullptr, D);  // c1
-        add(&p.w2, nullptr, D);                // c2
+        add(&p.w1, sw ? &p.w1b : nullptr, D1);  // c1
+        add(&p.w2, nullptr, D2);                // c2
         if (grads) {
-            add(&p.g1, nullptr, D);
+            add(&p.g1, nullptr, D1);
             if (sw) add(&p.g1b, nullptr, D);
-            add(&p.g2, nullptr, D);
+            add(&p.g2, nullptr, D2);
         }
     }
     return off;
@@ -491,8 +527,10 @@ extern "C" ecospa_status_t ecospa_score_pairs(const ecospa_pair_t* pairs, int32_
             Q.rope = pr.rope;
             Q.d_off = d_off;
             Q.seg_start = segs;
-            Q.inv_numel1 = static_cast<float>(1.0 / (static_cast<double>(pr.w1.other_dim) * pr.seg_len));
-            Q.inv_numel2 = static_cast<float>(1.0 / (static_cast<double>(pr.w2.other_dim) * pr.seg_len));
+            Q.rep1 = static_cast<int16_t>(std::max(1, pr.w1_rep));
+            Q.rep2 = static_cast<int16_t>(std::max(1, pr.w2_rep));
+            Q.inv_numel1 = static_cast<float>(1.0 / (static_cast<double>(pr.w1.other_dim) * pr.seg_len * Q.rep1));
+            Q.inv_numel2 = static_cast<float>(1.0 / (static_cast<double>(pr.w2.other_dim) * pr.seg_len * Q.rep2));
             d_off += pr.n_seg * pr.seg_len;
             segs += pr.n_seg;
             seg_off += pr.n_seg;

@@ -307,3 +307,22 @@ def test_shared_dimension_limit(lib):
                                   C.c_void_p(0x4000), 1 << 30, None) == 3
     g = B.Gather(_fake_mat(0x10000, other=2, ld=D), _fake_mat(0x80000000, other=2, ld=64), 0x9000, 32, D)
     assert lib.ecospa_compact_tensors(C.addressof((B.Gather * 1)(g)), 1, None) == 3
+
+
+def test_grouped_pairs_are_validated_on_the_host(lib):
+    null = B.Mat(None, 0, 0, 0, 0)
+    ups, ws = C.c_void_p(0x3000), C.c_void_p(0x4000)
+    wq = _fake_mat(0x100000, other=64, ld=256)                 # 4 query heads of 64 side by side
+    wk = _fake_mat(0x200000, other=64, ld=64)
+    ok = B.Pair(B.PAIR_PLAIN, 1, 64, 0, wq, null, wk, null, null, null, 4, 1)
+    assert lib.ecospa_score_workspace_bytes(C.addressof((B.Pair * 1)(ok)), 1) > 0
+    # the stacked side must cover rep * D shared indices
+    short = B.Pair(B.PAIR_PLAIN, 1, 64, 0, _fake_mat(0x100000, other=64, ld=128), null, wk, null, null, null, 4, 1)
+    assert lib.ecospa_score_pairs(C.addressof((B.Pair * 1)(short)), 1, 1.0, ups, None, None, ws, 1 << 24, None) == 1
+    # grouped heads with rotation pairs or with a gated FFN pair are not defined
+    rope = B.Pair(B.PAIR_PLAIN, 1, 64, 1, wq, null, wk, null, null, null, 4, 1)
+    assert lib.ecospa_score_pairs(C.addressof((B.Pair * 1)(rope)), 1, 1.0, ups, None, None, ws, 1 << 24, None) == 1
+    sw = B.Pair(B.PAIR_SWIGLU, 1, 64, 0, wq, wq, wk, null, null, null, 4, 1)
+    assert lib.ecospa_score_pairs(C.addressof((B.Pair * 1)(sw)), 1, 1.0, ups, None, None, ws, 1 << 24, None) == 1
+    neg = B.Pair(B.PAIR_PLAIN, 1, 64, 0, wq, null, wk, null, null, null, -2, 1)
+    assert lib.ecospa_score_pairs(C.addressof((B.Pair * 1)(neg)), 1, 1.0, ups, None, None, ws, 1 << 24, None) == 1
