@@ -150,3 +150,30 @@ def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: f
     B.ecospa_compact_tensors(jobs, stream=stream)
     info = {"k": new_widths, "kept": kept_lists, "fisher": fis, "chosen": chosen, "upsilon": ups, "n_chosen": m}
     return out_groups, info
+
+
+def total_params(groups: Sequence[Group]) -> int:
+    """Param(W_t) of Algorithm 1 restricted to the coupled pairs: elements of every W_1 (gate and up) and W_2."""
+    return sum(g.n_params() for g in groups)
+
+
+def run_to_budget(groups: Sequence[Group], budget: int, n_samples: float, top_k_ratio: float, theta: float,
+                  l1: bool = True, k_min: int = 1, refresh=None, max_passes: int = 1000, stream=None):
+    """Algorithm 1's outer rule: while the model is larger than the target size c (`budget`, in parameters of the
+    coupled pairs), run one pass of the body.  `refresh(groups, t)` stands for the optimizer update between two
+    passes (it may overwrite the weights and gradients of the groups in place); without it the compacted gradients
+    of the previous pass are reused.  Stops early when a pass removes nothing (every chosen pair is at k_min or
+    within theta).  Returns (groups, history) with one entry per pass: parameters before / after and the pass info."""
+    history = []
+    t = 0
+    while total_params(groups) > budget and t < max_passes:
+        if refresh is not None:
+            refresh(groups, t)
+        before = total_params(groups)
+        groups, info = step(groups, n_samples, top_k_ratio, theta, l1=l1, k_min=k_min, stream=stream)
+        after = total_params(groups)
+        history.append({"pass": t, "params_before": before, "params_after": after, "info": info})
+        t += 1
+        if after == before:
+            break
+    return groups, history

@@ -28,3 +28,12 @@ def test_uniform_group_is_one_descriptor_and_ragged_group_one_per_pair():
     assert all(p.w1.ld == 16 and p.w2.ld == d_m for p in pairs[1:])                            # pitches stay
     assert [p.rope for p in pairs] == [0, 2, 2, 2]
     assert r.n_params() == 12 * 2 * d_m
+
+
+def test_run_to_budget_stops_without_a_pass_when_the_model_is_small_enough():
+    import torch
+    from paper_2511_11641_b200 import algorithm1 as A1
+    g = A1.Group(torch.zeros(4, 6), torch.zeros(6, 4), 0, 1, [3, 3])
+    assert A1.total_params([g]) == 6 * (4 + 4)
+    out, hist = A1.run_to_budget([g], 48, 1.0, 0.3, 0.9)          # already at the target: nothing is launched
+    assert hist == [] and out[0] is g

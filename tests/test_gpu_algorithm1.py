@@ -132,3 +132,46 @@ def test_two_passes_match_the_oracle(name, rope):
             for (tg, lay), (tr, _) in zip(g.aux, sp["aux"]):
                 assert same_bytes(tg, tr, lay, D)
     assert any(len(set(g.widths)) > 1 for g in groups)          # the second pass did run on ragged groups
+
+
+def spec_params(specs):
+    n = 0
+    for sp in specs:
+        D = sum(sp["widths"])
+        o1 = sp["w1"].shape[0] if sp["layout1"] == 0 else sp["w1"].shape[1]
+        o2 = sp["w2"].shape[0] if sp["layout2"] == 0 else sp["w2"].shape[1]
+        n += D * (o1 * (2 if sp.get("w1b") is not None else 1) + o2)
+    return n
+
+
+@pytest.mark.parametrize("name", ["tails768", "tiny_swiglu"])
+def test_run_to_budget_matches_the_oracle_loop(name):
+    """Algorithm 1's `if Param(W_t) > c` rule as a loop: the GPU driver and an oracle-side loop (same decisions on the
+    same fp32 vectors, oracle compaction) shrink two copies of the model pass by pass to the same sizes and bytes,
+    and stop at the same pass."""
+    wl = WL.WORKLOADS[name]
+    specs = make_groups(wl)
+    groups = [to_gpu(sp) for sp in specs]
+    n_samples = float(wl.tokens)
+    start = spec_params(specs)
+    assert A1.total_params(groups) == start
+    budget = int(0.72 * start)
+    ratio, theta, k_min = 0.4, 0.9, 2
+    groups, hist = A1.run_to_budget(groups, budget, n_samples, ratio, theta, k_min=k_min)
+    torch.cuda.synchronize()
+    assert len(hist) >= 2, "the budget must take more than one pass"
+    for h in hist:                                   # replay the same passes on the oracle's copy
+        assert spec_params(specs) == h["params_before"] and h["params_before"] > budget
+        specs = oracle_pass(specs, h["info"], n_samples, ratio, theta, k_min)
+        assert spec_params(specs) == h["params_after"]
+    assert A1.total_params(groups) == spec_params(specs)
+    assert A1.total_params(groups) <= budget or hist[-1]["params_after"] == hist[-1]["params_before"]
+    assert hist[-1]["params_before"] > budget            # no pass ran once the target was met
+    for g, sp in zip(groups, specs):
+        assert g.widths == sp["widths"]
+        D = sum(sp["widths"])
+        for nm, lay in (("w1", sp["layout1"]), ("w1b", sp["layout1"]), ("w2", sp["layout2"])):
+            if sp.get(nm) is not None:
+                assert same_bytes(getattr(g, nm), sp[nm], lay, D), nm
+        for (tg, lay), (tr, _) in zip(g.aux, sp["aux"]):
+            assert same_bytes(tg, tr, lay, D)
