@@ -32,7 +32,7 @@ if ROOT not in sys.path:
 # DRAM bytes (read + write) per gemm_kernel launch, averaged over the eight GEMM launches of a layer:
 # `dram__bytes_read.sum + dram__bytes_write.sum` of one ncu capture of this build per workload (one layer captured;
 # per-launch traffic does not depend on the number of layers).  Workloads without a capture: None.
-NCU_GEMM_TRAFFIC_BYTES = {"gpt2m": 45.3e6, "llama1b": 213.7e6}
+NCU_GEMM_TRAFFIC_BYTES = {"gpt2m": 45.3e6, "llama1b": 213.3e6}
 # DRAM bytes per step of sumsq_kernel + gather_kernel on 8 gpt2m layers under ncu (grow in proportion to the layers)
 NCU_SPARSIFY_TRAFFIC_BYTES_PER_LAYER = {"gpt2m": 889.3e6 / 8}
 
@@ -281,7 +281,7 @@ class Model:
         self.attention_fwd()
         B.ecospa_coupled_vo_fwd_o(o["Ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws, **self.lay)
         self.L.ffn_fwd_bwd(a["x"], a["dy"], self.act, c["w1"], c["w2"], k, self.ffn, w1bc=c.get("w1b"),
-                           b1c=c.get("b1"), b2=self.w[l].get("b2"), **self.lay)
+                           b1c=c.get("b1"), b2=self.w[l].get("b2"), bias_grads=self.wl.bias, **self.lay)
         B.ecospa_coupled_vo_bwd_o(o["Ctx"], c["wo"], n, a["dout"], o["dCtx"], o["dWo"], o["dbo"] if bias else None,
                                   workspace=self.proj_ws, **self.lay)
         self.attention_bwd()
@@ -311,7 +311,7 @@ class Model:
         B.ecospa_coupled_vo_fwd_o(a["ctx"], c["wo"], n, o["Out"], workspace=self.proj_ws, **self.lay)
         # FFN forward + backward
         self.L.ffn_fwd_bwd(a["x"], a["dy"], self.act, c["w1"], c["w2"], k, self.ffn, w1bc=c.get("w1b"),
-                           b1c=c.get("b1"), b2=self.w[l].get("b2"), **self.lay)
+                           b1c=c.get("b1"), b2=self.w[l].get("b2"), bias_grads=self.wl.bias, **self.lay)
         # backward: what dOut gives (dCtx, dW_O), then what dQ, dK, dV give (dW_Q, dW_K, dW_V, dX)
         B.ecospa_coupled_vo_bwd_o(a["ctx"], c["wo"], n, a["dout"], o["dCtx"], o["dWo"], o["dbo"] if bias else None,
                                   workspace=self.proj_ws, **self.lay)

@@ -35,9 +35,10 @@ def ffn_buffers(T: int, d_m: int, k: int, act: int, dtype: torch.dtype, device, 
 
 
 def ffn_fwd_bwd(X, dY, act: int, w1c, w2c, k: int, buf: Dict[str, torch.Tensor], w1bc=None, b1c=None, b2=None,
-                **layouts) -> None:
+                bias_grads: bool = True, **layouts) -> None:
+    """bias_grads=False: the layer has no biases, so db1 / db2 (column sums of dH / dY) are not asked for."""
     B.ecospa_coupled_ffn_fwd(X, act, w1c, w2c, k, buf["Y"], buf["H"], buf["A"], w1b_c=w1bc, Hb=buf.get("Hb"),
                              b1_c=b1c, b2=b2, workspace=buf["ws"], **layouts)
     B.ecospa_coupled_ffn_bwd(X, act, w1c, w2c, k, buf["H"], buf["A"], dY, buf["dX"], buf["dW1"], buf["dW2"],
-                             w1b_c=w1bc, Hb=buf.get("Hb"), dW1b_c=buf.get("dW1b"), db1_c=buf.get("db1"),
-                             db2=buf["db2"], workspace=buf["ws"], **layouts)
+                             w1b_c=w1bc, Hb=buf.get("Hb"), dW1b_c=buf.get("dW1b"), db1_c=buf.get("db1") if bias_grads else None,
+                             db2=buf["db2"] if bias_grads else None, workspace=buf["ws"], **layouts)
