@@ -259,33 +259,22 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                 const uint32_t sb = g & 1;
                 if (!(ok = mbar_wait(s_full(sb), (g >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
                 tc_fence_after();
-                // Row maximum over all 128 keys of the block, read by every thread of the row for itself (four TMEM
-                // reads instead of one): no exchange, so the softmax warps do not meet once per key block and their
-                // phases (loads, exponentials, stores) drift apart and overlap.
+                const int kv0 = j * kTile + part * 32;                // first key of this thread's columns
                 uint32_t r[32];
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-                const bool tile_masked = j * kTile + kTile > limit;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t t[32];
-                    tc_ld32(t_lane + kColS + sb * kTile + c * 32, t);
-                    tc_wait_ld();
-                    if (tile_masked) {                                // keys past the limit count as -inf
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (j * kTile + c * 32 + i >= limit) t[i] = 0xff800000u;
-                    }
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(t[i]));
-                }
-                const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-                tc_ld32(t_lane + kColS + sb * kTile + part * 32, r);      // this thread's own 32 scores
+                tc_ld32(t_lane + kColS + sb * kTile + part * 32, r);
                 tc_wait_ld();
-                if (tile_masked) {
+                if (kv0 + 32 > limit) {                               // keys past the limit count as -inf
 #pragma unroll
                     for (int i = 0; i < 32; ++i)
-                        if (j * kTile + part * 32 + i >= limit) r[i] = 0xff800000u;
+                        if (kv0 + i >= limit) r[i] = 0xff800000u;
                 }
+                // maximum over this thread's columns (four independent chains), then over the row
+                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
+                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), mo[3];
+                if (!(ok = exchange(mx, mo))) break;
+                mx = fmaxf(fmaxf(mx, mo[0]), fmaxf(mo[1], mo[2]));
                 const float m_new = fmaxf(m, mx * P.scale_log2e);
                 const float alpha = ex2(m - m_new);
                 if (j > 0) {
