@@ -249,6 +249,15 @@ ecospa_status_t ecospa_pack_kept(const int32_t* slots, const int32_t* src, const
  * (used to pad every head's block of a compacted tensor to the width the attention kernels need).
  */
 ecospa_status_t ecospa_compact_tensors(const ecospa_gather_t* jobs, int32_t n_jobs, void* stream);
+/* In-place variant of the same removal (Algorithm 1 shrinks the matrices and the optimizer moments it holds; a caller
+ * that cannot afford a second copy of them uses this form): every job must have out.ptr == in.ptr and out.ld == in.ld.
+ * The kept part moves to the front of the shared axis (columns [0, n_kept) of a SHARED_COLS tensor, zero pad up to the
+ * next 16-byte boundary as above; rows [0, n_kept) of a SHARED_ROWS tensor); what lies behind it afterwards is
+ * unspecified.  Every kept index must be at least its position in the list, kept[c] >= c (true of any ascending list,
+ * and of lists whose blocks are padded with -1 entries to no more than the blocks' original width): that is what makes
+ * a front-to-back walk safe; -1 entries give zeros.
+ * Same bytes as ecospa_compact_tensors on the kept part; slower (one warp walks a row or a 512-byte column stripe). */
+ecospa_status_t ecospa_compact_tensors_inplace(const ecospa_gather_t* jobs, int32_t n_jobs, void* stream);
 ecospa_status_t ecospa_compact_pair(const ecospa_pair_t* pair, const int32_t* kept, int32_t n_kept,
                                     const ecospa_mat_t* aux_in, const ecospa_mat_t* aux_out, int32_t n_aux,
                                     const ecospa_mat_t* w1_out, const ecospa_mat_t* w1b_out,

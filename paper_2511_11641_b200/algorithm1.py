@@ -91,10 +91,12 @@ def describe(groups: Sequence[Group]):
 
 
 def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: float, l1: bool = True,
-         k_min: int = 1, stream=None):
+         k_min: int = 1, stream=None, in_place: bool = False):
     """One pass of Algorithm 1's body: importance of every pair, the top-K share of the least important pairs,
     their scores, removal of the lowest-scored aligned indices while the remaining score mass exceeds theta, and
-    the physical removal from every tensor of the group.  Returns (new groups, info)."""
+    the physical removal from every tensor of the group.  Returns (new groups, info).
+    in_place: the tensors shrink inside their own storage (no second copy of the model and its optimizer state):
+    the new groups hold the same buffers, whose leading columns / rows are the kept part."""
     assert k_min >= 1 and all(w >= 1 for g in groups for w in g.widths)
     dev = groups[0].w1.device
     pairs, n_seg, seg_len, where, rope = describe(groups)
@@ -140,6 +142,10 @@ def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: f
         def shrink(t, layout):
             if t is None:
                 return None
+            if in_place:
+                v = _trim(t, layout, D)
+                jobs.append(B.gather(v, v, layout, kept, n_kept, D))
+                return t                                   # same storage and pitch; `widths` says what is valid
             o = alloc_compacted(_trim(t, layout, D), layout, n_kept)
             jobs.append(B.gather(_trim(t, layout, D), o, layout, kept, n_kept, D))
             return o
@@ -147,7 +153,7 @@ def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: f
                    w1b=shrink(g.w1b, g.layout1), g1=shrink(g.g1, g.layout1), g2=shrink(g.g2, g.layout2),
                    g1b=shrink(g.g1b, g.layout1), aux=[(shrink(t, lay), lay) for t, lay in g.aux], rope=g.rope)
         out_groups.append(ng)
-    B.ecospa_compact_tensors(jobs, stream=stream)
+    (B.ecospa_compact_tensors_inplace if in_place else B.ecospa_compact_tensors)(jobs, stream=stream)
     info = {"k": new_widths, "kept": kept_lists, "fisher": fis, "chosen": chosen, "upsilon": ups, "n_chosen": m}
     return out_groups, info
 
@@ -158,7 +164,8 @@ def total_params(groups: Sequence[Group]) -> int:
 
 
 def run_to_budget(groups: Sequence[Group], budget: int, n_samples: float, top_k_ratio: float, theta: float,
-                  l1: bool = True, k_min: int = 1, refresh=None, max_passes: int = 1000, stream=None):
+                  l1: bool = True, k_min: int = 1, refresh=None, max_passes: int = 1000, stream=None,
+                  in_place: bool = False):
     """Algorithm 1's outer rule: while the model is larger than the target size c (`budget`, in parameters of the
     coupled pairs), run one pass of the body.  `refresh(groups, t)` stands for the optimizer update between two
     passes (it may overwrite the weights and gradients of the groups in place); without it the compacted gradients
@@ -170,7 +177,7 @@ def run_to_budget(groups: Sequence[Group], budget: int, n_samples: float, top_k_
         if refresh is not None:
             refresh(groups, t)
         before = total_params(groups)
-        groups, info = step(groups, n_samples, top_k_ratio, theta, l1=l1, k_min=k_min, stream=stream)
+        groups, info = step(groups, n_samples, top_k_ratio, theta, l1=l1, k_min=k_min, stream=stream, in_place=in_place)
         after = total_params(groups)
         history.append({"pass": t, "params_before": before, "params_after": after, "info": info})
         t += 1

@@ -250,6 +250,17 @@ def ecospa_compact_tensors(jobs: Sequence[Gather], stream=None) -> None:
         raise EcospaError(st, "ecospa_compact_tensors")
 
 
+def ecospa_compact_tensors_inplace(jobs: Sequence[Gather], stream=None) -> None:
+    """Jobs whose output is their input (same pointer and pitch): the kept part moves to the front."""
+    arr = (Gather * len(jobs))(*jobs)
+    fn = lib().ecospa_compact_tensors_inplace
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+    st = fn(C.addressof(arr), len(jobs), _stream(stream))
+    if st != 0:
+        raise EcospaError(st, "ecospa_compact_tensors_inplace")
+
+
 def ecospa_compact_pair(p: Pair, kept: torch.Tensor, n_kept: int, w1_out: torch.Tensor, w2_out: torch.Tensor,
                         w1b_out: Optional[torch.Tensor] = None,
                         aux: Sequence[Tuple[torch.Tensor, torch.Tensor, int]] = (), stream=None) -> None:

@@ -232,12 +232,154 @@ ecospa_status_t compact_impl(const ecospa_gather_t* jobs, int32_t n_jobs, cudaSt
     return ECOSPA_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// In-place variant: out == in (same base, same pitch); the kept part moves to the front of the shared axis.
+// Kept indices are ascending, so kept[c] >= c: a destination is never a source that is still needed later, as long
+// as one owner walks the shared axis front to back and reads a batch before it writes it.
+//   shared-cols: a warp owns a row; it gathers a batch of columns into registers, then writes the batch.
+//   shared-rows: a warp owns a 512-byte stripe of columns of every row; it reads the stripe of 8 source rows, then
+//                writes them to their destination rows.
+// One job per launch grid slice; far fewer bytes in flight than the out-of-place kernel (memory saved, not time).
+// ------------------------------------------------------------------------------------------------
+struct InplaceJob {
+    void* base;
+    const int32_t* kept;
+    int64_t ld;            // elements
+    int32_t other, D, n_kept, esize, layout, warp_start, n_warps, pad_;
+};
+constexpr int kMaxInplaceJobs = 128;
+struct InplaceParams {
+    int32_t n_jobs, pad_;
+    InplaceJob jobs[kMaxInplaceJobs];
+};
+
+template <typename E>
+__device__ __forceinline__ void inplace_cols_row(const InplaceJob& J, int row, int lane) {
+    constexpr int kPer = 8;                              // columns per lane per batch
+    E* p = static_cast<E*>(J.base) + static_cast<int64_t>(row) * J.ld;
+    const int v = 16 / static_cast<int>(sizeof(E));
+    const int64_t padded = static_cast<int64_t>((J.n_kept + v - 1) / v) * v;
+    const int out_cols = static_cast<int>(padded < J.ld ? padded : J.ld);   // kept columns + zero pad
+    for (int c0 = 0; c0 < out_cols; c0 += 32 * kPer) {
+        E val[kPer];
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) {
+            const int c = c0 + e * 32 + lane;
+            int k = c < J.n_kept ? __ldg(J.kept + c) : -1;
+            k = k < 0 ? -1 : min(k, J.D - 1);
+            val[e] = k >= 0 ? p[k] : E(0);
+        }
+        __syncwarp();                                    // every source of the batch is read before any of it is written
+#pragma unroll
+        for (int e = 0; e < kPer; ++e) {
+            const int c = c0 + e * 32 + lane;
+            if (c < out_cols) p[c] = val[e];
+        }
+        __syncwarp();
+    }
+}
+
+__global__ void __launch_bounds__(128) gather_inplace_kernel(const __grid_constant__ InplaceParams P) {
+    const int gw = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    int ji = 0;
+    while (ji + 1 < P.n_jobs && P.jobs[ji + 1].warp_start <= gw) ++ji;
+    const InplaceJob& J = P.jobs[ji];
+    const int w = gw - J.warp_start;
+    if (w >= J.n_warps) return;
+    if (J.layout == ECOSPA_SHARED_COLS) {
+        if (J.esize == 2) inplace_cols_row<uint16_t>(J, w, lane); else inplace_cols_row<uint32_t>(J, w, lane);
+        return;
+    }
+    // shared rows: this warp's stripe = bytes [512 w, 512 w + 512) of every row (2-byte units: every element size divides)
+    const int64_t row_bytes = static_cast<int64_t>(J.other) * J.esize, pitch = J.ld * J.esize;
+    const int64_t b0 = 512ll * w + 16 * lane;
+    char* base = static_cast<char*>(J.base);
+    const bool vec = (reinterpret_cast<uintptr_t>(base) & 15u) == 0 && pitch % 16 == 0 && b0 + 16 <= row_bytes;
+    for (int r0 = 0; r0 < J.n_kept; r0 += 8) {
+        uint4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (r0 + u < J.n_kept) {
+                int k = __ldg(J.kept + r0 + u);
+                if (k >= 0 && b0 < row_bytes) {
+                    const char* src = base + static_cast<int64_t>(min(k, J.D - 1)) * pitch + b0;
+                    if (vec) {
+                        v[u] = *reinterpret_cast<const uint4*>(src);
+                    } else {
+                        uint16_t* h = reinterpret_cast<uint16_t*>(&v[u]);
+                        for (int e = 0; e < 8; ++e)
+                            if (b0 + 2 * e < row_bytes) h[e] = *reinterpret_cast<const uint16_t*>(src + 2 * e);
+                    }
+                }
+            }
+        }
+        __syncwarp();
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (r0 + u < J.n_kept && b0 < row_bytes) {
+                char* dst = base + static_cast<int64_t>(r0 + u) * pitch + b0;
+                if (vec) {
+                    *reinterpret_cast<uint4*>(dst) = v[u];
+                } else {
+                    const uint16_t* h = reinterpret_cast<const uint16_t*>(&v[u]);
+                    for (int e = 0; e < 8; ++e)
+                        if (b0 + 2 * e < row_bytes) *reinterpret_cast<uint16_t*>(dst + 2 * e) = h[e];
+                }
+            }
+        }
+        __syncwarp();
+    }
+}
+
+ecospa_status_t compact_inplace_impl(const ecospa_gather_t* jobs, int32_t n_jobs, cudaStream_t stream) {
+    if (!jobs || n_jobs < 1) return ECOSPA_ERR_INVALID;
+    for (int i = 0; i < n_jobs; ++i) {
+        const ecospa_gather_t& g = jobs[i];
+        if (!g.in.ptr || !g.kept || g.out.ptr != g.in.ptr || g.out.ld != g.in.ld) return ECOSPA_ERR_INVALID;
+        if (g.in.dtype != g.out.dtype || g.in.layout != g.out.layout || g.in.other_dim != g.out.other_dim) return ECOSPA_ERR_INVALID;
+        if (g.in.dtype != ECOSPA_F32 && g.in.dtype != ECOSPA_BF16) return ECOSPA_ERR_INVALID;
+        if (g.in.layout != ECOSPA_SHARED_COLS && g.in.layout != ECOSPA_SHARED_ROWS) return ECOSPA_ERR_INVALID;
+        if (g.in.other_dim < 1 || g.in.other_dim > INT32_MAX || g.in.ld > INT32_MAX) return ECOSPA_ERR_INVALID;
+        if (g.n_kept < 0 || g.shared_dim < 1 || g.n_kept > g.shared_dim) return ECOSPA_ERR_INVALID;
+        if (g.in.ld < (g.in.layout == ECOSPA_SHARED_COLS ? g.shared_dim : g.in.other_dim)) return ECOSPA_ERR_INVALID;
+        if (reinterpret_cast<uintptr_t>(g.in.ptr) % elem_bytes(g.in.dtype)) return ECOSPA_ERR_ALIGNMENT;
+    }
+    static thread_local InplaceParams ip;
+    int i = 0;
+    while (i < n_jobs) {
+        int nj = 0, warps = 0;
+        for (; i < n_jobs && nj < kMaxInplaceJobs; ++i) {
+            const ecospa_gather_t& g = jobs[i];
+            if (g.n_kept == 0) continue;
+            InplaceJob& J = ip.jobs[nj++];
+            J = InplaceJob{};
+            const int eb = elem_bytes(g.in.dtype);
+            J.base = g.in.ptr; J.kept = g.kept; J.ld = g.in.ld;
+            J.other = static_cast<int32_t>(g.in.other_dim); J.D = g.shared_dim; J.n_kept = g.n_kept;
+            J.esize = eb; J.layout = g.in.layout; J.warp_start = warps;
+            J.n_warps = g.in.layout == ECOSPA_SHARED_COLS ? J.other : static_cast<int32_t>(ceil_div(static_cast<int64_t>(J.other) * eb, 512));
+            warps += J.n_warps;
+        }
+        if (nj == 0) continue;
+        ip.n_jobs = nj;
+        gather_inplace_kernel<<<static_cast<unsigned>(ceil_div(warps, 4)), 128, 0, stream>>>(ip);
+        ecospa_status_t st = check_launch("gather_inplace_kernel");
+        if (st != ECOSPA_OK) return st;
+    }
+    return ECOSPA_OK;
+}
+
 }  // namespace ecospa
 
 using namespace ecospa;
 
 extern "C" ecospa_status_t ecospa_compact_tensors(const ecospa_gather_t* jobs, int32_t n_jobs, void* stream) {
     return compact_impl(jobs, n_jobs, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" ecospa_status_t ecospa_compact_tensors_inplace(const ecospa_gather_t* jobs, int32_t n_jobs, void* stream) {
+    return compact_inplace_impl(jobs, n_jobs, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" ecospa_status_t ecospa_compact_pair(const ecospa_pair_t* pair, const int32_t* kept, int32_t n_kept,

@@ -326,3 +326,18 @@ def test_grouped_pairs_are_validated_on_the_host(lib):
     assert lib.ecospa_score_pairs(C.addressof((B.Pair * 1)(sw)), 1, 1.0, ups, None, None, ws, 1 << 24, None) == 1
     neg = B.Pair(B.PAIR_PLAIN, 1, 64, 0, wq, null, wk, null, null, null, -2, 1)
     assert lib.ecospa_score_pairs(C.addressof((B.Pair * 1)(neg)), 1, 1.0, ups, None, None, ws, 1 << 24, None) == 1
+
+
+def test_in_place_compaction_rejects_jobs_that_are_not_in_place(lib):
+    fn = lib.ecospa_compact_tensors_inplace
+    fn.restype = C.c_int
+    fn.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
+    kept = 0x9000
+    m = _fake_mat(0x10000, other=8, ld=64)
+    ok_shape = B.Gather(m, _fake_mat(0x20000, other=8, ld=64), kept, 32, 64)          # another buffer
+    assert fn(C.addressof((B.Gather * 1)(ok_shape)), 1, None) == 1
+    other_pitch = B.Gather(m, _fake_mat(0x10000, other=8, ld=32), kept, 32, 64)       # same base, other pitch
+    assert fn(C.addressof((B.Gather * 1)(other_pitch)), 1, None) == 1
+    assert fn(None, 1, None) == 1
+    too_many = B.Gather(m, m, kept, 65, 64)
+    assert fn(C.addressof((B.Gather * 1)(too_many)), 1, None) == 1

@@ -111,15 +111,19 @@ def same_bytes(gpu_t, ref, layout, D):
     return torch.equal(g.view(view), ref.contiguous().view(view))
 
 
-@pytest.mark.parametrize("name,rope", [("tails768", 0), ("tiny_swiglu", 0), ("tails768", B.ROPE_HALF),
-                                       ("tiny_swiglu", B.ROPE_INTERLEAVED)])
-def test_two_passes_match_the_oracle(name, rope):
+@pytest.mark.parametrize("name,rope,in_place", [("tails768", 0, False), ("tiny_swiglu", 0, False), ("tails768", B.ROPE_HALF, False),
+                                                ("tiny_swiglu", B.ROPE_INTERLEAVED, False), ("tails768", 0, True),
+                                                ("tiny_swiglu", 0, True)])
+def test_two_passes_match_the_oracle(name, rope, in_place):
+    """in_place: the tensors (weights, gradients, fp32 moments, biases) shrink inside their own storage."""
     wl = WL.WORKLOADS[name]
     specs = make_groups(wl, rope=rope)
     groups = [to_gpu(sp) for sp in specs]
     n_samples = float(wl.tokens)
+    ptrs = [g.w1.data_ptr() for g in groups]
     for ratio, theta in ((0.5, 0.9), (0.6, 0.8)):
-        groups, info = A1.step(groups, n_samples, ratio, theta, l1=True, k_min=2)
+        groups, info = A1.step(groups, n_samples, ratio, theta, l1=True, k_min=2, in_place=in_place)
+        assert [g.w1.data_ptr() for g in groups] == ptrs or not in_place
         torch.cuda.synchronize()
         specs = oracle_pass(specs, info, n_samples, ratio, theta, 2)
         for g, sp in zip(groups, specs):

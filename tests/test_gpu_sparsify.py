@@ -455,3 +455,47 @@ def test_reestimation_sweep_one_layer():
             names = ["wq", "wk", "wo", "w1", "w1b", "w2", "gq", "go", "g1", "g1b", "g2"] if s10 in (1, 5, 9) else []
             kept = select_and_compact_vs_oracle(wl, allt, d_all, ups, s, names)
             assert len(kept) == 2 * wl.n_heads * WL.kept_count(wl.d_h, s) + WL.kept_count(wl.d_ffn, s)
+
+
+def test_in_place_compaction_equals_out_of_place():
+    """ecospa_compact_tensors_inplace moves the kept part to the front of each tensor's own storage: same bytes as the
+    out-of-place call (and the oracle) on the kept part, for bf16 and fp32, both layouts, a 1-D bias, odd pitches, and a
+    kept list with "no index" entries."""
+    wl = WL.WORKLOADS["tails768"]
+    w = WL.layer_weights(wl, 0)
+    gen = torch.Generator().manual_seed(6)
+    t = {"w1": w["w1"], "w2": w["w2"], "b1": w["b1"], "m1": torch.randn(w["w1"].shape, generator=gen),
+         "m2": torch.randn(w["w2"].shape, generator=gen)}
+    lay = {"w1": 0, "w2": 1, "b1": 0, "m1": 0, "m2": 1}
+    r = np.random.default_rng(8)
+    for k_ffn, pads in ((1337, 0), (2044, 0), (1073, 7)):
+        kept = np.sort(r.choice(wl.d_ffn, size=k_ffn, replace=False)).astype(np.int32)
+        if pads:                                          # "no index" entries that pad two blocks, as for padded heads:
+            half = wl.d_ffn // 2                          # every real entry still satisfies kept[c] >= c
+            lo, hi = kept[kept < half], kept[kept >= half]
+            kept = np.concatenate([lo, -np.ones(3, np.int32), hi, -np.ones(pads - 3, np.int32)]).astype(np.int32)
+        n = len(kept)
+        kd = torch.from_numpy(kept).to(DEV)
+        jobs, bufs = [], {}
+        for nm, src in t.items():
+            d = src.to(DEV).clone()
+            bufs[nm] = d
+            jobs.append(B.gather(d, d, lay[nm], kd, n, wl.d_ffn))
+        B.ecospa_compact_tensors_inplace(jobs)
+        torch.cuda.synchronize()
+        for nm, src in t.items():
+            ref = O.compact(src, lay[nm], kept)
+            d = bufs[nm].cpu()
+            got = d[:n] if src.dim() == 1 else (d[:, :n] if lay[nm] == 0 else d[:n])
+            view = torch.int16 if src.element_size() == 2 else torch.int32
+            assert torch.equal(got.contiguous().view(view), ref.contiguous().view(view)), (nm, k_ffn)
+    # an odd pitch and a base that is only 2-byte aligned (element-wise path of the shared-rows stripe)
+    src = w["w2"][:, :701].contiguous()
+    buf = torch.zeros(src.shape[0] * 705 + 1, dtype=src.dtype, device=DEV)
+    v = buf[1:].as_strided(src.shape, (705, 1))
+    v.copy_(src)
+    kept = np.sort(r.choice(wl.d_ffn, size=900, replace=False)).astype(np.int32)
+    kd = torch.from_numpy(kept).to(DEV)
+    B.ecospa_compact_tensors_inplace([B.gather(v, v, 1, kd, 900, wl.d_ffn)])
+    ref = O.compact(src, 1, kept)
+    assert torch.equal(v[:900].cpu().contiguous().view(torch.int16), ref.view(torch.int16))
