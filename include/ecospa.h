@@ -235,6 +235,48 @@ ecospa_status_t ecospa_pack_kept(const int32_t* slots, const int32_t* src, const
                                  const int32_t* add, int32_t n_segs, int32_t* out, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * One pass of the body of Algorithm 1 over whole groups of pairs (everything between "if Param(W_t) > c" and the
+ * end of the loop body): importance of every pair, the n_choose pairs with the smallest importance, their scores,
+ * removal of the lowest-scored aligned indices while the remaining score mass exceeds theta, and the removal of the
+ * same rows / columns from every tensor of the group (gradients, optimizer moments, biases).
+ *
+ * A group = the tensors that live on one shared axis: the six tensors of ecospa_pair_t plus n_aux further ones (HOST
+ * array `aux`; a 1-D bias is other_dim = 1, SHARED_COLS), and the widths of its pairs (HOST, n_pairs entries; the pairs sit
+ * side by side on the shared axis, sum of widths = its extent; after a pass the widths differ from pair to pair; width 0
+ * = a pair that has lost every index and takes no part).
+ * ecospa_alg1_plan     enqueues scoring, pair choice and threshold selection, waits for the stream (the one
+ *                      synchronisation: the counts size what follows) and writes the new width of every pair to
+ *                      k_host (HOST, one entry per pair of every group, in order).  Gradients are required.
+ * ecospa_alg1_apply    enqueues the removal: into the tensors of out[g] (same structure, caller-allocated for the
+ *                      widths in k_host, padded pitches as in step 3), or, with in_place != 0, inside the tensors
+ *                      themselves (out may be NULL; see ecospa_compact_tensors_inplace).  Must follow a plan call on the same
+ *                      groups with the same workspace.
+ * workspace: DEVICE, ecospa_alg1_workspace_bytes, 16-byte aligned; between the two calls it holds the scores,
+ * importance values, choice flags and kept lists; ecospa_alg1_offsets gives their byte offsets
+ * (offsets[0..3] = upsilon, importance, choice flags, kept lists; offsets[4..5] = total shared indices and pairs described),
+ * in the order of the described pairs (groups in order, pairs of width 0 left out).  theta, l1, k_min as in
+ * ecospa_select_aligned_threshold.  */
+typedef struct {
+    ecospa_mat_t w1, w1b, w2;   /* w1b: SwiGLU up matrix or absent */
+    ecospa_mat_t g1, g1b, g2;
+    const ecospa_mat_t* aux;    /* HOST [n_aux] */
+    int32_t n_aux;
+    int32_t n_pairs;
+    const int32_t* widths;      /* HOST [n_pairs] */
+    int32_t rope;               /* ecospa_rope_t of the group's pairs */
+    int32_t reserved_;
+} ecospa_group_t;
+
+size_t ecospa_alg1_workspace_bytes(const ecospa_group_t* groups, int32_t n_groups);
+ecospa_status_t ecospa_alg1_offsets(const ecospa_group_t* groups, int32_t n_groups, int64_t* offsets);
+ecospa_status_t ecospa_alg1_plan(const ecospa_group_t* groups, int32_t n_groups, double n_samples, int32_t n_choose,
+                                 double theta, int32_t l1, int32_t k_min, void* workspace, size_t workspace_bytes,
+                                 int32_t* k_host, void* stream);
+ecospa_status_t ecospa_alg1_apply(const ecospa_group_t* groups, int32_t n_groups, const int32_t* k_host,
+                                  const ecospa_group_t* out, int32_t in_place, void* workspace, size_t workspace_bytes,
+                                  void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Step 3: physical removal.   Definition 1: drop column j of W_1 and row j of W_2 for every removed j
  * "keeping the original pairings"; Alg. 1 also drops the same rows/columns of the optimizer moments.
  *

@@ -90,71 +90,65 @@ def describe(groups: Sequence[Group]):
     return pairs, n_seg, seg_len, where, rope
 
 
+def _c_group(g: Group, with_grads: bool = True) -> "B.Group":
+    D = g.D
+    t = lambda nm, lay: _trim(getattr(g, nm), lay, D)
+    return B.group(t("w1", g.layout1), t("w2", g.layout2), g.layout1, g.layout2, g.widths, w1b=t("w1b", g.layout1),
+                   g1=t("g1", g.layout1) if with_grads else None, g2=t("g2", g.layout2) if with_grads else None,
+                   g1b=t("g1b", g.layout1) if with_grads else None, aux=[(_trim(a, lay, D), lay) for a, lay in g.aux],
+                   rope=g.rope)
+
+
 def step(groups: Sequence[Group], n_samples: float, top_k_ratio: float, theta: float, l1: bool = True,
          k_min: int = 1, stream=None, in_place: bool = False):
     """One pass of Algorithm 1's body: importance of every pair, the top-K share of the least important pairs,
     their scores, removal of the lowest-scored aligned indices while the remaining score mass exceeds theta, and
     the physical removal from every tensor of the group.  Returns (new groups, info).
+    The pass itself is two library calls (ecospa_alg1_plan, which reads the data-dependent kept counts back, and
+    ecospa_alg1_apply); this function describes the groups, allocates the compacted tensors in between and wraps
+    what the workspace holds afterwards.
     in_place: the tensors shrink inside their own storage (no second copy of the model and its optimizer state):
     the new groups hold the same buffers, whose leading columns / rows are the kept part."""
-    assert k_min >= 1 and all(w >= 1 for g in groups for w in g.widths)
+    assert k_min >= 1
     dev = groups[0].w1.device
-    pairs, n_seg, seg_len, where, rope = describe(groups)
-    total_segs = sum(n_seg)
-    total_d = sum(a * b for a, b in zip(n_seg, seg_len))
-    i32, f32 = torch.int32, torch.float32
-    ups = torch.empty(total_d, dtype=f32, device=dev)
-    fis = torch.empty(total_segs, dtype=f32, device=dev)
-    ws = torch.empty(max(16, B.ecospa_score_workspace_bytes(pairs)), dtype=torch.uint8, device=dev)
-    B.ecospa_score_pairs(pairs, float(n_samples), ups, None, fis, ws, stream=stream)
-    m = min(total_segs, int(top_k_ratio * total_segs + 0.5))
-    chosen = torch.empty(total_segs, dtype=i32, device=dev)
-    B.ecospa_choose_pairs(fis, m, chosen, stream=stream)
-    slots = torch.empty(total_d, dtype=i32, device=dev)
-    k_out = torch.empty(total_segs, dtype=i32, device=dev)
-    B.ecospa_select_aligned_threshold(ups, n_seg, seg_len, theta, slots, k_out, l1=l1, k_min=k_min, chosen=chosen,
-                                      rope=rope if any(rope) else None, stream=stream)
-    k = k_out.cpu().tolist()                 # the one read-back: the counts size everything that follows
-
-    # per group: the kept list of the whole shared axis, then one gather per tensor
-    new_widths: List[List[int]] = [[] for _ in groups]
-    src: List[List[int]] = [[] for _ in groups]
-    add: List[List[int]] = [[] for _ in groups]
-    kk: List[List[int]] = [[] for _ in groups]
-    seg, d_off = 0, 0
-    for (gi, off), ns, sl in zip(where, n_seg, seg_len):
-        for s in range(ns):
-            new_widths[gi].append(k[seg]); kk[gi].append(k[seg])
-            src[gi].append(d_off + s * sl); add[gi].append(off)      # slot indices are relative to the described pair group
-            seg += 1
-        d_off += ns * sl
-    out_groups, kept_lists, jobs = [], [], []
-    for gi, g in enumerate(groups):
-        n_kept = sum(kk[gi])
-        dst, run = [], 0
-        for v in kk[gi]:
-            dst.append(run); run += v
-        kept = torch.empty(max(n_kept, 1), dtype=i32, device=dev)
-        B.ecospa_pack_kept(slots, src[gi], dst, kk[gi], add[gi], kept, stream=stream)
-        kept_lists.append(kept[:n_kept])
-        D = g.D
+    cg = [_c_group(g) for g in groups]
+    ws = torch.empty(max(16, B.ecospa_alg1_workspace_bytes(cg)), dtype=torch.uint8, device=dev)
+    live = sum(1 for g in groups for w in g.widths if w > 0)
+    m = min(live, int(top_k_ratio * live + 0.5))
+    k = B.ecospa_alg1_plan(cg, float(n_samples), m, theta, l1, k_min, ws, stream=stream)
+    new_widths, pos = [], 0
+    for g in groups:
+        new_widths.append(k[pos:pos + len(g.widths)])
+        pos += len(g.widths)
+    out_groups = []
+    for g, nw in zip(groups, new_widths):
+        n_kept, D = sum(nw), g.D
 
         def shrink(t, layout):
             if t is None:
                 return None
-            if in_place:
-                v = _trim(t, layout, D)
-                jobs.append(B.gather(v, v, layout, kept, n_kept, D))
-                return t                                   # same storage and pitch; `widths` says what is valid
-            o = alloc_compacted(_trim(t, layout, D), layout, n_kept)
-            jobs.append(B.gather(_trim(t, layout, D), o, layout, kept, n_kept, D))
-            return o
-        ng = Group(shrink(g.w1, g.layout1), shrink(g.w2, g.layout2), g.layout1, g.layout2, new_widths[gi],
-                   w1b=shrink(g.w1b, g.layout1), g1=shrink(g.g1, g.layout1), g2=shrink(g.g2, g.layout2),
-                   g1b=shrink(g.g1b, g.layout1), aux=[(shrink(t, lay), lay) for t, lay in g.aux], rope=g.rope)
-        out_groups.append(ng)
-    (B.ecospa_compact_tensors_inplace if in_place else B.ecospa_compact_tensors)(jobs, stream=stream)
-    info = {"k": new_widths, "kept": kept_lists, "fisher": fis, "chosen": chosen, "upsilon": ups, "n_chosen": m}
+            return t if in_place else alloc_compacted(_trim(t, layout, D), layout, n_kept)
+        out_groups.append(Group(shrink(g.w1, g.layout1), shrink(g.w2, g.layout2), g.layout1, g.layout2, list(nw),
+                                w1b=shrink(g.w1b, g.layout1), g1=shrink(g.g1, g.layout1), g2=shrink(g.g2, g.layout2),
+                                g1b=shrink(g.g1b, g.layout1), aux=[(shrink(t, lay), lay) for t, lay in g.aux], rope=g.rope))
+    if in_place:
+        B.ecospa_alg1_apply(cg, k, None, ws, in_place=True, stream=stream)
+    else:
+        # the output descriptors carry the buffers as allocated (padded pitch); their widths are not read
+        og = []
+        for g, ng in zip(groups, out_groups):
+            og.append(B.group(ng.w1, ng.w2, g.layout1, g.layout2, ng.widths, w1b=ng.w1b, g1=ng.g1, g2=ng.g2, g1b=ng.g1b,
+                              aux=ng.aux, rope=g.rope))
+        B.ecospa_alg1_apply(cg, k, og, ws, in_place=False, stream=stream)
+    o_ups, o_fis, o_chosen, o_kept, total_d, total_pairs = B.ecospa_alg1_offsets(cg)
+    f32v = lambda off, n: ws[off:off + 4 * n].view(torch.float32)
+    i32v = lambda off, n: ws[off:off + 4 * n].view(torch.int32)
+    kept_lists, ko = [], 0
+    for nw in new_widths:
+        kept_lists.append(i32v(o_kept + 4 * ko, sum(nw)))
+        ko += sum(nw)
+    info = {"k": [list(nw) for nw in new_widths], "kept": kept_lists, "fisher": f32v(o_fis, total_pairs),
+            "chosen": i32v(o_chosen, total_pairs), "upsilon": f32v(o_ups, total_d), "n_chosen": m, "workspace": ws}
     return out_groups, info
 
 

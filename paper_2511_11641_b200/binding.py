@@ -559,6 +559,71 @@ def ecospa_pad_kept(kept: torch.Tensor, src: Sequence[int], dst: Sequence[int], 
               _stream(stream)), "ecospa_pad_kept")
 
 
+# ---------------------------------------------------------------------------------------------
+# one pass of Algorithm 1's body over groups of pairs
+# ---------------------------------------------------------------------------------------------
+
+class Group(C.Structure):
+    _fields_ = [("w1", Mat), ("w1b", Mat), ("w2", Mat), ("g1", Mat), ("g1b", Mat), ("g2", Mat), ("aux", C.c_void_p),
+                ("n_aux", C.c_int32), ("n_pairs", C.c_int32), ("widths", C.c_void_p), ("rope", C.c_int32),
+                ("reserved_", C.c_int32)]
+
+
+def group(w1, w2, layout1: int, layout2: int, widths: Sequence[int], w1b=None, g1=None, g2=None, g1b=None,
+          aux: Sequence[Tuple[Optional[torch.Tensor], int]] = (), rope: int = 0) -> Group:
+    """Descriptor of the tensors on one shared axis; aux = (tensor, layout) pairs (a 1-D tensor is a bias)."""
+    n_aux = len(aux)
+    a_arr = (Mat * max(1, n_aux))(*[mat(t, lay) for t, lay in aux])
+    w_arr = (C.c_int32 * len(widths))(*[int(v) for v in widths])
+    g = Group(mat(w1, layout1), mat(w1b, layout1), mat(w2, layout2), mat(g1, layout1), mat(g1b, layout1), mat(g2, layout2),
+              C.addressof(a_arr) if n_aux else None, n_aux, len(widths), C.addressof(w_arr), rope, 0)
+    g._keep = (a_arr, w_arr, w1, w2, w1b, g1, g2, g1b, [t for t, _ in aux])
+    return g
+
+
+def _alg1(name, restype, argtypes):
+    f = getattr(lib(), name)
+    f.restype, f.argtypes = restype, argtypes
+    return f
+
+
+def ecospa_alg1_workspace_bytes(groups: Sequence[Group]) -> int:
+    arr = (Group * len(groups))(*groups)
+    return int(_alg1("ecospa_alg1_workspace_bytes", C.c_size_t, [C.c_void_p, C.c_int32])(C.addressof(arr), len(groups)))
+
+
+def ecospa_alg1_offsets(groups: Sequence[Group]) -> List[int]:
+    arr = (Group * len(groups))(*groups)
+    out = (C.c_int64 * 6)()
+    _check(_alg1("ecospa_alg1_offsets", C.c_int, [C.c_void_p, C.c_int32, C.c_void_p])(C.addressof(arr), len(groups), C.addressof(out)),
+           "ecospa_alg1_offsets")
+    return [int(v) for v in out]
+
+
+def ecospa_alg1_plan(groups: Sequence[Group], n_samples: float, n_choose: int, theta: float, l1: bool, k_min: int,
+                     workspace: torch.Tensor, stream=None) -> List[int]:
+    """Returns the new width of every pair of every group (synchronises the stream)."""
+    arr = (Group * len(groups))(*groups)
+    n = sum(g.n_pairs for g in groups)
+    k = (C.c_int32 * n)()
+    f = _alg1("ecospa_alg1_plan", C.c_int, [C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_double, C.c_int32, C.c_int32,
+                                            C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p])
+    _check(f(C.addressof(arr), len(groups), float(n_samples), int(n_choose), float(theta), int(bool(l1)), int(k_min),
+             workspace.data_ptr(), workspace.numel(), C.addressof(k), _stream(stream)), "ecospa_alg1_plan")
+    return list(k)
+
+
+def ecospa_alg1_apply(groups: Sequence[Group], k: Sequence[int], out: Optional[Sequence[Group]], workspace: torch.Tensor,
+                      in_place: bool = False, stream=None) -> None:
+    arr = (Group * len(groups))(*groups)
+    oarr = (Group * len(out))(*out) if out is not None else None
+    ka = (C.c_int32 * len(k))(*[int(v) for v in k])
+    f = _alg1("ecospa_alg1_apply", C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t,
+                                             C.c_void_p])
+    _check(f(C.addressof(arr), len(groups), C.addressof(ka), C.addressof(oarr) if oarr is not None else None,
+             int(bool(in_place)), workspace.data_ptr(), workspace.numel(), _stream(stream)), "ecospa_alg1_apply")
+
+
 def ecospa_launch_count() -> int:
     f = lib().ecospa_launch_count
     f.restype = C.c_uint64

@@ -341,3 +341,69 @@ def test_in_place_compaction_rejects_jobs_that_are_not_in_place(lib):
     assert fn(None, 1, None) == 1
     too_many = B.Gather(m, m, kept, 65, 64)
     assert fn(C.addressof((B.Gather * 1)(too_many)), 1, None) == 1
+
+
+def test_algorithm1_pass_rejects_bad_arguments_without_launching(lib):
+    null = B.Mat(None, 0, 0, 0, 0)
+    w1 = _fake_mat(0x10000, ld=128)
+    w2 = _fake_mat(0x20000, layout=B.SHARED_ROWS)
+    g1 = _fake_mat(0x30000, ld=128)
+    g2 = _fake_mat(0x40000, layout=B.SHARED_ROWS)
+    widths = (C.c_int32 * 2)(64, 64)
+
+    def grp(w1=w1, w2=w2, g1=g1, g2=g2, n_pairs=2, wptr=C.addressof(widths), n_aux=0, aux=None):
+        return B.Group(w1, null, w2, g1, null, g2, aux, n_aux, n_pairs, wptr, 0, 0)
+
+    def arr(g):
+        a = (B.Group * 1)(g)
+        return a, C.addressof(a)
+
+    size = lib.ecospa_alg1_workspace_bytes
+    size.restype, size.argtypes = C.c_size_t, [C.c_void_p, C.c_int32]
+    plan = lib.ecospa_alg1_plan
+    plan.restype = C.c_int
+    plan.argtypes = [C.c_void_p, C.c_int32, C.c_double, C.c_int32, C.c_double, C.c_int32, C.c_int32, C.c_void_p, C.c_size_t,
+                     C.c_void_p, C.c_void_p]
+    apply_ = lib.ecospa_alg1_apply
+    apply_.restype = C.c_int
+    apply_.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]
+    offs = lib.ecospa_alg1_offsets
+    offs.restype, offs.argtypes = C.c_int, [C.c_void_p, C.c_int32, C.c_void_p]
+
+    keep, good = arr(grp())
+    need = size(good, 1)
+    assert need > 6 * 128 * 4 and need % 256 == 0
+    out6 = (C.c_int64 * 6)()
+    assert offs(good, 1, C.addressof(out6)) == 0 and out6[4] == 128 and out6[5] == 2 and out6[0] == 0
+    assert offs(good, 1, None) == 1
+    k = (C.c_int32 * 2)(32, 32)
+    ws = 0x100000
+    # no groups / no counts / negative pair count to choose
+    assert plan(None, 1, 8.0, 1, 0.5, 1, 1, ws, need, C.addressof(k), None) == 1
+    assert plan(good, 1, 8.0, 1, 0.5, 1, 1, ws, need, None, None) == 1
+    assert plan(good, 1, 8.0, -1, 0.5, 1, 1, ws, need, C.addressof(k), None) == 1
+    # importance needs the gradients
+    kp, nograd = arr(grp(g1=null))
+    assert plan(nograd, 1, 8.0, 1, 0.5, 1, 1, ws, need, C.addressof(k), None) == 1
+    # a group without widths, with a negative width, with aux announced but absent
+    kp, bad = arr(grp(wptr=None))
+    assert size(bad, 1) == 0 and plan(bad, 1, 8.0, 1, 0.5, 1, 1, ws, need, C.addressof(k), None) == 1
+    neg = (C.c_int32 * 2)(64, -1)
+    kp, bad = arr(grp(wptr=C.addressof(neg)))
+    assert size(bad, 1) == 0
+    kp, bad = arr(grp(n_aux=1))
+    assert size(bad, 1) == 0
+    # every pair empty: nothing to describe
+    zero = (C.c_int32 * 2)(0, 0)
+    kp, bad = arr(grp(wptr=C.addressof(zero)))
+    assert size(bad, 1) == 0
+    # workspace too small / absent / misaligned
+    assert plan(good, 1, 8.0, 1, 0.5, 1, 1, ws, need - 1, C.addressof(k), None) != 0
+    assert plan(good, 1, 8.0, 1, 0.5, 1, 1, None, need, C.addressof(k), None) != 0
+    assert plan(good, 1, 8.0, 1, 0.5, 1, 1, ws + 4, need, C.addressof(k), None) != 0
+    # apply: out of place without outputs, counts larger than the pair, workspace too small
+    assert apply_(good, 1, C.addressof(k), None, 0, ws, need, None) == 1
+    big = (C.c_int32 * 2)(65, 1)
+    assert apply_(good, 1, C.addressof(big), None, 1, ws, need, None) == 1
+    assert apply_(good, 1, C.addressof(k), None, 1, ws, need - 1, None) != 0
+    assert apply_(good, 1, None, None, 1, ws, need, None) == 1

@@ -179,3 +179,28 @@ def test_run_to_budget_matches_the_oracle_loop(name):
                 assert same_bytes(getattr(g, nm), sp[nm], lay, D), nm
         for (tg, lay), (tr, _) in zip(g.aux, sp["aux"]):
             assert same_bytes(tg, tr, lay, D)
+
+
+def test_a_pair_that_lost_every_index_takes_no_part():
+    """A group described with an empty pair in the middle gives the same pass as the group without it (the empty
+    pair keeps width 0 and is neither scored nor chosen); the reference pass is the oracle-checked one above."""
+    wl = WL.WORKLOADS["tails768"]
+    specs = make_groups(wl)
+    n_samples = float(wl.tokens)
+    ref_groups, ref_info = A1.step([to_gpu(sp) for sp in specs], n_samples, 0.5, 0.85, k_min=2)
+    holed = []
+    for sp in specs:
+        sp = dict(sp)
+        w = list(sp["widths"])
+        sp["widths"] = w[:1] + [0] + w[1:]
+        holed.append(to_gpu(sp))
+    groups, info = A1.step(holed, n_samples, 0.5, 0.85, k_min=2)
+    torch.cuda.synchronize()
+    assert info["n_chosen"] == ref_info["n_chosen"]
+    assert torch.equal(info["fisher"], ref_info["fisher"]) and torch.equal(info["chosen"], ref_info["chosen"])
+    for g, r in zip(groups, ref_groups):
+        assert g.widths == r.widths[:1] + [0] + r.widths[1:]
+        for nm in ("w1", "w2", "g1", "g2"):
+            assert torch.equal(getattr(g, nm), getattr(r, nm))
+        for (a, _), (b, _) in zip(g.aux, r.aux):
+            assert torch.equal(a, b)
