@@ -8,20 +8,22 @@
 // Q K^T, and a zero column of V^c gives a zero column of Ctx) and off_h a multiple of 8, so that every tile load starts
 // on a 16-byte boundary and every contraction is a whole number of 16-deep MMA steps.
 //
-// Forward kernel, one CTA per SM, 576 threads.  A work item is (sequence b, head h, 128 query rows); a CTA walks a
-// static list of items (for causal attention the long ones first).
-//   warp 0      producer: one lane issues the TMA loads of the item's Q tile (2 buffers) and of every K / V tile
-//               (2 stages); a tile is one or two 64-column blocks of 128 rows x 128 bytes, 128-byte swizzle
-//   warp 1      owns TMEM (512 columns: two 128-column score buffers, one output tile of up to 128 columns); one lane
-//               issues S = Q K^T (K-major operands) and O_tile = P V (P from shared memory, V as stored = MN-major)
-//   warps 2..17 softmax, thread = (query row = TMEM lane, quarter of the 128 key columns): row maximum over the score
-//               tile (the four threads of a row exchange their maxima through shared memory), p = 2^(s*c - m) with the
-//               running maximum m, P as bf16 into shared memory (K-major, swizzled) for the second product, and the
-//               running output O = O * 2^(m_old - m_new) + O_tile in registers (each thread its quarter of the columns);
-//               at the end O / l and the row's log-sum-exp are written
-// The score tile of key block j+1 is issued before P V of block j, so the tensor pipe works while the softmax of the
-// next block runs.  Every mbarrier wait is bounded; on expiry the CTA records a code (11 producer, 12 MMA issuer,
-// 13 softmax) in the device status word, lets copies land, frees TMEM and returns.
+// Forward kernel, one CTA per SM, 320 threads.  A work item is (sequence b, head h, two neighbouring tiles of 128 query
+// rows); a CTA walks a static list of items (for causal attention the long ones first).  The two query tiles are two
+// streams that share the K / V tiles and run half a step apart.
+//   warp 0      producer: one lane issues the TMA loads of the item's two Q tiles and of every K / V tile (rings of 2
+//               stages); a tile is one or two 64-column blocks of 128 rows x 128 bytes, 128-byte swizzle
+//   warp 1      owns TMEM (512 columns: a 128-column score tile and an output tile per stream, and the probabilities as
+//               packed bf16); one lane issues S = Q K^T (K-major operands from shared memory) and O_tile = P V (P read
+//               from TMEM, V as stored = MN-major) for both streams
+//   warps 2..5  softmax of stream 0, warps 6..9 of stream 1; thread = query row = TMEM lane, all 128 key columns, so
+//               nothing is exchanged between threads.  Per key block: pass 1 reads the score tile for the row maximum,
+//               folds the previous output tile (O = O * 2^(m_old - m_new) + O_tile, in registers); pass 2 reads the
+//               scores again, p = 2^(s*c - m), packs P to bf16 and writes it to TMEM for the second product.
+// Pass 2 is bound by the exponential unit, pass 1 and the waits on the tensor pipe are not: a token (two mbarriers)
+// lets only one stream at a time through pass 2, so one stream exponentiates while the other reads maxima, folds and
+// waits for its products.  Every mbarrier wait is bounded; on expiry the CTA records a code (11 producer, 12 MMA
+// issuer, 13 softmax) in the device status word, lets copies land, frees TMEM and returns.
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -44,11 +46,9 @@ using namespace tc;
 constexpr int kTile = 128;                  // query rows and key rows per tile
 constexpr int kBlockBytes = kTile * 128;    // one 64-column block of a 128-row tile
 constexpr int kMaxHeads = 128;
-constexpr int kFwdParts = 4;
-constexpr int kFwdThreads = 64 + kFwdParts * 128;   // producer warp, MMA warp, four sets of four softmax warps
+constexpr int kFwdThreads = 64 + 2 * 128;   // producer warp, MMA warp, two streams of four softmax warps
 constexpr int kBwdThreads = 64 + 4 * 128;   // producer warp, MMA warp, four sets of four compute warps
 constexpr int kTmemCols = 512;
-constexpr uint32_t kColS = 0, kColO = 256;  // TMEM columns: score buffers at 0 and 128, output tile at 256
 
 struct HeadLayout {
     int32_t qk_off[kMaxHeads], qk_w[kMaxHeads], vo_off[kMaxHeads], vo_w[kMaxHeads];
@@ -67,44 +67,65 @@ struct AttnFwdParams {
 };
 
 struct Item {
-    int b, h, qt, n_kv;
+    int b, h, qp, n_a, n_b, n;   // query tiles 2 qp and 2 qp + 1 with n_a and n_b key blocks (0: no such tile), n = the larger
 };
 __device__ __forceinline__ Item decode_item(int it, int n_qt, int n_heads, int batch, int n_kt, int causal) {
     Item I;
     const int per = n_heads * batch;
-    I.qt = n_qt - 1 - it / per;             // long (late) query tiles first
+    const int n_qp = (n_qt + 1) >> 1;
+    I.qp = n_qp - 1 - it / per;             // long (late) query tiles first
     const int rem = it % per;
     I.h = rem / batch;
     I.b = rem % batch;
-    I.n_kv = causal ? min(n_kt, I.qt + 1) : n_kt;
+    const int qa = 2 * I.qp, qb = qa + 1;
+    I.n_a = causal ? min(n_kt, qa + 1) : n_kt;
+    I.n_b = qb < n_qt ? (causal ? min(n_kt, qb + 1) : n_kt) : 0;
+    I.n = max(I.n_a, I.n_b);
     return I;
 }
 
 template <int NB>   // 64-column blocks per tile: 1 (every head at most 64 wide) or 2
+struct FwdCfg {
+    static constexpr int kTileBytes = NB * kBlockBytes;
+    static constexpr int QS = NB == 1 ? 2 : 1;                     // buffers of the pair of Q tiles
+    static constexpr int kSmem = (2 * QS + 4) * kTileBytes + 1024 + 256;
+    static constexpr int kOCols = NB * 64;                          // columns of an output tile
+    static constexpr int CH = NB == 1 ? 32 : 16;                    // score columns a thread holds at a time (two such buffers)
+    // TMEM columns of stream x: scores, output tile, probabilities (narrow heads: a region of their own, so that the
+    // next score tile never waits for the second product; wide heads: over the scores they were made from)
+    static __device__ __forceinline__ uint32_t col_s(uint32_t x) { return 128u * x; }
+    static __device__ __forceinline__ uint32_t col_o(uint32_t x) { return 256u + kOCols * x; }
+    static __device__ __forceinline__ uint32_t col_p(uint32_t x) { return NB == 1 ? 384u + 64u * x : 128u * x; }
+};
+
+template <int NB>
 __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_constant__ AttnFwdParams P) {
-    constexpr int kTileBytes = NB * kBlockBytes;
-    constexpr int QS = NB == 1 ? 2 : 1;                      // buffers of the Q tile (wide heads: one, to fit shared memory)
+    using Cfg = FwdCfg<NB>;
+    constexpr int kTileBytes = Cfg::kTileBytes;
+    constexpr int QS = Cfg::QS;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw_addr);
-    const uint32_t sQ = base, sK = sQ + QS * kTileBytes, sV = sK + 2 * kTileBytes, sP = sV + 2 * kTileBytes;
-    float* xchg = reinterpret_cast<float*>(smem + (QS + 4) * kTileBytes + 2 * kBlockBytes);   // [2 phases][4 parts][128 rows]
-    uint8_t* tail = smem + (QS + 4) * kTileBytes + 2 * kBlockBytes + 2 * kFwdParts * kTile * 4;
+    const uint32_t sQ = base, sK = sQ + 2 * QS * kTileBytes, sV = sK + 2 * kTileBytes;
+    uint8_t* tail = smem + (2 * QS + 4) * kTileBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 20 * 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 20 * 8 + 8);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 24 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 24 * 8 + 8);
     const uint32_t bar0 = smem_u32(bars);
     auto q_full = [&](uint32_t s) { return bar0 + 8u * s; };
     auto q_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };
-    // K and V tiles have rings of their own: a K stage is free as soon as the score product that read it is done (one
-    // step earlier than the V stage), so the load of the next K tile is not held up by the second product
+    // K and V tiles have rings of their own: a K stage is free as soon as the score products that read it are done
+    // (one step earlier than the V stage), so the load of the next K tile is not held up by the second products
     auto k_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
     auto k_empty = [&](uint32_t s) { return bar0 + 8u * (6 + s); };
-    auto s_full = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
-    const uint32_t p_full = bar0 + 8u * 10, o_full = bar0 + 8u * 11, x_ready = bar0 + 8u * 12;
-    auto v_full = [&](uint32_t s) { return bar0 + 8u * (13 + s); };
-    auto v_empty = [&](uint32_t s) { return bar0 + 8u * (15 + s); };
+    auto v_full = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
+    auto v_empty = [&](uint32_t s) { return bar0 + 8u * (10 + s); };
+    // per stream: score tile complete, probabilities written, output tile complete, pass-2 token
+    auto s_full = [&](uint32_t x) { return bar0 + 8u * (12 + x); };
+    auto p_full = [&](uint32_t x) { return bar0 + 8u * (14 + x); };
+    auto o_full = [&](uint32_t x) { return bar0 + 8u * (16 + x); };
+    auto token = [&](uint32_t x) { return bar0 + 8u * (18 + x); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_kt = (P.seq + kTile - 1) / kTile;
@@ -117,10 +138,10 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             mbar_init(v_full(s), 1);
             mbar_init(v_empty(s), 1);
             mbar_init(s_full(s), 1);
+            mbar_init(p_full(s), 128);
+            mbar_init(o_full(s), 1);
+            mbar_init(token(s), 128);
         }
-        mbar_init(p_full, kFwdThreads - 64);
-        mbar_init(o_full, 1);
-        mbar_init(x_ready, kFwdThreads - 64);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.map_q);
@@ -145,10 +166,13 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                 const int row0 = I.b * P.seq;
                 const uint32_t qs = qi % QS;
                 if (!(ok = mbar_wait(q_empty(qs), ((qi / QS) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
-                mbar_expect_tx(q_full(qs), nbq * kBlockBytes);
-                for (int blk = 0; blk < nbq; ++blk)
-                    tma_load_2d(sQ + qs * kTileBytes + blk * kBlockBytes, &P.map_q, qoff + 64 * blk, row0 + I.qt * kTile, q_full(qs));
-                for (int j = 0; j < I.n_kv; ++j, ++g) {
+                const int n_tiles = I.n_b > 0 ? 2 : 1;
+                mbar_expect_tx(q_full(qs), n_tiles * nbq * kBlockBytes);
+                for (int x = 0; x < n_tiles; ++x)
+                    for (int blk = 0; blk < nbq; ++blk)
+                        tma_load_2d(sQ + (2 * qs + x) * kTileBytes + blk * kBlockBytes, &P.map_q, qoff + 64 * blk,
+                                    row0 + (2 * I.qp + x) * kTile, q_full(qs));
+                for (int j = 0; j < I.n; ++j, ++g) {
                     const uint32_t st = g & 1;
                     if (!(ok = mbar_wait(k_empty(st), ((g >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
                     mbar_expect_tx(k_full(st), nbq * kBlockBytes);
@@ -164,7 +188,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
-            uint32_t g = 0, qi = 0;
+            uint32_t g = 0, qi = 0, cp[2] = {0, 0};       // cp[x]: probability tiles of stream x consumed so far
             bool ok = true;
             for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++qi) {
                 const Item I = decode_item(it, P.n_qt, P.n_heads, P.batch, n_kt, P.causal);
@@ -173,166 +197,177 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                 if (!(ok = mbar_wait(q_full(qs), (qi / QS) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
                 const uint32_t idesc_s = make_idesc(kTile, kTile, 0, 0);
                 const uint32_t idesc_o = make_idesc(kTile, wv, 0, 1);
-                // S = Q K^T of key block gg into score buffer gg & 1
-                auto issue_scores = [&](uint32_t gg) -> bool {
-                    const uint32_t st = gg & 1;
-                    if (!mbar_wait(k_full(st), (gg >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns)) return false;
-                    tc_fence_after();
+                // S_x = Q_x K^T with the K tile in ring stage st
+                auto scores = [&](uint32_t x, uint32_t st) {
                     for (int ks = 0; ks < (wq >> 4); ++ks) {
                         const uint32_t o = (ks >> 2) * kBlockBytes + (ks & 3) * 32;
-                        tc_mma_bf16(tmem_base + kColS + st * kTile, make_smem_desc(sQ + qs * kTileBytes + o, 16, 1024),
+                        tc_mma_bf16(tmem_base + Cfg::col_s(x), make_smem_desc(sQ + (2 * qs + x) * kTileBytes + o, 16, 1024),
                                     make_smem_desc(sK + st * kTileBytes + o, 16, 1024), idesc_s, ks != 0 ? 1u : 0u);
                     }
-                    tc_commit(s_full(st));
-                    tc_commit(k_empty(st));
+                    tc_commit(s_full(x));
+                };
+                // O_tile_x = P_x V over the 128 keys of the block in ring stage st
+                auto outputs = [&](uint32_t x, uint32_t st) -> bool {
+                    if (!mbar_wait(p_full(x), cp[x] & 1u, abort_flag, 12, P.status, P.wait_limit_ns)) return false;
+                    ++cp[x];
+                    tc_fence_after();
+                    for (int ks = 0; ks < kTile / 16; ++ks)
+                        tc_mma_bf16_ts(tmem_base + Cfg::col_o(x), tmem_base + Cfg::col_p(x) + 8 * ks,
+                                       make_smem_desc(sV + st * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc_o, ks != 0 ? 1u : 0u);
+                    tc_commit(o_full(x));
                     return true;
                 };
-                if (!(ok = issue_scores(g))) break;
-                for (int j = 0; j < I.n_kv; ++j, ++g) {
-                    if (j + 1 < I.n_kv && !(ok = issue_scores(g + 1))) break;
-                    if (!(ok = mbar_wait(p_full, g & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
-                    const uint32_t st = g & 1;
+                if (!(ok = mbar_wait(k_full(g & 1), (g >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                scores(0, g & 1);
+                if (I.n_b > 0) scores(1, g & 1);
+                tc_commit(k_empty(g & 1));
+                for (int j = 0; j < I.n; ++j, ++g) {
+                    const uint32_t st = g & 1, nx = (g + 1) & 1;
                     if (!(ok = mbar_wait(v_full(st), (g >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                    if (j + 1 < I.n && !(ok = mbar_wait(k_full(nx), ((g + 1) >> 1) & 1u, abort_flag, 12, P.status, P.wait_limit_ns))) break;
                     tc_fence_after();
-                    for (int ks = 0; ks < kTile / 16; ++ks)   // O_tile = P V over the 128 keys of the block
-                        tc_mma_bf16(tmem_base + kColO, make_smem_desc(sP + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
-                                    make_smem_desc(sV + st * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc_o, ks != 0 ? 1u : 0u);
-                    tc_commit(o_full);
+                    if (j < I.n_a && !(ok = outputs(0, st))) break;
+                    if (j + 1 < I.n_a) scores(0, nx);
+                    if (j < I.n_b && !(ok = outputs(1, st))) break;
                     tc_commit(v_empty(st));
+                    if (j + 1 < I.n_b) scores(1, nx);
+                    if (j + 1 < I.n) tc_commit(k_empty(nx));
                 }
                 if (ok) tc_commit(q_empty(qs));
             }
         }
     } else {
         // ------------------------------------------------------------------ softmax
-        // Thread = (query row, quarter of the key block's columns): warps 2..5 take columns [0, 32) of the 128 keys,
-        // warps 6..9 [32, 64), and so on, so every scheduler has four softmax warps to interleave.  A thread keeps its
-        // 32 scores in registers (one TMEM read per block).  The four threads of a row agree on the row maximum
-        // through shared memory once per key block; each keeps the sum of its own probabilities (added once, at the
-        // end) and folds its own quarter of the output columns.
-        const int part = (warp - 2) >> 2;
+        const uint32_t x = static_cast<uint32_t>(warp - 2) >> 2;           // stream
         const int row = (warp & 3) * 32 + lane;
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-        // this thread's 32 columns = four 16-byte chunks of block part / 2 of the row's image
-        const uint32_t p_row = sP + (part >> 1) * kBlockBytes + row * 128;
-        const int chunk0 = (part & 1) * 4;
-        const int swz = row & 7;
-        constexpr int kOwn = NB * 16;                                   // output columns this thread folds
-        uint32_t g = 0, xph = 0;
+        const uint32_t tS = t_lane + Cfg::col_s(x), tO = t_lane + Cfg::col_o(x), tP = t_lane + Cfg::col_p(x);
+        constexpr int CH = Cfg::CH, NC = kTile / CH;
+        constexpr int kOwn = Cfg::kOCols;
+        uint32_t cs = 0, turn = 0;                                          // tiles of this stream so far; turns of the token
         bool ok = true;
         const int64_t T = static_cast<int64_t>(P.batch) * P.seq;
         for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x) {
             const Item I = decode_item(it, P.n_qt, P.n_heads, P.batch, n_kt, P.causal);
+            const int n_own = x == 0 ? I.n_a : I.n_b;
             const int wv = P.heads.vo_w[I.h];
-            const int q_pos = I.qt * kTile + row;                     // position of this row in its sequence
-            const int limit = P.causal ? min(P.seq, q_pos + 1) : P.seq;   // keys [0, limit) are visible
+            const int q_pos = (2 * I.qp + static_cast<int>(x)) * kTile + row;   // position of this row in its sequence
+            const int limit = P.causal ? min(P.seq, q_pos + 1) : P.seq;     // keys [0, limit) are visible
             float m = -INFINITY, l = 0.f, alpha_prev = 0.f;
             float o[kOwn];
 #pragma unroll
             for (int i = 0; i < kOwn; ++i) o[i] = 0.f;
-            // O = O * a + O_tile (the output tile of the previous key block), this thread's columns
+            // O = O * a + O_tile (the output tile of the previous key block)
             auto fold_output = [&](float a) {
 #pragma unroll
-                for (int c = 0; c < NB; ++c) {
-                    const int col = part * kOwn + c * 16;
-                    if (col < wv) {
+                for (int c = 0; c < kOwn / 16; ++c) {
+                    if (c * 16 < wv) {
                         uint32_t r[16];
-                        tc_ld16(t_lane + kColO + col, r);
-                        tc_wait_ld();
+                        tc_ld16(tO + c * 16, r);
+                        tc_wait_ld(r);
 #pragma unroll
                         for (int i = 0; i < 16; ++i) o[c * 16 + i] = fmaf(o[c * 16 + i], a, __uint_as_float(r[i]));
                     }
                 }
             };
-            // values of the row's other threads: through xchg[phase & 1][part][row], one mbarrier phase per exchange
-            auto exchange = [&](float v, float (&others)[3]) -> bool {
-                float* buf = xchg + (xph & 1) * kFwdParts * kTile;
-                buf[part * kTile + row] = v;
-                mbar_arrive(x_ready);
-                if (!mbar_wait(x_ready, xph & 1u, abort_flag, 13, P.status, P.wait_limit_ns)) return false;
-#pragma unroll
-                for (int k = 0; k < 3; ++k) others[k] = buf[((part + 1 + k) & 3) * kTile + row];
-                ++xph;
-                return true;
-            };
-            for (int j = 0; j < I.n_kv; ++j, ++g) {
-                const uint32_t sb = g & 1;
-                if (!(ok = mbar_wait(s_full(sb), (g >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
-                tc_fence_after();
-                const int kv0 = j * kTile + part * 32;                // first key of this thread's columns
-                uint32_t r[32];
-                tc_ld32(t_lane + kColS + sb * kTile + part * 32, r);
-                tc_wait_ld();
-                if (kv0 + 32 > limit) {                               // keys past the limit count as -inf
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (kv0 + i >= limit) r[i] = 0xff800000u;
-                }
-                // maximum over this thread's columns (four independent chains), then over the row
-                float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(r[i]));
-                float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), mo[3];
-                if (!(ok = exchange(mx, mo))) break;
-                mx = fmaxf(fmaxf(mx, mo[0]), fmaxf(mo[1], mo[2]));
-                const float m_new = fmaxf(m, mx * P.scale_log2e);
-                const float alpha = ex2(m - m_new);
-                if (j > 0) {
-                    if (!(ok = mbar_wait(o_full, (g - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+            for (int j = 0; j < I.n; ++j, ++turn) {
+                const bool active = j < n_own;
+                const int kv_base = j * kTile;
+                const bool masked = kv_base + kTile > limit;               // keys past the limit count as -inf
+                float m_new = m, alpha = 1.f;
+                if (active) {
+                    if (!(ok = mbar_wait(s_full(x), cs & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
                     tc_fence_after();
-                    fold_output(alpha_prev);
-                }
-                // p = 2^(s * c - m_new) (2^-inf = 0 for the masked keys), row sum, P as bf16 into shared memory
-                float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+                    // pass 1: row maximum (four independent chains); the next chunk is in flight while one is reduced
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+                    uint32_t ra[CH], rb[CH];
+                    tc_ld(tS, ra);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    float p[8];
+                    for (int c = 0; c < NC; ++c) {
+                        uint32_t(&cur)[CH] = (c & 1) ? rb : ra;
+                        uint32_t(&nxt)[CH] = (c & 1) ? ra : rb;
+                        tc_wait_ld(cur);
+                        if (c + 1 < NC) tc_ld(tS + (c + 1) * CH, nxt);
+                        if (masked) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        p[i] = ex2(fmaf(__uint_as_float(r[8 * q + i]), P.scale_log2e, -m_new));
-                        rs4[i & 3] += p[i];
+                            for (int i = 0; i < CH; ++i)
+                                if (kv_base + c * CH + i >= limit) cur[i] = 0xff800000u;
+                        }
+#pragma unroll
+                        for (int i = 0; i < CH; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(cur[i]));
                     }
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(p_row + (((chunk0 + q) ^ swz) << 4)),
-                                 "r"(pack_bf16(p[0], p[1])), "r"(pack_bf16(p[2], p[3])), "r"(pack_bf16(p[4], p[5])),
-                                 "r"(pack_bf16(p[6], p[7]))
-                                 : "memory");
+                    const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+                    m_new = fmaxf(m, mx * P.scale_log2e);
+                    alpha = ex2(m - m_new);
+                    if (j > 0) {
+                        if (!(ok = mbar_wait(o_full(x), (cs - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                        tc_fence_after();
+                        fold_output(alpha_prev);
+                    }
                 }
-                fence_async_smem();
-                tc_fence_before();
-                mbar_arrive(p_full);
-                l = fmaf(l, alpha, (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
-                m = m_new;
-                alpha_prev = alpha;
+                // the token: stream 0 goes first, then the streams alternate
+                if (!(ok = mbar_wait(token(x), x == 0 ? (turn & 1u) ^ 1u : turn & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+                if (active) {
+                    // pass 2: p = 2^(s * c - m_new) (2^-inf = 0 for the masked keys), row sum, P as packed bf16 into TMEM
+                    uint32_t ra[CH], rb[CH];
+                    tc_ld(tS, ra);
+#pragma unroll
+                    for (int c = 0; c < NC; ++c) {
+                        uint32_t(&cur)[CH] = (c & 1) ? rb : ra;
+                        uint32_t(&nxt)[CH] = (c & 1) ? ra : rb;
+                        tc_wait_ld(cur);
+                        if (c + 1 < NC) tc_ld(tS + (c + 1) * CH, nxt);
+                        if (masked) {
+#pragma unroll
+                            for (int i = 0; i < CH; ++i)
+                                if (kv_base + c * CH + i >= limit) cur[i] = 0xff800000u;
+                        }
+                        uint32_t pk[CH / 2];
+#pragma unroll
+                        for (int i = 0; i < CH; i += 2) {
+                            const float p0 = ex2(fmaf(__uint_as_float(cur[i]), P.scale_log2e, -m_new));
+                            const float p1 = ex2(fmaf(__uint_as_float(cur[i + 1]), P.scale_log2e, -m_new));
+                            rs4[(i >> 1) & 3] += p0 + p1;
+                            pk[i >> 1] = pack_bf16(p0, p1);
+                        }
+                        tc_st(tP + c * (CH / 2), pk);
+                    }
+                }
+                mbar_arrive(token(x ^ 1u));
+                if (active) {
+                    tc_wait_st();
+                    tc_fence_before();
+                    mbar_arrive(p_full(x));
+                    l = fmaf(l, alpha, (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]));
+                    m = m_new;
+                    alpha_prev = alpha;
+                    ++cs;
+                }
             }
             if (!ok) break;
-            if (!(ok = mbar_wait(o_full, (g - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
-            tc_fence_after();
-            fold_output(alpha_prev);
-            float lo[3];
-            if (!(ok = exchange(l, lo))) break;
-            {   // every thread of the row adds the four partial sums in the order of the parts
-                float lp[4];
-                lp[part] = l;
+            if (n_own > 0) {
+                if (!(ok = mbar_wait(o_full(x), (cs - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                fold_output(alpha_prev);
+                if (q_pos < P.seq) {
+                    const int64_t t = static_cast<int64_t>(I.b) * P.seq + q_pos;
+                    const float inv = 1.f / l;
+                    uint16_t* dst = P.ctx + t * P.ld_ctx + P.heads.vo_off[I.h];
 #pragma unroll
-                for (int k = 0; k < 3; ++k) lp[(part + 1 + k) & 3] = lo[k];
-                l = (lp[0] + lp[1]) + (lp[2] + lp[3]);
-            }
-            if (q_pos < P.seq) {
-                const int64_t t = static_cast<int64_t>(I.b) * P.seq + q_pos;
-                const float inv = 1.f / l;
-                uint16_t* dst = P.ctx + t * P.ld_ctx + P.heads.vo_off[I.h] + part * kOwn;
-#pragma unroll
-                for (int c = 0; c < NB * 2; ++c) {
-                    if (part * kOwn + c * 8 < wv) {
-                        uint4 v;
-                        v.x = pack_bf16(o[c * 8 + 0] * inv, o[c * 8 + 1] * inv);
-                        v.y = pack_bf16(o[c * 8 + 2] * inv, o[c * 8 + 3] * inv);
-                        v.z = pack_bf16(o[c * 8 + 4] * inv, o[c * 8 + 5] * inv);
-                        v.w = pack_bf16(o[c * 8 + 6] * inv, o[c * 8 + 7] * inv);
-                        *reinterpret_cast<uint4*>(dst + c * 8) = v;
+                    for (int c = 0; c < kOwn / 8; ++c) {
+                        if (c * 8 < wv) {
+                            uint4 v;
+                            v.x = pack_bf16(o[c * 8 + 0] * inv, o[c * 8 + 1] * inv);
+                            v.y = pack_bf16(o[c * 8 + 2] * inv, o[c * 8 + 3] * inv);
+                            v.z = pack_bf16(o[c * 8 + 4] * inv, o[c * 8 + 5] * inv);
+                            v.w = pack_bf16(o[c * 8 + 6] * inv, o[c * 8 + 7] * inv);
+                            *reinterpret_cast<uint4*>(dst + c * 8) = v;
+                        }
                     }
+                    P.lse[static_cast<int64_t>(I.h) * T + t] = m * 0.6931471805599453f + logf(l);
                 }
-                if (part == 0) P.lse[static_cast<int64_t>(I.h) * T + t] = m * 0.6931471805599453f + logf(l);
             }
         }
     }
@@ -845,9 +880,6 @@ ecospa_status_t check_mat(const void* p, int64_t ld, int64_t cols) {
     return ECOSPA_OK;
 }
 
-template <typename Params>
-size_t fwd_smem_bytes(int nb) { return static_cast<size_t>((nb == 1 ? 6 : 5) * nb + 2) * kBlockBytes + 2 * kFwdParts * kTile * 4 + 1024 + 256; }
-
 }  // namespace
 
 }  // namespace ecospa
@@ -879,7 +911,7 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
     P.n_heads = heads->n_heads;
     P.n_qt = static_cast<int32_t>(ceil_div(seq, kTile));
     P.causal = causal != 0;
-    const int64_t items = static_cast<int64_t>(P.n_qt) * P.n_heads * batch;
+    const int64_t items = static_cast<int64_t>((P.n_qt + 1) / 2) * P.n_heads * batch;   // pairs of query tiles
     if (items > INT32_MAX) return ECOSPA_ERR_UNSUPPORTED;
     P.n_items = static_cast<int32_t>(items);
     P.scale_log2e = scale * 1.4426950408889634f;
@@ -889,15 +921,14 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
     P.status = status;
     P.wait_limit_ns = engine_wait_limit_ns();
     const int nb = max_w > 64 ? 2 : 1;
-    const size_t smem = fwd_smem_bytes<AttnFwdParams>(nb);
+    const size_t smem = nb == 1 ? FwdCfg<1>::kSmem : FwdCfg<2>::kSmem;
     static std::once_flag once[64];
     int dev = 0;
     cudaGetDevice(&dev);
     cudaError_t e = cudaSuccess;
     std::call_once(once[dev & 63], [&] {
-        e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fwd_smem_bytes<AttnFwdParams>(1)));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(fwd_smem_bytes<AttnFwdParams>(2)));
+        e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<1>::kSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<2>::kSmem);
     });
     if (e != cudaSuccess) {
         set_cuda_error(e, "attention setup");
