@@ -8,9 +8,11 @@
 // Q K^T, and a zero column of V^c gives a zero column of Ctx) and off_h a multiple of 8, so that every tile load starts
 // on a 16-byte boundary and every contraction is a whole number of 16-deep MMA steps.
 //
-// Forward kernel, one CTA per SM, 320 threads.  A work item is (sequence b, head h, two neighbouring tiles of 128 query
-// rows); a CTA walks a static list of items (for causal attention the long ones first).  The two query tiles are two
-// streams that share the K / V tiles and run half a step apart.
+// Two forward kernels, one CTA per SM.  Output heads up to 32 wide (with Q/K heads up to 64) take the kernel of
+// independent key streams further down (attn_fwd_ms_kernel); wider heads take the kernel described here, 320 threads.
+// A work item is (sequence b, head h, two neighbouring tiles of 128 query rows); a CTA walks a static list of items
+// (for causal attention the long ones first).  The two query tiles are two streams that share the K / V tiles and run
+// half a step apart.
 //   warp 0      producer: one lane issues the TMA loads of the item's two Q tiles and of every K / V tile (rings of 2
 //               stages); a tile is one or two 64-column blocks of 128 rows x 128 bytes, 128-byte swizzle
 //   warp 1      owns TMEM (512 columns: a 128-column score tile and an output tile per stream, and the probabilities as
@@ -381,6 +383,451 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// forward, heads up to 64 wide: NS independent streams per CTA
+// ------------------------------------------------------------------------------------------------
+// A work item is (sequence b, head h, one tile of 128 query rows).  A K / V tile holds NS slices of 64 keys; stream x
+// (four warps, thread = query row) owns slice x of every tile and keeps a softmax of its own over its keys: reference
+// exponent m_x, sum l_x, and the output O_x = sum_j P_x(j) V_x(j) accumulating in TMEM.  At the end of the item the NS
+// partial results of a row are merged (M = max m_x, weights 2^(m_x - M)).  The streams never wait for one another inside
+// an item, so while one waits for its products the others keep the exponential unit busy.
+// One pass per score slice: p = 2^(s*c - m) with the reference m the stream already has; m moves only when a score
+// exceeds it by more than 32 (2^32 headroom in fp32 / bf16, whose relative precision does not depend on the scale), in
+// which case the row's l, O and the probabilities already written for the slice are rescaled first, so no exponent
+// can overflow.  The first slice of an item starts from m = -1e30 and takes that path once.
+// A stream has two score buffers: S_x of slice G + 1 is computed while the stream exponentiates slice G, so a stream goes
+// from one slice to the next without waiting for the tensor pipe.  The probabilities of a slice overwrite the first half
+// of the score buffer they were made from (chunk c of 32 scores becomes 16 packed columns at 16 c, inside columns
+// that are already in registers).  TMEM columns of stream x: score buffers at 128 x and 128 x + 64, output 128 NS + OC x.
+template <int NS, int OC>
+struct MsCfg {
+    // per stream: one warp that loads the stream's K / V slices and issues its products, and four softmax warps
+    static constexpr int kThreads = 32 * NS + 128 * NS;
+    static constexpr int kSlice = 64;
+    static constexpr int kKeys = NS * kSlice;                 // keys per K / V tile
+    static constexpr int kSliceBytes = kSlice * 128;          // one slice: 64 rows x 128 bytes
+    static constexpr int kStages = 3;                         // K and V slices per stream: slice s uses stage s % 3
+    static constexpr int kRingBytes = NS * 2 * kStages * kSliceBytes;
+    static constexpr int kMergeBytes = 2 * NS * kTile * 4;    // m and l of every stream and row
+    static constexpr int kSmem = 2 * kBlockBytes + kRingBytes + kMergeBytes + 1024 + 512;
+    static __device__ __forceinline__ uint32_t col_s(uint32_t x, uint32_t buf) { return 128u * x + 64u * buf; }
+    static __device__ __forceinline__ uint32_t col_o(uint32_t x) { return 128u * NS + OC * x; }
+    static_assert(128 * NS + OC * NS <= kTmemCols, "TMEM columns");
+};
+
+struct MsItem {
+    int b, h, qt, lim;          // lim: last key position any row of the tile sees
+};
+__device__ __forceinline__ MsItem ms_decode(int it, int n_qt, int n_heads, int batch, int seq, int causal) {
+    MsItem I;
+    const int per = n_heads * batch;
+    I.qt = n_qt - 1 - it / per;             // long (late) query tiles first
+    const int rem = it % per;
+    I.h = rem / batch;
+    I.b = rem % batch;
+    I.lim = causal ? min(I.qt * kTile + kTile - 1, seq - 1) : seq - 1;
+    return I;
+}
+// K / V tiles in which slice x has a visible key
+__device__ __forceinline__ int ms_steps(int lim, int x, int keys_per_tile) {
+    const int first = 64 * x;
+    return lim >= first ? (lim - first) / keys_per_tile + 1 : 0;
+}
+
+struct RowState {
+    float m, l, rs;
+};
+// The rare path of a slice: a score exceeds the row's reference exponent by more than 32.  Moves the reference to that
+// score and rescales what was computed with the old one: the sums, the output row in TMEM (o_groups 16-column groups; 0
+// while the stream has no output yet) and the probability chunks of this slice written so far.  Called by whole warps.
+__device__ __forceinline__ RowState rescale_row(RowState s, float cm, uint32_t tO, int o_groups, uint32_t tP, int chunks_done) {
+    const bool need = cm - s.m > 32.f;
+    const float m_new = need ? cm : s.m;
+    const float f = need ? ex2(s.m - m_new) : 1.f;
+    tc_wait_st();                            // the chunks written so far are read back below
+    for (int g = 0; g < o_groups; ++g) {
+        uint32_t r[16];
+        tc_ld16(tO + 16 * g, r);
+        tc_wait_ld(r);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+        tc_st(tO + 16 * g, r);
+    }
+    for (int c = 0; c < chunks_done; ++c) {
+        uint32_t r[16];
+        tc_ld16(tP + 16 * c, r);
+        tc_wait_ld(r);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) r[i] = pack_bf16(bf16_lo(r[i]) * f, bf16_hi(r[i]) * f);
+        tc_st(tP + 16 * c, r);
+    }
+    tc_wait_st();
+    RowState o;
+    o.m = m_new;
+    o.l = s.l * f;
+    o.rs = s.rs * f;
+    return o;
+}
+
+template <int NS, int OC>
+__global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel(const __grid_constant__ AttnFwdParams P) {
+    using Cfg = MsCfg<NS, OC>;
+    constexpr int kSliceB = Cfg::kSliceBytes, kKeys = Cfg::kKeys, ST = Cfg::kStages;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw_addr = smem_u32(smem_raw);
+    const uint32_t base = (raw_addr + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw_addr);
+    const uint32_t sQ = base, sK = sQ + 2 * kBlockBytes, sV = sK + NS * ST * kSliceB;   // K / V: [stream][stage] slices
+    float* merge = reinterpret_cast<float*>(smem + 2 * kBlockBytes + Cfg::kRingBytes);   // [m | l][stream][row]
+    uint8_t* tail = smem + 2 * kBlockBytes + Cfg::kRingBytes + Cfg::kMergeBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 60 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 60 * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto q_full = [&](uint32_t s) { return bar0 + 8u * s; };
+    auto q_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };     // one arrival per stream and item
+    // Per stream and score buffer (slice G uses buffer G & 1): probabilities written; the product that read them done.
+    // Two barriers each, because a stream runs ahead of its issuer by one slice: with one barrier the phases of slices
+    // G and G + 1 could both complete before the waiter has looked at the first.
+    auto p_full = [&](uint32_t x, uint32_t buf) { return bar0 + 8u * (4 + 2 * x + buf); };
+    auto pv_done = [&](uint32_t x, uint32_t buf) { return bar0 + 8u * (42 + 2 * x + buf); };
+    auto s_full = [&](uint32_t x, uint32_t buf) { return bar0 + 8u * (12 + 2 * x + buf); };   // scores in buffer buf of stream x
+    auto kv_full = [&](uint32_t x, uint32_t b) { return bar0 + 8u * (20 + 2 * x + b); };      // the loads event G needs (b = G & 1) landed
+    const uint32_t merge_a = bar0 + 8u * 40, merge_b = bar0 + 8u * 41;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < 2; ++s) {
+            mbar_init(q_full(s), 1);
+            mbar_init(q_empty(s), NS);
+            for (uint32_t x = 0; x < NS; ++x) {
+                mbar_init(kv_full(x, s), 1);
+                mbar_init(s_full(x, s), 1);
+                mbar_init(p_full(x, s), 128);
+                mbar_init(pv_done(x, s), 1);
+            }
+        }
+        mbar_init(merge_a, 128 * NS);
+        mbar_init(merge_b, 128 * NS);
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&P.map_q);
+        prefetch_tensormap(&P.map_k);
+        prefetch_tensormap(&P.map_v);
+    }
+    if (warp == 0) tmem_alloc(smem_u32(tmem_holder), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_holder;
+
+    if (warp < NS) {
+        // ------------------------------------------------------------------ loader and MMA issuer of stream x
+        // The stream's slices form one sequence G = 0, 1, ... across the CTA's items (items in which the stream has no
+        // visible key are skipped).  Event G: the probabilities of slice G are written -> O_x += P_x V_x (slice G), then
+        // S_x of slice G + 2 into the score buffer that slice G occupied, then the loads of the K slice G + 3 and of the V
+        // slice G + 1.  Their stages (slice s uses stage s % 3) are free: S(G) was read by the softmax, and P V(G - 2) was
+        // issued before S(G), whose completion signal covers it.  Both loads report to the barrier event G + 1 waits on.
+        // This thread shares its scheduler with the stream's softmax warps, so the loop is kept short: slices are
+        // described by three packed registers produced once (next()) and handed from stage to stage.
+        if (lane == 0) {
+            const uint32_t x = warp;
+            const uint32_t tS = tmem_base + Cfg::col_s(x, 0), tO = tmem_base + Cfg::col_o(x);
+            const uint32_t idesc_s = make_idesc(kTile, 64, 0, 0);
+            const uint32_t sKx = sK + x * ST * kSliceB, sVx = sV + x * ST * kSliceB;
+            const uint64_t dq0 = make_smem_desc(sQ, 16, 1024), dk0 = make_smem_desc(sKx, 16, 1024),
+                           dv0 = make_smem_desc(sVx, kBlockBytes, 1024);
+            // meta bits: 0 valid, 1 first slice of its item, 2 last, 3 Q buffer, 4 phase of that buffer, 5-7 contraction
+            // steps of the scores, 8-11 output width / 16, 12-.. items skipped just before (first slices and the end mark)
+            struct SD {
+                int row;            // first key row of the slice in the K / V tensors
+                int qrow;           // first row of the item's query tile
+                uint32_t cols;      // first Q/K column | first V column << 16
+                uint32_t meta;
+            };
+            // generator of the stream's slice sequence
+            int g_it = static_cast<int>(blockIdx.x) - static_cast<int>(gridDim.x), g_J = 0, g_n = 0, g_row = 0, g_qrow = 0;
+            uint32_t g_cols = 0, g_meta = 0, g_qi = ~0u, g_skip = 0;
+            auto next = [&]() {
+                SD d;
+                if (g_J >= g_n) {
+                    for (;;) {
+                        g_it += gridDim.x;
+                        ++g_qi;
+                        if (g_it >= P.n_items) {   // end mark; it carries the Q buffers still to hand back
+                            d.row = 0;
+                            d.cols = 0;
+                            d.meta = ((g_qi & 1u) << 3) | (g_skip << 12);
+                            g_skip = 0;
+                            g_it -= gridDim.x;      // stay at the end: later calls give the mark again, with no count
+                            --g_qi;
+                            g_J = g_n = 0;
+                            d.qrow = 0;
+                            return d;
+                        }
+                        const MsItem I = ms_decode(g_it, P.n_qt, P.n_heads, P.batch, P.seq, P.causal);
+                        g_n = ms_steps(I.lim, x, kKeys);
+                        if (g_n == 0) {
+                            ++g_skip;
+                            continue;
+                        }
+                        g_J = 0;
+                        g_row = I.b * P.seq + 64 * static_cast<int>(x);
+                        g_qrow = I.b * P.seq + I.qt * kTile;
+                        g_cols = static_cast<uint32_t>(P.heads.qk_off[I.h]) | (static_cast<uint32_t>(P.heads.vo_off[I.h]) << 16);
+                        g_meta = 1u | ((g_qi & 1u) << 3) | (((g_qi >> 1) & 1u) << 4) | (static_cast<uint32_t>(P.heads.qk_w[I.h] >> 4) << 5) |
+                                 (static_cast<uint32_t>(P.heads.vo_w[I.h] >> 4) << 8);
+                        break;
+                    }
+                }
+                d.row = g_row + g_J * kKeys;
+                d.qrow = g_qrow;
+                d.cols = g_cols;
+                d.meta = g_meta | (g_J == 0 ? 2u | (g_skip << 12) : 0u) | (g_J == g_n - 1 ? 4u : 0u);
+                if (g_J == 0) g_skip = 0;
+                ++g_J;
+                return d;
+            };
+            bool ok = true;
+            // K slice of d into stage st (stream 0: with the Q tile of the item when d is its first slice)
+            auto load_k = [&](const SD& d, uint32_t st, uint32_t bar) -> bool {
+                if (x == 0 && (d.meta & 2u)) {
+                    const uint32_t qs = (d.meta >> 3) & 1u, ph = (d.meta >> 4) & 1u;
+                    if (!mbar_wait(q_empty(qs), ph ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns)) return false;
+                    mbar_expect_tx(q_full(qs), kBlockBytes);
+                    tma_load_2d(sQ + qs * kBlockBytes, &P.map_q, d.cols & 0xffffu, d.qrow, q_full(qs));
+                }
+                tma_load_2d(sKx + st * kSliceB, &P.map_k, d.cols & 0xffffu, d.row, bar);
+                return true;
+            };
+            auto load_v = [&](const SD& d, uint32_t st, uint32_t bar) {
+                tma_load_2d(sVx + st * kSliceB, &P.map_v, d.cols >> 16, d.row, bar);
+            };
+            auto hand_back = [&](uint32_t qs_of_item, uint32_t n) {   // Q buffers of the n items before the one whose buffer is given
+                for (uint32_t k = 1; k <= n; ++k) tc_commit(q_empty((qs_of_item + k) & 1u));
+            };
+            // S_x of slice d (its K slice in stage st) into score buffer buf
+            auto scores = [&](SD& d, uint32_t st, uint32_t buf) -> bool {
+                const uint32_t qs = (d.meta >> 3) & 1u;
+                if (!(d.meta & 1u)) {               // the end mark: only the hand-backs, once
+                    hand_back(qs, d.meta >> 12);
+                    d.meta &= 0xfffu;
+                    return true;
+                }
+                if (d.meta & 2u) {
+                    hand_back(qs, d.meta >> 12);
+                    if (!mbar_wait(q_full(qs), (d.meta >> 4) & 1u, abort_flag, 12, P.status, P.wait_limit_ns)) return false;
+                    tc_fence_after();
+                }
+                const uint64_t dq = dq0 + qs * (kBlockBytes >> 4), dk = dk0 + st * (kSliceB >> 4);
+                const uint32_t ksteps = (d.meta >> 5) & 7u, t = tS + 64 * buf;
+                tc_mma_bf16(t, dq, dk, idesc_s, 0u);
+                if (ksteps > 1) tc_mma_bf16(t, dq + 2, dk + 2, idesc_s, 1u);
+                if (ksteps > 2) tc_mma_bf16(t, dq + 4, dk + 4, idesc_s, 1u);
+                if (ksteps > 3) tc_mma_bf16(t, dq + 6, dk + 6, idesc_s, 1u);
+                tc_commit(s_full(x, buf));
+                if (d.meta & 4u) tc_commit(q_empty(qs));
+                return true;
+            };
+            SD d0 = next(), d1 = next(), d2 = next(), d3;
+            {   // start: K slices 0..2 and V slice 0 on the barrier event 0 waits on
+                const uint32_t nk = (d0.meta & 1u) + (d1.meta & 1u) + (d2.meta & 1u);
+                if (nk) mbar_expect_tx(kv_full(x, 0), (nk + 1) * kSliceB);
+                if (d0.meta & 1u) {
+                    ok = load_k(d0, 0, kv_full(x, 0));
+                    load_v(d0, 0, kv_full(x, 0));
+                }
+                if (ok && (d1.meta & 1u)) ok = load_k(d1, 1, kv_full(x, 0));
+                if (ok && (d2.meta & 1u)) ok = load_k(d2, 2, kv_full(x, 0));
+                if (ok && nk) ok = mbar_wait(kv_full(x, 0), 0u, abort_flag, 12, P.status, P.wait_limit_ns);
+                tc_fence_after();
+                ok = ok && scores(d0, 0, 0) && scores(d1, 1, 1);
+            }
+            uint32_t G = 0, st0 = 0;                // st0 = G % 3
+            while (ok && (d0.meta & 1u)) {
+                const uint32_t buf = G & 1u, ph = (G >> 1) & 1u;
+                const uint32_t st1 = st0 == 2 ? 0 : st0 + 1, st2 = st1 == 2 ? 0 : st1 + 1;
+                if (!(ok = mbar_wait(p_full(x, buf), ph, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                if (G > 0 && !(ok = mbar_wait(kv_full(x, buf), ph, abort_flag, 12, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                {   // O_x += P_x V_x over the slice's 64 keys
+                    const uint32_t idesc_o = make_idesc(kTile, ((d0.meta >> 8) & 15u) << 4, 0, 1);
+                    const uint64_t dv = dv0 + st0 * (kSliceB >> 4);
+                    const uint32_t tP = tS + 64 * buf;
+                    tc_mma_bf16_ts(tO, tP, dv, idesc_o, (d0.meta & 2u) ? 0u : 1u);
+                    tc_mma_bf16_ts(tO, tP + 8, dv + 128, idesc_o, 1u);
+                    tc_mma_bf16_ts(tO, tP + 16, dv + 256, idesc_o, 1u);
+                    tc_mma_bf16_ts(tO, tP + 24, dv + 384, idesc_o, 1u);
+                    tc_commit(pv_done(x, buf));
+                }
+                if (!(ok = scores(d2, st2, buf))) break;      // slice G + 2
+                d3 = next();                                   // slice G + 3
+                {
+                    const uint32_t nb = (d3.meta & 1u) + (d1.meta & 1u), bar = kv_full(x, buf ^ 1u);
+                    if (nb) mbar_expect_tx(bar, nb * kSliceB);
+                    if ((d3.meta & 1u) && !(ok = load_k(d3, st0, bar))) break;
+                    if (d1.meta & 1u) load_v(d1, st1, bar);
+                }
+                d0 = d1;
+                d1 = d2;
+                d2 = d3;
+                st0 = st1;
+                ++G;
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ softmax streams
+        const uint32_t x = static_cast<uint32_t>(warp - NS) >> 2;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+        const uint32_t tS0 = t_lane + Cfg::col_s(x, 0), tO = t_lane + Cfg::col_o(x);
+        constexpr int CH = 32, NC = 64 / CH;
+        uint32_t cs = 0, mi = 0;             // slices of this stream so far, items
+        bool ok = true, pending_b = false;
+        const int64_t T = static_cast<int64_t>(P.batch) * P.seq;
+        for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++mi) {
+            const MsItem I = ms_decode(it, P.n_qt, P.n_heads, P.batch, P.seq, P.causal);
+            const int n_own = ms_steps(I.lim, x, kKeys);
+            const int wv = P.heads.vo_w[I.h];
+            const int q_pos = I.qt * kTile + row;
+            const int limit = P.causal ? min(P.seq, q_pos + 1) : P.seq;     // keys [0, limit) are visible
+            RowState rsx;
+            rsx.m = -1e30f;
+            rsx.l = 0.f;
+            for (int j = 0; j < n_own; ++j) {
+                if (!(ok = mbar_wait(s_full(x, cs & 1), (cs >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                const uint32_t tS = tS0 + 64 * (cs & 1), tP = tS;    // the probabilities go over the scores they came from
+                const int kv_base = j * kKeys + 64 * static_cast<int>(x);
+                const bool masked = kv_base + 64 > limit;                   // keys past the limit count as -inf
+                float rs4[4] = {0.f, 0.f, 0.f, 0.f};
+                uint32_t ra[CH], rb[CH];
+                tc_ld(tS, ra);
+#pragma unroll
+                for (int c = 0; c < NC; ++c) {
+                    uint32_t(&cur)[CH] = (c & 1) ? rb : ra;
+                    uint32_t(&nxt)[CH] = (c & 1) ? ra : rb;
+                    tc_wait_ld(cur);
+                    if (c + 1 < NC) tc_ld(tS + (c + 1) * CH, nxt);
+                    if (masked) {
+#pragma unroll
+                        for (int i = 0; i < CH; ++i)
+                            if (kv_base + c * CH + i >= limit) cur[i] = 0xff800000u;
+                    }
+                    float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+                    for (int i = 0; i < CH; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(cur[i]));
+                    const float cm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * P.scale_log2e;
+                    if (__any_sync(0xffffffffu, cm - rsx.m > 32.f)) {
+                        // the output row is touched: the product of the previous slice must have landed
+                        if (j > 0 && !(ok = mbar_wait(pv_done(x, (cs - 1) & 1), ((cs - 1) >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                        tc_fence_after();
+                        rsx.rs = (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+                        rsx = rescale_row(rsx, cm, tO, j > 0 ? wv >> 4 : 0, tP, c);
+                        rs4[0] = rsx.rs;
+                        rs4[1] = rs4[2] = rs4[3] = 0.f;
+                    }
+                    const float neg_m = -rsx.m;
+                    uint32_t pk[CH / 2];
+#pragma unroll
+                    for (int i = 0; i < CH; i += 2) {
+                        const float p0 = ex2(fmaf(__uint_as_float(cur[i]), P.scale_log2e, neg_m));
+                        const float p1 = ex2(fmaf(__uint_as_float(cur[i + 1]), P.scale_log2e, neg_m));
+                        rs4[(i >> 1) & 3] += p0 + p1;
+                        pk[i >> 1] = pack_bf16(p0, p1);
+                    }
+                    tc_st(tP + c * (CH / 2), pk);
+                }
+                if (!ok) break;
+                tc_wait_st();
+                tc_fence_before();
+                if (pending_b) {   // the output regions of the previous item have been read by every stream
+                    if (!(ok = mbar_wait(merge_b, (mi - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                    pending_b = false;
+                }
+                mbar_arrive(p_full(x, cs & 1));
+                rsx.l += (rs4[0] + rs4[1]) + (rs4[2] + rs4[3]);
+                ++cs;
+            }
+            if (!ok) break;
+            if (n_own > 0) {   // the stream's last product of the item
+                if (!(ok = mbar_wait(pv_done(x, (cs - 1) & 1), ((cs - 1) >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+            }
+            if (pending_b) {       // (a stream without slices in this item)
+                if (!(ok = mbar_wait(merge_b, (mi - 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+                pending_b = false;
+            }
+            // merge of the row's NS partial results
+            merge[x * kTile + row] = rsx.m;
+            merge[(NS + x) * kTile + row] = rsx.l;
+            mbar_arrive(merge_a);
+            if (!(ok = mbar_wait(merge_a, mi & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
+            float gk[NS], M = -INFINITY, L = 0.f;
+#pragma unroll
+            for (int k = 0; k < NS; ++k)
+                if (ms_steps(I.lim, k, kKeys) > 0) M = fmaxf(M, merge[k * kTile + row]);
+#pragma unroll
+            for (int k = 0; k < NS; ++k) {
+                gk[k] = 0.f;
+                if (ms_steps(I.lim, k, kKeys) > 0) {
+                    gk[k] = ex2(merge[k * kTile + row] - M);
+                    L = fmaf(merge[(NS + k) * kTile + row], gk[k], L);
+                }
+            }
+            const float inv = 1.f / L;
+            const bool live = q_pos < P.seq;
+            const int64_t t = static_cast<int64_t>(I.b) * P.seq + q_pos;
+            for (int grp = x; grp < (wv >> 4); grp += NS) {   // this stream's share of the output columns
+                float acc[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) acc[i] = 0.f;
+#pragma unroll
+                for (int k = 0; k < NS; ++k) {
+                    if (ms_steps(I.lim, k, kKeys) > 0) {
+                        uint32_t r[16];
+                        tc_ld16(t_lane + Cfg::col_o(k) + 16 * grp, r);
+                        tc_wait_ld(r);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) acc[i] = fmaf(__uint_as_float(r[i]), gk[k], acc[i]);
+                    }
+                }
+                if (live) {
+                    uint16_t* dst = P.ctx + t * P.ld_ctx + P.heads.vo_off[I.h] + 16 * grp;
+                    uint4 v0, v1;
+                    v0.x = pack_bf16(acc[0] * inv, acc[1] * inv);
+                    v0.y = pack_bf16(acc[2] * inv, acc[3] * inv);
+                    v0.z = pack_bf16(acc[4] * inv, acc[5] * inv);
+                    v0.w = pack_bf16(acc[6] * inv, acc[7] * inv);
+                    v1.x = pack_bf16(acc[8] * inv, acc[9] * inv);
+                    v1.y = pack_bf16(acc[10] * inv, acc[11] * inv);
+                    v1.z = pack_bf16(acc[12] * inv, acc[13] * inv);
+                    v1.w = pack_bf16(acc[14] * inv, acc[15] * inv);
+                    *reinterpret_cast<uint4*>(dst) = v0;
+                    *reinterpret_cast<uint4*>(dst + 8) = v1;
+                }
+            }
+            if (x == 0 && live) P.lse[static_cast<int64_t>(I.h) * T + t] = M * 0.6931471805599453f + logf(L);
+            tc_fence_before();
+            mbar_arrive(merge_b);
+            pending_b = true;
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        const unsigned long long t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);   // copies still in flight land before the memory is released
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
         tc_fence_after();
         tmem_dealloc(tmem_base, kTmemCols);
     }
@@ -836,8 +1283,8 @@ EncodeFn attn_encode_fn() {
     });
     return fn;
 }
-// bf16 row-major (rows x cols, pitch ld) as tiles of 64 columns x 128 rows, 128-byte swizzle, zero fill outside
-ecospa_status_t encode_tile_map(CUtensorMap* out, const void* ptr, int64_t rows, int64_t cols, int64_t ld) {
+// bf16 row-major (rows x cols, pitch ld) as tiles of 64 columns x box_rows rows, 128-byte swizzle, zero fill outside
+ecospa_status_t encode_tile_map(CUtensorMap* out, const void* ptr, int64_t rows, int64_t cols, int64_t ld, int box_rows = kTile) {
     EncodeFn enc = attn_encode_fn();
     if (!enc) {
         set_cuda_error(cudaErrorNotSupported, "cuTensorMapEncodeTiled entry point");
@@ -845,7 +1292,7 @@ ecospa_status_t encode_tile_map(CUtensorMap* out, const void* ptr, int64_t rows,
     }
     const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
     const cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
-    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(kTile)};
+    const cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
     const cuuint32_t estr[2] = {1, 1};
     if (enc(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
@@ -903,15 +1350,20 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
     int* status = engine_status_ptr(&st);
     if (!status) return st;
     const int64_t T = batch * seq;
+    // output heads up to 32 wide (and Q/K heads up to 64): the stream kernel (K / V tiles as slices of 64 keys); wider
+    // heads: two query tiles per CTA, with one or two 64-column blocks per tile
+    int max_vo = 0;
+    for (int h = 0; h < heads->n_heads; ++h) max_vo = std::max<int>(max_vo, heads->vo_w[h]);
+    const bool streams = max_w <= 64 && max_vo <= 32;
     if ((st = encode_tile_map(&P.map_q, Qc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
-    if ((st = encode_tile_map(&P.map_k, Kc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
-    if ((st = encode_tile_map(&P.map_v, Vc, T, n_vo, ld_v)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_k, Kc, T, n_qk, ld_qk, streams ? 64 : kTile)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_v, Vc, T, n_vo, ld_v, streams ? 64 : kTile)) != ECOSPA_OK) return st;
     P.batch = static_cast<int32_t>(batch);
     P.seq = static_cast<int32_t>(seq);
     P.n_heads = heads->n_heads;
     P.n_qt = static_cast<int32_t>(ceil_div(seq, kTile));
     P.causal = causal != 0;
-    const int64_t items = static_cast<int64_t>((P.n_qt + 1) / 2) * P.n_heads * batch;   // pairs of query tiles
+    const int64_t items = static_cast<int64_t>(streams ? P.n_qt : (P.n_qt + 1) / 2) * P.n_heads * batch;
     if (items > INT32_MAX) return ECOSPA_ERR_UNSUPPORTED;
     P.n_items = static_cast<int32_t>(items);
     P.scale_log2e = scale * 1.4426950408889634f;
@@ -920,8 +1372,6 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
     P.lse = lse;
     P.status = status;
     P.wait_limit_ns = engine_wait_limit_ns();
-    const int nb = max_w > 64 ? 2 : 1;
-    const size_t smem = nb == 1 ? FwdCfg<1>::kSmem : FwdCfg<2>::kSmem;
     static std::once_flag once[64];
     int dev = 0;
     cudaGetDevice(&dev);
@@ -929,6 +1379,7 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
     std::call_once(once[dev & 63], [&] {
         e = cudaFuncSetAttribute(attn_fwd_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<1>::kSmem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdCfg<2>::kSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_fwd_ms_kernel<3, 32>, cudaFuncAttributeMaxDynamicSharedMemorySize, MsCfg<3, 32>::kSmem);
     });
     if (e != cudaSuccess) {
         set_cuda_error(e, "attention setup");
@@ -936,8 +1387,10 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
         return ECOSPA_ERR_CUDA;
     }
     const int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
-    if (nb == 1) attn_fwd_kernel<1><<<grid, kFwdThreads, smem, static_cast<cudaStream_t>(stream)>>>(P);
-    else attn_fwd_kernel<2><<<grid, kFwdThreads, smem, static_cast<cudaStream_t>(stream)>>>(P);
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (streams) attn_fwd_ms_kernel<3, 32><<<grid, MsCfg<3, 32>::kThreads, MsCfg<3, 32>::kSmem, cs>>>(P);
+    else if (max_w <= 64) attn_fwd_kernel<1><<<grid, kFwdThreads, FwdCfg<1>::kSmem, cs>>>(P);
+    else attn_fwd_kernel<2><<<grid, kFwdThreads, FwdCfg<2>::kSmem, cs>>>(P);
     return check_launch("attn_fwd_kernel");
 }
 

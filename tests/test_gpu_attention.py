@@ -122,6 +122,78 @@ def test_forward_llama1b_sized_sampled_heads(causal):
         np.testing.assert_allclose(got_lse[h, rows], ref["lse"][0], rtol=0, atol=2e-3)
 
 
+NARROW = [20, 21, 25, 26, 30, 16, 32]      # output heads at most 32 wide take the kernel with independent key streams
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("seq", [77, 192, 500, 1000])
+def test_forward_narrow_heads_several_items_per_block(seq, causal):
+    """Output heads up to 32 wide, Q/K heads up to 64 wide: sequences that are not multiples of the 192-key tile, more
+    (sequence, head, query tile) items than the GPU has blocks (so every block walks several items and its pipelines
+    cross item boundaries), causal and not."""
+    H = 40
+    k_qk = [RAGGED[i % len(RAGGED)] for i in range(H)]
+    k_vo = [NARROW[i % len(NARROW)] for i in range(H)]
+    run_forward(3, seq, k_qk, k_vo, causal, seed=seq + 1)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_scores_that_grow_along_the_sequence(causal):
+    """Logits that rise by far more than 32 binary orders of magnitude along the keys (and from one 64-key slice to the
+    next), so that the kernel's reference exponent has to move many times, in the middle of a slice too, with the running
+    sums, the output accumulator and the probabilities already written rescaled each time; rows 3 mod 4 fall instead."""
+    batch, seq, H, w = 2, 600, 5, 32
+    k_qk, k_vo = [w] * H, [w] * H
+    d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, k_qk, k_vo, seed=21)
+    T = batch * seq
+    pos = torch.arange(T) % seq
+    ramp = (pos.double() / seq * 40.0 + ((pos % 97) == 0) * 25.0).to(torch.float32)        # steps and isolated spikes
+    for h in range(H):
+        u = torch.zeros(w)
+        u[h % w] = 1.0
+        d["Q"][:, qo[h]: qo[h] + w] = (torch.where((torch.arange(T) % 4 == 3)[:, None], -3.0, 3.0) * u[None, :]).to(torch.bfloat16)
+        d["K"][:, qo[h]: qo[h] + w] = (d["K"][:, qo[h]: qo[h] + w].float() * 0.1 + ramp[:, None] * u[None, :]).to(torch.bfloat16)
+    dd = {k: v.to(DEV) for k, v in d.items()}
+    Ctx = torch.zeros((T, nv + 8), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+    scale = 1.0
+    B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, B.heads(qo, qw, vo, vw), scale, causal, Ctx, lse)
+    B.ecospa_device_status()
+    ref = O.attn_fwd(d["Q"], d["K"], d["V"], batch, seq, qo, k_qk, vo, k_vo, scale, causal)
+    assert np.ptp(ref["lse"]) > 100                      # the case does span far more than 2^32
+    got = Ctx.double().cpu().numpy()
+    assert np.all(np.isfinite(got))
+    for h in range(H):
+        cols = slice(vo[h], vo[h] + w)
+        per_row = np.linalg.norm(got[:, cols] - ref["Ctx"][:, cols], axis=1) / np.linalg.norm(ref["Ctx"][:, cols], axis=1)
+        assert per_row.max() <= 3 * TOL, (h, per_row.argmax(), per_row.max())
+    np.testing.assert_allclose(lse.double().cpu().numpy().reshape(H, T), ref["lse"], rtol=2e-4, atol=2e-3)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_forward_llama1b_step_shape_sampled_heads(causal):
+    """batch 4 x seq 2048, 32 heads of 32 kept columns (the benchmark's attention shape): sampled (sequence, head) pairs."""
+    batch, seq, H = 4, 2048, 32
+    d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, [32] * H, [32] * H, seed=12)
+    T = batch * seq
+    dd = {k: v.to(DEV) for k, v in d.items()}
+    Ctx = torch.zeros((T, nv + 8), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+    scale = 0.125
+    B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, B.heads(qo, qw, vo, vw), scale, causal, Ctx, lse)
+    B.ecospa_device_status()
+    got = Ctx.double().cpu().numpy()
+    got_lse = lse.double().cpu().numpy().reshape(H, T)
+    for b, h in ((0, 0), (3, 31), (1, 13)):
+        rows = slice(b * seq, (b + 1) * seq)
+        q = d["Q"][rows, qo[h]: qo[h] + 32].contiguous()
+        k = d["K"][rows, qo[h]: qo[h] + 32].contiguous()
+        v = d["V"][rows, vo[h]: vo[h] + 32].contiguous()
+        ref = O.attn_fwd(q, k, v, 1, seq, [0], [32], [0], [32], scale, causal)
+        assert rel(got[rows, vo[h]: vo[h] + 32], ref["Ctx"]) <= TOL, (b, h)
+        np.testing.assert_allclose(got_lse[h, rows], ref["lse"][0], rtol=0, atol=2e-3)
+
+
 # ---------------------------------------------------------------------------------------------
 # backward
 # ---------------------------------------------------------------------------------------------
