@@ -924,7 +924,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     using Cfg = BwdCfg<NB, MODE>;
     constexpr int kTileBytes = Cfg::kTileBytes;
     constexpr int RS = Cfg::kResStages, SS = Cfg::kStrStages;
-    constexpr uint32_t kColX = 0, kColY = 128, kColAcc1 = 256, kColAcc2 = 384;
+    // TMEM columns.  Heads up to 64 wide: the accumulators take 64 columns each and the bf16 operands of the
+    // accumulating products (P^T and dS^T, or dS) live in TMEM too, two values per column; wider heads: accumulators of
+    // 128 columns, those operands in shared memory.
+    constexpr bool kOpsInTmem = NB == 1;
+    constexpr uint32_t kColX = 0, kColY = 128, kColAcc1 = 256, kColAcc2 = kOpsInTmem ? 320 : 384, kColP = 384, kColDS = 448;
     constexpr int kCodeBase = MODE == 0 ? 14 : 17;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw_addr = smem_u32(smem_raw);
@@ -1041,19 +1045,21 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 if (!(ok = mbar_wait(r_full(rs), (ri / RS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                 const uint32_t idesc_x = make_idesc(kTile, kTile, 0, 0);
                 // X = Ra Sa^T (contraction over the Q/K width), Y = Rb Sb^T (over the V width) of step gg
+                const uint64_t d_ra = make_smem_desc(sRes + (2 * rs) * kTileBytes, 16, 1024),
+                               d_rb = make_smem_desc(sRes + (2 * rs + 1) * kTileBytes, 16, 1024);
                 auto issue_scores = [&](uint32_t gg) -> bool {
                     const uint32_t st = gg % SS;
                     if (!mbar_wait(t_full(st), (gg / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns)) return false;
                     tc_fence_after();
+                    const uint64_t d_sa = make_smem_desc(sStr + (2 * st) * kTileBytes, 16, 1024),
+                                   d_sb = make_smem_desc(sStr + (2 * st + 1) * kTileBytes, 16, 1024);
                     for (int ks = 0; ks < (wa >> 4); ++ks) {
-                        const uint32_t o = (ks >> 2) * kBlockBytes + (ks & 3) * 32;
-                        tc_mma_bf16(tmem_base + kColX, make_smem_desc(sRes + (2 * rs) * kTileBytes + o, 16, 1024),
-                                    make_smem_desc(sStr + (2 * st) * kTileBytes + o, 16, 1024), idesc_x, ks != 0 ? 1u : 0u);
+                        const uint32_t o = ((ks >> 2) * kBlockBytes + (ks & 3) * 32) >> 4;
+                        tc_mma_bf16(tmem_base + kColX, d_ra + o, d_sa + o, idesc_x, ks != 0 ? 1u : 0u);
                     }
                     for (int ks = 0; ks < (wb >> 4); ++ks) {
-                        const uint32_t o = (ks >> 2) * kBlockBytes + (ks & 3) * 32;
-                        tc_mma_bf16(tmem_base + kColY, make_smem_desc(sRes + (2 * rs + 1) * kTileBytes + o, 16, 1024),
-                                    make_smem_desc(sStr + (2 * st + 1) * kTileBytes + o, 16, 1024), idesc_x, ks != 0 ? 1u : 0u);
+                        const uint32_t o = ((ks >> 2) * kBlockBytes + (ks & 3) * 32) >> 4;
+                        tc_mma_bf16(tmem_base + kColY, d_rb + o, d_sb + o, idesc_x, ks != 0 ? 1u : 0u);
                     }
                     tc_commit(x_full);
                     return true;
@@ -1072,18 +1078,28 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     const uint32_t st = g % SS;
                     if (MODE == 0) {   // dV += P^T dCtx_i : B = streamed b tile, MN-major, N = V width
                         const uint32_t idesc = make_idesc(kTile, wb, 0, 1);
-                        for (int ks = 0; ks < kTile / 16; ++ks)
-                            tc_mma_bf16(tmem_base + kColAcc1, make_smem_desc(sOut + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
-                                        make_smem_desc(sStr + (2 * st + 1) * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc,
-                                        (i | ks) != 0 ? 1u : 0u);
+                        const uint64_t db = make_smem_desc(sStr + (2 * st + 1) * kTileBytes, kBlockBytes, 1024);
+#pragma unroll
+                        for (int ks = 0; ks < kTile / 16; ++ks) {
+                            if (kOpsInTmem)
+                                tc_mma_bf16_ts(tmem_base + kColAcc1, tmem_base + kColP + 8 * ks, db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
+                            else
+                                tc_mma_bf16(tmem_base + kColAcc1, make_smem_desc(sOut + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
+                                            db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
+                        }
                     }
                     {   // dK += dS^T Q_i  (MODE 1: dQ += dS K_j): B = streamed a tile, MN-major, N = Q/K width
                         const uint32_t idesc = make_idesc(kTile, wa, 0, 1);
                         const uint32_t sA = sOut + (MODE == 0 ? 2 * kBlockBytes : 0);
-                        for (int ks = 0; ks < kTile / 16; ++ks)
-                            tc_mma_bf16(tmem_base + kColAcc2, make_smem_desc(sA + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
-                                        make_smem_desc(sStr + (2 * st) * kTileBytes + ks * 2048, kBlockBytes, 1024), idesc,
-                                        (i | ks) != 0 ? 1u : 0u);
+                        const uint64_t db = make_smem_desc(sStr + (2 * st) * kTileBytes, kBlockBytes, 1024);
+#pragma unroll
+                        for (int ks = 0; ks < kTile / 16; ++ks) {
+                            if (kOpsInTmem)
+                                tc_mma_bf16_ts(tmem_base + kColAcc2, tmem_base + kColDS + 8 * ks, db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
+                            else
+                                tc_mma_bf16(tmem_base + kColAcc2, make_smem_desc(sA + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
+                                            db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
+                        }
                     }
                     tc_commit(out_empty);
                     tc_commit(t_empty(st));
@@ -1197,16 +1213,22 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 }
                 // the products that read the previous step's tiles from shared memory are done
                 if (!(ok = mbar_wait(out_empty, (g & 1u) ^ 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+                if (kOpsInTmem) {   // this thread's 32 columns = 16 packed columns of its TMEM lane
+                    if (MODE == 0) tc_st(t_lane + kColP + 16 * part, pk_p);
+                    tc_st(t_lane + kColDS + 16 * part, pk_ds);
+                    tc_wait_st();
+                } else {
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const int chunk = chunk0 + q;
-                    if (MODE == 0)
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + ((chunk ^ swz) << 4)),
-                                     "r"(pk_p[4 * q + 0]), "r"(pk_p[4 * q + 1]), "r"(pk_p[4 * q + 2]), "r"(pk_p[4 * q + 3]) : "memory");
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + (MODE == 0 ? 2 * kBlockBytes : 0) + ((chunk ^ swz) << 4)),
-                                 "r"(pk_ds[4 * q + 0]), "r"(pk_ds[4 * q + 1]), "r"(pk_ds[4 * q + 2]), "r"(pk_ds[4 * q + 3]) : "memory");
+                    for (int q = 0; q < 4; ++q) {
+                        const int chunk = chunk0 + q;
+                        if (MODE == 0)
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + ((chunk ^ swz) << 4)),
+                                         "r"(pk_p[4 * q + 0]), "r"(pk_p[4 * q + 1]), "r"(pk_p[4 * q + 2]), "r"(pk_p[4 * q + 3]) : "memory");
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + (MODE == 0 ? 2 * kBlockBytes : 0) + ((chunk ^ swz) << 4)),
+                                     "r"(pk_ds[4 * q + 0]), "r"(pk_ds[4 * q + 1]), "r"(pk_ds[4 * q + 2]), "r"(pk_ds[4 * q + 3]) : "memory");
+                    }
+                    fence_async_smem();
                 }
-                fence_async_smem();
                 tc_fence_before();
                 mbar_arrive(out_full);
             }
