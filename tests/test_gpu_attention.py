@@ -275,3 +275,50 @@ def test_backward_llama1b_sized_sampled_heads(causal):
         for name, c in (("dQ", cq), ("dK", cq), ("dV", cv)):
             e = rel(g[name][rows, c], ref[name])
             assert e <= TOL, (name, b, h, e)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("seq", [50, 77, 192, 500, 1000])
+def test_backward_narrow_heads_several_items_per_block(seq, causal):
+    """Heads at most 32 wide take the backward kernels that run two blocks per SM on 64-row streamed blocks: sequences
+    that are not multiples of 64 or 128, more (sequence, head, block) items than resident blocks, causal and not."""
+    H = 40 if seq < 1000 else 12
+    k_qk = [NARROW[(i + 1) % len(NARROW)] for i in range(H)]
+    k_vo = [NARROW[i % len(NARROW)] for i in range(H)]
+    run_backward(3, seq, k_qk, k_vo, causal, seed=seq + 2)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_llama1b_step_shape_sampled_heads_and_reruns(causal):
+    """batch 4 x seq 2048, 32 heads of 32 kept columns (the benchmark's attention shape): sampled (sequence, head) pairs
+    against the oracle, and a second run bit-identical to the first."""
+    batch, seq, H = 4, 2048, 32
+    d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, [32] * H, [32] * H, seed=13, with_grad=True)
+    T = batch * seq
+    dd = {k: v.to(DEV) for k, v in d.items()}
+    Ctx = torch.zeros((T, nv + 8), dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+    hd = B.heads(qo, qw, vo, vw)
+    scale = 0.125
+    B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, hd, scale, causal, Ctx, lse)
+    ws = torch.empty(B.ecospa_attn_workspace_bytes(batch, seq, H), dtype=torch.uint8, device=DEV)
+    runs = []
+    for _ in range(2):
+        z = lambda n: torch.zeros((T, n + 8), dtype=torch.bfloat16, device=DEV)
+        dQ, dK, dV = z(nq), z(nq), z(nv)
+        B.ecospa_coupled_attn_bwd(dd["Q"], dd["K"], dd["V"], Ctx, dd["dCtx"], lse, batch, seq, hd, scale, causal, dQ, dK, dV, ws)
+        B.ecospa_device_status()
+        runs.append((dQ, dK, dV))
+    for x, y in zip(*runs):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+    dQ, dK, dV = runs[0]
+    g = {"dQ": dQ.double().cpu().numpy(), "dK": dK.double().cpu().numpy(), "dV": dV.double().cpu().numpy()}
+    for b, h in ((0, 0), (3, 31), (2, 14)):
+        rows = slice(b * seq, (b + 1) * seq)
+        cq, cv = slice(qo[h], qo[h] + 32), slice(vo[h], vo[h] + 32)
+        sub = lambda t, c: t[rows, c].contiguous()
+        ref = O.attn_bwd(sub(d["Q"], cq), sub(d["K"], cq), sub(d["V"], cv), sub(d["dCtx"], cv), 1, seq, [0], [32], [0], [32],
+                         scale, causal)
+        for name, c in (("dQ", cq), ("dK", cq), ("dV", cv)):
+            e = rel(g[name][rows, c], ref[name])
+            assert e <= TOL, (name, b, h, e)
