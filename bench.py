@@ -457,7 +457,7 @@ def attention_report(wl, m, r):
     exp_peak = 148 * 16 * sm * 1e6          # exponentials per second
     return {"ms": r["ms_attn"], "TFLOP/s": fl / r["ms_attn"] / 1e9, "flops": fl, "frac_of_nominal_2250": fl / r["ms_attn"] / 1e9 / 2250.0,
             "causal": m.causal, "head_widths": f"{m.plan['qk'][0]} of {wl.d_h} (padded to {m.qk_w[0]})",
-            "roofline": {"bound": "alu", "kernel": "attn_fwd_kernel + attn_bwd_kernel x2", "achieved": 3 * pairs / (r["ms_attn"] * 1e-3) / 1e12,
+            "roofline": {"bound": "alu", "kernel": ("attn_fwd_ms_kernel" if max(m.vo_w) <= 32 and max(m.qk_w) <= 64 else "attn_fwd_kernel") + " + attn_bwd_kernel x2", "achieved": 3 * pairs / (r["ms_attn"] * 1e-3) / 1e12,
                          "peak": exp_peak / 1e12, "unit": "T exp/s", "frac": 3 * pairs / (r["ms_attn"] * 1e-3) / exp_peak,
                          "peak_source": f"16 ex2/clk/SM x 148 SMs x {sm:.0f} MHz (sampled)"},
             "clocks": r["clocks_attn"]}
