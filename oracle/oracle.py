@@ -398,3 +398,46 @@ def fisher_pair_gqa(g1, g2, layout1: int, layout2: int, n_groups: int, seg_len: 
     other1, _ = _shared_dims(g1, layout1)
     other2, _ = _shared_dims(g2, layout2)
     return 0.5 * (s1 / (other1 * rep1 * seg_len) + s2 / (other2 * rep2 * seg_len)) / n_samples
+
+
+# ---------------------------------------------------------------------------
+# attention core for grouped-query models (Sec. 3.1, "Extension to GQA"): the query heads of a group read the K and V
+# columns of the group's one K/V head.  Written as the definition: every query head is given a copy of its group's K and V
+# columns and the per-head routines above are called; the gradients of the copies of a group are added.
+# ---------------------------------------------------------------------------
+
+def _expand_kv(K, V, rep, qk_off, qk_w, vo_off, vo_w, k_off, v_off, n_q, n_v):
+    import torch
+    T = K.shape[0]
+    Ke = torch.zeros((T, n_q), dtype=K.dtype)
+    Ve = torch.zeros((T, n_v), dtype=V.dtype)
+    for h in range(len(qk_off)):
+        g = h // rep
+        Ke[:, qk_off[h]: qk_off[h] + qk_w[h]] = K[:, k_off[g]: k_off[g] + qk_w[h]]
+        Ve[:, vo_off[h]: vo_off[h] + vo_w[h]] = V[:, v_off[g]: v_off[g] + vo_w[h]]
+    return Ke, Ve
+
+
+def attn_fwd_gqa(Q, K, V, batch: int, seq: int, qk_off, qk_w, vo_off, vo_w, k_off, v_off, scale: float, causal: bool = False):
+    """Q (T x n_q) and the returned Ctx hold one block per query head (qk_off / vo_off), K and V one block per K/V head
+    (k_off / v_off; head h reads group h // rep, rep = query heads per K/V head, and has the widths qk_w[h], vo_w[h])."""
+    rep = len(qk_off) // len(k_off)
+    n_v = max(o + w for o, w in zip(vo_off, vo_w))
+    Ke, Ve = _expand_kv(K, V, rep, qk_off, qk_w, vo_off, vo_w, k_off, v_off, Q.shape[1], n_v)
+    return attn_fwd(Q, Ke, Ve, batch, seq, qk_off, qk_w, vo_off, vo_w, scale, causal)
+
+
+def attn_bwd_gqa(Q, K, V, dCtx, batch: int, seq: int, qk_off, qk_w, vo_off, vo_w, k_off, v_off, scale: float, causal: bool = False):
+    """dQ in Q's layout; dK, dV in the layout of K and V: the sum over the query heads of each group."""
+    rep = len(qk_off) // len(k_off)
+    n_v = max(o + w for o, w in zip(vo_off, vo_w))
+    Ke, Ve = _expand_kv(K, V, rep, qk_off, qk_w, vo_off, vo_w, k_off, v_off, Q.shape[1], n_v)
+    dC = dCtx[:, :n_v].contiguous() if dCtx.shape[1] != n_v else dCtx
+    r = attn_bwd(Q, Ke, Ve, dC, batch, seq, qk_off, qk_w, vo_off, vo_w, scale, causal)
+    dK = np.zeros((K.shape[0], K.shape[1]), dtype=np.float64)
+    dV = np.zeros((V.shape[0], V.shape[1]), dtype=np.float64)
+    for h in range(len(qk_off)):
+        g = h // rep
+        dK[:, k_off[g]: k_off[g] + qk_w[h]] += r["dK"][:, qk_off[h]: qk_off[h] + qk_w[h]]
+        dV[:, v_off[g]: v_off[g] + vo_w[h]] += r["dV"][:, vo_off[h]: vo_off[h] + vo_w[h]]
+    return {"dQ": r["dQ"], "dK": dK, "dV": dV}
