@@ -447,11 +447,20 @@ ecospa_status_t ecospa_coupled_ffn_bwd(const void* X, int64_t ldx, int64_t T, in
  * that owns the query block).  A device-side wait that expires records codes 11-13 (forward), 14-19 (backward).
  */
 typedef struct {
-    int32_t n_heads;
-    const int32_t* qk_off; /* HOST [n_heads] first column of head h in Qc / Kc */
+    int32_t n_heads;       /* query heads */
+    const int32_t* qk_off; /* HOST [n_heads] first column of head h in Qc (and in Kc, unless K/V heads are shared) */
     const int32_t* qk_w;   /* HOST [n_heads] its (padded) width */
-    const int32_t* vo_off; /* HOST [n_heads] first column of head h in Vc / Ctx */
+    const int32_t* vo_off; /* HOST [n_heads] first column of head h in Ctx / dCtx (and in Vc, unless K/V heads are shared) */
     const int32_t* vo_w;   /* HOST [n_heads] its (padded) width */
+    /* Grouped-query models (Sec. 3.1, "Extension to GQA"): n_kv_heads > 0 says that n_heads / n_kv_heads consecutive
+     * query heads read the K and V columns of one K/V head, head h those of head g = h / (n_heads / n_kv_heads).  Kc,
+     * dKc then hold one block per K/V head at k_off[g] (width qk_w of its query heads, which share the group's kept
+     * indices and hence its widths: anything else is ECOSPA_ERR_INVALID), Vc, dVc one at v_off[g] (width vo_w); dKc and
+     * dVc receive the sum over the group's query heads.  Pitches stay as documented (Kc shares ld_qk with Qc).
+     * n_kv_heads == 0 (a zeroed tail of the struct): every query head has its own K/V head, k_off / v_off are not read. */
+    int32_t n_kv_heads;
+    const int32_t* k_off;  /* HOST [n_kv_heads] */
+    const int32_t* v_off;  /* HOST [n_kv_heads] */
 } ecospa_heads_t;
 
 size_t ecospa_attn_workspace_bytes(int64_t batch, int64_t seq, int32_t n_heads);

@@ -498,15 +498,23 @@ def ecospa_coupled_ffn_bwd(X, act: int, w1_c, w2_c, k: int, H, A, dY, dX, dW1_c,
 
 class Heads(C.Structure):
     _fields_ = [("n_heads", C.c_int32), ("qk_off", C.c_void_p), ("qk_w", C.c_void_p), ("vo_off", C.c_void_p),
-                ("vo_w", C.c_void_p)]
+                ("vo_w", C.c_void_p), ("n_kv_heads", C.c_int32), ("k_off", C.c_void_p), ("v_off", C.c_void_p)]
 
 
-def heads(qk_off: Sequence[int], qk_w: Sequence[int], vo_off: Sequence[int], vo_w: Sequence[int]) -> Heads:
-    """Descriptor of the per-head column blocks of Qc / Kc (qk_*) and of Vc / Ctx (vo_*)."""
+def heads(qk_off: Sequence[int], qk_w: Sequence[int], vo_off: Sequence[int], vo_w: Sequence[int],
+          k_off: Optional[Sequence[int]] = None, v_off: Optional[Sequence[int]] = None) -> Heads:
+    """Descriptor of the per-head column blocks of Qc / Kc (qk_*) and of Vc / Ctx (vo_*).  Grouped-query models: k_off,
+    v_off = first columns of the K/V heads in Kc and Vc (len(qk_off) // len(k_off) query heads read each of them)."""
     n = len(qk_off)
     assert len(qk_w) == n and len(vo_off) == n and len(vo_w) == n
     arrs = [(C.c_int32 * n)(*[int(x) for x in v]) for v in (qk_off, qk_w, vo_off, vo_w)]
-    h = Heads(n, *[C.addressof(a) for a in arrs])
+    if k_off is None:
+        h = Heads(n, *[C.addressof(a) for a in arrs], 0, None, None)
+    else:
+        assert v_off is not None and len(v_off) == len(k_off)
+        kv = [(C.c_int32 * len(k_off))(*[int(x) for x in v]) for v in (k_off, v_off)]
+        h = Heads(n, *[C.addressof(a) for a in arrs], len(k_off), C.addressof(kv[0]), C.addressof(kv[1]))
+        arrs += kv
     h._keep = arrs
     return h
 

@@ -53,7 +53,9 @@ constexpr int kBwdThreads = 64 + 4 * 128;   // producer warp, MMA warp, four set
 constexpr int kTmemCols = 512;
 
 struct HeadLayout {
-    int32_t qk_off[kMaxHeads], qk_w[kMaxHeads], vo_off[kMaxHeads], vo_w[kMaxHeads];
+    int32_t qk_off[kMaxHeads], qk_w[kMaxHeads], vo_off[kMaxHeads], vo_w[kMaxHeads];   // per query head: Q^c and Ctx columns, widths
+    int32_t k_off[kMaxHeads], v_off[kMaxHeads];   // per query head: first column of its K/V head in K^c and in V^c
+    int32_t rep;                                   // query heads per K/V head (1: every head its own)
 };
 
 struct AttnFwdParams {
@@ -163,7 +165,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             bool ok = true;
             for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++qi) {
                 const Item I = decode_item(it, P.n_qt, P.n_heads, P.batch, n_kt, P.causal);
-                const int qoff = P.heads.qk_off[I.h], voff = P.heads.vo_off[I.h];
+                const int qoff = P.heads.qk_off[I.h], koff = P.heads.k_off[I.h], voff = P.heads.v_off[I.h];
                 const int nbq = (P.heads.qk_w[I.h] + 63) >> 6, nbv = (P.heads.vo_w[I.h] + 63) >> 6;
                 const int row0 = I.b * P.seq;
                 const uint32_t qs = qi % QS;
@@ -179,7 +181,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                     if (!(ok = mbar_wait(k_empty(st), ((g >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
                     mbar_expect_tx(k_full(st), nbq * kBlockBytes);
                     for (int blk = 0; blk < nbq; ++blk)
-                        tma_load_2d(sK + st * kTileBytes + blk * kBlockBytes, &P.map_k, qoff + 64 * blk, row0 + j * kTile, k_full(st));
+                        tma_load_2d(sK + st * kTileBytes + blk * kBlockBytes, &P.map_k, koff + 64 * blk, row0 + j * kTile, k_full(st));
                     if (!(ok = mbar_wait(v_empty(st), ((g >> 1) & 1u) ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns))) break;
                     mbar_expect_tx(v_full(st), nbv * kBlockBytes);
                     for (int blk = 0; blk < nbv; ++blk)
@@ -547,12 +549,13 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
             struct SD {
                 int row;            // first key row of the slice in the K / V tensors
                 int qrow;           // first row of the item's query tile
-                uint32_t cols;      // first Q/K column | first V column << 16
+                uint32_t qcol;      // first column of the head in Q^c
+                uint32_t cols;      // first column of the head's K/V head in K^c | in V^c << 16
                 uint32_t meta;
             };
             // generator of the stream's slice sequence
             int g_it = static_cast<int>(blockIdx.x) - static_cast<int>(gridDim.x), g_J = 0, g_n = 0, g_row = 0, g_qrow = 0;
-            uint32_t g_cols = 0, g_meta = 0, g_qi = ~0u, g_skip = 0;
+            uint32_t g_cols = 0, g_qcol = 0, g_meta = 0, g_qi = ~0u, g_skip = 0;
             auto next = [&]() {
                 SD d;
                 if (g_J >= g_n) {
@@ -562,6 +565,7 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
                         if (g_it >= P.n_items) {   // end mark; it carries the Q buffers still to hand back
                             d.row = 0;
                             d.cols = 0;
+                            d.qcol = 0;
                             d.meta = ((g_qi & 1u) << 3) | (g_skip << 12);
                             g_skip = 0;
                             g_it -= gridDim.x;      // stay at the end: later calls give the mark again, with no count
@@ -579,7 +583,8 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
                         g_J = 0;
                         g_row = I.b * P.seq + 64 * static_cast<int>(x);
                         g_qrow = I.b * P.seq + I.qt * kTile;
-                        g_cols = static_cast<uint32_t>(P.heads.qk_off[I.h]) | (static_cast<uint32_t>(P.heads.vo_off[I.h]) << 16);
+                        g_cols = static_cast<uint32_t>(P.heads.k_off[I.h]) | (static_cast<uint32_t>(P.heads.v_off[I.h]) << 16);
+                        g_qcol = static_cast<uint32_t>(P.heads.qk_off[I.h]);
                         g_meta = 1u | ((g_qi & 1u) << 3) | (((g_qi >> 1) & 1u) << 4) | (static_cast<uint32_t>(P.heads.qk_w[I.h] >> 4) << 5) |
                                  (static_cast<uint32_t>(P.heads.vo_w[I.h] >> 4) << 8);
                         break;
@@ -587,6 +592,7 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
                 }
                 d.row = g_row + g_J * kKeys;
                 d.qrow = g_qrow;
+                d.qcol = g_qcol;
                 d.cols = g_cols;
                 d.meta = g_meta | (g_J == 0 ? 2u | (g_skip << 12) : 0u) | (g_J == g_n - 1 ? 4u : 0u);
                 if (g_J == 0) g_skip = 0;
@@ -600,7 +606,7 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
                     const uint32_t qs = (d.meta >> 3) & 1u, ph = (d.meta >> 4) & 1u;
                     if (!mbar_wait(q_empty(qs), ph ^ 1u, abort_flag, 11, P.status, P.wait_limit_ns)) return false;
                     mbar_expect_tx(q_full(qs), kBlockBytes);
-                    tma_load_2d(sQ + qs * kBlockBytes, &P.map_q, d.cols & 0xffffu, d.qrow, q_full(qs));
+                    tma_load_2d(sQ + qs * kBlockBytes, &P.map_q, d.qcol, d.qrow, q_full(qs));
                 }
                 tma_load_2d(sKx + st * kSliceB, &P.map_k, d.cols & 0xffffu, d.row, bar);
                 return true;
@@ -977,25 +983,28 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     tc_fence_after();
     const uint32_t tmem_base = *tmem_holder;
 
-    // item -> (sequence, head, owned block, number of steps, first streamed block)
+    // item -> (sequence, head, owned block, steps, first streamed block).  MODE 0 owns a key block of a K/V head and
+    // walks the query blocks of every query head that reads it, one head after the other (h = the first of them).
     struct BItem {
-        int b, h, own, n_steps, first;
+        int b, h, own, n_steps, n_per, first;
     };
+    const int grp = MODE == 0 ? P.heads.rep : 1;
     auto decode = [&](int it) {
         BItem I;
-        const int per = P.n_heads * P.batch;
+        const int per = (P.n_heads / grp) * P.batch;
         const int a = it / per;
         I.own = MODE == 0 ? a : P.n_t - 1 - a;                 // causal: the blocks with the most steps first
         const int rem = it % per;
-        I.h = rem / P.batch;
+        I.h = (rem / P.batch) * grp;
         I.b = rem % P.batch;
         if (MODE == 0) {
             I.first = P.causal ? I.own : 0;                    // query blocks at or after the key block
-            I.n_steps = P.n_t - I.first;
+            I.n_per = P.n_t - I.first;
         } else {
             I.first = 0;
-            I.n_steps = P.causal ? I.own + 1 : P.n_t;          // key blocks up to the query block
+            I.n_per = P.causal ? I.own + 1 : P.n_t;            // key blocks up to the query block
         }
+        I.n_steps = I.n_per * grp;
         return I;
     };
     // which tensor maps / head columns the resident and streamed "a" (Q/K side) and "b" (V/dCtx side) tiles use
@@ -1011,25 +1020,31 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             bool ok = true;
             for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
                 const BItem I = decode(it);
-                const int qoff = P.heads.qk_off[I.h], voff = P.heads.vo_off[I.h];
+                // columns of the resident tiles: MODE 0 the K/V head's block of K^c and V^c, MODE 1 the query head's of Q^c and dCtx
+                const int ra_off = MODE == 0 ? P.heads.k_off[I.h] : P.heads.qk_off[I.h];
+                const int rb_off = MODE == 0 ? P.heads.v_off[I.h] : P.heads.vo_off[I.h];
                 const int nba = (P.heads.qk_w[I.h] + 63) >> 6, nbb = (P.heads.vo_w[I.h] + 63) >> 6;
                 const int row0 = I.b * P.seq;
                 const uint32_t rs = ri % RS;
                 if (!(ok = mbar_wait(r_empty(rs), ((ri / RS) & 1u) ^ 1u, abort_flag, kCodeBase, P.status, P.wait_limit_ns))) break;
                 mbar_expect_tx(r_full(rs), (nba + nbb) * kBlockBytes);
                 for (int blk = 0; blk < nba; ++blk)
-                    tma_load_2d(sRes + (2 * rs) * kTileBytes + blk * kBlockBytes, map_ra, qoff + 64 * blk, row0 + I.own * kTile, r_full(rs));
+                    tma_load_2d(sRes + (2 * rs) * kTileBytes + blk * kBlockBytes, map_ra, ra_off + 64 * blk, row0 + I.own * kTile, r_full(rs));
                 for (int blk = 0; blk < nbb; ++blk)
-                    tma_load_2d(sRes + (2 * rs + 1) * kTileBytes + blk * kBlockBytes, map_rb, voff + 64 * blk, row0 + I.own * kTile, r_full(rs));
+                    tma_load_2d(sRes + (2 * rs + 1) * kTileBytes + blk * kBlockBytes, map_rb, rb_off + 64 * blk, row0 + I.own * kTile, r_full(rs));
                 for (int i = 0; i < I.n_steps; ++i, ++g) {
                     const uint32_t st = g % SS;
                     if (!(ok = mbar_wait(t_empty(st), ((g / SS) & 1u) ^ 1u, abort_flag, kCodeBase, P.status, P.wait_limit_ns))) break;
                     mbar_expect_tx(t_full(st), (nba + nbb) * kBlockBytes);
-                    const int y = row0 + (I.first + i) * kTile;
+                    // streamed tiles: MODE 0 the query block of query head h + i / n_per, MODE 1 the key block of the K/V head
+                    const int hq = I.h + i / I.n_per;
+                    const int sa_off = MODE == 0 ? P.heads.qk_off[hq] : P.heads.k_off[I.h];
+                    const int sb_off = MODE == 0 ? P.heads.vo_off[hq] : P.heads.v_off[I.h];
+                    const int y = row0 + (I.first + i % I.n_per) * kTile;
                     for (int blk = 0; blk < nba; ++blk)
-                        tma_load_2d(sStr + (2 * st) * kTileBytes + blk * kBlockBytes, map_sa, qoff + 64 * blk, y, t_full(st));
+                        tma_load_2d(sStr + (2 * st) * kTileBytes + blk * kBlockBytes, map_sa, sa_off + 64 * blk, y, t_full(st));
                     for (int blk = 0; blk < nbb; ++blk)
-                        tma_load_2d(sStr + (2 * st + 1) * kTileBytes + blk * kBlockBytes, map_sb, voff + 64 * blk, y, t_full(st));
+                        tma_load_2d(sStr + (2 * st + 1) * kTileBytes + blk * kBlockBytes, map_sb, sb_off + 64 * blk, y, t_full(st));
                 }
             }
         }
@@ -1131,8 +1146,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
             const BItem I = decode(it);
             const int own_pos = I.own * kTile + row;                 // position of this thread's row in the sequence
-            const float* lse_h = P.lse + static_cast<int64_t>(I.h) * T + static_cast<int64_t>(I.b) * P.seq;
-            const float* d_h = P.dvec + static_cast<int64_t>(I.h) * T + static_cast<int64_t>(I.b) * P.seq;
+            // log-sum-exp and row dots of query head hq of this sequence
+            auto lse_of = [&](int hq) { return P.lse + static_cast<int64_t>(hq) * T + static_cast<int64_t>(I.b) * P.seq; };
+            auto d_of = [&](int hq) { return P.dvec + static_cast<int64_t>(hq) * T + static_cast<int64_t>(I.b) * P.seq; };
+            const float* lse_h = lse_of(I.h);
+            const float* d_h = d_of(I.h);
             // MODE 1: this row's log-sum-exp (base 2) and row dot.  MODE 0 (threads of part 0 only): the values of
             // query `row` of the next query block, fetched one step ahead and staged in shared memory for all rows.
             float lse_r = 0.f, d_r = 0.f;
@@ -1149,7 +1167,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 }
             }
             for (int i = 0; i < I.n_steps; ++i, ++g) {
-                const int other0 = (I.first + i) * kTile;            // first position of the streamed block
+                const int other0 = (I.first + i % I.n_per) * kTile;  // first position of the streamed block
                 float* vb = vec + (g & 1) * 2 * kTile;
                 if (MODE == 0) {
                     if (part == 0) {
@@ -1161,10 +1179,12 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     if (!(ok = mbar_wait(vec_ready, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
                     if (part == 0) {
                         lse_r = d_r = 0.f;
-                        const int qp = other0 + kTile + row;         // prefetch for the next query block
+                        // prefetch for the next step: the next query block of this head, or the first one of the next head
+                        const int hn = I.h + (i + 1) / I.n_per;
+                        const int qp = (I.first + (i + 1) % I.n_per) * kTile + row;
                         if (i + 1 < I.n_steps && qp < P.seq) {
-                            lse_r = lse_h[qp] * kLog2e;
-                            d_r = d_h[qp];
+                            lse_r = lse_of(hn)[qp] * kLog2e;
+                            d_r = d_of(hn)[qp];
                         }
                     }
                 }
@@ -1263,8 +1283,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 }
             };
             if (MODE == 0) {
-                write_acc(kColAcc1, P.heads.vo_w[I.h], P.dv + t * P.ld_dv + P.heads.vo_off[I.h], 1.f);
-                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dk + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale);
+                write_acc(kColAcc1, P.heads.vo_w[I.h], P.dv + t * P.ld_dv + P.heads.v_off[I.h], 1.f);
+                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dk + t * P.ld_dqk + P.heads.k_off[I.h], P.scale);
             } else {
                 write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale);
             }
@@ -1324,21 +1344,32 @@ ecospa_status_t encode_tile_map(CUtensorMap* out, const void* ptr, int64_t rows,
     return ECOSPA_OK;
 }
 
-// Host-only checks shared by the forward and the backward call; fills the layout and the total widths.
-ecospa_status_t check_heads(const ecospa_heads_t* heads, HeadLayout& L, int64_t& n_qk, int64_t& n_vo, int& max_w) {
+// Host-only checks shared by the forward and the backward call; fills the layout and the widths of the tensors: Q^c
+// (n_qk), Ctx (n_vo), K^c (n_k) and V^c (n_v; the last two equal the first two unless K/V heads are shared).
+ecospa_status_t check_heads(const ecospa_heads_t* heads, HeadLayout& L, int64_t& n_qk, int64_t& n_vo, int64_t& n_k, int64_t& n_v,
+                            int& max_w) {
     if (!heads || !heads->qk_off || !heads->qk_w || !heads->vo_off || !heads->vo_w) return ECOSPA_ERR_INVALID;
-    if (heads->n_heads < 1) return ECOSPA_ERR_INVALID;
+    if (heads->n_heads < 1 || heads->n_kv_heads < 0) return ECOSPA_ERR_INVALID;
     if (heads->n_heads > kMaxHeads) return ECOSPA_ERR_UNSUPPORTED;
-    n_qk = n_vo = 0;
+    const int n_kv = heads->n_kv_heads;
+    if (n_kv > 0 && (!heads->k_off || !heads->v_off || heads->n_heads % n_kv != 0)) return ECOSPA_ERR_INVALID;
+    const int rep = n_kv > 0 ? heads->n_heads / n_kv : 1;
+    L.rep = rep;
+    n_qk = n_vo = n_k = n_v = 0;
     max_w = 0;
     for (int h = 0; h < heads->n_heads; ++h) {
         const int32_t qo = heads->qk_off[h], qw = heads->qk_w[h], vo = heads->vo_off[h], vw = heads->vo_w[h];
-        if (qo < 0 || vo < 0 || qw < 1 || vw < 1) return ECOSPA_ERR_INVALID;
+        const int32_t ko = n_kv > 0 ? heads->k_off[h / rep] : qo, vko = n_kv > 0 ? heads->v_off[h / rep] : vo;
+        if (qo < 0 || vo < 0 || ko < 0 || vko < 0 || qw < 1 || vw < 1) return ECOSPA_ERR_INVALID;
         if (qw > 128 || vw > 128) return ECOSPA_ERR_UNSUPPORTED;
-        if ((qw & 15) || (vw & 15) || (qo & 7) || (vo & 7)) return ECOSPA_ERR_ALIGNMENT;
-        L.qk_off[h] = qo; L.qk_w[h] = qw; L.vo_off[h] = vo; L.vo_w[h] = vw;
+        if ((qw & 15) || (vw & 15) || (qo & 7) || (vo & 7) || (ko & 7) || (vko & 7)) return ECOSPA_ERR_ALIGNMENT;
+        // the query heads of a group share the group's kept indices, hence its widths
+        if (h % rep != 0 && (qw != heads->qk_w[h - h % rep] || vw != heads->vo_w[h - h % rep])) return ECOSPA_ERR_INVALID;
+        L.qk_off[h] = qo; L.qk_w[h] = qw; L.vo_off[h] = vo; L.vo_w[h] = vw; L.k_off[h] = ko; L.v_off[h] = vko;
         n_qk = std::max<int64_t>(n_qk, qo + qw);
         n_vo = std::max<int64_t>(n_vo, vo + vw);
+        n_k = std::max<int64_t>(n_k, ko + qw);
+        n_v = std::max<int64_t>(n_v, vko + vw);
         max_w = std::max(max_w, std::max(qw, vw));
     }
     return ECOSPA_OK;
@@ -1359,14 +1390,14 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
                                                    int64_t batch, int64_t seq, const ecospa_heads_t* heads, float scale,
                                                    int32_t causal, void* Ctx, int64_t ld_ctx, float* lse, void* stream) {
     static thread_local AttnFwdParams P;
-    int64_t n_qk = 0, n_vo = 0;
+    int64_t n_qk = 0, n_vo = 0, n_k = 0, n_v = 0;
     int max_w = 0;
-    ecospa_status_t st = check_heads(heads, P.heads, n_qk, n_vo, max_w);
+    ecospa_status_t st = check_heads(heads, P.heads, n_qk, n_vo, n_k, n_v, max_w);
     if (st != ECOSPA_OK) return st;
     if (batch < 1 || seq < 1 || batch * seq > INT32_MAX || !lse) return ECOSPA_ERR_INVALID;
     if (!(scale > 0.f) || !std::isfinite(scale)) return ECOSPA_ERR_INVALID;
-    if ((st = check_mat(Qc, ld_qk, n_qk)) != ECOSPA_OK || (st = check_mat(Kc, ld_qk, n_qk)) != ECOSPA_OK ||
-        (st = check_mat(Vc, ld_v, n_vo)) != ECOSPA_OK || (st = check_mat(Ctx, ld_ctx, n_vo)) != ECOSPA_OK)
+    if ((st = check_mat(Qc, ld_qk, n_qk)) != ECOSPA_OK || (st = check_mat(Kc, ld_qk, n_k)) != ECOSPA_OK ||
+        (st = check_mat(Vc, ld_v, n_v)) != ECOSPA_OK || (st = check_mat(Ctx, ld_ctx, n_vo)) != ECOSPA_OK)
         return st;
     if (reinterpret_cast<uintptr_t>(lse) & 3u) return ECOSPA_ERR_ALIGNMENT;
     int* status = engine_status_ptr(&st);
@@ -1378,8 +1409,8 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
     for (int h = 0; h < heads->n_heads; ++h) max_vo = std::max<int>(max_vo, heads->vo_w[h]);
     const bool streams = max_w <= 64 && max_vo <= 32;
     if ((st = encode_tile_map(&P.map_q, Qc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
-    if ((st = encode_tile_map(&P.map_k, Kc, T, n_qk, ld_qk, streams ? 64 : kTile)) != ECOSPA_OK) return st;
-    if ((st = encode_tile_map(&P.map_v, Vc, T, n_vo, ld_v, streams ? 64 : kTile)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_k, Kc, T, n_k, ld_qk, streams ? 64 : kTile)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_v, Vc, T, n_v, ld_v, streams ? 64 : kTile)) != ECOSPA_OK) return st;
     P.batch = static_cast<int32_t>(batch);
     P.seq = static_cast<int32_t>(seq);
     P.n_heads = heads->n_heads;
@@ -1430,16 +1461,16 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     static thread_local AttnBwdParams P;
     static thread_local DotParams D;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    int64_t n_qk = 0, n_vo = 0;
+    int64_t n_qk = 0, n_vo = 0, n_k = 0, n_v = 0;
     int max_w = 0;
-    ecospa_status_t st = check_heads(heads, P.heads, n_qk, n_vo, max_w);
+    ecospa_status_t st = check_heads(heads, P.heads, n_qk, n_vo, n_k, n_v, max_w);
     if (st != ECOSPA_OK) return st;
     if (batch < 1 || seq < 1 || batch * seq > INT32_MAX || !lse) return ECOSPA_ERR_INVALID;
     if (!(scale > 0.f) || !std::isfinite(scale)) return ECOSPA_ERR_INVALID;
-    if ((st = check_mat(Qc, ld_qk, n_qk)) != ECOSPA_OK || (st = check_mat(Kc, ld_qk, n_qk)) != ECOSPA_OK ||
-        (st = check_mat(Vc, ld_v, n_vo)) != ECOSPA_OK || (st = check_mat(Ctx, ld_ctx, n_vo)) != ECOSPA_OK ||
+    if ((st = check_mat(Qc, ld_qk, n_qk)) != ECOSPA_OK || (st = check_mat(Kc, ld_qk, n_k)) != ECOSPA_OK ||
+        (st = check_mat(Vc, ld_v, n_v)) != ECOSPA_OK || (st = check_mat(Ctx, ld_ctx, n_vo)) != ECOSPA_OK ||
         (st = check_mat(dCtx, ld_dctx, n_vo)) != ECOSPA_OK || (st = check_mat(dQc, ld_dqk, n_qk)) != ECOSPA_OK ||
-        (st = check_mat(dKc, ld_dqk, n_qk)) != ECOSPA_OK || (st = check_mat(dVc, ld_dv, n_vo)) != ECOSPA_OK)
+        (st = check_mat(dKc, ld_dqk, n_k)) != ECOSPA_OK || (st = check_mat(dVc, ld_dv, n_v)) != ECOSPA_OK)
         return st;
     if (reinterpret_cast<uintptr_t>(lse) & 3u) return ECOSPA_ERR_ALIGNMENT;
     if (n_vo / 8 > kDotMaxVecs) return ECOSPA_ERR_UNSUPPORTED;
@@ -1449,8 +1480,8 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     if (!status) return st;
     const int64_t T = batch * seq;
     if ((st = encode_tile_map(&P.map_q, Qc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
-    if ((st = encode_tile_map(&P.map_k, Kc, T, n_qk, ld_qk)) != ECOSPA_OK) return st;
-    if ((st = encode_tile_map(&P.map_v, Vc, T, n_vo, ld_v)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_k, Kc, T, n_k, ld_qk)) != ECOSPA_OK) return st;
+    if ((st = encode_tile_map(&P.map_v, Vc, T, n_v, ld_v)) != ECOSPA_OK) return st;
     if ((st = encode_tile_map(&P.map_do, dCtx, T, n_vo, ld_dctx)) != ECOSPA_OK) return st;
     float* dvec = static_cast<float*>(workspace);
     P.batch = static_cast<int32_t>(batch);
@@ -1499,11 +1530,16 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     D.n_vecs = static_cast<int32_t>(n_vo / 8);
     attn_rowdot_kernel<<<static_cast<unsigned>(ceil_div(T, kDotWarps)), 32 * kDotWarps, 0, stream>>>(D);
     if ((st = check_launch("attn_rowdot_kernel")) != ECOSPA_OK) return st;
-    const int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
     const int nb = max_w > 64 ? 2 : 1;
+    // dK, dV: one item per (sequence, K/V head, key block); dQ: one per (sequence, query head, query block)
+    const int items_q = P.n_items;
+    P.n_items = items_q / P.heads.rep;
+    int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
     if (nb == 1) attn_bwd_kernel<1, 0><<<grid, kBwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
     else attn_bwd_kernel<2, 0><<<grid, kBwdThreads, BwdCfg<2, 0>::kSmem, stream>>>(P);
     if ((st = check_launch("attn_bwd_kernel (dK, dV)")) != ECOSPA_OK) return st;
+    P.n_items = items_q;
+    grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
     if (nb == 1) attn_bwd_kernel<1, 1><<<grid, kBwdThreads, BwdCfg<1, 1>::kSmem, stream>>>(P);
     else attn_bwd_kernel<2, 1><<<grid, kBwdThreads, BwdCfg<2, 1>::kSmem, stream>>>(P);
     return check_launch("attn_bwd_kernel (dQ)");

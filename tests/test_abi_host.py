@@ -407,3 +407,53 @@ def test_algorithm1_pass_rejects_bad_arguments_without_launching(lib):
     assert apply_(good, 1, C.addressof(big), None, 1, ws, need, None) == 1
     assert apply_(good, 1, C.addressof(k), None, 1, ws, need - 1, None) != 0
     assert apply_(good, 1, None, None, 1, ws, need, None) == 1
+
+
+def test_attention_calls_reject_bad_arguments_without_launching(lib):
+    fwd = lib.ecospa_coupled_attn_fwd
+    fwd.restype = C.c_int
+    fwd.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int64, C.c_int64, C.c_void_p, C.c_float,
+                    C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+    bwd = lib.ecospa_coupled_attn_bwd
+    bwd.restype = C.c_int
+    bwd.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64,
+                    C.c_void_p, C.c_int64, C.c_int64, C.c_void_p, C.c_float, C.c_int32, C.c_void_p, C.c_void_p, C.c_int64,
+                    C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+    wsb = lib.ecospa_attn_workspace_bytes
+    wsb.restype, wsb.argtypes = C.c_size_t, [C.c_int64, C.c_int64, C.c_int32]
+    assert wsb(2, 128, 4) >= 2 * 128 * 4 * 4 and wsb(0, 128, 4) == 0 and wsb(2, 0, 4) == 0 and wsb(2, 128, 0) == 0
+    Q, K, V, Ctx, lse = 0x10000, 0x20000, 0x30000, 0x40000, 0x50000
+
+    def f(hd, q=Q, k=K, ld_qk=64, v=V, ld_v=64, batch=2, seq=128, scale=0.125, ctx=Ctx, ld_ctx=64, l=lse):
+        return fwd(q, k, ld_qk, v, ld_v, batch, seq, C.addressof(hd) if hd is not None else None, scale, 0, ctx, ld_ctx, l, None)
+
+    good = B.heads([0, 32], [32, 32], [0, 32], [32, 32])
+    # every check below fails before the first CUDA call; the good descriptor itself is used for the pointer / pitch cases
+    assert f(None) == 1
+    assert f(B.heads([0, 32], [32, 24], [0, 32], [32, 32])) == 2          # width not a multiple of 16
+    assert f(B.heads([0, 36], [32, 32], [0, 32], [32, 32])) == 2          # offset not a multiple of 8
+    assert f(B.heads([0, 32], [32, 144], [0, 32], [32, 32])) == 3         # wider than 128
+    assert f(B.heads([0, 32], [32, 0], [0, 32], [32, 32])) == 1
+    assert f(B.heads([0, -8], [32, 32], [0, 32], [32, 32])) == 1
+    assert f(B.heads(list(range(0, 16 * 129, 16)), [16] * 129, list(range(0, 16 * 129, 16)), [16] * 129), ld_qk=4096, ld_v=4096, ld_ctx=4096) == 3
+    assert f(good, batch=0) == 1 and f(good, seq=0) == 1 and f(good, l=None) == 1
+    assert f(good, scale=0.0) == 1 and f(good, scale=float("nan")) == 1 and f(good, scale=-1.0) == 1
+    assert f(good, q=None) == 1 and f(good, ctx=None) == 1
+    assert f(good, ld_qk=60) == 1                                         # pitch smaller than the heads' columns
+    assert f(good, ld_v=68) == 2 and f(good, q=Q + 2) == 2 and f(good, l=lse + 2) == 2
+    # grouped-query descriptors
+    assert f(B.heads([0, 32, 64], [32] * 3, [0, 32, 64], [32] * 3, k_off=[0, 32], v_off=[0, 32]), ld_qk=96, ld_v=96, ld_ctx=96) == 1   # 3 % 2
+    assert f(B.heads([0, 32], [32, 16], [0, 32], [32, 32], k_off=[0], v_off=[0])) == 1     # widths differ inside a group
+    assert f(B.heads([0, 32], [32, 32], [0, 32], [32, 32], k_off=[4], v_off=[0])) == 2
+    h = B.heads([0, 32], [32, 32], [0, 32], [32, 32], k_off=[0], v_off=[0])
+    h.k_off = None
+    assert f(h) == 1
+    h = B.heads([0, 32], [32, 32], [0, 32], [32, 32])
+    h.n_kv_heads = -1
+    assert f(h) == 1
+
+    def g(hd, ws=0x90000, ws_bytes=1 << 20, dq=0x60000, dk=0x70000, dv=0x80000, ld_dqk=64, ld_dv=64, dctx=0xa0000):
+        return bwd(Q, K, 64, V, 64, Ctx, 64, dctx, 64, lse, 2, 128, C.addressof(hd), 0.125, 1, dq, dk, ld_dqk, dv, ld_dv, ws, ws_bytes, None)
+
+    assert g(good, ws=None) == 6 and g(good, ws_bytes=16) == 6 and g(good, ws=0x90004) == 2
+    assert g(good, dq=None) == 1 and g(good, dctx=None) == 1 and g(good, ld_dqk=62) == 1 and g(good, ld_dv=68) == 2

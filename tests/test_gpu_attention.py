@@ -322,3 +322,84 @@ def test_backward_llama1b_step_shape_sampled_heads_and_reruns(causal):
         for name, c in (("dQ", cq), ("dK", cq), ("dV", cv)):
             e = rel(g[name][rows, c], ref[name])
             assert e <= TOL, (name, b, h, e)
+
+
+# ---------------------------------------------------------------------------------------------
+# grouped-query models: several query heads read one K/V head
+# ---------------------------------------------------------------------------------------------
+
+def run_gqa(batch, seq, k_qk_g, k_vo_g, rep, causal, seed=0, d_h=64):
+    """k_qk_g / k_vo_g: kept widths per K/V group (its query heads share them).  Forward and backward against the oracle."""
+    G = len(k_qk_g)
+    k_qk = [k_qk_g[h // rep] for h in range(G * rep)]
+    k_vo = [k_vo_g[h // rep] for h in range(G * rep)]
+    qo, qw, nq = BL.padded_head_layout(k_qk)
+    vo, vw, nvo = BL.padded_head_layout(k_vo)
+    ko, kw, nk = BL.padded_head_layout(k_qk_g)
+    vko, vkw, nv = BL.padded_head_layout(k_vo_g)
+    T = batch * seq
+    g = torch.Generator().manual_seed(seed)
+
+    def fill(n, off, k):
+        t = torch.zeros((T, n + 8), dtype=torch.bfloat16)
+        for h in range(len(k)):
+            t[:, off[h]: off[h] + k[h]] = torch.randn((T, k[h]), generator=g).to(torch.bfloat16)
+        return t
+
+    Q, dC = fill(nq, qo, k_qk), fill(nvo, vo, k_vo)
+    K = torch.zeros((T, nq + 8), dtype=torch.bfloat16)          # K^c shares the pitch of Q^c
+    K[:, :nk + 8] = fill(nk, ko, k_qk_g)
+    V = fill(nv, vko, k_vo_g)
+    dev = lambda t: t.to(DEV)
+    Qd, Kd, Vd, dCd = dev(Q), dev(K), dev(V), dev(dC)
+    Ctx = torch.full((T, nvo + 8), 7.0, dtype=torch.bfloat16, device=DEV)
+    lse = torch.zeros(G * rep * T, dtype=torch.float32, device=DEV)
+    hd = B.heads(qo, qw, vo, vw, k_off=ko, v_off=vko)
+    scale = 1.0 / np.sqrt(d_h)
+    B.ecospa_coupled_attn_fwd(Qd, Kd, Vd, batch, seq, hd, scale, causal, Ctx, lse)
+    dQ = torch.full((T, nq + 8), 7.0, dtype=torch.bfloat16, device=DEV)
+    dK = torch.full((T, nq + 8), 7.0, dtype=torch.bfloat16, device=DEV)
+    dV = torch.full((T, nv + 8), 7.0, dtype=torch.bfloat16, device=DEV)
+    ws = torch.empty(B.ecospa_attn_workspace_bytes(batch, seq, G * rep), dtype=torch.uint8, device=DEV)
+    B.ecospa_coupled_attn_bwd(Qd, Kd, Vd, Ctx, dCd, lse, batch, seq, hd, scale, causal, dQ, dK, dV, ws)
+    B.ecospa_device_status()
+    ref = O.attn_fwd_gqa(Q, K, V, batch, seq, qo, k_qk, vo, k_vo, ko, vko, scale, causal)
+    rb = O.attn_bwd_gqa(Q, K, V, dC, batch, seq, qo, k_qk, vo, k_vo, ko, vko, scale, causal)
+    got = Ctx.double().cpu().numpy()
+    for h in range(G * rep):
+        for b in range(batch):
+            rows = slice(b * seq, (b + 1) * seq)
+            assert rel(got[rows, vo[h]: vo[h] + k_vo[h]], ref["Ctx"][rows, vo[h]: vo[h] + k_vo[h]]) <= TOL, ("Ctx", h, b)
+            assert rel(dQ.double().cpu().numpy()[rows, qo[h]: qo[h] + k_qk[h]], rb["dQ"][rows, qo[h]: qo[h] + k_qk[h]]) <= TOL, ("dQ", h, b)
+    np.testing.assert_allclose(lse.double().cpu().numpy().reshape(G * rep, T), ref["lse"], rtol=0, atol=2e-3)
+    gK, gV = dK.double().cpu().numpy(), dV.double().cpu().numpy()
+    for gi in range(G):
+        for b in range(batch):
+            rows = slice(b * seq, (b + 1) * seq)
+            assert rel(gK[rows, ko[gi]: ko[gi] + k_qk_g[gi]], rb["dK"][rows, ko[gi]: ko[gi] + k_qk_g[gi]]) <= TOL, ("dK", gi, b)
+            assert rel(gV[rows, vko[gi]: vko[gi] + k_vo_g[gi]], rb["dV"][rows, vko[gi]: vko[gi] + k_vo_g[gi]]) <= TOL, ("dV", gi, b)
+    assert torch.all(dK[:, nk:] == 7.0) and torch.all(dV[:, nv:] == 7.0) and torch.all(Ctx[:, nvo:] == 7.0)
+    return dQ, dK, dV
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("rep,seq", [(2, 77), (4, 300), (8, 200)])
+def test_grouped_query_attention_narrow_heads(rep, seq, causal):
+    """4 or 5 K/V heads with ragged kept widths up to 32 (the kernel with key streams in the forward pass)."""
+    run_gqa(2, seq, [20, 32, 26, 16, 30][: 5 if rep < 8 else 4], [25, 16, 32, 21, 30][: 5 if rep < 8 else 4], rep, causal, seed=rep + seq)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_grouped_query_attention_wide_heads(causal):
+    """Widths up to 64 and up to 128: the kernels with one and two 64-column blocks per tile."""
+    run_gqa(2, 200, [64, 37, 48], [30, 64, 50], 4, causal, seed=3)
+    run_gqa(1, 260, [128, 96], [72, 128], 2, causal, seed=4, d_h=128)
+
+
+def test_grouped_query_attention_llama_shape_rerun_bit_identical():
+    """8 K/V heads x 4 query heads of 32 kept columns, 2 x 1024 tokens, causal: more items than CTAs; two runs agree bit
+    for bit (the sums over a group's query heads are taken by one CTA in a fixed order)."""
+    a = run_gqa(2, 1024, [32] * 8, [32] * 8, 4, True, seed=5)
+    b = run_gqa(2, 1024, [32] * 8, [32] * 8, 4, True, seed=5)
+    for x, y in zip(a, b):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
