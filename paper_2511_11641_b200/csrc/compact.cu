@@ -247,33 +247,96 @@ struct InplaceJob {
     int64_t ld;            // elements
     int32_t other, D, n_kept, esize, layout, warp_start, n_warps, pad_;
 };
-constexpr int kMaxInplaceJobs = 128;
+constexpr int kMaxInplaceJobs = 512;      // (28 KB of kernel parameters)
 struct InplaceParams {
     int32_t n_jobs, pad_;
     InplaceJob jobs[kMaxInplaceJobs];
 };
 
+constexpr int kInplaceRows = 4;          // rows a warp compacts with one read of the kept list
+constexpr int kInplaceStageBytes = 2048; // staging space per row and chunk of 256 outputs
+
+// Shared-cols tensor, rows [row0, row0 + n_rows) of one warp.  The kept list is walked in chunks of 256 outputs (8 per
+// lane); the sources of a chunk span kept[first] .. kept[last], which is read into shared memory with wide loads (all of
+// the warp's rows at once, to have enough bytes in flight) and written back compacted with wide stores.  In place this
+// is safe because every output index of a chunk is below every source index of the chunks after it (kept[c] >= c) and
+// the chunk's own sources are all staged before its first store.  A chunk whose sources span more than the staging
+// space (about one kept column in four or fewer) falls back to element-wise moves, read before written in the same way.
 template <typename E>
-__device__ __forceinline__ void inplace_cols_row(const InplaceJob& J, int row, int lane) {
-    constexpr int kPer = 8;                              // columns per lane per batch
-    E* p = static_cast<E*>(J.base) + static_cast<int64_t>(row) * J.ld;
-    const int v = 16 / static_cast<int>(sizeof(E));
-    const int64_t padded = static_cast<int64_t>((J.n_kept + v - 1) / v) * v;
+__device__ __forceinline__ void inplace_cols_rows(const InplaceJob& J, int row0, int n_rows, int lane, uint8_t* stage_raw) {
+    constexpr int V = 16 / static_cast<int>(sizeof(E));          // elements per 16-byte vector
+    constexpr int kWindow = kInplaceStageBytes / static_cast<int>(sizeof(E));
+    constexpr int kPer = 8;
+    const int64_t padded = static_cast<int64_t>((J.n_kept + V - 1) / V) * V;
     const int out_cols = static_cast<int>(padded < J.ld ? padded : J.ld);   // kept columns + zero pad
+    E* base = static_cast<E*>(J.base);
+    const bool aligned = (reinterpret_cast<uintptr_t>(base) & 15u) == 0 && (J.ld * sizeof(E)) % 16 == 0;
     for (int c0 = 0; c0 < out_cols; c0 += 32 * kPer) {
-        E val[kPer];
+        int k[kPer];
+        int lo = INT32_MAX, hi = -1;
 #pragma unroll
         for (int e = 0; e < kPer; ++e) {
-            const int c = c0 + e * 32 + lane;
-            int k = c < J.n_kept ? __ldg(J.kept + c) : -1;
-            k = k < 0 ? -1 : min(k, J.D - 1);
-            val[e] = k >= 0 ? p[k] : E(0);
+            const int c = c0 + lane * kPer + e;
+            int v = c < J.n_kept ? __ldg(J.kept + c) : -1;
+            v = v < 0 ? -1 : min(v, J.D - 1);
+            k[e] = v;
+            if (v >= 0) {
+                lo = min(lo, v);
+                hi = max(hi, v);
+            }
         }
-        __syncwarp();                                    // every source of the batch is read before any of it is written
 #pragma unroll
-        for (int e = 0; e < kPer; ++e) {
-            const int c = c0 + e * 32 + lane;
-            if (c < out_cols) p[c] = val[e];
+        for (int o = 16; o > 0; o >>= 1) {
+            lo = min(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+            hi = max(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+        }
+        const int s0 = hi >= 0 ? (lo / V) * V : 0;               // window start, on a vector boundary of the row
+        const int span = hi >= 0 ? hi + 1 - s0 : 0;
+        const bool staged = span <= kWindow;
+        alignas(16) E val[kInplaceRows][kPer];
+        if (staged) {
+#pragma unroll
+            for (int r = 0; r < kInplaceRows; ++r) {
+                if (r < n_rows) {
+                    const E* p = base + static_cast<int64_t>(row0 + r) * J.ld + s0;
+                    E* st = reinterpret_cast<E*>(stage_raw + r * kInplaceStageBytes);
+                    if (aligned) {
+                        for (int v = lane * V; v < span; v += 32 * V)   // (the pitch is a whole number of vectors)
+                            *reinterpret_cast<uint4*>(st + v) = *reinterpret_cast<const uint4*>(p + v);
+                    } else {
+                        for (int v = lane; v < span; v += 32) st[v] = p[v];
+                    }
+                }
+            }
+            __syncwarp();
+#pragma unroll
+            for (int r = 0; r < kInplaceRows; ++r) {
+                const E* st = reinterpret_cast<const E*>(stage_raw + r * kInplaceStageBytes);
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) val[r][e] = (r < n_rows && k[e] >= 0) ? st[k[e] - s0] : E(0);
+            }
+        } else {
+#pragma unroll
+            for (int r = 0; r < kInplaceRows; ++r) {
+                const E* p = base + static_cast<int64_t>(row0 + (r < n_rows ? r : 0)) * J.ld;
+#pragma unroll
+                for (int e = 0; e < kPer; ++e) val[r][e] = (r < n_rows && k[e] >= 0) ? p[k[e]] : E(0);
+            }
+        }
+        __syncwarp();                                            // every source of the chunk is read before any of it is written
+        const int c = c0 + lane * kPer;
+#pragma unroll
+        for (int r = 0; r < kInplaceRows; ++r) {
+            if (r >= n_rows) continue;
+            E* p = base + static_cast<int64_t>(row0 + r) * J.ld;
+            if (aligned && c + kPer <= out_cols) {
+                *reinterpret_cast<uint4*>(p + c) = *reinterpret_cast<const uint4*>(val[r]);
+                if (sizeof(E) == 4) *reinterpret_cast<uint4*>(p + c + 4) = *reinterpret_cast<const uint4*>(val[r] + 4);
+            } else {
+#pragma unroll
+                for (int e = 0; e < kPer; ++e)
+                    if (c + e < out_cols) p[c + e] = val[r][e];
+            }
         }
         __syncwarp();
     }
@@ -287,44 +350,49 @@ __global__ void __launch_bounds__(128) gather_inplace_kernel(const __grid_consta
     const int w = gw - J.warp_start;
     if (w >= J.n_warps) return;
     if (J.layout == ECOSPA_SHARED_COLS) {
-        if (J.esize == 2) inplace_cols_row<uint16_t>(J, w, lane); else inplace_cols_row<uint32_t>(J, w, lane);
+        __shared__ __align__(16) uint8_t stage_all[4][kInplaceRows * kInplaceStageBytes];
+        const int row0 = w * kInplaceRows, n_rows = min(kInplaceRows, J.other - row0);
+        if (J.esize == 2) inplace_cols_rows<uint16_t>(J, row0, n_rows, lane, stage_all[threadIdx.x >> 5]);
+        else inplace_cols_rows<uint32_t>(J, row0, n_rows, lane, stage_all[threadIdx.x >> 5]);
         return;
     }
-    // shared rows: this warp's stripe = bytes [512 w, 512 w + 512) of every row (2-byte units: every element size divides)
+    // shared rows: this warp's stripe = bytes [128 w, 128 w + 128) of every row (4 bytes per lane; 2-byte units at a ragged
+    // end: every element size divides them).  Rows move in batches of 32, each batch read before it is written; narrow
+    // stripes because the batches of a stripe must follow one another, so the stripes are where the parallelism is.
+    constexpr int kBatch = 32;
     const int64_t row_bytes = static_cast<int64_t>(J.other) * J.esize, pitch = J.ld * J.esize;
-    const int64_t b0 = 512ll * w + 16 * lane;
+    const int64_t b0 = 128ll * w + 4 * lane;
     char* base = static_cast<char*>(J.base);
-    const bool vec = (reinterpret_cast<uintptr_t>(base) & 15u) == 0 && pitch % 16 == 0 && b0 + 16 <= row_bytes;
-    for (int r0 = 0; r0 < J.n_kept; r0 += 8) {
-        uint4 v[8];
+    if (b0 >= row_bytes) return;
+    const bool vec = (reinterpret_cast<uintptr_t>(base) & 3u) == 0 && pitch % 4 == 0 && b0 + 4 <= row_bytes;
+    for (int r0 = 0; r0 < J.n_kept; r0 += kBatch) {
+        uint32_t v[kBatch];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            v[u] = make_uint4(0, 0, 0, 0);
+        for (int u = 0; u < kBatch; ++u) {
+            v[u] = 0;
             if (r0 + u < J.n_kept) {
-                int k = __ldg(J.kept + r0 + u);
-                if (k >= 0 && b0 < row_bytes) {
+                const int k = __ldg(J.kept + r0 + u);
+                if (k >= 0) {
                     const char* src = base + static_cast<int64_t>(min(k, J.D - 1)) * pitch + b0;
                     if (vec) {
-                        v[u] = *reinterpret_cast<const uint4*>(src);
-                    } else {
-                        uint16_t* h = reinterpret_cast<uint16_t*>(&v[u]);
-                        for (int e = 0; e < 8; ++e)
-                            if (b0 + 2 * e < row_bytes) h[e] = *reinterpret_cast<const uint16_t*>(src + 2 * e);
+                        v[u] = *reinterpret_cast<const uint32_t*>(src);
+                    } else {                                     // unaligned tensor or the 2-byte tail of a row: halves
+                        v[u] = *reinterpret_cast<const uint16_t*>(src);
+                        if (b0 + 4 <= row_bytes) v[u] |= static_cast<uint32_t>(*reinterpret_cast<const uint16_t*>(src + 2)) << 16;
                     }
                 }
             }
         }
         __syncwarp();
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            if (r0 + u < J.n_kept && b0 < row_bytes) {
+        for (int u = 0; u < kBatch; ++u) {
+            if (r0 + u < J.n_kept) {
                 char* dst = base + static_cast<int64_t>(r0 + u) * pitch + b0;
                 if (vec) {
-                    *reinterpret_cast<uint4*>(dst) = v[u];
+                    *reinterpret_cast<uint32_t*>(dst) = v[u];
                 } else {
-                    const uint16_t* h = reinterpret_cast<const uint16_t*>(&v[u]);
-                    for (int e = 0; e < 8; ++e)
-                        if (b0 + 2 * e < row_bytes) *reinterpret_cast<uint16_t*>(dst + 2 * e) = h[e];
+                    *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(v[u]);
+                    if (b0 + 4 <= row_bytes) *reinterpret_cast<uint16_t*>(dst + 2) = static_cast<uint16_t>(v[u] >> 16);
                 }
             }
         }
@@ -358,7 +426,8 @@ ecospa_status_t compact_inplace_impl(const ecospa_gather_t* jobs, int32_t n_jobs
             J.base = g.in.ptr; J.kept = g.kept; J.ld = g.in.ld;
             J.other = static_cast<int32_t>(g.in.other_dim); J.D = g.shared_dim; J.n_kept = g.n_kept;
             J.esize = eb; J.layout = g.in.layout; J.warp_start = warps;
-            J.n_warps = g.in.layout == ECOSPA_SHARED_COLS ? J.other : static_cast<int32_t>(ceil_div(static_cast<int64_t>(J.other) * eb, 512));
+            J.n_warps = g.in.layout == ECOSPA_SHARED_COLS ? static_cast<int32_t>(ceil_div(static_cast<int64_t>(J.other), static_cast<int64_t>(kInplaceRows)))
+                                                           : static_cast<int32_t>(ceil_div(static_cast<int64_t>(J.other) * eb, 128));
             warps += J.n_warps;
         }
         if (nj == 0) continue;

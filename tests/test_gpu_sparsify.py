@@ -468,7 +468,7 @@ def test_in_place_compaction_equals_out_of_place():
          "m2": torch.randn(w["w2"].shape, generator=gen)}
     lay = {"w1": 0, "w2": 1, "b1": 0, "m1": 0, "m2": 1}
     r = np.random.default_rng(8)
-    for k_ffn, pads in ((1337, 0), (2044, 0), (1073, 7)):
+    for k_ffn, pads in ((1337, 0), (2044, 0), (1073, 7), (150, 0)):      # 150: sources too far apart to stage a chunk
         kept = np.sort(r.choice(wl.d_ffn, size=k_ffn, replace=False)).astype(np.int32)
         if pads:                                          # "no index" entries that pad two blocks, as for padded heads:
             half = wl.d_ffn // 2                          # every real entry still satisfies kept[c] >= c
@@ -499,3 +499,12 @@ def test_in_place_compaction_equals_out_of_place():
     B.ecospa_compact_tensors_inplace([B.gather(v, v, 1, kd, 900, wl.d_ffn)])
     ref = O.compact(src, 1, kept)
     assert torch.equal(v[:900].cpu().contiguous().view(torch.int16), ref.view(torch.int16))
+    # the same for a shared-cols tensor (element-wise loads and stores of the staged path)
+    src = w["w1"][:37].contiguous()
+    pitch = wl.d_ffn + 3
+    buf = torch.zeros(src.shape[0] * pitch + 1, dtype=src.dtype, device=DEV)
+    v = buf[1:].as_strided(src.shape, (pitch, 1))
+    v.copy_(src)
+    B.ecospa_compact_tensors_inplace([B.gather(v, v, 0, kd, 900, wl.d_ffn)])
+    ref = O.compact(src, 0, kept)
+    assert torch.equal(v[:, :900].cpu().contiguous().view(torch.int16), ref.view(torch.int16))
