@@ -18,7 +18,7 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def make_groups(wl, with_moments=True, rope=0):
+def make_groups(wl, with_moments=True, rope=0, galore_rank=0):
     w = WL.layer_weights(wl, 0)
     g = WL.layer_grads(wl, 0)
     gen = torch.Generator().manual_seed(11)
@@ -35,6 +35,16 @@ def make_groups(wl, with_moments=True, rope=0):
     if with_moments:
         qk["aux"] += [(mom(w["wq"]), 0), (mom(w["wk"]), 0)]
         ffn["aux"] += [(mom(w["w1"]), 0), (mom(w["w2"]), 1)]
+    if galore_rank:
+        # Optimizer states kept in a rank-r projected space (the memory-saving optimizer of the paper's LLaMA runs): the
+        # projection acts on the short side of a weight, so the moments keep the shared axis: r x D beside a d_m x D
+        # weight (shared columns), D x r beside a D x d_m weight (shared rows).  First and second moment each.
+        r_ = galore_rank
+        D_attn, D_ffn = h * dh, wl.d_ffn
+        for _ in range(2):
+            qk["aux"] += [(torch.rand((r_, D_attn), generator=gen), 0), (torch.rand((r_, D_attn), generator=gen), 0)]
+            vo["aux"] += [(torch.rand((r_, D_attn), generator=gen), 0), (torch.rand((D_attn, r_), generator=gen), 1)]
+            ffn["aux"] += [(torch.rand((r_, D_ffn), generator=gen), 0), (torch.rand((D_ffn, r_), generator=gen), 1)]
     if wl.bias:
         qk["aux"] += [(w["bq"], 0), (w["bk"], 0)]
         vo["aux"] += [(w["bv"], 0)]
@@ -179,6 +189,25 @@ def test_run_to_budget_matches_the_oracle_loop(name):
                 assert same_bytes(getattr(g, nm), sp[nm], lay, D), nm
         for (tg, lay), (tr, _) in zip(g.aux, sp["aux"]):
             assert same_bytes(tg, tr, lay, D)
+
+
+@pytest.mark.parametrize("in_place", [False, True])
+def test_projected_optimizer_states_follow_the_pass(in_place):
+    """Rank-24 projected first and second moments (r x D and D x r, fp32) ride along as further tensors of their groups:
+    after two passes they hold exactly the kept columns / rows, like the weights."""
+    wl = WL.WORKLOADS["tails768"]
+    specs = make_groups(wl, with_moments=False, galore_rank=24)
+    groups = [to_gpu(sp) for sp in specs]
+    n_samples = float(wl.tokens)
+    for ratio, theta in ((0.5, 0.9), (0.7, 0.85)):
+        groups, info = A1.step(groups, n_samples, ratio, theta, l1=True, k_min=2, in_place=in_place)
+        torch.cuda.synchronize()
+        specs = oracle_pass(specs, info, n_samples, ratio, theta, 2)
+        for g, sp in zip(groups, specs):
+            D = sum(sp["widths"])
+            assert len(g.aux) == len(sp["aux"]) >= 4
+            for (tg, lay), (tr, _) in zip(g.aux, sp["aux"]):
+                assert same_bytes(tg, tr, lay, D)
 
 
 def test_a_pair_that_lost_every_index_takes_no_part():
