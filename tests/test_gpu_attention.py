@@ -403,3 +403,14 @@ def test_grouped_query_attention_llama_shape_rerun_bit_identical():
     b = run_gqa(2, 1024, [32] * 8, [32] * 8, 4, True, seed=5)
     for x, y in zip(a, b):
         assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_long_sequence_and_many_heads(causal):
+    """One sequence of 6000 positions (not a multiple of any tile size; 32 slices per stream in the narrow-head forward
+    kernel, 47 blocks in the others) on two heads, forward and backward, in full; and 128 heads (the most the descriptor
+    takes) on a short one."""
+    run_backward(1, 6000, [32, 20], [32, 26], causal, seed=31)
+    run_forward(1, 6000, [64, 37], [64, 48], causal, seed=32)
+    run_forward(1, 130, [16] * 128, [16] * 128, causal, seed=33)
+    run_backward(1, 130, [16] * 128, [16] * 128, causal, seed=34)
