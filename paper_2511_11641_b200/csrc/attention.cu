@@ -49,7 +49,8 @@ constexpr int kTile = 128;                  // query rows and key rows per tile
 constexpr int kBlockBytes = kTile * 128;    // one 64-column block of a 128-row tile
 constexpr int kMaxHeads = 128;
 constexpr int kFwdThreads = 64 + 2 * 128;   // producer warp, MMA warp, two streams of four softmax warps
-constexpr int kBwdThreads = 64 + 4 * 128;   // producer warp, MMA warp, four sets of four compute warps
+constexpr int kBwdComputeWarps = 16;
+constexpr int kBwdThreads = 64 + 4 * 128 + 32;   // producer warp, MMA warp, four sets of four compute warps, a second MMA warp
 constexpr int kTmemCols = 512;
 
 struct HeadLayout {
@@ -919,8 +920,10 @@ template <int NB, int MODE>
 struct BwdCfg {
     static constexpr int kTileBytes = NB * kBlockBytes;
     static constexpr int kResStages = NB == 1 ? 2 : 1;                         // buffers of the resident pair of tiles
-    static constexpr int kStrStages = (NB == 1 || MODE == 1) ? 2 : 1;          // stages of the streamed pair of tiles
-    static constexpr int kOutTiles = MODE == 0 ? 2 : 1;                        // P^T and dS^T, or dS
+    // stages of the streamed pair of tiles.  Three where they fit (a fourth changes nothing): a stage is free again only when the accumulating
+    // products that read it are done, a whole step after the score products, and the next load must be under way by then
+    static constexpr int kStrStages = NB == 1 ? 3 : (MODE == 1 ? 2 : 1);
+    static constexpr int kOutTiles = NB == 1 ? 0 : (MODE == 0 ? 2 : 1);        // P^T and dS^T, or dS (narrow heads: in TMEM)
     static constexpr int kVecBytes = MODE == 0 ? 2 * 2 * kTile * 4 : 0;        // lse and D of a query block, two buffers
     static constexpr int kSmem = 2 * kTileBytes * (kResStages + kStrStages) + kOutTiles * 2 * kBlockBytes + kVecBytes + 1024 + 256;
 };
@@ -934,6 +937,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     // accumulating products (P^T and dS^T, or dS) live in TMEM too, two values per column; wider heads: accumulators of
     // 128 columns, those operands in shared memory.
     constexpr bool kOpsInTmem = NB == 1;
+    // key-block kernel on narrow heads: dV from warp 1, dK from warp 18 (a thread issues one product per ~72 clocks, and 20
+    // of them per step from one thread would take longer than the step's exponentials)
+    constexpr bool kSplit = NB == 1 && MODE == 0;
+    constexpr uint32_t kAccIssuers = kSplit ? 2 : 1;
     constexpr uint32_t kColX = 0, kColY = 128, kColAcc1 = 256, kColAcc2 = kOpsInTmem ? 320 : 384, kColP = 384, kColDS = 448;
     constexpr int kCodeBase = MODE == 0 ? 14 : 17;
     extern __shared__ uint8_t smem_raw[];
@@ -946,30 +953,34 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     float* vec = reinterpret_cast<float*>(vec_raw);                               // [2 buffers][lse2 | D][128]
     uint8_t* tail = vec_raw + Cfg::kVecBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
-    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 16 * 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * 8 + 8);
+    uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 24 * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 24 * 8 + 8);
     const uint32_t bar0 = smem_u32(bars);
     auto r_full = [&](uint32_t s) { return bar0 + 8u * s; };
     auto r_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };
     auto t_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
-    auto t_empty = [&](uint32_t s) { return bar0 + 8u * (6 + s); };
-    const uint32_t x_full = bar0 + 8u * 8, out_full = bar0 + 8u * 9, out_empty = bar0 + 8u * 10, acc_full = bar0 + 8u * 11,
-                   acc_empty = bar0 + 8u * 12, vec_ready = bar0 + 8u * 13;
+    auto t_empty = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
+    const uint32_t x_full = bar0 + 8u * 12, out_full = bar0 + 8u * 13, out_empty = bar0 + 8u * 14, acc_full = bar0 + 8u * 15,
+                   acc_empty = bar0 + 8u * 16, vec_ready = bar0 + 8u * 17, xy_free = bar0 + 8u * 18;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < 2; ++s) {
             mbar_init(r_full(s), 1);
             mbar_init(r_empty(s), 1);
+        }
+        for (uint32_t s = 0; s < 4; ++s) {
             mbar_init(t_full(s), 1);
-            mbar_init(t_empty(s), 1);
+            mbar_init(t_empty(s), kAccIssuers);
         }
         mbar_init(x_full, 1);
-        mbar_init(out_full, kBwdThreads - 64);
-        mbar_init(out_empty, 1);
-        mbar_init(acc_full, 1);
-        mbar_init(acc_empty, kBwdThreads - 64);
-        mbar_init(vec_ready, kBwdThreads - 64);   // every compute thread arrives: no waiter can fall two phases behind
+        // barriers the compute threads arrive on: one arrival per warp (its lanes meet first), not one per thread
+        mbar_init(out_full, kBwdComputeWarps);
+        mbar_init(out_empty, kAccIssuers);
+        mbar_init(acc_full, kAccIssuers);
+        mbar_init(acc_empty, kBwdComputeWarps);
+        mbar_init(vec_ready, kBwdComputeWarps);   // every compute warp arrives: no waiter can fall two phases behind
+        mbar_init(xy_free, kBwdComputeWarps);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.map_q);
@@ -1081,11 +1092,16 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 };
                 if (!(ok = issue_scores(g))) break;
                 for (int i = 0; i < I.n_steps; ++i, ++g) {
+                    // With two stages the next step's score products are issued as soon as every compute thread has the
+                    // scores of this step in registers (it says so half way through its step), so that they are complete
+                    // by the time the threads come back for them.
+                    if (SS > 1 && i + 1 < I.n_steps) {
+                        if (!(ok = mbar_wait(xy_free, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                        tc_fence_after();
+                        if (!(ok = issue_scores(g + 1))) break;
+                    }
                     if (!(ok = mbar_wait(out_full, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                     tc_fence_after();
-                    // with two stages the next step's score products go first, so that the compute warps can start on them
-                    // while the accumulating products of this step run
-                    if (SS > 1 && i + 1 < I.n_steps && !(ok = issue_scores(g + 1))) break;
                     if (i == 0) {   // the accumulators of the previous item have been read out
                         if (!(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                         tc_fence_after();
@@ -1103,7 +1119,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                                             db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
                         }
                     }
-                    {   // dK += dS^T Q_i  (MODE 1: dQ += dS K_j): B = streamed a tile, MN-major, N = Q/K width
+                    if (!kSplit) {   // dK += dS^T Q_i  (MODE 1: dQ += dS K_j): B = streamed a tile, MN-major, N = Q/K width
                         const uint32_t idesc = make_idesc(kTile, wa, 0, 1);
                         const uint32_t sA = sOut + (MODE == 0 ? 2 * kBlockBytes : 0);
                         const uint64_t db = make_smem_desc(sStr + (2 * st) * kTileBytes, kBlockBytes, 1024);
@@ -1125,6 +1141,31 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_commit(acc_full);
                     tc_commit(r_empty(rs));
                 }
+            }
+        }
+    } else if (warp == 2 + kBwdComputeWarps) {
+        // ------------------------------------------------------------------ second MMA issuer (key-block kernel, narrow heads)
+        if (kSplit && lane == 0) {
+            uint32_t g = 0, ri = 0;
+            bool ok = true;
+            for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
+                const BItem I = decode(it);
+                const uint32_t idesc = make_idesc(kTile, P.heads.qk_w[I.h], 0, 1);
+                for (int i = 0; i < I.n_steps; ++i, ++g) {
+                    const uint32_t st = g % SS;
+                    if (!(ok = mbar_wait(t_full(st), (g / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                    if (!(ok = mbar_wait(out_full, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                    if (i == 0 && !(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                    tc_fence_after();
+                    // dK += dS^T Q_i : B = streamed a tile, MN-major, N = Q/K width
+                    const uint64_t db = make_smem_desc(sStr + (2 * st) * kTileBytes, kBlockBytes, 1024);
+#pragma unroll
+                    for (int ks = 0; ks < kTile / 16; ++ks)
+                        tc_mma_bf16_ts(tmem_base + kColAcc2, tmem_base + kColDS + 8 * ks, db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
+                    tc_commit(out_empty);
+                    tc_commit(t_empty(st));
+                }
+                if (ok) tc_commit(acc_full);
             }
         }
     } else {
@@ -1174,7 +1215,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         vb[row] = lse_r;
                         vb[kTile + row] = d_r;
                     }
-                    mbar_arrive(vec_ready);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(vec_ready);
                     // (a bounded wait instead of a block barrier: a thread that gave up is not waited for)
                     if (!(ok = mbar_wait(vec_ready, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
                     if (part == 0) {
@@ -1201,6 +1243,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_ld16(t_lane + kColX + col0 + 16 * hh, rx);
                     tc_ld16(t_lane + kColY + col0 + 16 * hh, ry);
                     tc_wait_ld();
+                    if (hh == 1) {                                    // this thread's last read of the step's score tiles
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(xy_free);
+                    }
                     if (masked) {                                     // pairs outside the mask count as -inf (p = 0)
 #pragma unroll
                         for (int e = 0; e < 16; ++e) {
@@ -1250,7 +1297,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     fence_async_smem();
                 }
                 tc_fence_before();
-                mbar_arrive(out_full);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(out_full);
             }
             if (!ok) break;
             // the accumulators of this item are complete: write them out (every thread its quarter of the columns)
@@ -1289,7 +1337,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale);
             }
             tc_fence_before();
-            mbar_arrive(acc_empty);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty);
         }
     }
 
