@@ -50,7 +50,7 @@ constexpr int kBlockBytes = kTile * 128;    // one 64-column block of a 128-row 
 constexpr int kMaxHeads = 128;
 constexpr int kFwdThreads = 64 + 2 * 128;   // producer warp, MMA warp, two streams of four softmax warps
 constexpr int kBwdComputeWarps = 16;
-constexpr int kBwdThreads = 64 + 4 * 128 + 32;   // producer warp, MMA warp, four sets of four compute warps, a second MMA warp
+constexpr int kBwdThreads = 64 + 4 * 128 + 64;   // producer warp, MMA warp, four sets of four compute warps, two more MMA warps
 constexpr int kTmemCols = 512;
 
 struct HeadLayout {
@@ -937,9 +937,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     // accumulating products (P^T and dS^T, or dS) live in TMEM too, two values per column; wider heads: accumulators of
     // 128 columns, those operands in shared memory.
     constexpr bool kOpsInTmem = NB == 1;
-    // key-block kernel on narrow heads: dV from warp 1, dK from warp 18 (a thread issues one product per ~72 clocks, and 20
-    // of them per step from one thread would take longer than the step's exponentials)
-    constexpr bool kSplit = NB == 1 && MODE == 0;
+    // Narrow heads: three issuing threads (a thread issues one product per ~72 clocks, and the 12-20 of a step from one
+    // thread, with its waits, take longer than the step's exponentials).  Warp 1 issues the score products only; warps
+    // 18 and 19 the accumulating ones: dV and dK in the key-block kernel, the two halves of the contraction of dQ (into
+    // two accumulators that are added at the end) in the query-block kernel.
+    constexpr bool kSplit = NB == 1;
     constexpr uint32_t kAccIssuers = kSplit ? 2 : 1;
     constexpr uint32_t kColX = 0, kColY = 128, kColAcc1 = 256, kColAcc2 = kOpsInTmem ? 320 : 384, kColP = 384, kColDS = 448;
     constexpr int kCodeBase = MODE == 0 ? 14 : 17;
@@ -1090,6 +1092,17 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_commit(x_full);
                     return true;
                 };
+                if (kSplit) {
+                    // score products only: those of step g + 1 as soon as every compute thread has the scores of step g in
+                    // registers (it says so half way through its step), also across the boundary between two items
+                    for (int i = 0; ok && i < I.n_steps; ++i, ++g) {
+                        if (g > 0 && !(ok = mbar_wait(xy_free, (g - 1) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                        tc_fence_after();
+                        ok = issue_scores(g);
+                    }
+                    if (ok) tc_commit(r_empty(rs));
+                    continue;
+                }
                 if (!(ok = issue_scores(g))) break;
                 for (int i = 0; i < I.n_steps; ++i, ++g) {
                     // With two stages the next step's score products are issued as soon as every compute thread has the
@@ -1143,25 +1156,30 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 }
             }
         }
-    } else if (warp == 2 + kBwdComputeWarps) {
-        // ------------------------------------------------------------------ second MMA issuer (key-block kernel, narrow heads)
+    } else if (warp >= 2 + kBwdComputeWarps) {
+        // ------------------------------------------------------------------ issuers of the accumulating products (narrow heads)
         if (kSplit && lane == 0) {
+            const int which = warp - (2 + kBwdComputeWarps);        // 0: dV (key-block kernel) / first half of dQ; 1: dK / second half
             uint32_t g = 0, ri = 0;
             bool ok = true;
             for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
                 const BItem I = decode(it);
-                const uint32_t idesc = make_idesc(kTile, P.heads.qk_w[I.h], 0, 1);
+                const int wn = (MODE == 0 && which == 0) ? P.heads.vo_w[I.h] : P.heads.qk_w[I.h];
+                const uint32_t idesc = make_idesc(kTile, wn, 0, 1);
+                // key-block kernel: dV += P^T dCtx_i (B = streamed b tile) / dK += dS^T Q_i (B = streamed a tile), all 8 steps
+                // of the contraction; query-block kernel: dQ += dS K_j (B = streamed a tile), steps 0-3 / 4-7
+                const uint32_t acc_col = MODE == 0 ? (which == 0 ? kColAcc1 : kColAcc2) : (which == 0 ? kColAcc2 : kColAcc1);
+                const uint32_t a_col = (MODE == 0 && which == 0) ? kColP : kColDS;
+                const int ks0 = MODE == 0 ? 0 : 4 * which, ks1 = MODE == 0 ? kTile / 16 : 4 * which + 4;
                 for (int i = 0; i < I.n_steps; ++i, ++g) {
                     const uint32_t st = g % SS;
                     if (!(ok = mbar_wait(t_full(st), (g / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                     if (!(ok = mbar_wait(out_full, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                     if (i == 0 && !(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                     tc_fence_after();
-                    // dK += dS^T Q_i : B = streamed a tile, MN-major, N = Q/K width
-                    const uint64_t db = make_smem_desc(sStr + (2 * st) * kTileBytes, kBlockBytes, 1024);
-#pragma unroll
-                    for (int ks = 0; ks < kTile / 16; ++ks)
-                        tc_mma_bf16_ts(tmem_base + kColAcc2, tmem_base + kColDS + 8 * ks, db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
+                    const uint64_t db = make_smem_desc(sStr + (2 * st + ((MODE == 0 && which == 0) ? 1 : 0)) * kTileBytes, kBlockBytes, 1024);
+                    for (int ks = ks0; ks < ks1; ++ks)
+                        tc_mma_bf16_ts(tmem_base + acc_col, tmem_base + a_col + 8 * ks, db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
                     tc_commit(out_empty);
                     tc_commit(t_empty(st));
                 }
@@ -1306,7 +1324,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             tc_fence_after();
             const bool live = own_pos < P.seq;
             const int64_t t = static_cast<int64_t>(I.b) * P.seq + own_pos;
-            auto write_acc = [&](uint32_t colbase, int w, uint16_t* dst, float mul) {
+            auto write_acc = [&](uint32_t colbase, int w, uint16_t* dst, float mul, bool two = false, uint32_t colbase2 = 0) {
 #pragma unroll
                 for (int c = 0; c < NB; ++c) {
                     const int col = part * (NB * 16) + c * 16;
@@ -1314,6 +1332,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         uint32_t r[16];
                         tc_ld16(t_lane + colbase + col, r);
                         tc_wait_ld();
+                        if (two) {                               // the contraction was split over two accumulators
+                            uint32_t r2[16];
+                            tc_ld16(t_lane + colbase2 + col, r2);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) + __uint_as_float(r2[e]));
+                        }
                         if (live) {
                             uint4 v0, v1;
                             v0.x = pack_bf16(__uint_as_float(r[0]) * mul, __uint_as_float(r[1]) * mul);
@@ -1334,7 +1359,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 write_acc(kColAcc1, P.heads.vo_w[I.h], P.dv + t * P.ld_dv + P.heads.v_off[I.h], 1.f);
                 write_acc(kColAcc2, P.heads.qk_w[I.h], P.dk + t * P.ld_dqk + P.heads.k_off[I.h], P.scale);
             } else {
-                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale);
+                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale, kSplit, kColAcc1);
             }
             tc_fence_before();
             __syncwarp();
