@@ -858,20 +858,35 @@ struct DotParams {
     HeadLayout heads;
     const uint16_t* ctx;
     const uint16_t* dctx;
-    float* out;                        // [n_heads][T]
+    const float* lse;                  // [n_heads][T], natural logarithm (from the forward call)
+    float* vecs;                       // [2][n_heads][batch][seq_pad]: -lse * log2(e), then the row dots D; zero past seq
     int64_t ld_ctx, ld_dctx, T;
-    int32_t n_heads, n_vecs;
+    int32_t n_heads, n_vecs, batch, seq, seq_pad;
 };
+// One warp per position of the padded sequences: the per-head row dots D_t = sum_c dCtx[t, c] Ctx[t, c] and the
+// log-sum-exp in the form the backward kernels use, in a layout whose 128-position blocks are whole, 512-byte aligned
+// runs (so that a block's vectors can be copied to shared memory in bulk).
 __global__ void __launch_bounds__(32 * kDotWarps) attn_rowdot_kernel(const __grid_constant__ DotParams P) {
     __shared__ float part[kDotWarps][kDotMaxVecs];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t t = static_cast<int64_t>(blockIdx.x) * kDotWarps + warp;
-    if (t >= P.T) return;
+    const int64_t tp = static_cast<int64_t>(blockIdx.x) * kDotWarps + warp;      // position in the padded layout
+    if (tp >= static_cast<int64_t>(P.batch) * P.seq_pad) return;
+    const int b = static_cast<int>(tp / P.seq_pad), pos = static_cast<int>(tp % P.seq_pad);
+    const int64_t per_arr = static_cast<int64_t>(P.n_heads) * P.batch * P.seq_pad;
+    if (pos >= P.seq) {
+        for (int h = lane; h < P.n_heads; h += 32) {
+            const int64_t o = (static_cast<int64_t>(h) * P.batch + b) * P.seq_pad + pos;
+            P.vecs[o] = 0.f;
+            P.vecs[per_arr + o] = 0.f;
+        }
+        return;
+    }
+    const int64_t t = static_cast<int64_t>(b) * P.seq + pos;
     const uint16_t* a = P.ctx + t * P.ld_ctx;
-    const uint16_t* b = P.dctx + t * P.ld_dctx;
+    const uint16_t* bb = P.dctx + t * P.ld_dctx;
     for (int v = lane; v < P.n_vecs; v += 32) {
         const uint4 x = *reinterpret_cast<const uint4*>(a + 8 * v);
-        const uint4 y = *reinterpret_cast<const uint4*>(b + 8 * v);
+        const uint4 y = *reinterpret_cast<const uint4*>(bb + 8 * v);
         float s = bf16_lo(x.x) * bf16_lo(y.x);
         s = fmaf(bf16_hi(x.x), bf16_hi(y.x), s);
         s = fmaf(bf16_lo(x.y), bf16_lo(y.y), s);
@@ -887,7 +902,9 @@ __global__ void __launch_bounds__(32 * kDotWarps) attn_rowdot_kernel(const __gri
         const int v0 = P.heads.vo_off[h] >> 3, nv = P.heads.vo_w[h] >> 3;
         float s = 0.f;
         for (int i = 0; i < nv; ++i) s += part[warp][v0 + i];
-        P.out[static_cast<int64_t>(h) * P.T + t] = s;
+        const int64_t o = (static_cast<int64_t>(h) * P.batch + b) * P.seq_pad + pos;
+        P.vecs[o] = -P.lse[static_cast<int64_t>(h) * P.T + t] * 1.4426950408889634f;
+        P.vecs[per_arr + o] = s;
     }
 }
 
@@ -897,7 +914,8 @@ struct AttnBwdParams {
     int32_t batch, seq, n_heads, n_t, causal, n_items;
     float scale_log2e, scale;
     const float* lse;                  // [n_heads][T], natural logarithm
-    const float* dvec;                 // [n_heads][T] row dots D
+    const float* vecs;                 // [2][n_heads][batch][seq_pad]: -lse * log2(e) and the row dots D (attn_rowdot_kernel)
+    int32_t seq_pad;
     uint16_t* dq;
     uint16_t* dk;
     uint16_t* dv;
@@ -924,7 +942,7 @@ struct BwdCfg {
     // products that read it are done, a whole step after the score products, and the next load must be under way by then
     static constexpr int kStrStages = NB == 1 ? 3 : (MODE == 1 ? 2 : 1);
     static constexpr int kOutTiles = NB == 1 ? 0 : (MODE == 0 ? 2 : 1);        // P^T and dS^T, or dS (narrow heads: in TMEM)
-    static constexpr int kVecBytes = MODE == 0 ? 2 * 2 * kTile * 4 : 0;        // lse and D of a query block, two buffers
+    static constexpr int kVecBytes = MODE == 0 ? kStrStages * 2 * kTile * 4 : 0;   // -lse2 and D of a query block, per streamed stage
     static constexpr int kSmem = 2 * kTileBytes * (kResStages + kStrStages) + kOutTiles * 2 * kBlockBytes + kVecBytes + 1024 + 256;
 };
 
@@ -952,7 +970,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     // resident: [stage][a | b], streamed: [stage][a | b], out tiles, vectors, barriers
     const uint32_t sRes = base, sStr = sRes + 2 * kTileBytes * RS, sOut = sStr + 2 * kTileBytes * SS;
     uint8_t* vec_raw = smem + 2 * kTileBytes * (RS + SS) + Cfg::kOutTiles * 2 * kBlockBytes;
-    float* vec = reinterpret_cast<float*>(vec_raw);                               // [2 buffers][lse2 | D][128]
+    float* vec = reinterpret_cast<float*>(vec_raw);                               // [stage][-lse2 | D][128]
     uint8_t* tail = vec_raw + Cfg::kVecBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
     uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(tail + 24 * 8);
@@ -963,7 +981,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     auto t_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
     auto t_empty = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
     const uint32_t x_full = bar0 + 8u * 12, out_full = bar0 + 8u * 13, out_empty = bar0 + 8u * 14, acc_full = bar0 + 8u * 15,
-                   acc_empty = bar0 + 8u * 16, vec_ready = bar0 + 8u * 17, xy_free = bar0 + 8u * 18;
+                   acc_empty = bar0 + 8u * 16, xy_free = bar0 + 8u * 17;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -981,7 +999,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         mbar_init(out_empty, kAccIssuers);
         mbar_init(acc_full, kAccIssuers);
         mbar_init(acc_empty, kBwdComputeWarps);
-        mbar_init(vec_ready, kBwdComputeWarps);   // every compute warp arrives: no waiter can fall two phases behind
         mbar_init(xy_free, kBwdComputeWarps);
         *abort_flag = 0;
         fence_barrier_init();
@@ -1048,9 +1065,16 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 for (int i = 0; i < I.n_steps; ++i, ++g) {
                     const uint32_t st = g % SS;
                     if (!(ok = mbar_wait(t_empty(st), ((g / SS) & 1u) ^ 1u, abort_flag, kCodeBase, P.status, P.wait_limit_ns))) break;
-                    mbar_expect_tx(t_full(st), (nba + nbb) * kBlockBytes);
+                    mbar_expect_tx(t_full(st), (nba + nbb) * kBlockBytes + (MODE == 0 ? 2 * kTile * 4 : 0));
                     // streamed tiles: MODE 0 the query block of query head h + i / n_per, MODE 1 the key block of the K/V head
                     const int hq = I.h + i / I.n_per;
+                    if (MODE == 0) {   // with the query block's per-query vectors
+                        const int64_t o = (static_cast<int64_t>(hq) * P.batch + I.b) * P.seq_pad + (I.first + i % I.n_per) * kTile;
+                        const int64_t per_arr = static_cast<int64_t>(P.n_heads) * P.batch * P.seq_pad;
+                        const uint32_t dst = smem_u32(vec) + st * 2 * kTile * 4;
+                        bulk_load(dst, P.vecs + o, kTile * 4, t_full(st));
+                        bulk_load(dst + kTile * 4, P.vecs + per_arr + o, kTile * 4, t_full(st));
+                    }
                     const int sa_off = MODE == 0 ? P.heads.qk_off[hq] : P.heads.k_off[I.h];
                     const int sb_off = MODE == 0 ? P.heads.vo_off[hq] : P.heads.v_off[I.h];
                     const int y = row0 + (I.first + i % I.n_per) * kTile;
@@ -1201,55 +1225,24 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         uint32_t g = 0, ri = 0;
         bool ok = true;
         const int64_t T = static_cast<int64_t>(P.batch) * P.seq;
-        constexpr float kLog2e = 1.4426950408889634f;
         for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
             const BItem I = decode(it);
             const int own_pos = I.own * kTile + row;                 // position of this thread's row in the sequence
-            // log-sum-exp and row dots of query head hq of this sequence
-            auto lse_of = [&](int hq) { return P.lse + static_cast<int64_t>(hq) * T + static_cast<int64_t>(I.b) * P.seq; };
-            auto d_of = [&](int hq) { return P.dvec + static_cast<int64_t>(hq) * T + static_cast<int64_t>(I.b) * P.seq; };
-            const float* lse_h = lse_of(I.h);
-            const float* d_h = d_of(I.h);
-            // MODE 1: this row's log-sum-exp (base 2) and row dot.  MODE 0 (threads of part 0 only): the values of
-            // query `row` of the next query block, fetched one step ahead and staged in shared memory for all rows.
+            // MODE 1: this row's -log-sum-exp (base 2) and row dot (zeros past the end of the sequence).  MODE 0: the values of
+            // the step's 128 queries arrive in shared memory with the step's tiles.
             float lse_r = 0.f, d_r = 0.f;
             if (MODE == 1) {
-                if (own_pos < P.seq) {
-                    lse_r = lse_h[own_pos] * kLog2e;
-                    d_r = d_h[own_pos];
-                }
-            } else if (part == 0) {
-                const int qp = I.first * kTile + row;
-                if (qp < P.seq) {
-                    lse_r = lse_h[qp] * kLog2e;
-                    d_r = d_h[qp];
-                }
+                const int64_t o = (static_cast<int64_t>(I.h) * P.batch + I.b) * P.seq_pad + own_pos;
+                lse_r = P.vecs[o];
+                d_r = P.vecs[static_cast<int64_t>(P.n_heads) * P.batch * P.seq_pad + o];
             }
             for (int i = 0; i < I.n_steps; ++i, ++g) {
                 const int other0 = (I.first + i % I.n_per) * kTile;  // first position of the streamed block
-                float* vb = vec + (g & 1) * 2 * kTile;
-                if (MODE == 0) {
-                    if (part == 0) {
-                        vb[row] = lse_r;
-                        vb[kTile + row] = d_r;
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(vec_ready);
-                    // (a bounded wait instead of a block barrier: a thread that gave up is not waited for)
-                    if (!(ok = mbar_wait(vec_ready, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
-                    if (part == 0) {
-                        lse_r = d_r = 0.f;
-                        // prefetch for the next step: the next query block of this head, or the first one of the next head
-                        const int hn = I.h + (i + 1) / I.n_per;
-                        const int qp = (I.first + (i + 1) % I.n_per) * kTile + row;
-                        if (i + 1 < I.n_steps && qp < P.seq) {
-                            lse_r = lse_of(hn)[qp] * kLog2e;
-                            d_r = d_of(hn)[qp];
-                        }
-                    }
-                }
+                const float* vb = vec + (g % SS) * 2 * kTile;
                 if (!(ok = mbar_wait(x_full, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
                 tc_fence_after();
+                // (the step's loads landed long ago; this thread reads the vectors among them, so it looks at their barrier itself)
+                if (MODE == 0 && !(ok = mbar_wait(t_full(g % SS), (g / SS) & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
                 // (query position, key position) of element (row, column c): MODE 0 rows are keys, MODE 1 rows are queries
                 const int q0 = MODE == 0 ? other0 : I.own * kTile, k0 = MODE == 0 ? I.own * kTile : other0;
                 const bool masked = q0 + kTile > P.seq || k0 + kTile > P.seq || (P.causal && q0 < k0 + kTile);
@@ -1287,7 +1280,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         float pe[4], de[4];
 #pragma unroll
                         for (int u = 0; u < 4; ++u) {
-                            pe[u] = ex2(fmaf(__uint_as_float(rx[e + u]), P.scale_log2e, -l2[u]));
+                            pe[u] = ex2(fmaf(__uint_as_float(rx[e + u]), P.scale_log2e, l2[u]));   // l2 = -lse * log2(e)
                             de[u] = pe[u] * (__uint_as_float(ry[e + u]) - dd[u]);
                         }
                         pk_p[8 * hh + (e >> 1)] = pack_bf16(pe[0], pe[1]);
@@ -1523,7 +1516,8 @@ extern "C" ecospa_status_t ecospa_coupled_attn_fwd(const void* Qc, const void* K
 
 extern "C" size_t ecospa_attn_workspace_bytes(int64_t batch, int64_t seq, int32_t n_heads) {
     if (batch < 1 || seq < 1 || n_heads < 1) return 0;
-    return static_cast<size_t>(batch) * seq * n_heads * 4 + 256;      // the row dots D, one fp32 per (head, token)
+    // two fp32 per (head, position of the sequences padded to whole blocks of 128): -lse * log2(e) and the row dots D
+    return static_cast<size_t>(batch) * ceil_div(seq, static_cast<int64_t>(kTile)) * kTile * n_heads * 8 + 256;
 }
 
 extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* Kc, int64_t ld_qk, const void* Vc, int64_t ld_v,
@@ -1557,7 +1551,7 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     if ((st = encode_tile_map(&P.map_k, Kc, T, n_k, ld_qk)) != ECOSPA_OK) return st;
     if ((st = encode_tile_map(&P.map_v, Vc, T, n_v, ld_v)) != ECOSPA_OK) return st;
     if ((st = encode_tile_map(&P.map_do, dCtx, T, n_vo, ld_dctx)) != ECOSPA_OK) return st;
-    float* dvec = static_cast<float*>(workspace);
+    float* vecs = static_cast<float*>(workspace);
     P.batch = static_cast<int32_t>(batch);
     P.seq = static_cast<int32_t>(seq);
     P.n_heads = heads->n_heads;
@@ -1569,7 +1563,8 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     P.scale = scale;
     P.scale_log2e = scale * 1.4426950408889634f;
     P.lse = lse;
-    P.dvec = dvec;
+    P.vecs = vecs;
+    P.seq_pad = static_cast<int32_t>(ceil_div(seq, static_cast<int64_t>(kTile)) * kTile);
     P.dq = static_cast<uint16_t*>(dQc);
     P.dk = static_cast<uint16_t*>(dKc);
     P.dv = static_cast<uint16_t*>(dVc);
@@ -1596,13 +1591,17 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     D.heads = P.heads;
     D.ctx = static_cast<const uint16_t*>(Ctx);
     D.dctx = static_cast<const uint16_t*>(dCtx);
-    D.out = dvec;
+    D.vecs = vecs;
+    D.lse = lse;
+    D.batch = static_cast<int32_t>(batch);
+    D.seq = static_cast<int32_t>(seq);
+    D.seq_pad = P.seq_pad;
     D.ld_ctx = ld_ctx;
     D.ld_dctx = ld_dctx;
     D.T = T;
     D.n_heads = heads->n_heads;
     D.n_vecs = static_cast<int32_t>(n_vo / 8);
-    attn_rowdot_kernel<<<static_cast<unsigned>(ceil_div(T, kDotWarps)), 32 * kDotWarps, 0, stream>>>(D);
+    attn_rowdot_kernel<<<static_cast<unsigned>(ceil_div(batch * D.seq_pad, static_cast<int64_t>(kDotWarps))), 32 * kDotWarps, 0, stream>>>(D);
     if ((st = check_launch("attn_rowdot_kernel")) != ECOSPA_OK) return st;
     const int nb = max_w > 64 ? 2 : 1;
     // dK, dV: one item per (sequence, K/V head, key block); dQ: one per (sequence, query head, query block)
