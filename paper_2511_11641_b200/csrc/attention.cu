@@ -726,10 +726,27 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
                         for (int i = 0; i < CH; ++i)
                             if (kv_base + c * CH + i >= limit) cur[i] = 0xff800000u;
                     }
+                    // The chunk's maximum and its exponentials (with the reference the row has) have no dependence on one
+                    // another, so they can be interleaved; only if some score exceeds the reference by more than 32 (rare) is
+                    // the row rescaled and the chunk exponentiated again.
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
                     for (int i = 0; i < CH; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(cur[i]));
                     const float cm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * P.scale_log2e;
+                    uint32_t pk[CH / 2];
+                    float cs4[4] = {0.f, 0.f, 0.f, 0.f};
+                    auto exponentiate = [&](float neg_m) {
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) cs4[q] = 0.f;
+#pragma unroll
+                        for (int i = 0; i < CH; i += 2) {
+                            const float p0 = ex2(fmaf(__uint_as_float(cur[i]), P.scale_log2e, neg_m));
+                            const float p1 = ex2(fmaf(__uint_as_float(cur[i + 1]), P.scale_log2e, neg_m));
+                            cs4[(i >> 1) & 3] += p0 + p1;
+                            pk[i >> 1] = pack_bf16(p0, p1);
+                        }
+                    };
+                    exponentiate(-rsx.m);
                     if (__any_sync(0xffffffffu, cm - rsx.m > 32.f)) {
                         // the output row is touched: the product of the previous slice must have landed
                         if (j > 0 && !(ok = mbar_wait(pv_done(x, (cs - 1) & 1), ((cs - 1) >> 1) & 1u, abort_flag, 13, P.status, P.wait_limit_ns))) break;
@@ -738,16 +755,10 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
                         rsx = rescale_row(rsx, cm, tO, j > 0 ? wv >> 4 : 0, tP, c);
                         rs4[0] = rsx.rs;
                         rs4[1] = rs4[2] = rs4[3] = 0.f;
+                        exponentiate(-rsx.m);
                     }
-                    const float neg_m = -rsx.m;
-                    uint32_t pk[CH / 2];
 #pragma unroll
-                    for (int i = 0; i < CH; i += 2) {
-                        const float p0 = ex2(fmaf(__uint_as_float(cur[i]), P.scale_log2e, neg_m));
-                        const float p1 = ex2(fmaf(__uint_as_float(cur[i + 1]), P.scale_log2e, neg_m));
-                        rs4[(i >> 1) & 3] += p0 + p1;
-                        pk[i >> 1] = pack_bf16(p0, p1);
-                    }
+                    for (int q = 0; q < 4; ++q) rs4[q] += cs4[q];
                     tc_st(tP + c * (CH / 2), pk);
                 }
                 if (!ok) break;
