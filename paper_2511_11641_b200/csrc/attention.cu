@@ -857,9 +857,9 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
 // Reverse mode of Ctx_h = P V_h, P = softmax(scale * Q_h K_h^T), with P recomputed from the saved log-sum-exp:
 //     dV = P^T dCtx,  dP = dCtx V^T,  dS = P (.) (dP - D),  D_t = sum_c dCtx[t, c] Ctx[t, c],
 //     dQ = scale * dS K,  dK = scale * dS^T Q.
-// Three launches: the row dots D (memory-bound), then one launch that owns key blocks (dK and dV accumulate in TMEM
-// over the query blocks) and one that owns query blocks (dQ accumulates over the key blocks).  Nothing is added
-// across CTAs, so the results do not depend on timing.
+// Three launches: the row dots D with the log-sum-exp in the form the other two use (memory-bound), then one launch that
+// owns key blocks (dK and dV accumulate in TMEM over the query blocks) and one that owns query blocks (dQ accumulates
+// over the key blocks).  Nothing is added across CTAs, so the results do not depend on timing.
 
 // D[h][t] for every head: a warp takes a row, every lane multiplies 16-byte vectors (8 columns, which never straddle a
 // head because offsets and widths are multiples of 8), and the per-vector partial sums are added per head in order.
@@ -935,16 +935,21 @@ struct AttnBwdParams {
     unsigned long long wait_limit_ns;
 };
 
-// MODE 0: a CTA owns a key block of a (sequence, head) and walks the query blocks: K, V resident, Q_i and dCtx_i
-//         streamed; X = S^T = K Q_i^T and Y = dP^T = V dCtx_i^T (thread = key row, columns = queries); P^T and dS^T go to
-//         shared memory; dV += P^T dCtx_i and dK += dS^T Q_i accumulate in TMEM.
+// MODE 0: a CTA owns a key block of a (sequence, K/V head) and walks the query blocks of the query heads that read it:
+//         K, V resident, Q_i and dCtx_i streamed (with the 128 queries' -lse*log2e and D, bulk-copied on the same
+//         barrier); X = S^T = K Q_i^T and Y = dP^T = V dCtx_i^T (thread = key row, columns = queries); P^T and dS^T are
+//         the A operands of dV += P^T dCtx_i and dK += dS^T Q_i, which accumulate in TMEM.
 // MODE 1: a CTA owns a query block and walks the key blocks: Q, dCtx resident, K_j and V_j streamed; X = S = Q K_j^T and
-//         Y = dP = dCtx V_j^T (thread = query row); dS goes to shared memory; dQ += dS K_j accumulates in TMEM.
+//         Y = dP = dCtx V_j^T (thread = query row); dS is the A operand of dQ += dS K_j, which accumulates in TMEM.
 // Streamed tiles serve twice: as K-major B operands of the score products and as MN-major B operands of the
-// accumulating ones (same bytes, other descriptor).  Warp roles as in the forward kernel, with sixteen compute warps
-// (thread = row, quarter of the columns).  The score products of
-// step i+1 are issued before the accumulating products of step i.  Wait codes: 14 / 15 / 16 (MODE 0 producer, issuer,
-// compute) and 17 / 18 / 19 (MODE 1).
+// accumulating ones (same bytes, other descriptor).  Warp 0 loads, warp 1 issues products, warps 2..17 compute (thread =
+// row, quarter of the columns), warps 18 and 19 issue products on narrow heads.
+// Heads up to 64 wide (NB = 1): the A operands go through TMEM as packed bf16; three stages of streamed tiles; the score
+// products of step i+1 are issued as soon as every compute thread has the score tiles of step i in registers; warp 1
+// issues the score products only, warps 18 and 19 the accumulating ones.  Wider heads (NB = 2): A operands through
+// shared memory, one or two stages, everything issued by warp 1, the score products of step i+1 before the accumulating
+// products of step i where there are two stages.
+// Wait codes: 14 / 15 / 16 (MODE 0 loads, products, compute) and 17 / 18 / 19 (MODE 1).
 template <int NB, int MODE>
 struct BwdCfg {
     static constexpr int kTileBytes = NB * kBlockBytes;
