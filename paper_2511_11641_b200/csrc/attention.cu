@@ -942,13 +942,14 @@ struct AttnBwdParams {
 // MODE 1: a CTA owns a query block and walks the key blocks: Q, dCtx resident, K_j and V_j streamed; X = S = Q K_j^T and
 //         Y = dP = dCtx V_j^T (thread = query row); dS is the A operand of dQ += dS K_j, which accumulates in TMEM.
 // Streamed tiles serve twice: as K-major B operands of the score products and as MN-major B operands of the
-// accumulating ones (same bytes, other descriptor).  Warp 0 loads, warp 1 issues products, warps 2..17 compute (thread =
-// row, quarter of the columns), warps 18 and 19 issue products on narrow heads.
-// Heads up to 64 wide (NB = 1): the A operands go through TMEM as packed bf16; three stages of streamed tiles; the score
-// products of step i+1 are issued as soon as every compute thread has the score tiles of step i in registers; warp 1
-// issues the score products only, warps 18 and 19 the accumulating ones.  Wider heads (NB = 2): A operands through
-// shared memory, one or two stages, everything issued by warp 1, the score products of step i+1 before the accumulating
-// products of step i where there are two stages.
+// accumulating ones (same bytes, other descriptor).  Warp 0 loads, warps 2..17 compute (thread = row, quarter of the
+// columns), and three threads issue products (a thread issues one product per ~72 clocks, and the 12-32 of a step from
+// one thread, with its waits, take longer than the step's exponentials): warp 1 the score products, those of step i+1 as
+// soon as every compute thread has the score tiles of step i in registers; warps 18 and 19 the accumulating ones: dV and
+// dK in the key-block kernel, the two halves of the contraction of dQ (into two accumulators that are added at the end)
+// in the query-block kernel.
+// Heads up to 64 wide (NB = 1): the A operands of the accumulating products go through TMEM as packed bf16; three stages
+// of streamed tiles.  Wider heads (NB = 2): those operands through shared memory, one or two stages.
 // Wait codes: 14 / 15 / 16 (MODE 0 loads, products, compute) and 17 / 18 / 19 (MODE 1).
 template <int NB, int MODE>
 struct BwdCfg {
@@ -971,12 +972,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     // accumulating products (P^T and dS^T, or dS) live in TMEM too, two values per column; wider heads: accumulators of
     // 128 columns, those operands in shared memory.
     constexpr bool kOpsInTmem = NB == 1;
-    // Narrow heads: three issuing threads (a thread issues one product per ~72 clocks, and the 12-20 of a step from one
-    // thread, with its waits, take longer than the step's exponentials).  Warp 1 issues the score products only; warps
-    // 18 and 19 the accumulating ones: dV and dK in the key-block kernel, the two halves of the contraction of dQ (into
-    // two accumulators that are added at the end) in the query-block kernel.
-    constexpr bool kSplit = NB == 1;
-    constexpr uint32_t kAccIssuers = kSplit ? 2 : 1;
+    constexpr uint32_t kAccIssuers = 2;
     constexpr uint32_t kColX = 0, kColY = 128, kColAcc1 = 256, kColAcc2 = kOpsInTmem ? 320 : 384, kColP = 384, kColDS = 448;
     constexpr int kCodeBase = MODE == 0 ? 14 : 17;
     extern __shared__ uint8_t smem_raw[];
@@ -1132,73 +1128,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     tc_commit(x_full);
                     return true;
                 };
-                if (kSplit) {
-                    // score products only: those of step g + 1 as soon as every compute thread has the scores of step g in
-                    // registers (it says so half way through its step), also across the boundary between two items
-                    for (int i = 0; ok && i < I.n_steps; ++i, ++g) {
-                        if (g > 0 && !(ok = mbar_wait(xy_free, (g - 1) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                        tc_fence_after();
-                        ok = issue_scores(g);
-                    }
-                    if (ok) tc_commit(r_empty(rs));
-                    continue;
-                }
-                if (!(ok = issue_scores(g))) break;
-                for (int i = 0; i < I.n_steps; ++i, ++g) {
-                    // With two stages the next step's score products are issued as soon as every compute thread has the
-                    // scores of this step in registers (it says so half way through its step), so that they are complete
-                    // by the time the threads come back for them.
-                    if (SS > 1 && i + 1 < I.n_steps) {
-                        if (!(ok = mbar_wait(xy_free, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                        tc_fence_after();
-                        if (!(ok = issue_scores(g + 1))) break;
-                    }
-                    if (!(ok = mbar_wait(out_full, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                // score products only: those of step g + 1 as soon as every compute thread has the scores of step g in
+                // registers (it says so half way through its step), also across the boundary between two items
+                for (int i = 0; ok && i < I.n_steps; ++i, ++g) {
+                    if (g > 0 && !(ok = mbar_wait(xy_free, (g - 1) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                     tc_fence_after();
-                    if (i == 0) {   // the accumulators of the previous item have been read out
-                        if (!(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                        tc_fence_after();
-                    }
-                    const uint32_t st = g % SS;
-                    if (MODE == 0) {   // dV += P^T dCtx_i : B = streamed b tile, MN-major, N = V width
-                        const uint32_t idesc = make_idesc(kTile, wb, 0, 1);
-                        const uint64_t db = make_smem_desc(sStr + (2 * st + 1) * kTileBytes, kBlockBytes, 1024);
-#pragma unroll
-                        for (int ks = 0; ks < kTile / 16; ++ks) {
-                            if (kOpsInTmem)
-                                tc_mma_bf16_ts(tmem_base + kColAcc1, tmem_base + kColP + 8 * ks, db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
-                            else
-                                tc_mma_bf16(tmem_base + kColAcc1, make_smem_desc(sOut + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
-                                            db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
-                        }
-                    }
-                    if (!kSplit) {   // dK += dS^T Q_i  (MODE 1: dQ += dS K_j): B = streamed a tile, MN-major, N = Q/K width
-                        const uint32_t idesc = make_idesc(kTile, wa, 0, 1);
-                        const uint32_t sA = sOut + (MODE == 0 ? 2 * kBlockBytes : 0);
-                        const uint64_t db = make_smem_desc(sStr + (2 * st) * kTileBytes, kBlockBytes, 1024);
-#pragma unroll
-                        for (int ks = 0; ks < kTile / 16; ++ks) {
-                            if (kOpsInTmem)
-                                tc_mma_bf16_ts(tmem_base + kColAcc2, tmem_base + kColDS + 8 * ks, db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
-                            else
-                                tc_mma_bf16(tmem_base + kColAcc2, make_smem_desc(sA + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
-                                            db + 128 * ks, idesc, (i | ks) != 0 ? 1u : 0u);
-                        }
-                    }
-                    tc_commit(out_empty);
-                    tc_commit(t_empty(st));
-                    // with one stage the next step's tiles can only be loaded once these products have released it
-                    if (SS == 1 && i + 1 < I.n_steps && !(ok = issue_scores(g + 1))) break;
+                    ok = issue_scores(g);
                 }
-                if (ok) {
-                    tc_commit(acc_full);
-                    tc_commit(r_empty(rs));
-                }
+                if (ok) tc_commit(r_empty(rs));
             }
         }
     } else if (warp >= 2 + kBwdComputeWarps) {
-        // ------------------------------------------------------------------ issuers of the accumulating products (narrow heads)
-        if (kSplit && lane == 0) {
+        // ------------------------------------------------------------------ issuers of the accumulating products
+        if (lane == 0) {
             const int which = warp - (2 + kBwdComputeWarps);        // 0: dV (key-block kernel) / first half of dQ; 1: dK / second half
             uint32_t g = 0, ri = 0;
             bool ok = true;
@@ -1210,6 +1152,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 // of the contraction; query-block kernel: dQ += dS K_j (B = streamed a tile), steps 0-3 / 4-7
                 const uint32_t acc_col = MODE == 0 ? (which == 0 ? kColAcc1 : kColAcc2) : (which == 0 ? kColAcc2 : kColAcc1);
                 const uint32_t a_col = (MODE == 0 && which == 0) ? kColP : kColDS;
+                const uint32_t sA = sOut + ((MODE == 0 && which == 1) ? 2 * kBlockBytes : 0);   // wide heads: the same operands in shared memory
                 const int ks0 = MODE == 0 ? 0 : 4 * which, ks1 = MODE == 0 ? kTile / 16 : 4 * which + 4;
                 for (int i = 0; i < I.n_steps; ++i, ++g) {
                     const uint32_t st = g % SS;
@@ -1218,8 +1161,13 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     if (i == 0 && !(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                     tc_fence_after();
                     const uint64_t db = make_smem_desc(sStr + (2 * st + ((MODE == 0 && which == 0) ? 1 : 0)) * kTileBytes, kBlockBytes, 1024);
-                    for (int ks = ks0; ks < ks1; ++ks)
-                        tc_mma_bf16_ts(tmem_base + acc_col, tmem_base + a_col + 8 * ks, db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
+                    for (int ks = ks0; ks < ks1; ++ks) {
+                        if (kOpsInTmem)
+                            tc_mma_bf16_ts(tmem_base + acc_col, tmem_base + a_col + 8 * ks, db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
+                        else
+                            tc_mma_bf16(tmem_base + acc_col, make_smem_desc(sA + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
+                                        db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
+                    }
                     tc_commit(out_empty);
                     tc_commit(t_empty(st));
                 }
@@ -1368,7 +1316,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 write_acc(kColAcc1, P.heads.vo_w[I.h], P.dv + t * P.ld_dv + P.heads.v_off[I.h], 1.f);
                 write_acc(kColAcc2, P.heads.qk_w[I.h], P.dk + t * P.ld_dqk + P.heads.k_off[I.h], P.scale);
             } else {
-                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale, kSplit, kColAcc1);
+                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale, true, kColAcc1);
             }
             tc_fence_before();
             __syncwarp();
