@@ -943,36 +943,49 @@ struct AttnBwdParams {
 //         Y = dP = dCtx V_j^T (thread = query row); dS is the A operand of dQ += dS K_j, which accumulates in TMEM.
 // Streamed tiles serve twice: as K-major B operands of the score products and as MN-major B operands of the
 // accumulating ones (same bytes, other descriptor).  Warp 0 loads, warps 2..17 compute (thread = row, quarter of the
-// columns), and three threads issue products (a thread issues one product per ~72 clocks, and the 12-32 of a step from
-// one thread, with its waits, take longer than the step's exponentials): warp 1 the score products, those of step i+1 as
-// soon as every compute thread has the score tiles of step i in registers; warps 18 and 19 the accumulating ones: dV and
-// dK in the key-block kernel, the two halves of the contraction of dQ (into two accumulators that are added at the end)
-// in the query-block kernel.
-// Heads up to 64 wide (NB = 1): the A operands of the accumulating products go through TMEM as packed bf16; three stages
-// of streamed tiles.  Wider heads (NB = 2): those operands through shared memory, one or two stages.
+// columns), and three threads issue products: a thread gets a tcgen05 instruction (product or commit) accepted every
+// 70-130 clocks, so the 25-40 of a step are spread evenly over them, and the score products of a step are issued as soon
+// as every compute thread has the previous score tiles in registers.
+// Heads up to 64 wide (NB = 1): warp 1 issues the score products; warps 18 and 19 the accumulating ones: dV and dK in the
+// key-block kernel, the two halves of the contraction of dQ (into two accumulators that are added at the end) in the
+// query-block kernel; their A operands go through TMEM as packed bf16; three stages of streamed tiles.
+// Wider heads (NB = 2): warp 1 issues X, warp 18 Y, warp 19 the accumulating products, whose A operands go through shared
+// memory; the key-block kernel takes the queries 64 at a time (three stages of half-size tiles, two buffers of score
+// tiles and of operands), the query-block kernel has two stages.
 // Wait codes: 14 / 15 / 16 (MODE 0 loads, products, compute) and 17 / 18 / 19 (MODE 1).
 template <int NB, int MODE>
 struct BwdCfg {
     static constexpr int kTileBytes = NB * kBlockBytes;
+    // rows of a streamed block.  The key-block kernel on wide heads walks the queries in half blocks: its two wide
+    // accumulators fill the tensor memory beside the score tiles, so P^T and dS^T go through shared memory, and only with
+    // half-size streamed tiles and operands is there room for more than one stage
+    static constexpr int kStep = (NB == 2 && MODE == 0) ? 64 : kTile;
+    static constexpr int kStrBlockBytes = kStep * 128;                         // 64 columns of a streamed block
+    static constexpr int kStrTileBytes = NB * kStrBlockBytes;
     static constexpr int kResStages = NB == 1 ? 2 : 1;                         // buffers of the resident pair of tiles
     // stages of the streamed pair of tiles.  Three where they fit (a fourth changes nothing): a stage is free again only when the accumulating
     // products that read it are done, a whole step after the score products, and the next load must be under way by then
-    static constexpr int kStrStages = NB == 1 ? 3 : (MODE == 1 ? 2 : 1);
+    static constexpr int kStrStages = (NB == 1 || MODE == 0) ? 3 : 2;
+    static constexpr int kOutTileBytes = (kStep / 64) * kBlockBytes;            // 128 rows x kStep columns of bf16
     static constexpr int kOutTiles = NB == 1 ? 0 : (MODE == 0 ? 2 : 1);        // P^T and dS^T, or dS (narrow heads: in TMEM)
-    static constexpr int kVecBytes = MODE == 0 ? kStrStages * 2 * kTile * 4 : 0;   // -lse2 and D of a query block, per streamed stage
-    static constexpr int kSmem = 2 * kTileBytes * (kResStages + kStrStages) + kOutTiles * 2 * kBlockBytes + kVecBytes + 1024 + 256;
+    static constexpr int kOutBufs = kStep == 64 ? 2 : 1;                       // half-block steps: room for two sets of them
+    static constexpr int kVecBytes = MODE == 0 ? kStrStages * 2 * kStep * 4 : 0;   // -lse2 and D of a query block, per streamed stage
+    static constexpr int kSmem = 2 * kTileBytes * kResStages + 2 * kStrTileBytes * kStrStages + kOutBufs * kOutTiles * kOutTileBytes +
+                                 kVecBytes + 1024 + 256;
+    static_assert(kSmem <= 232448, "shared memory of a block");
 };
 
 template <int NB, int MODE>
 __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ AttnBwdParams P) {
     using Cfg = BwdCfg<NB, MODE>;
-    constexpr int kTileBytes = Cfg::kTileBytes;
+    constexpr int kTileBytes = Cfg::kTileBytes, kStrTileBytes = Cfg::kStrTileBytes, kStrBlockBytes = Cfg::kStrBlockBytes;
+    constexpr int kStep = Cfg::kStep, kOutTileBytes = Cfg::kOutTileBytes;
     constexpr int RS = Cfg::kResStages, SS = Cfg::kStrStages;
     // TMEM columns.  Heads up to 64 wide: the accumulators take 64 columns each and the bf16 operands of the
     // accumulating products (P^T and dS^T, or dS) live in TMEM too, two values per column; wider heads: accumulators of
     // 128 columns, those operands in shared memory.
     constexpr bool kOpsInTmem = NB == 1;
-    constexpr uint32_t kAccIssuers = 2;
+    constexpr uint32_t kAccIssuers = NB == 1 ? 2 : 1, kScoreIssuers = NB == 1 ? 1 : 2;
     constexpr uint32_t kColX = 0, kColY = 128, kColAcc1 = 256, kColAcc2 = kOpsInTmem ? 320 : 384, kColP = 384, kColDS = 448;
     constexpr int kCodeBase = MODE == 0 ? 14 : 17;
     extern __shared__ uint8_t smem_raw[];
@@ -980,8 +993,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     const uint32_t base = (raw_addr + 1023u) & ~1023u;
     uint8_t* smem = smem_raw + (base - raw_addr);
     // resident: [stage][a | b], streamed: [stage][a | b], out tiles, vectors, barriers
-    const uint32_t sRes = base, sStr = sRes + 2 * kTileBytes * RS, sOut = sStr + 2 * kTileBytes * SS;
-    uint8_t* vec_raw = smem + 2 * kTileBytes * (RS + SS) + Cfg::kOutTiles * 2 * kBlockBytes;
+    const uint32_t sRes = base, sStr = sRes + 2 * kTileBytes * RS, sOut = sStr + 2 * kStrTileBytes * SS;
+    uint8_t* vec_raw = smem + 2 * kTileBytes * RS + 2 * kStrTileBytes * SS + Cfg::kOutBufs * Cfg::kOutTiles * kOutTileBytes;
     float* vec = reinterpret_cast<float*>(vec_raw);                               // [stage][-lse2 | D][128]
     uint8_t* tail = vec_raw + Cfg::kVecBytes;
     uint64_t* bars = reinterpret_cast<uint64_t*>(tail);
@@ -992,26 +1005,33 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     auto r_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };
     auto t_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
     auto t_empty = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
-    const uint32_t x_full = bar0 + 8u * 12, out_full = bar0 + 8u * 13, out_empty = bar0 + 8u * 14, acc_full = bar0 + 8u * 15,
-                   acc_empty = bar0 + 8u * 16, xy_free = bar0 + 8u * 17;
+    const uint32_t acc_full = bar0 + 8u * 15, acc_empty = bar0 + 8u * 16;
+    constexpr uint32_t kOB = Cfg::kOutBufs, kOutSetBytes = Cfg::kOutTiles * kOutTileBytes;
+    auto out_full = [&](uint32_t b) { return bar0 + 8u * (b ? 20 : 13); };
+    auto out_empty = [&](uint32_t b) { return bar0 + 8u * (b ? 21 : 14); };
+    // score tiles: one buffer of 128 columns each, or (half-block steps) two of 64, each with its own pair of barriers
+    constexpr uint32_t kXY = kStep == 64 ? 2 : 1;
+    auto x_full = [&](uint32_t b) { return bar0 + 8u * (b ? 18 : 12); };
+    auto xy_free = [&](uint32_t b) { return bar0 + 8u * (b ? 19 : 17); };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (uint32_t s = 0; s < 2; ++s) {
             mbar_init(r_full(s), 1);
-            mbar_init(r_empty(s), 1);
+            mbar_init(r_empty(s), kScoreIssuers);
         }
         for (uint32_t s = 0; s < 4; ++s) {
             mbar_init(t_full(s), 1);
             mbar_init(t_empty(s), kAccIssuers);
         }
-        mbar_init(x_full, 1);
-        // barriers the compute threads arrive on: one arrival per warp (its lanes meet first), not one per thread
-        mbar_init(out_full, kBwdComputeWarps);
-        mbar_init(out_empty, kAccIssuers);
+        for (uint32_t b = 0; b < 2; ++b) {
+            mbar_init(x_full(b), kScoreIssuers);
+            mbar_init(xy_free(b), kBwdComputeWarps);
+            mbar_init(out_full(b), kBwdComputeWarps);     // barriers the compute threads arrive on: one arrival per warp (its lanes meet first)
+            mbar_init(out_empty(b), kAccIssuers);
+        }
         mbar_init(acc_full, kAccIssuers);
         mbar_init(acc_empty, kBwdComputeWarps);
-        mbar_init(xy_free, kBwdComputeWarps);
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.map_q);
@@ -1040,8 +1060,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         I.h = (rem / P.batch) * grp;
         I.b = rem % P.batch;
         if (MODE == 0) {
-            I.first = P.causal ? I.own : 0;                    // query blocks at or after the key block
-            I.n_per = P.n_t - I.first;
+            I.first = P.causal ? I.own * (kTile / kStep) : 0;  // query blocks (of kStep queries) at or after the key block
+            I.n_per = (P.seq + kStep - 1) / kStep - I.first;
         } else {
             I.first = 0;
             I.n_per = P.causal ? I.own + 1 : P.n_t;            // key blocks up to the query block
@@ -1054,6 +1074,82 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     const CUtensorMap* map_rb = MODE == 0 ? &P.map_v : &P.map_do;
     const CUtensorMap* map_sa = MODE == 0 ? &P.map_q : &P.map_k;
     const CUtensorMap* map_sb = MODE == 0 ? &P.map_do : &P.map_v;
+
+    // The score products X = Ra Sa^T (contraction over the Q/K width) and / or Y = Rb Sb^T (over the V width) of every step:
+    // those of a step as soon as every compute thread has the previous scores of the same buffer in registers (it says so
+    // half way through its step), also across the boundary between two items.
+    auto score_role = [&](bool do_x, bool do_y) {
+        uint32_t g = 0, ri = 0;
+        bool ok = true;
+        for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
+            const BItem I = decode(it);
+            const int wa = P.heads.qk_w[I.h], wb = P.heads.vo_w[I.h];
+            const uint32_t rs = ri % RS;
+            if (!(ok = mbar_wait(r_full(rs), (ri / RS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+            const uint32_t idesc_x = make_idesc(kTile, kStep, 0, 0);
+            const uint64_t d_ra = make_smem_desc(sRes + (2 * rs) * kTileBytes, 16, 1024),
+                           d_rb = make_smem_desc(sRes + (2 * rs + 1) * kTileBytes, 16, 1024);
+            for (int i = 0; ok && i < I.n_steps; ++i, ++g) {
+                const uint32_t use = g / kXY, st = g % SS, xb = g % kXY;
+                if (use > 0 && !(ok = mbar_wait(xy_free(xb), (use - 1) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                if (!(ok = mbar_wait(t_full(st), (g / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                const uint64_t d_sa = make_smem_desc(sStr + (2 * st) * kStrTileBytes, 16, 1024),
+                               d_sb = make_smem_desc(sStr + (2 * st + 1) * kStrTileBytes, 16, 1024);
+                if (do_x) {
+                    for (int ks = 0; ks < (wa >> 4); ++ks) {
+                        const uint32_t o = ((ks >> 2) * kBlockBytes + (ks & 3) * 32) >> 4, os = ((ks >> 2) * kStrBlockBytes + (ks & 3) * 32) >> 4;
+                        tc_mma_bf16(tmem_base + kColX + xb * kStep, d_ra + o, d_sa + os, idesc_x, ks != 0 ? 1u : 0u);
+                    }
+                }
+                if (do_y) {
+                    for (int ks = 0; ks < (wb >> 4); ++ks) {
+                        const uint32_t o = ((ks >> 2) * kBlockBytes + (ks & 3) * 32) >> 4, os = ((ks >> 2) * kStrBlockBytes + (ks & 3) * 32) >> 4;
+                        tc_mma_bf16(tmem_base + kColY + xb * kStep, d_rb + o, d_sb + os, idesc_x, ks != 0 ? 1u : 0u);
+                    }
+                }
+                tc_commit(x_full(xb));
+            }
+            if (ok) tc_commit(r_empty(rs));
+        }
+    };
+    // The accumulating products number w0 .. w1 - 1 of every step.  Key-block kernel: 0 is dV += P^T dCtx_i (B = streamed b
+    // tile), 1 is dK += dS^T Q_i (B = streamed a tile), all steps of the contraction over the step's queries; query-block
+    // kernel: dQ += dS K_j (B = streamed a tile), 0 is steps 0-3 of the contraction, 1 is steps 4-7 (two accumulators).
+    auto acc_role = [&](int w0, int w1) {
+        uint32_t g = 0, ri = 0;
+        bool ok = true;
+        for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
+            const BItem I = decode(it);
+            for (int i = 0; i < I.n_steps; ++i, ++g) {
+                const uint32_t st = g % SS;
+                if (!(ok = mbar_wait(t_full(st), (g / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                const uint32_t ob = g % kOB;
+                if (!(ok = mbar_wait(out_full(ob), (g / kOB) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                if (i == 0 && !(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                tc_fence_after();
+                for (int which = w0; which < w1; ++which) {
+                    const int wn = (MODE == 0 && which == 0) ? P.heads.vo_w[I.h] : P.heads.qk_w[I.h];
+                    const uint32_t idesc = make_idesc(kTile, wn, 0, 1);
+                    const uint32_t acc_col = MODE == 0 ? (which == 0 ? kColAcc1 : kColAcc2) : (which == 0 ? kColAcc2 : kColAcc1);
+                    const uint32_t a_col = (MODE == 0 && which == 0) ? kColP : kColDS;                 // narrow heads: A operand in TMEM
+                    const uint32_t sA = sOut + ob * kOutSetBytes + ((MODE == 0 && which == 1) ? kOutTileBytes : 0);   // wide heads: in shared memory
+                    const int ks0 = MODE == 0 ? 0 : 4 * which, ks1 = MODE == 0 ? kStep / 16 : 4 * which + 4;
+                    const uint64_t db = make_smem_desc(sStr + (2 * st + ((MODE == 0 && which == 0) ? 1 : 0)) * kStrTileBytes, kStrBlockBytes, 1024);
+                    for (int ks = ks0; ks < ks1; ++ks) {
+                        if (kOpsInTmem)
+                            tc_mma_bf16_ts(tmem_base + acc_col, tmem_base + a_col + 8 * ks, db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
+                        else
+                            tc_mma_bf16(tmem_base + acc_col, make_smem_desc(sA + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
+                                        db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
+                    }
+                }
+                tc_commit(out_empty(ob));
+                tc_commit(t_empty(st));
+            }
+            if (ok) tc_commit(acc_full);
+        }
+    };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
@@ -1077,102 +1173,36 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 for (int i = 0; i < I.n_steps; ++i, ++g) {
                     const uint32_t st = g % SS;
                     if (!(ok = mbar_wait(t_empty(st), ((g / SS) & 1u) ^ 1u, abort_flag, kCodeBase, P.status, P.wait_limit_ns))) break;
-                    mbar_expect_tx(t_full(st), (nba + nbb) * kBlockBytes + (MODE == 0 ? 2 * kTile * 4 : 0));
+                    mbar_expect_tx(t_full(st), (nba + nbb) * kStrBlockBytes + (MODE == 0 ? 2 * kStep * 4 : 0));
                     // streamed tiles: MODE 0 the query block of query head h + i / n_per, MODE 1 the key block of the K/V head
                     const int hq = I.h + i / I.n_per;
                     if (MODE == 0) {   // with the query block's per-query vectors
-                        const int64_t o = (static_cast<int64_t>(hq) * P.batch + I.b) * P.seq_pad + (I.first + i % I.n_per) * kTile;
+                        const int64_t o = (static_cast<int64_t>(hq) * P.batch + I.b) * P.seq_pad + (I.first + i % I.n_per) * kStep;
                         const int64_t per_arr = static_cast<int64_t>(P.n_heads) * P.batch * P.seq_pad;
-                        const uint32_t dst = smem_u32(vec) + st * 2 * kTile * 4;
-                        bulk_load(dst, P.vecs + o, kTile * 4, t_full(st));
-                        bulk_load(dst + kTile * 4, P.vecs + per_arr + o, kTile * 4, t_full(st));
+                        const uint32_t dst = smem_u32(vec) + st * 2 * kStep * 4;
+                        bulk_load(dst, P.vecs + o, kStep * 4, t_full(st));
+                        bulk_load(dst + kStep * 4, P.vecs + per_arr + o, kStep * 4, t_full(st));
                     }
                     const int sa_off = MODE == 0 ? P.heads.qk_off[hq] : P.heads.k_off[I.h];
                     const int sb_off = MODE == 0 ? P.heads.vo_off[hq] : P.heads.v_off[I.h];
-                    const int y = row0 + (I.first + i % I.n_per) * kTile;
+                    const int y = row0 + (I.first + i % I.n_per) * kStep;
                     for (int blk = 0; blk < nba; ++blk)
-                        tma_load_2d(sStr + (2 * st) * kTileBytes + blk * kBlockBytes, map_sa, sa_off + 64 * blk, y, t_full(st));
+                        tma_load_2d(sStr + (2 * st) * kStrTileBytes + blk * kStrBlockBytes, map_sa, sa_off + 64 * blk, y, t_full(st));
                     for (int blk = 0; blk < nbb; ++blk)
-                        tma_load_2d(sStr + (2 * st + 1) * kTileBytes + blk * kBlockBytes, map_sb, sb_off + 64 * blk, y, t_full(st));
+                        tma_load_2d(sStr + (2 * st + 1) * kStrTileBytes + blk * kStrBlockBytes, map_sb, sb_off + 64 * blk, y, t_full(st));
                 }
             }
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            uint32_t g = 0, ri = 0;
-            bool ok = true;
-            for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
-                const BItem I = decode(it);
-                const int wa = P.heads.qk_w[I.h], wb = P.heads.vo_w[I.h];
-                const uint32_t rs = ri % RS;
-                if (!(ok = mbar_wait(r_full(rs), (ri / RS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                const uint32_t idesc_x = make_idesc(kTile, kTile, 0, 0);
-                // X = Ra Sa^T (contraction over the Q/K width), Y = Rb Sb^T (over the V width) of step gg
-                const uint64_t d_ra = make_smem_desc(sRes + (2 * rs) * kTileBytes, 16, 1024),
-                               d_rb = make_smem_desc(sRes + (2 * rs + 1) * kTileBytes, 16, 1024);
-                auto issue_scores = [&](uint32_t gg) -> bool {
-                    const uint32_t st = gg % SS;
-                    if (!mbar_wait(t_full(st), (gg / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns)) return false;
-                    tc_fence_after();
-                    const uint64_t d_sa = make_smem_desc(sStr + (2 * st) * kTileBytes, 16, 1024),
-                                   d_sb = make_smem_desc(sStr + (2 * st + 1) * kTileBytes, 16, 1024);
-                    for (int ks = 0; ks < (wa >> 4); ++ks) {
-                        const uint32_t o = ((ks >> 2) * kBlockBytes + (ks & 3) * 32) >> 4;
-                        tc_mma_bf16(tmem_base + kColX, d_ra + o, d_sa + o, idesc_x, ks != 0 ? 1u : 0u);
-                    }
-                    for (int ks = 0; ks < (wb >> 4); ++ks) {
-                        const uint32_t o = ((ks >> 2) * kBlockBytes + (ks & 3) * 32) >> 4;
-                        tc_mma_bf16(tmem_base + kColY, d_rb + o, d_sb + o, idesc_x, ks != 0 ? 1u : 0u);
-                    }
-                    tc_commit(x_full);
-                    return true;
-                };
-                // score products only: those of step g + 1 as soon as every compute thread has the scores of step g in
-                // registers (it says so half way through its step), also across the boundary between two items
-                for (int i = 0; ok && i < I.n_steps; ++i, ++g) {
-                    if (g > 0 && !(ok = mbar_wait(xy_free, (g - 1) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                    tc_fence_after();
-                    ok = issue_scores(g);
-                }
-                if (ok) tc_commit(r_empty(rs));
-            }
-        }
+        // ------------------------------------------------------------------ issuer of the score products
+        if (lane == 0) score_role(true, NB == 1);
     } else if (warp >= 2 + kBwdComputeWarps) {
-        // ------------------------------------------------------------------ issuers of the accumulating products
+        // ------------------------------------------------------------------ issuers of the accumulating products (wide heads: of Y, and of all accumulating products)
         if (lane == 0) {
-            const int which = warp - (2 + kBwdComputeWarps);        // 0: dV (key-block kernel) / first half of dQ; 1: dK / second half
-            uint32_t g = 0, ri = 0;
-            bool ok = true;
-            for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
-                const BItem I = decode(it);
-                const int wn = (MODE == 0 && which == 0) ? P.heads.vo_w[I.h] : P.heads.qk_w[I.h];
-                const uint32_t idesc = make_idesc(kTile, wn, 0, 1);
-                // key-block kernel: dV += P^T dCtx_i (B = streamed b tile) / dK += dS^T Q_i (B = streamed a tile), all 8 steps
-                // of the contraction; query-block kernel: dQ += dS K_j (B = streamed a tile), steps 0-3 / 4-7
-                const uint32_t acc_col = MODE == 0 ? (which == 0 ? kColAcc1 : kColAcc2) : (which == 0 ? kColAcc2 : kColAcc1);
-                const uint32_t a_col = (MODE == 0 && which == 0) ? kColP : kColDS;
-                const uint32_t sA = sOut + ((MODE == 0 && which == 1) ? 2 * kBlockBytes : 0);   // wide heads: the same operands in shared memory
-                const int ks0 = MODE == 0 ? 0 : 4 * which, ks1 = MODE == 0 ? kTile / 16 : 4 * which + 4;
-                for (int i = 0; i < I.n_steps; ++i, ++g) {
-                    const uint32_t st = g % SS;
-                    if (!(ok = mbar_wait(t_full(st), (g / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                    if (!(ok = mbar_wait(out_full, g & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                    if (i == 0 && !(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                    tc_fence_after();
-                    const uint64_t db = make_smem_desc(sStr + (2 * st + ((MODE == 0 && which == 0) ? 1 : 0)) * kTileBytes, kBlockBytes, 1024);
-                    for (int ks = ks0; ks < ks1; ++ks) {
-                        if (kOpsInTmem)
-                            tc_mma_bf16_ts(tmem_base + acc_col, tmem_base + a_col + 8 * ks, db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
-                        else
-                            tc_mma_bf16(tmem_base + acc_col, make_smem_desc(sA + (ks >> 2) * kBlockBytes + (ks & 3) * 32, 16, 1024),
-                                        db + 128 * ks, idesc, (i != 0 || ks != ks0) ? 1u : 0u);
-                    }
-                    tc_commit(out_empty);
-                    tc_commit(t_empty(st));
-                }
-                if (ok) tc_commit(acc_full);
-            }
+            const int which = warp - (2 + kBwdComputeWarps);
+            if (NB == 1) acc_role(which, which + 1);
+            else if (which == 0) score_role(false, true);
+            else acc_role(0, 2);
         }
     } else {
         // ------------------------------------------------------------------ compute
@@ -1180,7 +1210,8 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         // columns [0, 32), warps 6..9 [32, 64), and so on, so every scheduler has four compute warps to interleave.
         const int part = (warp - 2) >> 2;
         const int row = (warp & 3) * 32 + lane;
-        const int col0 = part * 32;                                    // this thread's columns of the streamed block
+        constexpr int kHalves = kStep / 64;                            // 16-column halves of this thread's columns
+        const int col0 = part * (kStep / 4);                           // this thread's columns of the streamed block
         const uint32_t t_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         // 32 columns = four 16-byte chunks of block col0 / 64 of the row's image
         const uint32_t out_row = sOut + (col0 >> 6) * kBlockBytes + row * 128;
@@ -1201,27 +1232,28 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 d_r = P.vecs[static_cast<int64_t>(P.n_heads) * P.batch * P.seq_pad + o];
             }
             for (int i = 0; i < I.n_steps; ++i, ++g) {
-                const int other0 = (I.first + i % I.n_per) * kTile;  // first position of the streamed block
-                const float* vb = vec + (g % SS) * 2 * kTile;
-                if (!(ok = mbar_wait(x_full, g & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+                const int other0 = (I.first + i % I.n_per) * kStep;  // first position of the streamed block
+                const float* vb = vec + (g % SS) * 2 * kStep;
+                const uint32_t xb = g % kXY;
+                if (!(ok = mbar_wait(x_full(xb), (g / kXY) & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
                 tc_fence_after();
                 // (the step's loads landed long ago; this thread reads the vectors among them, so it looks at their barrier itself)
                 if (MODE == 0 && !(ok = mbar_wait(t_full(g % SS), (g / SS) & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
                 // (query position, key position) of element (row, column c): MODE 0 rows are keys, MODE 1 rows are queries
                 const int q0 = MODE == 0 ? other0 : I.own * kTile, k0 = MODE == 0 ? I.own * kTile : other0;
-                const bool masked = q0 + kTile > P.seq || k0 + kTile > P.seq || (P.causal && q0 < k0 + kTile);
+                const bool masked = q0 + (MODE == 0 ? kStep : kTile) > P.seq || k0 + kTile > P.seq || (P.causal && q0 < k0 + kTile);
                 // two halves of 16 columns: probabilities and dS are packed to bf16 pairs as soon as they exist
                 uint32_t pk_p[16], pk_ds[16];
 #pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
+                for (int hh = 0; hh < kHalves; ++hh) {
                     uint32_t rx[16], ry[16];
-                    tc_ld16(t_lane + kColX + col0 + 16 * hh, rx);
-                    tc_ld16(t_lane + kColY + col0 + 16 * hh, ry);
+                    tc_ld16(t_lane + kColX + xb * kStep + col0 + 16 * hh, rx);
+                    tc_ld16(t_lane + kColY + xb * kStep + col0 + 16 * hh, ry);
                     tc_wait_ld();
-                    if (hh == 1) {                                    // this thread's last read of the step's score tiles
+                    if (hh == kHalves - 1) {                          // this thread's last read of the step's score tiles
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(xy_free);
+                        if (lane == 0) mbar_arrive(xy_free(xb));
                     }
                     if (masked) {                                     // pairs outside the mask count as -inf (p = 0)
 #pragma unroll
@@ -1237,7 +1269,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                         float l2[4] = {lse_r, lse_r, lse_r, lse_r}, dd[4] = {d_r, d_r, d_r, d_r};
                         if (MODE == 0) {
                             const float4 a4 = *reinterpret_cast<const float4*>(vb + col0 + 16 * hh + e);
-                            const float4 b4 = *reinterpret_cast<const float4*>(vb + kTile + col0 + 16 * hh + e);
+                            const float4 b4 = *reinterpret_cast<const float4*>(vb + kStep + col0 + 16 * hh + e);
                             l2[0] = a4.x; l2[1] = a4.y; l2[2] = a4.z; l2[3] = a4.w;
                             dd[0] = b4.x; dd[1] = b4.y; dd[2] = b4.z; dd[3] = b4.w;
                         }
@@ -1254,26 +1286,27 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     }
                 }
                 // the products that read the previous step's tiles from shared memory are done
-                if (!(ok = mbar_wait(out_empty, (g & 1u) ^ 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
+                const uint32_t ob = g % kOB;
+                if (!(ok = mbar_wait(out_empty(ob), ((g / kOB) & 1u) ^ 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
                 if (kOpsInTmem) {   // this thread's 32 columns = 16 packed columns of its TMEM lane
                     if (MODE == 0) tc_st(t_lane + kColP + 16 * part, pk_p);
                     tc_st(t_lane + kColDS + 16 * part, pk_ds);
                     tc_wait_st();
                 } else {
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
+                    for (int q = 0; q < 2 * kHalves; ++q) {
                         const int chunk = chunk0 + q;
                         if (MODE == 0)
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + ((chunk ^ swz) << 4)),
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + ob * kOutSetBytes + ((chunk ^ swz) << 4)),
                                          "r"(pk_p[4 * q + 0]), "r"(pk_p[4 * q + 1]), "r"(pk_p[4 * q + 2]), "r"(pk_p[4 * q + 3]) : "memory");
-                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + (MODE == 0 ? 2 * kBlockBytes : 0) + ((chunk ^ swz) << 4)),
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(out_row + ob * kOutSetBytes + (MODE == 0 ? kOutTileBytes : 0) + ((chunk ^ swz) << 4)),
                                      "r"(pk_ds[4 * q + 0]), "r"(pk_ds[4 * q + 1]), "r"(pk_ds[4 * q + 2]), "r"(pk_ds[4 * q + 3]) : "memory");
                     }
                     fence_async_smem();
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(out_full);
+                if (lane == 0) mbar_arrive(out_full(ob));
             }
             if (!ok) break;
             // the accumulators of this item are complete: write them out (every thread its quarter of the columns)
@@ -1572,8 +1605,14 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     const int items_q = P.n_items;
     P.n_items = items_q / P.heads.rep;
     int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
-    if (nb == 1) attn_bwd_kernel<1, 0><<<grid, kBwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
-    else attn_bwd_kernel<2, 0><<<grid, kBwdThreads, BwdCfg<2, 0>::kSmem, stream>>>(P);
+    if (nb == 1) {
+        attn_bwd_kernel<1, 0><<<grid, kBwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
+    } else {   // wide heads: the streamed query blocks are half blocks
+        AttnBwdParams P0 = P;
+        if ((st = encode_tile_map(&P0.map_q, Qc, T, n_qk, ld_qk, BwdCfg<2, 0>::kStep)) != ECOSPA_OK) return st;
+        if ((st = encode_tile_map(&P0.map_do, dCtx, T, n_vo, ld_dctx, BwdCfg<2, 0>::kStep)) != ECOSPA_OK) return st;
+        attn_bwd_kernel<2, 0><<<grid, kBwdThreads, BwdCfg<2, 0>::kSmem, stream>>>(P0);
+    }
     if ((st = check_launch("attn_bwd_kernel (dK, dV)")) != ECOSPA_OK) return st;
     P.n_items = items_q;
     grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
