@@ -239,6 +239,18 @@ def test_backward_wide_heads(causal):
     run_backward(2, 200, [96, 128, 72, 33, 64], [128, 17, 100, 64, 80], causal, seed=6, d_h=128)
 
 
+@pytest.mark.parametrize("causal", [False, True])
+def test_backward_wide_heads_several_items_per_block(causal):
+    """Heads wider than 64 (the key-block kernel takes their queries 64 at a time): 3 x 9 x 6 key blocks are more items
+    than resident blocks, and 650 positions leave a ragged last half block of queries."""
+    k_qk = [96, 128, 72, 65, 128, 80, 112, 128, 100]
+    k_vo = [128, 70, 100, 128, 66, 128, 96, 120, 128]
+    a = run_backward(3, 650, k_qk, k_vo, causal, seed=11, d_h=128)
+    b = run_backward(3, 650, k_qk, k_vo, causal, seed=11, d_h=128)
+    for x, y in zip(a, b):
+        assert torch.equal(x.view(torch.int16), y.view(torch.int16))
+
+
 def test_backward_block_config_in_full_and_bit_identical_reruns():
     for causal in (False, True):
         a = run_backward(4, 128, [32] * 4, [32] * 4, causal, seed=2)
@@ -280,8 +292,8 @@ def test_backward_llama1b_sized_sampled_heads(causal):
 @pytest.mark.parametrize("causal", [False, True])
 @pytest.mark.parametrize("seq", [50, 77, 192, 500, 1000])
 def test_backward_narrow_heads_several_items_per_block(seq, causal):
-    """Heads at most 32 wide take the backward kernels that run two blocks per SM on 64-row streamed blocks: sequences
-    that are not multiples of 64 or 128, more (sequence, head, block) items than resident blocks, causal and not."""
+    """Heads at most 32 wide: sequences that are not multiples of 64 or 128, more (sequence, head, block) items than
+    resident blocks (so that a block's products run on into its next item), causal and not."""
     H = 40 if seq < 1000 else 12
     k_qk = [NARROW[(i + 1) % len(NARROW)] for i in range(H)]
     k_vo = [NARROW[i % len(NARROW)] for i in range(H)]
