@@ -1244,6 +1244,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 const bool masked = q0 + (MODE == 0 ? kStep : kTile) > P.seq || k0 + kTile > P.seq || (P.causal && q0 < k0 + kTile);
                 // two halves of 16 columns: probabilities and dS are packed to bf16 pairs as soon as they exist
                 uint32_t pk_p[16], pk_ds[16];
+                const f32x2 c2 = pack2(P.scale_log2e, P.scale_log2e), neg1 = pack2(-1.f, -1.f);
 #pragma unroll
                 for (int hh = 0; hh < kHalves; ++hh) {
                     uint32_t rx[16], ry[16];
@@ -1266,23 +1267,26 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                     }
 #pragma unroll
                     for (int e = 0; e < 16; e += 4) {
-                        float l2[4] = {lse_r, lse_r, lse_r, lse_r}, dd[4] = {d_r, d_r, d_r, d_r};
+                        // packed fp32 arithmetic around the exponentials: the step is bound by issue slots as much as by the
+                        // exponential unit.  l2 = -lse * log2(e); p = 2^(s * c + l2); dS = p * (dP - D)
+                        f32x2 l2a = pack2(lse_r, lse_r), l2b = l2a, dda = pack2(d_r, d_r), ddb = dda;
                         if (MODE == 0) {
                             const float4 a4 = *reinterpret_cast<const float4*>(vb + col0 + 16 * hh + e);
                             const float4 b4 = *reinterpret_cast<const float4*>(vb + kStep + col0 + 16 * hh + e);
-                            l2[0] = a4.x; l2[1] = a4.y; l2[2] = a4.z; l2[3] = a4.w;
-                            dd[0] = b4.x; dd[1] = b4.y; dd[2] = b4.z; dd[3] = b4.w;
+                            l2a = pack2(a4.x, a4.y); l2b = pack2(a4.z, a4.w);
+                            dda = pack2(b4.x, b4.y); ddb = pack2(b4.z, b4.w);
                         }
-                        float pe[4], de[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            pe[u] = ex2(fmaf(__uint_as_float(rx[e + u]), P.scale_log2e, l2[u]));   // l2 = -lse * log2(e)
-                            de[u] = pe[u] * (__uint_as_float(ry[e + u]) - dd[u]);
-                        }
-                        pk_p[8 * hh + (e >> 1)] = pack_bf16(pe[0], pe[1]);
-                        pk_p[8 * hh + (e >> 1) + 1] = pack_bf16(pe[2], pe[3]);
-                        pk_ds[8 * hh + (e >> 1)] = pack_bf16(de[0], de[1]);
-                        pk_ds[8 * hh + (e >> 1) + 1] = pack_bf16(de[2], de[3]);
+                        float x0, x1, x2, x3;
+                        unpack2(fma2(pack2(rx[e], rx[e + 1]), c2, l2a), x0, x1);
+                        unpack2(fma2(pack2(rx[e + 2], rx[e + 3]), c2, l2b), x2, x3);
+                        const float p0 = ex2(x0), p1 = ex2(x1), p2 = ex2(x2), p3 = ex2(x3);
+                        float d0, d1, d2, d3;
+                        unpack2(mul2(pack2(p0, p1), fma2(dda, neg1, pack2(ry[e], ry[e + 1]))), d0, d1);
+                        unpack2(mul2(pack2(p2, p3), fma2(ddb, neg1, pack2(ry[e + 2], ry[e + 3]))), d2, d3);
+                        pk_p[8 * hh + (e >> 1)] = pack_bf16(p0, p1);
+                        pk_p[8 * hh + (e >> 1) + 1] = pack_bf16(p2, p3);
+                        pk_ds[8 * hh + (e >> 1)] = pack_bf16(d0, d1);
+                        pk_ds[8 * hh + (e >> 1) + 1] = pack_bf16(d2, d3);
                     }
                 }
                 // the products that read the previous step's tiles from shared memory are done
