@@ -265,6 +265,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
             for (int i = 0; i < kOwn; ++i) o[i] = 0.f;
             // O = O * a + O_tile (the output tile of the previous key block)
             auto fold_output = [&](float a) {
+                const f32x2 a2 = pack2(a, a);
 #pragma unroll
                 for (int c = 0; c < kOwn / 16; ++c) {
                     if (c * 16 < wv) {
@@ -272,7 +273,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                         tc_ld16(tO + c * 16, r);
                         tc_wait_ld(r);
 #pragma unroll
-                        for (int i = 0; i < 16; ++i) o[c * 16 + i] = fmaf(o[c * 16 + i], a, __uint_as_float(r[i]));
+                        for (int i = 0; i < 16; i += 2)     // (packed fp32: half the issue slots)
+                            unpack2(fma2(pack2(o[c * 16 + i], o[c * 16 + i + 1]), a2, pack2(r[i], r[i + 1])), o[c * 16 + i], o[c * 16 + i + 1]);
                     }
                 }
             };
@@ -317,6 +319,8 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                 if (active) {
                     // pass 2: p = 2^(s * c - m_new) (2^-inf = 0 for the masked keys), row sum, P as packed bf16 into TMEM
                     uint32_t ra[CH], rb[CH];
+                    const f32x2 c2 = pack2(P.scale_log2e, P.scale_log2e), nm2 = pack2(-m_new, -m_new);
+                    f32x2 acc2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
                     tc_ld(tS, ra);
 #pragma unroll
                     for (int c = 0; c < NC; ++c) {
@@ -332,13 +336,16 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                         uint32_t pk[CH / 2];
 #pragma unroll
                         for (int i = 0; i < CH; i += 2) {
-                            const float p0 = ex2(fmaf(__uint_as_float(cur[i]), P.scale_log2e, -m_new));
-                            const float p1 = ex2(fmaf(__uint_as_float(cur[i + 1]), P.scale_log2e, -m_new));
-                            rs4[(i >> 1) & 3] += p0 + p1;
+                            float x0, x1;
+                            unpack2(fma2(pack2(cur[i], cur[i + 1]), c2, nm2), x0, x1);
+                            const float p0 = ex2(x0), p1 = ex2(x1);
+                            acc2[(i >> 1) & 1] = add2(acc2[(i >> 1) & 1], pack2(p0, p1));
                             pk[i >> 1] = pack_bf16(p0, p1);
                         }
                         tc_st(tP + c * (CH / 2), pk);
                     }
+                    unpack2(acc2[0], rs4[0], rs4[1]);
+                    unpack2(acc2[1], rs4[2], rs4[3]);
                 }
                 mbar_arrive(token(x ^ 1u));
                 if (active) {
