@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(kFwdThreads, 1) attn_fwd_kernel(const __grid_c
                                 if (kv_base + c * CH + i >= limit) cur[i] = 0xff800000u;
                         }
 #pragma unroll
-                        for (int i = 0; i < CH; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(cur[i]));
+                        for (int i = 0; i < CH; i += 2) mx4[(i >> 1) & 3] = max3(mx4[(i >> 1) & 3], __uint_as_float(cur[i]), __uint_as_float(cur[i + 1]));
                     }
                     const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
                     m_new = fmaxf(m, mx * P.scale_log2e);
@@ -738,7 +738,7 @@ __global__ void __launch_bounds__(MsCfg<NS, OC>::kThreads, 1) attn_fwd_ms_kernel
                     // the row rescaled and the chunk exponentiated again.
                     float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-                    for (int i = 0; i < CH; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], __uint_as_float(cur[i]));
+                    for (int i = 0; i < CH; i += 2) mx4[(i >> 1) & 3] = max3(mx4[(i >> 1) & 3], __uint_as_float(cur[i]), __uint_as_float(cur[i + 1]));
                     const float cm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * P.scale_log2e;
                     uint32_t pk[CH / 2];
                     float cs4[4] = {0.f, 0.f, 0.f, 0.f};
