@@ -418,6 +418,78 @@ def test_grouped_query_attention_llama_shape_rerun_bit_identical():
 
 
 @pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("seq", [63, 65, 129])
+def test_short_sequences_all_kernels(seq, causal):
+    """Lengths around the 64- and 128-position block sizes; one call per kernel family: narrow (key streams), up to 64
+    wide, up to 128 wide (half blocks of queries in the backward pass)."""
+    for k_qk, k_vo, d_h in (([16, 30], [32, 16], 64), ([64, 40], [48, 64], 64), ([128, 80], [96, 128], 128)):
+        run_forward(2, seq, k_qk, k_vo, causal, seed=100 + seq, d_h=d_h)
+        run_backward(2, seq, k_qk, k_vo, causal, seed=200 + seq, d_h=d_h)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_two_positions(causal):
+    """seq = 2.  dS = P (dP - D) cancels when one key dominates (dP of that key ~ D), and the kernels take D from the
+    bf16 context rows the forward call stored, the oracle from its own fp64 ones: each D_i is off by up to 2^-8 of
+    sum_c |dCtx_ic Ctx_ic|, which moves dQ_i by scale |dD_i| |sum_j P_ij K_j| <= scale |dD_i| max_j |K_j| and dK_j by
+    scale |dD_i| P_ij |Q_i|.  The comparison allows for that on top of the relative tolerance; dV does not involve D."""
+    for k_qk, k_vo, d_h in (([16, 30], [32, 16], 64), ([64, 40], [48, 64], 64), ([128, 80], [96, 128], 128)):
+        batch, seq, H = 8, 2, len(k_qk)
+        run_forward(batch, seq, k_qk, k_vo, causal, seed=7, d_h=d_h)
+        d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, k_qk, k_vo, 8, with_grad=True)
+        dd = {k: v.to(DEV) for k, v in d.items()}
+        T = batch * seq
+        Ctx = torch.zeros((T, nv), dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+        hd = B.heads(qo, qw, vo, vw)
+        scale = 1.0 / np.sqrt(d_h)
+        B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, hd, scale, causal, Ctx, lse)
+        dQ, dK, dV = (torch.zeros((T, n), dtype=torch.bfloat16, device=DEV) for n in (nq, nq, nv))
+        ws = torch.empty(B.ecospa_attn_workspace_bytes(batch, seq, H), dtype=torch.uint8, device=DEV)
+        B.ecospa_coupled_attn_bwd(dd["Q"], dd["K"], dd["V"], Ctx, dd["dCtx"], lse, batch, seq, hd, scale, causal, dQ, dK, dV, ws)
+        B.ecospa_device_status()
+        ref = O.attn_bwd(d["Q"], d["K"], d["V"], d["dCtx"], batch, seq, qo, k_qk, vo, k_vo, scale, causal)
+        fwd = O.attn_fwd(d["Q"], d["K"], d["V"], batch, seq, qo, k_qk, vo, k_vo, scale, causal)
+        Qn, Kn, dCn = (d[k].double().numpy() for k in ("Q", "K", "dCtx"))
+        for h in range(H):
+            cq, cv = slice(qo[h], qo[h] + k_qk[h]), slice(vo[h], vo[h] + k_vo[h])
+            dD = 2.0 ** -8 * np.abs(dCn[:, cv] * fwd["Ctx"][:, cv]).sum(axis=1)          # per query position
+            slack = scale * np.linalg.norm(dD) * max(np.linalg.norm(Kn[:, cq], axis=1).max(), np.linalg.norm(Qn[:, cq], axis=1).max())
+            for name, got_t in (("dQ", dQ), ("dK", dK)):
+                got = got_t.double().cpu().numpy()[:, cq]
+                err = np.linalg.norm(got - ref[name][:, cq])
+                assert err <= TOL * np.linalg.norm(ref[name][:, cq]) + slack, (name, h, err, slack)
+            assert rel(dV.double().cpu().numpy()[:, cv], ref["dV"][:, cv]) <= TOL, ("dV", h)
+
+
+@pytest.mark.parametrize("causal", [False, True])
+def test_single_position(causal):
+    """seq = 1: the softmax is over one key, so Ctx = V, dV = dCtx and dQ = dK = 0 (dS = P (dP - D) with P = 1 and
+    D = dP); the kernels get the zeros only up to the rounding of two differently ordered fp32 sums."""
+    for k_qk, k_vo, d_h in (([16, 30], [32, 16], 64), ([64, 40], [48, 64], 64), ([128, 80], [96, 128], 128)):
+        batch, seq, H = 3, 1, len(k_qk)
+        run_forward(batch, seq, k_qk, k_vo, causal, seed=5, d_h=d_h)
+        d, (qo, qw, nq), (vo, vw, nv) = make_inputs(batch, seq, k_qk, k_vo, 6, with_grad=True)
+        dd = {k: v.to(DEV) for k, v in d.items()}
+        T = batch * seq
+        Ctx = torch.zeros((T, nv), dtype=torch.bfloat16, device=DEV)
+        lse = torch.zeros(H * T, dtype=torch.float32, device=DEV)
+        hd = B.heads(qo, qw, vo, vw)
+        scale = 1.0 / np.sqrt(d_h)
+        B.ecospa_coupled_attn_fwd(dd["Q"], dd["K"], dd["V"], batch, seq, hd, scale, causal, Ctx, lse)
+        dQ, dK, dV = (torch.zeros((T, n), dtype=torch.bfloat16, device=DEV) for n in (nq, nq, nv))
+        ws = torch.empty(B.ecospa_attn_workspace_bytes(batch, seq, H), dtype=torch.uint8, device=DEV)
+        B.ecospa_coupled_attn_bwd(dd["Q"], dd["K"], dd["V"], Ctx, dd["dCtx"], lse, batch, seq, hd, scale, causal, dQ, dK, dV, ws)
+        B.ecospa_device_status()
+        for h in range(H):
+            cv = slice(vo[h], vo[h] + k_vo[h])
+            assert torch.equal(Ctx[:, cv].cpu(), d["V"][:, cv]), "Ctx = V"
+            assert torch.equal(dV[:, cv].cpu(), d["dCtx"][:, cv]), "dV = dCtx"
+        big = float(d["dCtx"].double().abs().max() * d["V"].double().abs().max() * max(max(k_vo), 1))
+        assert float(dQ.double().abs().max()) <= 1e-5 * big and float(dK.double().abs().max()) <= 1e-5 * big
+
+
+@pytest.mark.parametrize("causal", [False, True])
 def test_long_sequence_and_many_heads(causal):
     """One sequence of 6000 positions (not a multiple of any tile size; 32 slices per stream in the narrow-head forward
     kernel, 47 blocks in the others) on two heads, forward and backward, in full; and 128 heads (the most the descriptor
