@@ -946,7 +946,7 @@ struct AttnBwdParams {
 };
 
 // MODE 0: a CTA owns a key block of a (sequence, K/V head) and walks the query blocks of the query heads that read it:
-//         K, V resident, Q_i and dCtx_i streamed (with the 128 queries' -lse*log2e and D, bulk-copied on the same
+//         K, V resident, Q_i and dCtx_i streamed (with the step's queries' -lse*log2e and D, bulk-copied on the same
 //         barrier); X = S^T = K Q_i^T and Y = dP^T = V dCtx_i^T (thread = key row, columns = queries); P^T and dS^T are
 //         the A operands of dV += P^T dCtx_i and dK += dS^T Q_i, which accumulate in TMEM.
 // MODE 1: a CTA owns a query block and walks the key blocks: Q, dCtx resident, K_j and V_j streamed; X = S = Q K_j^T and
