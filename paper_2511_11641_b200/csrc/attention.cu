@@ -985,7 +985,7 @@ struct BwdCfg {
     static_assert(kSmem <= 232448, "shared memory of a block");
 };
 
-template <int NB, int MODE>
+template <int NB, int MODE, int NACC = 1>   // NACC = 2: every head at most 32 wide, the accumulators of two items side by side
 __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_constant__ AttnBwdParams P) {
     using Cfg = BwdCfg<NB, MODE>;
     constexpr int kTileBytes = Cfg::kTileBytes, kStrTileBytes = Cfg::kStrTileBytes, kStrBlockBytes = Cfg::kStrBlockBytes;
@@ -1015,7 +1015,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
     auto r_empty = [&](uint32_t s) { return bar0 + 8u * (2 + s); };
     auto t_full = [&](uint32_t s) { return bar0 + 8u * (4 + s); };
     auto t_empty = [&](uint32_t s) { return bar0 + 8u * (8 + s); };
-    const uint32_t acc_full = bar0 + 8u * 15, acc_empty = bar0 + 8u * 16;
+    // accumulators: one set, or two (heads at most 32 wide) that the items take in turn, each with its own pair of barriers
+    auto acc_full = [&](uint32_t a) { return bar0 + 8u * (a ? 22 : 15); };
+    auto acc_empty = [&](uint32_t a) { return bar0 + 8u * (a ? 23 : 16); };
+    constexpr uint32_t n_acc = NACC;
+    static_assert(NACC == 1 || NB == 1, "two sets of accumulators need the narrow layout");
     constexpr uint32_t kOB = Cfg::kOutBufs, kOutSetBytes = Cfg::kOutTiles * kOutTileBytes;
     auto out_full = [&](uint32_t b) { return bar0 + 8u * (b ? 20 : 13); };
     auto out_empty = [&](uint32_t b) { return bar0 + 8u * (b ? 21 : 14); };
@@ -1040,8 +1044,10 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
             mbar_init(out_full(b), kBwdComputeWarps);     // barriers the compute threads arrive on: one arrival per warp (its lanes meet first)
             mbar_init(out_empty(b), kAccIssuers);
         }
-        mbar_init(acc_full, kAccIssuers);
-        mbar_init(acc_empty, kBwdComputeWarps);
+        for (uint32_t a = 0; a < 2; ++a) {
+            mbar_init(acc_full(a), kAccIssuers);
+            mbar_init(acc_empty(a), kBwdComputeWarps);
+        }
         *abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&P.map_q);
@@ -1131,17 +1137,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         bool ok = true;
         for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
             const BItem I = decode(it);
+            const uint32_t as = ri % n_acc;
+            const uint32_t acc1 = n_acc == 2 ? kColAcc1 + 64 * as : kColAcc1, acc2 = n_acc == 2 ? kColAcc1 + 64 * as + 32 : kColAcc2;
             for (int i = 0; i < I.n_steps; ++i, ++g) {
                 const uint32_t st = g % SS;
                 if (!(ok = mbar_wait(t_full(st), (g / SS) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                 const uint32_t ob = g % kOB;
                 if (!(ok = mbar_wait(out_full(ob), (g / kOB) & 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
-                if (i == 0 && !(ok = mbar_wait(acc_empty, (ri & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
+                if (i == 0 && !(ok = mbar_wait(acc_empty(as), ((ri / n_acc) & 1u) ^ 1u, abort_flag, kCodeBase + 1, P.status, P.wait_limit_ns))) break;
                 tc_fence_after();
                 for (int which = w0; which < w1; ++which) {
                     const int wn = (MODE == 0 && which == 0) ? P.heads.vo_w[I.h] : P.heads.qk_w[I.h];
                     const uint32_t idesc = make_idesc(kTile, wn, 0, 1);
-                    const uint32_t acc_col = MODE == 0 ? (which == 0 ? kColAcc1 : kColAcc2) : (which == 0 ? kColAcc2 : kColAcc1);
+                    const uint32_t acc_col = (MODE == 0) == (which == 0) ? acc1 : acc2;
                     const uint32_t a_col = (MODE == 0 && which == 0) ? kColP : kColDS;                 // narrow heads: A operand in TMEM
                     const uint32_t sA = sOut + ob * kOutSetBytes + ((MODE == 0 && which == 1) ? kOutTileBytes : 0);   // wide heads: in shared memory
                     const int ks0 = MODE == 0 ? 0 : 4 * which, ks1 = MODE == 0 ? kStep / 16 : 4 * which + 4;
@@ -1157,7 +1165,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 tc_commit(out_empty(ob));
                 tc_commit(t_empty(st));
             }
-            if (ok) tc_commit(acc_full);
+            if (ok) tc_commit(acc_full(as));
         }
     };
 
@@ -1230,6 +1238,63 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
         uint32_t g = 0, ri = 0;
         bool ok = true;
         const int64_t T = static_cast<int64_t>(P.batch) * P.seq;
+        struct Pend {
+            int h, b, own;
+            uint32_t ri;
+            bool on;
+        };
+        Pend pend = {0, 0, 0, 0, false};
+        // writes an item's accumulators out once they are complete (every thread its quarter of the columns) and releases them
+        auto flush = [&](const Pend& d) -> bool {
+            const uint32_t as = d.ri % n_acc;
+            const uint32_t acc1 = n_acc == 2 ? kColAcc1 + 64 * as : kColAcc1, acc2 = n_acc == 2 ? kColAcc1 + 64 * as + 32 : kColAcc2;
+            if (!mbar_wait(acc_full(as), (d.ri / n_acc) & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns)) return false;
+            tc_fence_after();
+            const int pos = d.own * kTile + row;
+            const bool live = pos < P.seq;
+            const int64_t t = static_cast<int64_t>(d.b) * P.seq + pos;
+            auto write_acc = [&](uint32_t colbase, int w, uint16_t* dst, float mul, bool two = false, uint32_t colbase2 = 0) {
+#pragma unroll
+                for (int c = 0; c < NB; ++c) {
+                    const int col = part * (NB * 16) + c * 16;
+                    if (col < w) {
+                        uint32_t r[16];
+                        tc_ld16(t_lane + colbase + col, r);
+                        tc_wait_ld();
+                        if (two) {                               // the contraction was split over two accumulators
+                            uint32_t r2[16];
+                            tc_ld16(t_lane + colbase2 + col, r2);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) + __uint_as_float(r2[e]));
+                        }
+                        if (live) {
+                            uint4 v0, v1;
+                            v0.x = pack_bf16(__uint_as_float(r[0]) * mul, __uint_as_float(r[1]) * mul);
+                            v0.y = pack_bf16(__uint_as_float(r[2]) * mul, __uint_as_float(r[3]) * mul);
+                            v0.z = pack_bf16(__uint_as_float(r[4]) * mul, __uint_as_float(r[5]) * mul);
+                            v0.w = pack_bf16(__uint_as_float(r[6]) * mul, __uint_as_float(r[7]) * mul);
+                            v1.x = pack_bf16(__uint_as_float(r[8]) * mul, __uint_as_float(r[9]) * mul);
+                            v1.y = pack_bf16(__uint_as_float(r[10]) * mul, __uint_as_float(r[11]) * mul);
+                            v1.z = pack_bf16(__uint_as_float(r[12]) * mul, __uint_as_float(r[13]) * mul);
+                            v1.w = pack_bf16(__uint_as_float(r[14]) * mul, __uint_as_float(r[15]) * mul);
+                            *reinterpret_cast<uint4*>(dst + col) = v0;
+                            *reinterpret_cast<uint4*>(dst + col + 8) = v1;
+                        }
+                    }
+                }
+            };
+            if (MODE == 0) {
+                write_acc(acc1, P.heads.vo_w[d.h], P.dv + t * P.ld_dv + P.heads.v_off[d.h], 1.f);
+                write_acc(acc2, P.heads.qk_w[d.h], P.dk + t * P.ld_dqk + P.heads.k_off[d.h], P.scale);
+            } else {
+                write_acc(acc2, P.heads.qk_w[d.h], P.dq + t * P.ld_dqk + P.heads.qk_off[d.h], P.scale, true, acc1);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(as));
+            return true;
+        };
         for (int it = blockIdx.x; ok && it < P.n_items; it += gridDim.x, ++ri) {
             const BItem I = decode(it);
             const int own_pos = I.own * kTile + row;                 // position of this thread's row in the sequence
@@ -1321,54 +1386,19 @@ __global__ void __launch_bounds__(kBwdThreads, 1) attn_bwd_kernel(const __grid_c
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(out_full(ob));
+                if (i == 0 && pend.on) {   // the previous item's accumulators, now that this item's first step is on its way
+                    if (!(ok = flush(pend))) break;
+                    pend.on = false;
+                }
             }
             if (!ok) break;
-            // the accumulators of this item are complete: write them out (every thread its quarter of the columns)
-            if (!(ok = mbar_wait(acc_full, ri & 1u, abort_flag, kCodeBase + 2, P.status, P.wait_limit_ns))) break;
-            tc_fence_after();
-            const bool live = own_pos < P.seq;
-            const int64_t t = static_cast<int64_t>(I.b) * P.seq + own_pos;
-            auto write_acc = [&](uint32_t colbase, int w, uint16_t* dst, float mul, bool two = false, uint32_t colbase2 = 0) {
-#pragma unroll
-                for (int c = 0; c < NB; ++c) {
-                    const int col = part * (NB * 16) + c * 16;
-                    if (col < w) {
-                        uint32_t r[16];
-                        tc_ld16(t_lane + colbase + col, r);
-                        tc_wait_ld();
-                        if (two) {                               // the contraction was split over two accumulators
-                            uint32_t r2[16];
-                            tc_ld16(t_lane + colbase2 + col, r2);
-                            tc_wait_ld();
-#pragma unroll
-                            for (int e = 0; e < 16; ++e) r[e] = __float_as_uint(__uint_as_float(r[e]) + __uint_as_float(r2[e]));
-                        }
-                        if (live) {
-                            uint4 v0, v1;
-                            v0.x = pack_bf16(__uint_as_float(r[0]) * mul, __uint_as_float(r[1]) * mul);
-                            v0.y = pack_bf16(__uint_as_float(r[2]) * mul, __uint_as_float(r[3]) * mul);
-                            v0.z = pack_bf16(__uint_as_float(r[4]) * mul, __uint_as_float(r[5]) * mul);
-                            v0.w = pack_bf16(__uint_as_float(r[6]) * mul, __uint_as_float(r[7]) * mul);
-                            v1.x = pack_bf16(__uint_as_float(r[8]) * mul, __uint_as_float(r[9]) * mul);
-                            v1.y = pack_bf16(__uint_as_float(r[10]) * mul, __uint_as_float(r[11]) * mul);
-                            v1.z = pack_bf16(__uint_as_float(r[12]) * mul, __uint_as_float(r[13]) * mul);
-                            v1.w = pack_bf16(__uint_as_float(r[14]) * mul, __uint_as_float(r[15]) * mul);
-                            *reinterpret_cast<uint4*>(dst + col) = v0;
-                            *reinterpret_cast<uint4*>(dst + col + 8) = v1;
-                        }
-                    }
-                }
-            };
-            if (MODE == 0) {
-                write_acc(kColAcc1, P.heads.vo_w[I.h], P.dv + t * P.ld_dv + P.heads.v_off[I.h], 1.f);
-                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dk + t * P.ld_dqk + P.heads.k_off[I.h], P.scale);
-            } else {
-                write_acc(kColAcc2, P.heads.qk_w[I.h], P.dq + t * P.ld_dqk + P.heads.qk_off[I.h], P.scale, true, kColAcc1);
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(acc_empty);
+            // the accumulators of this item: written out now, or (two sets) after the first step of the CTA's next item, when
+            // the last products into them have long landed
+            const Pend cur = {I.h, I.b, I.own, ri, true};
+            if (n_acc == 2) pend = cur;
+            else if (!(ok = flush(cur))) break;
         }
+        if (ok && pend.on) flush(pend);
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -1589,6 +1619,8 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     cudaError_t e = cudaSuccess;
     std::call_once(once[dev & 63], [&] {
         e = cudaFuncSetAttribute(attn_bwd_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<1, 0>::kSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<1, 0, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<1, 0>::kSmem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<1, 1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<1, 1>::kSmem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<2, 0>::kSmem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<1, 1>::kSmem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(attn_bwd_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, BwdCfg<2, 1>::kSmem);
@@ -1620,7 +1652,8 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     P.n_items = items_q / P.heads.rep;
     int grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
     if (nb == 1) {
-        attn_bwd_kernel<1, 0><<<grid, kBwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
+        if (max_w <= 32) attn_bwd_kernel<1, 0, 2><<<grid, kBwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
+        else attn_bwd_kernel<1, 0><<<grid, kBwdThreads, BwdCfg<1, 0>::kSmem, stream>>>(P);
     } else {   // wide heads: the streamed query blocks are half blocks
         AttnBwdParams P0 = P;
         if ((st = encode_tile_map(&P0.map_q, Qc, T, n_qk, ld_qk, BwdCfg<2, 0>::kStep)) != ECOSPA_OK) return st;
@@ -1630,7 +1663,8 @@ extern "C" ecospa_status_t ecospa_coupled_attn_bwd(const void* Qc, const void* K
     if ((st = check_launch("attn_bwd_kernel (dK, dV)")) != ECOSPA_OK) return st;
     P.n_items = items_q;
     grid = std::min<int>(P.n_items, std::max(1, engine_num_sms()));
-    if (nb == 1) attn_bwd_kernel<1, 1><<<grid, kBwdThreads, BwdCfg<1, 1>::kSmem, stream>>>(P);
+    if (nb == 1 && max_w <= 32) attn_bwd_kernel<1, 1, 2><<<grid, kBwdThreads, BwdCfg<1, 1>::kSmem, stream>>>(P);
+    else if (nb == 1) attn_bwd_kernel<1, 1><<<grid, kBwdThreads, BwdCfg<1, 1>::kSmem, stream>>>(P);
     else attn_bwd_kernel<2, 1><<<grid, kBwdThreads, BwdCfg<2, 1>::kSmem, stream>>>(P);
     return check_launch("attn_bwd_kernel (dQ)");
 }
